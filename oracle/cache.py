@@ -1,0 +1,282 @@
+"""ORACLE — TEST INFRASTRUCTURE ONLY.
+
+The hybrid paged KV cache of Section 3.3 as an fp64 state machine with the
+same four operations as the library boundary:
+
+    append_kv                 "Incremental Cache Update": a new K/V row goes to
+                              the current dense page and takes part in attention
+                              at once; a new dense slot opens at a page boundary.
+    compress_eligible_pages   "Page-Wise Low-Rank KV Cache Construction": every
+                              completed page outside the sink region and the
+                              local window is replaced, once, by its rank-r
+                              truncated-SVD factors (Eq. 2); the dense slot is
+                              released; factor pages are never revisited.
+    decode_attention          "Attention over Mixed KV Pages": softmax attention
+                              (Eq. 1) over dense rows and reconstructed factor
+                              pages, for every query head of every sequence.
+    page_table                (kind, slot) of each logical page.
+
+Readings where the paper is silent (slot allocation policy, per-layer token
+counts, GQA head mapping) are written next to the code that takes them.
+"""
+from dataclasses import dataclass, field
+
+import numpy as np
+
+from . import attention as _att
+from . import svd as _svd
+
+DENSE, FACTOR = 0, 1
+
+
+@dataclass
+class OracleConfig:
+    n_layers: int
+    n_kv_heads: int
+    n_q_heads: int
+    head_dim: int
+    page_size: int
+    rank_k: int
+    rank_v: int
+    sink_tokens: int
+    recent_tokens: int
+    max_seqs: int
+    n_dense_slots: int
+    n_factor_slots: int
+    softmax_scale: float = 0.0          # 0 => 1/sqrt(head_dim)  (Eq. 1)
+
+
+class PoolExhausted(RuntimeError):
+    pass
+
+
+class _FreeList:
+    """Reading (paper only says storage is preallocated and dense slots are
+    released): slots are handed out in the caller's order array; a released slot
+    goes on a stack that is popped before the order array is consumed further."""
+
+    def __init__(self, order):
+        self.order = [int(x) for x in order]
+        self.next = 0
+        self.stack = []
+
+    def alloc(self):
+        if self.stack:
+            return self.stack.pop()
+        if self.next >= len(self.order):
+            raise PoolExhausted()
+        s = self.order[self.next]
+        self.next += 1
+        return s
+
+    def release(self, s):
+        self.stack.append(int(s))
+
+    def in_use(self):
+        return self.next - len(self.stack)
+
+
+@dataclass
+class _SeqLayer:
+    n_tokens: int = 0
+    kinds: list = field(default_factory=list)
+    slots: list = field(default_factory=list)
+
+
+def eligible_range(n_tokens: int, P: int, sink_tokens: int, recent_tokens: int):
+    """Closed form of the eligibility rule: with n_c = floor(T/P) completed
+    pages, n_s = S/P sink pages and n_w = W/P window pages, page p may be
+    factorized iff n_s <= p < n_c - n_w.  The n_w most recently completed pages
+    and the incomplete page stay dense; the paper's default dense region (one
+    sink page, the most recently completed page, the current incomplete page)
+    is S = W = P.  Returns (lo, hi) with hi >= lo."""
+    n_c = n_tokens // P
+    lo = sink_tokens // P
+    hi = max(lo, n_c - recent_tokens // P)
+    return lo, hi
+
+
+class OracleCache:
+    def __init__(self, cfg: OracleConfig, dense_slot_order=None, factor_slot_order=None):
+        assert cfg.n_q_heads % cfg.n_kv_heads == 0
+        assert cfg.sink_tokens % cfg.page_size == 0 and cfg.recent_tokens % cfg.page_size == 0
+        assert 0 < cfg.rank_k <= cfg.page_size and 0 < cfg.rank_v <= cfg.page_size
+        assert cfg.page_size <= cfg.head_dim
+        self.cfg = cfg
+        self.scale = cfg.softmax_scale if cfg.softmax_scale > 0 else 1.0 / np.sqrt(cfg.head_dim)
+        self.dense_free = _FreeList(range(cfg.n_dense_slots) if dense_slot_order is None else dense_slot_order)
+        self.factor_free = _FreeList(range(cfg.n_factor_slots) if factor_slot_order is None else factor_slot_order)
+        # slot -> arrays.  A slot is one logical page of one layer, all KV heads.
+        self.dense = {}      # slot -> (K [H_kv,P,d], V [H_kv,P,d]) fp64
+        self.factor = {}     # slot -> dict(A_k [H,P,r_k], B_k [H,r_k,d], A_v, B_v) fp64
+        self.sigma = {}      # slot -> (sigma_k [H,P], sigma_v [H,P]) sorted descending
+        self.state = {}      # (seq, layer) -> _SeqLayer
+        self.pages_compressed = 0
+
+    # ------------------------------------------------------------------ append
+    def _sl(self, seq, layer):
+        assert 0 <= seq < self.cfg.max_seqs and 0 <= layer < self.cfg.n_layers
+        return self.state.setdefault((seq, layer), _SeqLayer())
+
+    def append_kv(self, layer, seq_ids, n_new, k, v):
+        """k, v: [sum(n_new), H_kv, d] (values exactly representable in bf16,
+        widened to fp64 by the caller).  Token counts are kept per (seq, layer):
+        this call advances only `layer`'s count."""
+        c = self.cfg
+        k = np.asarray(k, dtype=np.float64)
+        v = np.asarray(v, dtype=np.float64)
+        assert k.shape == v.shape == (int(sum(n_new)), c.n_kv_heads, c.head_dim)
+        row = 0
+        for seq, n in zip(seq_ids, n_new):
+            sl = self._sl(int(seq), layer)
+            for _ in range(int(n)):
+                t = sl.n_tokens
+                p, r = divmod(t, c.page_size)
+                if r == 0:
+                    slot = self.dense_free.alloc()
+                    self.dense[slot] = (np.zeros((c.n_kv_heads, c.page_size, c.head_dim)),
+                                        np.zeros((c.n_kv_heads, c.page_size, c.head_dim)))
+                    sl.kinds.append(DENSE)
+                    sl.slots.append(slot)
+                Kp, Vp = self.dense[sl.slots[p]]
+                Kp[:, r, :] = k[row]
+                Vp[:, r, :] = v[row]
+                sl.n_tokens = t + 1
+                row += 1
+
+    # ---------------------------------------------------------------- compress
+    def eligible(self, seq, layer):
+        sl = self.state.get((seq, layer))
+        if sl is None:
+            return []
+        c = self.cfg
+        lo, hi = eligible_range(sl.n_tokens, c.page_size, c.sink_tokens, c.recent_tokens)
+        return [p for p in range(lo, hi) if sl.kinds[p] == DENSE]
+
+    def compress_eligible_pages(self, layer=-1):
+        """Processes eligible pages in ascending (seq, layer, page) order; for
+        each: allocate a factor slot, factorize every KV head's K page (rank r_k)
+        and V page (rank r_v), then release the dense slot.  Returns the number
+        of logical pages converted."""
+        c = self.cfg
+        layers = range(c.n_layers) if layer < 0 else [layer]
+        work = []
+        for seq in range(c.max_seqs):
+            for ly in layers:
+                for p in self.eligible(seq, ly):
+                    work.append((seq, ly, p))
+        if not work:
+            return 0
+        Ks = np.stack([self.dense[self.state[(s, ly)].slots[p]][0] for s, ly, p in work])  # [n,H,P,d]
+        Vs = np.stack([self.dense[self.state[(s, ly)].slots[p]][1] for s, ly, p in work])
+        n, H = Ks.shape[0], c.n_kv_heads
+        A_k, B_k, s_k = _svd.page_factors(Ks.reshape(n * H, c.page_size, c.head_dim), c.rank_k)
+        A_v, B_v, s_v = _svd.page_factors(Vs.reshape(n * H, c.page_size, c.head_dim), c.rank_v)
+        for i, (seq, ly, p) in enumerate(work):
+            sl = self.state[(seq, ly)]
+            fslot = self.factor_free.alloc()
+            sel = slice(i * H, (i + 1) * H)
+            self.factor[fslot] = dict(A_k=A_k[sel].copy(), B_k=B_k[sel].copy(),
+                                      A_v=A_v[sel].copy(), B_v=B_v[sel].copy())
+            self.sigma[fslot] = (s_k[sel].copy(), s_v[sel].copy())
+            dslot = sl.slots[p]
+            del self.dense[dslot]
+            self.dense_free.release(dslot)
+            sl.kinds[p] = FACTOR
+            sl.slots[p] = fslot
+        self.pages_compressed += len(work)
+        return len(work)
+
+    # ------------------------------------------------------------------ attend
+    def gather_kv(self, seq, layer, kv_head):
+        """Stack the logical pages of one (seq, layer, kv head) into K_all,
+        V_all [T, d]; factor pages are materialised as A B."""
+        c = self.cfg
+        sl = self.state[(seq, layer)]
+        Ks, Vs = [], []
+        n_pages = -(-sl.n_tokens // c.page_size)
+        for p in range(n_pages):
+            rows = min(c.page_size, sl.n_tokens - p * c.page_size)
+            if sl.kinds[p] == DENSE:
+                Kp, Vp = self.dense[sl.slots[p]]
+                Ks.append(Kp[kv_head, :rows])
+                Vs.append(Vp[kv_head, :rows])
+            else:
+                f = self.factor[sl.slots[p]]
+                Ks.append(f["A_k"][kv_head] @ f["B_k"][kv_head])
+                Vs.append(f["A_v"][kv_head] @ f["B_v"][kv_head])
+        return np.concatenate(Ks), np.concatenate(Vs)
+
+    def decode_attention(self, layer, seq_ids, q):
+        """q: [n_seqs, H_q, d].  Query head h reads KV head h // G, G = H_q/H_kv
+        (the grouped-query convention of the model runtime the paper builds on;
+        the paper omits the head index).  Returns [n_seqs, H_q, d] fp64."""
+        c = self.cfg
+        q = np.asarray(q, dtype=np.float64)
+        G = c.n_q_heads // c.n_kv_heads
+        out = np.zeros((len(seq_ids), c.n_q_heads, c.head_dim))
+        for i, seq in enumerate(seq_ids):
+            sl = self.state.get((int(seq), layer))
+            if sl is None or sl.n_tokens == 0:
+                raise ValueError("attention over an empty sequence")
+            for kvh in range(c.n_kv_heads):
+                K_all, V_all = self.gather_kv(int(seq), layer, kvh)
+                for g in range(G):
+                    h = kvh * G + g
+                    out[i, h] = _att.attention_plain(q[i, h], K_all, V_all, self.scale)
+        return out
+
+    def decode_attention_pagewise(self, layer, seq_ids, q):
+        """Same result through Eq. 4 (factor pages evaluated from factors, never
+        materialised) and Eq. 5 (merge).  Used to check the algebra only."""
+        c = self.cfg
+        q = np.asarray(q, dtype=np.float64)
+        G = c.n_q_heads // c.n_kv_heads
+        out = np.zeros((len(seq_ids), c.n_q_heads, c.head_dim))
+        for i, seq in enumerate(seq_ids):
+            sl = self.state[(int(seq), layer)]
+            n_pages = -(-sl.n_tokens // c.page_size)
+            for h in range(c.n_q_heads):
+                kvh = h // G
+                states = []
+                for p in range(n_pages):
+                    rows = min(c.page_size, sl.n_tokens - p * c.page_size)
+                    if sl.kinds[p] == DENSE:
+                        Kp, Vp = self.dense[sl.slots[p]]
+                        states.append(_att.page_state_dense(q[i, h], Kp[kvh, :rows], Vp[kvh, :rows], self.scale))
+                    else:
+                        f = self.factor[sl.slots[p]]
+                        states.append(_att.page_state_factor(q[i, h], f["A_k"][kvh], f["B_k"][kvh],
+                                                             f["A_v"][kvh], f["B_v"][kvh], self.scale))
+                out[i, h] = _att.merge_page_states(states)
+        return out
+
+    # ------------------------------------------------------------- bookkeeping
+    def page_table(self, seq, layer):
+        sl = self.state.get((seq, layer), _SeqLayer())
+        return list(sl.kinds), list(sl.slots), sl.n_tokens
+
+    def set_factors(self, slot, A_k, B_k, A_v, B_v):
+        """Replace a factor slot's contents (used to evaluate attention over
+        factors produced elsewhere, e.g. rounded to the storage type)."""
+        self.factor[slot] = dict(A_k=np.asarray(A_k, np.float64), B_k=np.asarray(B_k, np.float64),
+                                 A_v=np.asarray(A_v, np.float64), B_v=np.asarray(B_v, np.float64))
+
+    def free_seq(self, seq):
+        """Release every slot of a sequence, layers ascending, pages ascending."""
+        for ly in range(self.cfg.n_layers):
+            sl = self.state.pop((seq, ly), None)
+            if sl is None:
+                continue
+            for kind, slot in zip(sl.kinds, sl.slots):
+                if kind == DENSE:
+                    del self.dense[slot]
+                    self.dense_free.release(slot)
+                else:
+                    del self.factor[slot]
+                    self.sigma.pop(slot, None)
+                    self.factor_free.release(slot)
+
+    def stats(self):
+        return dict(dense_in_use=self.dense_free.in_use(), factor_in_use=self.factor_free.in_use(),
+                    pages_compressed=self.pages_compressed)
