@@ -1,0 +1,226 @@
+/*
+ * pkv.h — C ABI of the PuzzleKV decode hot path for NVIDIA B200 (sm_100a).
+ *
+ * What the library does (paper: Section 3.3).  Each (layer, KV head) of a
+ * sequence is split into pages of P tokens.  The sink pages and a moving window
+ * of recent pages are kept as dense bf16 rows; every other completed page is
+ * replaced, once, by its rank-r truncated-SVD factors (Eq. 2)
+ *        K_page ~= A_k B_k,  V_page ~= A_v B_v,   A: P x r,  B: r x d,
+ * (A is the paper's L, B the paper's R).  Decode attention (Eq. 4, Eq. 5)
+ * evaluates factor pages straight from the factors and merges all pages with an
+ * online softmax; historical K/V is never rebuilt.
+ *
+ * Conventions
+ *  - Every function returns a pkv_status (0 = PKV_OK, negative = error).  No
+ *    exception or abort crosses this boundary.  pkv_last_error() gives a
+ *    message for the most recent failure on that cache.
+ *  - Ownership: the caller allocates every device buffer and passes raw device
+ *    pointers; pkv_query_sizes() says how large each must be.  The library owns
+ *    only host-side metadata (page tables, free lists, a pinned staging ring)
+ *    and never allocates or frees device memory.  Buffers must stay valid until
+ *    pkv_destroy_cache().
+ *  - Pointers marked [device] are device addresses on the current CUDA device,
+ *    [host] are ordinary host addresses.  bf16 = IEEE bfloat16 bit pattern.
+ *  - All device work is enqueued on the `stream` argument (a cudaStream_t passed
+ *    as void*); calls are asynchronous unless stated.  Operations on one cache
+ *    must be issued on one stream (or the caller orders the streams).
+ *  - One cache object is not thread-safe; use one host thread per cache.
+ *  - Supported shapes: head_dim = 128, page_size = 64, rank_k = rank_v in
+ *    {8,16,24,32}, 1 <= n_q_heads / n_kv_heads <= 8.  Anything else returns
+ *    PKV_ERR_UNSUPPORTED from pkv_init_cache().
+ *  - Dry-run mode: if dense_pool, factor_pool, meta and workspace are all NULL
+ *    in pkv_init_cache(), no CUDA call is ever made; append / compress /
+ *    free_seq update the page tables exactly as they would with device buffers
+ *    (k, v, q, out may then be NULL) and pkv_decode_attention() only validates
+ *    its arguments.  Useful for capacity planning.
+ */
+#ifndef PKV_H
+#define PKV_H
+
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef struct pkv_cache pkv_cache;
+typedef int32_t pkv_status;
+
+#define PKV_OK                   0
+#define PKV_ERR_INVALID_ARG     (-1)  /* bad pointer, size, layer, count, or an empty sequence in attention */
+#define PKV_ERR_POOL_EXHAUSTED  (-2)  /* no free dense / factor slot, or a sequence exceeds max_pages_per_seq; state unchanged */
+#define PKV_ERR_BAD_SEQ         (-3)  /* sequence id outside [0, max_seqs) or repeated within one call */
+#define PKV_ERR_CUDA            (-4)  /* a CUDA runtime call failed; message holds cudaGetErrorString */
+#define PKV_ERR_NOT_CONVERGED   (-5)  /* reported by pkv_get_stats users: some page hit the Jacobi sweep cap (factors still written) */
+#define PKV_ERR_UNSUPPORTED     (-6)  /* shape outside the supported set */
+#define PKV_ERR_DEVICE_TIMEOUT  (-7)  /* a bounded in-kernel wait gave up (seen via pkv_get_stats); results of that call are invalid */
+
+#define PKV_KIND_DENSE  0
+#define PKV_KIND_FACTOR 1
+
+typedef struct pkv_config {
+    int32_t n_layers;
+    int32_t n_kv_heads;         /* H_kv */
+    int32_t n_q_heads;          /* H_q, a multiple of H_kv; query head h reads KV head h / (H_q/H_kv) */
+    int32_t head_dim;           /* d */
+    int32_t page_size;          /* P tokens per page */
+    int32_t rank_k, rank_v;     /* r_K, r_V of Eq. 2 */
+    int32_t sink_tokens;        /* S, multiple of P: the first S tokens stay dense for ever */
+    int32_t recent_tokens;      /* W, multiple of P: the W/P most recently completed pages and the incomplete page stay dense */
+    int32_t max_seqs;           /* sequence ids are 0 .. max_seqs-1 */
+    int32_t max_pages_per_seq;  /* ceil(max context / P) */
+    int64_t n_dense_slots;      /* pool capacities; one slot = one logical page of one layer, all KV heads */
+    int64_t n_factor_slots;
+    float   softmax_scale;      /* 0 => 1/sqrt(head_dim)  (Eq. 1) */
+    int32_t jacobi_max_sweeps;  /* 0 => default (16) */
+    float   jacobi_tol;         /* 0 => default; rotation skipped when |g_pq| <= tol*sqrt(g_pp*g_qq) */
+    int32_t n_ctas;             /* decode grid size; 0 => one CTA per SM of the current device (148 in dry-run) */
+    int32_t decode_variant;     /* 0 = tensor-core pipeline kernel (the product path); 1 = scalar fp32 kernel that
+                                   evaluates the same equations one unit at a time, kept as a debugging reference */
+} pkv_config;
+
+typedef struct pkv_sizes {
+    int64_t dense_slot_bytes;   /* H_kv * 2 * P * d * 2 */
+    int64_t factor_slot_bytes;  /* H_kv * 2 * (P*r_k + r_k*d + P*r_v + r_v*d) bytes; Eq. 3 is factor_slot_bytes / dense_slot_bytes */
+    int64_t dense_pool_bytes;   /* n_dense_slots * dense_slot_bytes */
+    int64_t factor_pool_bytes;
+    int64_t meta_bytes;         /* device page tables, token counts, decode plans, status words */
+    int64_t workspace_bytes;    /* split-K partial states, merge tickets, compression work list */
+} pkv_sizes;
+
+typedef struct pkv_stats {
+    int64_t dense_slots_in_use;
+    int64_t factor_slots_in_use;
+    int64_t pages_compressed;        /* logical pages (one layer, all KV heads) converted so far */
+    int64_t page_svds_not_converged; /* K or V pages whose Jacobi iteration hit the sweep cap */
+    int64_t device_timeouts;         /* bounded in-kernel waits that gave up (must be 0) */
+    int64_t last_decode_bytes;       /* algorithmic HBM bytes of the most recent pkv_decode_attention call:
+                                        factor blobs + valid dense rows + q + out */
+    int64_t last_decode_units;       /* work units (factor pages + dense blocks) of that call */
+} pkv_stats;
+
+/* Sizes of the caller-allocated buffers for a configuration.  Validates cfg. */
+pkv_status pkv_query_sizes(const pkv_config *cfg, pkv_sizes *out);
+
+/*
+ * Section 3.3 "Page-Wise Low-Rank KV Cache Construction": creates an empty
+ * hybrid cache over caller-owned storage.
+ *   dense_pool, factor_pool, meta, workspace  [device] buffers of at least the
+ *       sizes from pkv_query_sizes(), 256-byte aligned.  Contents need not be
+ *       initialised; meta and workspace are initialised here (synchronously).
+ *   dense_slot_order, factor_slot_order  [host] permutations of
+ *       0..n_*_slots-1 giving the order in which physical slots are handed out
+ *       (a shuffled physical pool); NULL = identity.  A released slot is reused
+ *       (last released first) before the order array is consumed further.
+ *   out  receives the cache handle.
+ * The storage format inside the pools is private (rows are stored with a
+ * 16-byte-chunk XOR swizzle so that a page can be copied linearly into shared
+ * memory and read without bank conflicts); use pkv_read_* / pkv_write_factors
+ * to look inside.
+ */
+pkv_status pkv_init_cache(const pkv_config *cfg, void *dense_pool, void *factor_pool,
+                          void *meta, void *workspace,
+                          const int32_t *dense_slot_order, const int32_t *factor_slot_order,
+                          pkv_cache **out);
+
+/*
+ * Section 3.3 "Incremental Cache Update": appends new key/value rows to the
+ * current dense page of each listed sequence in one layer; a new dense slot is
+ * taken at each page boundary.  The rows take part in the next attention call.
+ *   seq_ids [host] n_seqs distinct ids;  n_new [host] tokens per sequence (>= 0)
+ *   k, v    [device] bf16 [sum(n_new), H_kv, d], tokens of seq_ids[0] first.
+ * Token counts are kept per (sequence, layer); this call advances `layer` only.
+ * On PKV_ERR_POOL_EXHAUSTED nothing has been appended.
+ */
+pkv_status pkv_append_kv(pkv_cache *c, int32_t layer, int32_t n_seqs, const int32_t *seq_ids,
+                         const int32_t *n_new, const void *k, const void *v, void *stream);
+
+/*
+ * Section 3.3, Eq. 2 and the Gram-matrix route described after Eq. 3: converts
+ * every eligible page of `layer` (-1 = all layers) to factors.  A page p of a
+ * sequence with T tokens is eligible iff S/P <= p < floor(T/P) - W/P and it is
+ * still dense.  Pages are taken in ascending (sequence, layer, page) order; for
+ * each, a factor slot is allocated, the K and V page of every KV head are
+ * factorized on the GPU (G = X X^T in fp32, cyclic Jacobi eigen-solve in shared
+ * memory, A = top-r eigenvectors, B = A^T X, both rounded to bf16), then the
+ * dense slot is released.  Factor pages are never revisited.
+ *   n_pages_compressed [host, may be NULL] logical pages converted by this call.
+ * If the factor pool runs out, the pages converted so far stay converted and
+ * PKV_ERR_POOL_EXHAUSTED is returned.
+ */
+pkv_status pkv_compress_eligible_pages(pkv_cache *c, int32_t layer, int64_t *n_pages_compressed,
+                                       void *stream);
+
+/*
+ * Section 3.3 "Attention over Mixed KV Pages", Eq. 4 and Eq. 5: one query per
+ * sequence and query head attends over all tokens of that sequence in `layer`.
+ *   seq_ids [host] n_seqs distinct ids, each with at least one token in `layer`
+ *   q       [device] bf16 [n_seqs, H_q, d]
+ *   out     [device] bf16 [n_seqs, H_q, d]
+ *   out_f32 [device, may be NULL] the same result before rounding, fp32
+ * Scores use softmax_scale; accumulation is fp32.  The result does not depend
+ * on physical slot placement and is bit-identical from run to run.
+ */
+pkv_status pkv_decode_attention(pkv_cache *c, int32_t layer, int32_t n_seqs, const int32_t *seq_ids,
+                                const void *q, void *out, float *out_f32, void *stream);
+
+/*
+ * The same call for callers whose queries and results live in host memory:
+ * copies q_host -> q_stage, runs pkv_decode_attention, copies out_stage ->
+ * out_host, all on `stream` (asynchronous if the host buffers are pinned).
+ *   q_host, out_host [host] bf16 [n_seqs, H_q, d];  q_stage, out_stage [device]
+ *   caller-owned staging buffers of the same size.
+ */
+pkv_status pkv_decode_attention_host(pkv_cache *c, int32_t layer, int32_t n_seqs, const int32_t *seq_ids,
+                                     const void *q_host, void *out_host, void *q_stage, void *out_stage,
+                                     void *stream);
+
+/* Page table of one (sequence, layer) from the host mirror: kinds[i] in
+ * {PKV_KIND_DENSE, PKV_KIND_FACTOR}, slots[i] the physical slot, for i <
+ * *n_pages (arrays [host] of capacity max_pages_per_seq; may be NULL). */
+pkv_status pkv_get_page_table(const pkv_cache *c, int32_t seq, int32_t layer, int32_t *kinds,
+                              int32_t *slots, int32_t *n_pages, int32_t *n_tokens);
+
+/*
+ * The split of the most recent pkv_decode_attention() call on `layer` over CTAs
+ * (host mirror; for tests and tuning).  Work units are ordered by (position in
+ * seq_ids, KV head, unit); a unit is one factor page or one block of 16 or 32
+ * rows of a dense page.  CTA j owns the units from cta_starts[3j..3j+2] =
+ * (position, KV head, unit) up to the start of CTA j+1; entry n_used_ctas is the
+ * end sentinel (n_seqs, 0, 0).  seg_parts[2s], seg_parts[2s+1] = first CTA and
+ * number of CTAs that hold a partial softmax state of segment s = position *
+ * H_kv + KV head.  Arrays [host]: cta_starts 3*(n_ctas+1) ints, seg_parts
+ * 2*n_seqs*H_kv ints; any pointer may be NULL.
+ */
+pkv_status pkv_get_decode_plan(const pkv_cache *c, int32_t layer, int32_t *n_used_ctas, int32_t *cta_starts,
+                               int32_t *n_segs, int32_t *seg_parts);
+
+/* Counters; synchronises `stream` to read the device status words. */
+pkv_status pkv_get_stats(pkv_cache *c, pkv_stats *out, void *stream);
+
+/* Releases every slot of a sequence (layers ascending, pages ascending). */
+pkv_status pkv_free_seq(pkv_cache *c, int32_t seq);
+
+/* Frees host metadata only; the caller's device buffers are untouched. */
+pkv_status pkv_destroy_cache(pkv_cache *c);
+
+const char *pkv_last_error(const pkv_cache *c);
+
+/*
+ * Inspection helpers (asynchronous on `stream`).  They translate the private
+ * pool format to plain row-major bf16 in caller-owned [device] buffers:
+ *   pkv_read_factors : A_k [P, r_k], B_k [r_k, d], A_v [P, r_v], B_v [r_v, d]
+ *   pkv_write_factors: the reverse (overwrites one KV head of a factor slot)
+ *   pkv_read_dense   : K [P, d], V [P, d] of one KV head of a dense slot
+ */
+pkv_status pkv_read_factors(pkv_cache *c, int64_t factor_slot, int32_t kv_head, void *A_k, void *B_k,
+                            void *A_v, void *B_v, void *stream);
+pkv_status pkv_write_factors(pkv_cache *c, int64_t factor_slot, int32_t kv_head, const void *A_k,
+                             const void *B_k, const void *A_v, const void *B_v, void *stream);
+pkv_status pkv_read_dense(pkv_cache *c, int64_t dense_slot, int32_t kv_head, void *K, void *V,
+                          void *stream);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* PKV_H */

@@ -24,6 +24,7 @@ from dataclasses import dataclass, field
 import numpy as np
 
 from . import attention as _att
+from . import bf16 as _bf16
 from . import svd as _svd
 
 DENSE, FACTOR = 0, 1
@@ -261,6 +262,13 @@ class OracleCache:
         factors produced elsewhere, e.g. rounded to the storage type)."""
         self.factor[slot] = dict(A_k=np.asarray(A_k, np.float64), B_k=np.asarray(B_k, np.float64),
                                  A_v=np.asarray(A_v, np.float64), B_v=np.asarray(B_v, np.float64))
+
+    def round_factors_to_storage_type(self):
+        """Applies the storage step to every factor page: A and B rounded to
+        bf16 (the type dense pages are stored in; Eq. 3 counts elements of one
+        type).  Attention afterwards reads the stored values, still in fp64."""
+        for slot, f in self.factor.items():
+            self.factor[slot] = {k: _bf16.round_to_bf16(v) for k, v in f.items()}
 
     def free_seq(self, seq):
         """Release every slot of a sequence, layers ascending, pages ascending."""

@@ -1,0 +1,756 @@
+// Host side of the library: configuration, page tables, free lists, eligibility,
+// decode planning (split of the page list over CTAs) and the C ABI.  All device
+// work is delegated to the launchers declared in pkv_internal.h.
+#include <algorithm>
+#include <cmath>
+#include <cstdarg>
+#include <cstdio>
+#include <cstring>
+#include <new>
+#include <string>
+#include <vector>
+
+#include "pkv_internal.h"
+
+using namespace pkv;
+
+namespace {
+
+struct FreeList {
+    // Slots are handed out in the caller's order; a released slot is reused
+    // (last released first) before the order array is consumed further.
+    std::vector<int32_t> order, stack;
+    size_t next = 0;
+    int64_t available() const { return (int64_t)(order.size() - next + stack.size()); }
+    int32_t alloc() {
+        if (!stack.empty()) { int32_t s = stack.back(); stack.pop_back(); return s; }
+        return order[next++];
+    }
+    void release(int32_t s) { stack.push_back(s); }
+    int64_t in_use() const { return (int64_t)next - (int64_t)stack.size(); }
+};
+
+struct SeqLayer {
+    int32_t n_tokens = 0;
+    int32_t f_end = 0;                 // pages [sink_pages, f_end) are factor pages
+    uint64_t version = 0;              // bumped whenever the page list changes
+    std::vector<int32_t> slots;
+};
+
+struct PlanCache {
+    bool valid = false;
+    std::vector<int32_t> seq_ids;
+    std::vector<uint64_t> versions;
+    int n_segs = 0;
+    int64_t units = 0;
+    std::vector<PlanCta> ctas;         // n_used + 1 entries (last = end sentinel)
+    std::vector<PlanSeg> segs;
+};
+
+// Pinned staging ring for host -> device metadata uploads.
+struct Stager {
+    static constexpr int kChunks = 32;
+    static constexpr size_t kChunkBytes = 128 * 1024;
+    unsigned char *base = nullptr;
+    cudaEvent_t ev[kChunks];
+    bool pending[kChunks];
+    int cur = 0;
+    size_t used = 0;
+    bool dirty = false;
+};
+
+}  // namespace
+
+struct pkv_cache {
+    pkv_config cfg;
+    Geometry geo;
+    MetaLayout ml;
+    WorkspaceLayout wl;
+    bool dry = false;
+    unsigned char *dense_pool = nullptr, *factor_pool = nullptr, *meta = nullptr, *workspace = nullptr;
+    FreeList dense_free, factor_free;
+    std::vector<SeqLayer> sl;          // [max_seqs * n_layers]
+    std::vector<PlanCache> plans;      // [n_layers]
+    std::vector<int32_t> stamp;        // duplicate detection
+    int32_t stamp_gen = 0;
+    Stager stg;
+    std::string err;
+    int64_t pages_compressed = 0;
+    int64_t last_decode_bytes = 0, last_decode_units = 0;
+
+    SeqLayer &at(int seq, int layer) { return sl[(size_t)seq * cfg.n_layers + layer]; }
+    const SeqLayer &at(int seq, int layer) const { return sl[(size_t)seq * cfg.n_layers + layer]; }
+};
+
+namespace {
+
+pkv_status fail(pkv_cache *c, pkv_status code, const char *fmt, ...) {
+    if (c) {
+        char buf[512];
+        va_list ap;
+        va_start(ap, fmt);
+        vsnprintf(buf, sizeof buf, fmt, ap);
+        va_end(ap);
+        c->err = buf;
+    }
+    return code;
+}
+
+#define PKV_CUDA(c, call)                                                                         \
+    do {                                                                                          \
+        cudaError_t e_ = (call);                                                                  \
+        if (e_ != cudaSuccess)                                                                    \
+            return fail((c), PKV_ERR_CUDA, "%s failed: %s", #call, cudaGetErrorString(e_));        \
+    } while (0)
+
+pkv_status validate(const pkv_config *cfg, const char **why) {
+    *why = "";
+    if (!cfg) { *why = "cfg is NULL"; return PKV_ERR_INVALID_ARG; }
+    if (cfg->n_layers <= 0 || cfg->n_kv_heads <= 0 || cfg->n_q_heads <= 0 || cfg->max_seqs <= 0 ||
+        cfg->max_pages_per_seq <= 0 || cfg->n_dense_slots <= 0 || cfg->n_factor_slots < 0) {
+        *why = "counts must be positive"; return PKV_ERR_INVALID_ARG;
+    }
+    if (cfg->n_q_heads % cfg->n_kv_heads) { *why = "n_q_heads must be a multiple of n_kv_heads"; return PKV_ERR_INVALID_ARG; }
+    if (cfg->page_size <= 0 || cfg->rank_k <= 0 || cfg->rank_v <= 0 || cfg->rank_k > cfg->page_size ||
+        cfg->rank_v > cfg->page_size || cfg->page_size > cfg->head_dim) {
+        *why = "need 0 < rank <= page_size <= head_dim"; return PKV_ERR_INVALID_ARG;
+    }
+    if (cfg->sink_tokens < 0 || cfg->recent_tokens < 0 || cfg->sink_tokens % cfg->page_size ||
+        cfg->recent_tokens % cfg->page_size) {
+        *why = "sink_tokens and recent_tokens must be non-negative multiples of page_size"; return PKV_ERR_INVALID_ARG;
+    }
+    if (cfg->softmax_scale < 0.f || cfg->jacobi_max_sweeps < 0 || cfg->jacobi_tol < 0.f || cfg->n_ctas < 0 ||
+        cfg->decode_variant < 0 || cfg->decode_variant > 1) {
+        *why = "negative scale / sweep cap / tolerance / n_ctas, or unknown decode_variant"; return PKV_ERR_INVALID_ARG;
+    }
+    if (cfg->n_dense_slots > INT32_MAX || cfg->n_factor_slots > INT32_MAX) {
+        *why = "slot counts must fit in int32"; return PKV_ERR_INVALID_ARG;
+    }
+    if (cfg->head_dim != kHeadDim) { *why = "only head_dim = 128 is supported"; return PKV_ERR_UNSUPPORTED; }
+    if (cfg->page_size != kPage) { *why = "only page_size = 64 is supported"; return PKV_ERR_UNSUPPORTED; }
+    if (cfg->rank_k != cfg->rank_v || cfg->rank_k % 8 || cfg->rank_k > 32) {
+        *why = "only rank_k = rank_v in {8,16,24,32} is supported"; return PKV_ERR_UNSUPPORTED;
+    }
+    if (cfg->n_q_heads / cfg->n_kv_heads > kMaxGroup) { *why = "only n_q_heads/n_kv_heads <= 8 is supported"; return PKV_ERR_UNSUPPORTED; }
+    return PKV_OK;
+}
+
+long long align_up(long long x, long long a) { return (x + a - 1) / a * a; }
+
+void derive(const pkv_config &cfg, int n_ctas, Geometry &g, MetaLayout &ml, WorkspaceLayout &wl) {
+    const int P = cfg.page_size, d = cfg.head_dim;
+    g.n_layers = cfg.n_layers; g.n_kv_heads = cfg.n_kv_heads; g.n_q_heads = cfg.n_q_heads;
+    g.group = cfg.n_q_heads / cfg.n_kv_heads;
+    g.rank_k = cfg.rank_k; g.rank_v = cfg.rank_v;
+    g.max_seqs = cfg.max_seqs; g.max_pages = cfg.max_pages_per_seq;
+    g.sink_pages = cfg.sink_tokens / P; g.recent_pages = cfg.recent_tokens / P;
+    g.ak_off = 0;
+    g.bk_off = g.ak_off + P * cfg.rank_k * 2;
+    g.av_off = g.bk_off + cfg.rank_k * d * 2;
+    g.bv_off = g.av_off + P * cfg.rank_v * 2;
+    g.blob_bytes = g.bv_off + cfg.rank_v * d * 2;
+    g.dense_head_bytes = 2 * P * d * 2;
+    g.dense_slot_bytes = (long long)cfg.n_kv_heads * g.dense_head_bytes;
+    g.factor_slot_bytes = (long long)cfg.n_kv_heads * g.blob_bytes;
+    g.stage_bytes = std::max(g.blob_bytes, 8192);
+    g.block_tokens = g.stage_bytes >= 16384 ? 32 : 16;
+    g.blocks_per_page = P / g.block_tokens;
+    const int fixed = kConsumerWarps * kPartialFloats * 4 + 2048;
+    g.n_stages = std::min(24, (kSmemBudget - fixed) / g.stage_bytes);
+    g.n_ctas = n_ctas;
+    const float scale = cfg.softmax_scale > 0.f ? cfg.softmax_scale : 1.0f / std::sqrt((float)d);
+    g.scale_log2e = scale * 1.4426950408889634f;
+    g.jacobi_max_sweeps = cfg.jacobi_max_sweeps > 0 ? cfg.jacobi_max_sweeps : 16;
+    g.jacobi_tol = cfg.jacobi_tol > 0.f ? cfg.jacobi_tol : 1e-5f;
+
+    long long off = 0;
+    ml.page_table = off; off = align_up(off + 4LL * cfg.max_seqs * cfg.n_layers * cfg.max_pages_per_seq, 256);
+    ml.n_tokens = off;   off = align_up(off + 4LL * cfg.max_seqs * cfg.n_layers, 256);
+    long long p = sizeof(PlanHeader);
+    ml.plan_cta = p;   p = align_up(p + (long long)sizeof(PlanCta) * (n_ctas + 1), 16);
+    ml.plan_entry = p; p = align_up(p + (long long)sizeof(PlanEntry) * cfg.max_seqs, 16);
+    ml.plan_seg = p;   p = align_up(p + (long long)sizeof(PlanSeg) * cfg.max_seqs * cfg.n_kv_heads, 256);
+    ml.plan_stride = p;
+    ml.plans = off;      off = align_up(off + p * cfg.n_layers, 256);
+    ml.append_desc = off; off = align_up(off + (long long)sizeof(AppendDesc) * cfg.max_seqs, 256);
+    ml.status = off;     off = align_up(off + 4LL * kStatusWords, 256);
+    ml.total = off;
+
+    wl.n_partials = (long long)n_ctas + (long long)cfg.max_seqs * cfg.n_kv_heads;
+    long long w = 0;
+    wl.partials = w; w = align_up(w + wl.n_partials * kPartialFloats * 4, 256);
+    wl.worklist = w; w = align_up(w + (long long)sizeof(int2) * kCompressChunk, 256);
+    wl.total = w;
+}
+
+int default_ctas(bool dry) {
+    if (dry) return 148;
+    int dev = 0, sms = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess) return 148;
+    if (cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess || sms <= 0) return 148;
+    return sms;
+}
+
+// ---- staging ring -----------------------------------------------------------
+pkv_status stager_init(pkv_cache *c) {
+    Stager &s = c->stg;
+    PKV_CUDA(c, cudaHostAlloc((void **)&s.base, Stager::kChunks * Stager::kChunkBytes, cudaHostAllocDefault));
+    for (int i = 0; i < Stager::kChunks; ++i) {
+        PKV_CUDA(c, cudaEventCreateWithFlags(&s.ev[i], cudaEventDisableTiming));
+        s.pending[i] = false;
+    }
+    return PKV_OK;
+}
+
+// Moves to the next chunk, recording an event for the one just used.
+pkv_status stager_flush(pkv_cache *c, cudaStream_t st) {
+    Stager &s = c->stg;
+    if (!s.dirty) return PKV_OK;
+    PKV_CUDA(c, cudaEventRecord(s.ev[s.cur], st));
+    s.pending[s.cur] = true;
+    s.cur = (s.cur + 1) % Stager::kChunks;
+    s.used = 0;
+    s.dirty = false;
+    if (s.pending[s.cur]) {
+        PKV_CUDA(c, cudaEventSynchronize(s.ev[s.cur]));
+        s.pending[s.cur] = false;
+    }
+    return PKV_OK;
+}
+
+// Copies `bytes` of host data to device address `dst` through the ring.
+pkv_status upload(pkv_cache *c, void *dst, const void *src, size_t bytes, cudaStream_t st) {
+    Stager &s = c->stg;
+    const unsigned char *p = (const unsigned char *)src;
+    unsigned char *d = (unsigned char *)dst;
+    while (bytes > 0) {
+        if (s.used == Stager::kChunkBytes) {
+            pkv_status r = stager_flush(c, st);
+            if (r != PKV_OK) return r;
+        }
+        size_t n = std::min(bytes, Stager::kChunkBytes - s.used);
+        unsigned char *h = s.base + (size_t)s.cur * Stager::kChunkBytes + s.used;
+        memcpy(h, p, n);
+        PKV_CUDA(c, cudaMemcpyAsync(d, h, n, cudaMemcpyHostToDevice, st));
+        s.used += align_up((long long)n, 16);
+        if (s.used > Stager::kChunkBytes) s.used = Stager::kChunkBytes;
+        s.dirty = true;
+        p += n; d += n; bytes -= n;
+    }
+    return PKV_OK;
+}
+
+int *dev_page_table_row(pkv_cache *c, int seq, int layer) {
+    return (int *)(c->meta + c->ml.page_table) +
+           ((size_t)seq * c->cfg.n_layers + layer) * (size_t)c->cfg.max_pages_per_seq;
+}
+
+pkv_status check_seq_list(pkv_cache *c, int32_t n_seqs, const int32_t *seq_ids) {
+    if (n_seqs <= 0 || n_seqs > c->cfg.max_seqs || !seq_ids)
+        return fail(c, PKV_ERR_INVALID_ARG, "n_seqs must be in [1, max_seqs] and seq_ids non-NULL");
+    if (++c->stamp_gen == INT32_MAX) { std::fill(c->stamp.begin(), c->stamp.end(), 0); c->stamp_gen = 1; }
+    for (int i = 0; i < n_seqs; ++i) {
+        int s = seq_ids[i];
+        if (s < 0 || s >= c->cfg.max_seqs) return fail(c, PKV_ERR_BAD_SEQ, "sequence id %d out of range", s);
+        if (c->stamp[s] == c->stamp_gen) return fail(c, PKV_ERR_BAD_SEQ, "sequence id %d repeated", s);
+        c->stamp[s] = c->stamp_gen;
+    }
+    return PKV_OK;
+}
+
+// ---- decode planning ----------------------------------------------------------
+struct HeadShape { int d0_units, nf, d1_units, units; long long cost; };
+
+HeadShape head_shape(const Geometry &g, int n_pages, int f_begin, int f_end, long long cf, long long cd) {
+    HeadShape h;
+    int fb = std::min(f_begin, n_pages), fe = std::min(std::max(f_end, fb), n_pages);
+    h.d0_units = fb * g.blocks_per_page;
+    h.nf = fe - fb;
+    h.d1_units = (n_pages - fe) * g.blocks_per_page;
+    h.units = h.d0_units + h.nf + h.d1_units;
+    h.cost = (long long)(h.d0_units + h.d1_units) * cd + (long long)h.nf * cf;
+    return h;
+}
+
+// Smallest unit index u whose start cost (cost of units [0,u)) is >= rem.
+int first_unit_at_or_after(const HeadShape &h, long long rem, long long cf, long long cd) {
+    if (rem <= 0) return 0;
+    long long c0 = (long long)h.d0_units * cd;
+    if (rem <= c0) return (int)((rem + cd - 1) / cd);
+    rem -= c0;
+    long long c1 = (long long)h.nf * cf;
+    if (rem <= c1) return h.d0_units + (int)((rem + cf - 1) / cf);
+    rem -= c1;
+    return h.d0_units + h.nf + (int)std::min<long long>((rem + cd - 1) / cd, h.d1_units);
+}
+
+pkv_status build_plan(pkv_cache *c, int layer, int n_seqs, const int32_t *seq_ids, cudaStream_t st) {
+    const Geometry &g = c->geo;
+    PlanCache &pc = c->plans[layer];
+    const int H = g.n_kv_heads, N = g.n_ctas;
+    const long long cf = g.blob_bytes + 2048, cd = (long long)g.block_tokens * 2 * kRowBytes + 2048;
+
+    std::vector<PlanEntry> entries(n_seqs);
+    std::vector<HeadShape> shapes(n_seqs);
+    long long total_cost = 0, total_units = 0;
+    for (int i = 0; i < n_seqs; ++i) {
+        const SeqLayer &s = c->at(seq_ids[i], layer);
+        int n_pages = (s.n_tokens + kPage - 1) / kPage;
+        entries[i] = PlanEntry{seq_ids[i], n_pages, g.sink_pages, s.f_end};
+        shapes[i] = head_shape(g, n_pages, g.sink_pages, s.f_end, cf, cd);
+        total_cost += shapes[i].cost * H;
+        total_units += (long long)shapes[i].units * H;
+    }
+    // Cut the (entry, head, unit) sequence where the running cost crosses j * total / N.
+    std::vector<PlanCta> ctas;
+    ctas.reserve(N + 1);
+    {
+        int i = 0, h = 0;
+        long long base = 0;          // cost before (i, h)
+        for (int j = 0; j < N; ++j) {
+            long long b = (total_cost * j) / N;
+            while (i < n_seqs && base + shapes[i].cost <= b) {
+                base += shapes[i].cost;
+                if (++h == H) { h = 0; ++i; }
+            }
+            if (i >= n_seqs) break;
+            int u = first_unit_at_or_after(shapes[i], b - base, cf, cd);
+            PlanCta pos{i, h, u, 0};
+            if (u >= shapes[i].units) {          // start of the next (entry, head)
+                pos.unit = 0;
+                pos.head = h + 1;
+                if (pos.head == H) { pos.head = 0; pos.entry = i + 1; }
+                if (pos.entry >= n_seqs) break;
+            }
+            if (!ctas.empty() && ctas.back().entry == pos.entry && ctas.back().head == pos.head &&
+                ctas.back().unit == pos.unit)
+                continue;                         // empty range: drop it
+            ctas.push_back(pos);
+        }
+    }
+    const int n_used = (int)ctas.size();
+    ctas.push_back(PlanCta{n_seqs, 0, 0, 0});    // end sentinel
+    // Which CTAs hold a partial state of each (entry, head) segment.
+    const int n_segs = n_seqs * H;
+    std::vector<PlanSeg> segs(n_segs, PlanSeg{0, 0});
+    for (int j = 0; j < n_used; ++j) {
+        int g0 = ctas[j].entry * H + ctas[j].head;
+        int g1 = ctas[j + 1].entry * H + ctas[j + 1].head;     // segment of the first unit NOT in the range
+        if (ctas[j + 1].unit == 0) g1 -= 1;                    // range ends exactly at a segment boundary
+        for (int s = g0; s <= g1 && s < n_segs; ++s) {
+            if (segs[s].n_parts == 0) segs[s].cta_first = j;
+            segs[s].n_parts += 1;
+        }
+    }
+    PlanHeader hdr{n_seqs, n_used, n_segs, (int)std::min<long long>(total_units, INT32_MAX)};
+
+    pc.valid = true;
+    pc.seq_ids.assign(seq_ids, seq_ids + n_seqs);
+    pc.versions.resize(n_seqs);
+    for (int i = 0; i < n_seqs; ++i) pc.versions[i] = c->at(seq_ids[i], layer).version;
+    pc.n_segs = n_segs;
+    pc.units = total_units;
+    pc.ctas = ctas;
+    pc.segs = segs;
+
+    if (c->dry) return PKV_OK;
+    unsigned char *plan = c->meta + c->ml.plans + c->ml.plan_stride * layer;
+    pkv_status r;
+    if ((r = upload(c, plan, &hdr, sizeof hdr, st)) != PKV_OK) return r;
+    if ((r = upload(c, plan + c->ml.plan_cta, ctas.data(), sizeof(PlanCta) * ctas.size(), st)) != PKV_OK) return r;
+    if ((r = upload(c, plan + c->ml.plan_entry, entries.data(), sizeof(PlanEntry) * n_seqs, st)) != PKV_OK) return r;
+    if ((r = upload(c, plan + c->ml.plan_seg, segs.data(), sizeof(PlanSeg) * n_segs, st)) != PKV_OK) return r;
+    return stager_flush(c, st);
+}
+
+bool plan_is_current(pkv_cache *c, int layer, int n_seqs, const int32_t *seq_ids) {
+    const PlanCache &pc = c->plans[layer];
+    if (!pc.valid || (int)pc.seq_ids.size() != n_seqs) return false;
+    for (int i = 0; i < n_seqs; ++i) {
+        if (pc.seq_ids[i] != seq_ids[i]) return false;
+        if (pc.versions[i] != c->at(seq_ids[i], layer).version) return false;
+    }
+    return true;
+}
+
+}  // namespace
+
+// =============================================================================
+extern "C" {
+
+pkv_status pkv_query_sizes(const pkv_config *cfg, pkv_sizes *out) {
+    const char *why;
+    pkv_status r = validate(cfg, &why);
+    if (r != PKV_OK) return r;
+    if (!out) return PKV_ERR_INVALID_ARG;
+    Geometry g; MetaLayout ml; WorkspaceLayout wl;
+    // meta / workspace sizes depend on the grid size; use the larger of the request and 256 CTAs
+    int n_ctas = cfg->n_ctas > 0 ? cfg->n_ctas : 256;
+    derive(*cfg, n_ctas, g, ml, wl);
+    out->dense_slot_bytes = g.dense_slot_bytes;
+    out->factor_slot_bytes = g.factor_slot_bytes;
+    out->dense_pool_bytes = g.dense_slot_bytes * cfg->n_dense_slots;
+    out->factor_pool_bytes = g.factor_slot_bytes * cfg->n_factor_slots;
+    out->meta_bytes = ml.total;
+    out->workspace_bytes = wl.total;
+    return PKV_OK;
+}
+
+pkv_status pkv_init_cache(const pkv_config *cfg, void *dense_pool, void *factor_pool, void *meta,
+                          void *workspace, const int32_t *dense_slot_order,
+                          const int32_t *factor_slot_order, pkv_cache **out) {
+    const char *why;
+    pkv_status r = validate(cfg, &why);
+    if (r != PKV_OK) return r;
+    if (!out) return PKV_ERR_INVALID_ARG;
+    const bool dry = !dense_pool && !factor_pool && !meta && !workspace;
+    if (!dry && (!dense_pool || !meta || !workspace || (!factor_pool && cfg->n_factor_slots > 0)))
+        return PKV_ERR_INVALID_ARG;
+    if (!dry && (((uintptr_t)dense_pool | (uintptr_t)factor_pool | (uintptr_t)meta | (uintptr_t)workspace) & 255))
+        return PKV_ERR_INVALID_ARG;
+    pkv_cache *c = new (std::nothrow) pkv_cache();
+    if (!c) return PKV_ERR_INVALID_ARG;
+    c->cfg = *cfg;
+    c->dry = dry;
+    int n_ctas = cfg->n_ctas > 0 ? cfg->n_ctas : default_ctas(dry);
+    if (cfg->n_ctas == 0 && n_ctas > 256) n_ctas = 256;      // pkv_query_sizes() sized the buffers for <= 256
+    derive(*cfg, n_ctas, c->geo, c->ml, c->wl);
+    c->dense_pool = (unsigned char *)dense_pool; c->factor_pool = (unsigned char *)factor_pool;
+    c->meta = (unsigned char *)meta; c->workspace = (unsigned char *)workspace;
+    auto fill = [](FreeList &f, const int32_t *order, int64_t n) -> bool {
+        f.order.resize((size_t)n);
+        std::vector<char> seen((size_t)n, 0);
+        for (int64_t i = 0; i < n; ++i) {
+            int32_t s = order ? order[i] : (int32_t)i;
+            if (s < 0 || s >= n || seen[s]) return false;
+            seen[s] = 1;
+            f.order[(size_t)i] = s;
+        }
+        return true;
+    };
+    if (!fill(c->dense_free, dense_slot_order, cfg->n_dense_slots) ||
+        !fill(c->factor_free, factor_slot_order, cfg->n_factor_slots)) {
+        delete c;
+        return PKV_ERR_INVALID_ARG;               // slot order is not a permutation
+    }
+    c->sl.resize((size_t)cfg->max_seqs * cfg->n_layers);
+    for (auto &s : c->sl) s.f_end = c->geo.sink_pages;
+    c->plans.resize(cfg->n_layers);
+    c->stamp.assign(cfg->max_seqs, 0);
+    if (!dry) {
+        cudaError_t e = cudaMemset(c->meta, 0, (size_t)c->ml.total);
+        if (e == cudaSuccess) e = cudaMemset(c->workspace, 0, (size_t)c->wl.total);
+        if (e == cudaSuccess) e = decode_kernel_setup();
+        if (e == cudaSuccess) e = cudaDeviceSynchronize();
+        if (e != cudaSuccess || stager_init(c) != PKV_OK) { delete c; return PKV_ERR_CUDA; }
+    }
+    *out = c;
+    return PKV_OK;
+}
+
+pkv_status pkv_destroy_cache(pkv_cache *c) {
+    if (!c) return PKV_ERR_INVALID_ARG;
+    if (!c->dry && c->stg.base) {
+        for (int i = 0; i < Stager::kChunks; ++i) {
+            if (c->stg.pending[i]) cudaEventSynchronize(c->stg.ev[i]);
+            cudaEventDestroy(c->stg.ev[i]);
+        }
+        cudaFreeHost(c->stg.base);
+    }
+    delete c;
+    return PKV_OK;
+}
+
+const char *pkv_last_error(const pkv_cache *c) { return c ? c->err.c_str() : "cache is NULL"; }
+
+pkv_status pkv_append_kv(pkv_cache *c, int32_t layer, int32_t n_seqs, const int32_t *seq_ids,
+                         const int32_t *n_new, const void *k, const void *v, void *stream) {
+    if (!c) return PKV_ERR_INVALID_ARG;
+    cudaStream_t st = (cudaStream_t)stream;
+    if (layer < 0 || layer >= c->cfg.n_layers) return fail(c, PKV_ERR_INVALID_ARG, "layer %d out of range", layer);
+    pkv_status r = check_seq_list(c, n_seqs, seq_ids);
+    if (r != PKV_OK) return r;
+    if (!n_new) return fail(c, PKV_ERR_INVALID_ARG, "n_new is NULL");
+    long long n_tok = 0, need = 0;
+    for (int i = 0; i < n_seqs; ++i) {
+        if (n_new[i] < 0) return fail(c, PKV_ERR_INVALID_ARG, "n_new[%d] is negative", i);
+        const SeqLayer &s = c->at(seq_ids[i], layer);
+        long long after = ((long long)s.n_tokens + n_new[i] + kPage - 1) / kPage;
+        if (after > c->cfg.max_pages_per_seq)
+            return fail(c, PKV_ERR_POOL_EXHAUSTED, "sequence %d would exceed max_pages_per_seq", seq_ids[i]);
+        need += after - (long long)s.slots.size();
+        n_tok += n_new[i];
+    }
+    if (need > c->dense_free.available())
+        return fail(c, PKV_ERR_POOL_EXHAUSTED, "dense pool exhausted: need %lld slots, %lld free", need,
+                    (long long)c->dense_free.available());
+    if (!c->dry && n_tok > 0 && (!k || !v)) return fail(c, PKV_ERR_INVALID_ARG, "k or v is NULL");
+    if (n_tok == 0) return PKV_OK;
+
+    std::vector<AppendDesc> desc;
+    desc.reserve(n_seqs);
+    long long tok = 0;
+    for (int i = 0; i < n_seqs; ++i) {
+        if (n_new[i] == 0) continue;
+        SeqLayer &s = c->at(seq_ids[i], layer);
+        desc.push_back(AppendDesc{seq_ids[i], s.n_tokens, (int)tok, n_new[i]});
+        int before = (int)s.slots.size();
+        int after = (s.n_tokens + n_new[i] + kPage - 1) / kPage;
+        for (int p = before; p < after; ++p) s.slots.push_back(c->dense_free.alloc());
+        s.n_tokens += n_new[i];
+        tok += n_new[i];
+        if (after > before) {
+            s.version++;
+            if (!c->dry) {
+                r = upload(c, dev_page_table_row(c, seq_ids[i], layer) + before, s.slots.data() + before,
+                           sizeof(int32_t) * (after - before), st);
+                if (r != PKV_OK) return r;
+            }
+        }
+    }
+    if (c->dry) return PKV_OK;
+    AppendDesc *ddesc = (AppendDesc *)(c->meta + c->ml.append_desc);
+    if ((r = upload(c, ddesc, desc.data(), sizeof(AppendDesc) * desc.size(), st)) != PKV_OK) return r;
+    if ((r = stager_flush(c, st)) != PKV_OK) return r;
+    PKV_CUDA(c, launch_append(c->geo, c->dense_pool, (const int *)(c->meta + c->ml.page_table),
+                              (int *)(c->meta + c->ml.n_tokens), ddesc, (int)desc.size(), n_tok, layer, k, v, st));
+    return PKV_OK;
+}
+
+pkv_status pkv_compress_eligible_pages(pkv_cache *c, int32_t layer, int64_t *n_pages_compressed,
+                                       void *stream) {
+    if (!c) return PKV_ERR_INVALID_ARG;
+    cudaStream_t st = (cudaStream_t)stream;
+    if (n_pages_compressed) *n_pages_compressed = 0;
+    if (layer < -1 || layer >= c->cfg.n_layers) return fail(c, PKV_ERR_INVALID_ARG, "layer %d out of range", layer);
+    const Geometry &g = c->geo;
+    const int l0 = layer < 0 ? 0 : layer, l1 = layer < 0 ? c->cfg.n_layers : layer + 1;
+    std::vector<int2> work;
+    int64_t done = 0;
+    bool exhausted = false;
+    pkv_status r;
+    auto flush_work = [&]() -> pkv_status {
+        if (work.empty() || c->dry) { work.clear(); return PKV_OK; }
+        int2 *dwl = (int2 *)(c->workspace + c->wl.worklist);
+        pkv_status rr = upload(c, dwl, work.data(), sizeof(int2) * work.size(), st);
+        if (rr != PKV_OK) return rr;
+        if ((rr = stager_flush(c, st)) != PKV_OK) return rr;
+        PKV_CUDA(c, launch_compress(g, c->dense_pool, c->factor_pool, dwl, (int)work.size(),
+                                    (int *)(c->meta + c->ml.status), st));
+        work.clear();
+        return PKV_OK;
+    };
+    // Page-table uploads of converted pages are queued behind the kernel that reads the dense slots.
+    struct Flip { int seq, layer, first, last; };
+    std::vector<Flip> flips;
+    auto flush_flips = [&]() -> pkv_status {
+        for (const Flip &f : flips) {
+            if (c->dry) break;
+            const SeqLayer &s = c->at(f.seq, f.layer);
+            pkv_status rr = upload(c, dev_page_table_row(c, f.seq, f.layer) + f.first, s.slots.data() + f.first,
+                                   sizeof(int32_t) * (f.last - f.first), st);
+            if (rr != PKV_OK) return rr;
+        }
+        flips.clear();
+        return stager_flush(c, st);
+    };
+    for (int seq = 0; seq < c->cfg.max_seqs && !exhausted; ++seq) {
+        for (int ly = l0; ly < l1 && !exhausted; ++ly) {
+            SeqLayer &s = c->at(seq, ly);
+            const int n_c = s.n_tokens / kPage;
+            const int hi = std::max(g.sink_pages, n_c - g.recent_pages);   // eligible: sink_pages <= p < hi
+            if (s.f_end >= hi) continue;
+            const int first = s.f_end;
+            for (int p = s.f_end; p < hi; ++p) {
+                if (c->factor_free.available() == 0) { exhausted = true; break; }
+                int32_t fs = c->factor_free.alloc();
+                int32_t ds = s.slots[p];
+                work.push_back(make_int2(ds, fs));
+                s.slots[p] = fs;
+                c->dense_free.release(ds);
+                s.f_end = p + 1;
+                ++done;
+                if ((int)work.size() == kCompressChunk) {
+                    flips.push_back(Flip{seq, ly, first, s.f_end});
+                    if ((r = flush_work()) != PKV_OK) return r;
+                    if ((r = flush_flips()) != PKV_OK) return r;
+                }
+            }
+            if (s.f_end > first) {
+                s.version++;
+                flips.push_back(Flip{seq, ly, first, s.f_end});
+            }
+        }
+    }
+    if ((r = flush_work()) != PKV_OK) return r;
+    if ((r = flush_flips()) != PKV_OK) return r;
+    c->pages_compressed += done;
+    if (n_pages_compressed) *n_pages_compressed = done;
+    if (exhausted) return fail(c, PKV_ERR_POOL_EXHAUSTED, "factor pool exhausted after %lld pages", (long long)done);
+    return PKV_OK;
+}
+
+pkv_status pkv_decode_attention(pkv_cache *c, int32_t layer, int32_t n_seqs, const int32_t *seq_ids,
+                                const void *q, void *out, float *out_f32, void *stream) {
+    if (!c) return PKV_ERR_INVALID_ARG;
+    cudaStream_t st = (cudaStream_t)stream;
+    if (layer < 0 || layer >= c->cfg.n_layers) return fail(c, PKV_ERR_INVALID_ARG, "layer %d out of range", layer);
+    pkv_status r = check_seq_list(c, n_seqs, seq_ids);
+    if (r != PKV_OK) return r;
+    for (int i = 0; i < n_seqs; ++i)
+        if (c->at(seq_ids[i], layer).n_tokens == 0)
+            return fail(c, PKV_ERR_INVALID_ARG, "sequence %d has no tokens in layer %d", seq_ids[i], layer);
+    if (!c->dry && (!q || !out)) return fail(c, PKV_ERR_INVALID_ARG, "q or out is NULL");
+    if (!plan_is_current(c, layer, n_seqs, seq_ids)) {
+        if ((r = build_plan(c, layer, n_seqs, seq_ids, st)) != PKV_OK) return r;
+    }
+    const PlanCache &pc = c->plans[layer];
+    int64_t bytes = 2LL * n_seqs * c->cfg.n_q_heads * kRowBytes;          // q and out
+    for (int i = 0; i < n_seqs; ++i) {
+        const SeqLayer &s = c->at(seq_ids[i], layer);
+        const int n_pages = (int)s.slots.size();
+        const int nf = std::min(s.f_end, n_pages) - std::min(c->geo.sink_pages, n_pages);
+        const bool last_dense = !(n_pages - 1 >= c->geo.sink_pages && n_pages - 1 < s.f_end);
+        int64_t rows = (int64_t)(n_pages - nf) * kPage;
+        if (last_dense) rows -= (int64_t)n_pages * kPage - s.n_tokens;  // unfilled rows of the last page are not read
+        bytes += (int64_t)c->geo.n_kv_heads * ((int64_t)nf * c->geo.blob_bytes + rows * 2 * kRowBytes);
+    }
+    c->last_decode_bytes = bytes;
+    c->last_decode_units = pc.units;
+    if (c->dry) return PKV_OK;
+    DecodeArgs a;
+    a.geo = c->geo;
+    a.dense_pool = c->dense_pool; a.factor_pool = c->factor_pool;
+    a.page_table = (const int *)(c->meta + c->ml.page_table);
+    a.n_tokens = (const int *)(c->meta + c->ml.n_tokens);
+    a.plan = c->meta + c->ml.plans + c->ml.plan_stride * layer;
+    a.plan_cta = c->ml.plan_cta; a.plan_entry = c->ml.plan_entry; a.plan_seg = c->ml.plan_seg;
+    a.q = q; a.out = out; a.out_f32 = out_f32;
+    a.partials = (float *)(c->workspace + c->wl.partials);
+    a.status = (int *)(c->meta + c->ml.status);
+    a.layer = layer;
+    a.variant = c->cfg.decode_variant;
+    PKV_CUDA(c, launch_decode(a, pc.n_segs, st));
+    return PKV_OK;
+}
+
+pkv_status pkv_decode_attention_host(pkv_cache *c, int32_t layer, int32_t n_seqs, const int32_t *seq_ids,
+                                     const void *q_host, void *out_host, void *q_stage, void *out_stage,
+                                     void *stream) {
+    if (!c) return PKV_ERR_INVALID_ARG;
+    if (c->dry) return pkv_decode_attention(c, layer, n_seqs, seq_ids, nullptr, nullptr, nullptr, stream);
+    if (!q_host || !out_host || !q_stage || !out_stage || n_seqs <= 0)
+        return fail(c, PKV_ERR_INVALID_ARG, "host or staging buffer is NULL");
+    cudaStream_t st = (cudaStream_t)stream;
+    const size_t bytes = (size_t)n_seqs * c->cfg.n_q_heads * kRowBytes;
+    PKV_CUDA(c, cudaMemcpyAsync(q_stage, q_host, bytes, cudaMemcpyHostToDevice, st));
+    pkv_status r = pkv_decode_attention(c, layer, n_seqs, seq_ids, q_stage, out_stage, nullptr, stream);
+    if (r != PKV_OK) return r;
+    PKV_CUDA(c, cudaMemcpyAsync(out_host, out_stage, bytes, cudaMemcpyDeviceToHost, st));
+    return PKV_OK;
+}
+
+pkv_status pkv_get_page_table(const pkv_cache *c, int32_t seq, int32_t layer, int32_t *kinds,
+                              int32_t *slots, int32_t *n_pages, int32_t *n_tokens) {
+    if (!c) return PKV_ERR_INVALID_ARG;
+    if (seq < 0 || seq >= c->cfg.max_seqs) return PKV_ERR_BAD_SEQ;
+    if (layer < 0 || layer >= c->cfg.n_layers) return PKV_ERR_INVALID_ARG;
+    const SeqLayer &s = c->at(seq, layer);
+    for (size_t p = 0; p < s.slots.size(); ++p) {
+        if (kinds) kinds[p] = ((int)p >= c->geo.sink_pages && (int)p < s.f_end) ? PKV_KIND_FACTOR : PKV_KIND_DENSE;
+        if (slots) slots[p] = s.slots[p];
+    }
+    if (n_pages) *n_pages = (int32_t)s.slots.size();
+    if (n_tokens) *n_tokens = s.n_tokens;
+    return PKV_OK;
+}
+
+pkv_status pkv_get_decode_plan(const pkv_cache *c, int32_t layer, int32_t *n_used_ctas, int32_t *cta_starts,
+                               int32_t *n_segs, int32_t *seg_parts) {
+    if (!c || layer < 0 || layer >= c->cfg.n_layers) return PKV_ERR_INVALID_ARG;
+    const PlanCache &pc = c->plans[layer];
+    if (!pc.valid) return PKV_ERR_INVALID_ARG;
+    if (n_used_ctas) *n_used_ctas = (int32_t)pc.ctas.size() - 1;
+    if (n_segs) *n_segs = pc.n_segs;
+    if (cta_starts)
+        for (size_t j = 0; j < pc.ctas.size(); ++j) {
+            cta_starts[3 * j] = pc.ctas[j].entry; cta_starts[3 * j + 1] = pc.ctas[j].head; cta_starts[3 * j + 2] = pc.ctas[j].unit;
+        }
+    if (seg_parts)
+        for (int s = 0; s < pc.n_segs; ++s) { seg_parts[2 * s] = pc.segs[s].cta_first; seg_parts[2 * s + 1] = pc.segs[s].n_parts; }
+    return PKV_OK;
+}
+
+pkv_status pkv_get_stats(pkv_cache *c, pkv_stats *out, void *stream) {
+    if (!c || !out) return PKV_ERR_INVALID_ARG;
+    memset(out, 0, sizeof *out);
+    out->dense_slots_in_use = c->dense_free.in_use();
+    out->factor_slots_in_use = c->factor_free.in_use();
+    out->pages_compressed = c->pages_compressed;
+    out->last_decode_bytes = c->last_decode_bytes;
+    out->last_decode_units = c->last_decode_units;
+    if (!c->dry) {
+        int32_t st[kStatusWords];
+        PKV_CUDA(c, cudaStreamSynchronize((cudaStream_t)stream));
+        PKV_CUDA(c, cudaMemcpy(st, c->meta + c->ml.status, sizeof st, cudaMemcpyDeviceToHost));
+        out->device_timeouts = st[0];
+        out->page_svds_not_converged = st[1];
+    }
+    return PKV_OK;
+}
+
+pkv_status pkv_free_seq(pkv_cache *c, int32_t seq) {
+    if (!c) return PKV_ERR_INVALID_ARG;
+    if (seq < 0 || seq >= c->cfg.max_seqs) return fail(c, PKV_ERR_BAD_SEQ, "sequence id %d out of range", seq);
+    for (int ly = 0; ly < c->cfg.n_layers; ++ly) {
+        SeqLayer &s = c->at(seq, ly);
+        for (size_t p = 0; p < s.slots.size(); ++p) {
+            if ((int)p >= c->geo.sink_pages && (int)p < s.f_end) c->factor_free.release(s.slots[p]);
+            else c->dense_free.release(s.slots[p]);
+        }
+        s.slots.clear();
+        s.n_tokens = 0;
+        s.f_end = c->geo.sink_pages;
+        s.version++;
+    }
+    return PKV_OK;
+}
+
+static pkv_status slot_args(pkv_cache *c, int64_t slot, int64_t n_slots, int32_t head) {
+    if (!c) return PKV_ERR_INVALID_ARG;
+    if (c->dry) return fail(c, PKV_ERR_INVALID_ARG, "no device buffers in dry-run mode");
+    if (slot < 0 || slot >= n_slots || head < 0 || head >= c->cfg.n_kv_heads)
+        return fail(c, PKV_ERR_INVALID_ARG, "slot or head out of range");
+    return PKV_OK;
+}
+
+pkv_status pkv_read_factors(pkv_cache *c, int64_t slot, int32_t head, void *A_k, void *B_k, void *A_v,
+                            void *B_v, void *stream) {
+    pkv_status r = slot_args(c, slot, c ? c->cfg.n_factor_slots : 0, head);
+    if (r != PKV_OK) return r;
+    if (!A_k || !B_k || !A_v || !B_v) return fail(c, PKV_ERR_INVALID_ARG, "output pointer is NULL");
+    const unsigned char *blob = c->factor_pool + slot * c->geo.factor_slot_bytes + (int64_t)head * c->geo.blob_bytes;
+    PKV_CUDA(c, launch_read_factors(c->geo, blob, A_k, B_k, A_v, B_v, (cudaStream_t)stream));
+    return PKV_OK;
+}
+
+pkv_status pkv_write_factors(pkv_cache *c, int64_t slot, int32_t head, const void *A_k, const void *B_k,
+                             const void *A_v, const void *B_v, void *stream) {
+    pkv_status r = slot_args(c, slot, c ? c->cfg.n_factor_slots : 0, head);
+    if (r != PKV_OK) return r;
+    if (!A_k || !B_k || !A_v || !B_v) return fail(c, PKV_ERR_INVALID_ARG, "input pointer is NULL");
+    unsigned char *blob = c->factor_pool + slot * c->geo.factor_slot_bytes + (int64_t)head * c->geo.blob_bytes;
+    PKV_CUDA(c, launch_write_factors(c->geo, blob, A_k, B_k, A_v, B_v, (cudaStream_t)stream));
+    return PKV_OK;
+}
+
+pkv_status pkv_read_dense(pkv_cache *c, int64_t slot, int32_t head, void *K, void *V, void *stream) {
+    pkv_status r = slot_args(c, slot, c ? c->cfg.n_dense_slots : 0, head);
+    if (r != PKV_OK) return r;
+    if (!K || !V) return fail(c, PKV_ERR_INVALID_ARG, "output pointer is NULL");
+    const unsigned char *base = c->dense_pool + slot * c->geo.dense_slot_bytes + (int64_t)head * c->geo.dense_head_bytes;
+    PKV_CUDA(c, launch_read_dense(c->geo, base, K, V, (cudaStream_t)stream));
+    return PKV_OK;
+}
+
+}  // extern "C"

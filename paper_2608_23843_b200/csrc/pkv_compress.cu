@@ -1,0 +1,222 @@
+// Batched per-page truncated SVD (paper: Eq. 2 and the Gram-matrix route that
+// follows Eq. 3).  One CTA factorizes one P x d page X (K or V of one KV head):
+//   G = X X^T (P x P, fp32, exact bf16 products)        -> shared memory
+//   cyclic Jacobi eigen-solve of G with Q accumulating the rotations (fp32)
+//   A = the r eigenvectors of largest eigenvalue, B = A^T X, both rounded to bf16
+// Pages are independent, so the grid is simply (work-list entries) x (KV heads) x (K|V).
+#include <cuda_bf16.h>
+
+#include "pkv_internal.h"
+
+namespace pkv {
+
+namespace {
+
+constexpr int kThreads = 256;
+constexpr int kWarps = kThreads / 32;
+constexpr int kGs = kPage + 1;            // padded row stride of G and Q (floats)
+constexpr int kXs = kHeadDim + 2;         // padded row stride of X (bf16): 65 words, odd
+
+struct CompressSmem {
+    float G[kPage * kGs];
+    float Q[kPage * kGs];
+    __nv_bfloat16 X[kPage * kXs];
+    float2 cs[kPage / 2];
+    float lam[kPage];
+    int order[kPage];
+    float red[kWarps];
+};
+
+// Round-robin tournament: in round rho (0..P-2) the P indices form P/2 disjoint
+// pairs; over P-1 rounds every pair meets exactly once.
+__device__ __forceinline__ void pair_of(int rho, int k, int &p, int &q) {
+    constexpr int m = kPage - 1;
+    int a, b;
+    if (k == 0) { a = m; b = rho; }
+    else { a = rho + k; if (a >= m) a -= m; b = rho - k; if (b < 0) b += m; }
+    p = min(a, b); q = max(a, b);
+}
+
+__global__ void __launch_bounds__(kThreads)
+compress_kernel(Geometry geo, const unsigned char *dense_pool, unsigned char *factor_pool,
+                const int2 *worklist, int *status) {
+    extern __shared__ __align__(16) unsigned char smem_raw[];
+    CompressSmem &S = *reinterpret_cast<CompressSmem *>(smem_raw);
+    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+    const int kv = blockIdx.x & 1;
+    const int head = (blockIdx.x >> 1) % geo.n_kv_heads;
+    const int entry = (blockIdx.x >> 1) / geo.n_kv_heads;
+    const int2 wk = worklist[entry];
+    const int rank = kv ? geo.rank_v : geo.rank_k;
+    const unsigned char *src = dense_pool + (long long)wk.x * geo.dense_slot_bytes +
+                               (long long)head * geo.dense_head_bytes + kv * (kPage * kRowBytes);
+    unsigned char *blob = factor_pool + (long long)wk.y * geo.factor_slot_bytes + (long long)head * geo.blob_bytes;
+    unsigned char *dstA = blob + (kv ? geo.av_off : geo.ak_off);
+    unsigned char *dstB = blob + (kv ? geo.bv_off : geo.bk_off);
+
+    // ---- load the page (undo the storage swizzle) ----
+    for (int i = tid; i < kPage * 16; i += kThreads) {
+        const int row = i >> 4, chunk = i & 15;
+        const uint4 val = *reinterpret_cast<const uint4 *>(src + row * kRowBytes + swz_chunk(row, chunk) * 16);
+        unsigned *dst = reinterpret_cast<unsigned *>(&S.X[row * kXs + chunk * 8]);
+        dst[0] = val.x; dst[1] = val.y; dst[2] = val.z; dst[3] = val.w;
+    }
+    __syncthreads();
+
+    // ---- Gram matrix: each thread a 4 x 4 tile ----
+    {
+        const int ti = tid >> 4, tj = tid & 15;
+        float acc[4][4] = {};
+        for (int k = 0; k < kHeadDim; k += 2) {
+            float2 a[4], b[4];
+#pragma unroll
+            for (int u = 0; u < 4; ++u) {
+                a[u] = __bfloat1622float2(*reinterpret_cast<const __nv_bfloat162 *>(&S.X[(4 * ti + u) * kXs + k]));
+                b[u] = __bfloat1622float2(*reinterpret_cast<const __nv_bfloat162 *>(&S.X[(4 * tj + u) * kXs + k]));
+            }
+#pragma unroll
+            for (int u = 0; u < 4; ++u)
+#pragma unroll
+                for (int w = 0; w < 4; ++w) acc[u][w] = fmaf(a[u].y, b[w].y, fmaf(a[u].x, b[w].x, acc[u][w]));
+        }
+#pragma unroll
+        for (int u = 0; u < 4; ++u)
+#pragma unroll
+            for (int w = 0; w < 4; ++w) {
+                S.G[(4 * ti + u) * kGs + 4 * tj + w] = acc[u][w];
+                S.Q[(4 * ti + u) * kGs + 4 * tj + w] = (4 * ti + u == 4 * tj + w) ? 1.f : 0.f;
+            }
+    }
+    __syncthreads();
+    // the upper triangle was computed in a different summation order than the lower: symmetrise exactly
+    for (int i = tid; i < kPage * kPage; i += kThreads) {
+        const int r = i / kPage, c = i % kPage;
+        if (r > c) S.G[r * kGs + c] = S.G[c * kGs + r];
+    }
+    // absolute floor below which an off-diagonal entry is rounding noise of the Gram matrix
+    float dmax = 0.f;
+    if (tid < kPage) dmax = fabsf(S.G[tid * kGs + tid]);
+    for (int o = 16; o; o >>= 1) dmax = fmaxf(dmax, __shfl_xor_sync(0xffffffffu, dmax, o));
+    if (lane == 0) S.red[warp] = dmax;
+    __syncthreads();
+    const float floor_abs = 2e-7f * fmaxf(S.red[0], S.red[1]);
+    const float tol = geo.jacobi_tol;
+
+    // ---- cyclic Jacobi sweeps ----
+    bool converged = false;
+    for (int sweep = 0; sweep < geo.jacobi_max_sweeps && !converged; ++sweep) {
+        int rotated = 0;
+        for (int rho = 0; rho < kPage - 1; ++rho) {
+            if (tid < kPage / 2) {
+                int p, q;
+                pair_of(rho, tid, p, q);
+                const float gpp = S.G[p * kGs + p], gqq = S.G[q * kGs + q], gpq = S.G[p * kGs + q];
+                float c = 1.f, s = 0.f;
+                if (fabsf(gpq) > fmaxf(tol * sqrtf(fabsf(gpp * gqq)), floor_abs)) {
+                    const float theta = (gqq - gpp) / (2.f * gpq);
+                    const float t = copysignf(1.f, theta) / (fabsf(theta) + sqrtf(1.f + theta * theta));
+                    c = rsqrtf(1.f + t * t);
+                    s = t * c;
+                    rotated = 1;
+                }
+                S.cs[tid] = make_float2(c, s);
+            }
+            __syncthreads();
+            // columns p, q of G and Q:  x_p' = c x_p - s x_q,  x_q' = s x_p + c x_q
+#pragma unroll
+            for (int kk = 0; kk < kPage / 2 / kWarps; ++kk) {
+                const int k = warp + kk * kWarps;
+                int p, q;
+                pair_of(rho, k, p, q);
+                const float2 cs = S.cs[k];
+                if (cs.y != 0.f) {
+#pragma unroll
+                    for (int half = 0; half < 2; ++half) {
+                        const int i = lane + 32 * half;
+                        float gp = S.G[i * kGs + p], gq = S.G[i * kGs + q];
+                        S.G[i * kGs + p] = cs.x * gp - cs.y * gq;
+                        S.G[i * kGs + q] = cs.y * gp + cs.x * gq;
+                        float qp = S.Q[i * kGs + p], qq = S.Q[i * kGs + q];
+                        S.Q[i * kGs + p] = cs.x * qp - cs.y * qq;
+                        S.Q[i * kGs + q] = cs.y * qp + cs.x * qq;
+                    }
+                }
+            }
+            __syncthreads();
+            // rows p, q of G
+#pragma unroll
+            for (int kk = 0; kk < kPage / 2 / kWarps; ++kk) {
+                const int k = warp + kk * kWarps;
+                int p, q;
+                pair_of(rho, k, p, q);
+                const float2 cs = S.cs[k];
+                if (cs.y != 0.f) {
+#pragma unroll
+                    for (int half = 0; half < 2; ++half) {
+                        const int j = lane + 32 * half;
+                        float gp = S.G[p * kGs + j], gq = S.G[q * kGs + j];
+                        S.G[p * kGs + j] = cs.x * gp - cs.y * gq;
+                        S.G[q * kGs + j] = cs.y * gp + cs.x * gq;
+                    }
+                }
+            }
+            __syncthreads();
+        }
+        converged = !__syncthreads_or(rotated);
+    }
+    if (!converged && tid == 0) atomicAdd(&status[1], 1);
+
+    // ---- order eigenvalues: descending, ties by lower index ----
+    if (tid < kPage) { S.lam[tid] = S.G[tid * kGs + tid]; S.order[tid] = tid; }
+    __syncthreads();
+    if (tid < kPage) {
+        const float li = S.lam[tid];
+        int r = 0;
+        for (int j = 0; j < kPage; ++j) {
+            const float lj = S.lam[j];
+            r += (lj > li) || (lj == li && j < tid);
+        }
+        S.order[r] = tid;       // r < P always; NaN eigenvalues may collide (outputs then unspecified)
+    }
+    __syncthreads();
+
+    // ---- A = Q[:, order[:r]] as bf16, row-major [P][r] ----
+    for (int i = tid; i < kPage * rank / 2; i += kThreads) {
+        const int row = i / (rank / 2), j = (i % (rank / 2)) * 2;
+        const float a0 = S.Q[row * kGs + S.order[j]], a1 = S.Q[row * kGs + S.order[j + 1]];
+        *reinterpret_cast<__nv_bfloat162 *>(dstA + (row * rank + j) * 2) = __floats2bfloat162_rn(a0, a1);
+    }
+    // ---- B = A^T X (fp32 eigenvectors, exact page), rows swizzled like dense rows ----
+    for (int i = tid; i < rank * (kHeadDim / 2); i += kThreads) {
+        const int j = i / (kHeadDim / 2), col = (i % (kHeadDim / 2)) * 2;
+        const int oj = S.order[j];
+        float b0 = 0.f, b1 = 0.f;
+#pragma unroll 8
+        for (int r = 0; r < kPage; ++r) {
+            const float a = S.Q[r * kGs + oj];
+            const float2 x = __bfloat1622float2(*reinterpret_cast<const __nv_bfloat162 *>(&S.X[r * kXs + col]));
+            b0 = fmaf(a, x.x, b0);
+            b1 = fmaf(a, x.y, b1);
+        }
+        *reinterpret_cast<__nv_bfloat162 *>(dstB + j * kRowBytes + swz_chunk(j, col >> 3) * 16 + (col & 7) * 2) =
+            __floats2bfloat162_rn(b0, b1);
+    }
+}
+
+}  // namespace
+
+cudaError_t launch_compress(const Geometry &geo, const unsigned char *dense_pool, unsigned char *factor_pool,
+                            const int2 *worklist, int n_entries, int *status, cudaStream_t st) {
+    static bool configured = false;
+    if (!configured) {
+        cudaError_t e = cudaFuncSetAttribute(compress_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                             (int)sizeof(CompressSmem));
+        if (e != cudaSuccess) return e;
+        configured = true;
+    }
+    const unsigned grid = (unsigned)n_entries * geo.n_kv_heads * 2;
+    compress_kernel<<<grid, kThreads, sizeof(CompressSmem), st>>>(geo, dense_pool, factor_pool, worklist, status);
+    return cudaGetLastError();
+}
+
+}  // namespace pkv

@@ -1,0 +1,727 @@
+// Decode attention over mixed dense / factor pages (paper: Eq. 4, Eq. 5).
+//
+// One launch covers one layer.  The (sequence, KV head, page) list is cut by the
+// host into byte-balanced contiguous ranges, one per persistent CTA.  Inside a
+// CTA a producer warp walks the page table and streams whole factor blobs / dense
+// row blocks into a shared-memory ring with bulk async copies (TMA, mbarrier
+// completion); eight consumer warps each take one unit at a time and evaluate
+//     q~ = B_k q          (tensor cores, bf16 x bf16 -> fp32)
+//     s  = A_k q~ * scale (q~ split into two bf16 terms so the exponent sees ~fp32)
+//     online softmax      (fp32, exp2 with the scale folded in)
+//     w  = A_v^T p,  o += B_v^T w
+// for all query heads that share the KV head, keeping (m, l, o) in registers.
+// K^ and V^ are never formed.  At the end of each (sequence, KV head) segment the
+// warps combine their states and the CTA writes one partial state; a small merge
+// kernel applies Eq. 5 across CTAs.  A scalar fp32 kernel with the same plan and
+// partial format exists as a debugging reference (decode_variant = 1).
+#include <cuda_bf16.h>
+
+#include "pkv_internal.h"
+
+namespace pkv {
+
+namespace {
+
+constexpr float kNegInf = -1e30f;      // finite stand-in for -inf: exp2(kNegInf - x) == 0, no NaN from inf - inf
+constexpr int kKindDense = 0, kKindFactor = 1, kKindEnd = 2;
+
+struct Range {
+    PlanCta start, end;
+    int n_used, seg_first, n_local_segs;
+};
+
+struct HeadUnits { int d0, nf, units, fb, fe; };
+
+__device__ __forceinline__ HeadUnits head_units(const Geometry &g, const PlanEntry &e) {
+    HeadUnits h;
+    h.fb = min(e.f_begin, e.n_pages);
+    h.fe = min(max(e.f_end, h.fb), e.n_pages);
+    h.d0 = h.fb * g.blocks_per_page;
+    h.nf = h.fe - h.fb;
+    h.units = h.d0 + h.nf + (e.n_pages - h.fe) * g.blocks_per_page;
+    return h;
+}
+
+// unit index within an (entry, head) run -> logical page, block inside the page, kind
+__device__ __forceinline__ void unit_to_page(const Geometry &g, const HeadUnits &h, int u, int &page, int &blk,
+                                             int &kind) {
+    if (u < h.d0) { page = u / g.blocks_per_page; blk = u % g.blocks_per_page; kind = kKindDense; }
+    else if (u < h.d0 + h.nf) { page = h.fb + (u - h.d0); blk = 0; kind = kKindFactor; }
+    else { int v = u - h.d0 - h.nf; page = h.fe + v / g.blocks_per_page; blk = v % g.blocks_per_page; kind = kKindDense; }
+}
+
+__device__ __forceinline__ bool load_range(const DecodeArgs &a, Range &r) {
+    const PlanHeader hdr = *reinterpret_cast<const PlanHeader *>(a.plan);
+    r.n_used = hdr.n_used_ctas;
+    if ((int)blockIdx.x >= hdr.n_used_ctas) return false;
+    const PlanCta *ctas = reinterpret_cast<const PlanCta *>(a.plan + a.plan_cta);
+    r.start = ctas[blockIdx.x];
+    r.end = ctas[blockIdx.x + 1];
+    const int H = a.geo.n_kv_heads;
+    r.seg_first = r.start.entry * H + r.start.head;
+    int seg_last = r.end.entry * H + r.end.head;
+    if (r.end.unit == 0) seg_last -= 1;
+    r.n_local_segs = seg_last - r.seg_first + 1;
+    return true;
+}
+
+// =============================================================================
+// Scalar reference kernel (debugging aid): same plan, same partial format.
+// =============================================================================
+__device__ __forceinline__ float bf16_at(const unsigned char *base, int byte_off) {
+    return __bfloat162float(*reinterpret_cast<const __nv_bfloat16 *>(base + byte_off));
+}
+__device__ __forceinline__ int swz_off(int row, int col) {     // byte offset of element (row, col) of a 256-byte-row matrix
+    return row * kRowBytes + swz_chunk(row, col >> 3) * 16 + (col & 7) * 2;
+}
+
+__global__ void __launch_bounds__(128) decode_scalar_kernel(const __grid_constant__ DecodeArgs a) {
+    Range rg;
+    if (!load_range(a, rg)) return;
+    const Geometry &g = a.geo;
+    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+    const int G = g.group, H = g.n_kv_heads, r_k = g.rank_k, r_v = g.rank_v;
+    __shared__ float qs[kMaxGroup][kHeadDim];
+    __shared__ float qt[kMaxGroup][32];
+    __shared__ float sc[kMaxGroup][kPage];
+    __shared__ float wv[kMaxGroup][32];
+    __shared__ float m_s[kMaxGroup], l_s[kMaxGroup], alpha_s[kMaxGroup];
+    float o[kMaxGroup];
+    const PlanEntry *entries = reinterpret_cast<const PlanEntry *>(a.plan + a.plan_entry);
+
+    PlanCta cur = rg.start;
+    while (!(cur.entry == rg.end.entry && cur.head == rg.end.head && cur.unit == rg.end.unit)) {
+        const PlanEntry e = entries[cur.entry];
+        const HeadUnits hu = head_units(g, e);
+        const bool last_run = cur.entry == rg.end.entry && cur.head == rg.end.head;
+        const int u_end = last_run ? rg.end.unit : hu.units;
+        const int T = a.n_tokens[(long long)e.seq * g.n_layers + a.layer];
+        // new segment: load q, reset state
+        __syncthreads();
+        for (int i = tid; i < G * kHeadDim; i += 128)
+            qs[i / kHeadDim][i % kHeadDim] = __bfloat162float(
+                reinterpret_cast<const __nv_bfloat16 *>(a.q)[((long long)cur.entry * g.n_q_heads + cur.head * G) * kHeadDim + i]);
+        if (tid < kMaxGroup) { m_s[tid] = kNegInf; l_s[tid] = 0.f; }
+        for (int gq = 0; gq < kMaxGroup; ++gq) o[gq] = 0.f;
+        __syncthreads();
+        for (int u = cur.unit; u < u_end; ++u) {
+            int page, blk, kind;
+            unit_to_page(g, hu, u, page, blk, kind);
+            const int slot = a.page_table[((long long)e.seq * g.n_layers + a.layer) * g.max_pages + page];
+            int rows;
+            const unsigned char *base;
+            if (kind == kKindFactor) {
+                rows = kPage;
+                base = a.factor_pool + (long long)slot * g.factor_slot_bytes + (long long)cur.head * g.blob_bytes;
+                for (int i = tid; i < G * r_k; i += 128) {           // q~ = B_k q
+                    const int gq = i / r_k, j = i % r_k;
+                    float acc = 0.f;
+                    for (int c = 0; c < kHeadDim; ++c) acc += bf16_at(base + g.bk_off, swz_off(j, c)) * qs[gq][c];
+                    qt[gq][j] = acc;
+                }
+                __syncthreads();
+                for (int i = tid; i < G * kPage; i += 128) {         // s = A_k q~ * scale
+                    const int gq = i / kPage, p = i % kPage;
+                    float acc = 0.f;
+                    for (int j = 0; j < r_k; ++j) acc += bf16_at(base + g.ak_off, (p * r_k + j) * 2) * qt[gq][j];
+                    sc[gq][p] = acc * g.scale_log2e;
+                }
+            } else {
+                const int row0 = blk * g.block_tokens;
+                rows = min(g.block_tokens, T - page * kPage - row0);
+                if (rows <= 0) continue;
+                base = a.dense_pool + (long long)slot * g.dense_slot_bytes + (long long)cur.head * g.dense_head_bytes;
+                for (int i = tid; i < G * rows; i += 128) {
+                    const int gq = i / rows, p = i % rows;
+                    float acc = 0.f;
+                    for (int c = 0; c < kHeadDim; ++c) acc += bf16_at(base, swz_off(row0 + p, c)) * qs[gq][c];
+                    sc[gq][p] = acc * g.scale_log2e;
+                }
+            }
+            __syncthreads();
+            for (int gq = warp; gq < G; gq += 4) {                   // online softmax, one warp per head
+                float mx = kNegInf;
+                for (int p = lane; p < rows; p += 32) mx = fmaxf(mx, sc[gq][p]);
+                for (int off = 16; off; off >>= 1) mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, off));
+                const float m_new = fmaxf(m_s[gq], mx);
+                float sum = 0.f;
+                for (int p = lane; p < rows; p += 32) { float e2 = exp2f(sc[gq][p] - m_new); sc[gq][p] = e2; sum += e2; }
+                for (int off = 16; off; off >>= 1) sum += __shfl_xor_sync(0xffffffffu, sum, off);
+                if (lane == 0) {
+                    const float al = exp2f(m_s[gq] - m_new);
+                    alpha_s[gq] = al;
+                    l_s[gq] = l_s[gq] * al + sum;
+                    m_s[gq] = m_new;
+                }
+            }
+            __syncthreads();
+            if (kind == kKindFactor) {
+                for (int i = tid; i < G * r_v; i += 128) {           // w = A_v^T p
+                    const int gq = i / r_v, j = i % r_v;
+                    float acc = 0.f;
+                    for (int p = 0; p < kPage; ++p) acc += sc[gq][p] * bf16_at(base + g.av_off, (p * r_v + j) * 2);
+                    wv[gq][j] = acc;
+                }
+                __syncthreads();
+                for (int gq = 0; gq < G; ++gq) {                     // o = o*alpha + B_v^T w
+                    float acc = 0.f;
+                    for (int j = 0; j < r_v; ++j) acc += wv[gq][j] * bf16_at(base + g.bv_off, swz_off(j, tid));
+                    o[gq] = o[gq] * alpha_s[gq] + acc;
+                }
+            } else {
+                const int row0 = blk * g.block_tokens;
+                for (int gq = 0; gq < G; ++gq) {
+                    float acc = 0.f;
+                    for (int p = 0; p < rows; ++p)
+                        acc += sc[gq][p] * bf16_at(base + kPage * kRowBytes, swz_off(row0 + p, tid));
+                    o[gq] = o[gq] * alpha_s[gq] + acc;
+                }
+            }
+            __syncthreads();
+        }
+        // segment (or range) done: write the partial state
+        const int seg = cur.entry * H + cur.head;
+        float *part = a.partials + ((long long)blockIdx.x + seg) * kPartialFloats;
+        for (int gq = 0; gq < kMaxGroup; ++gq) part[gq * kHeadDim + tid] = gq < G ? o[gq] : 0.f;
+        if (tid < kMaxGroup) {
+            part[kMaxGroup * kHeadDim + tid] = tid < G ? m_s[tid] : kNegInf;
+            part[kMaxGroup * kHeadDim + kMaxGroup + tid] = tid < G ? l_s[tid] : 0.f;
+        }
+        if (last_run) break;
+        cur.unit = 0;
+        if (++cur.head == H) { cur.head = 0; ++cur.entry; }
+    }
+}
+
+// =============================================================================
+// Eq. 5 across CTAs: one block per (entry, KV head) segment.
+// =============================================================================
+__global__ void __launch_bounds__(256) merge_kernel(const __grid_constant__ DecodeArgs a) {
+    const Geometry &g = a.geo;
+    const int seg = blockIdx.x;
+    const PlanSeg ps = reinterpret_cast<const PlanSeg *>(a.plan + a.plan_seg)[seg];
+    const int entry = seg / g.n_kv_heads, head = seg % g.n_kv_heads;
+    const int hq = threadIdx.x >> 5, d4 = (threadIdx.x & 31) * 4;
+    if (hq >= g.group) return;
+    const float *part = a.partials + ((long long)ps.cta_first + seg) * kPartialFloats;
+    float M = kNegInf;
+    for (int k = 0; k < ps.n_parts; ++k) M = fmaxf(M, part[(long long)k * kPartialFloats + kMaxGroup * kHeadDim + hq]);
+    float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
+    float L = 0.f;
+    for (int k = 0; k < ps.n_parts; ++k) {
+        const float *pk = part + (long long)k * kPartialFloats;
+        const float w = exp2f(pk[kMaxGroup * kHeadDim + hq] - M);
+        const float4 o = *reinterpret_cast<const float4 *>(pk + hq * kHeadDim + d4);
+        acc.x += w * o.x; acc.y += w * o.y; acc.z += w * o.z; acc.w += w * o.w;
+        L += w * pk[kMaxGroup * kHeadDim + kMaxGroup + hq];
+    }
+    const float inv = 1.f / L;
+    acc.x *= inv; acc.y *= inv; acc.z *= inv; acc.w *= inv;
+    const long long off = ((long long)entry * g.n_q_heads + head * g.group + hq) * kHeadDim + d4;
+    __nv_bfloat162 lo = __floats2bfloat162_rn(acc.x, acc.y), hi = __floats2bfloat162_rn(acc.z, acc.w);
+    uint2 packed;
+    packed.x = *reinterpret_cast<unsigned *>(&lo);
+    packed.y = *reinterpret_cast<unsigned *>(&hi);
+    *reinterpret_cast<uint2 *>(reinterpret_cast<__nv_bfloat16 *>(a.out) + off) = packed;
+    if (a.out_f32) *reinterpret_cast<float4 *>(a.out_f32 + off) = acc;
+}
+
+// =============================================================================
+// Tensor-core pipeline kernel.
+// =============================================================================
+__device__ __forceinline__ uint32_t smem_u32(const void *p) { return (uint32_t)__cvta_generic_to_shared(p); }
+
+__device__ __forceinline__ void mbar_init(uint32_t bar, uint32_t count) {
+    asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(bar), "r"(count));
+}
+__device__ __forceinline__ void mbar_arrive(uint32_t bar) {
+    asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(bar) : "memory");
+}
+__device__ __forceinline__ void mbar_arrive_expect_tx(uint32_t bar, uint32_t bytes) {
+    asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(bytes) : "memory");
+}
+__device__ __forceinline__ bool mbar_try_wait(uint32_t bar, uint32_t parity) {
+    uint32_t ok;
+    asm volatile(
+        "{\n\t.reg .pred p;\n\t"
+        "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
+        "selp.u32 %0, 1, 0, p;\n\t}"
+        : "=r"(ok) : "r"(bar), "r"(parity) : "memory");
+    return ok != 0;
+}
+// Bounded wait: gives up after ~2e9 clocks (about a second) and reports failure.
+__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity) {
+    if (mbar_try_wait(bar, parity)) return true;
+    const long long t0 = clock64();
+    while (!mbar_try_wait(bar, parity)) {
+        if (clock64() - t0 > 2000000000LL) return false;
+    }
+    return true;
+}
+__device__ __forceinline__ void bulk_g2s(uint32_t dst, const void *src, uint32_t bytes, uint32_t bar) {
+    asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];"
+                 ::"r"(dst), "l"(src), "r"(bytes), "r"(bar) : "memory");
+}
+__device__ __forceinline__ void ldsm_x4(uint32_t (&r)[4], uint32_t addr) {
+    asm volatile("ldmatrix.sync.aligned.m8n8.x4.shared.b16 {%0,%1,%2,%3}, [%4];"
+                 : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]) : "r"(addr));
+}
+__device__ __forceinline__ void ldsm_x4_t(uint32_t (&r)[4], uint32_t addr) {
+    asm volatile("ldmatrix.sync.aligned.m8n8.x4.trans.shared.b16 {%0,%1,%2,%3}, [%4];"
+                 : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]) : "r"(addr));
+}
+__device__ __forceinline__ void ldsm_x2(uint32_t (&r)[2], uint32_t addr) {
+    asm volatile("ldmatrix.sync.aligned.m8n8.x2.shared.b16 {%0,%1}, [%2];" : "=r"(r[0]), "=r"(r[1]) : "r"(addr));
+}
+__device__ __forceinline__ void ldsm_x2_t(uint32_t (&r)[2], uint32_t addr) {
+    asm volatile("ldmatrix.sync.aligned.m8n8.x2.trans.shared.b16 {%0,%1}, [%2];" : "=r"(r[0]), "=r"(r[1]) : "r"(addr));
+}
+__device__ __forceinline__ void mma16816(float (&d)[4], uint32_t a0, uint32_t a1, uint32_t a2, uint32_t a3,
+                                         uint32_t b0, uint32_t b1) {
+    asm volatile("mma.sync.aligned.m16n8k16.row.col.f32.bf16.bf16.f32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, {%0,%1,%2,%3};"
+                 : "+f"(d[0]), "+f"(d[1]), "+f"(d[2]), "+f"(d[3])
+                 : "r"(a0), "r"(a1), "r"(a2), "r"(a3), "r"(b0), "r"(b1));
+}
+__device__ __forceinline__ void mma1688(float (&d)[4], uint32_t a0, uint32_t a1, uint32_t b0) {
+    asm volatile("mma.sync.aligned.m16n8k8.row.col.f32.bf16.bf16.f32 {%0,%1,%2,%3}, {%4,%5}, {%6}, {%0,%1,%2,%3};"
+                 : "+f"(d[0]), "+f"(d[1]), "+f"(d[2]), "+f"(d[3]) : "r"(a0), "r"(a1), "r"(b0));
+}
+__device__ __forceinline__ uint32_t movm_t(uint32_t x) {
+    uint32_t y;
+    asm volatile("movmatrix.sync.aligned.m8n8.trans.b16 %0, %1;" : "=r"(y) : "r"(x));
+    return y;
+}
+// two floats -> packed bf16x2 (lo in the low half), round to nearest even
+__device__ __forceinline__ uint32_t pack_bf16(float lo, float hi) {
+    uint32_t r;
+    asm("cvt.rn.bf16x2.f32 %0, %1, %2;" : "=r"(r) : "f"(hi), "f"(lo));
+    return r;
+}
+__device__ __forceinline__ float bf16lo_f(uint32_t x) { return __uint_as_float(x << 16); }
+__device__ __forceinline__ float bf16hi_f(uint32_t x) { return __uint_as_float(x & 0xffff0000u); }
+
+struct StageDesc { int kind, rows, seg, pad; };
+
+template <int R>
+struct Tc {
+    static constexpr int kBlob = 2 * (kPage * R + R * kHeadDim) * 2;
+    static constexpr int kStage = kBlob > 8192 ? kBlob : 8192;
+    static constexpr int kDB = kStage >= 16384 ? 32 : 16;      // dense block tokens
+    static constexpr int kAk = 0, kBk = kPage * R * 2, kAv = kBk + R * kHeadDim * 2, kBv = kAv + kPage * R * 2;
+    static constexpr int kNT = R / 8;                          // 8-wide rank tiles
+};
+
+// Per-warp running state for the query heads 2t, 2t+1 (t = lane & 3) of one KV head.
+struct WarpState {
+    float o[8][4];        // o[i]: (d = 16i+g, heads 2t,2t+1), (d = 16i+8+g, heads 2t,2t+1);  g = lane >> 2
+    float m[2], l[2];     // l is this lane's share; summed over g at flush time
+};
+
+template <int NTOK>       // softmax over NTOK/16 score tiles; returns p in place and the movmatrix'ed bf16 copies
+__device__ __forceinline__ void online_softmax(float (&s)[4][4], WarpState &st, uint32_t (&T0)[4], uint32_t (&T1)[4]) {
+    constexpr int NI = NTOK / 16;
+    float mx0 = kNegInf, mx1 = kNegInf;
+#pragma unroll
+    for (int i = 0; i < NI; ++i) {
+        mx0 = fmaxf(mx0, fmaxf(s[i][0], s[i][2]));
+        mx1 = fmaxf(mx1, fmaxf(s[i][1], s[i][3]));
+    }
+#pragma unroll
+    for (int off = 4; off <= 16; off <<= 1) {
+        mx0 = fmaxf(mx0, __shfl_xor_sync(0xffffffffu, mx0, off));
+        mx1 = fmaxf(mx1, __shfl_xor_sync(0xffffffffu, mx1, off));
+    }
+    const float mn0 = fmaxf(st.m[0], mx0), mn1 = fmaxf(st.m[1], mx1);
+    const float al0 = exp2f(st.m[0] - mn0), al1 = exp2f(st.m[1] - mn1);
+    st.m[0] = mn0; st.m[1] = mn1;
+    float sum0 = 0.f, sum1 = 0.f;
+#pragma unroll
+    for (int i = 0; i < NI; ++i) {
+        s[i][0] = exp2f(s[i][0] - mn0); s[i][2] = exp2f(s[i][2] - mn0);
+        s[i][1] = exp2f(s[i][1] - mn1); s[i][3] = exp2f(s[i][3] - mn1);
+        sum0 += s[i][0] + s[i][2];
+        sum1 += s[i][1] + s[i][3];
+    }
+    st.l[0] = st.l[0] * al0 + sum0;
+    st.l[1] = st.l[1] * al1 + sum1;
+    if (__any_sync(0xffffffffu, al0 != 1.f || al1 != 1.f)) {
+#pragma unroll
+        for (int i = 0; i < 8; ++i) { st.o[i][0] *= al0; st.o[i][1] *= al1; st.o[i][2] *= al0; st.o[i][3] *= al1; }
+    }
+#pragma unroll
+    for (int i = 0; i < NI; ++i) {
+        T0[i] = movm_t(pack_bf16(s[i][0], s[i][1]));   // (head g; tokens 16i+2t, +1)
+        T1[i] = movm_t(pack_bf16(s[i][2], s[i][3]));   // (head g; tokens 16i+8+2t, +1)
+    }
+}
+
+template <int R>
+__device__ __forceinline__ void factor_unit(uint32_t sb, const uint32_t (&qf)[8][2], float scale, WarpState &st, int lane) {
+    using C = Tc<R>;
+    const int l7 = lane & 7, mi = lane >> 3;
+    // ---- q~^T [G][R] = q [G][d] . B_k^T ----
+    float qt[C::kNT][4];
+    uint32_t qhi[C::kNT], qlo[C::kNT];
+#pragma unroll
+    for (int j = 0; j < C::kNT; ++j) {
+        qt[j][0] = qt[j][1] = qt[j][2] = qt[j][3] = 0.f;
+#pragma unroll
+        for (int qd = 0; qd < 4; ++qd) {
+            uint32_t b[4];
+            ldsm_x4(b, sb + C::kBk + (8 * j + l7) * kRowBytes + (((4 * qd + mi) ^ l7) << 4));
+            mma16816(qt[j], qf[2 * qd][0], 0u, qf[2 * qd][1], 0u, b[0], b[1]);
+            mma16816(qt[j], qf[2 * qd + 1][0], 0u, qf[2 * qd + 1][1], 0u, b[2], b[3]);
+        }
+        const float x0 = qt[j][0] * scale, x1 = qt[j][1] * scale;
+        qhi[j] = pack_bf16(x0, x1);
+        qlo[j] = pack_bf16(x0 - bf16lo_f(qhi[j]), x1 - bf16hi_f(qhi[j]));
+    }
+    // ---- s [P][G] = A_k [P][R] . q~ ----
+    float s[4][4];
+#pragma unroll
+    for (int i = 0; i < 4; ++i) {
+        s[i][0] = s[i][1] = s[i][2] = s[i][3] = 0.f;
+#pragma unroll
+        for (int kk = 0; kk < R / 16; ++kk) {
+            uint32_t av[4];
+            ldsm_x4(av, sb + C::kAk + (16 * i + (mi & 1) * 8 + l7) * (2 * R) + ((2 * kk + (mi >> 1)) << 4));
+            mma16816(s[i], av[0], av[1], av[2], av[3], qhi[2 * kk], qhi[2 * kk + 1]);
+            mma16816(s[i], av[0], av[1], av[2], av[3], qlo[2 * kk], qlo[2 * kk + 1]);
+        }
+        if (R % 16 == 8) {
+            uint32_t av[2];
+            ldsm_x2(av, sb + C::kAk + (16 * i + (mi & 1) * 8 + l7) * (2 * R) + ((R / 8 - 1) << 4));
+            mma1688(s[i], av[0], av[1], qhi[C::kNT - 1]);
+            mma1688(s[i], av[0], av[1], qlo[C::kNT - 1]);
+        }
+    }
+    uint32_t T0[4], T1[4];
+    online_softmax<kPage>(s, st, T0, T1);
+    // ---- w^T [G][R] = p^T [G][P] . A_v [P][R] ----
+    uint32_t wh[C::kNT];
+#pragma unroll
+    for (int j = 0; j < C::kNT; ++j) {
+        float wt[4] = {0.f, 0.f, 0.f, 0.f};
+#pragma unroll
+        for (int qd = 0; qd < 2; ++qd) {
+            uint32_t b[4];
+            ldsm_x4_t(b, sb + C::kAv + (16 * (2 * qd + (mi >> 1)) + (mi & 1) * 8 + l7) * (2 * R) + (j << 4));
+            mma16816(wt, T0[2 * qd], 0u, T1[2 * qd], 0u, b[0], b[1]);
+            mma16816(wt, T0[2 * qd + 1], 0u, T1[2 * qd + 1], 0u, b[2], b[3]);
+        }
+        wh[j] = pack_bf16(wt[0], wt[1]);
+    }
+    // ---- o [d][G] += B_v^T [d][R] . w ----
+#pragma unroll
+    for (int i = 0; i < 8; ++i) {
+#pragma unroll
+        for (int kk = 0; kk < R / 16; ++kk) {
+            uint32_t av[4];
+            ldsm_x4_t(av, sb + C::kBv + (16 * kk + (mi >> 1) * 8 + l7) * kRowBytes + (((2 * i + (mi & 1)) ^ l7) << 4));
+            mma16816(st.o[i], av[0], av[1], av[2], av[3], wh[2 * kk], wh[2 * kk + 1]);
+        }
+        if (R % 16 == 8) {
+            uint32_t av[2];
+            ldsm_x2_t(av, sb + C::kBv + (R - 8 + l7) * kRowBytes + (((2 * i + (mi & 1)) ^ l7) << 4));
+            mma1688(st.o[i], av[0], av[1], wh[C::kNT - 1]);
+        }
+    }
+}
+
+template <int R>
+__device__ __forceinline__ void dense_unit(uint32_t sb, unsigned char *sp, int rows, const uint32_t (&qf)[8][2],
+                                           float scale, WarpState &st, int lane) {
+    using C = Tc<R>;
+    constexpr int DB = C::kDB, NI = DB / 16;
+    const int l7 = lane & 7, mi = lane >> 3, g = lane >> 2;
+    if (rows < DB) {
+        // unfilled V rows hold stale bytes: zero them so that 0 * garbage cannot make a NaN
+        uint4 *v = reinterpret_cast<uint4 *>(sp + DB * kRowBytes + rows * kRowBytes);
+        for (int i = lane; i < (DB - rows) * 16; i += 32) v[i] = make_uint4(0u, 0u, 0u, 0u);
+        __syncwarp();
+    }
+    float s[4][4];
+#pragma unroll
+    for (int i = 0; i < NI; ++i) {
+        s[i][0] = s[i][1] = s[i][2] = s[i][3] = 0.f;
+#pragma unroll
+        for (int kk = 0; kk < 8; ++kk) {
+            uint32_t av[4];
+            ldsm_x4(av, sb + (16 * i + (mi & 1) * 8 + l7) * kRowBytes + (((2 * kk + (mi >> 1)) ^ l7) << 4));
+            mma16816(s[i], av[0], av[1], av[2], av[3], qf[kk][0], qf[kk][1]);
+        }
+        const bool v0 = 16 * i + g < rows, v1 = 16 * i + 8 + g < rows;
+        s[i][0] = v0 ? s[i][0] * scale : kNegInf; s[i][1] = v0 ? s[i][1] * scale : kNegInf;
+        s[i][2] = v1 ? s[i][2] * scale : kNegInf; s[i][3] = v1 ? s[i][3] * scale : kNegInf;
+    }
+    uint32_t T0[4], T1[4];
+    online_softmax<DB>(s, st, T0, T1);
+#pragma unroll
+    for (int ii = 0; ii < 8; ++ii) {
+#pragma unroll
+        for (int i = 0; i < NI; ++i) {
+            uint32_t av[4];
+            ldsm_x4_t(av, sb + DB * kRowBytes + (16 * i + (mi >> 1) * 8 + l7) * kRowBytes +
+                              (((2 * ii + (mi & 1)) ^ l7) << 4));
+            mma16816(st.o[ii], av[0], av[1], av[2], av[3], T0[i], T1[i]);
+        }
+    }
+}
+
+__device__ __forceinline__ void reset_state(WarpState &st) {
+#pragma unroll
+    for (int i = 0; i < 8; ++i) st.o[i][0] = st.o[i][1] = st.o[i][2] = st.o[i][3] = 0.f;
+    st.m[0] = st.m[1] = kNegInf;
+    st.l[0] = st.l[1] = 0.f;
+}
+
+__device__ __forceinline__ void load_q(const DecodeArgs &a, int seg, uint32_t (&qf)[8][2], int lane) {
+    const int H = a.geo.n_kv_heads, G = a.geo.group;
+    const int entry = seg / H, head = seg % H, g = lane >> 2, t = lane & 3;
+    if (g < G) {
+        const uint32_t *q = reinterpret_cast<const uint32_t *>(
+            reinterpret_cast<const __nv_bfloat16 *>(a.q) + ((long long)entry * a.geo.n_q_heads + head * G + g) * kHeadDim);
+#pragma unroll
+        for (int kk = 0; kk < 8; ++kk) { qf[kk][0] = __ldg(q + 8 * kk + t); qf[kk][1] = __ldg(q + 8 * kk + 4 + t); }
+    } else {
+#pragma unroll
+        for (int kk = 0; kk < 8; ++kk) qf[kk][0] = qf[kk][1] = 0u;
+    }
+}
+
+// All consumer warps combine their states of one segment; the CTA writes one partial.
+__device__ __forceinline__ void flush_segment(const DecodeArgs &a, float *comb, WarpState &st, int seg, int warp, int lane,
+                                              int ctid) {
+    const int g = lane >> 2, t = lane & 3;
+    float l0 = st.l[0], l1 = st.l[1];
+#pragma unroll
+    for (int off = 4; off <= 16; off <<= 1) {
+        l0 += __shfl_xor_sync(0xffffffffu, l0, off);
+        l1 += __shfl_xor_sync(0xffffffffu, l1, off);
+    }
+    float *mine = comb + warp * kPartialFloats;
+#pragma unroll
+    for (int i = 0; i < 8; ++i) {
+        mine[(2 * t) * kHeadDim + 16 * i + g] = st.o[i][0];
+        mine[(2 * t + 1) * kHeadDim + 16 * i + g] = st.o[i][1];
+        mine[(2 * t) * kHeadDim + 16 * i + 8 + g] = st.o[i][2];
+        mine[(2 * t + 1) * kHeadDim + 16 * i + 8 + g] = st.o[i][3];
+    }
+    if (g == 0) {
+        mine[kMaxGroup * kHeadDim + 2 * t] = st.m[0];
+        mine[kMaxGroup * kHeadDim + 2 * t + 1] = st.m[1];
+        mine[kMaxGroup * kHeadDim + kMaxGroup + 2 * t] = l0;
+        mine[kMaxGroup * kHeadDim + kMaxGroup + 2 * t + 1] = l1;
+    }
+    asm volatile("bar.sync 1, %0;" ::"n"(kConsumerWarps * 32) : "memory");
+    {
+        const int hq = ctid >> 5, d4 = (ctid & 31) * 4;
+        float M = kNegInf;
+#pragma unroll
+        for (int w = 0; w < kConsumerWarps; ++w) M = fmaxf(M, comb[w * kPartialFloats + kMaxGroup * kHeadDim + hq]);
+        float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
+        float L = 0.f;
+#pragma unroll
+        for (int w = 0; w < kConsumerWarps; ++w) {
+            const float *cw = comb + w * kPartialFloats;
+            const float f = exp2f(cw[kMaxGroup * kHeadDim + hq] - M);
+            const float4 o = *reinterpret_cast<const float4 *>(cw + hq * kHeadDim + d4);
+            acc.x += f * o.x; acc.y += f * o.y; acc.z += f * o.z; acc.w += f * o.w;
+            L += f * cw[kMaxGroup * kHeadDim + kMaxGroup + hq];
+        }
+        float *part = a.partials + ((long long)blockIdx.x + seg) * kPartialFloats;
+        *reinterpret_cast<float4 *>(part + hq * kHeadDim + d4) = acc;
+        if ((ctid & 31) == 0) {
+            part[kMaxGroup * kHeadDim + hq] = M;
+            part[kMaxGroup * kHeadDim + kMaxGroup + hq] = L;
+        }
+    }
+    asm volatile("bar.sync 1, %0;" ::"n"(kConsumerWarps * 32) : "memory");
+}
+
+template <int R>
+__global__ void __launch_bounds__(kDecodeThreads, 1) decode_tc_kernel(const __grid_constant__ DecodeArgs a) {
+    using C = Tc<R>;
+    Range rg;
+    if (!load_range(a, rg)) return;
+    const Geometry &geo = a.geo;
+    const int S = geo.n_stages;
+    extern __shared__ __align__(1024) unsigned char smem[];
+    unsigned char *stages = smem;
+    float *comb = reinterpret_cast<float *>(smem + (size_t)S * C::kStage);
+    unsigned long long *full_bar = reinterpret_cast<unsigned long long *>(comb + kConsumerWarps * kPartialFloats);
+    unsigned long long *empty_bar = full_bar + S;
+    StageDesc *descs = reinterpret_cast<StageDesc *>(empty_bar + S);
+    volatile int *abort_flag = reinterpret_cast<volatile int *>(descs + S);
+
+    const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+    if (tid == 0) {
+        for (int s = 0; s < S; ++s) { mbar_init(smem_u32(full_bar + s), 1); mbar_init(smem_u32(empty_bar + s), 1); }
+        *abort_flag = 0;
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    }
+    __syncthreads();
+
+    if (warp == kConsumerWarps) {
+        // ------------------------------ producer ------------------------------
+        const PlanEntry *entries = reinterpret_cast<const PlanEntry *>(a.plan + a.plan_entry);
+        int k = 0, seg_local = 0;
+        bool ok = true;
+        PlanCta cur = rg.start;
+        while (ok && !(cur.entry == rg.end.entry && cur.head == rg.end.head && cur.unit == rg.end.unit)) {
+            const PlanEntry e = entries[cur.entry];
+            const HeadUnits hu = head_units(geo, e);
+            const bool last_run = cur.entry == rg.end.entry && cur.head == rg.end.head;
+            const int u_end = last_run ? rg.end.unit : hu.units;
+            const int T = a.n_tokens[(long long)e.seq * geo.n_layers + a.layer];
+            const int *pt = a.page_table + ((long long)e.seq * geo.n_layers + a.layer) * geo.max_pages;
+            for (int u0 = cur.unit; u0 < u_end && ok; u0 += 32) {
+                const int u = u0 + lane;
+                int kind = kKindDense, rows = 0;
+                const unsigned char *src = nullptr;
+                if (u < u_end) {
+                    int page, blk;
+                    unit_to_page(geo, hu, u, page, blk, kind);
+                    const int slot = pt[page];
+                    if (kind == kKindFactor) {
+                        rows = kPage;
+                        src = a.factor_pool + (long long)slot * geo.factor_slot_bytes + (long long)cur.head * geo.blob_bytes;
+                    } else {
+                        rows = max(0, min(C::kDB, T - page * kPage - blk * C::kDB));
+                        src = a.dense_pool + (long long)slot * geo.dense_slot_bytes +
+                              (long long)cur.head * geo.dense_head_bytes + blk * C::kDB * kRowBytes;
+                    }
+                }
+                const int n_here = min(32, u_end - u0);
+                for (int j = 0; j < n_here && ok; ++j) {
+                    const int kind_j = __shfl_sync(0xffffffffu, kind, j);
+                    const int rows_j = __shfl_sync(0xffffffffu, rows, j);
+                    const unsigned long long src_j = __shfl_sync(0xffffffffu, (unsigned long long)src, j);
+                    if (lane == 0) {
+                        const int s = k % S;
+                        if (k >= S && !mbar_wait(smem_u32(empty_bar + s), ((k / S) - 1) & 1)) ok = false;
+                        if (ok) {
+                            descs[s] = StageDesc{kind_j, rows_j, seg_local, 0};
+                            const uint32_t bar = smem_u32(full_bar + s);
+                            const uint32_t dst = smem_u32(stages + (size_t)s * C::kStage);
+                            if (kind_j == kKindFactor) {
+                                mbar_arrive_expect_tx(bar, C::kBlob);
+                                bulk_g2s(dst, (const void *)src_j, C::kBlob, bar);
+                            } else if (rows_j > 0) {
+                                mbar_arrive_expect_tx(bar, 2 * rows_j * kRowBytes);
+                                bulk_g2s(dst, (const void *)src_j, rows_j * kRowBytes, bar);
+                                bulk_g2s(dst + C::kDB * kRowBytes, (const unsigned char *)src_j + kPage * kRowBytes,
+                                         rows_j * kRowBytes, bar);
+                            } else {
+                                mbar_arrive(bar);
+                            }
+                        }
+                    }
+                    ok = __shfl_sync(0xffffffffu, (int)ok, 0) != 0;
+                    ++k;
+                }
+            }
+            if (last_run) break;
+            cur.unit = 0;
+            if (++cur.head == geo.n_kv_heads) { cur.head = 0; ++cur.entry; }
+            ++seg_local;
+        }
+        // one end marker per consumer warp
+        for (int w = 0; w < kConsumerWarps && ok; ++w, ++k) {
+            if (lane == 0) {
+                const int s = k % S;
+                if (k >= S && !mbar_wait(smem_u32(empty_bar + s), ((k / S) - 1) & 1)) ok = false;
+                if (ok) {
+                    descs[s] = StageDesc{kKindEnd, 0, rg.n_local_segs, 0};
+                    mbar_arrive(smem_u32(full_bar + s));
+                }
+            }
+            ok = __shfl_sync(0xffffffffu, (int)ok, 0) != 0;
+        }
+        if (!ok && lane == 0) {
+            *abort_flag = 1;
+            atomicAdd(a.status, 1);
+            // let copies already in flight land before the CTA retires
+            for (int back = 1; back <= min(k, S); ++back) {
+                const int kk = k - back;
+                (void)mbar_wait(smem_u32(full_bar + kk % S), (kk / S) & 1);
+            }
+        }
+    } else {
+        // ------------------------------ consumers ------------------------------
+        WarpState st;
+        reset_state(st);
+        uint32_t qf[8][2];
+        int cur_seg = 0;
+        load_q(a, rg.seg_first, qf, lane);
+        bool ok = true;
+        for (int k = warp;; k += kConsumerWarps) {
+            const int s = k % S;
+            if (ok && (*abort_flag || !mbar_wait(smem_u32(full_bar + s), (k / S) & 1))) {
+                ok = false;
+                if (lane == 0) { *abort_flag = 1; atomicAdd(a.status, 1); }
+            }
+            StageDesc dsc = ok ? descs[s] : StageDesc{kKindEnd, 0, rg.n_local_segs, 0};
+            while (cur_seg < dsc.seg) {
+                flush_segment(a, comb, st, rg.seg_first + cur_seg, warp, lane, tid);
+                ++cur_seg;
+                reset_state(st);
+                if (cur_seg < rg.n_local_segs) load_q(a, rg.seg_first + cur_seg, qf, lane);
+            }
+            if (dsc.kind == kKindEnd) break;
+            if (dsc.rows > 0) {
+                const uint32_t sb = smem_u32(stages + (size_t)s * C::kStage);
+                if (dsc.kind == kKindFactor) {
+                    factor_unit<R>(sb, qf, geo.scale_log2e, st, lane);
+                } else {
+                    dense_unit<R>(sb, stages + (size_t)s * C::kStage, dsc.rows, qf, geo.scale_log2e, st, lane);
+                    if (dsc.rows < C::kDB) asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+                }
+            }
+            __syncwarp();
+            if (lane == 0) mbar_arrive(smem_u32(empty_bar + s));
+        }
+    }
+}
+
+template <int R>
+cudaError_t launch_tc(const DecodeArgs &a, cudaStream_t st) {
+    using C = Tc<R>;
+    const size_t smem = (size_t)a.geo.n_stages * C::kStage + kConsumerWarps * kPartialFloats * 4 +
+                        a.geo.n_stages * (8 + 8 + sizeof(StageDesc)) + 64;
+    decode_tc_kernel<R><<<a.geo.n_ctas, kDecodeThreads, smem, st>>>(a);
+    return cudaGetLastError();
+}
+
+}  // namespace
+
+cudaError_t decode_kernel_setup() {
+    cudaError_t e;
+    const int max_smem = kSmemBudget;
+    if ((e = cudaFuncSetAttribute(decode_tc_kernel<8>, cudaFuncAttributeMaxDynamicSharedMemorySize, max_smem)) != cudaSuccess) return e;
+    if ((e = cudaFuncSetAttribute(decode_tc_kernel<16>, cudaFuncAttributeMaxDynamicSharedMemorySize, max_smem)) != cudaSuccess) return e;
+    if ((e = cudaFuncSetAttribute(decode_tc_kernel<24>, cudaFuncAttributeMaxDynamicSharedMemorySize, max_smem)) != cudaSuccess) return e;
+    if ((e = cudaFuncSetAttribute(decode_tc_kernel<32>, cudaFuncAttributeMaxDynamicSharedMemorySize, max_smem)) != cudaSuccess) return e;
+    return cudaSuccess;
+}
+
+cudaError_t launch_decode(const DecodeArgs &a, int n_segs, cudaStream_t st) {
+    cudaError_t e;
+    if (a.variant == 1) {
+        decode_scalar_kernel<<<a.geo.n_ctas, 128, 0, st>>>(a);
+        e = cudaGetLastError();
+    } else {
+        switch (a.geo.rank_k) {
+            case 8:  e = launch_tc<8>(a, st); break;
+            case 16: e = launch_tc<16>(a, st); break;
+            case 24: e = launch_tc<24>(a, st); break;
+            case 32: e = launch_tc<32>(a, st); break;
+            default: return cudaErrorInvalidValue;
+        }
+    }
+    if (e != cudaSuccess) return e;
+    merge_kernel<<<n_segs, 256, 0, st>>>(a);
+    return cudaGetLastError();
+}
+
+}  // namespace pkv

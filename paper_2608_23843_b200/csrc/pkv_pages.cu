@@ -1,0 +1,123 @@
+// Row scatter for pkv_append_kv and the format translators behind
+// pkv_read_factors / pkv_write_factors / pkv_read_dense.
+#include "pkv_internal.h"
+
+namespace pkv {
+
+namespace {
+
+// One thread moves one 16-byte chunk of one (token, KV head, K|V) row into the
+// swizzled dense page.  Block 0 also publishes the new token counts.
+__global__ void append_kernel(Geometry geo, unsigned char *dense_pool, const int *page_table, int *n_tokens,
+                              const AppendDesc *desc, int n_seqs, long long n_tok, int layer,
+                              const uint4 *k, const uint4 *v) {
+    const int H = geo.n_kv_heads;
+    const long long total = n_tok * H * 2 * 16;
+    for (long long idx = blockIdx.x * (long long)blockDim.x + threadIdx.x; idx < total;
+         idx += (long long)gridDim.x * blockDim.x) {
+        const int chunk = (int)(idx & 15);
+        long long rest = idx >> 4;
+        const int kv = (int)(rest & 1);
+        rest >>= 1;
+        const int h = (int)(rest % H);
+        const long long tok = rest / H;
+        // entry whose token range holds `tok`
+        int lo = 0, hi = n_seqs - 1;
+        while (lo < hi) {
+            int mid = (lo + hi + 1) >> 1;
+            if (desc[mid].tok_begin <= tok) lo = mid; else hi = mid - 1;
+        }
+        const AppendDesc e = desc[lo];
+        const int t = e.t_start + (int)(tok - e.tok_begin);
+        const int page = t / kPage, row = t % kPage;
+        const int slot = page_table[((long long)e.seq * geo.n_layers + layer) * geo.max_pages + page];
+        const uint4 val = (kv ? v : k)[(tok * H + h) * 16 + chunk];
+        unsigned char *dst = dense_pool + (long long)slot * geo.dense_slot_bytes + (long long)h * geo.dense_head_bytes +
+                             kv * (kPage * kRowBytes) + row * kRowBytes + swz_chunk(row, chunk) * 16;
+        *reinterpret_cast<uint4 *>(dst) = val;
+    }
+    if (blockIdx.x == 0) {
+        for (int i = threadIdx.x; i < n_seqs; i += blockDim.x) {
+            n_tokens[(long long)desc[i].seq * geo.n_layers + layer] = desc[i].t_start + desc[i].n_new;
+        }
+    }
+}
+
+// blob <-> row-major factors.  dir = 0: blob -> arrays, 1: arrays -> blob.
+__global__ void factor_io_kernel(Geometry geo, unsigned char *blob, unsigned short *A_k, unsigned short *B_k,
+                                 unsigned short *A_v, unsigned short *B_v, int dir) {
+    const int rk = geo.rank_k, rv = geo.rank_v;
+    const int nAk = kPage * rk, nBk = rk * kHeadDim, nAv = kPage * rv, nBv = rv * kHeadDim;
+    for (int i = blockIdx.x * blockDim.x + threadIdx.x; i < nAk + nBk + nAv + nBv; i += gridDim.x * blockDim.x) {
+        unsigned short *plain;
+        unsigned short *stored;
+        if (i < nAk) {                          // A_k: plain row-major [P][r_k]
+            plain = A_k + i;
+            stored = reinterpret_cast<unsigned short *>(blob + geo.ak_off) + i;
+        } else if (i < nAk + nBk) {             // B_k: rows of 256 B, chunk-swizzled
+            int j = i - nAk, row = j / kHeadDim, col = j % kHeadDim;
+            plain = B_k + j;
+            stored = reinterpret_cast<unsigned short *>(blob + geo.bk_off + row * kRowBytes +
+                                                        swz_chunk(row, col >> 3) * 16) + (col & 7);
+        } else if (i < nAk + nBk + nAv) {
+            int j = i - nAk - nBk;
+            plain = A_v + j;
+            stored = reinterpret_cast<unsigned short *>(blob + geo.av_off) + j;
+        } else {
+            int j = i - nAk - nBk - nAv, row = j / kHeadDim, col = j % kHeadDim;
+            plain = B_v + j;
+            stored = reinterpret_cast<unsigned short *>(blob + geo.bv_off + row * kRowBytes +
+                                                        swz_chunk(row, col >> 3) * 16) + (col & 7);
+        }
+        if (dir == 0) *plain = *stored; else *stored = *plain;
+    }
+}
+
+__global__ void dense_read_kernel(const unsigned char *head_base, unsigned short *K, unsigned short *V) {
+    for (int i = blockIdx.x * blockDim.x + threadIdx.x; i < 2 * kPage * kHeadDim; i += gridDim.x * blockDim.x) {
+        int kv = i / (kPage * kHeadDim), j = i % (kPage * kHeadDim), row = j / kHeadDim, col = j % kHeadDim;
+        const unsigned short *src = reinterpret_cast<const unsigned short *>(
+                                        head_base + kv * (kPage * kRowBytes) + row * kRowBytes +
+                                        swz_chunk(row, col >> 3) * 16) + (col & 7);
+        (kv ? V : K)[j] = *src;
+    }
+}
+
+}  // namespace
+
+cudaError_t launch_append(const Geometry &geo, unsigned char *dense_pool, const int *page_table,
+                          int *n_tokens, const AppendDesc *desc, int n_seqs, long long n_tok, int layer,
+                          const void *k, const void *v, cudaStream_t st) {
+    const long long total = n_tok * geo.n_kv_heads * 2 * 16;
+    const int threads = 256;
+    long long blocks = (total + threads - 1) / threads;
+    if (blocks > 148LL * 16) blocks = 148LL * 16;
+    if (blocks < 1) blocks = 1;
+    append_kernel<<<(unsigned)blocks, threads, 0, st>>>(geo, dense_pool, page_table, n_tokens, desc, n_seqs, n_tok,
+                                                        layer, (const uint4 *)k, (const uint4 *)v);
+    return cudaGetLastError();
+}
+
+cudaError_t launch_read_factors(const Geometry &geo, const unsigned char *blob, void *A_k, void *B_k,
+                                void *A_v, void *B_v, cudaStream_t st) {
+    factor_io_kernel<<<8, 256, 0, st>>>(geo, const_cast<unsigned char *>(blob), (unsigned short *)A_k,
+                                        (unsigned short *)B_k, (unsigned short *)A_v, (unsigned short *)B_v, 0);
+    return cudaGetLastError();
+}
+
+cudaError_t launch_write_factors(const Geometry &geo, unsigned char *blob, const void *A_k, const void *B_k,
+                                 const void *A_v, const void *B_v, cudaStream_t st) {
+    factor_io_kernel<<<8, 256, 0, st>>>(geo, blob, (unsigned short *)const_cast<void *>(A_k),
+                                        (unsigned short *)const_cast<void *>(B_k),
+                                        (unsigned short *)const_cast<void *>(A_v),
+                                        (unsigned short *)const_cast<void *>(B_v), 1);
+    return cudaGetLastError();
+}
+
+cudaError_t launch_read_dense(const Geometry &, const unsigned char *head_base, void *K, void *V,
+                              cudaStream_t st) {
+    dense_read_kernel<<<16, 256, 0, st>>>(head_base, (unsigned short *)K, (unsigned short *)V);
+    return cudaGetLastError();
+}
+
+}  // namespace pkv

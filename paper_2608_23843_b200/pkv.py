@@ -1,0 +1,304 @@
+"""ctypes binding of libpkv.so (see include/pkv.h): argument marshalling only.
+
+Module-level functions carry the C names (`pkv_init_cache`, `pkv_append_kv`,
+`pkv_compress_eligible_pages`, `pkv_decode_attention`, ...).  `Cache` is a
+convenience wrapper that allocates the caller-owned device buffers with torch
+and forwards to those functions; every computation runs in the CUDA library.
+There is no CPU fallback: if the library has not been built, loading fails.
+"""
+import ctypes
+import os
+
+import torch
+
+_HERE = os.path.dirname(os.path.abspath(__file__))
+LIB_PATH = os.path.join(_HERE, "libpkv.so")
+
+PKV_OK = 0
+PKV_ERR_INVALID_ARG = -1
+PKV_ERR_POOL_EXHAUSTED = -2
+PKV_ERR_BAD_SEQ = -3
+PKV_ERR_CUDA = -4
+PKV_ERR_NOT_CONVERGED = -5
+PKV_ERR_UNSUPPORTED = -6
+PKV_ERR_DEVICE_TIMEOUT = -7
+PKV_KIND_DENSE, PKV_KIND_FACTOR = 0, 1
+
+EXPORTS = [
+    "pkv_query_sizes", "pkv_init_cache", "pkv_append_kv", "pkv_compress_eligible_pages",
+    "pkv_decode_attention", "pkv_decode_attention_host", "pkv_get_page_table", "pkv_get_stats",
+    "pkv_free_seq", "pkv_destroy_cache", "pkv_last_error", "pkv_read_factors", "pkv_write_factors",
+    "pkv_read_dense", "pkv_get_decode_plan",
+]
+
+
+class PkvConfig(ctypes.Structure):
+    _fields_ = [
+        ("n_layers", ctypes.c_int32), ("n_kv_heads", ctypes.c_int32), ("n_q_heads", ctypes.c_int32),
+        ("head_dim", ctypes.c_int32), ("page_size", ctypes.c_int32), ("rank_k", ctypes.c_int32),
+        ("rank_v", ctypes.c_int32), ("sink_tokens", ctypes.c_int32), ("recent_tokens", ctypes.c_int32),
+        ("max_seqs", ctypes.c_int32), ("max_pages_per_seq", ctypes.c_int32),
+        ("n_dense_slots", ctypes.c_int64), ("n_factor_slots", ctypes.c_int64),
+        ("softmax_scale", ctypes.c_float), ("jacobi_max_sweeps", ctypes.c_int32),
+        ("jacobi_tol", ctypes.c_float), ("n_ctas", ctypes.c_int32), ("decode_variant", ctypes.c_int32),
+    ]
+
+
+class PkvSizes(ctypes.Structure):
+    _fields_ = [(n, ctypes.c_int64) for n in ("dense_slot_bytes", "factor_slot_bytes", "dense_pool_bytes",
+                                              "factor_pool_bytes", "meta_bytes", "workspace_bytes")]
+
+
+class PkvStats(ctypes.Structure):
+    _fields_ = [(n, ctypes.c_int64) for n in ("dense_slots_in_use", "factor_slots_in_use", "pages_compressed",
+                                              "page_svds_not_converged", "device_timeouts",
+                                              "last_decode_bytes", "last_decode_units")]
+
+
+class PkvError(RuntimeError):
+    def __init__(self, status, message=""):
+        super().__init__("pkv status %d: %s" % (status, message))
+        self.status = status
+
+
+_lib = None
+
+
+def lib():
+    """The loaded CUDA library.  Raises if it has not been built."""
+    global _lib
+    if _lib is None:
+        if not os.path.exists(LIB_PATH):
+            raise RuntimeError("libpkv.so is missing: build it with `python -m paper_2608_23843_b200.build` "
+                               "(there is no CPU fallback)")
+        L = ctypes.CDLL(LIB_PATH)
+        vp, i32, i64 = ctypes.c_void_p, ctypes.c_int32, ctypes.c_int64
+        ip = ctypes.POINTER(ctypes.c_int32)
+        L.pkv_query_sizes.argtypes = [ctypes.POINTER(PkvConfig), ctypes.POINTER(PkvSizes)]
+        L.pkv_init_cache.argtypes = [ctypes.POINTER(PkvConfig), vp, vp, vp, vp, ip, ip, ctypes.POINTER(vp)]
+        L.pkv_append_kv.argtypes = [vp, i32, i32, ip, ip, vp, vp, vp]
+        L.pkv_compress_eligible_pages.argtypes = [vp, i32, ctypes.POINTER(i64), vp]
+        L.pkv_decode_attention.argtypes = [vp, i32, i32, ip, vp, vp, vp, vp]
+        L.pkv_decode_attention_host.argtypes = [vp, i32, i32, ip, vp, vp, vp, vp, vp]
+        L.pkv_get_page_table.argtypes = [vp, i32, i32, ip, ip, ip, ip]
+        L.pkv_get_stats.argtypes = [vp, ctypes.POINTER(PkvStats), vp]
+        L.pkv_free_seq.argtypes = [vp, i32]
+        L.pkv_destroy_cache.argtypes = [vp]
+        L.pkv_last_error.argtypes = [vp]
+        L.pkv_last_error.restype = ctypes.c_char_p
+        L.pkv_read_factors.argtypes = [vp, i64, i32, vp, vp, vp, vp, vp]
+        L.pkv_write_factors.argtypes = [vp, i64, i32, vp, vp, vp, vp, vp]
+        L.pkv_read_dense.argtypes = [vp, i64, i32, vp, vp, vp]
+        L.pkv_get_decode_plan.argtypes = [vp, i32, ip, ip, ip, ip]
+        for name in EXPORTS:
+            if name != "pkv_last_error":
+                getattr(L, name).restype = ctypes.c_int32
+        _lib = L
+    return _lib
+
+
+def _ints(xs):
+    xs = [int(x) for x in xs]
+    return (ctypes.c_int32 * len(xs))(*xs), len(xs)
+
+
+def _ptr(t):
+    return None if t is None else ctypes.c_void_p(t.data_ptr())
+
+
+def _stream(stream):
+    if stream is None:
+        return None
+    if isinstance(stream, int):
+        return ctypes.c_void_p(stream)
+    return ctypes.c_void_p(stream.cuda_stream)
+
+
+# ---- functions with the C names -------------------------------------------------
+def pkv_query_sizes(cfg: PkvConfig) -> PkvSizes:
+    out = PkvSizes()
+    st = lib().pkv_query_sizes(ctypes.byref(cfg), ctypes.byref(out))
+    if st != PKV_OK:
+        raise PkvError(st, "pkv_query_sizes")
+    return out
+
+
+def pkv_init_cache(cfg, dense_pool, factor_pool, meta, workspace, dense_slot_order=None, factor_slot_order=None):
+    """Tensors (or None for all four = dry run) -> opaque handle."""
+    h = ctypes.c_void_p()
+    d_ord = f_ord = None
+    if dense_slot_order is not None:
+        d_ord, _ = _ints(dense_slot_order)
+    if factor_slot_order is not None:
+        f_ord, _ = _ints(factor_slot_order)
+    st = lib().pkv_init_cache(ctypes.byref(cfg), _ptr(dense_pool), _ptr(factor_pool), _ptr(meta), _ptr(workspace),
+                              d_ord, f_ord, ctypes.byref(h))
+    if st != PKV_OK:
+        raise PkvError(st, "pkv_init_cache")
+    return h
+
+
+def _check(handle, st):
+    if st != PKV_OK:
+        raise PkvError(st, lib().pkv_last_error(handle).decode())
+
+
+def pkv_append_kv(handle, layer, seq_ids, n_new, k, v, stream=None):
+    ids, n = _ints(seq_ids)
+    cnt, _ = _ints(n_new)
+    _check(handle, lib().pkv_append_kv(handle, layer, n, ids, cnt, _ptr(k), _ptr(v), _stream(stream)))
+
+
+def pkv_compress_eligible_pages(handle, layer=-1, stream=None) -> int:
+    n = ctypes.c_int64(0)
+    st = lib().pkv_compress_eligible_pages(handle, layer, ctypes.byref(n), _stream(stream))
+    _check(handle, st)
+    return int(n.value)
+
+
+def pkv_decode_attention(handle, layer, seq_ids, q, out, out_f32=None, stream=None):
+    ids, n = _ints(seq_ids)
+    _check(handle, lib().pkv_decode_attention(handle, layer, n, ids, _ptr(q), _ptr(out), _ptr(out_f32), _stream(stream)))
+
+
+def pkv_decode_attention_host(handle, layer, seq_ids, q_host, out_host, q_stage, out_stage, stream=None):
+    ids, n = _ints(seq_ids)
+    _check(handle, lib().pkv_decode_attention_host(handle, layer, n, ids, _ptr(q_host), _ptr(out_host),
+                                                   _ptr(q_stage), _ptr(out_stage), _stream(stream)))
+
+
+def pkv_get_page_table(handle, seq, layer, max_pages):
+    kinds = (ctypes.c_int32 * max_pages)()
+    slots = (ctypes.c_int32 * max_pages)()
+    n_pages, n_tokens = ctypes.c_int32(0), ctypes.c_int32(0)
+    st = lib().pkv_get_page_table(handle, seq, layer, kinds, slots, ctypes.byref(n_pages), ctypes.byref(n_tokens))
+    if st != PKV_OK:
+        raise PkvError(st, "pkv_get_page_table")
+    n = n_pages.value
+    return list(kinds[:n]), list(slots[:n]), int(n_tokens.value)
+
+
+def pkv_get_stats(handle, stream=None) -> dict:
+    s = PkvStats()
+    _check(handle, lib().pkv_get_stats(handle, ctypes.byref(s), _stream(stream)))
+    return {n: int(getattr(s, n)) for n, _ in PkvStats._fields_}
+
+
+def pkv_get_decode_plan(handle, layer, n_ctas, n_seqs, n_kv_heads):
+    """-> (cta_starts [(position, head, unit)] incl. end sentinel, seg_parts [(cta_first, n_parts)])."""
+    starts = (ctypes.c_int32 * (3 * (n_ctas + 1)))()
+    segs = (ctypes.c_int32 * (2 * n_seqs * n_kv_heads))()
+    n_used, n_segs = ctypes.c_int32(0), ctypes.c_int32(0)
+    st = lib().pkv_get_decode_plan(handle, layer, ctypes.byref(n_used), starts, ctypes.byref(n_segs), segs)
+    if st != PKV_OK:
+        raise PkvError(st, "pkv_get_decode_plan")
+    return ([tuple(starts[3 * j:3 * j + 3]) for j in range(n_used.value + 1)],
+            [tuple(segs[2 * s:2 * s + 2]) for s in range(n_segs.value)])
+
+
+def pkv_free_seq(handle, seq):
+    _check(handle, lib().pkv_free_seq(handle, seq))
+
+
+def pkv_destroy_cache(handle):
+    lib().pkv_destroy_cache(handle)
+
+
+def pkv_read_factors(handle, slot, kv_head, A_k, B_k, A_v, B_v, stream=None):
+    _check(handle, lib().pkv_read_factors(handle, slot, kv_head, _ptr(A_k), _ptr(B_k), _ptr(A_v), _ptr(B_v), _stream(stream)))
+
+
+def pkv_write_factors(handle, slot, kv_head, A_k, B_k, A_v, B_v, stream=None):
+    _check(handle, lib().pkv_write_factors(handle, slot, kv_head, _ptr(A_k), _ptr(B_k), _ptr(A_v), _ptr(B_v), _stream(stream)))
+
+
+def pkv_read_dense(handle, slot, kv_head, K, V, stream=None):
+    _check(handle, lib().pkv_read_dense(handle, slot, kv_head, _ptr(K), _ptr(V), _stream(stream)))
+
+
+# ---- convenience wrapper ----------------------------------------------------------
+def make_config(n_layers, n_kv_heads, n_q_heads, rank, sink_tokens, recent_tokens, max_seqs, max_pages_per_seq,
+                n_dense_slots, n_factor_slots, head_dim=128, page_size=64, rank_v=None, softmax_scale=0.0,
+                jacobi_max_sweeps=0, jacobi_tol=0.0, n_ctas=0, decode_variant=0) -> PkvConfig:
+    return PkvConfig(n_layers, n_kv_heads, n_q_heads, head_dim, page_size, rank, rank if rank_v is None else rank_v,
+                     sink_tokens, recent_tokens, max_seqs, max_pages_per_seq, n_dense_slots, n_factor_slots,
+                     softmax_scale, jacobi_max_sweeps, jacobi_tol, n_ctas, decode_variant)
+
+
+class Cache:
+    """Owns the device buffers (torch uint8 tensors) and the library handle."""
+
+    def __init__(self, cfg: PkvConfig, device="cuda", dense_slot_order=None, factor_slot_order=None, dry_run=False):
+        self.cfg = cfg
+        self.sizes = pkv_query_sizes(cfg)
+        self.dry_run = dry_run
+        if dry_run:
+            self.dense_pool = self.factor_pool = self.meta = self.workspace = None
+            self.stream = None
+        else:
+            self.device = torch.device(device)
+            mk = lambda n: torch.empty(max(int(n), 256), dtype=torch.uint8, device=self.device)
+            self.dense_pool, self.factor_pool = mk(self.sizes.dense_pool_bytes), mk(self.sizes.factor_pool_bytes)
+            self.meta, self.workspace = mk(self.sizes.meta_bytes), mk(self.sizes.workspace_bytes)
+        self.handle = pkv_init_cache(cfg, self.dense_pool, self.factor_pool, self.meta, self.workspace,
+                                     dense_slot_order, factor_slot_order)
+
+    def _st(self):
+        return None if self.dry_run else torch.cuda.current_stream(self.device)
+
+    def append_kv(self, layer, seq_ids, n_new, k=None, v=None):
+        pkv_append_kv(self.handle, layer, seq_ids, n_new, k, v, self._st())
+
+    def compress_eligible_pages(self, layer=-1):
+        return pkv_compress_eligible_pages(self.handle, layer, self._st())
+
+    def decode_attention(self, layer, seq_ids, q=None, out=None, out_f32=None):
+        if out is None and q is not None:
+            out = torch.empty_like(q)
+        pkv_decode_attention(self.handle, layer, seq_ids, q, out, out_f32, self._st())
+        return out
+
+    def decode_attention_host(self, layer, seq_ids, q_host, out_host, q_stage, out_stage):
+        pkv_decode_attention_host(self.handle, layer, seq_ids, q_host, out_host, q_stage, out_stage, self._st())
+
+    def page_table(self, seq, layer):
+        return pkv_get_page_table(self.handle, seq, layer, self.cfg.max_pages_per_seq)
+
+    def stats(self):
+        return pkv_get_stats(self.handle, self._st())
+
+    def free_seq(self, seq):
+        pkv_free_seq(self.handle, seq)
+
+    def read_factors(self, slot, kv_head):
+        c = self.cfg
+        mk = lambda *s: torch.empty(s, dtype=torch.bfloat16, device=self.device)
+        A_k, B_k = mk(c.page_size, c.rank_k), mk(c.rank_k, c.head_dim)
+        A_v, B_v = mk(c.page_size, c.rank_v), mk(c.rank_v, c.head_dim)
+        pkv_read_factors(self.handle, slot, kv_head, A_k, B_k, A_v, B_v, self._st())
+        return A_k, B_k, A_v, B_v
+
+    def write_factors(self, slot, kv_head, A_k, B_k, A_v, B_v):
+        ts = [t.to(device=self.device, dtype=torch.bfloat16).contiguous() for t in (A_k, B_k, A_v, B_v)]
+        pkv_write_factors(self.handle, slot, kv_head, *ts, self._st())
+        torch.cuda.current_stream(self.device).synchronize()     # keep `ts` alive until the copy kernel ran
+
+    def read_dense(self, slot, kv_head):
+        c = self.cfg
+        K = torch.empty((c.page_size, c.head_dim), dtype=torch.bfloat16, device=self.device)
+        V = torch.empty_like(K)
+        pkv_read_dense(self.handle, slot, kv_head, K, V, self._st())
+        return K, V
+
+    def close(self):
+        if self.handle is not None:
+            if not self.dry_run:
+                torch.cuda.synchronize(self.device)
+            pkv_destroy_cache(self.handle)
+            self.handle = None
+
+    def __del__(self):
+        try:
+            self.close()
+        except Exception:
+            pass

@@ -1,0 +1,233 @@
+"""Host logic of the CUDA library, exercised in dry-run mode (no GPU needed):
+exported symbols, page tables / eligibility / slot allocation bit-exact against
+the oracle's state machine, error codes, byte accounting and the decode plan."""
+import ctypes
+import os
+import re
+
+import numpy as np
+import pytest
+
+from oracle import accounting
+from oracle.cache import OracleCache, OracleConfig, PoolExhausted
+from paper_2608_23843_b200 import pkv
+
+ROOT = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
+
+
+@pytest.fixture(scope="module", autouse=True)
+def _built():
+    from paper_2608_23843_b200 import build
+    build.build()
+
+
+def test_library_exports_every_declared_symbol():
+    header = open(os.path.join(ROOT, "include", "pkv.h")).read()
+    header = re.sub(r"/\*.*?\*/", "", header, flags=re.S)
+    declared = set(re.findall(r"\b(pkv_[a-z_0-9]+)\s*\(", header))
+    assert declared, "no declarations parsed"
+    L = ctypes.CDLL(pkv.LIB_PATH)
+    for name in sorted(declared):
+        assert hasattr(L, name), "libpkv.so does not export %s" % name
+    assert declared == set(pkv.EXPORTS)
+
+
+def _pair(seed=None, **kw):
+    base = dict(n_layers=2, n_kv_heads=2, n_q_heads=8, rank=16, sink_tokens=64, recent_tokens=128,
+                max_seqs=4, max_pages_per_seq=64, n_dense_slots=96, n_factor_slots=96)
+    base.update(kw)
+    cfg = pkv.make_config(**base)
+    d_ord = f_ord = None
+    if seed is not None:
+        rng = np.random.default_rng(seed)
+        d_ord, f_ord = rng.permutation(base["n_dense_slots"]), rng.permutation(base["n_factor_slots"])
+    gpu = pkv.Cache(cfg, dry_run=True, dense_slot_order=d_ord, factor_slot_order=f_ord)
+    ocfg = OracleConfig(n_layers=base["n_layers"], n_kv_heads=base["n_kv_heads"], n_q_heads=base["n_q_heads"],
+                        head_dim=128, page_size=64, rank_k=base["rank"], rank_v=base["rank"],
+                        sink_tokens=base["sink_tokens"], recent_tokens=base["recent_tokens"],
+                        max_seqs=base["max_seqs"], n_dense_slots=base["n_dense_slots"],
+                        n_factor_slots=base["n_factor_slots"])
+    return gpu, OracleCache(ocfg, d_ord, f_ord), base
+
+
+def _oracle_append(orc, layer, seqs, n_new, H):
+    n = int(sum(n_new))
+    z = np.zeros((n, H, 128))
+    orc.append_kv(layer, seqs, n_new, z, z)
+
+
+def _same_tables(gpu, orc, base):
+    for s in range(base["max_seqs"]):
+        for ly in range(base["n_layers"]):
+            assert gpu.page_table(s, ly) == orc.page_table(s, ly), (s, ly)
+    st, ost = gpu.stats(), orc.stats()
+    assert st["dense_slots_in_use"] == ost["dense_in_use"]
+    assert st["factor_slots_in_use"] == ost["factor_in_use"]
+    assert st["pages_compressed"] == ost["pages_compressed"]
+
+
+def test_tiny_config_has_13_factor_pages():
+    gpu, orc, base = _pair(n_layers=1, n_kv_heads=1, n_q_heads=4, max_seqs=1)
+    gpu.append_kv(0, [0], [1024])
+    assert gpu.compress_eligible_pages() == 13
+    kinds, slots, T = gpu.page_table(0, 0)
+    assert T == 1024 and kinds == [0] + [1] * 13 + [0, 0]
+
+
+@pytest.mark.parametrize("seed", [0, 1, 2, 3])
+def test_random_schedule_matches_oracle_bit_exact(seed):
+    gpu, orc, base = _pair(seed=seed)
+    rng = np.random.default_rng(100 + seed)
+    H = base["n_kv_heads"]
+    for step in range(60):
+        op = rng.integers(0, 10)
+        if op < 6:
+            layer = int(rng.integers(0, base["n_layers"]))
+            k = int(rng.integers(1, base["max_seqs"] + 1))
+            seqs = [int(x) for x in rng.choice(base["max_seqs"], size=k, replace=False)]
+            n_new = [int(rng.choice([0, 1, 1, 1, 7, 64, 65, 200])) for _ in seqs]
+            try:
+                _oracle_append(orc, layer, seqs, n_new, H)
+                ok = True
+            except PoolExhausted:
+                pytest.skip("schedule overflowed the pool")   # not expected with these sizes
+            if ok:
+                gpu.append_kv(layer, seqs, n_new)
+        elif op < 9:
+            layer = int(rng.integers(-1, base["n_layers"]))
+            # the oracle factorizes zero pages here: cheap, and keeps slot numbering identical
+            assert gpu.compress_eligible_pages(layer) == orc.compress_eligible_pages(layer)
+        else:
+            s = int(rng.integers(0, base["max_seqs"]))
+            orc.free_seq(s)
+            gpu.free_seq(s)
+        _same_tables(gpu, orc, base)
+
+
+def test_incremental_conversion_is_one_page_per_boundary_step():
+    gpu, orc, base = _pair(n_layers=1, max_seqs=2, sink_tokens=64, recent_tokens=256)
+    gpu.append_kv(0, [0, 1], [8192 // 16, 8192 // 16])
+    gpu.compress_eligible_pages()
+    T0 = 8192 // 16
+    for t in range(T0, T0 + 130):
+        gpu.append_kv(0, [0, 1], [1, 1])
+        n = gpu.compress_eligible_pages(0)
+        assert n == (2 if (t + 1) % 64 == 0 else 0)
+    kinds, _, T = gpu.page_table(1, 0)
+    lo, hi = 1, T // 64 - 4
+    assert [i for i, k in enumerate(kinds) if k == 1] == list(range(lo, hi))
+
+
+def test_error_codes_and_unchanged_state_on_failure():
+    gpu, orc, base = _pair(n_dense_slots=3, n_factor_slots=1, n_layers=1)
+    with pytest.raises(pkv.PkvError) as e:
+        gpu.append_kv(0, [0], [64 * 4])
+    assert e.value.status == pkv.PKV_ERR_POOL_EXHAUSTED and gpu.page_table(0, 0) == ([], [], 0)
+    with pytest.raises(pkv.PkvError) as e:
+        gpu.append_kv(0, [0, 0], [1, 1])
+    assert e.value.status == pkv.PKV_ERR_BAD_SEQ
+    with pytest.raises(pkv.PkvError) as e:
+        gpu.append_kv(0, [9], [1])
+    assert e.value.status == pkv.PKV_ERR_BAD_SEQ
+    with pytest.raises(pkv.PkvError) as e:
+        gpu.append_kv(5, [0], [1])
+    assert e.value.status == pkv.PKV_ERR_INVALID_ARG
+    with pytest.raises(pkv.PkvError) as e:
+        gpu.decode_attention(0, [0])                                  # empty sequence
+    assert e.value.status == pkv.PKV_ERR_INVALID_ARG
+    gpu.append_kv(0, [0], [64 * 3])
+    gpu.free_seq(0)
+    gpu2, _, _ = _pair(n_dense_slots=8, n_factor_slots=1, n_layers=1, sink_tokens=0, recent_tokens=0)
+    gpu2.append_kv(0, [0], [64 * 3])
+    with pytest.raises(pkv.PkvError) as e:
+        gpu2.compress_eligible_pages()
+    assert e.value.status == pkv.PKV_ERR_POOL_EXHAUSTED
+    assert gpu2.page_table(0, 0)[0] == [1, 0, 0]                      # the page converted before exhaustion stays converted
+
+
+def test_config_validation():
+    ok = dict(n_layers=1, n_kv_heads=1, n_q_heads=4, rank=16, sink_tokens=64, recent_tokens=64, max_seqs=1,
+              max_pages_per_seq=4, n_dense_slots=4, n_factor_slots=4)
+    pkv.pkv_query_sizes(pkv.make_config(**ok))
+    for bad, status in [(dict(sink_tokens=10), pkv.PKV_ERR_INVALID_ARG), (dict(recent_tokens=65), pkv.PKV_ERR_INVALID_ARG),
+                        (dict(n_q_heads=3, n_kv_heads=2), pkv.PKV_ERR_INVALID_ARG), (dict(rank=0), pkv.PKV_ERR_INVALID_ARG),
+                        (dict(rank=65), pkv.PKV_ERR_INVALID_ARG), (dict(rank=12), pkv.PKV_ERR_UNSUPPORTED),
+                        (dict(head_dim=64, page_size=64), pkv.PKV_ERR_UNSUPPORTED), (dict(page_size=32), pkv.PKV_ERR_UNSUPPORTED),
+                        (dict(n_q_heads=16), pkv.PKV_ERR_UNSUPPORTED), (dict(rank=16, rank_v=8), pkv.PKV_ERR_UNSUPPORTED)]:
+        with pytest.raises(pkv.PkvError) as e:
+            pkv.pkv_query_sizes(pkv.make_config(**{**ok, **bad}))
+        assert e.value.status == status, bad
+    with pytest.raises(pkv.PkvError):
+        pkv.Cache(pkv.make_config(**ok), dry_run=True, dense_slot_order=[0, 0, 1, 2])   # not a permutation
+
+
+def test_slot_sizes_follow_storage_ratio_formula():
+    for r in (8, 16, 24, 32):
+        sz = pkv.pkv_query_sizes(pkv.make_config(n_layers=1, n_kv_heads=8, n_q_heads=32, rank=r, sink_tokens=64,
+                                                 recent_tokens=256, max_seqs=1, max_pages_per_seq=8,
+                                                 n_dense_slots=8, n_factor_slots=8))
+        assert sz.dense_slot_bytes == 8 * 2 * 64 * 128 * 2
+        assert sz.factor_slot_bytes / sz.dense_slot_bytes == accounting.page_storage_ratio(r, r, 64, 128)
+
+
+def _decode_bytes(T, P, S, W, r, H_kv, H_q):
+    n_pages = -(-T // P)
+    lo, hi = S // P, max(S // P, T // P - W // P)
+    nf = max(0, min(hi, n_pages) - min(lo, n_pages))
+    dense_rows = T - nf * P
+    return H_kv * (nf * 2 * (P * r + r * 128) * 2 + dense_rows * 2 * 128 * 2) + 2 * H_q * 128 * 2
+
+
+def test_decode_byte_accounting_long_context_layer():
+    # 64q/8kv, T=131072, r=24, 64 sink + 512 recent: 2039 factor pages + 9 dense pages per KV head
+    gpu, _, _ = _pair(n_layers=1, n_kv_heads=8, n_q_heads=64, rank=24, sink_tokens=64, recent_tokens=512,
+                      max_seqs=1, max_pages_per_seq=2048, n_dense_slots=2048, n_factor_slots=2048)
+    gpu.append_kv(0, [0], [131072])
+    assert gpu.compress_eligible_pages() == 2039
+    gpu.decode_attention(0, [0])
+    st = gpu.stats()
+    assert st["last_decode_bytes"] == _decode_bytes(131072, 64, 64, 512, 24, 8, 64) == 303054848
+    assert st["last_decode_units"] == 8 * (2039 + 9 * 2)
+
+
+@pytest.mark.parametrize("lengths,rank", [([1024], 16), ([32768] * 8, 24), ([2048, 65536, 3001, 40000, 2049, 9999], 8),
+                                          ([70, 64, 1, 129], 32)])
+def test_decode_plan_covers_every_unit_once_and_is_balanced(lengths, rank):
+    H, n = 8, len(lengths)
+    gpu, _, _ = _pair(n_layers=1, n_kv_heads=H, n_q_heads=32, rank=rank, sink_tokens=64, recent_tokens=256,
+                      max_seqs=n, max_pages_per_seq=1024, n_dense_slots=4096, n_factor_slots=4096)
+    gpu.append_kv(0, list(range(n)), lengths)
+    gpu.compress_eligible_pages()
+    order = list(range(n))[::-1]                                      # batch order != sequence id order
+    gpu.decode_attention(0, order)
+    st = gpu.stats()
+    assert st["last_decode_bytes"] == sum(_decode_bytes(lengths[s], 64, 64, 256, rank, H, 0) for s in order) + 2 * n * 32 * 256
+    starts, segs = pkv.pkv_get_decode_plan(gpu.handle, 0, 148, n, H)
+    nb = 2 if rank >= 24 else 4                                        # dense blocks per page
+    blob, blk = 2 * (64 * rank + rank * 128) * 2, (64 // nb) * 512
+
+    def units(s):
+        kinds = gpu.page_table(s, 0)[0]
+        return [("f", blob) if k == 1 else ("d", blk) for k in kinds for _ in range(1 if k == 1 else nb)]
+
+    per_head = [units(s) for s in order]
+    flat = [(i, h, u) for i in range(n) for h in range(H) for u in range(len(per_head[i]))]
+    assert len(flat) == st["last_decode_units"]
+    assert starts[0] == (0, 0, 0) and starts[-1] == (n, 0, 0)
+    idx = {pos: j for j, pos in enumerate(flat)}
+    idx[(n, 0, 0)] = len(flat)
+    cuts = [idx[s] for s in starts]
+    assert all(b > a for a, b in zip(cuts, cuts[1:])), "ranges must be non-empty and ordered"
+    assert len(cuts) - 1 <= 148
+    # balance (the split weighs a unit by its bytes plus a fixed 2 KiB of per-unit overhead):
+    # no CTA exceeds the mean by more than two units
+    cost = [per_head[i][u][1] + 2048 for (i, h, u) in flat]
+    loads = [sum(cost[a:b]) for a, b in zip(cuts, cuts[1:])]
+    if len(flat) >= 148:
+        assert max(loads) <= sum(cost) / 148 + 2 * (max(blob, blk) + 2048)
+    # segment bookkeeping: CTAs that touch segment s are exactly [first, first + n_parts)
+    for s in range(n * H):
+        touching = [j for j, (a, b) in enumerate(zip(cuts, cuts[1:]))
+                    if any(flat[x][0] * H + flat[x][1] == s for x in (a, b - 1)) or
+                    (flat[a][0] * H + flat[a][1] < s < flat[b - 1][0] * H + flat[b - 1][1])]
+        assert segs[s] == (touching[0], len(touching)), s

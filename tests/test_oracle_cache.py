@@ -200,3 +200,34 @@ def test_free_seq_returns_slots():
     c.compress_eligible_pages()
     c.free_seq(0)
     assert c.stats()["dense_in_use"] == 0 and c.stats()["factor_in_use"] == 0
+
+
+def test_bf16_storage_rounding_matches_library_and_hand_cases():
+    import torch
+    from oracle.bf16 import round_to_bf16
+    rng = np.random.default_rng(9)
+    x = np.concatenate([rng.standard_normal(5000) * 10.0 ** rng.integers(-6, 6, 5000), [0.0, -0.0, 1.0, 65504.0]])
+    ref = torch.tensor(x, dtype=torch.float64).to(torch.float32).to(torch.bfloat16).to(torch.float64).numpy()
+    assert (round_to_bf16(x) == ref).all()
+    # 1 + 2^-8 is a tie between 1 and 1 + 2^-7: ties go to the even mantissa (1.0);
+    # 1 + 3*2^-8 ties between 1+2^-7 (odd) and 1+2^-6 (even)
+    assert round_to_bf16(np.array([1 + 2.0 ** -8]))[0] == 1.0
+    assert round_to_bf16(np.array([1 + 3 * 2.0 ** -8]))[0] == 1 + 2.0 ** -6
+    assert round_to_bf16(np.array([1 + 2.0 ** -8 + 2.0 ** -20]))[0] == 1 + 2.0 ** -7
+
+
+def test_storage_rounding_keeps_tables_and_perturbs_factors_by_bf16_epsilon():
+    cfg = _cfg(n_kv_heads=1, n_q_heads=1)
+    rng = np.random.default_rng(10)
+    c = OracleCache(cfg)
+    k, v = _kv(rng, 64, cfg)
+    c.append_kv(0, [0], [64], k, v)
+    c.compress_eligible_pages()
+    before = {s: {n: a.copy() for n, a in f.items()} for s, f in c.factor.items()}
+    table = c.page_table(0, 0)
+    c.round_factors_to_storage_type()
+    assert c.page_table(0, 0) == table
+    for s, f in c.factor.items():
+        for n, a in f.items():
+            rel = np.abs(a - before[s][n]) / np.maximum(np.abs(before[s][n]), 1e-300)
+            assert rel.max() <= 2.0 ** -8 and rel.max() > 0
