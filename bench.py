@@ -1,0 +1,323 @@
+#!/usr/bin/env python
+"""Benchmark of the PuzzleKV decode hot path on B200.
+
+One "step" = one full decode step of the workload: pkv_decode_attention for
+every layer (mixed dense/factor attention over the whole context).  Inputs are
+seeded synthetic caches (19 GB for the default workload, far larger than L2),
+resident in HBM before the timed region.  Also reported: achieved HBM GB/s and
+roofline fraction of the decode kernel, page-SVD throughput of the prefill
+compression, the same step through host buffers (e2e), and the fp64 oracle
+timed on this machine's host cores on a bounded sample.
+
+  python bench.py [--gpus N] [--steps K] [--warmup W] [--workload NAME] [--impl reference]
+"""
+import argparse
+import json
+import math
+import os
+import statistics
+import subprocess
+import sys
+import threading
+import time
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+sys.path.insert(0, ROOT)
+
+WORKLOADS = {
+    # BASELINE config 2: Qwen3-32B-shaped long context
+    "qwen3_32b_128k": dict(n_layers=64, n_kv_heads=8, n_q_heads=64, batch=1, T=131072, rank=24,
+                           sink=64, recent=512, ragged=False, outliers=0.0),
+    # BASELINE config 1: Llama-3-8B-shaped decode layer
+    "llama3_8b_32k_b8": dict(n_layers=1, n_kv_heads=8, n_q_heads=32, batch=8, T=32768, rank=24,
+                             sink=64, recent=256, ragged=False, outliers=0.0),
+    # BASELINE config 4: ragged serving batch (rank chosen with --rank)
+    "ragged_b64": dict(n_layers=1, n_kv_heads=8, n_q_heads=32, batch=64, T=(2048, 65536), rank=24,
+                       sink=64, recent=256, ragged=True, outliers=0.02),
+    # BASELINE config 0: tiny (L2-resident; latency only)
+    "tiny": dict(n_layers=1, n_kv_heads=1, n_q_heads=4, batch=1, T=1024, rank=16, sink=64, recent=128,
+                 ragged=False, outliers=0.0),
+}
+SEED = 0
+
+
+def _peaks():
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(path):
+        with open(path) as f:
+            return float(json.load(f)["hbm_gbs"]), "measured (MEASURED_PEAKS.json hbm_gbs)"
+    return 6650.0, "fallback (6.65 TB/s)"
+
+
+class ClockSampler:
+    """Samples SM clocks and throttle reasons with nvidia-smi while the timed region runs."""
+
+    FIELDS = ("clocks.sm,clocks.max.sm,clocks_event_reasons.hw_slowdown,clocks_event_reasons.hw_thermal_slowdown,"
+              "clocks_event_reasons.sw_thermal_slowdown,clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, index):
+        self.index, self.rows, self.proc = index, [], None
+
+    def start(self):
+        try:
+            self.proc = subprocess.Popen(["nvidia-smi", "-i", str(self.index), "--query-gpu=" + self.FIELDS,
+                                          "--format=csv,noheader,nounits", "-lms", "100"],
+                                         stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
+            self.thread = threading.Thread(target=self._read, daemon=True)
+            self.thread.start()
+        except OSError:
+            self.proc = None
+
+    def _read(self):
+        for line in self.proc.stdout:
+            self.rows.append([x.strip() for x in line.split(",")])
+
+    def stop(self):
+        if self.proc is None:
+            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["nvidia-smi unavailable"]}
+        time.sleep(0.15)
+        self.proc.terminate()
+        try:
+            self.proc.wait(timeout=5)
+        except subprocess.TimeoutExpired:
+            self.proc.kill()
+        sm = [float(r[0]) for r in self.rows if len(r) >= 6 and r[0].replace(".", "").isdigit()]
+        mx = [float(r[1]) for r in self.rows if len(r) >= 6 and r[1].replace(".", "").isdigit()]
+        names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
+        reasons = sorted({names[i] for r in self.rows if len(r) >= 6 for i in range(4) if r[2 + i].startswith("Active")})
+        return {"sm_mhz": statistics.median(sm) if sm else None, "sm_max_mhz": max(mx) if mx else None,
+                "reasons": reasons, "samples": len(sm)}
+
+
+def build_workload(w, rank, device):
+    """Allocate the cache, generate each (layer, sequence) on the GPU, append and compress layer by layer."""
+    import torch
+    from paper_2608_23843_b200 import pkv, synth
+    P = 64
+    if w["ragged"]:
+        lengths = synth.loguniform_lengths(SEED, w["batch"], *w["T"])
+    else:
+        lengths = [w["T"]] * w["batch"]
+    pages = [-(-t // P) for t in lengths]
+    n_sink, n_win = w["sink"] // P, w["recent"] // P
+    n_factor = [max(0, t // P - n_win - n_sink) for t in lengths]
+    L = w["n_layers"]
+    n_factor_slots = L * sum(n_factor) + 1
+    # dense slots: what stays dense in every layer plus one layer's worth of transient pages
+    n_dense_slots = sum(pages) + L * sum(p - f for p, f in zip(pages, n_factor)) + 8
+    cfg = pkv.make_config(n_layers=L, n_kv_heads=w["n_kv_heads"], n_q_heads=w["n_q_heads"], rank=rank,
+                          sink_tokens=w["sink"], recent_tokens=w["recent"], max_seqs=w["batch"],
+                          max_pages_per_seq=max(pages), n_dense_slots=n_dense_slots, n_factor_slots=n_factor_slots)
+    cache = pkv.Cache(cfg, device, synth.slot_permutation(SEED, n_dense_slots, 0).tolist(),
+                      synth.slot_permutation(SEED, n_factor_slots, 1).tolist())
+    ids = list(range(w["batch"]))
+    svd_ms, n_svds = 0.0, 0
+    for layer in range(L):
+        for s in ids:
+            k, v = synth.make_kv(SEED, layer, s, lengths[s], w["n_kv_heads"], 128, P, device, w["outliers"])
+            cache.append_kv(layer, [s], [lengths[s]], k, v)
+            del k, v
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record()
+        n = cache.compress_eligible_pages(layer)
+        e1.record()
+        torch.cuda.synchronize()
+        svd_ms += e0.elapsed_time(e1)
+        n_svds += n * w["n_kv_heads"] * 2
+    return cfg, cache, lengths, dict(pages_per_s=(n_svds / (svd_ms * 1e-3) if svd_ms > 0 else None), n_page_svds=n_svds,
+                                     svd_ms=svd_ms)
+
+
+def oracle_sample(w, rank, steps):
+    """The fp64 oracle, as it stands, on one (layer 0, KV head 0) slice of sequence 0: page SVDs and
+    one decode call for the G query heads of that KV head.  Returns seconds per decode and pages/s."""
+    import torch
+    from oracle import svd as osvd
+    from oracle.cache import OracleCache, OracleConfig
+    from paper_2608_23843_b200 import synth
+    G = w["n_q_heads"] // w["n_kv_heads"]
+    T = synth.loguniform_lengths(SEED, w["batch"], *w["T"])[0] if w["ragged"] else w["T"]
+    k, v = synth.make_kv(SEED, 0, 0, T, w["n_kv_heads"], 128, 64, "cpu", w["outliers"])
+    k, v = k[:, :1].to(torch.float64).numpy(), v[:, :1].to(torch.float64).numpy()
+    n_pages = -(-T // 64)
+    orc = OracleCache(OracleConfig(n_layers=1, n_kv_heads=1, n_q_heads=G, head_dim=128, page_size=64, rank_k=rank,
+                                   rank_v=rank, sink_tokens=w["sink"], recent_tokens=w["recent"], max_seqs=1,
+                                   n_dense_slots=n_pages, n_factor_slots=n_pages))
+    orc.append_kv(0, [0], [T], k, v)
+    t0 = time.perf_counter()
+    n = orc.compress_eligible_pages(0)
+    t_svd = time.perf_counter() - t0
+    q = synth.make_q(SEED, 0, 0, 1, w["n_q_heads"], 128)[:, :G].to(torch.float64).numpy()
+    times = []
+    for _ in range(max(1, steps)):
+        t0 = time.perf_counter()
+        orc.decode_attention(0, [0], q)
+        times.append(time.perf_counter() - t0)
+    slices_per_step = w["n_layers"] * w["n_kv_heads"] * w["batch"]
+    return dict(decode_s=statistics.median(times), slices_per_step=slices_per_step,
+                pages_per_s=(2 * n / t_svd if t_svd > 0 else None), cores=osvd.n_threads(), T=T,
+                sample="sequence 0, layer 0, KV head 0 (1/%d of a step): %d page SVDs + %d-head decode over %d tokens; "
+                       "us/step extrapolated linearly in slices" % (slices_per_step, 2 * n, G, T))
+
+
+def run_reference(args, w, rank):
+    rank0 = int(os.environ.get("RANK", "0")) == 0
+    if not rank0:
+        return
+    o = oracle_sample(w, rank, args.steps + args.warmup)
+    us = o["decode_s"] * 1e6 * o["slices_per_step"]
+    line = {"impl": "reference", "metric": "decode_us_per_step", "value": us, "unit": "us", "n_gpus": args.gpus,
+            "steps": args.steps, "warmup": args.warmup, "ms_per_step": us / 1e3, "higher_is_better": False,
+            "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic",
+            "config": _config_dict(args, w, rank),
+            "cpu_baseline": {"value": us, "unit": "us", "cores": o["cores"], "kind": "oracle", "sample": o["sample"],
+                             "pages_per_s": o["pages_per_s"]},
+            "e2e": {"value": us, "unit": "us", "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0}}
+    print(json.dumps(line))
+
+
+def _config_dict(args, w, rank):
+    return {"workload": args.workload, "n_layers": w["n_layers"], "n_q_heads": w["n_q_heads"],
+            "n_kv_heads": w["n_kv_heads"], "head_dim": 128, "batch": w["batch"], "context": w["T"], "page_size": 64,
+            "rank": rank, "sink_tokens": w["sink"], "recent_tokens": w["recent"],
+            "l2": "inputs larger than L2 (no flush)" if args.workload != "tiny" else "L2-resident (latency only)",
+            "parallelism": "replicas x%d" % args.gpus}
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=20)
+    ap.add_argument("--warmup", type=int, default=5)
+    ap.add_argument("--workload", default="qwen3_32b_128k", choices=sorted(WORKLOADS))
+    ap.add_argument("--rank", type=int, default=0, help="override the workload's rank (8, 16, 24, 32)")
+    ap.add_argument("--impl", default="pkv", choices=["pkv", "reference"])
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    args = ap.parse_args()
+    w = WORKLOADS[args.workload]
+    rank = args.rank or w["rank"]
+    if args.impl == "reference":
+        run_reference(args, w, rank)
+        return
+
+    import torch
+    import torch.distributed as dist
+    from paper_2608_23843_b200 import pkv, synth
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    rk = int(os.environ.get("RANK", "0"))
+    local = int(os.environ.get("LOCAL_RANK", "0"))
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py needs a CUDA device; there is no CPU fallback")
+    torch.cuda.set_device(local)
+    device = torch.device("cuda", local)
+    if world > 1:
+        dist.init_process_group("nccl", device_id=device)
+    pkv.lib()                                             # fail loudly if the CUDA library is missing
+
+    cfg, cache, lengths, comp = build_workload(w, rank, device)
+    ids = list(range(w["batch"]))
+    L, Hq = w["n_layers"], w["n_q_heads"]
+    qs = [synth.make_q(SEED, layer, 0, w["batch"], Hq, 128, device) for layer in range(L)]
+    outs = [torch.empty_like(q) for q in qs]
+
+    def step():
+        for layer in range(L):
+            cache.decode_attention(layer, ids, qs[layer], outs[layer])
+
+    def barrier():
+        if world > 1:
+            dist.barrier()
+        torch.cuda.synchronize()
+
+    for _ in range(max(3, args.warmup)):
+        step()
+    bytes_per_step = 0
+    for layer in range(L):                                # algorithmic bytes, from the library's own accounting
+        cache.decode_attention(layer, ids, qs[layer], outs[layer])
+        bytes_per_step += cache.stats()["last_decode_bytes"]
+    sampler = ClockSampler(local)
+    sampler.start()
+    barrier()
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    e0.record()
+    for _ in range(args.steps):
+        step()
+    e1.record()
+    barrier()
+    clocks = sampler.stop()
+    ms = e0.elapsed_time(e1) / args.steps
+    # per-launch time of the decode kernel: every launch individually (includes its merge kernel)
+    per_launch = []
+    for _ in range(2):
+        for layer in range(L):
+            a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            a.record()
+            cache.decode_attention(layer, ids, qs[layer], outs[layer])
+            b.record()
+            per_launch.append((a, b))
+    torch.cuda.synchronize()
+    launch_ms = statistics.mean(a.elapsed_time(b) for a, b in per_launch)
+
+    # end to end: queries and results in pinned host memory, copies inside the timed region
+    q_host = [q.cpu().pin_memory() for q in qs]
+    out_host = [torch.empty_like(q).pin_memory() for q in q_host]
+    q_stage, out_stage = torch.empty_like(qs[0]), torch.empty_like(qs[0])
+
+    def step_host():
+        for layer in range(L):
+            cache.decode_attention_host(layer, ids, q_host[layer], out_host[layer], q_stage, out_stage)
+        torch.cuda.current_stream().synchronize()        # the caller reads the result on the host
+
+    for _ in range(3):
+        step_host()
+    barrier()
+    t0 = time.perf_counter()
+    h0, h1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    h0.record()
+    for _ in range(args.steps):
+        step_host()
+    h1.record()
+    barrier()
+    e2e_ms = max(h0.elapsed_time(h1), (time.perf_counter() - t0) * 1e3) / args.steps
+    st = cache.stats()
+    if st["device_timeouts"] or st["bad_slot_indices"] or (outs[0].float().isnan().any().item()):
+        raise SystemExit("decode produced timeouts or NaNs: %r" % st)
+
+    t = torch.tensor([ms, e2e_ms, launch_ms], device=device, dtype=torch.float64)
+    if world > 1:
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    ms, e2e_ms, launch_ms = [float(x) for x in t.tolist()]
+
+    if rk == 0:
+        peak, peak_src = _peaks()
+        bytes_per_launch = bytes_per_step / L
+        achieved = bytes_per_launch / (launch_ms * 1e-3) / 1e9
+        qbytes = sum(q.numel() * 2 for q in qs)
+        line = {
+            "metric": "decode_us_per_step", "value": ms * 1e3, "unit": "us", "n_gpus": world, "steps": args.steps,
+            "warmup": max(3, args.warmup), "ms_per_step": ms, "higher_is_better": False, "scaling": "weak",
+            "vs_baseline": None, "dtype": "bf16", "data": "synthetic", "config": _config_dict(args, w, rank),
+            "hbm_gbs": bytes_per_step / (ms * 1e-3) / 1e9 * world,
+            "frac_of_8tbs": bytes_per_step / (ms * 1e-3) / 8e12,
+            "algorithmic_bytes_per_step": bytes_per_step,
+            "pages_factorized_per_s": comp["pages_per_s"], "page_svds_timed": comp["n_page_svds"],
+            "roofline": {"bound": "hbm", "kernel": "decode_tc_kernel<%d> (+ merge_kernel)" % rank,
+                         "achieved": achieved, "peak": peak, "unit": "GB/s", "frac": achieved / peak,
+                         "peak_source": peak_src, "traffic": None, "launch_us": launch_ms * 1e3,
+                         "algorithmic_bytes_per_launch": bytes_per_launch},
+            "e2e": {"value": e2e_ms * 1e3, "unit": "us", "h2d_bytes_per_step": qbytes, "d2h_bytes_per_step": qbytes},
+            "gpu_launches": 2 * L * args.steps, "clocks": clocks,
+        }
+        if not args.no_cpu_baseline and world == 1:
+            o = oracle_sample(w, rank, 3)
+            line["cpu_baseline"] = {"value": o["decode_s"] * 1e6 * o["slices_per_step"], "unit": "us",
+                                    "cores": o["cores"], "kind": "oracle", "sample": o["sample"],
+                                    "pages_per_s": o["pages_per_s"]}
+        print(json.dumps(line))
+    cache.close()
+    if world > 1:
+        dist.destroy_process_group()
+
+
+if __name__ == "__main__":
+    main()

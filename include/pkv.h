@@ -94,6 +94,7 @@ typedef struct pkv_stats {
     int64_t pages_compressed;        /* logical pages (one layer, all KV heads) converted so far */
     int64_t page_svds_not_converged; /* K or V pages whose Jacobi iteration hit the sweep cap */
     int64_t device_timeouts;         /* bounded in-kernel waits that gave up (must be 0) */
+    int64_t bad_slot_indices;        /* page-table entries outside the pools met by a kernel (skipped; must be 0) */
     int64_t last_decode_bytes;       /* algorithmic HBM bytes of the most recent pkv_decode_attention call:
                                         factor blobs + valid dense rows + q + out */
     int64_t last_decode_units;       /* work units (factor pages + dense blocks) of that call */

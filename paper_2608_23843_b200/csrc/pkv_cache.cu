@@ -143,6 +143,7 @@ void derive(const pkv_config &cfg, int n_ctas, Geometry &g, MetaLayout &ml, Work
     g.group = cfg.n_q_heads / cfg.n_kv_heads;
     g.rank_k = cfg.rank_k; g.rank_v = cfg.rank_v;
     g.max_seqs = cfg.max_seqs; g.max_pages = cfg.max_pages_per_seq;
+    g.n_dense_slots = (int)cfg.n_dense_slots; g.n_factor_slots = (int)cfg.n_factor_slots;
     g.sink_pages = cfg.sink_tokens / P; g.recent_pages = cfg.recent_tokens / P;
     g.ak_off = 0;
     g.bk_off = g.ak_off + P * cfg.rank_k * 2;
@@ -513,7 +514,8 @@ pkv_status pkv_append_kv(pkv_cache *c, int32_t layer, int32_t n_seqs, const int3
     if ((r = upload(c, ddesc, desc.data(), sizeof(AppendDesc) * desc.size(), st)) != PKV_OK) return r;
     if ((r = stager_flush(c, st)) != PKV_OK) return r;
     PKV_CUDA(c, launch_append(c->geo, c->dense_pool, (const int *)(c->meta + c->ml.page_table),
-                              (int *)(c->meta + c->ml.n_tokens), ddesc, (int)desc.size(), n_tok, layer, k, v, st));
+                              (int *)(c->meta + c->ml.n_tokens), ddesc, (int)desc.size(), n_tok, layer, k, v,
+                              (int *)(c->meta + c->ml.status), st));
     return PKV_OK;
 }
 
@@ -695,6 +697,7 @@ pkv_status pkv_get_stats(pkv_cache *c, pkv_stats *out, void *stream) {
         PKV_CUDA(c, cudaMemcpy(st, c->meta + c->ml.status, sizeof st, cudaMemcpyDeviceToHost));
         out->device_timeouts = st[0];
         out->page_svds_not_converged = st[1];
+        out->bad_slot_indices = st[2];
     }
     return PKV_OK;
 }

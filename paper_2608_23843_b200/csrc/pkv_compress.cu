@@ -47,6 +47,10 @@ compress_kernel(Geometry geo, const unsigned char *dense_pool, unsigned char *fa
     const int head = (blockIdx.x >> 1) % geo.n_kv_heads;
     const int entry = (blockIdx.x >> 1) / geo.n_kv_heads;
     const int2 wk = worklist[entry];
+    if (wk.x < 0 || wk.x >= geo.n_dense_slots || wk.y < 0 || wk.y >= geo.n_factor_slots) {
+        if (tid == 0) atomicAdd(&status[2], 1);       // corrupt work list: skip the page, leave a mark
+        return;
+    }
     const int rank = kv ? geo.rank_v : geo.rank_k;
     const unsigned char *src = dense_pool + (long long)wk.x * geo.dense_slot_bytes +
                                (long long)head * geo.dense_head_bytes + kv * (kPage * kRowBytes);

@@ -258,6 +258,16 @@ __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity) {
     }
     return true;
 }
+// Bounded spin until the producer has armed unit k.
+__device__ __forceinline__ bool wait_issued(volatile int *issued, int k) {
+    if (*issued > k) return true;
+    const long long t0 = clock64();
+    while (*issued <= k) {
+        if (clock64() - t0 > 2000000000LL) return false;
+        __nanosleep(20);
+    }
+    return true;
+}
 __device__ __forceinline__ void bulk_g2s(uint32_t dst, const void *src, uint32_t bytes, uint32_t bar) {
     asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];"
                  ::"r"(dst), "l"(src), "r"(bytes), "r"(bar) : "memory");
@@ -553,11 +563,16 @@ __global__ void __launch_bounds__(kDecodeThreads, 1) decode_tc_kernel(const __gr
     unsigned long long *empty_bar = full_bar + S;
     StageDesc *descs = reinterpret_cast<StageDesc *>(empty_bar + S);
     volatile int *abort_flag = reinterpret_cast<volatile int *>(descs + S);
+    // Units armed so far.  A parity wait cannot tell phase n from phase n-2, and bulk copies may land out of
+    // order, so a consumer first makes sure that its unit has been armed (which the producer does only after
+    // the stage's previous occupant was consumed) and only then waits on the stage's barrier.
+    volatile int *issued = abort_flag + 1;
 
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
     if (tid == 0) {
         for (int s = 0; s < S; ++s) { mbar_init(smem_u32(full_bar + s), 1); mbar_init(smem_u32(empty_bar + s), 1); }
         *abort_flag = 0;
+        *issued = 0;
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     }
     __syncthreads();
@@ -583,7 +598,11 @@ __global__ void __launch_bounds__(kDecodeThreads, 1) decode_tc_kernel(const __gr
                     int page, blk;
                     unit_to_page(geo, hu, u, page, blk, kind);
                     const int slot = pt[page];
-                    if (kind == kKindFactor) {
+                    if (slot < 0 || slot >= (kind == kKindFactor ? geo.n_factor_slots : geo.n_dense_slots)) {
+                        atomicAdd(a.status + 2, 1);          // corrupt page table: skip the unit, leave a mark
+                        kind = kKindDense;
+                        rows = 0;
+                    } else if (kind == kKindFactor) {
                         rows = kPage;
                         src = a.factor_pool + (long long)slot * geo.factor_slot_bytes + (long long)cur.head * geo.blob_bytes;
                     } else {
@@ -615,6 +634,8 @@ __global__ void __launch_bounds__(kDecodeThreads, 1) decode_tc_kernel(const __gr
                             } else {
                                 mbar_arrive(bar);
                             }
+                            __threadfence_block();
+                            *issued = k + 1;
                         }
                     }
                     ok = __shfl_sync(0xffffffffu, (int)ok, 0) != 0;
@@ -634,6 +655,8 @@ __global__ void __launch_bounds__(kDecodeThreads, 1) decode_tc_kernel(const __gr
                 if (ok) {
                     descs[s] = StageDesc{kKindEnd, 0, rg.n_local_segs, 0};
                     mbar_arrive(smem_u32(full_bar + s));
+                    __threadfence_block();
+                    *issued = k + 1;
                 }
             }
             ok = __shfl_sync(0xffffffffu, (int)ok, 0) != 0;
@@ -657,7 +680,7 @@ __global__ void __launch_bounds__(kDecodeThreads, 1) decode_tc_kernel(const __gr
         bool ok = true;
         for (int k = warp;; k += kConsumerWarps) {
             const int s = k % S;
-            if (ok && (*abort_flag || !mbar_wait(smem_u32(full_bar + s), (k / S) & 1))) {
+            if (ok && (*abort_flag || !wait_issued(issued, k) || !mbar_wait(smem_u32(full_bar + s), (k / S) & 1))) {
                 ok = false;
                 if (lane == 0) { *abort_flag = 1; atomicAdd(a.status, 1); }
             }
@@ -669,6 +692,7 @@ __global__ void __launch_bounds__(kDecodeThreads, 1) decode_tc_kernel(const __gr
                 if (cur_seg < rg.n_local_segs) load_q(a, rg.seg_first + cur_seg, qf, lane);
             }
             if (dsc.kind == kKindEnd) break;
+            dsc.rows = min(dsc.rows, dsc.kind == kKindFactor ? kPage : C::kDB);
             if (dsc.rows > 0) {
                 const uint32_t sb = smem_u32(stages + (size_t)s * C::kStage);
                 if (dsc.kind == kKindFactor) {

@@ -15,7 +15,7 @@ constexpr int kMaxGroup = 8;           // query heads per KV head handled by the
 constexpr int kConsumerWarps = 8;      // decode kernel: warps that compute
 constexpr int kDecodeThreads = (kConsumerWarps + 1) * 32;
 constexpr int kPartialFloats = kMaxGroup * (kHeadDim + 2);   // o[8][128], m[8], l[8]
-constexpr int kStatusWords = 8;        // [0] device timeouts, [1] page SVDs not converged
+constexpr int kStatusWords = 8;        // [0] device timeouts, [1] page SVDs not converged, [2] slot indices out of range
 constexpr int kCompressChunk = 8192;   // work-list entries per compression launch
 constexpr int kSmemBudget = 227 * 1024;
 
@@ -24,6 +24,7 @@ struct Geometry {
     int n_layers, n_kv_heads, n_q_heads, group;   // group = H_q / H_kv
     int rank_k, rank_v;
     int max_seqs, max_pages;
+    int n_dense_slots, n_factor_slots;
     int sink_pages, recent_pages;
     // factor blob of one (slot, KV head): [A_k P x r_k][B_k r_k x d][A_v P x r_v][B_v r_v x d], bf16
     int ak_off, bk_off, av_off, bv_off, blob_bytes;
@@ -83,7 +84,7 @@ struct DecodeArgs {
 // Launchers (defined in the .cu files); all return the launch error.
 cudaError_t launch_append(const Geometry &geo, unsigned char *dense_pool, const int *page_table,
                           int *n_tokens, const AppendDesc *desc, int n_seqs, long long n_tok, int layer,
-                          const void *k, const void *v, cudaStream_t st);
+                          const void *k, const void *v, int *status, cudaStream_t st);
 cudaError_t launch_compress(const Geometry &geo, const unsigned char *dense_pool, unsigned char *factor_pool,
                             const int2 *worklist, int n_entries, int *status, cudaStream_t st);
 cudaError_t launch_decode(const DecodeArgs &a, int n_segs, cudaStream_t st);

@@ -10,7 +10,7 @@ namespace {
 // swizzled dense page.  Block 0 also publishes the new token counts.
 __global__ void append_kernel(Geometry geo, unsigned char *dense_pool, const int *page_table, int *n_tokens,
                               const AppendDesc *desc, int n_seqs, long long n_tok, int layer,
-                              const uint4 *k, const uint4 *v) {
+                              const uint4 *k, const uint4 *v, int *status) {
     const int H = geo.n_kv_heads;
     const long long total = n_tok * H * 2 * 16;
     for (long long idx = blockIdx.x * (long long)blockDim.x + threadIdx.x; idx < total;
@@ -31,6 +31,10 @@ __global__ void append_kernel(Geometry geo, unsigned char *dense_pool, const int
         const int t = e.t_start + (int)(tok - e.tok_begin);
         const int page = t / kPage, row = t % kPage;
         const int slot = page_table[((long long)e.seq * geo.n_layers + layer) * geo.max_pages + page];
+        if (slot < 0 || slot >= geo.n_dense_slots || page >= geo.max_pages) {
+            if (chunk == 0 && kv == 0 && h == 0) atomicAdd(status + 2, 1);   // corrupt page table: skip the row
+            continue;
+        }
         const uint4 val = (kv ? v : k)[(tok * H + h) * 16 + chunk];
         unsigned char *dst = dense_pool + (long long)slot * geo.dense_slot_bytes + (long long)h * geo.dense_head_bytes +
                              kv * (kPage * kRowBytes) + row * kRowBytes + swz_chunk(row, chunk) * 16;
@@ -87,14 +91,14 @@ __global__ void dense_read_kernel(const unsigned char *head_base, unsigned short
 
 cudaError_t launch_append(const Geometry &geo, unsigned char *dense_pool, const int *page_table,
                           int *n_tokens, const AppendDesc *desc, int n_seqs, long long n_tok, int layer,
-                          const void *k, const void *v, cudaStream_t st) {
+                          const void *k, const void *v, int *status, cudaStream_t st) {
     const long long total = n_tok * geo.n_kv_heads * 2 * 16;
     const int threads = 256;
     long long blocks = (total + threads - 1) / threads;
     if (blocks > 148LL * 16) blocks = 148LL * 16;
     if (blocks < 1) blocks = 1;
     append_kernel<<<(unsigned)blocks, threads, 0, st>>>(geo, dense_pool, page_table, n_tokens, desc, n_seqs, n_tok,
-                                                        layer, (const uint4 *)k, (const uint4 *)v);
+                                                        layer, (const uint4 *)k, (const uint4 *)v, status);
     return cudaGetLastError();
 }
 

@@ -51,7 +51,7 @@ class PkvSizes(ctypes.Structure):
 
 class PkvStats(ctypes.Structure):
     _fields_ = [(n, ctypes.c_int64) for n in ("dense_slots_in_use", "factor_slots_in_use", "pages_compressed",
-                                              "page_svds_not_converged", "device_timeouts",
+                                              "page_svds_not_converged", "device_timeouts", "bad_slot_indices",
                                               "last_decode_bytes", "last_decode_units")]
 
 
