@@ -74,9 +74,16 @@ typedef struct pkv_config {
     float   softmax_scale;      /* 0 => 1/sqrt(head_dim)  (Eq. 1) */
     int32_t jacobi_max_sweeps;  /* 0 => default (16) */
     float   jacobi_tol;         /* 0 => default; rotation skipped when |g_pq| <= tol*sqrt(g_pp*g_qq) */
-    int32_t n_ctas;             /* decode grid size; 0 => one CTA per SM of the current device (148 in dry-run) */
+    int32_t n_ctas;             /* decode grid size; 0 => SM count of the current device (148 in dry-run), doubled unless decode_overlap */
     int32_t decode_variant;     /* 0 = tensor-core pipeline kernel (the product path); 1 = scalar fp32 kernel that
                                    evaluates the same equations one unit at a time, kept as a debugging reference */
+    int32_t decode_overlap;     /* pkv_decode_attention is launched with programmatic stream serialization, so its
+                                   CTAs start as SMs free up.  0 (default): the kernel still waits for the preceding
+                                   kernel on the stream to finish before it reads the cache or q.  1: the caller
+                                   promises that the kernel enqueued just before each pkv_decode_attention call
+                                   writes neither this cache's pools nor q (typical: the previous layer's decode
+                                   with queries prepared in advance); the kernel then streams pages at once and
+                                   waits only before touching its shared workspace and `out`. */
 } pkv_config;
 
 typedef struct pkv_sizes {

@@ -120,7 +120,8 @@ pkv_status validate(const pkv_config *cfg, const char **why) {
         *why = "sink_tokens and recent_tokens must be non-negative multiples of page_size"; return PKV_ERR_INVALID_ARG;
     }
     if (cfg->softmax_scale < 0.f || cfg->jacobi_max_sweeps < 0 || cfg->jacobi_tol < 0.f || cfg->n_ctas < 0 ||
-        cfg->decode_variant < 0 || cfg->decode_variant > 1) {
+        cfg->decode_variant < 0 || cfg->decode_variant > 1 ||
+        cfg->decode_overlap < 0 || cfg->decode_overlap > 1) {
         *why = "negative scale / sweep cap / tolerance / n_ctas, or unknown decode_variant"; return PKV_ERR_INVALID_ARG;
     }
     if (cfg->n_dense_slots > INT32_MAX || cfg->n_factor_slots > INT32_MAX) {
@@ -156,8 +157,10 @@ void derive(const pkv_config &cfg, int n_ctas, Geometry &g, MetaLayout &ml, Work
     g.stage_bytes = std::max(g.blob_bytes, 8192);
     g.block_tokens = g.stage_bytes >= 16384 ? 32 : 16;
     g.blocks_per_page = P / g.block_tokens;
-    const int fixed = kConsumerWarps * kPartialFloats * 4 + 2048;
-    g.n_stages = std::min(24, (kSmemBudget - fixed) / g.stage_bytes);
+    // two CTAs are resident per SM (consecutive launches overlap, or the grid holds two CTAs per SM),
+    // so that one streams while the other is in its prologue or merging
+    const int fixed = kConsumerWarps * kPartialFloats * 4 + 1024 + 1024;
+    g.n_stages = std::min(16, (kSmemBudget / 2 - fixed) / g.stage_bytes);
     g.n_ctas = n_ctas;
     const float scale = cfg.softmax_scale > 0.f ? cfg.softmax_scale : 1.0f / std::sqrt((float)d);
     g.scale_log2e = scale * 1.4426950408889634f;
@@ -181,6 +184,7 @@ void derive(const pkv_config &cfg, int n_ctas, Geometry &g, MetaLayout &ml, Work
     long long w = 0;
     wl.partials = w; w = align_up(w + wl.n_partials * kPartialFloats * 4, 256);
     wl.worklist = w; w = align_up(w + (long long)sizeof(int2) * kCompressChunk, 256);
+    wl.tickets = w;  w = align_up(w + 4LL * cfg.max_seqs * cfg.n_kv_heads, 256);
     wl.total = w;
 }
 
@@ -385,8 +389,8 @@ pkv_status pkv_query_sizes(const pkv_config *cfg, pkv_sizes *out) {
     if (r != PKV_OK) return r;
     if (!out) return PKV_ERR_INVALID_ARG;
     Geometry g; MetaLayout ml; WorkspaceLayout wl;
-    // meta / workspace sizes depend on the grid size; use the larger of the request and 256 CTAs
-    int n_ctas = cfg->n_ctas > 0 ? cfg->n_ctas : 256;
+    // meta / workspace sizes depend on the grid size; the default grid never exceeds 512 CTAs
+    int n_ctas = cfg->n_ctas > 0 ? cfg->n_ctas : 512;
     derive(*cfg, n_ctas, g, ml, wl);
     out->dense_slot_bytes = g.dense_slot_bytes;
     out->factor_slot_bytes = g.factor_slot_bytes;
@@ -413,8 +417,10 @@ pkv_status pkv_init_cache(const pkv_config *cfg, void *dense_pool, void *factor_
     if (!c) return PKV_ERR_INVALID_ARG;
     c->cfg = *cfg;
     c->dry = dry;
-    int n_ctas = cfg->n_ctas > 0 ? cfg->n_ctas : default_ctas(dry);
-    if (cfg->n_ctas == 0 && n_ctas > 256) n_ctas = 256;      // pkv_query_sizes() sized the buffers for <= 256
+    // default grid: one CTA per SM when consecutive launches overlap (two launches share each SM),
+    // otherwise two CTAs per SM
+    int n_ctas = cfg->n_ctas > 0 ? cfg->n_ctas : default_ctas(dry) * (cfg->decode_overlap ? 1 : 2);
+    if (cfg->n_ctas == 0 && n_ctas > 512) n_ctas = 512;      // pkv_query_sizes() sized the buffers for <= 512
     derive(*cfg, n_ctas, c->geo, c->ml, c->wl);
     c->dense_pool = (unsigned char *)dense_pool; c->factor_pool = (unsigned char *)factor_pool;
     c->meta = (unsigned char *)meta; c->workspace = (unsigned char *)workspace;
@@ -629,9 +635,11 @@ pkv_status pkv_decode_attention(pkv_cache *c, int32_t layer, int32_t n_seqs, con
     a.plan_cta = c->ml.plan_cta; a.plan_entry = c->ml.plan_entry; a.plan_seg = c->ml.plan_seg;
     a.q = q; a.out = out; a.out_f32 = out_f32;
     a.partials = (float *)(c->workspace + c->wl.partials);
+    a.tickets = (int *)(c->workspace + c->wl.tickets);
     a.status = (int *)(c->meta + c->ml.status);
     a.layer = layer;
     a.variant = c->cfg.decode_variant;
+    a.overlap = c->cfg.decode_overlap;
     PKV_CUDA(c, launch_decode(a, pc.n_segs, st));
     return PKV_OK;
 }

@@ -11,9 +11,11 @@
 //     w  = A_v^T p,  o += B_v^T w
 // for all query heads that share the KV head, keeping (m, l, o) in registers.
 // K^ and V^ are never formed.  At the end of each (sequence, KV head) segment the
-// warps combine their states and the CTA writes one partial state; a small merge
-// kernel applies Eq. 5 across CTAs.  A scalar fp32 kernel with the same plan and
-// partial format exists as a debugging reference (decode_variant = 1).
+// warps combine their states; a segment split over several CTAs leaves one
+// partial state per CTA and the CTA that finishes last applies Eq. 5 across them
+// (ticket counter, no waiting).  A scalar fp32 kernel with the same plan and
+// partial format, followed by a separate merge kernel, exists as a debugging
+// reference (decode_variant = 1).
 #include <cuda_bf16.h>
 
 #include "pkv_internal.h"
@@ -499,63 +501,122 @@ __device__ __forceinline__ void load_q(const DecodeArgs &a, int seg, uint32_t (&
     }
 }
 
-// All consumer warps combine their states of one segment; the CTA writes one partial.
-__device__ __forceinline__ void flush_segment(const DecodeArgs &a, float *comb, WarpState &st, int seg, int warp, int lane,
-                                              int ctid) {
+// Writes the final result of one (entry, KV head) for query head hq, dims d4..d4+3.
+__device__ __forceinline__ void store_out(const DecodeArgs &a, int seg, int hq, int d4, float4 acc, float L) {
+    const Geometry &g = a.geo;
+    const int entry = seg / g.n_kv_heads, head = seg % g.n_kv_heads;
+    const float inv = 1.f / L;
+    acc.x *= inv; acc.y *= inv; acc.z *= inv; acc.w *= inv;
+    const long long off = ((long long)entry * g.n_q_heads + head * g.group + hq) * kHeadDim + d4;
+    __nv_bfloat162 lo = __floats2bfloat162_rn(acc.x, acc.y), hi = __floats2bfloat162_rn(acc.z, acc.w);
+    uint2 packed;
+    packed.x = *reinterpret_cast<unsigned *>(&lo);
+    packed.y = *reinterpret_cast<unsigned *>(&hi);
+    *reinterpret_cast<uint2 *>(reinterpret_cast<__nv_bfloat16 *>(a.out) + off) = packed;
+    if (a.out_f32) *reinterpret_cast<float4 *>(a.out_f32 + off) = acc;
+}
+
+#define PKV_CONSUMER_BARRIER() asm volatile("bar.sync 1, %0;" ::"n"(kConsumerWarps * 32) : "memory")
+
+// All consumer warps combine their states of one segment (Eq. 5 inside the CTA).  If the segment
+// lies wholly in this CTA the result is final; otherwise the CTA writes one partial state, takes a
+// ticket, and the CTA that draws the last ticket of the segment applies Eq. 5 across CTAs.  Partials
+// are always summed in CTA order, so the result does not depend on which CTA arrives last.
+__device__ __forceinline__ void flush_segment(const DecodeArgs &a, float *comb, volatile int *last_flag, WarpState &st,
+                                              int seg, int warp, int lane, int ctid, int n_active) {
+    constexpr int kThreads = kConsumerWarps * 32, kItems = kMaxGroup * 32;   // item = (query head, 4 dims)
     const int g = lane >> 2, t = lane & 3;
-    float l0 = st.l[0], l1 = st.l[1];
+    if (warp < n_active) {
+        float l0 = st.l[0], l1 = st.l[1];
 #pragma unroll
-    for (int off = 4; off <= 16; off <<= 1) {
-        l0 += __shfl_xor_sync(0xffffffffu, l0, off);
-        l1 += __shfl_xor_sync(0xffffffffu, l1, off);
-    }
-    float *mine = comb + warp * kPartialFloats;
+        for (int off = 4; off <= 16; off <<= 1) {
+            l0 += __shfl_xor_sync(0xffffffffu, l0, off);
+            l1 += __shfl_xor_sync(0xffffffffu, l1, off);
+        }
+        float *mine = comb + warp * kPartialFloats;
 #pragma unroll
-    for (int i = 0; i < 8; ++i) {
-        mine[(2 * t) * kHeadDim + 16 * i + g] = st.o[i][0];
-        mine[(2 * t + 1) * kHeadDim + 16 * i + g] = st.o[i][1];
-        mine[(2 * t) * kHeadDim + 16 * i + 8 + g] = st.o[i][2];
-        mine[(2 * t + 1) * kHeadDim + 16 * i + 8 + g] = st.o[i][3];
+        for (int i = 0; i < 8; ++i) {
+            mine[(2 * t) * kHeadDim + 16 * i + g] = st.o[i][0];
+            mine[(2 * t + 1) * kHeadDim + 16 * i + g] = st.o[i][1];
+            mine[(2 * t) * kHeadDim + 16 * i + 8 + g] = st.o[i][2];
+            mine[(2 * t + 1) * kHeadDim + 16 * i + 8 + g] = st.o[i][3];
+        }
+        if (g == 0) {
+            mine[kMaxGroup * kHeadDim + 2 * t] = st.m[0];
+            mine[kMaxGroup * kHeadDim + 2 * t + 1] = st.m[1];
+            mine[kMaxGroup * kHeadDim + kMaxGroup + 2 * t] = l0;
+            mine[kMaxGroup * kHeadDim + kMaxGroup + 2 * t + 1] = l1;
+        }
     }
-    if (g == 0) {
-        mine[kMaxGroup * kHeadDim + 2 * t] = st.m[0];
-        mine[kMaxGroup * kHeadDim + 2 * t + 1] = st.m[1];
-        mine[kMaxGroup * kHeadDim + kMaxGroup + 2 * t] = l0;
-        mine[kMaxGroup * kHeadDim + kMaxGroup + 2 * t + 1] = l1;
-    }
-    asm volatile("bar.sync 1, %0;" ::"n"(kConsumerWarps * 32) : "memory");
-    {
-        const int hq = ctid >> 5, d4 = (ctid & 31) * 4;
+    PKV_CONSUMER_BARRIER();
+    // partial states, tickets and (for a caller that reuses it) `out` may still be in use by the preceding launch
+    asm volatile("griddepcontrol.wait;" ::: "memory");
+    const PlanSeg ps = reinterpret_cast<const PlanSeg *>(a.plan + a.plan_seg)[seg];
+    float *part = a.partials + ((long long)blockIdx.x + seg) * kPartialFloats;
+    for (int item = ctid; item < kItems; item += kThreads) {
+        const int hq = item >> 5, d4 = (item & 31) * 4;
         float M = kNegInf;
-#pragma unroll
-        for (int w = 0; w < kConsumerWarps; ++w) M = fmaxf(M, comb[w * kPartialFloats + kMaxGroup * kHeadDim + hq]);
+        for (int w = 0; w < n_active; ++w) M = fmaxf(M, comb[w * kPartialFloats + kMaxGroup * kHeadDim + hq]);
         float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
         float L = 0.f;
-#pragma unroll
-        for (int w = 0; w < kConsumerWarps; ++w) {
+        for (int w = 0; w < n_active; ++w) {
             const float *cw = comb + w * kPartialFloats;
             const float f = exp2f(cw[kMaxGroup * kHeadDim + hq] - M);
             const float4 o = *reinterpret_cast<const float4 *>(cw + hq * kHeadDim + d4);
             acc.x += f * o.x; acc.y += f * o.y; acc.z += f * o.z; acc.w += f * o.w;
             L += f * cw[kMaxGroup * kHeadDim + kMaxGroup + hq];
         }
-        float *part = a.partials + ((long long)blockIdx.x + seg) * kPartialFloats;
-        *reinterpret_cast<float4 *>(part + hq * kHeadDim + d4) = acc;
-        if ((ctid & 31) == 0) {
-            part[kMaxGroup * kHeadDim + hq] = M;
-            part[kMaxGroup * kHeadDim + kMaxGroup + hq] = L;
+        if (ps.n_parts <= 1) {
+            if (hq < a.geo.group) store_out(a, seg, hq, d4, acc, L);
+        } else {
+            *reinterpret_cast<float4 *>(part + hq * kHeadDim + d4) = acc;
+            if ((item & 31) == 0) {
+                part[kMaxGroup * kHeadDim + hq] = M;
+                part[kMaxGroup * kHeadDim + kMaxGroup + hq] = L;
+            }
         }
     }
-    asm volatile("bar.sync 1, %0;" ::"n"(kConsumerWarps * 32) : "memory");
+    if (ps.n_parts > 1) {
+        __threadfence();
+        PKV_CONSUMER_BARRIER();
+        if (ctid == 0) *last_flag = (atomicAdd(a.tickets + seg, 1) == ps.n_parts - 1);
+        PKV_CONSUMER_BARRIER();
+        if (*last_flag) {
+            __threadfence();
+            const float *first = a.partials + ((long long)ps.cta_first + seg) * kPartialFloats;
+            for (int item = ctid; item < a.geo.group * 32; item += kThreads) {
+                const int hq = item >> 5, d4 = (item & 31) * 4;
+                float Mg = kNegInf;
+                for (int k = 0; k < ps.n_parts; ++k)
+                    Mg = fmaxf(Mg, __ldcg(first + (long long)k * kPartialFloats + kMaxGroup * kHeadDim + hq));
+                float4 tot = make_float4(0.f, 0.f, 0.f, 0.f);
+                float Lg = 0.f;
+#pragma unroll 4
+                for (int k = 0; k < ps.n_parts; ++k) {
+                    const float *pk = first + (long long)k * kPartialFloats;
+                    const float f = exp2f(__ldcg(pk + kMaxGroup * kHeadDim + hq) - Mg);
+                    const float4 o = __ldcg(reinterpret_cast<const float4 *>(pk + hq * kHeadDim + d4));
+                    tot.x += f * o.x; tot.y += f * o.y; tot.z += f * o.z; tot.w += f * o.w;
+                    Lg += f * __ldcg(pk + kMaxGroup * kHeadDim + kMaxGroup + hq);
+                }
+                store_out(a, seg, hq, d4, tot, Lg);
+            }
+            if (ctid == 0) a.tickets[seg] = 0;          // ready for the next launch
+        }
+    }
+    PKV_CONSUMER_BARRIER();
 }
 
 template <int R>
-__global__ void __launch_bounds__(kDecodeThreads, 1) decode_tc_kernel(const __grid_constant__ DecodeArgs a) {
+__global__ void __launch_bounds__(kDecodeThreads, 2) decode_tc_kernel(const __grid_constant__ DecodeArgs a) {
     using C = Tc<R>;
     Range rg;
     if (!load_range(a, rg)) return;
     const Geometry &geo = a.geo;
     const int S = geo.n_stages;
+    // A warp that has reached the next segment keeps its stage until every warp has; so no more warps may
+    // take units than there are stages.  The others only take part in the flush barriers.
+    const int W = min(kConsumerWarps, S);
     extern __shared__ __align__(1024) unsigned char smem[];
     unsigned char *stages = smem;
     float *comb = reinterpret_cast<float *>(smem + (size_t)S * C::kStage);
@@ -567,6 +628,7 @@ __global__ void __launch_bounds__(kDecodeThreads, 1) decode_tc_kernel(const __gr
     // order, so a consumer first makes sure that its unit has been armed (which the producer does only after
     // the stage's previous occupant was consumed) and only then waits on the stage's barrier.
     volatile int *issued = abort_flag + 1;
+    volatile int *last_flag = abort_flag + 2;
 
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
     if (tid == 0) {
@@ -576,6 +638,12 @@ __global__ void __launch_bounds__(kDecodeThreads, 1) decode_tc_kernel(const __gr
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     }
     __syncthreads();
+    // Programmatic dependent launch: let the next kernel on the stream begin as SMs free up.  Unless the caller
+    // vouched that the preceding kernel writes neither this cache nor q (overlap mode), wait for it to finish
+    // before reading anything it may have produced; in overlap mode only the shared partial-state workspace
+    // needs that wait (taken in flush_segment).
+    if (!a.overlap) asm volatile("griddepcontrol.wait;" ::: "memory");
+    asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
 
     if (warp == kConsumerWarps) {
         // ------------------------------ producer ------------------------------
@@ -648,7 +716,7 @@ __global__ void __launch_bounds__(kDecodeThreads, 1) decode_tc_kernel(const __gr
             ++seg_local;
         }
         // one end marker per consumer warp
-        for (int w = 0; w < kConsumerWarps && ok; ++w, ++k) {
+        for (int w = 0; w < W && ok; ++w, ++k) {
             if (lane == 0) {
                 const int s = k % S;
                 if (k >= S && !mbar_wait(smem_u32(empty_bar + s), ((k / S) - 1) & 1)) ok = false;
@@ -674,11 +742,16 @@ __global__ void __launch_bounds__(kDecodeThreads, 1) decode_tc_kernel(const __gr
         // ------------------------------ consumers ------------------------------
         WarpState st;
         reset_state(st);
+        if (warp >= W) {
+            for (int sg = 0; sg < rg.n_local_segs; ++sg)
+                flush_segment(a, comb, last_flag, st, rg.seg_first + sg, warp, lane, tid, W);
+            return;
+        }
         uint32_t qf[8][2];
         int cur_seg = 0;
         load_q(a, rg.seg_first, qf, lane);
         bool ok = true;
-        for (int k = warp;; k += kConsumerWarps) {
+        for (int k = warp;; k += W) {
             const int s = k % S;
             if (ok && (*abort_flag || !wait_issued(issued, k) || !mbar_wait(smem_u32(full_bar + s), (k / S) & 1))) {
                 ok = false;
@@ -686,7 +759,7 @@ __global__ void __launch_bounds__(kDecodeThreads, 1) decode_tc_kernel(const __gr
             }
             StageDesc dsc = ok ? descs[s] : StageDesc{kKindEnd, 0, rg.n_local_segs, 0};
             while (cur_seg < dsc.seg) {
-                flush_segment(a, comb, st, rg.seg_first + cur_seg, warp, lane, tid);
+                flush_segment(a, comb, last_flag, st, rg.seg_first + cur_seg, warp, lane, tid, W);
                 ++cur_seg;
                 reset_state(st);
                 if (cur_seg < rg.n_local_segs) load_q(a, rg.seg_first + cur_seg, qf, lane);
@@ -713,8 +786,17 @@ cudaError_t launch_tc(const DecodeArgs &a, cudaStream_t st) {
     using C = Tc<R>;
     const size_t smem = (size_t)a.geo.n_stages * C::kStage + kConsumerWarps * kPartialFloats * 4 +
                         a.geo.n_stages * (8 + 8 + sizeof(StageDesc)) + 64;
-    decode_tc_kernel<R><<<a.geo.n_ctas, kDecodeThreads, smem, st>>>(a);
-    return cudaGetLastError();
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3(a.geo.n_ctas);
+    cfg.blockDim = dim3(kDecodeThreads);
+    cfg.dynamicSmemBytes = smem;
+    cfg.stream = st;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = 1;
+    return cudaLaunchKernelEx(&cfg, decode_tc_kernel<R>, a);
 }
 
 }  // namespace
@@ -743,7 +825,7 @@ cudaError_t launch_decode(const DecodeArgs &a, int n_segs, cudaStream_t st) {
             default: return cudaErrorInvalidValue;
         }
     }
-    if (e != cudaSuccess) return e;
+    if (e != cudaSuccess || a.variant != 1) return e;
     merge_kernel<<<n_segs, 256, 0, st>>>(a);
     return cudaGetLastError();
 }

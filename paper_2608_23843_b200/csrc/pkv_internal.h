@@ -12,7 +12,7 @@ constexpr int kHeadDim = 128;          // d (only supported value)
 constexpr int kPage = 64;              // P (only supported value)
 constexpr int kRowBytes = kHeadDim * 2;
 constexpr int kMaxGroup = 8;           // query heads per KV head handled by the tensor-core kernel
-constexpr int kConsumerWarps = 8;      // decode kernel: warps that compute
+constexpr int kConsumerWarps = 4;      // decode kernel: warps that compute (two CTAs share an SM)
 constexpr int kDecodeThreads = (kConsumerWarps + 1) * 32;
 constexpr int kPartialFloats = kMaxGroup * (kHeadDim + 2);   // o[8][128], m[8], l[8]
 constexpr int kStatusWords = 8;        // [0] device timeouts, [1] page SVDs not converged, [2] slot indices out of range
@@ -60,6 +60,7 @@ struct WorkspaceLayout {
     long long partials;                // float [n_partials][kPartialFloats]
     long long n_partials;
     long long worklist;                // int2 [kCompressChunk]
+    long long tickets;                 // int [max_seqs * n_kv_heads]
     long long total;
 };
 
@@ -76,9 +77,11 @@ struct DecodeArgs {
     void *out;
     float *out_f32;
     float *partials;
+    int *tickets;                      // one per segment, zero between launches
     int *status;
     int layer;
     int variant;                       // 0 = tensor-core pipeline, 1 = scalar reference kernel
+    int overlap;                       // 1 = may stream KV before the preceding kernel has finished
 };
 
 // Launchers (defined in the .cu files); all return the launch error.
