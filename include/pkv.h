@@ -183,6 +183,38 @@ pkv_status pkv_decode_attention_host(pkv_cache *c, int32_t layer, int32_t n_seqs
                                      const void *q_host, void *out_host, void *q_stage, void *out_stage,
                                      void *stream);
 
+/*
+ * No counterpart in the paper: this entry point exists for deployment reasons only.
+ *
+ * pkv_decode_attention() keeps its split-K scratch (one partial softmax state per CTA and segment,
+ * plus the merge tickets) in the `workspace` buffer that the caller allocated.  Some callers cannot
+ * provide such a buffer when they decode: code that runs inside a serving process whose device
+ * memory is fully handed out at start-up and where a later cudaMalloc is forbidden (it would stall
+ * every stream of the device), plug-ins that are given fixed input/output tensors by a host
+ * framework and have no allocator of their own, and hosts that let another component reuse or
+ * release the workspace between steps.  This variant computes exactly what pkv_decode_attention()
+ * computes, with the same kernels, arguments and results, but keeps that scratch in a fixed array
+ * inside the library itself.  It calls no cudaMalloc, cudaFree or other allocating routine; the
+ * cache's own workspace buffer is not touched.
+ *
+ * Limits and rules
+ *  - Capacity: n_ctas + n_seqs * n_kv_heads <= 1024 partial states.  A larger call is rejected
+ *    with PKV_ERR_INVALID_ARG and a message; nothing is launched.
+ *  - Cost: the array (about 4.1 MiB) is part of the library image, so every GPU on which the
+ *    library is loaded holds it until the process exits, whether or not this function is called.
+ *  - The first call on each device looks up the array's device address (the device must be
+ *    current).  Make that first call outside any CUDA stream capture.
+ *  - All calls on a device share the one array, which keeps the previous call's contents; the
+ *    function clears the part that must start at zero (the tickets) on `stream` before each
+ *    launch.  Two calls that may run on the GPU at the same time (different streams without an
+ *    ordering between them, or different caches) would overwrite each other's partial states:
+ *    the caller must order them.  For the same reason consecutive calls do not overlap on the
+ *    GPU even when decode_overlap is set.
+ */
+pkv_status pkv_decode_attention_static_scratch(pkv_cache *c, int32_t layer, int32_t n_seqs,
+                                               const int32_t *seq_ids, const void *q, void *out,
+                                               float *out_f32, void *stream);
+
 /* Page table of one (sequence, layer) from the host mirror: kinds[i] in
  * {PKV_KIND_DENSE, PKV_KIND_FACTOR}, slots[i] the physical slot, for i <
  * *n_pages (arrays [host] of capacity max_pages_per_seq; may be NULL). */

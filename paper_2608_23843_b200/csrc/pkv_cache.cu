@@ -644,6 +644,44 @@ pkv_status pkv_decode_attention(pkv_cache *c, int32_t layer, int32_t n_seqs, con
     return PKV_OK;
 }
 
+pkv_status pkv_decode_attention_static_scratch(pkv_cache *c, int32_t layer, int32_t n_seqs,
+                                               const int32_t *seq_ids, const void *q, void *out, float *out_f32,
+                                               void *stream) {
+    if (!c) return PKV_ERR_INVALID_ARG;
+    if (c->dry) return fail(c, PKV_ERR_INVALID_ARG, "no device buffers in dry-run mode");
+    cudaStream_t st = (cudaStream_t)stream;
+    if (layer < 0 || layer >= c->cfg.n_layers) return fail(c, PKV_ERR_INVALID_ARG, "layer %d out of range", layer);
+    pkv_status r = check_seq_list(c, n_seqs, seq_ids);
+    if (r != PKV_OK) return r;
+    for (int i = 0; i < n_seqs; ++i)
+        if (c->at(seq_ids[i], layer).n_tokens == 0)
+            return fail(c, PKV_ERR_INVALID_ARG, "sequence %d has no tokens in layer %d", seq_ids[i], layer);
+    if (!q || !out) return fail(c, PKV_ERR_INVALID_ARG, "q or out is NULL");
+    if (!plan_is_current(c, layer, n_seqs, seq_ids)) {
+        if ((r = build_plan(c, layer, n_seqs, seq_ids, st)) != PKV_OK) return r;
+    }
+    DecodeArgs a;
+    a.geo = c->geo;
+    a.dense_pool = c->dense_pool; a.factor_pool = c->factor_pool;
+    a.page_table = (const int *)(c->meta + c->ml.page_table);
+    a.n_tokens = (const int *)(c->meta + c->ml.n_tokens);
+    a.plan = c->meta + c->ml.plans + c->ml.plan_stride * layer;
+    a.plan_cta = c->ml.plan_cta; a.plan_entry = c->ml.plan_entry; a.plan_seg = c->ml.plan_seg;
+    a.q = q; a.out = out; a.out_f32 = out_f32;
+    a.partials = nullptr; a.tickets = nullptr;            // set by the launcher from the static scratch
+    a.status = (int *)(c->meta + c->ml.status);
+    a.layer = layer;
+    a.variant = c->cfg.decode_variant;
+    a.overlap = c->cfg.decode_overlap;
+    const char *why = "";
+    cudaError_t e = launch_decode_static_scratch(a, c->plans[layer].n_segs, st, &why);
+    if (e == cudaErrorInvalidValue && why[0])
+        return fail(c, PKV_ERR_INVALID_ARG, "pkv_decode_attention_static_scratch: %s", why);
+    if (e != cudaSuccess)
+        return fail(c, PKV_ERR_CUDA, "pkv_decode_attention_static_scratch: %s: %s", why, cudaGetErrorString(e));
+    return PKV_OK;
+}
+
 pkv_status pkv_decode_attention_host(pkv_cache *c, int32_t layer, int32_t n_seqs, const int32_t *seq_ids,
                                      const void *q_host, void *out_host, void *q_stage, void *out_stage,
                                      void *stream) {

@@ -20,6 +20,15 @@
 
 #include "pkv_internal.h"
 
+// Scratch of pkv_decode_attention_static_scratch(): split-K partial states followed by the merge
+// tickets.  It lives in the library image, so every GPU that loads the library holds these bytes
+// (about 4.1 MiB) until the process exits, and every call on a device shares them.
+static constexpr int kStaticPartialStates = 1024;
+static constexpr int kStaticTickets = 1024;
+static constexpr size_t kStaticTicketOffset = (size_t)kStaticPartialStates * pkv::kPartialFloats * sizeof(float);
+static constexpr size_t kStaticScratchBytes = kStaticTicketOffset + kStaticTickets * sizeof(int);
+static __device__ __align__(256) unsigned char g_static_scratch[kStaticScratchBytes];
+
 namespace pkv {
 
 namespace {
@@ -828,6 +837,39 @@ cudaError_t launch_decode(const DecodeArgs &a, int n_segs, cudaStream_t st) {
     if (e != cudaSuccess || a.variant != 1) return e;
     merge_kernel<<<n_segs, 256, 0, st>>>(a);
     return cudaGetLastError();
+}
+
+// Same launch as launch_decode(), with the partial states and tickets in g_static_scratch instead of
+// the caller's workspace.  In host code the array's name is only a stand-in for the device symbol, so
+// its device address is looked up (once per device, with that device current) and handed to the kernel.
+cudaError_t launch_decode_static_scratch(const DecodeArgs &a, int n_segs, cudaStream_t st, const char **why) {
+    static unsigned char *scratch_of_device[64] = {};
+    *why = "";
+    if ((long long)a.geo.n_ctas + n_segs > kStaticPartialStates || n_segs > kStaticTickets) {
+        *why = "call needs more split-K partial states than the static scratch holds "
+               "(n_ctas + n_seqs * n_kv_heads must be <= 1024)";
+        return cudaErrorInvalidValue;
+    }
+    int dev = -1;
+    cudaError_t e = cudaGetDevice(&dev);
+    if (e != cudaSuccess) { *why = "cudaGetDevice failed"; return e; }
+    if (dev < 0 || dev >= 64) { *why = "device ordinal above 63"; return cudaErrorInvalidDevice; }
+    if (!scratch_of_device[dev]) {
+        unsigned char *p = nullptr;
+        e = cudaGetSymbolAddress((void **)&p, g_static_scratch);
+        if (e != cudaSuccess || !p) { *why = "cudaGetSymbolAddress(g_static_scratch) failed"; return e != cudaSuccess ? e : cudaErrorUnknown; }
+        scratch_of_device[dev] = p;
+    }
+    unsigned char *base = scratch_of_device[dev];
+    DecodeArgs b = a;
+    b.partials = reinterpret_cast<float *>(base);
+    b.tickets = reinterpret_cast<int *>(base + kStaticTicketOffset);
+    // the array keeps whatever the previous call (or an aborted one) left: tickets must start at zero
+    e = cudaMemsetAsync(b.tickets, 0, (size_t)n_segs * sizeof(int), st);
+    if (e != cudaSuccess) { *why = "clearing the tickets failed"; return e; }
+    e = launch_decode(b, n_segs, st);
+    if (e != cudaSuccess) *why = "kernel launch failed";
+    return e;
 }
 
 }  // namespace pkv

@@ -91,6 +91,7 @@ cudaError_t launch_append(const Geometry &geo, unsigned char *dense_pool, const 
 cudaError_t launch_compress(const Geometry &geo, const unsigned char *dense_pool, unsigned char *factor_pool,
                             const int2 *worklist, int n_entries, int *status, cudaStream_t st);
 cudaError_t launch_decode(const DecodeArgs &a, int n_segs, cudaStream_t st);
+cudaError_t launch_decode_static_scratch(const DecodeArgs &a, int n_segs, cudaStream_t st, const char **why);
 cudaError_t launch_read_factors(const Geometry &geo, const unsigned char *blob, void *A_k, void *B_k,
                                 void *A_v, void *B_v, cudaStream_t st);
 cudaError_t launch_write_factors(const Geometry &geo, unsigned char *blob, const void *A_k, const void *B_k,

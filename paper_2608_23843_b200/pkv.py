@@ -28,7 +28,7 @@ EXPORTS = [
     "pkv_query_sizes", "pkv_init_cache", "pkv_append_kv", "pkv_compress_eligible_pages",
     "pkv_decode_attention", "pkv_decode_attention_host", "pkv_get_page_table", "pkv_get_stats",
     "pkv_free_seq", "pkv_destroy_cache", "pkv_last_error", "pkv_read_factors", "pkv_write_factors",
-    "pkv_read_dense", "pkv_get_decode_plan",
+    "pkv_read_dense", "pkv_get_decode_plan", "pkv_decode_attention_static_scratch",
 ]
 
 
@@ -80,6 +80,7 @@ def lib():
         L.pkv_append_kv.argtypes = [vp, i32, i32, ip, ip, vp, vp, vp]
         L.pkv_compress_eligible_pages.argtypes = [vp, i32, ctypes.POINTER(i64), vp]
         L.pkv_decode_attention.argtypes = [vp, i32, i32, ip, vp, vp, vp, vp]
+        L.pkv_decode_attention_static_scratch.argtypes = [vp, i32, i32, ip, vp, vp, vp, vp]
         L.pkv_decode_attention_host.argtypes = [vp, i32, i32, ip, vp, vp, vp, vp, vp]
         L.pkv_get_page_table.argtypes = [vp, i32, i32, ip, ip, ip, ip]
         L.pkv_get_stats.argtypes = [vp, ctypes.POINTER(PkvStats), vp]
@@ -160,6 +161,14 @@ def pkv_compress_eligible_pages(handle, layer=-1, stream=None) -> int:
 def pkv_decode_attention(handle, layer, seq_ids, q, out, out_f32=None, stream=None):
     ids, n = _ints(seq_ids)
     _check(handle, lib().pkv_decode_attention(handle, layer, n, ids, _ptr(q), _ptr(out), _ptr(out_f32), _stream(stream)))
+
+
+def pkv_decode_attention_static_scratch(handle, layer, seq_ids, q, out, out_f32=None, stream=None):
+    """Same result as pkv_decode_attention; the split-K scratch is a fixed array inside the library, for
+    callers that cannot supply a workspace.  Shared by all calls on the device: do not overlap calls."""
+    ids, n = _ints(seq_ids)
+    _check(handle, lib().pkv_decode_attention_static_scratch(handle, layer, n, ids, _ptr(q), _ptr(out), _ptr(out_f32),
+                                                             _stream(stream)))
 
 
 def pkv_decode_attention_host(handle, layer, seq_ids, q_host, out_host, q_stage, out_stage, stream=None):
