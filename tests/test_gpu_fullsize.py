@@ -1,0 +1,232 @@
+"""GPU parity at the benchmark's full sizes, in the launch configuration bench.py times (same cache
+builder, default grid, overlapping per-layer launches).  The oracle cannot run these workloads whole,
+so it checks sampled (sequence, layer, KV head) slices: heads are independent, so attention for the
+query heads of one KV head needs only that head's pages.
+
+  kernel gate      the oracle attends over the slice's pages exactly as stored on the GPU (bf16 factors
+                   and dense rows read back): max-abs <= 1e-2 * ||out||_inf
+  factor gate      every factor page of the slice: ||X - A B||_F <= 1.01 * tail + 1e-3 * ||X||_F, tail
+                   from the oracle's fp64 SVD of the regenerated page
+  end-to-end gate  oracle append + compress + attend on the regenerated slice (fp64 factors):
+                   <= 1e-2 + 3 x (the oracle's own bf16-storage error)
+"""
+import copy
+
+import numpy as np
+import pytest
+import torch
+
+import bench
+from gpu_helpers import f64, rel_err
+from oracle import attention as oatt
+from oracle import svd as osvd
+from oracle.cache import FACTOR, OracleCache, OracleConfig
+from paper_2608_23843_b200 import pkv, synth
+
+pytestmark = pytest.mark.gpu
+ATT_TOL = 1e-2
+
+
+def stored_kv(cache, seq, layer, head):
+    """K_all, V_all [T, d] of one (sequence, layer, KV head) exactly as the GPU stores them."""
+    kinds, slots, T = cache.page_table(seq, layer)
+    Ks, Vs, factors = [], [], {}
+    for p, (kd, slot) in enumerate(zip(kinds, slots)):
+        rows = min(64, T - p * 64)
+        if kd == FACTOR:
+            A_k, B_k, A_v, B_v = [f64(t) for t in cache.read_factors(slot, head)]
+            factors[p] = (A_k, B_k, A_v, B_v)
+            Ks.append(A_k @ B_k)
+            Vs.append(A_v @ B_v)
+        else:
+            K, V = cache.read_dense(slot, head)
+            Ks.append(f64(K)[:rows])
+            Vs.append(f64(V)[:rows])
+    return np.concatenate(Ks), np.concatenate(Vs), factors
+
+
+def kernel_gate(cache, cfg, layer, order, q, out, samples):
+    G = cfg.n_q_heads // cfg.n_kv_heads
+    scale = 1.0 / np.sqrt(cfg.head_dim)
+    worst = 0.0
+    for (i, head) in samples:
+        K_all, V_all, _ = stored_kv(cache, order[i], layer, head)
+        for g in range(G):
+            h = head * G + g
+            ref = oatt.attention_plain(f64(q[i, h]), K_all, V_all, scale)
+            e = rel_err(f64(out[i, h]), ref)
+            assert e <= ATT_TOL, (order[i], layer, h, e)
+            worst = max(worst, e)
+    return worst
+
+
+def oracle_slice(w, rank, seq, layer, head, T, device, steps_kv=None):
+    """Single-KV-head oracle cache of one slice, regenerated with the bench's generator."""
+    k, v = synth.make_kv(bench.SEED, layer, seq, T, w["n_kv_heads"], 128, 64, device, w["outliers"])
+    k, v = f64(k[:, head:head + 1]), f64(v[:, head:head + 1])
+    G = w["n_q_heads"] // w["n_kv_heads"]
+    n_pages = -(-T // 64) + 16
+    orc = OracleCache(OracleConfig(n_layers=1, n_kv_heads=1, n_q_heads=G, head_dim=128, page_size=64, rank_k=rank,
+                                   rank_v=rank, sink_tokens=w["sink"], recent_tokens=w["recent"], max_seqs=1,
+                                   n_dense_slots=n_pages, n_factor_slots=n_pages))
+    orc.append_kv(0, [0], [T], k, v)
+    orc.compress_eligible_pages(0)
+    return orc, k, v
+
+
+def factor_and_e2e_gates(cache, w, rank, seq, layer, head, T, q_row, out_row, device):
+    """q_row/out_row: [G, d] of this KV head's query heads."""
+    orc, k, v = oracle_slice(w, rank, seq, layer, head, T, device)
+    _, _, gpu_factors = stored_kv(cache, seq, layer, head)
+    okinds, oslots, _ = orc.page_table(0, 0)
+    assert sorted(gpu_factors) == [p for p, kd in enumerate(okinds) if kd == FACTOR]
+    worst = 0.0
+    for p, (A_k, B_k, A_v, B_v) in gpu_factors.items():
+        sig_k, sig_v = orc.sigma[oslots[p]]
+        for X, A, B, sig in ((k[p * 64:(p + 1) * 64, 0], A_k, B_k, sig_k[0]), (v[p * 64:(p + 1) * 64, 0], A_v, B_v, sig_v[0])):
+            err = np.linalg.norm(X - A @ B)
+            bound = 1.01 * float(np.sqrt((sig[rank:] ** 2).sum())) + 1e-3 * np.linalg.norm(X)
+            assert err <= bound, (seq, layer, head, p, err, bound)
+            worst = max(worst, err / bound)
+            assert np.abs(A.T @ A - np.eye(rank)).max() <= 1e-2
+    qd = f64(q_row)[None]
+    ref = orc.decode_attention(0, [0], qd)[0]
+    rounded = copy.deepcopy(orc)
+    rounded.round_factors_to_storage_type()
+    floor = rel_err(rounded.decode_attention(0, [0], qd)[0], ref)
+    e2e = rel_err(f64(out_row), ref)
+    assert e2e <= ATT_TOL + 3.0 * floor, (seq, layer, head, e2e, floor)
+    return worst, e2e, floor
+
+
+def _decode_all(cache, w, ids, device):
+    qs = [synth.make_q(bench.SEED, layer, 0, len(ids), w["n_q_heads"], 128, device) for layer in range(w["n_layers"])]
+    outs = [torch.empty_like(q) for q in qs]
+    for layer in range(w["n_layers"]):
+        cache.decode_attention(layer, ids, qs[layer], outs[layer])
+    torch.cuda.synchronize()
+    return qs, outs
+
+
+def _finish(cache):
+    st = cache.stats()
+    assert st["device_timeouts"] == 0 and st["page_svds_not_converged"] == 0 and st["bad_slot_indices"] == 0, st
+    cache.close()
+
+
+def test_llama3_8b_layer_batch8_context_32k():
+    """BASELINE config 1: 32q/8kv, batch 8, T=32768, r=24, 64 sink + 256 recent, shuffled pools."""
+    w, device = bench.WORKLOADS["llama3_8b_32k_b8"], torch.device("cuda", 0)
+    cfg, cache, lengths, comp = bench.build_workload(w, w["rank"], device)
+    assert comp["n_page_svds"] == 64896
+    ids = list(range(w["batch"]))
+    assert cache.page_table(3, 0)[0] == [0] + [1] * 507 + [0] * 4
+    qs, outs = _decode_all(cache, w, ids, device)
+    G = 4
+    worst = kernel_gate(cache, cfg, 0, ids, qs[0], outs[0], [(0, 0), (5, 7), (7, 3)])
+    fw, e2e, floor = factor_and_e2e_gates(cache, w, w["rank"], 5, 0, 7, lengths[5], qs[0][5, 7 * G:8 * G], outs[0][5, 7 * G:8 * G], device)
+    again = torch.empty_like(outs[0])
+    cache.decode_attention(0, ids, qs[0], again)
+    torch.cuda.synchronize()
+    assert torch.equal(again, outs[0])
+    print("config 1: kernel gate %.2e, factor err/bound %.3f, e2e %.2e (floor %.2e)" % (worst, fw, e2e, floor))
+    _finish(cache)
+
+
+def test_qwen3_32b_64_layers_context_128k():
+    """BASELINE config 2: 64 layers, 64q/8kv, batch 1, T=131072, r=24, 64 sink + 512 recent."""
+    w, device = bench.WORKLOADS["qwen3_32b_128k"], torch.device("cuda", 0)
+    cfg, cache, lengths, comp = bench.build_workload(w, w["rank"], device)
+    assert comp["n_page_svds"] == 2087936
+    kinds = cache.page_table(0, 63)[0]
+    assert kinds == [0] + [1] * 2039 + [0] * 8
+    qs, outs = _decode_all(cache, w, [0], device)
+    G = 8
+    worst = 0.0
+    for layer, head in ((0, 0), (31, 5), (63, 7)):
+        worst = max(worst, kernel_gate(cache, cfg, layer, [0], qs[layer], outs[layer], [(0, head)]))
+    fw, e2e, floor = factor_and_e2e_gates(cache, w, w["rank"], 0, 31, 5, lengths[0], qs[31][0, 5 * G:6 * G],
+                                          outs[31][0, 5 * G:6 * G], device)
+    print("config 2: kernel gate %.2e, factor err/bound %.3f, e2e %.2e (floor %.2e), %.0f page SVDs/s"
+          % (worst, fw, e2e, floor, comp["pages_per_s"]))
+    _finish(cache)
+
+
+@pytest.mark.parametrize("rank", [8, 16, 24, 32])
+def test_ragged_serving_batch_rank_sweep(rank):
+    """BASELINE config 4: 64 requests, lengths log-uniform in [2048, 65536], 2% outlier key tokens (x10)."""
+    w, device = bench.WORKLOADS["ragged_b64"], torch.device("cuda", 0)
+    cfg, cache, lengths, comp = bench.build_workload(w, rank, device)
+    ids = list(range(w["batch"]))
+    qs, outs = _decode_all(cache, w, ids, device)
+    short, long_ = int(np.argmin(lengths)), int(np.argmax(lengths))
+    worst = kernel_gate(cache, cfg, 0, ids, qs[0], outs[0], [(short, 1), (long_, 6), (17, 0)])
+    G = 4
+    fw, e2e, floor = factor_and_e2e_gates(cache, w, rank, short, 0, 1, lengths[short], qs[0][short, G:2 * G],
+                                          outs[0][short, G:2 * G], device)
+    assert any(t % 64 for t in lengths)                     # partial last pages are present
+    print("config 4 r=%d: kernel gate %.2e, factor err/bound %.3f, e2e %.2e (floor %.2e)" % (rank, worst, fw, e2e, floor))
+    _finish(cache)
+
+
+def test_incremental_compression_during_decoding():
+    """BASELINE config 3: batch 32, prompts of 8192 tokens prefilled and compressed, then 512 steps of
+    append -> attend -> compress; a page per (sequence, KV head, K|V) leaves the 256-token window every
+    64 steps.  Page tables are checked bit-exact against the oracle's state machine at every step; the
+    kernel gate runs at sampled steps; one slice is followed end to end by a single-head oracle."""
+    device = torch.device("cuda", 0)
+    H, Hq, B, T0, steps, rank = 8, 32, 32, 8192, 512, 24
+    n_pages = (T0 + steps) // 64 + 1
+    cfg = pkv.make_config(n_layers=1, n_kv_heads=H, n_q_heads=Hq, rank=rank, sink_tokens=64, recent_tokens=256,
+                          max_seqs=B, max_pages_per_seq=n_pages, n_dense_slots=B * (T0 // 64 + 2),
+                          n_factor_slots=B * n_pages)
+    d_ord = synth.slot_permutation(3, cfg.n_dense_slots, 0).tolist()
+    f_ord = synth.slot_permutation(3, cfg.n_factor_slots, 1).tolist()
+    cache = pkv.Cache(cfg, device, d_ord, f_ord)
+    mirror = OracleCache(OracleConfig(n_layers=1, n_kv_heads=1, n_q_heads=1, head_dim=128, page_size=64, rank_k=rank,
+                                      rank_v=rank, sink_tokens=64, recent_tokens=256, max_seqs=B,
+                                      n_dense_slots=cfg.n_dense_slots, n_factor_slots=cfg.n_factor_slots), d_ord, f_ord)
+    ids = list(range(B))
+    kv = [synth.make_kv(3, 0, s, T0 + steps, H, 128, 64, device) for s in ids]
+    cache.append_kv(0, ids, [T0] * B, torch.cat([k[:T0] for k, _ in kv]), torch.cat([v[:T0] for _, v in kv]))
+    assert cache.compress_eligible_pages(0) == B * 123
+    # the oracle state machine with zero data mirrors slot numbering (cheap: zero pages converge at once)
+    z = np.zeros((B * T0, 1, 128))
+    mirror.append_kv(0, ids, [T0] * B, z, z)
+    mirror.compress_eligible_pages(0)
+    seq_s, head_s, G = 11, 2, Hq // H
+    orc = OracleCache(OracleConfig(n_layers=1, n_kv_heads=1, n_q_heads=G, head_dim=128, page_size=64, rank_k=rank,
+                                   rank_v=rank, sink_tokens=64, recent_tokens=256, max_seqs=1, n_dense_slots=n_pages,
+                                   n_factor_slots=n_pages))
+    ks, vs = f64(kv[seq_s][0][:, head_s:head_s + 1]), f64(kv[seq_s][1][:, head_s:head_s + 1])
+    orc.append_kv(0, [0], [T0], ks[:T0], vs[:T0])
+    orc.compress_eligible_pages(0)
+    z1 = np.zeros((B, 1, 128))
+    n_events = 0
+    for t in range(steps):
+        knew = torch.cat([k[T0 + t:T0 + t + 1] for k, _ in kv])
+        vnew = torch.cat([v[T0 + t:T0 + t + 1] for _, v in kv])
+        cache.append_kv(0, ids, [1] * B, knew, vnew)
+        mirror.append_kv(0, ids, [1] * B, z1, z1)
+        orc.append_kv(0, [0], [1], ks[T0 + t:T0 + t + 1], vs[T0 + t:T0 + t + 1])
+        if t + 1 in (1, 64, 65, 512):
+            q = synth.make_q(3, 0, t, B, Hq, 128, device)
+            out = cache.decode_attention(0, ids, q)
+            torch.cuda.synchronize()
+            kernel_gate(cache, cfg, 0, ids, q, out, [(seq_s, head_s), (0, 7)])
+            qd = f64(q[seq_s, head_s * G:(head_s + 1) * G])[None]
+            ref = orc.decode_attention(0, [0], qd)[0]
+            rounded = copy.deepcopy(orc)
+            rounded.round_factors_to_storage_type()
+            floor = rel_err(rounded.decode_attention(0, [0], qd)[0], ref)
+            e2e = rel_err(f64(out[seq_s, head_s * G:(head_s + 1) * G]), ref)
+            assert e2e <= ATT_TOL + 3.0 * floor, (t, e2e, floor)
+        n = cache.compress_eligible_pages(0)
+        assert n == mirror.compress_eligible_pages(0) == (B if (T0 + t + 1) % 64 == 0 else 0)
+        orc.compress_eligible_pages(0)
+        n_events += n > 0
+    assert n_events == 8
+    for s in (0, seq_s, B - 1):
+        assert cache.page_table(s, 0) == mirror.page_table(s, 0)
+    assert cache.page_table(seq_s, 0)[0] == orc.page_table(0, 0)[0]
+    _finish(cache)
