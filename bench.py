@@ -189,6 +189,17 @@ def _config_dict(args, w, rank):
             "parallelism": "replicas x%d" % args.gpus}
 
 
+def max_over_ranks(values, world, device="cpu"):
+    """Element-wise max of a list of floats over all ranks (identity when world == 1)."""
+    if world <= 1:
+        return [float(v) for v in values]
+    import torch
+    import torch.distributed as dist
+    t = torch.tensor(values, device=device, dtype=torch.float64)
+    dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    return [float(x) for x in t.tolist()]
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
@@ -300,10 +311,7 @@ def main():
     if st["device_timeouts"] or st["bad_slot_indices"] or (outs[0].float().isnan().any().item()):
         raise SystemExit("decode produced timeouts or NaNs: %r" % st)
 
-    t = torch.tensor([ms, e2e_ms, launch_ms], device=device, dtype=torch.float64)
-    if world > 1:
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-    ms, e2e_ms, launch_ms = [float(x) for x in t.tolist()]
+    ms, e2e_ms, launch_ms = max_over_ranks([ms, e2e_ms, launch_ms], world, device)
 
     if rk == 0:
         peak, peak_src = _peaks()
