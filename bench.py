@@ -39,6 +39,10 @@ WORKLOADS = {
                  ragged=False, outliers=0.0),
 }
 SEED = 0
+# DRAM bytes (read + write) per algorithmic byte of a decode launch, from the ncu capture summarised in
+# profiles/decode_tc_kernel_r24_llama3_8b_32k_b8.md: (608.92 MB read + 4.52 MB written) / 608.70 MB.  Every
+# unit is fetched once, so traffic scales with the units a launch processes.
+NCU_TRAFFIC_PER_ALGORITHMIC_BYTE = (608.9216e6 + 4.52096e6) / 608698368.0
 
 
 def _peaks():
@@ -328,7 +332,10 @@ def main():
             "pages_factorized_per_s": comp["pages_per_s"], "page_svds_timed": comp["n_page_svds"],
             "roofline": {"bound": "hbm", "kernel": "decode_tc_kernel<%d>" % rank,
                          "achieved": achieved, "peak": peak, "unit": "GB/s", "frac": achieved / peak,
-                         "peak_source": peak_src, "traffic": None, "launch_us": launch_ms * 1e3,
+                         "peak_source": peak_src,
+                         "traffic": bytes_per_launch * NCU_TRAFFIC_PER_ALGORITHMIC_BYTE,
+                         "traffic_source": "ncu dram__bytes_read+write of this kernel on the llama3_8b_32k_b8 launch, "
+                                           "scaled by algorithmic bytes", "launch_us": launch_ms * 1e3,
                          "algorithmic_bytes_per_launch": bytes_per_launch},
             "e2e": {"value": e2e_ms * 1e3, "unit": "us", "h2d_bytes_per_step": qbytes, "d2h_bytes_per_step": qbytes},
             "gpu_launches": L * args.steps, "clocks": clocks,

@@ -173,11 +173,13 @@ pkv_status pkv_decode_attention(pkv_cache *c, int32_t layer, int32_t n_seqs, con
                                 const void *q, void *out, float *out_f32, void *stream);
 
 /*
- * The same call for callers whose queries and results live in host memory:
- * copies q_host -> q_stage, runs pkv_decode_attention, copies out_stage ->
- * out_host, all on `stream` (asynchronous if the host buffers are pinned).
+ * The same call for callers whose queries and results live in host memory.
  *   q_host, out_host [host] bf16 [n_seqs, H_q, d];  q_stage, out_stage [device]
  *   caller-owned staging buffers of the same size.
+ * If both host buffers are pinned and device-mapped (cudaHostAlloc / cudaHostRegister), the kernel
+ * reads q_host and writes out_host across the bus directly and the staging buffers are not used;
+ * otherwise q_host is copied to q_stage, the kernel runs, and out_stage is copied to out_host, all on
+ * `stream`.  Either way out_host is valid once the work enqueued on `stream` has completed.
  */
 pkv_status pkv_decode_attention_host(pkv_cache *c, int32_t layer, int32_t n_seqs, const int32_t *seq_ids,
                                      const void *q_host, void *out_host, void *q_stage, void *out_stage,

@@ -34,3 +34,17 @@ def eligible_pages_token_form(T: int, P: int, sink_tokens: int, recent_tokens: i
             continue
         out.append(p)
     return out
+
+
+def hybrid_cache_bytes(T: int, P: int, sink_tokens: int, recent_tokens: int, r_k: int, r_v: int, d: int,
+                       n_layers: int, n_kv_heads: int, bytes_per_element: int = 2) -> int:
+    """Logical live footprint of the hybrid cache (Section 3.3 construction + Eq. 3): every
+    factorized page holds (r_k + r_v)(P + d) elements, every other token 2 d elements, per layer
+    and KV head.  Pages are factorized by the closed-form rule of cache.eligible_range."""
+    n_c = T // P
+    lo = sink_tokens // P
+    hi = max(lo, n_c - recent_tokens // P)
+    n_factor = hi - lo
+    dense_tokens = T - n_factor * P
+    per_head = n_factor * (r_k + r_v) * (P + d) + dense_tokens * 2 * d
+    return n_layers * n_kv_heads * per_head * bytes_per_element

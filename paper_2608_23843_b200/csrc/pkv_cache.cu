@@ -691,6 +691,16 @@ pkv_status pkv_decode_attention_host(pkv_cache *c, int32_t layer, int32_t n_seqs
         return fail(c, PKV_ERR_INVALID_ARG, "host or staging buffer is NULL");
     cudaStream_t st = (cudaStream_t)stream;
     const size_t bytes = (size_t)n_seqs * c->cfg.n_q_heads * kRowBytes;
+    // Pinned, device-mapped host buffers: the kernel reads q and writes out across the bus itself, so no
+    // copy operation sits between consecutive launches (they keep overlapping).  The bytes still cross
+    // the bus inside this call.  Anything else goes through the staging buffers.
+    auto mapped = [](const void *p) -> void * {
+        cudaPointerAttributes at;
+        if (cudaPointerGetAttributes(&at, p) != cudaSuccess) { cudaGetLastError(); return nullptr; }
+        return at.type == cudaMemoryTypeHost ? at.devicePointer : nullptr;
+    };
+    void *q_dev = mapped(q_host), *out_dev = mapped(out_host);
+    if (q_dev && out_dev) return pkv_decode_attention(c, layer, n_seqs, seq_ids, q_dev, out_dev, nullptr, stream);
     PKV_CUDA(c, cudaMemcpyAsync(q_stage, q_host, bytes, cudaMemcpyHostToDevice, st));
     pkv_status r = pkv_decode_attention(c, layer, n_seqs, seq_ids, q_stage, out_stage, nullptr, stream);
     if (r != PKV_OK) return r;

@@ -210,3 +210,25 @@ def test_degenerate_pages_do_not_hang_or_poison():
     torch.cuda.synchronize()
     st = pair.gpu.stats()
     assert st["device_timeouts"] == 0
+
+
+@pytest.mark.parametrize("pinned", [True, False])
+def test_host_buffer_decode_matches_device_buffer_decode(pinned):
+    """pkv_decode_attention_host: pinned buffers are read/written by the kernel itself, pageable ones staged."""
+    cfg = pkv.make_config(n_layers=1, n_kv_heads=2, n_q_heads=8, rank=16, sink_tokens=64, recent_tokens=128,
+                          max_seqs=2, max_pages_per_seq=32, n_dense_slots=64, n_factor_slots=64)
+    pair = Pair(cfg, seed=13, oracle=False)
+    for s, T in enumerate([1800, 333]):
+        k, v = gen_kv(13, 0, s, T, cfg)
+        pair.gpu.append_kv(0, [s], [T], k.cuda(), v.cuda())
+    pair.gpu.compress_eligible_pages(0)
+    q = synth.make_q(13, 0, 0, 2, 8, 128)
+    ref = pair.gpu.decode_attention(0, [0, 1], q.cuda())
+    q_host = q.clone().pin_memory() if pinned else q.clone()
+    out_host = torch.zeros_like(q).pin_memory() if pinned else torch.zeros_like(q)
+    q_stage, out_stage = torch.empty_like(ref), torch.empty_like(ref)
+    for _ in range(2):
+        out_host.zero_()
+        pair.gpu.decode_attention_host(0, [0, 1], q_host, out_host, q_stage, out_stage)
+        torch.cuda.synchronize()
+        assert torch.equal(out_host, ref.cpu())

@@ -231,3 +231,16 @@ def test_storage_rounding_keeps_tables_and_perturbs_factors_by_bf16_epsilon():
         for n, a in f.items():
             rel = np.abs(a - before[s][n]) / np.maximum(np.abs(before[s][n]), 1e-300)
             assert rel.max() <= 2.0 ** -8 and rel.max() > 0
+
+
+def test_footprint_table_printed_in_paper_weak_pin():
+    for L, H, d, P, S, W, rk, rv, raw_mib, comp_mib, steady, theory, rtol in _rows("footprint.txt"):
+        L, H, d, P, S, W, rk, rv = (int(x) for x in (L, H, d, P, S, W, rk, rv))
+        per_token = accounting.kv_cache_elements(L, H, 1, d) * 2
+        T = round(raw_mib * 2 ** 20 / per_token)
+        assert abs(T * per_token / 2 ** 20 - raw_mib) <= 0.01            # the raw figure is a whole token count
+        got = accounting.hybrid_cache_bytes(T, P, S, W, rk, rv, d, L, H) / 2 ** 20
+        assert abs(got - comp_mib) <= rtol * comp_mib
+        assert abs(got / raw_mib - steady) <= 2e-3
+        assert abs(accounting.page_storage_ratio(rk, rv, P, d) - theory) <= 1e-4
+        assert abs((steady - theory) - 0.0017) <= 2e-4                   # "0.17 percentage points above"
