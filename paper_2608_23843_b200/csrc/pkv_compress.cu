@@ -211,12 +211,15 @@ compress_kernel(Geometry geo, const unsigned char *dense_pool, unsigned char *fa
 
 cudaError_t launch_compress(const Geometry &geo, const unsigned char *dense_pool, unsigned char *factor_pool,
                             const int2 *worklist, int n_entries, int *status, cudaStream_t st) {
-    static bool configured = false;
-    if (!configured) {
-        cudaError_t e = cudaFuncSetAttribute(compress_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                             (int)sizeof(CompressSmem));
+    static bool configured[64] = {};         // the attribute is per device
+    int dev = 0;
+    cudaError_t e = cudaGetDevice(&dev);
+    if (e != cudaSuccess) return e;
+    if (dev < 0 || dev >= 64 || !configured[dev]) {
+        e = cudaFuncSetAttribute(compress_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                 (int)sizeof(CompressSmem));
         if (e != cudaSuccess) return e;
-        configured = true;
+        if (dev >= 0 && dev < 64) configured[dev] = true;
     }
     const unsigned grid = (unsigned)n_entries * geo.n_kv_heads * 2;
     compress_kernel<<<grid, kThreads, sizeof(CompressSmem), st>>>(geo, dense_pool, factor_pool, worklist, status);
