@@ -25,9 +25,11 @@
  *    as void*); calls are asynchronous unless stated.  Operations on one cache
  *    must be issued on one stream (or the caller orders the streams).
  *  - One cache object is not thread-safe; use one host thread per cache.
- *  - Supported shapes: head_dim = 128, page_size = 64, rank_k = rank_v in
- *    {8,16,24,32}, 1 <= n_q_heads / n_kv_heads <= 8.  Anything else returns
- *    PKV_ERR_UNSUPPORTED from pkv_init_cache().
+ *  - Supported shapes: head_dim = 128; page_size 16, 32 or 64; 1 <= rank_k,
+ *    rank_v <= min(32, page_size) with ceil(rank_k / 8) == ceil(rank_v / 8)
+ *    (e.g. the paper's default P = 32, (r_K, r_V) = (16, 14)); 1 <= n_q_heads /
+ *    n_kv_heads <= 8.  Anything else returns PKV_ERR_UNSUPPORTED from
+ *    pkv_init_cache().
  *  - Dry-run mode: if dense_pool, factor_pool, meta and workspace are all NULL
  *    in pkv_init_cache(), no CUDA call is ever made; append / compress /
  *    free_seq update the page tables exactly as they would with device buffers
@@ -88,7 +90,7 @@ typedef struct pkv_config {
 
 typedef struct pkv_sizes {
     int64_t dense_slot_bytes;   /* H_kv * 2 * P * d * 2 */
-    int64_t factor_slot_bytes;  /* H_kv * 2 * (P*r_k + r_k*d + P*r_v + r_v*d) bytes; Eq. 3 is factor_slot_bytes / dense_slot_bytes */
+    int64_t factor_slot_bytes;  /* H_kv * 2 * (r_k + r_v) * (P + d) bytes; Eq. 3 is factor_slot_bytes / dense_slot_bytes */
     int64_t dense_pool_bytes;   /* n_dense_slots * dense_slot_bytes */
     int64_t factor_pool_bytes;
     int64_t meta_bytes;         /* device page tables, token counts, decode plans, status words */
@@ -121,10 +123,10 @@ pkv_status pkv_query_sizes(const pkv_config *cfg, pkv_sizes *out);
  *       (a shuffled physical pool); NULL = identity.  A released slot is reused
  *       (last released first) before the order array is consumed further.
  *   out  receives the cache handle.
- * The storage format inside the pools is private (rows are stored with a
- * 16-byte-chunk XOR swizzle so that a page can be copied linearly into shared
- * memory and read without bank conflicts); use pkv_read_* / pkv_write_factors
- * to look inside.
+ * The storage format inside the pools is private (A factors are stored
+ * transposed, and all rows carry a 16-byte-chunk XOR swizzle, so that a page can
+ * be copied linearly into shared memory and read without bank conflicts); use
+ * pkv_read_* / pkv_write_factors to look inside.
  */
 pkv_status pkv_init_cache(const pkv_config *cfg, void *dense_pool, void *factor_pool,
                           void *meta, void *workspace,

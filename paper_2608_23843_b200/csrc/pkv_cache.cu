@@ -128,9 +128,11 @@ pkv_status validate(const pkv_config *cfg, const char **why) {
         *why = "slot counts must fit in int32"; return PKV_ERR_INVALID_ARG;
     }
     if (cfg->head_dim != kHeadDim) { *why = "only head_dim = 128 is supported"; return PKV_ERR_UNSUPPORTED; }
-    if (cfg->page_size != kPage) { *why = "only page_size = 64 is supported"; return PKV_ERR_UNSUPPORTED; }
-    if (cfg->rank_k != cfg->rank_v || cfg->rank_k % 8 || cfg->rank_k > 32) {
-        *why = "only rank_k = rank_v in {8,16,24,32} is supported"; return PKV_ERR_UNSUPPORTED;
+    if (cfg->page_size != 16 && cfg->page_size != 32 && cfg->page_size != 64) {
+        *why = "only page_size 16, 32 or 64 is supported"; return PKV_ERR_UNSUPPORTED;
+    }
+    if ((cfg->rank_k + 7) / 8 != (cfg->rank_v + 7) / 8 || cfg->rank_k > 32 || cfg->rank_v > 32) {
+        *why = "ranks must be <= 32 and round up to the same multiple of 8 for K and V"; return PKV_ERR_UNSUPPORTED;
     }
     if (cfg->n_q_heads / cfg->n_kv_heads > kMaxGroup) { *why = "only n_q_heads/n_kv_heads <= 8 is supported"; return PKV_ERR_UNSUPPORTED; }
     return PKV_OK;
@@ -142,7 +144,9 @@ void derive(const pkv_config &cfg, int n_ctas, Geometry &g, MetaLayout &ml, Work
     const int P = cfg.page_size, d = cfg.head_dim;
     g.n_layers = cfg.n_layers; g.n_kv_heads = cfg.n_kv_heads; g.n_q_heads = cfg.n_q_heads;
     g.group = cfg.n_q_heads / cfg.n_kv_heads;
+    g.page = P;
     g.rank_k = cfg.rank_k; g.rank_v = cfg.rank_v;
+    g.rank_tiles = (cfg.rank_k + 7) / 8;
     g.max_seqs = cfg.max_seqs; g.max_pages = cfg.max_pages_per_seq;
     g.n_dense_slots = (int)cfg.n_dense_slots; g.n_factor_slots = (int)cfg.n_factor_slots;
     g.sink_pages = cfg.sink_tokens / P; g.recent_pages = cfg.recent_tokens / P;
@@ -154,9 +158,12 @@ void derive(const pkv_config &cfg, int n_ctas, Geometry &g, MetaLayout &ml, Work
     g.dense_head_bytes = 2 * P * d * 2;
     g.dense_slot_bytes = (long long)cfg.n_kv_heads * g.dense_head_bytes;
     g.factor_slot_bytes = (long long)cfg.n_kv_heads * g.blob_bytes;
-    g.stage_bytes = std::max(g.blob_bytes, 8192);
-    g.block_tokens = g.stage_bytes >= 16384 ? 32 : 16;
+    // decode work units: a factor page or a block of rows of a dense page.  A stage must hold either, plus
+    // the rows that 8-row tile loads read past the last matrix when rank_v is not a multiple of 8.
+    g.block_tokens = (P >= 32 && g.rank_tiles >= 3) ? 32 : 16;
     g.blocks_per_page = P / g.block_tokens;
+    const int overread = (8 * g.rank_tiles - cfg.rank_v) * kRowBytes;
+    g.stage_bytes = (int)align_up(std::max(g.blob_bytes + overread, g.block_tokens * 2 * kRowBytes), 128);
     // two CTAs are resident per SM (consecutive launches overlap, or the grid holds two CTAs per SM),
     // so that one streams while the other is in its prologue or merging
     const int fixed = kConsumerWarps * kPartialFloats * 4 + 1024 + 1024;
@@ -300,7 +307,7 @@ pkv_status build_plan(pkv_cache *c, int layer, int n_seqs, const int32_t *seq_id
     long long total_cost = 0, total_units = 0;
     for (int i = 0; i < n_seqs; ++i) {
         const SeqLayer &s = c->at(seq_ids[i], layer);
-        int n_pages = (s.n_tokens + kPage - 1) / kPage;
+        int n_pages = (s.n_tokens + c->cfg.page_size - 1) / c->cfg.page_size;
         entries[i] = PlanEntry{seq_ids[i], n_pages, g.sink_pages, s.f_end};
         shapes[i] = head_shape(g, n_pages, g.sink_pages, s.f_end, cf, cd);
         total_cost += shapes[i].cost * H;
@@ -482,7 +489,7 @@ pkv_status pkv_append_kv(pkv_cache *c, int32_t layer, int32_t n_seqs, const int3
     for (int i = 0; i < n_seqs; ++i) {
         if (n_new[i] < 0) return fail(c, PKV_ERR_INVALID_ARG, "n_new[%d] is negative", i);
         const SeqLayer &s = c->at(seq_ids[i], layer);
-        long long after = ((long long)s.n_tokens + n_new[i] + kPage - 1) / kPage;
+        long long after = ((long long)s.n_tokens + n_new[i] + c->cfg.page_size - 1) / c->cfg.page_size;
         if (after > c->cfg.max_pages_per_seq)
             return fail(c, PKV_ERR_POOL_EXHAUSTED, "sequence %d would exceed max_pages_per_seq", seq_ids[i]);
         need += after - (long long)s.slots.size();
@@ -502,7 +509,7 @@ pkv_status pkv_append_kv(pkv_cache *c, int32_t layer, int32_t n_seqs, const int3
         SeqLayer &s = c->at(seq_ids[i], layer);
         desc.push_back(AppendDesc{seq_ids[i], s.n_tokens, (int)tok, n_new[i]});
         int before = (int)s.slots.size();
-        int after = (s.n_tokens + n_new[i] + kPage - 1) / kPage;
+        int after = (s.n_tokens + n_new[i] + c->cfg.page_size - 1) / c->cfg.page_size;
         for (int p = before; p < after; ++p) s.slots.push_back(c->dense_free.alloc());
         s.n_tokens += n_new[i];
         tok += n_new[i];
@@ -565,7 +572,7 @@ pkv_status pkv_compress_eligible_pages(pkv_cache *c, int32_t layer, int64_t *n_p
     for (int seq = 0; seq < c->cfg.max_seqs && !exhausted; ++seq) {
         for (int ly = l0; ly < l1 && !exhausted; ++ly) {
             SeqLayer &s = c->at(seq, ly);
-            const int n_c = s.n_tokens / kPage;
+            const int n_c = s.n_tokens / c->cfg.page_size;
             const int hi = std::max(g.sink_pages, n_c - g.recent_pages);   // eligible: sink_pages <= p < hi
             if (s.f_end >= hi) continue;
             const int first = s.f_end;
@@ -619,8 +626,8 @@ pkv_status pkv_decode_attention(pkv_cache *c, int32_t layer, int32_t n_seqs, con
         const int n_pages = (int)s.slots.size();
         const int nf = std::min(s.f_end, n_pages) - std::min(c->geo.sink_pages, n_pages);
         const bool last_dense = !(n_pages - 1 >= c->geo.sink_pages && n_pages - 1 < s.f_end);
-        int64_t rows = (int64_t)(n_pages - nf) * kPage;
-        if (last_dense) rows -= (int64_t)n_pages * kPage - s.n_tokens;  // unfilled rows of the last page are not read
+        int64_t rows = (int64_t)(n_pages - nf) * c->cfg.page_size;
+        if (last_dense) rows -= (int64_t)n_pages * c->cfg.page_size - s.n_tokens;  // unfilled rows of the last page are not read
         bytes += (int64_t)c->geo.n_kv_heads * ((int64_t)nf * c->geo.blob_bytes + rows * 2 * kRowBytes);
     }
     c->last_decode_bytes = bytes;

@@ -91,10 +91,10 @@ __global__ void __launch_bounds__(128) decode_scalar_kernel(const __grid_constan
     if (!load_range(a, rg)) return;
     const Geometry &g = a.geo;
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
-    const int G = g.group, H = g.n_kv_heads, r_k = g.rank_k, r_v = g.rank_v;
+    const int G = g.group, H = g.n_kv_heads, r_k = g.rank_k, r_v = g.rank_v, P = g.page;
     __shared__ float qs[kMaxGroup][kHeadDim];
     __shared__ float qt[kMaxGroup][32];
-    __shared__ float sc[kMaxGroup][kPage];
+    __shared__ float sc[kMaxGroup][kMaxPage];
     __shared__ float wv[kMaxGroup][32];
     __shared__ float m_s[kMaxGroup], l_s[kMaxGroup], alpha_s[kMaxGroup];
     float o[kMaxGroup];
@@ -122,7 +122,7 @@ __global__ void __launch_bounds__(128) decode_scalar_kernel(const __grid_constan
             int rows;
             const unsigned char *base;
             if (kind == kKindFactor) {
-                rows = kPage;
+                rows = P;
                 base = a.factor_pool + (long long)slot * g.factor_slot_bytes + (long long)cur.head * g.blob_bytes;
                 for (int i = tid; i < G * r_k; i += 128) {           // q~ = B_k q
                     const int gq = i / r_k, j = i % r_k;
@@ -131,15 +131,15 @@ __global__ void __launch_bounds__(128) decode_scalar_kernel(const __grid_constan
                     qt[gq][j] = acc;
                 }
                 __syncthreads();
-                for (int i = tid; i < G * kPage; i += 128) {         // s = A_k q~ * scale
-                    const int gq = i / kPage, p = i % kPage;
+                for (int i = tid; i < G * P; i += 128) {             // s = A_k q~ * scale
+                    const int gq = i / P, p = i % P;
                     float acc = 0.f;
-                    for (int j = 0; j < r_k; ++j) acc += bf16_at(base + g.ak_off, (p * r_k + j) * 2) * qt[gq][j];
+                    for (int j = 0; j < r_k; ++j) acc += bf16_at(base + g.ak_off, a_t_offset(P, j, p)) * qt[gq][j];
                     sc[gq][p] = acc * g.scale_log2e;
                 }
             } else {
                 const int row0 = blk * g.block_tokens;
-                rows = min(g.block_tokens, T - page * kPage - row0);
+                rows = min(g.block_tokens, T - page * P - row0);
                 if (rows <= 0) continue;
                 base = a.dense_pool + (long long)slot * g.dense_slot_bytes + (long long)cur.head * g.dense_head_bytes;
                 for (int i = tid; i < G * rows; i += 128) {
@@ -170,7 +170,7 @@ __global__ void __launch_bounds__(128) decode_scalar_kernel(const __grid_constan
                 for (int i = tid; i < G * r_v; i += 128) {           // w = A_v^T p
                     const int gq = i / r_v, j = i % r_v;
                     float acc = 0.f;
-                    for (int p = 0; p < kPage; ++p) acc += sc[gq][p] * bf16_at(base + g.av_off, (p * r_v + j) * 2);
+                    for (int p = 0; p < P; ++p) acc += sc[gq][p] * bf16_at(base + g.av_off, a_t_offset(P, j, p));
                     wv[gq][j] = acc;
                 }
                 __syncthreads();
@@ -184,7 +184,7 @@ __global__ void __launch_bounds__(128) decode_scalar_kernel(const __grid_constan
                 for (int gq = 0; gq < G; ++gq) {
                     float acc = 0.f;
                     for (int p = 0; p < rows; ++p)
-                        acc += sc[gq][p] * bf16_at(base + kPage * kRowBytes, swz_off(row0 + p, tid));
+                        acc += sc[gq][p] * bf16_at(base + P * kRowBytes, swz_off(row0 + p, tid));
                     o[gq] = o[gq] * alpha_s[gq] + acc;
                 }
             }
@@ -323,24 +323,26 @@ __device__ __forceinline__ float bf16hi_f(uint32_t x) { return __uint_as_float(x
 
 struct StageDesc { int kind, rows, seg, pad; };
 
-template <int R>
-struct Tc {
-    static constexpr int kBlob = 2 * (kPage * R + R * kHeadDim) * 2;
-    static constexpr int kStage = kBlob > 8192 ? kBlob : 8192;
-    static constexpr int kDB = kStage >= 16384 ? 32 : 16;      // dense block tokens
-    static constexpr int kAk = 0, kBk = kPage * R * 2, kAv = kBk + R * kHeadDim * 2, kBv = kAv + kPage * R * 2;
-    static constexpr int kNT = R / 8;                          // 8-wide rank tiles
-};
-
 // Per-warp running state for the query heads 2t, 2t+1 (t = lane & 3) of one KV head.
 struct WarpState {
     float o[8][4];        // o[i]: (d = 16i+g, heads 2t,2t+1), (d = 16i+8+g, heads 2t,2t+1);  g = lane >> 2
     float m[2], l[2];     // l is this lane's share; summed over g at flush time
 };
 
-template <int NTOK>       // softmax over NTOK/16 score tiles; returns p in place and the movmatrix'ed bf16 copies
+// Shapes fixed at compile time: P tokens per page, NT = ceil(rank / 8) rank tiles (K and V alike).
+template <int P, int NT>
+struct Tc {
+    static constexpr int kMT = P / 16;                                  // 16-token tiles per page
+    static constexpr int kDB = (P >= 32 && NT >= 3) ? 32 : 16;          // rows per dense block
+    static constexpr int kPitchA = 2 * P;                               // bytes per A^T row
+};
+
+// chunk swizzle of an A^T row as a function of the row's low bits (see swz_a_chunk)
+template <int P>
+__device__ __forceinline__ int a_swz(int l7) { return P == 64 ? l7 : (P == 32 ? (l7 >> 1) : (l7 >> 2)); }
+
+template <int NI>         // softmax over NI score tiles of 16 tokens; leaves p in place and its bf16, transposed copies
 __device__ __forceinline__ void online_softmax(float (&s)[4][4], WarpState &st, uint32_t (&T0)[4], uint32_t (&T1)[4]) {
-    constexpr int NI = NTOK / 16;
     float mx0 = kNegInf, mx1 = kNegInf;
 #pragma unroll
     for (int i = 0; i < NI; ++i) {
@@ -376,84 +378,93 @@ __device__ __forceinline__ void online_softmax(float (&s)[4][4], WarpState &st, 
     }
 }
 
-template <int R>
-__device__ __forceinline__ void factor_unit(uint32_t sb, const uint32_t (&qf)[8][2], float scale, WarpState &st, int lane) {
-    using C = Tc<R>;
-    const int l7 = lane & 7, mi = lane >> 3;
-    // ---- q~^T [G][R] = q [G][d] . B_k^T ----
-    float qt[C::kNT][4];
-    uint32_t qhi[C::kNT], qlo[C::kNT];
+// One factor page.  sb = shared address of the blob; ak/bk/av/bv = byte offsets of its four matrices;
+// rk, rv = true ranks (tile rows past them hold other finite data and are multiplied by exact zeros).
+template <int P, int NT>
+__device__ __forceinline__ void factor_unit(uint32_t sb, int ak, int bk, int av, int bv, int rk, int rv,
+                                            const uint32_t (&qf)[8][2], float scale, WarpState &st, int lane) {
+    using C = Tc<P, NT>;
+    const int l7 = lane & 7, mi = lane >> 3, t2 = (lane & 3) * 2;
+    const int asw = a_swz<P>(l7);
+    // ---- q~^T [G][r] = q [G][d] . B_k^T ----
+    uint32_t qhi[NT], qlo[NT];
 #pragma unroll
-    for (int j = 0; j < C::kNT; ++j) {
-        qt[j][0] = qt[j][1] = qt[j][2] = qt[j][3] = 0.f;
+    for (int j = 0; j < NT; ++j) {
+        float qt[4] = {0.f, 0.f, 0.f, 0.f};
 #pragma unroll
         for (int qd = 0; qd < 4; ++qd) {
             uint32_t b[4];
-            ldsm_x4(b, sb + C::kBk + (8 * j + l7) * kRowBytes + (((4 * qd + mi) ^ l7) << 4));
-            mma16816(qt[j], qf[2 * qd][0], 0u, qf[2 * qd][1], 0u, b[0], b[1]);
-            mma16816(qt[j], qf[2 * qd + 1][0], 0u, qf[2 * qd + 1][1], 0u, b[2], b[3]);
+            ldsm_x4(b, sb + bk + (8 * j + l7) * kRowBytes + (((4 * qd + mi) ^ l7) << 4));
+            mma16816(qt, qf[2 * qd][0], 0u, qf[2 * qd][1], 0u, b[0], b[1]);
+            mma16816(qt, qf[2 * qd + 1][0], 0u, qf[2 * qd + 1][1], 0u, b[2], b[3]);
         }
-        const float x0 = qt[j][0] * scale, x1 = qt[j][1] * scale;
+        const float x0 = (8 * j + t2 < rk) ? qt[0] * scale : 0.f;
+        const float x1 = (8 * j + t2 + 1 < rk) ? qt[1] * scale : 0.f;
         qhi[j] = pack_bf16(x0, x1);
         qlo[j] = pack_bf16(x0 - bf16lo_f(qhi[j]), x1 - bf16hi_f(qhi[j]));
     }
-    // ---- s [P][G] = A_k [P][R] . q~ ----
+    // ---- s [P][G] = A_k [P][r] . q~   (A_k^T in shared memory: transposed tile loads) ----
     float s[4][4];
 #pragma unroll
-    for (int i = 0; i < 4; ++i) {
+    for (int i = 0; i < C::kMT; ++i) {
         s[i][0] = s[i][1] = s[i][2] = s[i][3] = 0.f;
 #pragma unroll
-        for (int kk = 0; kk < R / 16; ++kk) {
-            uint32_t av[4];
-            ldsm_x4(av, sb + C::kAk + (16 * i + (mi & 1) * 8 + l7) * (2 * R) + ((2 * kk + (mi >> 1)) << 4));
-            mma16816(s[i], av[0], av[1], av[2], av[3], qhi[2 * kk], qhi[2 * kk + 1]);
-            mma16816(s[i], av[0], av[1], av[2], av[3], qlo[2 * kk], qlo[2 * kk + 1]);
+        for (int kk = 0; kk < NT / 2; ++kk) {
+            uint32_t a4[4];
+            ldsm_x4_t(a4, sb + ak + (16 * kk + (mi >> 1) * 8 + l7) * C::kPitchA + (((2 * i + (mi & 1)) ^ asw) << 4));
+            mma16816(s[i], a4[0], a4[1], a4[2], a4[3], qhi[2 * kk], qhi[2 * kk + 1]);
+            mma16816(s[i], a4[0], a4[1], a4[2], a4[3], qlo[2 * kk], qlo[2 * kk + 1]);
         }
-        if (R % 16 == 8) {
-            uint32_t av[2];
-            ldsm_x2(av, sb + C::kAk + (16 * i + (mi & 1) * 8 + l7) * (2 * R) + ((R / 8 - 1) << 4));
-            mma1688(s[i], av[0], av[1], qhi[C::kNT - 1]);
-            mma1688(s[i], av[0], av[1], qlo[C::kNT - 1]);
+        if (NT % 2) {
+            uint32_t a2[2];
+            ldsm_x2_t(a2, sb + ak + (8 * (NT - 1) + l7) * C::kPitchA + (((2 * i + (mi & 1)) ^ asw) << 4));
+            mma1688(s[i], a2[0], a2[1], qhi[NT - 1]);
+            mma1688(s[i], a2[0], a2[1], qlo[NT - 1]);
         }
     }
     uint32_t T0[4], T1[4];
-    online_softmax<kPage>(s, st, T0, T1);
-    // ---- w^T [G][R] = p^T [G][P] . A_v [P][R] ----
-    uint32_t wh[C::kNT];
+    online_softmax<C::kMT>(s, st, T0, T1);
+    // ---- w^T [G][r] = p^T [G][P] . A_v [P][r] ----
+    uint32_t wh[NT];
 #pragma unroll
-    for (int j = 0; j < C::kNT; ++j) {
+    for (int j = 0; j < NT; ++j) {
         float wt[4] = {0.f, 0.f, 0.f, 0.f};
 #pragma unroll
-        for (int qd = 0; qd < 2; ++qd) {
+        for (int qd = 0; qd < C::kMT / 2; ++qd) {
             uint32_t b[4];
-            ldsm_x4_t(b, sb + C::kAv + (16 * (2 * qd + (mi >> 1)) + (mi & 1) * 8 + l7) * (2 * R) + (j << 4));
+            ldsm_x4(b, sb + av + (8 * j + l7) * C::kPitchA + (((4 * qd + mi) ^ asw) << 4));
             mma16816(wt, T0[2 * qd], 0u, T1[2 * qd], 0u, b[0], b[1]);
             mma16816(wt, T0[2 * qd + 1], 0u, T1[2 * qd + 1], 0u, b[2], b[3]);
         }
-        wh[j] = pack_bf16(wt[0], wt[1]);
+        if (C::kMT % 2) {
+            uint32_t b[2];
+            ldsm_x2(b, sb + av + (8 * j + l7) * C::kPitchA + (((2 * (C::kMT - 1) + (mi & 1)) ^ asw) << 4));
+            mma16816(wt, T0[C::kMT - 1], 0u, T1[C::kMT - 1], 0u, b[0], b[1]);
+        }
+        wh[j] = pack_bf16((8 * j + t2 < rv) ? wt[0] : 0.f, (8 * j + t2 + 1 < rv) ? wt[1] : 0.f);
     }
-    // ---- o [d][G] += B_v^T [d][R] . w ----
+    // ---- o [d][G] += B_v^T [d][r] . w ----
 #pragma unroll
     for (int i = 0; i < 8; ++i) {
 #pragma unroll
-        for (int kk = 0; kk < R / 16; ++kk) {
-            uint32_t av[4];
-            ldsm_x4_t(av, sb + C::kBv + (16 * kk + (mi >> 1) * 8 + l7) * kRowBytes + (((2 * i + (mi & 1)) ^ l7) << 4));
-            mma16816(st.o[i], av[0], av[1], av[2], av[3], wh[2 * kk], wh[2 * kk + 1]);
+        for (int kk = 0; kk < NT / 2; ++kk) {
+            uint32_t a4[4];
+            ldsm_x4_t(a4, sb + bv + (16 * kk + (mi >> 1) * 8 + l7) * kRowBytes + (((2 * i + (mi & 1)) ^ l7) << 4));
+            mma16816(st.o[i], a4[0], a4[1], a4[2], a4[3], wh[2 * kk], wh[2 * kk + 1]);
         }
-        if (R % 16 == 8) {
-            uint32_t av[2];
-            ldsm_x2_t(av, sb + C::kBv + (R - 8 + l7) * kRowBytes + (((2 * i + (mi & 1)) ^ l7) << 4));
-            mma1688(st.o[i], av[0], av[1], wh[C::kNT - 1]);
+        if (NT % 2) {
+            uint32_t a2[2];
+            ldsm_x2_t(a2, sb + bv + (8 * (NT - 1) + l7) * kRowBytes + (((2 * i + (mi & 1)) ^ l7) << 4));
+            mma1688(st.o[i], a2[0], a2[1], wh[NT - 1]);
         }
     }
 }
 
-template <int R>
+// One block of DB rows of a dense page: K rows at sb, V rows at sb + DB*256; `rows` of them are valid.
+template <int DB>
 __device__ __forceinline__ void dense_unit(uint32_t sb, unsigned char *sp, int rows, const uint32_t (&qf)[8][2],
                                            float scale, WarpState &st, int lane) {
-    using C = Tc<R>;
-    constexpr int DB = C::kDB, NI = DB / 16;
+    constexpr int NI = DB / 16;
     const int l7 = lane & 7, mi = lane >> 3, g = lane >> 2;
     if (rows < DB) {
         // unfilled V rows hold stale bytes: zero them so that 0 * garbage cannot make a NaN
@@ -467,24 +478,24 @@ __device__ __forceinline__ void dense_unit(uint32_t sb, unsigned char *sp, int r
         s[i][0] = s[i][1] = s[i][2] = s[i][3] = 0.f;
 #pragma unroll
         for (int kk = 0; kk < 8; ++kk) {
-            uint32_t av[4];
-            ldsm_x4(av, sb + (16 * i + (mi & 1) * 8 + l7) * kRowBytes + (((2 * kk + (mi >> 1)) ^ l7) << 4));
-            mma16816(s[i], av[0], av[1], av[2], av[3], qf[kk][0], qf[kk][1]);
+            uint32_t a4[4];
+            ldsm_x4(a4, sb + (16 * i + (mi & 1) * 8 + l7) * kRowBytes + (((2 * kk + (mi >> 1)) ^ l7) << 4));
+            mma16816(s[i], a4[0], a4[1], a4[2], a4[3], qf[kk][0], qf[kk][1]);
         }
         const bool v0 = 16 * i + g < rows, v1 = 16 * i + 8 + g < rows;
         s[i][0] = v0 ? s[i][0] * scale : kNegInf; s[i][1] = v0 ? s[i][1] * scale : kNegInf;
         s[i][2] = v1 ? s[i][2] * scale : kNegInf; s[i][3] = v1 ? s[i][3] * scale : kNegInf;
     }
     uint32_t T0[4], T1[4];
-    online_softmax<DB>(s, st, T0, T1);
+    online_softmax<NI>(s, st, T0, T1);
 #pragma unroll
     for (int ii = 0; ii < 8; ++ii) {
 #pragma unroll
         for (int i = 0; i < NI; ++i) {
-            uint32_t av[4];
-            ldsm_x4_t(av, sb + DB * kRowBytes + (16 * i + (mi >> 1) * 8 + l7) * kRowBytes +
+            uint32_t a4[4];
+            ldsm_x4_t(a4, sb + DB * kRowBytes + (16 * i + (mi >> 1) * 8 + l7) * kRowBytes +
                               (((2 * ii + (mi & 1)) ^ l7) << 4));
-            mma16816(st.o[ii], av[0], av[1], av[2], av[3], T0[i], T1[i]);
+            mma16816(st.o[ii], a4[0], a4[1], a4[2], a4[3], T0[i], T1[i]);
         }
     }
 }
@@ -616,9 +627,9 @@ __device__ __forceinline__ void flush_segment(const DecodeArgs &a, float *comb, 
     PKV_CONSUMER_BARRIER();
 }
 
-template <int R>
+template <int P, int NT>
 __global__ void __launch_bounds__(kDecodeThreads, 2) decode_tc_kernel(const __grid_constant__ DecodeArgs a) {
-    using C = Tc<R>;
+    using C = Tc<P, NT>;
     Range rg;
     if (!load_range(a, rg)) return;
     const Geometry &geo = a.geo;
@@ -628,7 +639,8 @@ __global__ void __launch_bounds__(kDecodeThreads, 2) decode_tc_kernel(const __gr
     const int W = min(kConsumerWarps, S);
     extern __shared__ __align__(1024) unsigned char smem[];
     unsigned char *stages = smem;
-    float *comb = reinterpret_cast<float *>(smem + (size_t)S * C::kStage);
+    const int stage_bytes = geo.stage_bytes, blob_bytes = geo.blob_bytes;
+    float *comb = reinterpret_cast<float *>(smem + (size_t)S * stage_bytes);
     unsigned long long *full_bar = reinterpret_cast<unsigned long long *>(comb + kConsumerWarps * kPartialFloats);
     unsigned long long *empty_bar = full_bar + S;
     StageDesc *descs = reinterpret_cast<StageDesc *>(empty_bar + S);
@@ -645,6 +657,16 @@ __global__ void __launch_bounds__(kDecodeThreads, 2) decode_tc_kernel(const __gr
         *abort_flag = 0;
         *issued = 0;
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    }
+    if (stage_bytes > blob_bytes) {
+        // Tile loads of 8 rows read past a rank that is not a multiple of 8; past the last matrix that is the
+        // tail of the stage, which no copy of a factor page ever writes.  Those values are multiplied by exact
+        // zeros, so they only have to be finite: clear the tails once.
+        const int tail16 = (stage_bytes - blob_bytes) >> 4;
+        for (int i = tid; i < S * tail16; i += kDecodeThreads)
+            reinterpret_cast<uint4 *>(stages + (size_t)(i / tail16) * stage_bytes + blob_bytes)[i % tail16] =
+                make_uint4(0u, 0u, 0u, 0u);
+        asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
     }
     __syncthreads();
     // Programmatic dependent launch: let the next kernel on the stream begin as SMs free up.  Unless the caller
@@ -680,10 +702,10 @@ __global__ void __launch_bounds__(kDecodeThreads, 2) decode_tc_kernel(const __gr
                         kind = kKindDense;
                         rows = 0;
                     } else if (kind == kKindFactor) {
-                        rows = kPage;
+                        rows = P;
                         src = a.factor_pool + (long long)slot * geo.factor_slot_bytes + (long long)cur.head * geo.blob_bytes;
                     } else {
-                        rows = max(0, min(C::kDB, T - page * kPage - blk * C::kDB));
+                        rows = max(0, min(C::kDB, T - page * P - blk * C::kDB));
                         src = a.dense_pool + (long long)slot * geo.dense_slot_bytes +
                               (long long)cur.head * geo.dense_head_bytes + blk * C::kDB * kRowBytes;
                     }
@@ -699,14 +721,14 @@ __global__ void __launch_bounds__(kDecodeThreads, 2) decode_tc_kernel(const __gr
                         if (ok) {
                             descs[s] = StageDesc{kind_j, rows_j, seg_local, 0};
                             const uint32_t bar = smem_u32(full_bar + s);
-                            const uint32_t dst = smem_u32(stages + (size_t)s * C::kStage);
+                            const uint32_t dst = smem_u32(stages + (size_t)s * stage_bytes);
                             if (kind_j == kKindFactor) {
-                                mbar_arrive_expect_tx(bar, C::kBlob);
-                                bulk_g2s(dst, (const void *)src_j, C::kBlob, bar);
+                                mbar_arrive_expect_tx(bar, blob_bytes);
+                                bulk_g2s(dst, (const void *)src_j, blob_bytes, bar);
                             } else if (rows_j > 0) {
                                 mbar_arrive_expect_tx(bar, 2 * rows_j * kRowBytes);
                                 bulk_g2s(dst, (const void *)src_j, rows_j * kRowBytes, bar);
-                                bulk_g2s(dst + C::kDB * kRowBytes, (const unsigned char *)src_j + kPage * kRowBytes,
+                                bulk_g2s(dst + C::kDB * kRowBytes, (const unsigned char *)src_j + P * kRowBytes,
                                          rows_j * kRowBytes, bar);
                             } else {
                                 mbar_arrive(bar);
@@ -774,13 +796,14 @@ __global__ void __launch_bounds__(kDecodeThreads, 2) decode_tc_kernel(const __gr
                 if (cur_seg < rg.n_local_segs) load_q(a, rg.seg_first + cur_seg, qf, lane);
             }
             if (dsc.kind == kKindEnd) break;
-            dsc.rows = min(dsc.rows, dsc.kind == kKindFactor ? kPage : C::kDB);
+            dsc.rows = min(dsc.rows, dsc.kind == kKindFactor ? P : C::kDB);
             if (dsc.rows > 0) {
-                const uint32_t sb = smem_u32(stages + (size_t)s * C::kStage);
+                const uint32_t sb = smem_u32(stages + (size_t)s * stage_bytes);
                 if (dsc.kind == kKindFactor) {
-                    factor_unit<R>(sb, qf, geo.scale_log2e, st, lane);
+                    factor_unit<P, NT>(sb, geo.ak_off, geo.bk_off, geo.av_off, geo.bv_off, geo.rank_k, geo.rank_v, qf,
+                                       geo.scale_log2e, st, lane);
                 } else {
-                    dense_unit<R>(sb, stages + (size_t)s * C::kStage, dsc.rows, qf, geo.scale_log2e, st, lane);
+                    dense_unit<C::kDB>(sb, stages + (size_t)s * stage_bytes, dsc.rows, qf, geo.scale_log2e, st, lane);
                     if (dsc.rows < C::kDB) asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
                 }
             }
@@ -790,49 +813,54 @@ __global__ void __launch_bounds__(kDecodeThreads, 2) decode_tc_kernel(const __gr
     }
 }
 
-template <int R>
+size_t decode_smem_bytes(const Geometry &g) {
+    return (size_t)g.n_stages * g.stage_bytes + kConsumerWarps * kPartialFloats * 4 +
+           g.n_stages * (8 + 8 + sizeof(StageDesc)) + 64;
+}
+
+template <int P, int NT>
 cudaError_t launch_tc(const DecodeArgs &a, cudaStream_t st) {
-    using C = Tc<R>;
-    const size_t smem = (size_t)a.geo.n_stages * C::kStage + kConsumerWarps * kPartialFloats * 4 +
-                        a.geo.n_stages * (8 + 8 + sizeof(StageDesc)) + 64;
     cudaLaunchConfig_t cfg = {};
     cfg.gridDim = dim3(a.geo.n_ctas);
     cfg.blockDim = dim3(kDecodeThreads);
-    cfg.dynamicSmemBytes = smem;
+    cfg.dynamicSmemBytes = decode_smem_bytes(a.geo);
     cfg.stream = st;
     cudaLaunchAttribute attr[1];
     attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
     attr[0].val.programmaticStreamSerializationAllowed = 1;
     cfg.attrs = attr;
     cfg.numAttrs = 1;
-    return cudaLaunchKernelEx(&cfg, decode_tc_kernel<R>, a);
+    return cudaLaunchKernelEx(&cfg, decode_tc_kernel<P, NT>, a);
 }
+
+template <int P, int NT>
+cudaError_t setup_tc() {
+    return cudaFuncSetAttribute(decode_tc_kernel<P, NT>, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBudget / 2);
+}
+
+// the instantiated shapes: P in {16, 32, 64}, rank tiles 1..4 (1..2 for P = 16)
+#define PKV_FOR_EACH_SHAPE(X) \
+    X(16, 1) X(16, 2) X(32, 1) X(32, 2) X(32, 3) X(32, 4) X(64, 1) X(64, 2) X(64, 3) X(64, 4)
 
 }  // namespace
 
 cudaError_t decode_kernel_setup() {
     cudaError_t e;
-    const int max_smem = kSmemBudget;
-    if ((e = cudaFuncSetAttribute(decode_tc_kernel<8>, cudaFuncAttributeMaxDynamicSharedMemorySize, max_smem)) != cudaSuccess) return e;
-    if ((e = cudaFuncSetAttribute(decode_tc_kernel<16>, cudaFuncAttributeMaxDynamicSharedMemorySize, max_smem)) != cudaSuccess) return e;
-    if ((e = cudaFuncSetAttribute(decode_tc_kernel<24>, cudaFuncAttributeMaxDynamicSharedMemorySize, max_smem)) != cudaSuccess) return e;
-    if ((e = cudaFuncSetAttribute(decode_tc_kernel<32>, cudaFuncAttributeMaxDynamicSharedMemorySize, max_smem)) != cudaSuccess) return e;
+#define PKV_SETUP(P, NT) if ((e = setup_tc<P, NT>()) != cudaSuccess) return e;
+    PKV_FOR_EACH_SHAPE(PKV_SETUP)
+#undef PKV_SETUP
     return cudaSuccess;
 }
 
 cudaError_t launch_decode(const DecodeArgs &a, int n_segs, cudaStream_t st) {
-    cudaError_t e;
+    cudaError_t e = cudaErrorInvalidValue;
     if (a.variant == 1) {
         decode_scalar_kernel<<<a.geo.n_ctas, 128, 0, st>>>(a);
         e = cudaGetLastError();
     } else {
-        switch (a.geo.rank_k) {
-            case 8:  e = launch_tc<8>(a, st); break;
-            case 16: e = launch_tc<16>(a, st); break;
-            case 24: e = launch_tc<24>(a, st); break;
-            case 32: e = launch_tc<32>(a, st); break;
-            default: return cudaErrorInvalidValue;
-        }
+#define PKV_LAUNCH(P, NT) if (a.geo.page == P && a.geo.rank_tiles == NT) e = launch_tc<P, NT>(a, st);
+        PKV_FOR_EACH_SHAPE(PKV_LAUNCH)
+#undef PKV_LAUNCH
     }
     if (e != cudaSuccess || a.variant != 1) return e;
     merge_kernel<<<n_segs, 256, 0, st>>>(a);

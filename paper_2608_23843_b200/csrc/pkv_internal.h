@@ -9,7 +9,7 @@
 namespace pkv {
 
 constexpr int kHeadDim = 128;          // d (only supported value)
-constexpr int kPage = 64;              // P (only supported value)
+constexpr int kMaxPage = 64;           // P is 16, 32 or 64
 constexpr int kRowBytes = kHeadDim * 2;
 constexpr int kMaxGroup = 8;           // query heads per KV head handled by the tensor-core kernel
 constexpr int kConsumerWarps = 4;      // decode kernel: warps that compute (two CTAs share an SM)
@@ -22,11 +22,13 @@ constexpr int kSmemBudget = 227 * 1024;
 // Sizes derived from a validated pkv_config.  Plain data: passed to kernels by value.
 struct Geometry {
     int n_layers, n_kv_heads, n_q_heads, group;   // group = H_q / H_kv
+    int page;                          // P
     int rank_k, rank_v;
+    int rank_tiles;                    // ceil(rank / 8), the same for K and V
     int max_seqs, max_pages;
     int n_dense_slots, n_factor_slots;
     int sink_pages, recent_pages;
-    // factor blob of one (slot, KV head): [A_k P x r_k][B_k r_k x d][A_v P x r_v][B_v r_v x d], bf16
+    // factor blob of one (slot, KV head): [A_k^T r_k x P][B_k r_k x d][A_v^T r_v x P][B_v r_v x d], bf16
     int ak_off, bk_off, av_off, bv_off, blob_bytes;
     int dense_head_bytes;              // [K P x d][V P x d] of one KV head = 2*P*d*2
     long long dense_slot_bytes, factor_slot_bytes;
@@ -103,5 +105,17 @@ cudaError_t decode_kernel_setup();     // raises the dynamic shared-memory limit
 // Storage swizzle of a 256-byte row: 16-byte chunk c of row `row` lives at
 // chunk position c ^ (row & 7).  Applied to dense K/V rows and to B factors.
 __host__ __device__ inline int swz_chunk(int row, int chunk) { return chunk ^ (row & 7); }
+
+// A factors are stored transposed, [r][P]: rows of 2P bytes = P/8 chunks.  Eight consecutive rows must
+// land in eight different 16-byte bank groups of a 128-byte window, so the chunk index is XORed with
+// the row's position inside that window: P = 64 -> row & 7, P = 32 -> (row >> 1) & 3, P = 16 -> (row >> 2) & 1.
+__host__ __device__ inline int swz_a_chunk(int P, int row, int chunk) {
+    const int nch = P >> 3;
+    return chunk ^ (((row * nch) >> 3) & (nch - 1));
+}
+// byte offset of element (row r, token i) inside an A^T matrix
+__host__ __device__ inline int a_t_offset(int P, int r, int i) {
+    return r * 2 * P + swz_a_chunk(P, r, i >> 3) * 16 + (i & 7) * 2;
+}
 
 }  // namespace pkv

@@ -29,7 +29,7 @@ __global__ void append_kernel(Geometry geo, unsigned char *dense_pool, const int
         }
         const AppendDesc e = desc[lo];
         const int t = e.t_start + (int)(tok - e.tok_begin);
-        const int page = t / kPage, row = t % kPage;
+        const int page = t / geo.page, row = t % geo.page;
         const int slot = page_table[((long long)e.seq * geo.n_layers + layer) * geo.max_pages + page];
         if (slot < 0 || slot >= geo.n_dense_slots || page >= geo.max_pages) {
             if (chunk == 0 && kv == 0 && h == 0) atomicAdd(status + 2, 1);   // corrupt page table: skip the row
@@ -37,7 +37,7 @@ __global__ void append_kernel(Geometry geo, unsigned char *dense_pool, const int
         }
         const uint4 val = (kv ? v : k)[(tok * H + h) * 16 + chunk];
         unsigned char *dst = dense_pool + (long long)slot * geo.dense_slot_bytes + (long long)h * geo.dense_head_bytes +
-                             kv * (kPage * kRowBytes) + row * kRowBytes + swz_chunk(row, chunk) * 16;
+                             kv * (geo.page * kRowBytes) + row * kRowBytes + swz_chunk(row, chunk) * 16;
         *reinterpret_cast<uint4 *>(dst) = val;
     }
     if (blockIdx.x == 0) {
@@ -47,26 +47,28 @@ __global__ void append_kernel(Geometry geo, unsigned char *dense_pool, const int
     }
 }
 
-// blob <-> row-major factors.  dir = 0: blob -> arrays, 1: arrays -> blob.
+// blob <-> row-major factors.  dir = 0: blob -> arrays, 1: arrays -> blob.  The caller's A is [P][r]
+// row-major; the blob holds A^T with swizzled chunks, and B rows with the dense-row swizzle.
 __global__ void factor_io_kernel(Geometry geo, unsigned char *blob, unsigned short *A_k, unsigned short *B_k,
                                  unsigned short *A_v, unsigned short *B_v, int dir) {
-    const int rk = geo.rank_k, rv = geo.rank_v;
-    const int nAk = kPage * rk, nBk = rk * kHeadDim, nAv = kPage * rv, nBv = rv * kHeadDim;
+    const int P = geo.page, rk = geo.rank_k, rv = geo.rank_v;
+    const int nAk = P * rk, nBk = rk * kHeadDim, nAv = P * rv, nBv = rv * kHeadDim;
     for (int i = blockIdx.x * blockDim.x + threadIdx.x; i < nAk + nBk + nAv + nBv; i += gridDim.x * blockDim.x) {
         unsigned short *plain;
         unsigned short *stored;
-        if (i < nAk) {                          // A_k: plain row-major [P][r_k]
+        if (i < nAk) {
+            const int tok = i / rk, r = i % rk;
             plain = A_k + i;
-            stored = reinterpret_cast<unsigned short *>(blob + geo.ak_off) + i;
-        } else if (i < nAk + nBk) {             // B_k: rows of 256 B, chunk-swizzled
+            stored = reinterpret_cast<unsigned short *>(blob + geo.ak_off + a_t_offset(P, r, tok));
+        } else if (i < nAk + nBk) {
             int j = i - nAk, row = j / kHeadDim, col = j % kHeadDim;
             plain = B_k + j;
             stored = reinterpret_cast<unsigned short *>(blob + geo.bk_off + row * kRowBytes +
                                                         swz_chunk(row, col >> 3) * 16) + (col & 7);
         } else if (i < nAk + nBk + nAv) {
-            int j = i - nAk - nBk;
+            const int j = i - nAk - nBk, tok = j / rv, r = j % rv;
             plain = A_v + j;
-            stored = reinterpret_cast<unsigned short *>(blob + geo.av_off) + j;
+            stored = reinterpret_cast<unsigned short *>(blob + geo.av_off + a_t_offset(P, r, tok));
         } else {
             int j = i - nAk - nBk - nAv, row = j / kHeadDim, col = j % kHeadDim;
             plain = B_v + j;
@@ -77,11 +79,11 @@ __global__ void factor_io_kernel(Geometry geo, unsigned char *blob, unsigned sho
     }
 }
 
-__global__ void dense_read_kernel(const unsigned char *head_base, unsigned short *K, unsigned short *V) {
-    for (int i = blockIdx.x * blockDim.x + threadIdx.x; i < 2 * kPage * kHeadDim; i += gridDim.x * blockDim.x) {
-        int kv = i / (kPage * kHeadDim), j = i % (kPage * kHeadDim), row = j / kHeadDim, col = j % kHeadDim;
+__global__ void dense_read_kernel(int P, const unsigned char *head_base, unsigned short *K, unsigned short *V) {
+    for (int i = blockIdx.x * blockDim.x + threadIdx.x; i < 2 * P * kHeadDim; i += gridDim.x * blockDim.x) {
+        int kv = i / (P * kHeadDim), j = i % (P * kHeadDim), row = j / kHeadDim, col = j % kHeadDim;
         const unsigned short *src = reinterpret_cast<const unsigned short *>(
-                                        head_base + kv * (kPage * kRowBytes) + row * kRowBytes +
+                                        head_base + kv * (P * kRowBytes) + row * kRowBytes +
                                         swz_chunk(row, col >> 3) * 16) + (col & 7);
         (kv ? V : K)[j] = *src;
     }
@@ -118,9 +120,9 @@ cudaError_t launch_write_factors(const Geometry &geo, unsigned char *blob, const
     return cudaGetLastError();
 }
 
-cudaError_t launch_read_dense(const Geometry &, const unsigned char *head_base, void *K, void *V,
+cudaError_t launch_read_dense(const Geometry &geo, const unsigned char *head_base, void *K, void *V,
                               cudaStream_t st) {
-    dense_read_kernel<<<16, 256, 0, st>>>(head_base, (unsigned short *)K, (unsigned short *)V);
+    dense_read_kernel<<<16, 256, 0, st>>>(geo.page, head_base, (unsigned short *)K, (unsigned short *)V);
     return cudaGetLastError();
 }
 

@@ -43,6 +43,10 @@ def _check_reconstruction(pair, seq, layer, heads=None):
                 err = np.linalg.norm(X - A @ B)
                 tail = float(np.sqrt((sig[r:] ** 2).sum()))
                 bound = 1.01 * tail + 1e-3 * np.linalg.norm(X)
+                if r == cfg.page_size:
+                    # full rank: the optimal tail is zero and what is left is the bf16 rounding of the two
+                    # factors (about 0.0023 ||X|| rms), which the 1e-3 ||X|| allowance does not cover
+                    bound = 4e-3 * np.linalg.norm(X)
                 assert err <= bound, (seq, p, h, name, err, bound)
                 worst = max(worst, err / bound)
                 assert np.abs(A.T @ A - np.eye(r)).max() <= 1e-2
@@ -232,3 +236,41 @@ def test_host_buffer_decode_matches_device_buffer_decode(pinned):
         pair.gpu.decode_attention_host(0, [0, 1], q_host, out_host, q_stage, out_stage)
         torch.cuda.synchronize()
         assert torch.equal(out_host, ref.cpu())
+
+
+@pytest.mark.parametrize("P,rk,rv,G", [(32, 16, 14, 4), (32, 16, 16, 8), (16, 9, 9, 4), (64, 27, 27, 8), (64, 20, 17, 4),
+                                       (32, 8, 8, 2), (16, 16, 16, 8), (32, 32, 32, 4), (16, 3, 5, 1)])
+def test_other_page_sizes_and_ranks(P, rk, rv, G):
+    """The paper's default shape (P=32, ranks (16,14), one sink page, one window page), its page-size
+    ablation shapes (16,9,9) and (64,27,27), unequal and odd ranks, and full rank r = P."""
+    H = 2
+    lengths = [40 * P + 5, P, P + 6, 1, 2 * P + 1, 23 * P, 10 * P]
+    cfg = pkv.make_config(n_layers=1, n_kv_heads=H, n_q_heads=H * G, rank=rk, rank_v=rv, page_size=P,
+                          sink_tokens=P, recent_tokens=P if P == 32 else 2 * P, max_seqs=len(lengths),
+                          max_pages_per_seq=48, n_dense_slots=160, n_factor_slots=120)
+    pair = Pair(cfg, seed=P + rk)
+    for s, T in enumerate(lengths):
+        k, v = gen_kv(2, 0, s, T, cfg, outlier_prob=0.02)
+        _remember_pages(pair, s, 0, k, v)
+        cut = T // 2
+        if cut:
+            pair.append(0, [s], [k[:cut]], [v[:cut]])
+            pair.compress(0)
+        pair.append(0, [s], [k[cut:]], [v[cut:]])
+    pair.compress(-1)
+    pair.same_tables()
+    kinds = pair.gpu.page_table(0, 0)[0]
+    n_w = 1 if P == 32 else 2
+    assert kinds == [0] + [1] * (40 - 1 - n_w) + [0] * (n_w + 1)
+    order = [5, 0, 3, 6, 1, 2, 4]
+    q = synth.make_q(2, 0, 0, len(order), H * G, 128)
+    got, got32 = pair.decode(0, order, q)
+    worst = max(_check_reconstruction(pair, s, 0) for s in (0, 5))
+    g = attention_gates(pair, 0, order, q, got, got32)
+    assert_attention_gates(g)
+    again, _ = pair.decode(0, order, q)
+    assert (again == got).all()
+    st = pair.gpu.stats()
+    assert st["device_timeouts"] == 0 and st["page_svds_not_converged"] == 0 and st["bad_slot_indices"] == 0
+    print("P=%d r=(%d,%d) G=%d: e2e max %.2e (floor %.2e) kernel max %.2e recon/bound %.3f"
+          % (P, rk, rv, G, max(g["e2e"]), max(g["floor"]), max(g["kernel"]), worst))

@@ -43,7 +43,8 @@ def _pair(seed=None, **kw):
         d_ord, f_ord = rng.permutation(base["n_dense_slots"]), rng.permutation(base["n_factor_slots"])
     gpu = pkv.Cache(cfg, dry_run=True, dense_slot_order=d_ord, factor_slot_order=f_ord)
     ocfg = OracleConfig(n_layers=base["n_layers"], n_kv_heads=base["n_kv_heads"], n_q_heads=base["n_q_heads"],
-                        head_dim=128, page_size=64, rank_k=base["rank"], rank_v=base["rank"],
+                        head_dim=128, page_size=base.get("page_size", 64), rank_k=base["rank"],
+                        rank_v=base.get("rank_v", base["rank"]),
                         sink_tokens=base["sink_tokens"], recent_tokens=base["recent_tokens"],
                         max_seqs=base["max_seqs"], n_dense_slots=base["n_dense_slots"],
                         n_factor_slots=base["n_factor_slots"])
@@ -74,9 +75,13 @@ def test_tiny_config_has_13_factor_pages():
     assert T == 1024 and kinds == [0] + [1] * 13 + [0, 0]
 
 
-@pytest.mark.parametrize("seed", [0, 1, 2, 3])
-def test_random_schedule_matches_oracle_bit_exact(seed):
-    gpu, orc, base = _pair(seed=seed)
+@pytest.mark.parametrize("seed,shape", [(0, {}), (1, {}), (2, {}), (3, {}),
+                                        (4, dict(page_size=32, rank=16, rank_v=14, sink_tokens=32, recent_tokens=32,
+                                                 n_dense_slots=192, n_factor_slots=192, max_pages_per_seq=128)),
+                                        (5, dict(page_size=16, rank=9, sink_tokens=16, recent_tokens=48,
+                                                 n_dense_slots=384, n_factor_slots=384, max_pages_per_seq=256))])
+def test_random_schedule_matches_oracle_bit_exact(seed, shape):
+    gpu, orc, base = _pair(seed=seed, **shape)
     rng = np.random.default_rng(100 + seed)
     H = base["n_kv_heads"]
     for step in range(60):
@@ -151,23 +156,28 @@ def test_config_validation():
     pkv.pkv_query_sizes(pkv.make_config(**ok))
     for bad, status in [(dict(sink_tokens=10), pkv.PKV_ERR_INVALID_ARG), (dict(recent_tokens=65), pkv.PKV_ERR_INVALID_ARG),
                         (dict(n_q_heads=3, n_kv_heads=2), pkv.PKV_ERR_INVALID_ARG), (dict(rank=0), pkv.PKV_ERR_INVALID_ARG),
-                        (dict(rank=65), pkv.PKV_ERR_INVALID_ARG), (dict(rank=12), pkv.PKV_ERR_UNSUPPORTED),
-                        (dict(head_dim=64, page_size=64), pkv.PKV_ERR_UNSUPPORTED), (dict(page_size=32), pkv.PKV_ERR_UNSUPPORTED),
+                        (dict(rank=65), pkv.PKV_ERR_INVALID_ARG), (dict(rank=33), pkv.PKV_ERR_UNSUPPORTED),
+                        (dict(head_dim=64, page_size=64), pkv.PKV_ERR_UNSUPPORTED), (dict(page_size=48, sink_tokens=48, recent_tokens=48), pkv.PKV_ERR_UNSUPPORTED),
+                        (dict(page_size=16, rank=17, sink_tokens=16, recent_tokens=16), pkv.PKV_ERR_INVALID_ARG),
                         (dict(n_q_heads=16), pkv.PKV_ERR_UNSUPPORTED), (dict(rank=16, rank_v=8), pkv.PKV_ERR_UNSUPPORTED)]:
         with pytest.raises(pkv.PkvError) as e:
             pkv.pkv_query_sizes(pkv.make_config(**{**ok, **bad}))
         assert e.value.status == status, bad
+    for good in (dict(rank=12), dict(rank=16, rank_v=14, page_size=32, sink_tokens=32, recent_tokens=32),
+                 dict(rank=9, page_size=16, sink_tokens=16, recent_tokens=16), dict(rank=27)):
+        pkv.pkv_query_sizes(pkv.make_config(**{**ok, **good}))
     with pytest.raises(pkv.PkvError):
         pkv.Cache(pkv.make_config(**ok), dry_run=True, dense_slot_order=[0, 0, 1, 2])   # not a permutation
 
 
 def test_slot_sizes_follow_storage_ratio_formula():
-    for r in (8, 16, 24, 32):
-        sz = pkv.pkv_query_sizes(pkv.make_config(n_layers=1, n_kv_heads=8, n_q_heads=32, rank=r, sink_tokens=64,
-                                                 recent_tokens=256, max_seqs=1, max_pages_per_seq=8,
+    for P, rk, rv in [(64, 8, 8), (64, 16, 16), (64, 24, 24), (64, 32, 32), (64, 27, 27), (32, 16, 14), (32, 16, 16),
+                      (16, 9, 9)]:
+        sz = pkv.pkv_query_sizes(pkv.make_config(n_layers=1, n_kv_heads=8, n_q_heads=32, rank=rk, rank_v=rv, page_size=P,
+                                                 sink_tokens=P, recent_tokens=P, max_seqs=1, max_pages_per_seq=8,
                                                  n_dense_slots=8, n_factor_slots=8))
-        assert sz.dense_slot_bytes == 8 * 2 * 64 * 128 * 2
-        assert sz.factor_slot_bytes / sz.dense_slot_bytes == accounting.page_storage_ratio(r, r, 64, 128)
+        assert sz.dense_slot_bytes == 8 * 2 * P * 128 * 2
+        assert sz.factor_slot_bytes / sz.dense_slot_bytes == accounting.page_storage_ratio(rk, rv, P, 128)
 
 
 def _decode_bytes(T, P, S, W, r, H_kv, H_q):
