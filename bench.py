@@ -29,11 +29,17 @@ WORKLOADS = {
     "qwen3_32b_128k": dict(n_layers=64, n_kv_heads=8, n_q_heads=64, batch=1, T=131072, rank=24,
                            sink=64, recent=512, ragged=False, outliers=0.0),
     # BASELINE config 1: Llama-3-8B-shaped decode layer
-    "llama3_8b_32k_b8": dict(n_layers=1, n_kv_heads=8, n_q_heads=32, batch=8, T=32768, rank=24,
+    # (four independent layers of that shape are built and a step decodes one of them in turn, so that
+    # overlapping launches never stream the same bytes and cannot feed each other through L2)
+    "llama3_8b_32k_b8": dict(n_layers=4, layers_per_step=1, n_kv_heads=8, n_q_heads=32, batch=8, T=32768, rank=24,
                              sink=64, recent=256, ragged=False, outliers=0.0),
     # BASELINE config 4: ragged serving batch (rank chosen with --rank)
-    "ragged_b64": dict(n_layers=1, n_kv_heads=8, n_q_heads=32, batch=64, T=(2048, 65536), rank=24,
+    "ragged_b64": dict(n_layers=2, layers_per_step=1, n_kv_heads=8, n_q_heads=32, batch=64, T=(2048, 65536), rank=24,
                        sink=64, recent=256, ragged=True, outliers=0.02),
+    # The paper's own setting: Qwen3-8B shape (36 layers, 32q/8kv), 16K context, P=32, ranks (16,14),
+    # one sink page, last completed page + incomplete page dense
+    "qwen3_8b_16k_paper_default": dict(n_layers=36, n_kv_heads=8, n_q_heads=32, batch=1, T=16384 + 17, rank=16,
+                                       rank_v=14, page=32, sink=32, recent=32, ragged=False, outliers=0.0),
     # BASELINE config 0: tiny (L2-resident; latency only)
     "tiny": dict(n_layers=1, n_kv_heads=1, n_q_heads=4, batch=1, T=1024, rank=16, sink=64, recent=128,
                  ragged=False, outliers=0.0),
@@ -93,11 +99,11 @@ class ClockSampler:
                 "reasons": reasons, "samples": len(sm)}
 
 
-def build_workload(w, rank, device, overlap=1):
+def build_workload(w, rank, device, overlap=2, n_ctas=0):
     """Allocate the cache, generate each (layer, sequence) on the GPU, append and compress layer by layer."""
     import torch
     from paper_2608_23843_b200 import pkv, synth
-    P = 64
+    P = w.get("page", 64)
     if w["ragged"]:
         lengths = synth.loguniform_lengths(SEED, w["batch"], *w["T"])
     else:
@@ -110,9 +116,10 @@ def build_workload(w, rank, device, overlap=1):
     # dense slots: what stays dense in every layer plus one layer's worth of transient pages
     n_dense_slots = sum(pages) + L * sum(p - f for p, f in zip(pages, n_factor)) + 8
     cfg = pkv.make_config(n_layers=L, n_kv_heads=w["n_kv_heads"], n_q_heads=w["n_q_heads"], rank=rank,
+                          rank_v=w.get("rank_v", rank), page_size=P,
                           sink_tokens=w["sink"], recent_tokens=w["recent"], max_seqs=w["batch"],
                           max_pages_per_seq=max(pages), n_dense_slots=n_dense_slots, n_factor_slots=n_factor_slots,
-                          decode_overlap=overlap)
+                          decode_overlap=overlap, n_ctas=n_ctas)
     cache = pkv.Cache(cfg, device, synth.slot_permutation(SEED, n_dense_slots, 0).tolist(),
                       synth.slot_permutation(SEED, n_factor_slots, 1).tolist())
     ids = list(range(w["batch"]))
@@ -142,11 +149,12 @@ def oracle_sample(w, rank, steps):
     from paper_2608_23843_b200 import synth
     G = w["n_q_heads"] // w["n_kv_heads"]
     T = synth.loguniform_lengths(SEED, w["batch"], *w["T"])[0] if w["ragged"] else w["T"]
-    k, v = synth.make_kv(SEED, 0, 0, T, w["n_kv_heads"], 128, 64, "cpu", w["outliers"])
+    P = w.get("page", 64)
+    k, v = synth.make_kv(SEED, 0, 0, T, w["n_kv_heads"], 128, P, "cpu", w["outliers"])
     k, v = k[:, :1].to(torch.float64).numpy(), v[:, :1].to(torch.float64).numpy()
-    n_pages = -(-T // 64)
-    orc = OracleCache(OracleConfig(n_layers=1, n_kv_heads=1, n_q_heads=G, head_dim=128, page_size=64, rank_k=rank,
-                                   rank_v=rank, sink_tokens=w["sink"], recent_tokens=w["recent"], max_seqs=1,
+    n_pages = -(-T // P)
+    orc = OracleCache(OracleConfig(n_layers=1, n_kv_heads=1, n_q_heads=G, head_dim=128, page_size=P, rank_k=rank,
+                                   rank_v=w.get("rank_v", rank), sink_tokens=w["sink"], recent_tokens=w["recent"], max_seqs=1,
                                    n_dense_slots=n_pages, n_factor_slots=n_pages))
     orc.append_kv(0, [0], [T], k, v)
     t0 = time.perf_counter()
@@ -158,7 +166,7 @@ def oracle_sample(w, rank, steps):
         t0 = time.perf_counter()
         orc.decode_attention(0, [0], q)
         times.append(time.perf_counter() - t0)
-    slices_per_step = w["n_layers"] * w["n_kv_heads"] * w["batch"]
+    slices_per_step = w.get("layers_per_step", w["n_layers"]) * w["n_kv_heads"] * w["batch"]
     return dict(decode_s=statistics.median(times), slices_per_step=slices_per_step,
                 pages_per_s=(2 * n / t_svd if t_svd > 0 else None), cores=osvd.n_threads(), T=T,
                 sample="sequence 0, layer 0, KV head 0 (1/%d of a step): %d page SVDs + %d-head decode over %d tokens; "
@@ -182,14 +190,16 @@ def run_reference(args, w, rank):
 
 
 def _config_dict(args, w, rank):
-    return {"workload": args.workload, "n_layers": w["n_layers"], "n_q_heads": w["n_q_heads"],
-            "n_kv_heads": w["n_kv_heads"], "head_dim": 128, "batch": w["batch"], "context": w["T"], "page_size": 64,
-            "rank": rank, "sink_tokens": w["sink"], "recent_tokens": w["recent"],
+    return {"workload": args.workload, "n_layers": w["n_layers"], "layers_per_step": w.get("layers_per_step", w["n_layers"]), "n_q_heads": w["n_q_heads"],
+            "n_kv_heads": w["n_kv_heads"], "head_dim": 128, "batch": w["batch"], "context": w["T"],
+            "page_size": w.get("page", 64), "rank": rank, "rank_v": w.get("rank_v", rank), "sink_tokens": w["sink"], "recent_tokens": w["recent"],
             "l2": "inputs larger than L2 (no flush)" if args.workload != "tiny" else "L2-resident (latency only)",
-            "overlap": ("none: each launch waits for the previous one" if args.no_overlap else
-                        "consecutive per-layer launches overlap (programmatic dependent launch); valid here because "
-                        "queries are prepared in advance and no launch in the step writes the cache"),
-            "launch": "host launch per layer" if args.no_graph else "one CUDA graph replay per step (%d per-layer launches)" % w["n_layers"],
+            "overlap": ["0: each launch waits for the previous one",
+                        "1: consecutive per-layer launches overlap (programmatic dependent launch) and complete in order",
+                        "2: per-layer launches overlap freely (programmatic dependent launch, rotating split-K scratch, "
+                        "a draining launch every 15); valid here because queries are prepared in advance and no "
+                        "launch in the step writes the cache"][args.overlap],
+            "launch": "one CUDA graph replay per step (%d per-layer launches)" % w.get("layers_per_step", w["n_layers"]) if args.graph else "host launch per layer",
             "parallelism": "replicas x%d" % args.gpus}
 
 
@@ -213,9 +223,12 @@ def main():
     ap.add_argument("--rank", type=int, default=0, help="override the workload's rank (8, 16, 24, 32)")
     ap.add_argument("--impl", default="pkv", choices=["pkv", "reference"])
     ap.add_argument("--no-cpu-baseline", action="store_true")
-    ap.add_argument("--no-overlap", action="store_true",
-                    help="each layer's launch waits for the previous launch to finish before reading the cache")
-    ap.add_argument("--no-graph", action="store_true", help="launch every layer from the host instead of replaying a CUDA graph")
+    ap.add_argument("--overlap", type=int, default=2, choices=[0, 1, 2],
+                    help="decode_overlap mode of the cache: 0 = every launch waits for the previous one, 1 = launches "
+                         "overlap but complete in order, 2 = launches never wait for one another (default)")
+    ap.add_argument("--n-ctas", type=int, default=0, help="decode grid size (0 = library default)")
+    ap.add_argument("--graph", action="store_true",
+                    help="replay one CUDA graph per step instead of launching every layer from the host (overlap 0 or 1)")
     args = ap.parse_args()
     w = WORKLOADS[args.workload]
     rank = args.rank or w["rank"]
@@ -237,14 +250,19 @@ def main():
         dist.init_process_group("nccl", device_id=device)
     pkv.lib()                                             # fail loudly if the CUDA library is missing
 
-    cfg, cache, lengths, comp = build_workload(w, rank, device, 0 if args.no_overlap else 1)
+    cfg, cache, lengths, comp = build_workload(w, rank, device, args.overlap, args.n_ctas)
     ids = list(range(w["batch"]))
     L, Hq = w["n_layers"], w["n_q_heads"]
     qs = [synth.make_q(SEED, layer, 0, w["batch"], Hq, 128, device) for layer in range(L)]
     outs = [torch.empty_like(q) for q in qs]
 
+    lps = w.get("layers_per_step", L)
+    cursor = [0]
+
     def step():
-        for layer in range(L):
+        for _ in range(lps):
+            layer = cursor[0] % L
+            cursor[0] += 1
             cache.decode_attention(layer, ids, qs[layer], outs[layer])
 
     def barrier():
@@ -256,7 +274,9 @@ def main():
         step()
     torch.cuda.synchronize()
     eager_step = step
-    if not args.no_graph:
+    if args.graph:
+        if args.overlap == 2:
+            raise SystemExit("--graph needs --overlap 0 or 1 (mode 2 cannot be captured)")
         # one CUDA graph of the step's per-layer launches (plans are cached on the device, so the
         # captured launches read current page tables and token counts at replay time)
         side = torch.cuda.Stream()
@@ -272,7 +292,7 @@ def main():
         for _ in range(3):
             step()
     bytes_per_step = 0
-    for layer in range(L):                                # algorithmic bytes, from the library's own accounting
+    for layer in range(lps):                              # algorithmic bytes, from the library's own accounting
         cache.decode_attention(layer, ids, qs[layer], outs[layer])
         bytes_per_step += cache.stats()["last_decode_bytes"]
     sampler = ClockSampler(local)
@@ -288,7 +308,7 @@ def main():
     ms = e0.elapsed_time(e1) / args.steps
     # average duration of one decode-kernel launch over the timed region: the region holds nothing but
     # steps * L back-to-back launches of that kernel, so this includes the gaps between launches
-    launch_ms = ms / L
+    launch_ms = ms / lps
 
     # end to end: queries and results in pinned host memory, copies inside the timed region
     q_host = [q.cpu().pin_memory() for q in qs]
@@ -296,7 +316,9 @@ def main():
     q_stage, out_stage = torch.empty_like(qs[0]), torch.empty_like(qs[0])
 
     def step_host():
-        for layer in range(L):
+        for _ in range(lps):
+            layer = cursor[0] % L
+            cursor[0] += 1
             cache.decode_attention_host(layer, ids, q_host[layer], out_host[layer], q_stage, out_stage)
         torch.cuda.current_stream().synchronize()        # the caller reads the result on the host
 
@@ -319,9 +341,9 @@ def main():
 
     if rk == 0:
         peak, peak_src = _peaks()
-        bytes_per_launch = bytes_per_step / L
+        bytes_per_launch = bytes_per_step / lps
         achieved = bytes_per_launch / (launch_ms * 1e-3) / 1e9
-        qbytes = sum(q.numel() * 2 for q in qs)
+        qbytes = sum(q.numel() * 2 for q in qs[:lps])
         line = {
             "metric": "decode_us_per_step", "value": ms * 1e3, "unit": "us", "n_gpus": world, "steps": args.steps,
             "warmup": max(3, args.warmup), "ms_per_step": ms, "higher_is_better": False, "scaling": "weak",
@@ -330,7 +352,7 @@ def main():
             "frac_of_8tbs": bytes_per_step / (ms * 1e-3) / 8e12,
             "algorithmic_bytes_per_step": bytes_per_step,
             "pages_factorized_per_s": comp["pages_per_s"], "page_svds_timed": comp["n_page_svds"],
-            "roofline": {"bound": "hbm", "kernel": "decode_tc_kernel<%d>" % rank,
+            "roofline": {"bound": "hbm", "kernel": "decode_tc_kernel<P=%d, rank tiles=%d>" % (w.get("page", 64), (rank + 7) // 8),
                          "achieved": achieved, "peak": peak, "unit": "GB/s", "frac": achieved / peak,
                          "peak_source": peak_src,
                          "traffic": bytes_per_launch * NCU_TRAFFIC_PER_ALGORITHMIC_BYTE,
@@ -338,7 +360,7 @@ def main():
                                            "scaled by algorithmic bytes", "launch_us": launch_ms * 1e3,
                          "algorithmic_bytes_per_launch": bytes_per_launch},
             "e2e": {"value": e2e_ms * 1e3, "unit": "us", "h2d_bytes_per_step": qbytes, "d2h_bytes_per_step": qbytes},
-            "gpu_launches": L * args.steps, "clocks": clocks,
+            "gpu_launches": lps * args.steps, "clocks": clocks,
         }
         if not args.no_cpu_baseline and world == 1:
             o = oracle_sample(w, rank, 3)

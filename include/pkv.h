@@ -80,12 +80,23 @@ typedef struct pkv_config {
     int32_t decode_variant;     /* 0 = tensor-core pipeline kernel (the product path); 1 = scalar fp32 kernel that
                                    evaluates the same equations one unit at a time, kept as a debugging reference */
     int32_t decode_overlap;     /* pkv_decode_attention is launched with programmatic stream serialization, so its
-                                   CTAs start as SMs free up.  0 (default): the kernel still waits for the preceding
-                                   kernel on the stream to finish before it reads the cache or q.  1: the caller
-                                   promises that the kernel enqueued just before each pkv_decode_attention call
-                                   writes neither this cache's pools nor q (typical: the previous layer's decode
-                                   with queries prepared in advance); the kernel then streams pages at once and
-                                   waits only before touching its shared workspace and `out`. */
+                                   CTAs start as SMs free up.
+                                   0 (default): the kernel waits for the preceding kernel on the stream to finish
+                                      before it reads the cache or q.
+                                   1: the caller promises that the kernel enqueued just before each
+                                      pkv_decode_attention call writes neither this cache's pools nor q (typical:
+                                      the previous layer's decode with queries prepared in advance).  The kernel
+                                      streams pages at once and waits for the preceding kernel only before it
+                                      touches its shared workspace and `out`; launches complete in order.
+                                   2: the same promise for ALL decode launches that may be in flight, and `out`
+                                      buffers of consecutive calls must be distinct (or hold the same values).
+                                      Launches never wait for one another and may complete out of order; the
+                                      library rotates the split-K scratch over 16 sets and makes every 15th
+                                      launch an ordinary one, which starts only after all earlier work on the
+                                      stream has finished.  Not capturable into a CUDA graph (the call returns
+                                      PKV_ERR_UNSUPPORTED while the stream is capturing).
+                                   Work enqueued after a decode call by any other means (another kernel, a copy)
+                                   still starts only after that call has completed, in every mode. */
 } pkv_config;
 
 typedef struct pkv_sizes {
@@ -238,6 +249,15 @@ pkv_status pkv_get_page_table(const pkv_cache *c, int32_t seq, int32_t layer, in
  */
 pkv_status pkv_get_decode_plan(const pkv_cache *c, int32_t layer, int32_t *n_used_ctas, int32_t *cta_starts,
                                int32_t *n_segs, int32_t *seg_parts);
+
+/*
+ * Debugging aid.  When the environment variable PKV_DECODE_TRACE=1 is set at pkv_init_cache() time, every
+ * CTA of a decode launch records eight 64-bit time stamps in the workspace: [0] globaltimer (ns) at entry,
+ * [1] at exit, then SM clock counts: [2] entry, [3] first copy issued, [4] first unit's data arrived,
+ * [5] last unit of the CTA consumed, [6] exit, [7] units processed.  This call synchronises `stream` and
+ * copies the stamps of the most recent launch to out [host, n_ctas * 8 values].
+ */
+pkv_status pkv_get_decode_trace(pkv_cache *c, int64_t *out, int32_t n_ctas, void *stream);
 
 /* Counters; synchronises `stream` to read the device status words. */
 pkv_status pkv_get_stats(pkv_cache *c, pkv_stats *out, void *stream);

@@ -5,6 +5,7 @@
 #include <cmath>
 #include <cstdarg>
 #include <cstdio>
+#include <cstdlib>
 #include <cstring>
 #include <new>
 #include <string>
@@ -67,6 +68,7 @@ struct pkv_cache {
     MetaLayout ml;
     WorkspaceLayout wl;
     bool dry = false;
+    bool trace = false;                // PKV_DECODE_TRACE=1: CTAs write time stamps into the workspace
     unsigned char *dense_pool = nullptr, *factor_pool = nullptr, *meta = nullptr, *workspace = nullptr;
     FreeList dense_free, factor_free;
     std::vector<SeqLayer> sl;          // [max_seqs * n_layers]
@@ -77,6 +79,7 @@ struct pkv_cache {
     std::string err;
     int64_t pages_compressed = 0;
     int64_t last_decode_bytes = 0, last_decode_units = 0;
+    uint64_t decode_seq = 0;           // decode launches so far (decode_overlap = 2: picks the scratch buffer)
 
     SeqLayer &at(int seq, int layer) { return sl[(size_t)seq * cfg.n_layers + layer]; }
     const SeqLayer &at(int seq, int layer) const { return sl[(size_t)seq * cfg.n_layers + layer]; }
@@ -121,7 +124,7 @@ pkv_status validate(const pkv_config *cfg, const char **why) {
     }
     if (cfg->softmax_scale < 0.f || cfg->jacobi_max_sweeps < 0 || cfg->jacobi_tol < 0.f || cfg->n_ctas < 0 ||
         cfg->decode_variant < 0 || cfg->decode_variant > 1 ||
-        cfg->decode_overlap < 0 || cfg->decode_overlap > 1) {
+        cfg->decode_overlap < 0 || cfg->decode_overlap > 2) {
         *why = "negative scale / sweep cap / tolerance / n_ctas, or unknown decode_variant"; return PKV_ERR_INVALID_ARG;
     }
     if (cfg->n_dense_slots > INT32_MAX || cfg->n_factor_slots > INT32_MAX) {
@@ -189,9 +192,12 @@ void derive(const pkv_config &cfg, int n_ctas, Geometry &g, MetaLayout &ml, Work
 
     wl.n_partials = (long long)n_ctas + (long long)cfg.max_seqs * cfg.n_kv_heads;
     long long w = 0;
-    wl.partials = w; w = align_up(w + wl.n_partials * kPartialFloats * 4, 256);
+    wl.partials_stride = align_up(wl.n_partials * kPartialFloats * 4, 256);
+    wl.partials = w; w += wl.partials_stride * kDecodeBuffers;
     wl.worklist = w; w = align_up(w + (long long)sizeof(int2) * kCompressChunk, 256);
-    wl.tickets = w;  w = align_up(w + 4LL * cfg.max_seqs * cfg.n_kv_heads, 256);
+    wl.tickets_stride = align_up(4LL * cfg.max_seqs * cfg.n_kv_heads, 256);
+    wl.tickets = w;  w += wl.tickets_stride * kDecodeBuffers;
+    wl.trace = w;    w = align_up(w + 64LL * n_ctas, 256);
     wl.total = w;
 }
 
@@ -424,6 +430,7 @@ pkv_status pkv_init_cache(const pkv_config *cfg, void *dense_pool, void *factor_
     if (!c) return PKV_ERR_INVALID_ARG;
     c->cfg = *cfg;
     c->dry = dry;
+    { const char *t = getenv("PKV_DECODE_TRACE"); c->trace = t && t[0] == '1'; }
     // default grid: one CTA per SM when consecutive launches overlap (two launches share each SM),
     // otherwise two CTAs per SM
     int n_ctas = cfg->n_ctas > 0 ? cfg->n_ctas : default_ctas(dry) * (cfg->decode_overlap ? 1 : 2);
@@ -641,12 +648,28 @@ pkv_status pkv_decode_attention(pkv_cache *c, int32_t layer, int32_t n_seqs, con
     a.plan = c->meta + c->ml.plans + c->ml.plan_stride * layer;
     a.plan_cta = c->ml.plan_cta; a.plan_entry = c->ml.plan_entry; a.plan_seg = c->ml.plan_seg;
     a.q = q; a.out = out; a.out_f32 = out_f32;
-    a.partials = (float *)(c->workspace + c->wl.partials);
-    a.tickets = (int *)(c->workspace + c->wl.tickets);
+    // decode_overlap = 2: launches never wait for one another, so launches in flight must not share split-K
+    // scratch.  The scratch rotates over kDecodeBuffers sets and every (kDecodeBuffers-1)-th launch is a plain
+    // one (no programmatic serialization: it starts after all earlier work on the stream has finished), so
+    // between two users of a set the stream has always drained once.
+    int buf = 0;
+    a.plain_launch = 0;
+    if (c->cfg.decode_overlap == 2 && c->cfg.decode_variant == 0) {
+        cudaStreamCaptureStatus cap = cudaStreamCaptureStatusNone;
+        PKV_CUDA(c, cudaStreamIsCapturing(st, &cap));
+        if (cap != cudaStreamCaptureStatusNone)
+            return fail(c, PKV_ERR_UNSUPPORTED, "decode_overlap = 2 cannot be captured into a CUDA graph (use 0 or 1)");
+        buf = (int)(c->decode_seq % kDecodeBuffers);
+        a.plain_launch = (c->decode_seq % (kDecodeBuffers - 1)) == 0;
+        c->decode_seq++;
+    }
+    a.partials = (float *)(c->workspace + c->wl.partials + c->wl.partials_stride * buf);
+    a.tickets = (int *)(c->workspace + c->wl.tickets + c->wl.tickets_stride * buf);
     a.status = (int *)(c->meta + c->ml.status);
     a.layer = layer;
     a.variant = c->cfg.decode_variant;
     a.overlap = c->cfg.decode_overlap;
+    a.trace = c->trace ? (long long *)(c->workspace + c->wl.trace) : nullptr;
     PKV_CUDA(c, launch_decode(a, pc.n_segs, st));
     return PKV_OK;
 }
@@ -676,10 +699,12 @@ pkv_status pkv_decode_attention_static_scratch(pkv_cache *c, int32_t layer, int3
     a.plan_cta = c->ml.plan_cta; a.plan_entry = c->ml.plan_entry; a.plan_seg = c->ml.plan_seg;
     a.q = q; a.out = out; a.out_f32 = out_f32;
     a.partials = nullptr; a.tickets = nullptr;            // set by the launcher from the static scratch
+    a.plain_launch = 0;
     a.status = (int *)(c->meta + c->ml.status);
     a.layer = layer;
     a.variant = c->cfg.decode_variant;
     a.overlap = c->cfg.decode_overlap;
+    a.trace = nullptr;
     const char *why = "";
     cudaError_t e = launch_decode_static_scratch(a, c->plans[layer].n_segs, st, &why);
     if (e == cudaErrorInvalidValue && why[0])
@@ -743,6 +768,14 @@ pkv_status pkv_get_decode_plan(const pkv_cache *c, int32_t layer, int32_t *n_use
         }
     if (seg_parts)
         for (int s = 0; s < pc.n_segs; ++s) { seg_parts[2 * s] = pc.segs[s].cta_first; seg_parts[2 * s + 1] = pc.segs[s].n_parts; }
+    return PKV_OK;
+}
+
+pkv_status pkv_get_decode_trace(pkv_cache *c, int64_t *out, int32_t n_ctas, void *stream) {
+    if (!c || !out || c->dry || n_ctas <= 0 || n_ctas > c->geo.n_ctas) return PKV_ERR_INVALID_ARG;
+    if (!c->trace) return fail(c, PKV_ERR_INVALID_ARG, "tracing is off: set PKV_DECODE_TRACE=1 before pkv_init_cache");
+    PKV_CUDA(c, cudaStreamSynchronize((cudaStream_t)stream));
+    PKV_CUDA(c, cudaMemcpy(out, c->workspace + c->wl.trace, 64 * (size_t)n_ctas, cudaMemcpyDeviceToHost));
     return PKV_OK;
 }
 

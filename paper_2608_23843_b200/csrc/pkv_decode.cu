@@ -269,11 +269,19 @@ __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity) {
     }
     return true;
 }
+__device__ __forceinline__ int ld_acquire_smem(const volatile int *p) {
+    int v;
+    asm volatile("ld.acquire.cta.shared.b32 %0, [%1];" : "=r"(v) : "r"(smem_u32(const_cast<const int *>(p))) : "memory");
+    return v;
+}
+__device__ __forceinline__ void st_release_smem(volatile int *p, int v) {
+    asm volatile("st.release.cta.shared.b32 [%0], %1;" ::"r"(smem_u32(const_cast<int *>(p))), "r"(v) : "memory");
+}
 // Bounded spin until the producer has armed unit k.
 __device__ __forceinline__ bool wait_issued(volatile int *issued, int k) {
-    if (*issued > k) return true;
+    if (ld_acquire_smem(issued) > k) return true;
     const long long t0 = clock64();
-    while (*issued <= k) {
+    while (ld_acquire_smem(issued) <= k) {
         if (clock64() - t0 > 2000000000LL) return false;
         __nanosleep(20);
     }
@@ -569,8 +577,8 @@ __device__ __forceinline__ void flush_segment(const DecodeArgs &a, float *comb, 
         }
     }
     PKV_CONSUMER_BARRIER();
-    // partial states, tickets and (for a caller that reuses it) `out` may still be in use by the preceding launch
-    asm volatile("griddepcontrol.wait;" ::: "memory");
+    // overlap mode 1: partial states, tickets and `out` may still be in use by the preceding launch
+    if (a.overlap == 1) asm volatile("griddepcontrol.wait;" ::: "memory");
     const PlanSeg ps = reinterpret_cast<const PlanSeg *>(a.plan + a.plan_seg)[seg];
     float *part = a.partials + ((long long)blockIdx.x + seg) * kPartialFloats;
     for (int item = ctid; item < kItems; item += kThreads) {
@@ -607,11 +615,12 @@ __device__ __forceinline__ void flush_segment(const DecodeArgs &a, float *comb, 
             for (int item = ctid; item < a.geo.group * 32; item += kThreads) {
                 const int hq = item >> 5, d4 = (item & 31) * 4;
                 float Mg = kNegInf;
+#pragma unroll 8
                 for (int k = 0; k < ps.n_parts; ++k)
                     Mg = fmaxf(Mg, __ldcg(first + (long long)k * kPartialFloats + kMaxGroup * kHeadDim + hq));
                 float4 tot = make_float4(0.f, 0.f, 0.f, 0.f);
                 float Lg = 0.f;
-#pragma unroll 4
+#pragma unroll 8
                 for (int k = 0; k < ps.n_parts; ++k) {
                     const float *pk = first + (long long)k * kPartialFloats;
                     const float f = exp2f(__ldcg(pk + kMaxGroup * kHeadDim + hq) - Mg);
@@ -652,6 +661,13 @@ __global__ void __launch_bounds__(kDecodeThreads, 2) decode_tc_kernel(const __gr
     volatile int *last_flag = abort_flag + 2;
 
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+    long long *trace = a.trace ? a.trace + 8LL * blockIdx.x : nullptr;
+    if (trace && tid == 0) {
+        unsigned long long gt;
+        asm volatile("mov.u64 %0, %globaltimer;" : "=l"(gt));
+        trace[0] = (long long)gt;
+        trace[2] = clock64();
+    }
     if (tid == 0) {
         for (int s = 0; s < S; ++s) { mbar_init(smem_u32(full_bar + s), 1); mbar_init(smem_u32(empty_bar + s), 1); }
         *abort_flag = 0;
@@ -671,8 +687,8 @@ __global__ void __launch_bounds__(kDecodeThreads, 2) decode_tc_kernel(const __gr
     __syncthreads();
     // Programmatic dependent launch: let the next kernel on the stream begin as SMs free up.  Unless the caller
     // vouched that the preceding kernel writes neither this cache nor q (overlap mode), wait for it to finish
-    // before reading anything it may have produced; in overlap mode only the shared partial-state workspace
-    // needs that wait (taken in flush_segment).
+    // before reading anything it may have produced.  Mode 1 waits later, before the shared split-K scratch is
+    // touched (flush_segment); mode 2 never waits: the host rotates the scratch and drains the stream in time.
     if (!a.overlap) asm volatile("griddepcontrol.wait;" ::: "memory");
     asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
 
@@ -710,36 +726,36 @@ __global__ void __launch_bounds__(kDecodeThreads, 2) decode_tc_kernel(const __gr
                               (long long)cur.head * geo.dense_head_bytes + blk * C::kDB * kRowBytes;
                     }
                 }
+                // Lanes arm their own units, S at a time (one stage each); the counter of armed units is
+                // published after each group so that consumers can free the stages the next group needs.
                 const int n_here = min(32, u_end - u0);
-                for (int j = 0; j < n_here && ok; ++j) {
-                    const int kind_j = __shfl_sync(0xffffffffu, kind, j);
-                    const int rows_j = __shfl_sync(0xffffffffu, rows, j);
-                    const unsigned long long src_j = __shfl_sync(0xffffffffu, (unsigned long long)src, j);
-                    if (lane == 0) {
-                        const int s = k % S;
-                        if (k >= S && !mbar_wait(smem_u32(empty_bar + s), ((k / S) - 1) & 1)) ok = false;
-                        if (ok) {
-                            descs[s] = StageDesc{kind_j, rows_j, seg_local, 0};
+                for (int j0 = 0; j0 < n_here && ok; j0 += S) {
+                    const int cnt = min(S, n_here - j0);
+                    bool mine_ok = true;
+                    if (lane >= j0 && lane < j0 + cnt) {
+                        const int kj = k + lane, s = kj % S;
+                        if (kj >= S && !mbar_wait(smem_u32(empty_bar + s), ((kj / S) - 1) & 1)) mine_ok = false;
+                        if (mine_ok) {
+                            descs[s] = StageDesc{kind, rows, seg_local, 0};
                             const uint32_t bar = smem_u32(full_bar + s);
                             const uint32_t dst = smem_u32(stages + (size_t)s * stage_bytes);
-                            if (kind_j == kKindFactor) {
+                            if (kind == kKindFactor) {
                                 mbar_arrive_expect_tx(bar, blob_bytes);
-                                bulk_g2s(dst, (const void *)src_j, blob_bytes, bar);
-                            } else if (rows_j > 0) {
-                                mbar_arrive_expect_tx(bar, 2 * rows_j * kRowBytes);
-                                bulk_g2s(dst, (const void *)src_j, rows_j * kRowBytes, bar);
-                                bulk_g2s(dst + C::kDB * kRowBytes, (const unsigned char *)src_j + P * kRowBytes,
-                                         rows_j * kRowBytes, bar);
+                                bulk_g2s(dst, src, blob_bytes, bar);
+                            } else if (rows > 0) {
+                                mbar_arrive_expect_tx(bar, 2 * rows * kRowBytes);
+                                bulk_g2s(dst, src, rows * kRowBytes, bar);
+                                bulk_g2s(dst + C::kDB * kRowBytes, src + P * kRowBytes, rows * kRowBytes, bar);
                             } else {
                                 mbar_arrive(bar);
                             }
-                            __threadfence_block();
-                            *issued = k + 1;
                         }
                     }
-                    ok = __shfl_sync(0xffffffffu, (int)ok, 0) != 0;
-                    ++k;
+                    ok = __all_sync(0xffffffffu, mine_ok);
+                    if (ok && lane == 0) st_release_smem(issued, k + j0 + cnt);
+                    if (trace && lane == 0 && k + j0 == 0) trace[3] = clock64();
                 }
+                k += n_here;
             }
             if (last_run) break;
             cur.unit = 0;
@@ -754,8 +770,7 @@ __global__ void __launch_bounds__(kDecodeThreads, 2) decode_tc_kernel(const __gr
                 if (ok) {
                     descs[s] = StageDesc{kKindEnd, 0, rg.n_local_segs, 0};
                     mbar_arrive(smem_u32(full_bar + s));
-                    __threadfence_block();
-                    *issued = k + 1;
+                    st_release_smem(issued, k + 1);
                 }
             }
             ok = __shfl_sync(0xffffffffu, (int)ok, 0) != 0;
@@ -789,6 +804,8 @@ __global__ void __launch_bounds__(kDecodeThreads, 2) decode_tc_kernel(const __gr
                 if (lane == 0) { *abort_flag = 1; atomicAdd(a.status, 1); }
             }
             StageDesc dsc = ok ? descs[s] : StageDesc{kKindEnd, 0, rg.n_local_segs, 0};
+            if (trace && k == 0 && lane == 0) trace[4] = clock64();
+            if (trace && dsc.kind == kKindEnd && warp == 0 && lane == 0) { trace[5] = clock64(); trace[7] = k; }
             while (cur_seg < dsc.seg) {
                 flush_segment(a, comb, last_flag, st, rg.seg_first + cur_seg, warp, lane, tid, W);
                 ++cur_seg;
@@ -810,6 +827,12 @@ __global__ void __launch_bounds__(kDecodeThreads, 2) decode_tc_kernel(const __gr
             __syncwarp();
             if (lane == 0) mbar_arrive(smem_u32(empty_bar + s));
         }
+        if (trace && warp == 0 && lane == 0) {
+            unsigned long long gt;
+            asm volatile("mov.u64 %0, %globaltimer;" : "=l"(gt));
+            trace[1] = (long long)gt;
+            trace[6] = clock64();
+        }
     }
 }
 
@@ -829,7 +852,7 @@ cudaError_t launch_tc(const DecodeArgs &a, cudaStream_t st) {
     attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
     attr[0].val.programmaticStreamSerializationAllowed = 1;
     cfg.attrs = attr;
-    cfg.numAttrs = 1;
+    cfg.numAttrs = a.plain_launch ? 0 : 1;
     return cudaLaunchKernelEx(&cfg, decode_tc_kernel<P, NT>, a);
 }
 

@@ -12,11 +12,12 @@ constexpr int kHeadDim = 128;          // d (only supported value)
 constexpr int kMaxPage = 64;           // P is 16, 32 or 64
 constexpr int kRowBytes = kHeadDim * 2;
 constexpr int kMaxGroup = 8;           // query heads per KV head handled by the tensor-core kernel
-constexpr int kConsumerWarps = 4;      // decode kernel: warps that compute (two CTAs share an SM)
+constexpr int kConsumerWarps = 5;      // decode kernel: warps that compute (two CTAs share an SM; 6 warps x 168 regs x 2 fit the register file)
 constexpr int kDecodeThreads = (kConsumerWarps + 1) * 32;
 constexpr int kPartialFloats = kMaxGroup * (kHeadDim + 2);   // o[8][128], m[8], l[8]
 constexpr int kStatusWords = 8;        // [0] device timeouts, [1] page SVDs not converged, [2] slot indices out of range
 constexpr int kCompressChunk = 8192;   // work-list entries per compression launch
+constexpr int kDecodeBuffers = 16;     // decode_overlap = 2: rotating sets of split-K scratch (see pkv_decode_attention)
 constexpr int kSmemBudget = 227 * 1024;
 
 // Sizes derived from a validated pkv_config.  Plain data: passed to kernels by value.
@@ -59,10 +60,14 @@ struct MetaLayout {                    // byte offsets inside the caller's `meta
 };
 
 struct WorkspaceLayout {
-    long long partials;                // float [n_partials][kPartialFloats]
+    long long partials;                // float [kDecodeBuffers][n_partials][kPartialFloats]
     long long n_partials;
+    long long partials_stride;         // bytes of one buffer
+    long long tickets_stride;
+
     long long worklist;                // int2 [kCompressChunk]
     long long tickets;                 // int [max_seqs * n_kv_heads]
+    long long trace;                   // long long [n_ctas][8]
     long long total;
 };
 
@@ -80,10 +85,13 @@ struct DecodeArgs {
     float *out_f32;
     float *partials;
     int *tickets;                      // one per segment, zero between launches
+
     int *status;
     int layer;
     int variant;                       // 0 = tensor-core pipeline, 1 = scalar reference kernel
-    int overlap;                       // 1 = may stream KV before the preceding kernel has finished
+    int overlap;                       // 0 wait at entry, 1 wait before the first partial state is written, 2 never wait
+    int plain_launch;                  // launch without programmatic serialization (drains the stream first)
+    long long *trace;                  // NULL, or [n_ctas][8] time stamps written by each CTA (debugging)
 };
 
 // Launchers (defined in the .cu files); all return the launch error.

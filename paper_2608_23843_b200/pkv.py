@@ -28,7 +28,7 @@ EXPORTS = [
     "pkv_query_sizes", "pkv_init_cache", "pkv_append_kv", "pkv_compress_eligible_pages",
     "pkv_decode_attention", "pkv_decode_attention_host", "pkv_get_page_table", "pkv_get_stats",
     "pkv_free_seq", "pkv_destroy_cache", "pkv_last_error", "pkv_read_factors", "pkv_write_factors",
-    "pkv_read_dense", "pkv_get_decode_plan", "pkv_decode_attention_static_scratch",
+    "pkv_read_dense", "pkv_get_decode_plan", "pkv_decode_attention_static_scratch", "pkv_get_decode_trace",
 ]
 
 
@@ -92,6 +92,7 @@ def lib():
         L.pkv_write_factors.argtypes = [vp, i64, i32, vp, vp, vp, vp, vp]
         L.pkv_read_dense.argtypes = [vp, i64, i32, vp, vp, vp]
         L.pkv_get_decode_plan.argtypes = [vp, i32, ip, ip, ip, ip]
+        L.pkv_get_decode_trace.argtypes = [vp, ctypes.POINTER(ctypes.c_int64), i32, vp]
         for name in EXPORTS:
             if name != "pkv_last_error":
                 getattr(L, name).restype = ctypes.c_int32
@@ -204,6 +205,13 @@ def pkv_get_decode_plan(handle, layer, n_ctas, n_seqs, n_kv_heads):
         raise PkvError(st, "pkv_get_decode_plan")
     return ([tuple(starts[3 * j:3 * j + 3]) for j in range(n_used.value + 1)],
             [tuple(segs[2 * s:2 * s + 2]) for s in range(n_segs.value)])
+
+
+def pkv_get_decode_trace(handle, n_ctas, stream=None):
+    """Per-CTA time stamps of the last decode launch (needs PKV_DECODE_TRACE=1 at init): list of 8-tuples."""
+    buf = (ctypes.c_int64 * (8 * n_ctas))()
+    _check(handle, lib().pkv_get_decode_trace(handle, buf, n_ctas, _stream(stream)))
+    return [tuple(buf[8 * i:8 * i + 8]) for i in range(n_ctas)]
 
 
 def pkv_free_seq(handle, seq):

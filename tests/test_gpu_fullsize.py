@@ -30,9 +30,10 @@ ATT_TOL = 1e-2
 def stored_kv(cache, seq, layer, head):
     """K_all, V_all [T, d] of one (sequence, layer, KV head) exactly as the GPU stores them."""
     kinds, slots, T = cache.page_table(seq, layer)
+    P = cache.cfg.page_size
     Ks, Vs, factors = [], [], {}
     for p, (kd, slot) in enumerate(zip(kinds, slots)):
-        rows = min(64, T - p * 64)
+        rows = min(P, T - p * P)
         if kd == FACTOR:
             A_k, B_k, A_v, B_v = [f64(t) for t in cache.read_factors(slot, head)]
             factors[p] = (A_k, B_k, A_v, B_v)
@@ -62,12 +63,13 @@ def kernel_gate(cache, cfg, layer, order, q, out, samples):
 
 def oracle_slice(w, rank, seq, layer, head, T, device, steps_kv=None):
     """Single-KV-head oracle cache of one slice, regenerated with the bench's generator."""
-    k, v = synth.make_kv(bench.SEED, layer, seq, T, w["n_kv_heads"], 128, 64, device, w["outliers"])
+    P = w.get("page", 64)
+    k, v = synth.make_kv(bench.SEED, layer, seq, T, w["n_kv_heads"], 128, P, device, w["outliers"])
     k, v = f64(k[:, head:head + 1]), f64(v[:, head:head + 1])
     G = w["n_q_heads"] // w["n_kv_heads"]
-    n_pages = -(-T // 64) + 16
-    orc = OracleCache(OracleConfig(n_layers=1, n_kv_heads=1, n_q_heads=G, head_dim=128, page_size=64, rank_k=rank,
-                                   rank_v=rank, sink_tokens=w["sink"], recent_tokens=w["recent"], max_seqs=1,
+    n_pages = -(-T // P) + 16
+    orc = OracleCache(OracleConfig(n_layers=1, n_kv_heads=1, n_q_heads=G, head_dim=128, page_size=P, rank_k=rank,
+                                   rank_v=w.get("rank_v", rank), sink_tokens=w["sink"], recent_tokens=w["recent"], max_seqs=1,
                                    n_dense_slots=n_pages, n_factor_slots=n_pages))
     orc.append_kv(0, [0], [T], k, v)
     orc.compress_eligible_pages(0)
@@ -81,14 +83,15 @@ def factor_and_e2e_gates(cache, w, rank, seq, layer, head, T, q_row, out_row, de
     okinds, oslots, _ = orc.page_table(0, 0)
     assert sorted(gpu_factors) == [p for p, kd in enumerate(okinds) if kd == FACTOR]
     worst = 0.0
+    P, rank_v = w.get("page", 64), w.get("rank_v", rank)
     for p, (A_k, B_k, A_v, B_v) in gpu_factors.items():
         sig_k, sig_v = orc.sigma[oslots[p]]
-        for X, A, B, sig in ((k[p * 64:(p + 1) * 64, 0], A_k, B_k, sig_k[0]), (v[p * 64:(p + 1) * 64, 0], A_v, B_v, sig_v[0])):
+        for X, A, B, sig, r in ((k[p * P:(p + 1) * P, 0], A_k, B_k, sig_k[0], rank), (v[p * P:(p + 1) * P, 0], A_v, B_v, sig_v[0], rank_v)):
             err = np.linalg.norm(X - A @ B)
-            bound = 1.01 * float(np.sqrt((sig[rank:] ** 2).sum())) + 1e-3 * np.linalg.norm(X)
+            bound = 1.01 * float(np.sqrt((sig[r:] ** 2).sum())) + 1e-3 * np.linalg.norm(X)
             assert err <= bound, (seq, layer, head, p, err, bound)
             worst = max(worst, err / bound)
-            assert np.abs(A.T @ A - np.eye(rank)).max() <= 1e-2
+            assert np.abs(A.T @ A - np.eye(r)).max() <= 1e-2
     qd = f64(q_row)[None]
     ref = orc.decode_attention(0, [0], qd)[0]
     rounded = copy.deepcopy(orc)
@@ -118,7 +121,7 @@ def test_llama3_8b_layer_batch8_context_32k():
     """BASELINE config 1: 32q/8kv, batch 8, T=32768, r=24, 64 sink + 256 recent, shuffled pools."""
     w, device = bench.WORKLOADS["llama3_8b_32k_b8"], torch.device("cuda", 0)
     cfg, cache, lengths, comp = bench.build_workload(w, w["rank"], device)
-    assert comp["n_page_svds"] == 64896
+    assert comp["n_page_svds"] == 64896 * w["n_layers"]
     ids = list(range(w["batch"]))
     assert cache.page_table(3, 0)[0] == [0] + [1] * 507 + [0] * 4
     qs, outs = _decode_all(cache, w, ids, device)
@@ -148,6 +151,26 @@ def test_qwen3_32b_64_layers_context_128k():
     fw, e2e, floor = factor_and_e2e_gates(cache, w, w["rank"], 0, 31, 5, lengths[0], qs[31][0, 5 * G:6 * G],
                                           outs[31][0, 5 * G:6 * G], device)
     print("config 2: kernel gate %.2e, factor err/bound %.3f, e2e %.2e (floor %.2e), %.0f page SVDs/s"
+          % (worst, fw, e2e, floor, comp["pages_per_s"]))
+    _finish(cache)
+
+
+def test_paper_default_shape_qwen3_8b_16k():
+    """The paper's own setting: 36 layers, 32q/8kv, 16K context, P=32, ranks (16,14), one sink page and the
+    last completed page + incomplete page dense (the context here ends with a 17-token incomplete page)."""
+    w, device = bench.WORKLOADS["qwen3_8b_16k_paper_default"], torch.device("cuda", 0)
+    cfg, cache, lengths, comp = bench.build_workload(w, w["rank"], device)
+    assert cache.page_table(0, 35)[0] == [0] + [1] * 510 + [0, 0]
+    sz = cache.sizes
+    assert sz.factor_slot_bytes / sz.dense_slot_bytes == 0.5859375             # Eq. 3 at (16,14), P=32, d=128
+    qs, outs = _decode_all(cache, w, [0], device)
+    G = 4
+    worst = 0.0
+    for layer, head in ((0, 0), (17, 3), (35, 7)):
+        worst = max(worst, kernel_gate(cache, cfg, layer, [0], qs[layer], outs[layer], [(0, head)]))
+    fw, e2e, floor = factor_and_e2e_gates(cache, w, w["rank"], 0, 17, 3, lengths[0], qs[17][0, 3 * G:4 * G],
+                                          outs[17][0, 3 * G:4 * G], device)
+    print("paper default: kernel gate %.2e, factor err/bound %.3f, e2e %.2e (floor %.2e), %.0f page SVDs/s"
           % (worst, fw, e2e, floor, comp["pages_per_s"]))
     _finish(cache)
 

@@ -274,3 +274,32 @@ def test_other_page_sizes_and_ranks(P, rk, rv, G):
     assert st["device_timeouts"] == 0 and st["page_svds_not_converged"] == 0 and st["bad_slot_indices"] == 0
     print("P=%d r=(%d,%d) G=%d: e2e max %.2e (floor %.2e) kernel max %.2e recon/bound %.3f"
           % (P, rk, rv, G, max(g["e2e"]), max(g["floor"]), max(g["kernel"]), worst))
+
+
+@pytest.mark.parametrize("overlap", [1, 2])
+def test_overlapping_launches_give_the_serialised_result(overlap):
+    """Many back-to-back decode launches over three layers with decode_overlap 1 and 2 (launches overlap on
+    the GPU; mode 2 rotates the split-K scratch and drains the stream every 15 launches): every launch must
+    reproduce, bit for bit, what a cache with decode_overlap = 0 computes."""
+    H, G, L, lengths = 2, 4, 3, [2600, 700]
+    outs = {}
+    for mode in (0, overlap):
+        cfg = pkv.make_config(n_layers=L, n_kv_heads=H, n_q_heads=H * G, rank=24, sink_tokens=64, recent_tokens=256,
+                              max_seqs=2, max_pages_per_seq=48, n_dense_slots=400, n_factor_slots=300,
+                              decode_overlap=mode, n_ctas=148)
+        pair = Pair(cfg, seed=17, oracle=False)
+        for layer in range(L):
+            for s, T in enumerate(lengths):
+                k, v = gen_kv(17, layer, s, T, cfg)
+                pair.gpu.append_kv(layer, [s], [T], k.cuda(), v.cuda())
+        pair.gpu.compress_eligible_pages(-1)
+        qs = [synth.make_q(17, i % L, i, 2, H * G, 128).cuda() for i in range(50)]
+        res = [torch.empty_like(q) for q in qs]
+        torch.cuda.synchronize()
+        for i, q in enumerate(qs):
+            pair.gpu.decode_attention(i % L, [0, 1], q, res[i])
+        torch.cuda.synchronize()
+        assert pair.gpu.stats()["device_timeouts"] == 0
+        outs[mode] = [r.cpu() for r in res]
+    for a, b in zip(outs[0], outs[overlap]):
+        assert torch.equal(a, b)
