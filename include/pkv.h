@@ -79,6 +79,12 @@ typedef struct pkv_config {
     int32_t n_ctas;             /* decode grid size; 0 => SM count of the current device (148 in dry-run), doubled unless decode_overlap */
     int32_t decode_variant;     /* 0 = tensor-core pipeline kernel (the product path); 1 = scalar fp32 kernel that
                                    evaluates the same equations one unit at a time, kept as a debugging reference */
+    float   jacobi_energy_tol;  /* the sweeps also stop once a sweep raises the energy captured by the r largest
+                                   diagonal entries (= ||A^T X||_F^2 of the factors it would give) by less than this
+                                   fraction of the energy left outside them (= the squared reconstruction error):
+                                   the remaining rotations only polish eigenvectors inside near-degenerate clusters
+                                   and cannot improve A B measurably.  0 => default 1e-4; negative => off (iterate
+                                   until no rotation exceeds jacobi_tol) */
     int32_t decode_overlap;     /* pkv_decode_attention is launched with programmatic stream serialization, so its
                                    CTAs start as SMs free up.
                                    0 (default): the kernel waits for the preceding kernel on the stream to finish

@@ -176,6 +176,7 @@ void derive(const pkv_config &cfg, int n_ctas, Geometry &g, MetaLayout &ml, Work
     g.scale_log2e = scale * 1.4426950408889634f;
     g.jacobi_max_sweeps = cfg.jacobi_max_sweeps > 0 ? cfg.jacobi_max_sweeps : 16;
     g.jacobi_tol = cfg.jacobi_tol > 0.f ? cfg.jacobi_tol : 1e-5f;
+    g.jacobi_energy_tol = cfg.jacobi_energy_tol == 0.f ? 1e-4f : cfg.jacobi_energy_tol;
 
     long long off = 0;
     ml.page_table = off; off = align_up(off + 4LL * cfg.max_seqs * cfg.n_layers * cfg.max_pages_per_seq, 256);

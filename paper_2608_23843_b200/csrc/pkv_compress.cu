@@ -14,6 +14,12 @@ namespace {
 
 constexpr int kXs = kHeadDim + 2;         // padded row stride of X (bf16): 65 words, odd
 
+// Rotation pairs of every round for P = 16, 32, 64 (offsets 0, 15*8, 15*8 + 31*16), written once per device by
+// the host.  A pair is stored as (first, second); for P = 64 the orientation is chosen so that the 32 first
+// members of a round fall into 32 different shared-memory banks (index mod 32), and so do the second members.
+__constant__ uchar2 c_pairs[15 * 8 + 31 * 16 + 63 * 32];
+__host__ __device__ constexpr int pair_table_offset(int P) { return P == 16 ? 0 : (P == 32 ? 15 * 8 : 15 * 8 + 31 * 16); }
+
 template <int P>
 struct Shape {
     static constexpr int kThreads = 4 * P;              // 256 / 128 / 64
@@ -21,6 +27,10 @@ struct Shape {
     static constexpr int kGs = P + 1;                   // padded row stride of G and Q (floats)
     static constexpr int kPairsPerWarp = (P / 2) / kWarps;   // = 4 for every P
     static constexpr int kHalves = (P + 31) / 32;       // 32-row groups a warp walks in the column phase
+    // 2 x 2 block update of G: lanes run over the column pair b, a warp covers kRowPairsPerIter row pairs at once
+    static constexpr int kLanesPerRowPair = (P / 2) < 32 ? (P / 2) : 32;
+    static constexpr int kRowPairsPerIter = 32 / kLanesPerRowPair;
+    static constexpr int kBlockIters = (P / 2) / (kWarps * kRowPairsPerIter);
 };
 
 template <int P>
@@ -29,6 +39,7 @@ struct CompressSmem {
     float Q[P * (P + 1)];
     __nv_bfloat16 X[P * kXs];
     float2 cs[P / 2];
+    uchar2 pairs[(P - 1) * (P / 2)];   // this page size's rows of c_pairs (lanes index it divergently)
     float lam[P];
     int order[P];
     float red[Shape<P>::kWarps];
@@ -36,13 +47,12 @@ struct CompressSmem {
 
 // Round-robin tournament: in round rho (0..P-2) the P indices form P/2 disjoint
 // pairs; over P-1 rounds every pair meets exactly once.
-template <int P>
-__device__ __forceinline__ void pair_of(int rho, int k, int &p, int &q) {
-    constexpr int m = P - 1;
+inline void pair_of(int P, int rho, int k, int &p, int &q) {
+    const int m = P - 1;
     int a, b;
     if (k == 0) { a = m; b = rho; }
     else { a = rho + k; if (a >= m) a -= m; b = rho - k; if (b < 0) b += m; }
-    p = min(a, b); q = max(a, b);
+    p = a < b ? a : b; q = a < b ? b : a;
 }
 
 template <int P>
@@ -119,15 +129,33 @@ compress_kernel(Geometry geo, const unsigned char *dense_pool, unsigned char *fa
     for (int w = 0; w < kWarps; ++w) gmax = fmaxf(gmax, S.red[w]);
     const float floor_abs = 2e-7f * gmax;
     const float tol = geo.jacobi_tol;
+    // trace(G) = ||X||_F^2: with the energy captured by the r largest diagonal entries it gives the squared
+    // reconstruction error the current Q would yield (used by the early-stopping rule below)
+    float tr = tid < P ? S.G[tid * kGs + tid] : 0.f;
+    for (int o = 16; o; o >>= 1) tr += __shfl_xor_sync(0xffffffffu, tr, o);
+    __syncthreads();
+    if (lane == 0) S.red[warp] = tr;
+    __syncthreads();
+    float trace = 0.f;
+#pragma unroll
+    for (int w = 0; w < kWarps; ++w) trace += S.red[w];
+    float captured_prev = -1.f;
 
     // ---- cyclic Jacobi sweeps ----
+    // The P/2 rotations of a round act on disjoint index pairs, so G' = J^T G J splits into (P/2)^2 independent
+    // 2 x 2 blocks: block (a, b) = rows of pair a, columns of pair b, becomes J_a^T . block . J_b.  One thread
+    // owns a block, reads and writes only its four entries, and G passes through shared memory once per round.
+    // Blocks below the diagonal are computed as the transpose of their mirror image (G stays bitwise symmetric).
+    for (int i = tid; i < (P - 1) * (P / 2); i += kThreads) S.pairs[i] = c_pairs[pair_table_offset(P) + i];
+    __syncthreads();
+    const uchar2 *pairs = S.pairs;
     bool converged = false;
     for (int sweep = 0; sweep < geo.jacobi_max_sweeps && !converged; ++sweep) {
         int rotated = 0;
         for (int rho = 0; rho < P - 1; ++rho) {
+            const uchar2 *pr = pairs + rho * (P / 2);
             if (tid < P / 2) {
-                int p, q;
-                pair_of<P>(rho, tid, p, q);
+                const int p = pr[tid].x, q = pr[tid].y;
                 const float gpp = S.G[p * kGs + p], gqq = S.G[q * kGs + q], gpq = S.G[p * kGs + q];
                 float c = 1.f, s = 0.f;
                 if (fabsf(gpq) > fmaxf(tol * sqrtf(fabsf(gpp * gqq)), floor_abs)) {
@@ -140,22 +168,44 @@ compress_kernel(Geometry geo, const unsigned char *dense_pool, unsigned char *fa
                 S.cs[tid] = make_float2(c, s);
             }
             __syncthreads();
-            // columns p, q of G and Q:  x_p' = c x_p - s x_q,  x_q' = s x_p + c x_q
+            {
+                const int bb = lane % Sh::kLanesPerRowPair;
+                const uchar2 pb = pr[bb];
+                const float2 cb = S.cs[bb];
+#pragma unroll
+                for (int it = 0; it < Sh::kBlockIters; ++it) {
+                    const int aa = warp * Sh::kRowPairsPerIter + lane / Sh::kLanesPerRowPair +
+                                   it * (kWarps * Sh::kRowPairsPerIter);
+                    const uchar2 pa = pr[aa];
+                    const float2 ca = S.cs[aa];
+                    if (ca.y == 0.f && cb.y == 0.f) continue;
+                    float x00 = S.G[pa.x * kGs + pb.x], x01 = S.G[pa.x * kGs + pb.y];
+                    float x10 = S.G[pa.y * kGs + pb.x], x11 = S.G[pa.y * kGs + pb.y];
+                    const bool lower = aa > bb;
+                    const float cl = lower ? cb.x : ca.x, sl = lower ? cb.y : ca.y;     // applied first
+                    const float cr = lower ? ca.x : cb.x, sr = lower ? ca.y : cb.y;     // applied second
+                    if (lower) { const float t = x01; x01 = x10; x10 = t; }
+                    const float y00 = cl * x00 - sl * x10, y01 = cl * x01 - sl * x11;
+                    const float y10 = sl * x00 + cl * x10, y11 = sl * x01 + cl * x11;
+                    float z00 = cr * y00 - sr * y01, z01 = sr * y00 + cr * y01;
+                    float z10 = cr * y10 - sr * y11, z11 = sr * y10 + cr * y11;
+                    if (lower) { const float t = z01; z01 = z10; z10 = t; }
+                    S.G[pa.x * kGs + pb.x] = z00; S.G[pa.x * kGs + pb.y] = z01;
+                    S.G[pa.y * kGs + pb.x] = z10; S.G[pa.y * kGs + pb.y] = z11;
+                }
+            }
+            // columns p, q of Q:  x_p' = c x_p - s x_q,  x_q' = s x_p + c x_q
 #pragma unroll
             for (int kk = 0; kk < Sh::kPairsPerWarp; ++kk) {
                 const int k = warp + kk * kWarps;
-                int p, q;
-                pair_of<P>(rho, k, p, q);
                 const float2 cs = S.cs[k];
                 if (cs.y != 0.f) {
+                    const int p = pr[k].x, q = pr[k].y;
 #pragma unroll
                     for (int half = 0; half < Sh::kHalves; ++half) {
                         const int i = lane + 32 * half;
                         if (i < P) {
-                            float gp = S.G[i * kGs + p], gq = S.G[i * kGs + q];
-                            S.G[i * kGs + p] = cs.x * gp - cs.y * gq;
-                            S.G[i * kGs + q] = cs.y * gp + cs.x * gq;
-                            float qp = S.Q[i * kGs + p], qq = S.Q[i * kGs + q];
+                            const float qp = S.Q[i * kGs + p], qq = S.Q[i * kGs + q];
                             S.Q[i * kGs + p] = cs.x * qp - cs.y * qq;
                             S.Q[i * kGs + q] = cs.y * qp + cs.x * qq;
                         }
@@ -163,28 +213,33 @@ compress_kernel(Geometry geo, const unsigned char *dense_pool, unsigned char *fa
                 }
             }
             __syncthreads();
-            // rows p, q of G
-#pragma unroll
-            for (int kk = 0; kk < Sh::kPairsPerWarp; ++kk) {
-                const int k = warp + kk * kWarps;
-                int p, q;
-                pair_of<P>(rho, k, p, q);
-                const float2 cs = S.cs[k];
-                if (cs.y != 0.f) {
-#pragma unroll
-                    for (int half = 0; half < Sh::kHalves; ++half) {
-                        const int j = lane + 32 * half;
-                        if (j < P) {
-                            float gp = S.G[p * kGs + j], gq = S.G[q * kGs + j];
-                            S.G[p * kGs + j] = cs.x * gp - cs.y * gq;
-                            S.G[q * kGs + j] = cs.y * gp + cs.x * gq;
-                        }
-                    }
-                }
-            }
-            __syncthreads();
         }
         converged = !__syncthreads_or(rotated);
+        if (!converged && geo.jacobi_energy_tol >= 0.f) {
+            // energy captured by the r largest diagonal entries after this sweep
+            if (tid < P) S.lam[tid] = S.G[tid * kGs + tid];
+            __syncthreads();
+            float mine = 0.f;
+            if (tid < P) {
+                const float li = S.lam[tid];
+                int r = 0;
+                for (int j = 0; j < P; ++j) {
+                    const float lj = S.lam[j];
+                    r += (lj > li) || (lj == li && j < tid);
+                }
+                if (r < rank) mine = li;
+            }
+            for (int o = 16; o; o >>= 1) mine += __shfl_xor_sync(0xffffffffu, mine, o);
+            if (lane == 0) S.red[warp] = mine;
+            __syncthreads();
+            float captured = 0.f;
+#pragma unroll
+            for (int w = 0; w < kWarps; ++w) captured += S.red[w];
+            __syncthreads();
+            if (captured_prev >= 0.f && captured - captured_prev <= geo.jacobi_energy_tol * fmaxf(trace - captured, 0.f))
+                converged = true;
+            captured_prev = captured;
+        }
     }
     if (!converged && tid == 0) atomicAdd(&status[1], 1);
 
@@ -226,10 +281,48 @@ compress_kernel(Geometry geo, const unsigned char *dense_pool, unsigned char *fa
     }
 }
 
+// Round-robin pairs of every round.  For P = 64 each pair is oriented (first, second) so that the first members
+// of a round have distinct indices mod 32 (and hence so do the second members): mark x first and its partner y
+// second; y ^ 32 shares y's bank, so it must be a first member; continue from there until the cycle closes.
+void fill_pair_table(int P, uchar2 *out) {
+    const int B = P / 2;
+    for (int rho = 0; rho < P - 1; ++rho) {
+        int partner[kMaxPage], role[kMaxPage];      // role: 0 unknown, 1 first, 2 second
+        for (int k = 0; k < B; ++k) {
+            int p, q;
+            pair_of(P, rho, k, p, q);
+            partner[p] = q; partner[q] = p;
+            role[p] = P == 64 ? 0 : 1; role[q] = P == 64 ? 0 : 2;
+        }
+        if (P == 64) {
+            for (int start = 0; start < P; ++start) {
+                int x = start;
+                while (role[x] == 0) {
+                    role[x] = 1;
+                    const int y = partner[x];
+                    role[y] = 2;
+                    x = y ^ 32;
+                }
+            }
+        }
+        int k = 0;
+        for (int x = 0; x < P; ++x)
+            if (role[x] == 1) out[rho * B + k++] = make_uchar2((unsigned char)x, (unsigned char)partner[x]);
+    }
+}
+
+cudaError_t upload_pair_tables() {
+    static uchar2 host[15 * 8 + 31 * 16 + 63 * 32];
+    fill_pair_table(16, host + pair_table_offset(16));
+    fill_pair_table(32, host + pair_table_offset(32));
+    fill_pair_table(64, host + pair_table_offset(64));
+    return cudaMemcpyToSymbol(c_pairs, host, sizeof host);
+}
+
 template <int P>
 cudaError_t launch_p(const Geometry &geo, const unsigned char *dense_pool, unsigned char *factor_pool,
                      const int2 *worklist, int n_entries, int *status, cudaStream_t st) {
-    static bool configured[64] = {};         // the attribute is per device
+    static bool configured[64] = {};         // attribute and constant table are per device
     int dev = 0;
     cudaError_t e = cudaGetDevice(&dev);
     if (e != cudaSuccess) return e;
@@ -237,6 +330,7 @@ cudaError_t launch_p(const Geometry &geo, const unsigned char *dense_pool, unsig
         e = cudaFuncSetAttribute(compress_kernel<P>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                  (int)sizeof(CompressSmem<P>));
         if (e != cudaSuccess) return e;
+        if ((e = upload_pair_tables()) != cudaSuccess) return e;
         if (dev >= 0 && dev < 64) configured[dev] = true;
     }
     const unsigned grid = (unsigned)n_entries * geo.n_kv_heads * 2;

@@ -39,6 +39,7 @@ struct Geometry {
     float scale_log2e;                 // softmax_scale * log2(e)
     int jacobi_max_sweeps;
     float jacobi_tol;
+    float jacobi_energy_tol;           // < 0: off
 };
 
 // Device-resident decode plan of one layer (written by the host when the batch
