@@ -102,7 +102,10 @@ typedef struct pkv_config {
                                       stream has finished.  Not capturable into a CUDA graph (the call returns
                                       PKV_ERR_UNSUPPORTED while the stream is capturing).
                                    Work enqueued after a decode call by any other means (another kernel, a copy)
-                                   still starts only after that call has completed, in every mode. */
+                                   still starts only after that call has completed, in every mode, and a decode
+                                   call that follows a pkv_append_kv or pkv_compress_eligible_pages call on this
+                                   cache always waits for it: the promise concerns other writers (of q, or of the
+                                   pools through their raw pointers) only. */
 } pkv_config;
 
 typedef struct pkv_sizes {

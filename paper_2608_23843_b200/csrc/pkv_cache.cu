@@ -80,6 +80,7 @@ struct pkv_cache {
     int64_t pages_compressed = 0;
     int64_t last_decode_bytes = 0, last_decode_units = 0;
     uint64_t decode_seq = 0;           // decode launches so far (decode_overlap = 2: picks the scratch buffer)
+    bool cache_written = true;         // an append or compression kernel was enqueued since the last decode launch
 
     SeqLayer &at(int seq, int layer) { return sl[(size_t)seq * cfg.n_layers + layer]; }
     const SeqLayer &at(int seq, int layer) const { return sl[(size_t)seq * cfg.n_layers + layer]; }
@@ -534,6 +535,7 @@ pkv_status pkv_append_kv(pkv_cache *c, int32_t layer, int32_t n_seqs, const int3
     AppendDesc *ddesc = (AppendDesc *)(c->meta + c->ml.append_desc);
     if ((r = upload(c, ddesc, desc.data(), sizeof(AppendDesc) * desc.size(), st)) != PKV_OK) return r;
     if ((r = stager_flush(c, st)) != PKV_OK) return r;
+    c->cache_written = true;
     PKV_CUDA(c, launch_append(c->geo, c->dense_pool, (const int *)(c->meta + c->ml.page_table),
                               (int *)(c->meta + c->ml.n_tokens), ddesc, (int)desc.size(), n_tok, layer, k, v,
                               (int *)(c->meta + c->ml.status), st));
@@ -558,6 +560,7 @@ pkv_status pkv_compress_eligible_pages(pkv_cache *c, int32_t layer, int64_t *n_p
         pkv_status rr = upload(c, dwl, work.data(), sizeof(int2) * work.size(), st);
         if (rr != PKV_OK) return rr;
         if ((rr = stager_flush(c, st)) != PKV_OK) return rr;
+        c->cache_written = true;
         PKV_CUDA(c, launch_compress(g, c->dense_pool, c->factor_pool, dwl, (int)work.size(),
                                     (int *)(c->meta + c->ml.status), st));
         work.clear();
@@ -654,14 +657,17 @@ pkv_status pkv_decode_attention(pkv_cache *c, int32_t layer, int32_t n_seqs, con
     // one (no programmatic serialization: it starts after all earlier work on the stream has finished), so
     // between two users of a set the stream has always drained once.
     int buf = 0;
-    a.plain_launch = 0;
+    // whatever the overlap mode, a decode that follows this library's own append / compression kernels is
+    // launched the ordinary way, after everything before it on the stream has finished
+    a.plain_launch = c->cache_written ? 1 : 0;
+    c->cache_written = false;
     if (c->cfg.decode_overlap == 2 && c->cfg.decode_variant == 0) {
         cudaStreamCaptureStatus cap = cudaStreamCaptureStatusNone;
         PKV_CUDA(c, cudaStreamIsCapturing(st, &cap));
         if (cap != cudaStreamCaptureStatusNone)
             return fail(c, PKV_ERR_UNSUPPORTED, "decode_overlap = 2 cannot be captured into a CUDA graph (use 0 or 1)");
         buf = (int)(c->decode_seq % kDecodeBuffers);
-        a.plain_launch = (c->decode_seq % (kDecodeBuffers - 1)) == 0;
+        if ((c->decode_seq % (kDecodeBuffers - 1)) == 0) a.plain_launch = 1;
         c->decode_seq++;
     }
     a.partials = (float *)(c->workspace + c->wl.partials + c->wl.partials_stride * buf);
@@ -700,7 +706,8 @@ pkv_status pkv_decode_attention_static_scratch(pkv_cache *c, int32_t layer, int3
     a.plan_cta = c->ml.plan_cta; a.plan_entry = c->ml.plan_entry; a.plan_seg = c->ml.plan_seg;
     a.q = q; a.out = out; a.out_f32 = out_f32;
     a.partials = nullptr; a.tickets = nullptr;            // set by the launcher from the static scratch
-    a.plain_launch = 0;
+    a.plain_launch = 0;                                   // the launcher's memset already orders it after earlier work
+    c->cache_written = false;
     a.status = (int *)(c->meta + c->ml.status);
     a.layer = layer;
     a.variant = c->cfg.decode_variant;

@@ -303,3 +303,31 @@ def test_overlapping_launches_give_the_serialised_result(overlap):
         outs[mode] = [r.cpu() for r in res]
     for a, b in zip(outs[0], outs[overlap]):
         assert torch.equal(a, b)
+
+
+@pytest.mark.parametrize("overlap", [1, 2])
+def test_overlap_modes_stay_correct_when_appends_and_compressions_are_interleaved(overlap):
+    """append -> attend -> compress per step on one stream: a decode that follows the library's own writes
+    is launched the ordinary way in every overlap mode, so the results equal those of decode_overlap = 0."""
+    H, G, T0, steps = 2, 4, 900, 70
+    outs = {}
+    for mode in (0, overlap):
+        cfg = pkv.make_config(n_layers=1, n_kv_heads=H, n_q_heads=H * G, rank=16, sink_tokens=64, recent_tokens=128,
+                              max_seqs=1, max_pages_per_seq=24, n_dense_slots=24, n_factor_slots=24,
+                              decode_overlap=mode, n_ctas=148)
+        pair = Pair(cfg, seed=19, oracle=False)
+        k, v = gen_kv(19, 0, 0, T0 + steps, cfg)
+        kd, vd = k.cuda(), v.cuda()
+        pair.gpu.append_kv(0, [0], [T0], kd[:T0], vd[:T0])
+        pair.gpu.compress_eligible_pages(0)
+        res = []
+        for t in range(steps):
+            pair.gpu.append_kv(0, [0], [1], kd[T0 + t:T0 + t + 1], vd[T0 + t:T0 + t + 1])
+            q = synth.make_q(19, 0, t, 1, H * G, 128).cuda()
+            res.append(pair.gpu.decode_attention(0, [0], q))
+            res.append(pair.gpu.decode_attention(0, [0], q))      # a second launch right behind the first
+            pair.gpu.compress_eligible_pages(0)
+        torch.cuda.synchronize()
+        outs[mode] = [r.cpu() for r in res]
+    for a, b in zip(outs[0], outs[overlap]):
+        assert torch.equal(a, b)
