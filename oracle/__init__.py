@@ -12,6 +12,7 @@ attention   softmax attention: the plain definition (Eq. 1) and the page-wise
             factor form with online-softmax merge (Eq. 4, Eq. 5)
 cache       the hybrid paged cache state machine (Section 3.3: construction,
             mixed attention, incremental update)
+quant       INT4 quantization of the factors (Section 4.3)
 bf16        bf16 storage rounding of factors (integer arithmetic on bit patterns)
 accounting  storage-ratio and size formulas (Eq. 3, Section 1)
 

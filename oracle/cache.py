@@ -25,6 +25,7 @@ import numpy as np
 
 from . import attention as _att
 from . import bf16 as _bf16
+from . import quant as _quant
 from . import svd as _svd
 
 DENSE, FACTOR = 0, 1
@@ -45,6 +46,7 @@ class OracleConfig:
     n_dense_slots: int
     n_factor_slots: int
     softmax_scale: float = 0.0          # 0 => 1/sqrt(head_dim)  (Eq. 1)
+    factor_bits: int = 16               # 4 => factors are INT4-quantized when a page is converted (Section 4.3)
 
 
 class PoolExhausted(RuntimeError):
@@ -179,6 +181,11 @@ class OracleCache:
             sel = slice(i * H, (i + 1) * H)
             self.factor[fslot] = dict(A_k=A_k[sel].copy(), B_k=B_k[sel].copy(),
                                       A_v=A_v[sel].copy(), B_v=B_v[sel].copy())
+            if c.factor_bits == 4:
+                f = self.factor[fslot]
+                for h in range(H):
+                    f["A_k"][h], f["B_k"][h], f["A_v"][h], f["B_v"][h] = _quant.quantized_page_factors(
+                        f["A_k"][h], f["B_k"][h], f["A_v"][h], f["B_v"][h])
             self.sigma[fslot] = (s_k[sel].copy(), s_v[sel].copy())
             dslot = sl.slots[p]
             del self.dense[dslot]
