@@ -99,7 +99,7 @@ class ClockSampler:
                 "reasons": reasons, "samples": len(sm)}
 
 
-def build_workload(w, rank, device, overlap=2, n_ctas=0):
+def build_workload(w, rank, device, overlap=2, n_ctas=0, factor_bits=16):
     """Allocate the cache, generate each (layer, sequence) on the GPU, append and compress layer by layer."""
     import torch
     from paper_2608_23843_b200 import pkv, synth
@@ -119,7 +119,7 @@ def build_workload(w, rank, device, overlap=2, n_ctas=0):
                           rank_v=w.get("rank_v", rank), page_size=P,
                           sink_tokens=w["sink"], recent_tokens=w["recent"], max_seqs=w["batch"],
                           max_pages_per_seq=max(pages), n_dense_slots=n_dense_slots, n_factor_slots=n_factor_slots,
-                          decode_overlap=overlap, n_ctas=n_ctas)
+                          decode_overlap=overlap, n_ctas=n_ctas, factor_bits=factor_bits)
     cache = pkv.Cache(cfg, device, synth.slot_permutation(SEED, n_dense_slots, 0).tolist(),
                       synth.slot_permutation(SEED, n_factor_slots, 1).tolist())
     ids = list(range(w["batch"]))
@@ -140,7 +140,7 @@ def build_workload(w, rank, device, overlap=2, n_ctas=0):
                                      svd_ms=svd_ms)
 
 
-def oracle_sample(w, rank, steps):
+def oracle_sample(w, rank, steps, factor_bits=16):
     """The fp64 oracle, as it stands, on one (layer 0, KV head 0) slice of sequence 0: page SVDs and
     one decode call for the G query heads of that KV head.  Returns seconds per decode and pages/s."""
     import torch
@@ -155,7 +155,7 @@ def oracle_sample(w, rank, steps):
     n_pages = -(-T // P)
     orc = OracleCache(OracleConfig(n_layers=1, n_kv_heads=1, n_q_heads=G, head_dim=128, page_size=P, rank_k=rank,
                                    rank_v=w.get("rank_v", rank), sink_tokens=w["sink"], recent_tokens=w["recent"], max_seqs=1,
-                                   n_dense_slots=n_pages, n_factor_slots=n_pages))
+                                   n_dense_slots=n_pages, n_factor_slots=n_pages, factor_bits=factor_bits))
     orc.append_kv(0, [0], [T], k, v)
     t0 = time.perf_counter()
     n = orc.compress_eligible_pages(0)
@@ -177,7 +177,7 @@ def run_reference(args, w, rank):
     rank0 = int(os.environ.get("RANK", "0")) == 0
     if not rank0:
         return
-    o = oracle_sample(w, rank, args.steps + args.warmup)
+    o = oracle_sample(w, rank, args.steps + args.warmup, args.factor_bits)
     us = o["decode_s"] * 1e6 * o["slices_per_step"]
     line = {"impl": "reference", "metric": "decode_us_per_step", "value": us, "unit": "us", "n_gpus": args.gpus,
             "steps": args.steps, "warmup": args.warmup, "ms_per_step": us / 1e3, "higher_is_better": False,
@@ -192,7 +192,7 @@ def run_reference(args, w, rank):
 def _config_dict(args, w, rank):
     return {"workload": args.workload, "n_layers": w["n_layers"], "layers_per_step": w.get("layers_per_step", w["n_layers"]), "n_q_heads": w["n_q_heads"],
             "n_kv_heads": w["n_kv_heads"], "head_dim": 128, "batch": w["batch"], "context": w["T"],
-            "page_size": w.get("page", 64), "rank": rank, "rank_v": w.get("rank_v", rank), "sink_tokens": w["sink"], "recent_tokens": w["recent"],
+            "page_size": w.get("page", 64), "rank": rank, "rank_v": w.get("rank_v", rank), "factor_bits": args.factor_bits, "sink_tokens": w["sink"], "recent_tokens": w["recent"],
             "l2": "inputs larger than L2 (no flush)" if args.workload != "tiny" else "L2-resident (latency only)",
             "overlap": ["0: each launch waits for the previous one",
                         "1: consecutive per-layer launches overlap (programmatic dependent launch) and complete in order",
@@ -227,6 +227,7 @@ def main():
                     help="decode_overlap mode of the cache: 0 = every launch waits for the previous one, 1 = launches "
                          "overlap but complete in order, 2 = launches never wait for one another (default)")
     ap.add_argument("--n-ctas", type=int, default=0, help="decode grid size (0 = library default)")
+    ap.add_argument("--factor-bits", type=int, default=16, choices=[4, 16], help="factor storage: bf16 or INT4 (paper, Section 4.3)")
     ap.add_argument("--graph", action="store_true",
                     help="replay one CUDA graph per step instead of launching every layer from the host (overlap 0 or 1)")
     args = ap.parse_args()
@@ -250,7 +251,7 @@ def main():
         dist.init_process_group("nccl", device_id=device)
     pkv.lib()                                             # fail loudly if the CUDA library is missing
 
-    cfg, cache, lengths, comp = build_workload(w, rank, device, args.overlap, args.n_ctas)
+    cfg, cache, lengths, comp = build_workload(w, rank, device, args.overlap, args.n_ctas, args.factor_bits)
     ids = list(range(w["batch"]))
     L, Hq = w["n_layers"], w["n_q_heads"]
     qs = [synth.make_q(SEED, layer, 0, w["batch"], Hq, 128, device) for layer in range(L)]
@@ -363,7 +364,7 @@ def main():
             "gpu_launches": lps * args.steps, "clocks": clocks,
         }
         if not args.no_cpu_baseline and world == 1:
-            o = oracle_sample(w, rank, 3)
+            o = oracle_sample(w, rank, 3, args.factor_bits)
             line["cpu_baseline"] = {"value": o["decode_s"] * 1e6 * o["slices_per_step"], "unit": "us",
                                     "cores": o["cores"], "kind": "oracle", "sample": o["sample"],
                                     "pages_per_s": o["pages_per_s"]}

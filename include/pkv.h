@@ -85,6 +85,12 @@ typedef struct pkv_config {
                                    the remaining rotations only polish eigenvectors inside near-degenerate clusters
                                    and cannot improve A B measurably.  0 => default 1e-4; negative => off (iterate
                                    until no rotation exceeds jacobi_tol) */
+    int32_t factor_bits;        /* 0 or 16: factors stored in bf16.  4: INT4 factors (Section 4.3): the singular
+                                   values are split evenly, A~ = A Sigma^(1/2), B~ = Sigma^(-1/2) B, and each matrix is
+                                   quantized symmetrically to 4 bits with one bf16 scale per column of A~_K, B~_K and
+                                   B~_V and per row (token) of A~_V; scale = max|x|/7, codes in [-7, 7].  Attention
+                                   reads bf16(code * scale).  pkv_read_factors returns those dequantised values;
+                                   pkv_write_factors is not available in this mode. */
     int32_t decode_overlap;     /* pkv_decode_attention is launched with programmatic stream serialization, so its
                                    CTAs start as SMs free up.
                                    0 (default): the kernel waits for the preceding kernel on the stream to finish
@@ -110,7 +116,9 @@ typedef struct pkv_config {
 
 typedef struct pkv_sizes {
     int64_t dense_slot_bytes;   /* H_kv * 2 * P * d * 2 */
-    int64_t factor_slot_bytes;  /* H_kv * 2 * (r_k + r_v) * (P + d) bytes; Eq. 3 is factor_slot_bytes / dense_slot_bytes */
+    int64_t factor_slot_bytes;  /* bf16 factors: H_kv * 2 * (r_k + r_v) * (P + d) bytes, so that Eq. 3 is
+                                   factor_slot_bytes / dense_slot_bytes; INT4 factors: H_kv * ((r_k + r_v)(P + d)/2
+                                   + 2 * (ceil8(r_k) + 2d + P)) bytes rounded up to 16 per KV head */
     int64_t dense_pool_bytes;   /* n_dense_slots * dense_slot_bytes */
     int64_t factor_pool_bytes;
     int64_t meta_bytes;         /* device page tables, token counts, decode plans, status words */

@@ -125,8 +125,9 @@ pkv_status validate(const pkv_config *cfg, const char **why) {
     }
     if (cfg->softmax_scale < 0.f || cfg->jacobi_max_sweeps < 0 || cfg->jacobi_tol < 0.f || cfg->n_ctas < 0 ||
         cfg->decode_variant < 0 || cfg->decode_variant > 1 ||
-        cfg->decode_overlap < 0 || cfg->decode_overlap > 2) {
-        *why = "negative scale / sweep cap / tolerance / n_ctas, or unknown decode_variant"; return PKV_ERR_INVALID_ARG;
+        cfg->decode_overlap < 0 || cfg->decode_overlap > 2 ||
+        (cfg->factor_bits != 0 && cfg->factor_bits != 4 && cfg->factor_bits != 16)) {
+        *why = "negative scale / sweep cap / tolerance / n_ctas, or unknown decode_variant / decode_overlap / factor_bits"; return PKV_ERR_INVALID_ARG;
     }
     if (cfg->n_dense_slots > INT32_MAX || cfg->n_factor_slots > INT32_MAX) {
         *why = "slot counts must fit in int32"; return PKV_ERR_INVALID_ARG;
@@ -158,7 +159,15 @@ void derive(const pkv_config &cfg, int n_ctas, Geometry &g, MetaLayout &ml, Work
     g.bk_off = g.ak_off + P * cfg.rank_k * 2;
     g.av_off = g.bk_off + cfg.rank_k * d * 2;
     g.bv_off = g.av_off + P * cfg.rank_v * 2;
-    g.blob_bytes = g.bv_off + cfg.rank_v * d * 2;
+    g.blob16_bytes = g.bv_off + cfg.rank_v * d * 2;
+    g.factor_bits = cfg.factor_bits == 4 ? 4 : 16;
+    g.codes_bytes = (int)align_up(g.blob16_bytes / 4, 16);
+    g.sak_off = 0;
+    g.sbk_off = g.sak_off + 2 * (int)align_up(cfg.rank_k, 8);
+    g.sav_off = g.sbk_off + 2 * d;
+    g.sbv_off = g.sav_off + 2 * P;
+    const int scales_bytes = g.sbv_off + 2 * d;
+    g.blob_bytes = g.factor_bits == 4 ? (int)align_up(g.codes_bytes + scales_bytes, 16) : g.blob16_bytes;
     g.dense_head_bytes = 2 * P * d * 2;
     g.dense_slot_bytes = (long long)cfg.n_kv_heads * g.dense_head_bytes;
     g.factor_slot_bytes = (long long)cfg.n_kv_heads * g.blob_bytes;
@@ -167,7 +176,9 @@ void derive(const pkv_config &cfg, int n_ctas, Geometry &g, MetaLayout &ml, Work
     g.block_tokens = (P >= 32 && g.rank_tiles >= 3) ? 32 : 16;
     g.blocks_per_page = P / g.block_tokens;
     const int overread = (8 * g.rank_tiles - cfg.rank_v) * kRowBytes;
-    g.stage_bytes = (int)align_up(std::max(g.blob_bytes + overread, g.block_tokens * 2 * kRowBytes), 128);
+    g.unpack_bytes = (int)align_up(g.blob16_bytes + overread, 16);
+    const int factor_stage = g.factor_bits == 4 ? g.unpack_bytes + (g.blob_bytes - g.codes_bytes) : g.unpack_bytes;
+    g.stage_bytes = (int)align_up(std::max(factor_stage, g.block_tokens * 2 * kRowBytes), 128);
     // two CTAs are resident per SM (consecutive launches overlap, or the grid holds two CTAs per SM),
     // so that one streams while the other is in its prologue or merging
     const int fixed = kConsumerWarps * kPartialFloats * 4 + 1024 + 1024;
@@ -846,6 +857,7 @@ pkv_status pkv_write_factors(pkv_cache *c, int64_t slot, int32_t head, const voi
     pkv_status r = slot_args(c, slot, c ? c->cfg.n_factor_slots : 0, head);
     if (r != PKV_OK) return r;
     if (!A_k || !B_k || !A_v || !B_v) return fail(c, PKV_ERR_INVALID_ARG, "input pointer is NULL");
+    if (c->geo.factor_bits == 4) return fail(c, PKV_ERR_UNSUPPORTED, "pkv_write_factors is not available with INT4 factors");
     unsigned char *blob = c->factor_pool + slot * c->geo.factor_slot_bytes + (int64_t)head * c->geo.blob_bytes;
     PKV_CUDA(c, launch_write_factors(c->geo, blob, A_k, B_k, A_v, B_v, (cudaStream_t)stream));
     return PKV_OK;

@@ -45,6 +45,26 @@ struct CompressSmem {
     float red[Shape<P>::kWarps];
 };
 
+// Extra shared memory of the INT4 epilogue (placed behind CompressSmem<P>).
+struct QuantSmem {
+    float B[32 * kHeadDim];        // B = A^T X in fp32, rank rows
+    float root[32], inv[32];       // sqrt(sigma_j) and its inverse (0 for a zero row)
+    float s_rank[32];              // stored (bf16-valued) scales: per rank column of A~ (keys)
+    float s_tok[kMaxPage];         //                              per token of A~ (values)
+    float s_ch[kHeadDim];          //                              per channel of B~
+};
+
+__device__ __forceinline__ float bf16_round(float v) {
+    return __bfloat162float(__float2bfloat16_rn(v));
+}
+// symmetric INT4 code of x for a stored scale: round half to even, clipped to [-7, 7] (0 if the scale is 0),
+// returned in its stored form code + 8
+__device__ __forceinline__ unsigned int4_code(float x, float scale) {
+    if (!(scale > 0.f)) return 8u;
+    const float q = fminf(fmaxf(rintf(x / scale), -7.f), 7.f);
+    return (unsigned)((int)q + 8);
+}
+
 // Round-robin tournament: in round rho (0..P-2) the P indices form P/2 disjoint
 // pairs; over P-1 rounds every pair meets exactly once.
 inline void pair_of(int P, int rho, int k, int &p, int &q) {
@@ -257,6 +277,88 @@ compress_kernel(Geometry geo, const unsigned char *dense_pool, unsigned char *fa
     }
     __syncthreads();
 
+    if (geo.factor_bits == 4) {
+        // ---- INT4 factors (paper, Section 4.3): A~ = A Sigma^(1/2), B~ = Sigma^(-1/2) B, symmetric 4-bit codes ----
+        QuantSmem &Z = *reinterpret_cast<QuantSmem *>(smem_raw + ((sizeof(CompressSmem<P>) + 15) / 16) * 16);
+        for (int i = tid; i < rank * (kHeadDim / 2); i += kThreads) {
+            const int j = i / (kHeadDim / 2), col = (i % (kHeadDim / 2)) * 2;
+            const int oj = S.order[j];
+            float b0 = 0.f, b1 = 0.f;
+#pragma unroll 8
+            for (int r = 0; r < P; ++r) {
+                const float a = S.Q[r * kGs + oj];
+                const float2 x = __bfloat1622float2(*reinterpret_cast<const __nv_bfloat162 *>(&S.X[r * kXs + col]));
+                b0 = fmaf(a, x.x, b0);
+                b1 = fmaf(a, x.y, b1);
+            }
+            Z.B[j * kHeadDim + col] = b0;
+            Z.B[j * kHeadDim + col + 1] = b1;
+        }
+        __syncthreads();
+        if (tid < rank) {                                   // sigma_j = ||B_j||
+            float ss = 0.f;
+            for (int c = 0; c < kHeadDim; ++c) ss = fmaf(Z.B[tid * kHeadDim + c], Z.B[tid * kHeadDim + c], ss);
+            const float root = sqrtf(sqrtf(ss));
+            Z.root[tid] = root;
+            Z.inv[tid] = root > 0.f ? 1.f / root : 0.f;
+        }
+        __syncthreads();
+        // scales = max|x| / 7, stored in bf16: keys per rank column of A~, values per token of A~; B~ per channel
+        unsigned char *sc_base = blob + geo.codes_bytes;
+        if (!kv) {
+            if (tid < rank) {
+                const int oj = S.order[tid];
+                float m = 0.f;
+                for (int i = 0; i < P; ++i) m = fmaxf(m, fabsf(S.Q[i * kGs + oj]));
+                const float sc = bf16_round(m * Z.root[tid] / 7.f);
+                Z.s_rank[tid] = sc;
+                *reinterpret_cast<__nv_bfloat16 *>(sc_base + geo.sak_off + 2 * tid) = __float2bfloat16_rn(sc);
+            } else if (tid < ((rank + 7) & ~7)) {           // padding entries of the rank-scale array
+                *reinterpret_cast<__nv_bfloat16 *>(sc_base + geo.sak_off + 2 * tid) = __float2bfloat16_rn(0.f);
+            }
+        } else if (tid < P) {
+            float m = 0.f;
+            for (int j = 0; j < rank; ++j) m = fmaxf(m, fabsf(S.Q[tid * kGs + S.order[j]] * Z.root[j]));
+            const float sc = bf16_round(m / 7.f);
+            Z.s_tok[tid] = sc;
+            *reinterpret_cast<__nv_bfloat16 *>(sc_base + geo.sav_off + 2 * tid) = __float2bfloat16_rn(sc);
+        }
+        for (int c = tid; c < kHeadDim; c += kThreads) {
+            float m = 0.f;
+            for (int j = 0; j < rank; ++j) m = fmaxf(m, fabsf(Z.B[j * kHeadDim + c] * Z.inv[j]));
+            const float sc = bf16_round(m / 7.f);
+            Z.s_ch[c] = sc;
+            *reinterpret_cast<__nv_bfloat16 *>(sc_base + (kv ? geo.sbv_off : geo.sbk_off) + 2 * c) = __float2bfloat16_rn(sc);
+        }
+        __syncthreads();
+        // one 32-bit word of codes per 16-byte chunk of the bf16 form: A^T region, then B region of this matrix pair
+        unsigned *words = reinterpret_cast<unsigned *>(blob);
+        const int a_base = (kv ? geo.av_off : geo.ak_off) >> 4, b_base = (kv ? geo.bv_off : geo.bk_off) >> 4;
+        const int a_words = rank * (P / 8), b_words = rank * (kHeadDim / 8);
+        for (int w = tid; w < a_words + b_words; w += kThreads) {
+            unsigned word = 0u;
+            if (w < a_words) {
+                const int j = w / (P / 8), lc = swz_a_chunk(P, j, w % (P / 8));     // stored chunk -> logical chunk
+                const int oj = S.order[j];
+#pragma unroll
+                for (int e = 0; e < 8; ++e) {
+                    const int tok = lc * 8 + e;
+                    const float x = S.Q[tok * kGs + oj] * Z.root[j];
+                    word |= int4_code(x, kv ? Z.s_tok[tok] : Z.s_rank[j]) << int4_nibble_shift(e);
+                }
+                words[a_base + w] = word;
+            } else {
+                const int wb = w - a_words, j = wb / (kHeadDim / 8), lc = (wb % (kHeadDim / 8)) ^ (j & 7);
+#pragma unroll
+                for (int e = 0; e < 8; ++e) {
+                    const int c = lc * 8 + e;
+                    word |= int4_code(Z.B[j * kHeadDim + c] * Z.inv[j], Z.s_ch[c]) << int4_nibble_shift(e);
+                }
+                words[b_base + wb] = word;
+            }
+        }
+        return;
+    }
     // ---- A^T [r][P] = Q[:, order[:r]]^T as bf16, chunk-swizzled rows ----
     for (int i = tid; i < rank * (P / 2); i += kThreads) {
         const int j = i / (P / 2), tok = (i % (P / 2)) * 2;
@@ -328,14 +430,14 @@ cudaError_t launch_p(const Geometry &geo, const unsigned char *dense_pool, unsig
     if (e != cudaSuccess) return e;
     if (dev < 0 || dev >= 64 || !configured[dev]) {
         e = cudaFuncSetAttribute(compress_kernel<P>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                 (int)sizeof(CompressSmem<P>));
+                                 (int)(sizeof(CompressSmem<P>) + 16 + sizeof(QuantSmem)));
         if (e != cudaSuccess) return e;
         if ((e = upload_pair_tables()) != cudaSuccess) return e;
         if (dev >= 0 && dev < 64) configured[dev] = true;
     }
     const unsigned grid = (unsigned)n_entries * geo.n_kv_heads * 2;
-    compress_kernel<P><<<grid, Shape<P>::kThreads, sizeof(CompressSmem<P>), st>>>(geo, dense_pool, factor_pool,
-                                                                                   worklist, status);
+    const size_t smem = sizeof(CompressSmem<P>) + (geo.factor_bits == 4 ? 16 + sizeof(QuantSmem) : 0);
+    compress_kernel<P><<<grid, Shape<P>::kThreads, smem, st>>>(geo, dense_pool, factor_pool, worklist, status);
     return cudaGetLastError();
 }
 

@@ -127,14 +127,14 @@ __global__ void __launch_bounds__(128) decode_scalar_kernel(const __grid_constan
                 for (int i = tid; i < G * r_k; i += 128) {           // q~ = B_k q
                     const int gq = i / r_k, j = i % r_k;
                     float acc = 0.f;
-                    for (int c = 0; c < kHeadDim; ++c) acc += bf16_at(base + g.bk_off, swz_off(j, c)) * qs[gq][c];
+                    for (int c = 0; c < kHeadDim; ++c) acc += blob_value(g, base, 1, j, c) * qs[gq][c];
                     qt[gq][j] = acc;
                 }
                 __syncthreads();
                 for (int i = tid; i < G * P; i += 128) {             // s = A_k q~ * scale
                     const int gq = i / P, p = i % P;
                     float acc = 0.f;
-                    for (int j = 0; j < r_k; ++j) acc += bf16_at(base + g.ak_off, a_t_offset(P, j, p)) * qt[gq][j];
+                    for (int j = 0; j < r_k; ++j) acc += blob_value(g, base, 0, j, p) * qt[gq][j];
                     sc[gq][p] = acc * g.scale_log2e;
                 }
             } else {
@@ -170,13 +170,13 @@ __global__ void __launch_bounds__(128) decode_scalar_kernel(const __grid_constan
                 for (int i = tid; i < G * r_v; i += 128) {           // w = A_v^T p
                     const int gq = i / r_v, j = i % r_v;
                     float acc = 0.f;
-                    for (int p = 0; p < P; ++p) acc += sc[gq][p] * bf16_at(base + g.av_off, a_t_offset(P, j, p));
+                    for (int p = 0; p < P; ++p) acc += sc[gq][p] * blob_value(g, base, 2, j, p);
                     wv[gq][j] = acc;
                 }
                 __syncthreads();
                 for (int gq = 0; gq < G; ++gq) {                     // o = o*alpha + B_v^T w
                     float acc = 0.f;
-                    for (int j = 0; j < r_v; ++j) acc += wv[gq][j] * bf16_at(base + g.bv_off, swz_off(j, tid));
+                    for (int j = 0; j < r_v; ++j) acc += wv[gq][j] * blob_value(g, base, 3, j, tid);
                     o[gq] = o[gq] * alpha_s[gq] + acc;
                 }
             } else {
@@ -384,6 +384,71 @@ __device__ __forceinline__ void online_softmax(float (&s)[4][4], WarpState &st, 
         T0[i] = movm_t(pack_bf16(s[i][0], s[i][1]));   // (head g; tokens 16i+2t, +1)
         T1[i] = movm_t(pack_bf16(s[i][2], s[i][3]));   // (head g; tokens 16i+8+2t, +1)
     }
+}
+
+// One 16-byte chunk of the bf16 form from its 32-bit word of INT4 codes (see unpack_int4).
+template <int P>
+__device__ __forceinline__ void unpack_chunk(unsigned char *sp, const unsigned char *scales, const Geometry &g, int w,
+                                             uint32_t cw) {
+    const int off = w << 4;
+    uint4 raw;                                        // eight bf16 scales, or one replicated
+    if (off < g.bk_off) {
+        const unsigned short s1 = *reinterpret_cast<const unsigned short *>(scales + g.sak_off + 2 * (off / (2 * P)));
+        raw.x = raw.y = raw.z = raw.w = (uint32_t)s1 * 0x10001u;
+    } else if (off < g.av_off) {
+        const int o = off - g.bk_off, r = o >> 8, lc = ((o & 255) >> 4) ^ (r & 7);
+        raw = *reinterpret_cast<const uint4 *>(scales + g.sbk_off + lc * 16);
+    } else if (off < g.bv_off) {
+        const int o = off - g.av_off, r = o / (2 * P), lc = swz_a_chunk(P, r, (o % (2 * P)) >> 4);
+        raw = *reinterpret_cast<const uint4 *>(scales + g.sav_off + lc * 16);
+    } else {
+        const int o = off - g.bv_off, r = o >> 8, lc = ((o & 255) >> 4) ^ (r & 7);
+        raw = *reinterpret_cast<const uint4 *>(scales + g.sbv_off + lc * 16);
+    }
+    const uint32_t sw[4] = {raw.x, raw.y, raw.z, raw.w};
+    uint32_t outw[4];
+    // (word >> 4j) & 0x000F000F | 0x43004300 is the bf16 pair (128 + u0, 128 + u1) with u = code + 8;
+    // subtracting 136 is exact, the product with the scale rounds once: bf16(code * scale)
+    const __nv_bfloat162 k136 = __floats2bfloat162_rn(136.f, 136.f);
+#pragma unroll
+    for (int k = 0; k < 4; ++k) {
+        const uint32_t x = ((cw >> (4 * k)) & 0x000F000Fu) | 0x43004300u;
+        const __nv_bfloat162 c = __hsub2(*reinterpret_cast<const __nv_bfloat162 *>(&x), k136);
+        const __nv_bfloat162 v = __hmul2(c, *reinterpret_cast<const __nv_bfloat162 *>(&sw[k]));
+        outw[k] = *reinterpret_cast<const uint32_t *>(&v);
+    }
+    *reinterpret_cast<uint4 *>(sp + off) = make_uint4(outw[0], outw[1], outw[2], outw[3]);
+}
+
+// INT4 blob -> bf16 form, in place.  The stage holds [ ... codes | scales ]: the codes end where the bf16 form
+// (plus tile over-read) ends, so chunk w of the bf16 form (bytes 16w..16w+15) is always written behind the code
+// word w it comes from, and a group of 128 chunks never reaches the code words of later groups (a group reads all
+// of its words before it writes).  Values are bf16(code * scale), the definition of the stored factor.
+template <int P>
+__device__ __forceinline__ void unpack_int4(unsigned char *sp, const Geometry &g, int lane) {
+    const int n_words = g.blob16_bytes >> 4;
+    const uint32_t *codes = reinterpret_cast<const uint32_t *>(sp + g.unpack_bytes - g.codes_bytes);
+    const unsigned char *scales = sp + g.unpack_bytes;
+    for (int w0 = 0; w0 < n_words; w0 += 128) {
+        uint32_t cw[4];
+#pragma unroll
+        for (int k = 0; k < 4; ++k) {
+            const int w = w0 + 32 * k + lane;
+            cw[k] = w < n_words ? codes[w] : 0u;
+        }
+        __syncwarp();
+#pragma unroll
+        for (int k = 0; k < 4; ++k) {
+            const int w = w0 + 32 * k + lane;
+            if (w < n_words) unpack_chunk<P>(sp, scales, g, w, cw[k]);
+        }
+        __syncwarp();
+    }
+    if (g.unpack_bytes > g.blob16_bytes) {                // tile over-read area: left-over code bytes must not look like NaN
+        for (int i = lane; i < ((g.unpack_bytes - g.blob16_bytes) >> 4); i += 32)
+            reinterpret_cast<uint4 *>(sp + g.blob16_bytes)[i] = make_uint4(0u, 0u, 0u, 0u);
+    }
+    __syncwarp();
 }
 
 // One factor page.  sb = shared address of the blob; ak/bk/av/bv = byte offsets of its four matrices;
@@ -649,6 +714,9 @@ __global__ void __launch_bounds__(kDecodeThreads, 2) decode_tc_kernel(const __gr
     extern __shared__ __align__(1024) unsigned char smem[];
     unsigned char *stages = smem;
     const int stage_bytes = geo.stage_bytes, blob_bytes = geo.blob_bytes;
+    const bool int4 = geo.factor_bits == 4;
+    // INT4 blobs land so that their codes end where the unpacked form ends and the scales follow it
+    const int land_off = int4 ? geo.unpack_bytes - geo.codes_bytes : 0;
     float *comb = reinterpret_cast<float *>(smem + (size_t)S * stage_bytes);
     unsigned long long *full_bar = reinterpret_cast<unsigned long long *>(comb + kConsumerWarps * kPartialFloats);
     unsigned long long *empty_bar = full_bar + S;
@@ -674,7 +742,7 @@ __global__ void __launch_bounds__(kDecodeThreads, 2) decode_tc_kernel(const __gr
         *issued = 0;
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     }
-    if (stage_bytes > blob_bytes) {
+    if (!int4 && stage_bytes > blob_bytes) {
         // Tile loads of 8 rows read past a rank that is not a multiple of 8; past the last matrix that is the
         // tail of the stage, which no copy of a factor page ever writes.  Those values are multiplied by exact
         // zeros, so they only have to be finite: clear the tails once.
@@ -741,7 +809,7 @@ __global__ void __launch_bounds__(kDecodeThreads, 2) decode_tc_kernel(const __gr
                             const uint32_t dst = smem_u32(stages + (size_t)s * stage_bytes);
                             if (kind == kKindFactor) {
                                 mbar_arrive_expect_tx(bar, blob_bytes);
-                                bulk_g2s(dst, src, blob_bytes, bar);
+                                bulk_g2s(dst + land_off, src, blob_bytes, bar);
                             } else if (rows > 0) {
                                 mbar_arrive_expect_tx(bar, 2 * rows * kRowBytes);
                                 bulk_g2s(dst, src, rows * kRowBytes, bar);
@@ -817,12 +885,15 @@ __global__ void __launch_bounds__(kDecodeThreads, 2) decode_tc_kernel(const __gr
             if (dsc.rows > 0) {
                 const uint32_t sb = smem_u32(stages + (size_t)s * stage_bytes);
                 if (dsc.kind == kKindFactor) {
+                    if (int4) unpack_int4<P>(stages + (size_t)s * stage_bytes, geo, lane);
                     factor_unit<P, NT>(sb, geo.ak_off, geo.bk_off, geo.av_off, geo.bv_off, geo.rank_k, geo.rank_v, qf,
                                        geo.scale_log2e, st, lane);
                 } else {
                     dense_unit<C::kDB>(sb, stages + (size_t)s * stage_bytes, dsc.rows, qf, geo.scale_log2e, st, lane);
                     if (dsc.rows < C::kDB) asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
                 }
+                // the unpacked form was written with ordinary stores into bytes the next bulk copy will overwrite
+                if (int4 && dsc.kind == kKindFactor) asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
             }
             __syncwarp();
             if (lane == 0) mbar_arrive(smem_u32(empty_bar + s));

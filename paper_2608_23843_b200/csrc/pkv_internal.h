@@ -30,7 +30,15 @@ struct Geometry {
     int n_dense_slots, n_factor_slots;
     int sink_pages, recent_pages;
     // factor blob of one (slot, KV head): [A_k^T r_k x P][B_k r_k x d][A_v^T r_v x P][B_v r_v x d], bf16
-    int ak_off, bk_off, av_off, bv_off, blob_bytes;
+    // (these offsets describe the bf16 form, which is also what INT4 blobs are unpacked to in shared memory)
+    int ak_off, bk_off, av_off, bv_off;
+    int blob16_bytes;                  // size of the bf16 form
+    int blob_bytes;                    // stored size of a blob in the factor pool (= blob16_bytes for bf16 factors)
+    int factor_bits;                   // 16 or 4
+    // INT4 blobs: [codes: one 32-bit word per 16-byte chunk of the bf16 form][bf16 scales: A~_K per rank column
+    // (padded to 8), B~_K per channel, A~_V per token, B~_V per channel]
+    int codes_bytes, sak_off, sbk_off, sav_off, sbv_off;     // scale offsets are relative to the scales' start
+    int unpack_bytes;                  // bf16 form + tile over-read, rounded to 16: INT4 scales land right behind it
     int dense_head_bytes;              // [K P x d][V P x d] of one KV head = 2*P*d*2
     long long dense_slot_bytes, factor_slot_bytes;
     // decode work units: a factor page, or a block of `block_tokens` rows of a dense page
@@ -126,5 +134,36 @@ __host__ __device__ inline int swz_a_chunk(int P, int row, int chunk) {
 __host__ __device__ inline int a_t_offset(int P, int r, int i) {
     return r * 2 * P + swz_a_chunk(P, r, i >> 3) * 16 + (i & 7) * 2;
 }
+
+// INT4 code words: element e (0..7) of a 16-byte chunk of the bf16 form sits in nibble (e >> 1) + 4 * (e & 1),
+// stored as code + 8 (1..15).  With that order (word >> 4j) & 0x000F000F holds elements 2j and 2j+1 in its two
+// halves, which is how the decode kernel turns a word into four bf16 pairs.
+__host__ __device__ inline int int4_nibble_shift(int e) { return 4 * ((e >> 1) + 4 * (e & 1)); }
+
+#ifdef __CUDACC__
+// Value of one factor element as attention reads it.  which: 0 = A_k(r, token i), 1 = B_k(r, channel i),
+// 2 = A_v(r, token i), 3 = B_v(r, channel i).  bf16 factors are read as stored; INT4 factors are
+// bf16(code * scale) with the scale of the element's column or row (see Geometry).
+__device__ inline float blob_value(const Geometry &g, const unsigned char *blob, int which, int r, int i) {
+    const int P = g.page;
+    int off;                                   // byte offset in the bf16 form
+    if (which == 0) off = g.ak_off + a_t_offset(P, r, i);
+    else if (which == 2) off = g.av_off + a_t_offset(P, r, i);
+    else off = (which == 1 ? g.bk_off : g.bv_off) + r * kRowBytes + swz_chunk(r, i >> 3) * 16 + (i & 7) * 2;
+    if (g.factor_bits != 4) {
+        const unsigned short raw = *reinterpret_cast<const unsigned short *>(blob + off);
+        return __uint_as_float((unsigned)raw << 16);
+    }
+    const unsigned word = reinterpret_cast<const unsigned *>(blob)[off >> 4];
+    const int code = (int)((word >> int4_nibble_shift((off & 15) >> 1)) & 0xFu) - 8;
+    const int soff = which == 0 ? g.sak_off + 2 * r : which == 1 ? g.sbk_off + 2 * i
+                   : which == 2 ? g.sav_off + 2 * i : g.sbv_off + 2 * i;
+    const unsigned short sraw = *reinterpret_cast<const unsigned short *>(blob + g.codes_bytes + soff);
+    const float v = (float)code * __uint_as_float((unsigned)sraw << 16);
+    unsigned u = __float_as_uint(v);           // round to bf16, ties to even (v is finite)
+    u += 0x7fffu + ((u >> 16) & 1u);
+    return __uint_as_float(u & 0xffff0000u);
+}
+#endif
 
 }  // namespace pkv

@@ -47,35 +47,34 @@ __global__ void append_kernel(Geometry geo, unsigned char *dense_pool, const int
     }
 }
 
-// blob <-> row-major factors.  dir = 0: blob -> arrays, 1: arrays -> blob.  The caller's A is [P][r]
-// row-major; the blob holds A^T with swizzled chunks, and B rows with the dense-row swizzle.
+// blob <-> row-major factors.  dir = 0: blob -> arrays (INT4 blobs are dequantised), 1: arrays -> blob (bf16
+// blobs only).  The caller's A is [P][r] row-major; the blob holds A^T with swizzled chunks, and B rows with
+// the dense-row swizzle.
 __global__ void factor_io_kernel(Geometry geo, unsigned char *blob, unsigned short *A_k, unsigned short *B_k,
                                  unsigned short *A_v, unsigned short *B_v, int dir) {
     const int P = geo.page, rk = geo.rank_k, rv = geo.rank_v;
     const int nAk = P * rk, nBk = rk * kHeadDim, nAv = P * rv, nBv = rv * kHeadDim;
     for (int i = blockIdx.x * blockDim.x + threadIdx.x; i < nAk + nBk + nAv + nBv; i += gridDim.x * blockDim.x) {
         unsigned short *plain;
-        unsigned short *stored;
+        int which, r, e, off;
         if (i < nAk) {
-            const int tok = i / rk, r = i % rk;
-            plain = A_k + i;
-            stored = reinterpret_cast<unsigned short *>(blob + geo.ak_off + a_t_offset(P, r, tok));
+            which = 0; r = i % rk; e = i / rk; plain = A_k + i;
+            off = geo.ak_off + a_t_offset(P, r, e);
         } else if (i < nAk + nBk) {
-            int j = i - nAk, row = j / kHeadDim, col = j % kHeadDim;
-            plain = B_k + j;
-            stored = reinterpret_cast<unsigned short *>(blob + geo.bk_off + row * kRowBytes +
-                                                        swz_chunk(row, col >> 3) * 16) + (col & 7);
+            const int j = i - nAk;
+            which = 1; r = j / kHeadDim; e = j % kHeadDim; plain = B_k + j;
+            off = geo.bk_off + r * kRowBytes + swz_chunk(r, e >> 3) * 16 + (e & 7) * 2;
         } else if (i < nAk + nBk + nAv) {
-            const int j = i - nAk - nBk, tok = j / rv, r = j % rv;
-            plain = A_v + j;
-            stored = reinterpret_cast<unsigned short *>(blob + geo.av_off + a_t_offset(P, r, tok));
+            const int j = i - nAk - nBk;
+            which = 2; r = j % rv; e = j / rv; plain = A_v + j;
+            off = geo.av_off + a_t_offset(P, r, e);
         } else {
-            int j = i - nAk - nBk - nAv, row = j / kHeadDim, col = j % kHeadDim;
-            plain = B_v + j;
-            stored = reinterpret_cast<unsigned short *>(blob + geo.bv_off + row * kRowBytes +
-                                                        swz_chunk(row, col >> 3) * 16) + (col & 7);
+            const int j = i - nAk - nBk - nAv;
+            which = 3; r = j / kHeadDim; e = j % kHeadDim; plain = B_v + j;
+            off = geo.bv_off + r * kRowBytes + swz_chunk(r, e >> 3) * 16 + (e & 7) * 2;
         }
-        if (dir == 0) *plain = *stored; else *stored = *plain;
+        if (dir == 0) *plain = (unsigned short)(__float_as_uint(blob_value(geo, blob, which, r, e)) >> 16);
+        else *reinterpret_cast<unsigned short *>(blob + off) = *plain;
     }
 }
 

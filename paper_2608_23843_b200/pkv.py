@@ -41,7 +41,7 @@ class PkvConfig(ctypes.Structure):
         ("n_dense_slots", ctypes.c_int64), ("n_factor_slots", ctypes.c_int64),
         ("softmax_scale", ctypes.c_float), ("jacobi_max_sweeps", ctypes.c_int32),
         ("jacobi_tol", ctypes.c_float), ("n_ctas", ctypes.c_int32), ("decode_variant", ctypes.c_int32),
-        ("jacobi_energy_tol", ctypes.c_float), ("decode_overlap", ctypes.c_int32),
+        ("jacobi_energy_tol", ctypes.c_float), ("factor_bits", ctypes.c_int32), ("decode_overlap", ctypes.c_int32),
     ]
 
 
@@ -238,10 +238,10 @@ def pkv_read_dense(handle, slot, kv_head, K, V, stream=None):
 def make_config(n_layers, n_kv_heads, n_q_heads, rank, sink_tokens, recent_tokens, max_seqs, max_pages_per_seq,
                 n_dense_slots, n_factor_slots, head_dim=128, page_size=64, rank_v=None, softmax_scale=0.0,
                 jacobi_max_sweeps=0, jacobi_tol=0.0, n_ctas=0, decode_variant=0, decode_overlap=0,
-                jacobi_energy_tol=0.0) -> PkvConfig:
+                jacobi_energy_tol=0.0, factor_bits=0) -> PkvConfig:
     return PkvConfig(n_layers, n_kv_heads, n_q_heads, head_dim, page_size, rank, rank if rank_v is None else rank_v,
                      sink_tokens, recent_tokens, max_seqs, max_pages_per_seq, n_dense_slots, n_factor_slots,
-                     softmax_scale, jacobi_max_sweeps, jacobi_tol, n_ctas, decode_variant, jacobi_energy_tol, decode_overlap)
+                     softmax_scale, jacobi_max_sweeps, jacobi_tol, n_ctas, decode_variant, jacobi_energy_tol, factor_bits, decode_overlap)
 
 
 class Cache:

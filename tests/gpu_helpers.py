@@ -17,7 +17,7 @@ def oracle_config(cfg: pkv.PkvConfig) -> OracleConfig:
                         head_dim=cfg.head_dim, page_size=cfg.page_size, rank_k=cfg.rank_k, rank_v=cfg.rank_v,
                         sink_tokens=cfg.sink_tokens, recent_tokens=cfg.recent_tokens, max_seqs=cfg.max_seqs,
                         n_dense_slots=cfg.n_dense_slots, n_factor_slots=cfg.n_factor_slots,
-                        softmax_scale=cfg.softmax_scale)
+                        softmax_scale=cfg.softmax_scale, factor_bits=4 if cfg.factor_bits == 4 else 16)
 
 
 class Pair:

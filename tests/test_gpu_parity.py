@@ -331,3 +331,70 @@ def test_overlap_modes_stay_correct_when_appends_and_compressions_are_interleave
         outs[mode] = [r.cpu() for r in res]
     for a, b in zip(outs[0], outs[overlap]):
         assert torch.equal(a, b)
+
+
+@pytest.mark.parametrize("P,rk,rv,G", [(32, 16, 14, 4), (64, 24, 24, 8), (16, 9, 9, 4), (64, 8, 8, 2)])
+def test_int4_factors(P, rk, rv, G):
+    """INT4 factor storage (Section 4.3): the GPU quantizes in the compression kernel and unpacks in the decode
+    kernel.  Kernel gate: the oracle attends over the GPU's own dequantised factors (<= 1e-2).  Factor gate: the
+    GPU's quantized reconstruction error is no worse than the oracle's INT4 error for the same page (x1.15).
+    End to end against the oracle's INT4 cache: 1e-2 + 3 x the error INT4 causes inside the oracle."""
+    import copy
+    from oracle import quant
+    from oracle.cache import OracleCache
+    H = 2
+    lengths = [30 * P + 7, 3 * P, 12 * P]
+    cfg = pkv.make_config(n_layers=1, n_kv_heads=H, n_q_heads=H * G, rank=rk, rank_v=rv, page_size=P, sink_tokens=P,
+                          recent_tokens=2 * P, max_seqs=3, max_pages_per_seq=40, n_dense_slots=120, n_factor_slots=100,
+                          factor_bits=4)
+    sz = pkv.pkv_query_sizes(cfg)
+    ratio = sz.factor_slot_bytes / sz.dense_slot_bytes
+    assert abs(ratio - quant.int4_page_storage_ratio(rk, rv, P, 128)) <= 40.0 / (2 * P * 128 * 2)      # padding only
+    pair = Pair(cfg, seed=P + rk + 1)
+    ocfg16 = copy.copy(pair.orc.cfg)
+    ocfg16.factor_bits = 16
+    exact = OracleCache(ocfg16, pair.orc.dense_free.order, pair.orc.factor_free.order)
+    for s, T in enumerate(lengths):
+        k, v = gen_kv(4, 0, s, T, cfg)
+        _remember_pages(pair, s, 0, k, v)
+        pair.append(0, [s], [k], [v])
+        exact.append_kv(0, [s], [T], f64(k), f64(v))
+    pair.compress(0)
+    exact.compress_eligible_pages(0)
+    pair.same_tables()
+    # factor gate + "really 4 bits" on the first factor pages of sequence 0
+    kinds, slots, _ = pair.gpu.page_table(0, 0)
+    checked = 0
+    for p, (kd, slot) in enumerate(zip(kinds, slots)):
+        if kd != FACTOR or checked >= 6:
+            continue
+        checked += 1
+        for h in range(H):
+            A_k, B_k, A_v, B_v = [f64(t) for t in pair.gpu.read_factors(slot, h)]
+            assert all(len(np.unique(np.abs(A_k[:, j]))) <= 8 for j in range(rk))          # |codes| in 0..7, one scale per column
+            assert all(len(np.unique(np.abs(A_v[i, :]))) <= 8 for i in range(P))           # one scale per token
+            assert all(len(np.unique(np.abs(B_k[:, c]))) <= 8 for c in range(128))
+            assert all(len(np.unique(np.abs(B_v[:, c]))) <= 8 for c in range(128))
+            of = pair.orc.factor[slot]
+            for name, A, B, oa, ob in (("K", A_k, B_k, of["A_k"][h], of["B_k"][h]), ("V", A_v, B_v, of["A_v"][h], of["B_v"][h])):
+                X = pair.pages[(0, 0, p, h, name)]
+                err, ref = np.linalg.norm(X - A @ B), np.linalg.norm(X - oa @ ob)
+                assert err <= 1.15 * ref + 1e-3 * np.linalg.norm(X), (p, h, name, err, ref)
+    order = [2, 0, 1]
+    q = synth.make_q(4, 0, 0, 3, H * G, 128)
+    got, got32 = pair.decode(0, order, q)
+    g = attention_gates(pair, 0, order, q, got, got32)            # kernel gate: oracle over the GPU's dequantised factors
+    ref4 = pair.orc.decode_attention(0, order, f64(q))
+    ref16 = exact.decode_attention(0, order, f64(q))
+    for i in range(3):
+        assert g["kernel"][i] <= 4e-3 and g["kernel_bf16"][i] <= ATT_TOL, (i, g["kernel"][i])
+        floor4 = rel_err(ref4[i], ref16[i])
+        assert rel_err(got[i], ref4[i]) <= ATT_TOL + 3.0 * floor4, (i, rel_err(got[i], ref4[i]), floor4)
+    with pytest.raises(pkv.PkvError) as e:
+        pair.gpu.write_factors(slots[1], 0, *pair.gpu.read_factors(slots[1], 0))
+    assert e.value.status == pkv.PKV_ERR_UNSUPPORTED
+    st = pair.gpu.stats()
+    assert st["device_timeouts"] == 0 and st["page_svds_not_converged"] == 0 and st["bad_slot_indices"] == 0
+    print("int4 P=%d r=(%d,%d): kernel %.2e, e2e vs int4 oracle %.2e, int4 noise %.2e, storage ratio %.4f"
+          % (P, rk, rv, max(g["kernel"]), max(rel_err(got[i], ref4[i]) for i in range(3)),
+             max(rel_err(ref4[i], ref16[i]) for i in range(3)), ratio))
