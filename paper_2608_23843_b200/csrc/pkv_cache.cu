@@ -161,7 +161,11 @@ void derive(const pkv_config &cfg, int n_ctas, Geometry &g, MetaLayout &ml, Work
     g.bv_off = g.av_off + P * cfg.rank_v * 2;
     g.blob16_bytes = g.bv_off + cfg.rank_v * d * 2;
     g.factor_bits = cfg.factor_bits == 4 ? 4 : 16;
-    g.codes_bytes = (int)align_up(g.blob16_bytes / 4, 16);
+    g.cak_off = 0;
+    g.cbk_off = g.cak_off + 4 * int4_a_words(P, g.rank_tiles);
+    g.cav_off = g.cbk_off + 4 * int4_b_words(d, g.rank_tiles);
+    g.cbv_off = g.cav_off + 4 * int4_b_words(P, g.rank_tiles);
+    g.codes_bytes = g.cbv_off + 4 * int4_a_words(d, g.rank_tiles);
     g.sak_off = 0;
     g.sbk_off = g.sak_off + 2 * (int)align_up(cfg.rank_k, 8);
     g.sav_off = g.sbk_off + 2 * d;
@@ -173,11 +177,10 @@ void derive(const pkv_config &cfg, int n_ctas, Geometry &g, MetaLayout &ml, Work
     g.factor_slot_bytes = (long long)cfg.n_kv_heads * g.blob_bytes;
     // decode work units: a factor page or a block of rows of a dense page.  A stage must hold either, plus
     // the rows that 8-row tile loads read past the last matrix when rank_v is not a multiple of 8.
-    g.block_tokens = (P >= 32 && g.rank_tiles >= 3) ? 32 : 16;
+    g.block_tokens = (g.factor_bits != 4 && P >= 32 && g.rank_tiles >= 3) ? 32 : 16;
     g.blocks_per_page = P / g.block_tokens;
     const int overread = (8 * g.rank_tiles - cfg.rank_v) * kRowBytes;
-    g.unpack_bytes = (int)align_up(g.blob16_bytes + overread, 16);
-    const int factor_stage = g.factor_bits == 4 ? g.unpack_bytes + (g.blob_bytes - g.codes_bytes) : g.unpack_bytes;
+    const int factor_stage = g.factor_bits == 4 ? g.blob_bytes : (int)align_up(g.blob16_bytes + overread, 16);
     g.stage_bytes = (int)align_up(std::max(factor_stage, g.block_tokens * 2 * kRowBytes), 128);
     // two CTAs are resident per SM (consecutive launches overlap, or the grid holds two CTAs per SM),
     // so that one streams while the other is in its prologue or merging

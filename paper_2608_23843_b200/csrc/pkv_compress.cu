@@ -331,31 +331,33 @@ compress_kernel(Geometry geo, const unsigned char *dense_pool, unsigned char *fa
             *reinterpret_cast<__nv_bfloat16 *>(sc_base + (kv ? geo.sbv_off : geo.sbk_off) + 2 * c) = __float2bfloat16_rn(sc);
         }
         __syncthreads();
-        // one 32-bit word of codes per 16-byte chunk of the bf16 form: A^T region, then B region of this matrix pair
-        unsigned *words = reinterpret_cast<unsigned *>(blob);
-        const int a_base = (kv ? geo.av_off : geo.ak_off) >> 4, b_base = (kv ? geo.bv_off : geo.bk_off) >> 4;
-        const int a_words = rank * (P / 8), b_words = rank * (kHeadDim / 8);
+        // code words in operand-register order (see int4_a_pos / int4_b_pos): A~ region, then B~ region of this
+        // matrix pair; ranks past the true rank and registers past the last one hold zero codes
+        const int NT = geo.rank_tiles;
+        const int a_words = kv ? int4_b_words(P, NT) : int4_a_words(P, NT);
+        const int b_words = kv ? int4_a_words(kHeadDim, NT) : int4_b_words(kHeadDim, NT);
+        unsigned *wa = reinterpret_cast<unsigned *>(blob + (kv ? geo.cav_off : geo.cak_off));
+        unsigned *wb = reinterpret_cast<unsigned *>(blob + (kv ? geo.cbv_off : geo.cbk_off));
         for (int w = tid; w < a_words + b_words; w += kThreads) {
+            const bool is_a = w < a_words;
+            const int wl = is_a ? w : w - a_words, ln = wl & 31, wq = wl >> 5;
             unsigned word = 0u;
-            if (w < a_words) {
-                const int j = w / (P / 8), lc = swz_a_chunk(P, j, w % (P / 8));     // stored chunk -> logical chunk
-                const int oj = S.order[j];
 #pragma unroll
-                for (int e = 0; e < 8; ++e) {
-                    const int tok = lc * 8 + e;
-                    const float x = S.Q[tok * kGs + oj] * Z.root[j];
-                    word |= int4_code(x, kv ? Z.s_tok[tok] : Z.s_rank[j]) << int4_nibble_shift(e);
+            for (int e = 0; e < 8; ++e) {
+                const int t = e >> 1, h = e & 1, n = 4 * wq + t;
+                int x = 0, j = 0;                  // x: token (A~) or channel (B~); j: rank
+                unsigned code = 8u;
+                if (is_a) {
+                    const bool ok = kv ? int4_b_elem(P, NT, ln, n, h, x, j) : int4_a_elem(P, NT, ln, n, h, x, j);
+                    if (ok && j < rank)
+                        code = int4_code(S.Q[x * kGs + S.order[j]] * Z.root[j], kv ? Z.s_tok[x] : Z.s_rank[j]);
+                } else {
+                    const bool ok = kv ? int4_a_elem(kHeadDim, NT, ln, n, h, x, j) : int4_b_elem(kHeadDim, NT, ln, n, h, x, j);
+                    if (ok && j < rank) code = int4_code(Z.B[j * kHeadDim + x] * Z.inv[j], Z.s_ch[x]);
                 }
-                words[a_base + w] = word;
-            } else {
-                const int wb = w - a_words, j = wb / (kHeadDim / 8), lc = (wb % (kHeadDim / 8)) ^ (j & 7);
-#pragma unroll
-                for (int e = 0; e < 8; ++e) {
-                    const int c = lc * 8 + e;
-                    word |= int4_code(Z.B[j * kHeadDim + c] * Z.inv[j], Z.s_ch[c]) << int4_nibble_shift(e);
-                }
-                words[b_base + wb] = word;
+                word |= code << (4 * (t + 4 * h));
             }
+            (is_a ? wa : wb)[wl] = word;
         }
         return;
     }

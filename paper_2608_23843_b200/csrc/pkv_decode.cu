@@ -337,11 +337,13 @@ struct WarpState {
     float m[2], l[2];     // l is this lane's share; summed over g at flush time
 };
 
-// Shapes fixed at compile time: P tokens per page, NT = ceil(rank / 8) rank tiles (K and V alike).
-template <int P, int NT>
+// Shapes fixed at compile time: P tokens per page, NT = ceil(rank / 8) rank tiles (K and V alike), I4 = factors
+// stored as INT4 codes.
+template <int P, int NT, bool I4 = false>
 struct Tc {
     static constexpr int kMT = P / 16;                                  // 16-token tiles per page
-    static constexpr int kDB = (P >= 32 && NT >= 3) ? 32 : 16;          // rows per dense block
+    // rows per dense block: 32 where a stage has to be that large for a bf16 factor page anyway
+    static constexpr int kDB = (!I4 && P >= 32 && NT >= 3) ? 32 : 16;
     static constexpr int kPitchA = 2 * P;                               // bytes per A^T row
 };
 
@@ -386,69 +388,16 @@ __device__ __forceinline__ void online_softmax(float (&s)[4][4], WarpState &st, 
     }
 }
 
-// One 16-byte chunk of the bf16 form from its 32-bit word of INT4 codes (see unpack_int4).
-template <int P>
-__device__ __forceinline__ void unpack_chunk(unsigned char *sp, const unsigned char *scales, const Geometry &g, int w,
-                                             uint32_t cw) {
-    const int off = w << 4;
-    uint4 raw;                                        // eight bf16 scales, or one replicated
-    if (off < g.bk_off) {
-        const unsigned short s1 = *reinterpret_cast<const unsigned short *>(scales + g.sak_off + 2 * (off / (2 * P)));
-        raw.x = raw.y = raw.z = raw.w = (uint32_t)s1 * 0x10001u;
-    } else if (off < g.av_off) {
-        const int o = off - g.bk_off, r = o >> 8, lc = ((o & 255) >> 4) ^ (r & 7);
-        raw = *reinterpret_cast<const uint4 *>(scales + g.sbk_off + lc * 16);
-    } else if (off < g.bv_off) {
-        const int o = off - g.av_off, r = o / (2 * P), lc = swz_a_chunk(P, r, (o % (2 * P)) >> 4);
-        raw = *reinterpret_cast<const uint4 *>(scales + g.sav_off + lc * 16);
-    } else {
-        const int o = off - g.bv_off, r = o >> 8, lc = ((o & 255) >> 4) ^ (r & 7);
-        raw = *reinterpret_cast<const uint4 *>(scales + g.sbv_off + lc * 16);
-    }
-    const uint32_t sw[4] = {raw.x, raw.y, raw.z, raw.w};
-    uint32_t outw[4];
-    // (word >> 4j) & 0x000F000F | 0x43004300 is the bf16 pair (128 + u0, 128 + u1) with u = code + 8;
-    // subtracting 136 is exact, the product with the scale rounds once: bf16(code * scale)
-    const __nv_bfloat162 k136 = __floats2bfloat162_rn(136.f, 136.f);
-#pragma unroll
-    for (int k = 0; k < 4; ++k) {
-        const uint32_t x = ((cw >> (4 * k)) & 0x000F000Fu) | 0x43004300u;
-        const __nv_bfloat162 c = __hsub2(*reinterpret_cast<const __nv_bfloat162 *>(&x), k136);
-        const __nv_bfloat162 v = __hmul2(c, *reinterpret_cast<const __nv_bfloat162 *>(&sw[k]));
-        outw[k] = *reinterpret_cast<const uint32_t *>(&v);
-    }
-    *reinterpret_cast<uint4 *>(sp + off) = make_uint4(outw[0], outw[1], outw[2], outw[3]);
+__device__ __forceinline__ uint32_t lds32(uint32_t addr) {
+    uint32_t v;
+    asm volatile("ld.shared.b32 %0, [%1];" : "=r"(v) : "r"(addr));
+    return v;
 }
-
-// INT4 blob -> bf16 form, in place.  The stage holds [ ... codes | scales ]: the codes end where the bf16 form
-// (plus tile over-read) ends, so chunk w of the bf16 form (bytes 16w..16w+15) is always written behind the code
-// word w it comes from, and a group of 128 chunks never reaches the code words of later groups (a group reads all
-// of its words before it writes).  Values are bf16(code * scale), the definition of the stored factor.
-template <int P>
-__device__ __forceinline__ void unpack_int4(unsigned char *sp, const Geometry &g, int lane) {
-    const int n_words = g.blob16_bytes >> 4;
-    const uint32_t *codes = reinterpret_cast<const uint32_t *>(sp + g.unpack_bytes - g.codes_bytes);
-    const unsigned char *scales = sp + g.unpack_bytes;
-    for (int w0 = 0; w0 < n_words; w0 += 128) {
-        uint32_t cw[4];
-#pragma unroll
-        for (int k = 0; k < 4; ++k) {
-            const int w = w0 + 32 * k + lane;
-            cw[k] = w < n_words ? codes[w] : 0u;
-        }
-        __syncwarp();
-#pragma unroll
-        for (int k = 0; k < 4; ++k) {
-            const int w = w0 + 32 * k + lane;
-            if (w < n_words) unpack_chunk<P>(sp, scales, g, w, cw[k]);
-        }
-        __syncwarp();
-    }
-    if (g.unpack_bytes > g.blob16_bytes) {                // tile over-read area: left-over code bytes must not look like NaN
-        for (int i = lane; i < ((g.unpack_bytes - g.blob16_bytes) >> 4); i += 32)
-            reinterpret_cast<uint4 *>(sp + g.blob16_bytes)[i] = make_uint4(0u, 0u, 0u, 0u);
-    }
-    __syncwarp();
+// one bf16 from shared memory, copied into both halves of a register
+__device__ __forceinline__ uint32_t lds16x2(uint32_t addr) {
+    uint32_t v;
+    asm volatile("ld.shared.u16 %0, [%1];" : "=r"(v) : "r"(addr));
+    return v * 0x10001u;
 }
 
 // One factor page.  sb = shared address of the blob; ak/bk/av/bv = byte offsets of its four matrices;
@@ -532,6 +481,124 @@ __device__ __forceinline__ void factor_unit(uint32_t sb, int ak, int bk, int av,
         }
     }
 }
+
+// Register n (a compile-time constant after unrolling) of this lane out of its code words: the two codes as
+// bf16(code * scale).  (word >> 4t) & 0x000F000F | 0x43004300 is the bf16 pair (128 + u_lo, 128 + u_hi) with
+// u = code + 8; subtracting 136 is exact and the product with the scale pair rounds once.
+__device__ __forceinline__ uint32_t int4_pair(uint32_t word, int t, uint32_t scale2) {
+    const uint32_t x = ((word >> (4 * t)) & 0x000F000Fu) | 0x43004300u;
+    uint32_t c, v;
+    asm("sub.rn.bf16x2 %0, %1, %2;" : "=r"(c) : "r"(x), "r"(0x43084308u));
+    asm("mul.rn.bf16x2 %0, %1, %2;" : "=r"(v) : "r"(c), "r"(scale2));
+    return v;
+}
+#define PKV_I4(words, n, scale2) int4_pair((words)[(n) >> 2], (n) & 3, (scale2))
+
+// One factor page stored as INT4 codes in operand-register order (see int4_a_pos / int4_b_pos): the same four
+// products as factor_unit, with every operand register made from its codes and scales in registers.  Ranks
+// past the true ones are stored as zero codes, so nothing needs masking.
+template <int P, int NT>
+__device__ __forceinline__ void factor_unit_int4(uint32_t sb, const Geometry &g, const uint32_t (&qf)[8][2],
+                                                 WarpState &st, int lane) {
+    using C = Tc<P, NT>;
+    constexpr int kMT = C::kMT;
+    constexpr int kWA = (kMT * 2 * NT + 3) / 4;        // words per lane: A~_K
+    constexpr int kWV = (NT * (P / 8) + 3) / 4;        //                 A~_V
+    constexpr int kWR = (8 * 2 * NT + 3) / 4;          //                 B~_V
+    const int gq = lane >> 2, c2 = (lane & 3) * 2;
+    const uint32_t sc = sb + g.codes_bytes, lane4 = lane * 4;
+    // ---- q~^T [G][r] = q [G][d] . B~_K^T   (scales per channel: pairs d = 16 kk + 8 b + 2c, +1) ----
+    uint32_t qhi[NT], qlo[NT];
+    {
+        uint32_t sk[16];
+#pragma unroll
+        for (int i = 0; i < 16; ++i) sk[i] = lds32(sc + g.sbk_off + 2 * (8 * i + c2));
+#pragma unroll
+        for (int j = 0; j < NT; ++j) {
+            float qt[4] = {0.f, 0.f, 0.f, 0.f};
+#pragma unroll
+            for (int wq = 0; wq < 4; ++wq) {
+                const uint32_t w = lds32(sb + g.cbk_off + (j * 4 + wq) * 128 + lane4);
+                mma16816(qt, qf[2 * wq][0], 0u, qf[2 * wq][1], 0u, int4_pair(w, 0, sk[4 * wq]), int4_pair(w, 1, sk[4 * wq + 1]));
+                mma16816(qt, qf[2 * wq + 1][0], 0u, qf[2 * wq + 1][1], 0u, int4_pair(w, 2, sk[4 * wq + 2]),
+                         int4_pair(w, 3, sk[4 * wq + 3]));
+            }
+            const float x0 = qt[0] * g.scale_log2e, x1 = qt[1] * g.scale_log2e;
+            qhi[j] = pack_bf16(x0, x1);
+            qlo[j] = pack_bf16(x0 - bf16lo_f(qhi[j]), x1 - bf16hi_f(qhi[j]));
+        }
+    }
+    // ---- s [P][G] = A~_K [P][r] . q~   (scales per rank: pairs 8 jt + 2c, +1) ----
+    float s[4][4];
+    {
+        uint32_t sa[NT], wa[kWA];
+#pragma unroll
+        for (int jt = 0; jt < NT; ++jt) sa[jt] = lds32(sc + g.sak_off + 2 * (8 * jt + c2));
+#pragma unroll
+        for (int w = 0; w < kWA; ++w) wa[w] = lds32(sb + g.cak_off + w * 128 + lane4);
+#pragma unroll
+        for (int i = 0; i < kMT; ++i) {
+            s[i][0] = s[i][1] = s[i][2] = s[i][3] = 0.f;
+#pragma unroll
+            for (int kk = 0; kk < NT / 2; ++kk) {
+                const int n0 = i * 2 * NT + 4 * kk;
+                const uint32_t a0 = PKV_I4(wa, n0, sa[2 * kk]), a1 = PKV_I4(wa, n0 + 1, sa[2 * kk]);
+                const uint32_t a2 = PKV_I4(wa, n0 + 2, sa[2 * kk + 1]), a3 = PKV_I4(wa, n0 + 3, sa[2 * kk + 1]);
+                mma16816(s[i], a0, a1, a2, a3, qhi[2 * kk], qhi[2 * kk + 1]);
+                mma16816(s[i], a0, a1, a2, a3, qlo[2 * kk], qlo[2 * kk + 1]);
+            }
+            if (NT % 2) {
+                const int n0 = i * 2 * NT + 4 * (NT / 2);
+                const uint32_t a0 = PKV_I4(wa, n0, sa[NT - 1]), a1 = PKV_I4(wa, n0 + 1, sa[NT - 1]);
+                mma1688(s[i], a0, a1, qhi[NT - 1]);
+                mma1688(s[i], a0, a1, qlo[NT - 1]);
+            }
+        }
+    }
+    uint32_t T0[4], T1[4];
+    online_softmax<kMT>(s, st, T0, T1);
+    // ---- w^T [G][r] = p^T [G][P] . A~_V [P][r]   (scales per token: pairs 16 kk + 8 b + 2c, +1) ----
+    uint32_t wh[NT];
+    {
+        uint32_t sv[2 * kMT], wv[kWV];
+#pragma unroll
+        for (int i = 0; i < 2 * kMT; ++i) sv[i] = lds32(sc + g.sav_off + 2 * (8 * i + c2));
+#pragma unroll
+        for (int w = 0; w < kWV; ++w) wv[w] = lds32(sb + g.cav_off + w * 128 + lane4);
+#pragma unroll
+        for (int j = 0; j < NT; ++j) {
+            float wt[4] = {0.f, 0.f, 0.f, 0.f};
+#pragma unroll
+            for (int kk = 0; kk < kMT; ++kk) {
+                const int n0 = j * (P / 8) + 2 * kk;
+                mma16816(wt, T0[kk], 0u, T1[kk], 0u, PKV_I4(wv, n0, sv[2 * kk]), PKV_I4(wv, n0 + 1, sv[2 * kk + 1]));
+            }
+            wh[j] = pack_bf16(wt[0], wt[1]);
+        }
+    }
+    // ---- o [d][G] += B~_V^T [d][r] . w   (scales per channel = per row of the operand) ----
+    {
+        uint32_t wr[kWR];
+#pragma unroll
+        for (int w = 0; w < kWR; ++w) wr[w] = lds32(sb + g.cbv_off + w * 128 + lane4);
+#pragma unroll
+        for (int i = 0; i < 8; ++i) {
+            const uint32_t s0 = lds16x2(sc + g.sbv_off + 2 * (16 * i + gq)), s1 = lds16x2(sc + g.sbv_off + 2 * (16 * i + 8 + gq));
+#pragma unroll
+            for (int kk = 0; kk < NT / 2; ++kk) {
+                const int n0 = i * 2 * NT + 4 * kk;
+                mma16816(st.o[i], PKV_I4(wr, n0, s0), PKV_I4(wr, n0 + 1, s1), PKV_I4(wr, n0 + 2, s0), PKV_I4(wr, n0 + 3, s1),
+                         wh[2 * kk], wh[2 * kk + 1]);
+            }
+            if (NT % 2) {
+                const int n0 = i * 2 * NT + 4 * (NT / 2);
+                mma1688(st.o[i], PKV_I4(wr, n0, s0), PKV_I4(wr, n0 + 1, s1), wh[NT - 1]);
+            }
+        }
+    }
+}
+#undef PKV_I4
+
 
 // One block of DB rows of a dense page: K rows at sb, V rows at sb + DB*256; `rows` of them are valid.
 template <int DB>
@@ -701,9 +768,9 @@ __device__ __forceinline__ void flush_segment(const DecodeArgs &a, float *comb, 
     PKV_CONSUMER_BARRIER();
 }
 
-template <int P, int NT>
+template <int P, int NT, bool I4>
 __global__ void __launch_bounds__(kDecodeThreads, 2) decode_tc_kernel(const __grid_constant__ DecodeArgs a) {
-    using C = Tc<P, NT>;
+    using C = Tc<P, NT, I4>;
     Range rg;
     if (!load_range(a, rg)) return;
     const Geometry &geo = a.geo;
@@ -714,9 +781,6 @@ __global__ void __launch_bounds__(kDecodeThreads, 2) decode_tc_kernel(const __gr
     extern __shared__ __align__(1024) unsigned char smem[];
     unsigned char *stages = smem;
     const int stage_bytes = geo.stage_bytes, blob_bytes = geo.blob_bytes;
-    const bool int4 = geo.factor_bits == 4;
-    // INT4 blobs land so that their codes end where the unpacked form ends and the scales follow it
-    const int land_off = int4 ? geo.unpack_bytes - geo.codes_bytes : 0;
     float *comb = reinterpret_cast<float *>(smem + (size_t)S * stage_bytes);
     unsigned long long *full_bar = reinterpret_cast<unsigned long long *>(comb + kConsumerWarps * kPartialFloats);
     unsigned long long *empty_bar = full_bar + S;
@@ -742,7 +806,7 @@ __global__ void __launch_bounds__(kDecodeThreads, 2) decode_tc_kernel(const __gr
         *issued = 0;
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     }
-    if (!int4 && stage_bytes > blob_bytes) {
+    if (!I4 && stage_bytes > blob_bytes) {
         // Tile loads of 8 rows read past a rank that is not a multiple of 8; past the last matrix that is the
         // tail of the stage, which no copy of a factor page ever writes.  Those values are multiplied by exact
         // zeros, so they only have to be finite: clear the tails once.
@@ -809,7 +873,7 @@ __global__ void __launch_bounds__(kDecodeThreads, 2) decode_tc_kernel(const __gr
                             const uint32_t dst = smem_u32(stages + (size_t)s * stage_bytes);
                             if (kind == kKindFactor) {
                                 mbar_arrive_expect_tx(bar, blob_bytes);
-                                bulk_g2s(dst + land_off, src, blob_bytes, bar);
+                                bulk_g2s(dst, src, blob_bytes, bar);
                             } else if (rows > 0) {
                                 mbar_arrive_expect_tx(bar, 2 * rows * kRowBytes);
                                 bulk_g2s(dst, src, rows * kRowBytes, bar);
@@ -885,15 +949,13 @@ __global__ void __launch_bounds__(kDecodeThreads, 2) decode_tc_kernel(const __gr
             if (dsc.rows > 0) {
                 const uint32_t sb = smem_u32(stages + (size_t)s * stage_bytes);
                 if (dsc.kind == kKindFactor) {
-                    if (int4) unpack_int4<P>(stages + (size_t)s * stage_bytes, geo, lane);
-                    factor_unit<P, NT>(sb, geo.ak_off, geo.bk_off, geo.av_off, geo.bv_off, geo.rank_k, geo.rank_v, qf,
-                                       geo.scale_log2e, st, lane);
+                    if (I4) factor_unit_int4<P, NT>(sb, geo, qf, st, lane);
+                    else factor_unit<P, NT>(sb, geo.ak_off, geo.bk_off, geo.av_off, geo.bv_off, geo.rank_k, geo.rank_v, qf,
+                                            geo.scale_log2e, st, lane);
                 } else {
                     dense_unit<C::kDB>(sb, stages + (size_t)s * stage_bytes, dsc.rows, qf, geo.scale_log2e, st, lane);
                     if (dsc.rows < C::kDB) asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
                 }
-                // the unpacked form was written with ordinary stores into bytes the next bulk copy will overwrite
-                if (int4 && dsc.kind == kKindFactor) asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
             }
             __syncwarp();
             if (lane == 0) mbar_arrive(smem_u32(empty_bar + s));
@@ -912,7 +974,7 @@ size_t decode_smem_bytes(const Geometry &g) {
            g.n_stages * (8 + 8 + sizeof(StageDesc)) + 64;
 }
 
-template <int P, int NT>
+template <int P, int NT, bool I4>
 cudaError_t launch_tc(const DecodeArgs &a, cudaStream_t st) {
     cudaLaunchConfig_t cfg = {};
     cfg.gridDim = dim3(a.geo.n_ctas);
@@ -924,12 +986,14 @@ cudaError_t launch_tc(const DecodeArgs &a, cudaStream_t st) {
     attr[0].val.programmaticStreamSerializationAllowed = 1;
     cfg.attrs = attr;
     cfg.numAttrs = a.plain_launch ? 0 : 1;
-    return cudaLaunchKernelEx(&cfg, decode_tc_kernel<P, NT>, a);
+    return cudaLaunchKernelEx(&cfg, decode_tc_kernel<P, NT, I4>, a);
 }
 
 template <int P, int NT>
 cudaError_t setup_tc() {
-    return cudaFuncSetAttribute(decode_tc_kernel<P, NT>, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBudget / 2);
+    cudaError_t e = cudaFuncSetAttribute(decode_tc_kernel<P, NT, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBudget / 2);
+    if (e != cudaSuccess) return e;
+    return cudaFuncSetAttribute(decode_tc_kernel<P, NT, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBudget / 2);
 }
 
 // the instantiated shapes: P in {16, 32, 64}, rank tiles 1..4 (1..2 for P = 16)
@@ -952,7 +1016,8 @@ cudaError_t launch_decode(const DecodeArgs &a, int n_segs, cudaStream_t st) {
         decode_scalar_kernel<<<a.geo.n_ctas, 128, 0, st>>>(a);
         e = cudaGetLastError();
     } else {
-#define PKV_LAUNCH(P, NT) if (a.geo.page == P && a.geo.rank_tiles == NT) e = launch_tc<P, NT>(a, st);
+#define PKV_LAUNCH(P, NT) if (a.geo.page == P && a.geo.rank_tiles == NT) \
+            e = a.geo.factor_bits == 4 ? launch_tc<P, NT, true>(a, st) : launch_tc<P, NT, false>(a, st);
         PKV_FOR_EACH_SHAPE(PKV_LAUNCH)
 #undef PKV_LAUNCH
     }

@@ -29,16 +29,16 @@ struct Geometry {
     int max_seqs, max_pages;
     int n_dense_slots, n_factor_slots;
     int sink_pages, recent_pages;
-    // factor blob of one (slot, KV head): [A_k^T r_k x P][B_k r_k x d][A_v^T r_v x P][B_v r_v x d], bf16
-    // (these offsets describe the bf16 form, which is also what INT4 blobs are unpacked to in shared memory)
+    // bf16 factor blob of one (slot, KV head): [A_k^T r_k x P][B_k r_k x d][A_v^T r_v x P][B_v r_v x d]
     int ak_off, bk_off, av_off, bv_off;
     int blob16_bytes;                  // size of the bf16 form
     int blob_bytes;                    // stored size of a blob in the factor pool (= blob16_bytes for bf16 factors)
     int factor_bits;                   // 16 or 4
-    // INT4 blobs: [codes: one 32-bit word per 16-byte chunk of the bf16 form][bf16 scales: A~_K per rank column
-    // (padded to 8), B~_K per channel, A~_V per token, B~_V per channel]
+    // INT4 blobs: [codes of A~_K][codes of B~_K][codes of A~_V][codes of B~_V][bf16 scales: A~_K per rank column
+    // (padded to 8), B~_K per channel, A~_V per token, B~_V per channel].  Codes are stored in the register order
+    // of the mma operand each matrix is read as (see int4_a_pos / int4_b_pos).
+    int cak_off, cbk_off, cav_off, cbv_off;                  // byte offsets of the four code regions
     int codes_bytes, sak_off, sbk_off, sav_off, sbv_off;     // scale offsets are relative to the scales' start
-    int unpack_bytes;                  // bf16 form + tile over-read, rounded to 16: INT4 scales land right behind it
     int dense_head_bytes;              // [K P x d][V P x d] of one KV head = 2*P*d*2
     long long dense_slot_bytes, factor_slot_bytes;
     // decode work units: a factor page, or a block of `block_tokens` rows of a dense page
@@ -135,10 +135,51 @@ __host__ __device__ inline int a_t_offset(int P, int r, int i) {
     return r * 2 * P + swz_a_chunk(P, r, i >> 3) * 16 + (i & 7) * 2;
 }
 
-// INT4 code words: element e (0..7) of a 16-byte chunk of the bf16 form sits in nibble (e >> 1) + 4 * (e & 1),
-// stored as code + 8 (1..15).  With that order (word >> 4j) & 0x000F000F holds elements 2j and 2j+1 in its two
-// halves, which is how the decode kernel turns a word into four bf16 pairs.
-__host__ __device__ inline int int4_nibble_shift(int e) { return 4 * ((e >> 1) + 4 * (e & 1)); }
+// ---- INT4 code layout -------------------------------------------------------------------------------------
+// Codes are stored as code + 8 (1..15; 8 = zero) in the order in which the decode kernel's tensor-core
+// instructions want their operands, so that a lane turns one 32-bit word into four operand registers without a
+// shared-memory round trip.  An operand register holds two bf16 values; a lane (g = lane >> 2, c = lane & 3)
+// numbers the registers it needs from one matrix n = 0, 1, ...; register n lives in the lane's word n >> 2 at
+// nibbles t and t + 4 (t = n & 3, low and high half), so that (word >> 4t) & 0x000F000F is the pair.  Word w
+// of lane l sits at 32-bit index 32 w + l of the matrix's code region.  NT = ceil(rank / 8); ranks up to 8 NT
+// are stored, the ones past the true rank as zeros.
+//   "A-type" (m16 x k16 row operand; rows m = tokens of A~_K or channels of B~_V, contraction over ranks):
+//       16-row tile i = m >> 4 owns registers i * 2NT ...: per 16-rank step four, (rows g, g+8) x (ranks 2c, 2c+8),
+//       then two for a last 8-rank step.
+//   "B-type" (k16 x n8 col operand; contraction index k = channels of B~_K or tokens of A~_V, columns = ranks):
+//       rank tile j owns registers j * (K/8) ...: register 2 kk + b holds k = 16 kk + 8 b + 2c (+1), rank 8 j + g.
+__host__ __device__ inline int int4_a_words(int M, int NT) { return (((M / 16) * 2 * NT + 3) / 4) * 32; }
+__host__ __device__ inline int int4_b_words(int K, int NT) { return ((NT * (K / 8) + 3) / 4) * 32; }
+// element (row m, rank r) -> 32-bit word index and bit shift of its nibble
+__host__ __device__ inline void int4_a_pos(int NT, int m, int r, int &word, int &shift) {
+    const int i = m >> 4, q0 = (m >> 3) & 1, g = m & 7, full = NT / 2;
+    int e, c;
+    if (r < 16 * full) { e = 4 * (r >> 4) + 2 * ((r >> 3) & 1) + q0; c = (r & 7) >> 1; }
+    else               { e = 4 * full + q0; c = (r - 16 * full) >> 1; }
+    const int n = i * 2 * NT + e;
+    word = (n >> 2) * 32 + 4 * g + c;
+    shift = 4 * ((n & 3) + 4 * (r & 1));
+}
+__host__ __device__ inline void int4_b_pos(int K, int k, int r, int &word, int &shift) {
+    const int n = (r >> 3) * (K / 8) + 2 * (k >> 4) + ((k >> 3) & 1);
+    word = (n >> 2) * 32 + 4 * (r & 7) + ((k & 7) >> 1);
+    shift = 4 * ((n & 3) + 4 * (k & 1));
+}
+// the inverse: half h of register n of `lane` -> (m, r) / (k, r); false past the last register
+__host__ __device__ inline bool int4_a_elem(int M, int NT, int lane, int n, int h, int &m, int &r) {
+    if (n >= (M / 16) * 2 * NT) return false;
+    const int i = n / (2 * NT), e = n % (2 * NT), g = lane >> 2, c = lane & 3, full = NT / 2;
+    if (e < 4 * full) { m = 16 * i + 8 * (e & 1) + g; r = 16 * (e >> 2) + 8 * ((e >> 1) & 1) + 2 * c + h; }
+    else              { m = 16 * i + 8 * (e - 4 * full) + g; r = 16 * full + 2 * c + h; }
+    return true;
+}
+__host__ __device__ inline bool int4_b_elem(int K, int NT, int lane, int n, int h, int &k, int &r) {
+    if (n >= NT * (K / 8)) return false;
+    const int j = n / (K / 8), rem = n % (K / 8), g = lane >> 2, c = lane & 3;
+    r = 8 * j + g;
+    k = 16 * (rem >> 1) + 8 * (rem & 1) + 2 * c + h;
+    return true;
+}
 
 #ifdef __CUDACC__
 // Value of one factor element as attention reads it.  which: 0 = A_k(r, token i), 1 = B_k(r, channel i),
@@ -146,16 +187,21 @@ __host__ __device__ inline int int4_nibble_shift(int e) { return 4 * ((e >> 1) +
 // bf16(code * scale) with the scale of the element's column or row (see Geometry).
 __device__ inline float blob_value(const Geometry &g, const unsigned char *blob, int which, int r, int i) {
     const int P = g.page;
-    int off;                                   // byte offset in the bf16 form
-    if (which == 0) off = g.ak_off + a_t_offset(P, r, i);
-    else if (which == 2) off = g.av_off + a_t_offset(P, r, i);
-    else off = (which == 1 ? g.bk_off : g.bv_off) + r * kRowBytes + swz_chunk(r, i >> 3) * 16 + (i & 7) * 2;
     if (g.factor_bits != 4) {
+        int off;
+        if (which == 0) off = g.ak_off + a_t_offset(P, r, i);
+        else if (which == 2) off = g.av_off + a_t_offset(P, r, i);
+        else off = (which == 1 ? g.bk_off : g.bv_off) + r * kRowBytes + swz_chunk(r, i >> 3) * 16 + (i & 7) * 2;
         const unsigned short raw = *reinterpret_cast<const unsigned short *>(blob + off);
         return __uint_as_float((unsigned)raw << 16);
     }
-    const unsigned word = reinterpret_cast<const unsigned *>(blob)[off >> 4];
-    const int code = (int)((word >> int4_nibble_shift((off & 15) >> 1)) & 0xFu) - 8;
+    int w, shift, region;
+    if (which == 0)      { int4_a_pos(g.rank_tiles, i, r, w, shift); region = g.cak_off; }
+    else if (which == 1) { int4_b_pos(kHeadDim, i, r, w, shift);     region = g.cbk_off; }
+    else if (which == 2) { int4_b_pos(P, i, r, w, shift);            region = g.cav_off; }
+    else                 { int4_a_pos(g.rank_tiles, i, r, w, shift); region = g.cbv_off; }
+    const unsigned word = reinterpret_cast<const unsigned *>(blob + region)[w];
+    const int code = (int)((word >> shift) & 0xFu) - 8;
     const int soff = which == 0 ? g.sak_off + 2 * r : which == 1 ? g.sbk_off + 2 * i
                    : which == 2 ? g.sav_off + 2 * i : g.sbv_off + 2 * i;
     const unsigned short sraw = *reinterpret_cast<const unsigned short *>(blob + g.codes_bytes + soff);

@@ -335,8 +335,8 @@ def test_overlap_modes_stay_correct_when_appends_and_compressions_are_interleave
 
 @pytest.mark.parametrize("P,rk,rv,G", [(32, 16, 14, 4), (64, 24, 24, 8), (16, 9, 9, 4), (64, 8, 8, 2)])
 def test_int4_factors(P, rk, rv, G):
-    """INT4 factor storage (Section 4.3): the GPU quantizes in the compression kernel and unpacks in the decode
-    kernel.  Kernel gate: the oracle attends over the GPU's own dequantised factors (<= 1e-2).  Factor gate: the
+    """INT4 factor storage (Section 4.3): the GPU quantizes in the compression kernel and dequantises in the
+    decode kernel's registers.  Kernel gate: the oracle attends over the GPU's own dequantised factors (<= 1e-2).  Factor gate: the
     GPU's quantized reconstruction error is no worse than the oracle's INT4 error for the same page (x1.15).
     End to end against the oracle's INT4 cache: 1e-2 + 3 x the error INT4 causes inside the oracle."""
     import copy
@@ -349,7 +349,10 @@ def test_int4_factors(P, rk, rv, G):
                           factor_bits=4)
     sz = pkv.pkv_query_sizes(cfg)
     ratio = sz.factor_slot_bytes / sz.dense_slot_bytes
-    assert abs(ratio - quant.int4_page_storage_ratio(rk, rv, P, 128)) <= 40.0 / (2 * P * 128 * 2)      # padding only
+    # the pool stores ranks in tiles of 8 (zero codes past the true rank); apart from that, padding only
+    rk8, rv8 = -(-rk // 8) * 8, -(-rv // 8) * 8
+    padded = quant.int4_page_storage_ratio(rk, rv, P, 128) + ((rk8 - rk) + (rv8 - rv)) * (P + 128) / 2 / (2 * P * 128 * 2)
+    assert abs(ratio - padded) <= 160.0 / (2 * P * 128 * 2), (ratio, padded)
     pair = Pair(cfg, seed=P + rk + 1)
     ocfg16 = copy.copy(pair.orc.cfg)
     ocfg16.factor_bits = 16
