@@ -40,6 +40,10 @@ WORKLOADS = {
     # one sink page, last completed page + incomplete page dense
     "qwen3_8b_16k_paper_default": dict(n_layers=36, n_kv_heads=8, n_q_heads=32, batch=1, T=16384 + 17, rank=16,
                                        rank_v=14, page=32, sink=32, recent=32, ragged=False, outliers=0.0),
+    # BASELINE config 3: serving loop.  Prompts are prefilled and compressed; a step is append (one token per
+    # sequence) -> decode -> compress_eligible, so every 64th step factorizes one page per (sequence, KV head, K|V)
+    "serving_b32_8k": dict(n_layers=1, n_kv_heads=8, n_q_heads=32, batch=32, T=8192, rank=24, sink=64, recent=256,
+                           ragged=False, outliers=0.0, serving=True),
     # BASELINE config 0: tiny (L2-resident; latency only)
     "tiny": dict(n_layers=1, n_kv_heads=1, n_q_heads=4, batch=1, T=1024, rank=16, sink=64, recent=128,
                  ragged=False, outliers=0.0),
@@ -99,8 +103,10 @@ class ClockSampler:
                 "reasons": reasons, "samples": len(sm)}
 
 
-def build_workload(w, rank, device, overlap=2, n_ctas=0, factor_bits=16):
-    """Allocate the cache, generate each (layer, sequence) on the GPU, append and compress layer by layer."""
+def build_workload(w, rank, device, overlap=2, n_ctas=0, factor_bits=16, grow=0, keep_kv=False):
+    """Allocate the cache, generate each (layer, sequence) on the GPU, append and compress layer by layer.
+    grow: tokens every sequence may still gain afterwards (sizes the pools and page tables); keep_kv: also
+    return the generated K/V of layer 0 including those `grow` tokens (serving loop)."""
     import torch
     from paper_2608_23843_b200 import pkv, synth
     P = w.get("page", 64)
@@ -108,9 +114,9 @@ def build_workload(w, rank, device, overlap=2, n_ctas=0, factor_bits=16):
         lengths = synth.loguniform_lengths(SEED, w["batch"], *w["T"])
     else:
         lengths = [w["T"]] * w["batch"]
-    pages = [-(-t // P) for t in lengths]
+    pages = [-(-(t + grow) // P) for t in lengths]
     n_sink, n_win = w["sink"] // P, w["recent"] // P
-    n_factor = [max(0, t // P - n_win - n_sink) for t in lengths]
+    n_factor = [max(0, (t + grow) // P - n_win - n_sink) for t in lengths]
     L = w["n_layers"]
     n_factor_slots = L * sum(n_factor) + 1
     # dense slots: what stays dense in every layer plus one layer's worth of transient pages
@@ -124,10 +130,13 @@ def build_workload(w, rank, device, overlap=2, n_ctas=0, factor_bits=16):
                       synth.slot_permutation(SEED, n_factor_slots, 1).tolist())
     ids = list(range(w["batch"]))
     svd_ms, n_svds = 0.0, 0
+    kept = []
     for layer in range(L):
         for s in ids:
-            k, v = synth.make_kv(SEED, layer, s, lengths[s], w["n_kv_heads"], 128, P, device, w["outliers"])
-            cache.append_kv(layer, [s], [lengths[s]], k, v)
+            k, v = synth.make_kv(SEED, layer, s, lengths[s] + grow, w["n_kv_heads"], 128, P, device, w["outliers"])
+            cache.append_kv(layer, [s], [lengths[s]], k[:lengths[s]], v[:lengths[s]])
+            if keep_kv and layer == 0:
+                kept.append((k[lengths[s]:].clone(), v[lengths[s]:].clone()))
             del k, v
         e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
         e0.record()
@@ -136,8 +145,142 @@ def build_workload(w, rank, device, overlap=2, n_ctas=0, factor_bits=16):
         torch.cuda.synchronize()
         svd_ms += e0.elapsed_time(e1)
         n_svds += n * w["n_kv_heads"] * 2
-    return cfg, cache, lengths, dict(pages_per_s=(n_svds / (svd_ms * 1e-3) if svd_ms > 0 else None), n_page_svds=n_svds,
-                                     svd_ms=svd_ms)
+    comp = dict(pages_per_s=(n_svds / (svd_ms * 1e-3) if svd_ms > 0 else None), n_page_svds=n_svds, svd_ms=svd_ms)
+    if keep_kv:
+        comp["new_k"] = torch.stack([k for k, _ in kept], 1).contiguous()      # [grow][batch][H_kv][d]
+        comp["new_v"] = torch.stack([v for _, v in kept], 1).contiguous()
+    return cfg, cache, lengths, comp
+
+
+def run_serving(args, w, rank, device, world, rk, local):
+    """BASELINE config 3: `steps` iterations of append (one token per sequence) -> decode -> compress on one
+    layer, timed as a whole and call by call with CUDA events on the launching stream."""
+    import torch
+    from paper_2608_23843_b200 import synth
+    B, Hq, P = w["batch"], w["n_q_heads"], w.get("page", 64)
+    warm = max(3, args.warmup)
+    total = warm + 2 * args.steps + 3           # device-resident pass, host-buffer pass, warm-ups
+    cfg, cache, lengths, comp = build_workload(w, rank, device, 0, args.n_ctas, args.factor_bits, grow=total, keep_kv=True)
+    ids = list(range(B))
+    new_k, new_v = comp["new_k"], comp["new_v"]
+    qs = [synth.make_q(SEED, 0, t, B, Hq, 128, device) for t in range(8)]
+    out = torch.empty_like(qs[0])
+    cursor = [0]
+    events = []
+
+    def step(record):
+        t = cursor[0]
+        cursor[0] += 1
+        ev = [torch.cuda.Event(enable_timing=True) for _ in range(4)] if record else None
+        if record:
+            ev[0].record()
+        cache.append_kv(0, ids, [1] * B, new_k[t], new_v[t])
+        if record:
+            ev[1].record()
+        cache.decode_attention(0, ids, qs[t % 8], out)
+        if record:
+            ev[2].record()
+        n = cache.compress_eligible_pages(0)
+        if record:
+            ev[3].record()
+            events.append((ev, n))
+
+    def barrier():
+        if world > 1:
+            import torch.distributed as dist
+            dist.barrier()
+        torch.cuda.synchronize()
+
+    for _ in range(warm):
+        step(False)
+    cache.decode_attention(0, ids, qs[0], out)
+    bytes_per_step = cache.stats()["last_decode_bytes"]
+    sampler = ClockSampler(local)
+    sampler.start()
+    barrier()
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    e0.record()
+    for _ in range(args.steps):
+        step(True)
+    e1.record()
+    barrier()
+    clocks = sampler.stop()
+    ms = e0.elapsed_time(e1) / args.steps
+    app = [ev[0].elapsed_time(ev[1]) * 1e3 for ev, _ in events]
+    att = [ev[1].elapsed_time(ev[2]) * 1e3 for ev, _ in events]
+    cmp_all = [(ev[2].elapsed_time(ev[3]) * 1e3, n) for ev, n in events]
+    cmp_event = [(us, n) for us, n in cmp_all if n > 0]
+
+    def pct(xs, p):
+        xs = sorted(xs)
+        return xs[min(len(xs) - 1, int(p * len(xs)))] if xs else None
+
+    # end to end: the step's new K/V rows and q come from pinned host memory, the result goes back to it
+    hk, hv = new_k.cpu().pin_memory(), new_v.cpu().pin_memory()
+    hq = [q.cpu().pin_memory() for q in qs]
+    hout = torch.empty_like(hq[0]).pin_memory()
+    dk, dv = torch.empty_like(new_k[0]), torch.empty_like(new_v[0])
+    q_stage, out_stage = torch.empty_like(qs[0]), torch.empty_like(qs[0])
+
+    def step_host():
+        t = cursor[0]
+        cursor[0] += 1
+        dk.copy_(hk[t], non_blocking=True)
+        dv.copy_(hv[t], non_blocking=True)
+        cache.append_kv(0, ids, [1] * B, dk, dv)
+        cache.decode_attention_host(0, ids, hq[t % 8], hout, q_stage, out_stage)
+        cache.compress_eligible_pages(0)
+        torch.cuda.current_stream().synchronize()
+
+    for _ in range(3):
+        step_host()
+    barrier()
+    t0 = time.perf_counter()
+    for _ in range(args.steps):
+        step_host()
+    barrier()
+    e2e_ms = (time.perf_counter() - t0) * 1e3 / args.steps
+    st = cache.stats()
+    if st["device_timeouts"] or st["bad_slot_indices"] or out.float().isnan().any().item():
+        raise SystemExit("decode produced timeouts or NaNs: %r" % st)
+    att_mean = statistics.mean(att)
+    ms, e2e_ms, att_mean = max_over_ranks([ms, e2e_ms, att_mean], world, device)
+    if rk == 0:
+        peak, peak_src = _peaks()
+        achieved = bytes_per_step / (att_mean * 1e-6) / 1e9
+        n_event_svds = sum(n for _, n in cmp_event) * w["n_kv_heads"] * 2
+        step_bytes = 2 * B * w["n_kv_heads"] * 128 * 2 + 2 * B * Hq * 128 * 2
+        line = {
+            "metric": "decode_us_per_step", "value": ms * 1e3, "unit": "us", "n_gpus": world, "steps": args.steps,
+            "warmup": warm, "ms_per_step": ms, "higher_is_better": False, "scaling": "weak", "vs_baseline": None,
+            "dtype": "bf16", "data": "synthetic", "config": dict(_config_dict(args, w, rank),
+                step="append (1 token per sequence) + decode + compress_eligible on one layer", overlap="0"),
+            "append_us": {"mean": statistics.mean(app), "p99": pct(app, 0.99)},
+            "attention_us": {"mean": statistics.mean(att), "p99": pct(att, 0.99)},
+            "compress_us": {"mean_no_event": statistics.mean([us for us, n in cmp_all if n == 0] or [0.0]),
+                            "mean_event": statistics.mean([us for us, _ in cmp_event]) if cmp_event else None,
+                            "event_steps": len(cmp_event),
+                            "pages_per_s_event": (n_event_svds / (sum(us for us, _ in cmp_event) * 1e-6)) if cmp_event else None},
+            "step_us_p99": pct([a + b + c for a, b, (c, _) in zip(app, att, cmp_all)], 0.99),
+            "algorithmic_bytes_per_step": bytes_per_step,
+            "pages_factorized_per_s": comp["pages_per_s"], "page_svds_timed": comp["n_page_svds"],
+            "roofline": {"bound": "hbm", "kernel": "decode_tc_kernel<P=%d, rank tiles=%d>" % (P, (rank + 7) // 8),
+                         "achieved": achieved, "peak": peak, "unit": "GB/s", "frac": achieved / peak,
+                         "peak_source": peak_src, "traffic": bytes_per_step * NCU_TRAFFIC_PER_ALGORITHMIC_BYTE,
+                         "traffic_source": "ncu dram__bytes_read+write of this kernel on the llama3_8b_32k_b8 launch, "
+                                           "scaled by algorithmic bytes",
+                         "launch_us": att_mean, "algorithmic_bytes_per_launch": bytes_per_step},
+            "e2e": {"value": e2e_ms * 1e3, "unit": "us", "h2d_bytes_per_step": step_bytes - B * Hq * 128 * 2,
+                    "d2h_bytes_per_step": B * Hq * 128 * 2},
+            "gpu_launches": args.steps * 2 + len(cmp_event), "clocks": clocks,
+        }
+        if not args.no_cpu_baseline and world == 1:
+            o = oracle_sample(w, rank, 3, args.factor_bits)
+            line["cpu_baseline"] = {"value": o["decode_s"] * 1e6 * o["slices_per_step"], "unit": "us",
+                                    "cores": o["cores"], "kind": "oracle", "sample": o["sample"] + " (attention only)",
+                                    "pages_per_s": o["pages_per_s"]}
+        print(json.dumps(line))
+    cache.close()
 
 
 def oracle_sample(w, rank, steps, factor_bits=16):
@@ -251,6 +394,11 @@ def main():
         dist.init_process_group("nccl", device_id=device)
     pkv.lib()                                             # fail loudly if the CUDA library is missing
 
+    if w.get("serving"):
+        run_serving(args, w, rank, device, world, rk, local)
+        if world > 1:
+            dist.destroy_process_group()
+        return
     cfg, cache, lengths, comp = build_workload(w, rank, device, args.overlap, args.n_ctas, args.factor_bits)
     ids = list(range(w["batch"]))
     L, Hq = w["n_layers"], w["n_q_heads"]

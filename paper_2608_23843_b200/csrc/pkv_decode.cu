@@ -339,11 +339,13 @@ struct WarpState {
 
 // Shapes fixed at compile time: P tokens per page, NT = ceil(rank / 8) rank tiles (K and V alike), I4 = factors
 // stored as INT4 codes.
-template <int P, int NT, bool I4 = false>
+// rows per dense block: 32 where a stage has to be that large for a bf16 factor page anyway
+template <int P, int NT, bool I4>
+constexpr int kDenseBlock = (!I4 && P >= 32 && NT >= 3) ? 32 : 16;
+
+template <int P, int NT>
 struct Tc {
     static constexpr int kMT = P / 16;                                  // 16-token tiles per page
-    // rows per dense block: 32 where a stage has to be that large for a bf16 factor page anyway
-    static constexpr int kDB = (!I4 && P >= 32 && NT >= 3) ? 32 : 16;
     static constexpr int kPitchA = 2 * P;                               // bytes per A^T row
 };
 
@@ -744,24 +746,47 @@ __device__ __forceinline__ void flush_segment(const DecodeArgs &a, float *comb, 
         if (*last_flag) {
             __threadfence();
             const float *first = a.partials + ((long long)ps.cta_first + seg) * kPartialFloats;
-            for (int item = ctid; item < a.geo.group * 32; item += kThreads) {
-                const int hq = item >> 5, d4 = (item & 31) * 4;
-                float Mg = kNegInf;
-#pragma unroll 8
-                for (int k = 0; k < ps.n_parts; ++k)
-                    Mg = fmaxf(Mg, __ldcg(first + (long long)k * kPartialFloats + kMaxGroup * kHeadDim + hq));
-                float4 tot = make_float4(0.f, 0.f, 0.f, 0.f);
-                float Lg = 0.f;
-#pragma unroll 8
-                for (int k = 0; k < ps.n_parts; ++k) {
-                    const float *pk = first + (long long)k * kPartialFloats;
-                    const float f = exp2f(__ldcg(pk + kMaxGroup * kHeadDim + hq) - Mg);
-                    const float4 o = __ldcg(reinterpret_cast<const float4 *>(pk + hq * kHeadDim + d4));
-                    tot.x += f * o.x; tot.y += f * o.y; tot.z += f * o.z; tot.w += f * o.w;
-                    Lg += f * __ldcg(pk + kMaxGroup * kHeadDim + kMaxGroup + hq);
+            // A thread owns items ctid and ctid + kThreads and walks the parts in CTA order with a running
+            // maximum (one pass); eight parts' loads are in flight at a time, because with dozens of parts
+            // it is the latency of these loads that the rest of the GPU waits for.
+            constexpr int kBatch = 8;
+            const int n_items = a.geo.group * 32, np = ps.n_parts;
+            const bool has[2] = {ctid < n_items, ctid + kThreads < n_items};
+            const int hq[2] = {has[0] ? ctid >> 5 : 0, has[1] ? (ctid + kThreads) >> 5 : 0};
+            const int d4 = (ctid & 31) * 4;                       // kThreads is a multiple of 32
+            float4 tot[2] = {make_float4(0.f, 0.f, 0.f, 0.f), make_float4(0.f, 0.f, 0.f, 0.f)};
+            float Mr[2] = {kNegInf, kNegInf}, Lr[2] = {0.f, 0.f};
+            for (int k0 = 0; k0 < np; k0 += kBatch) {
+                float4 o[2][kBatch];
+                float m[2][kBatch], l[2][kBatch];
+#pragma unroll
+                for (int j = 0; j < kBatch; ++j) {
+                    const float *pk = first + (long long)min(k0 + j, np - 1) * kPartialFloats;
+#pragma unroll
+                    for (int e = 0; e < 2; ++e) {
+                        o[e][j] = __ldcg(reinterpret_cast<const float4 *>(pk + hq[e] * kHeadDim + d4));
+                        m[e][j] = __ldcg(pk + kMaxGroup * kHeadDim + hq[e]);
+                        l[e][j] = __ldcg(pk + kMaxGroup * kHeadDim + kMaxGroup + hq[e]);
+                    }
                 }
-                store_out(a, seg, hq, d4, tot, Lg);
+#pragma unroll
+                for (int j = 0; j < kBatch; ++j) {
+                    if (k0 + j < np) {
+#pragma unroll
+                        for (int e = 0; e < 2; ++e) {
+                            const float Mn = fmaxf(Mr[e], m[e][j]);
+                            const float fa = exp2f(Mr[e] - Mn), fb = exp2f(m[e][j] - Mn);
+                            tot[e].x = tot[e].x * fa + fb * o[e][j].x; tot[e].y = tot[e].y * fa + fb * o[e][j].y;
+                            tot[e].z = tot[e].z * fa + fb * o[e][j].z; tot[e].w = tot[e].w * fa + fb * o[e][j].w;
+                            Lr[e] = Lr[e] * fa + fb * l[e][j];
+                            Mr[e] = Mn;
+                        }
+                    }
+                }
             }
+#pragma unroll
+            for (int e = 0; e < 2; ++e)
+                if (has[e]) store_out(a, seg, hq[e], d4, tot[e], Lr[e]);
             if (ctid == 0) a.tickets[seg] = 0;          // ready for the next launch
         }
     }
@@ -770,7 +795,7 @@ __device__ __forceinline__ void flush_segment(const DecodeArgs &a, float *comb, 
 
 template <int P, int NT, bool I4>
 __global__ void __launch_bounds__(kDecodeThreads, 2) decode_tc_kernel(const __grid_constant__ DecodeArgs a) {
-    using C = Tc<P, NT, I4>;
+    constexpr int kDB = kDenseBlock<P, NT, I4>;
     Range rg;
     if (!load_range(a, rg)) return;
     const Geometry &geo = a.geo;
@@ -853,9 +878,9 @@ __global__ void __launch_bounds__(kDecodeThreads, 2) decode_tc_kernel(const __gr
                         rows = P;
                         src = a.factor_pool + (long long)slot * geo.factor_slot_bytes + (long long)cur.head * geo.blob_bytes;
                     } else {
-                        rows = max(0, min(C::kDB, T - page * P - blk * C::kDB));
+                        rows = max(0, min(kDB, T - page * P - blk * kDB));
                         src = a.dense_pool + (long long)slot * geo.dense_slot_bytes +
-                              (long long)cur.head * geo.dense_head_bytes + blk * C::kDB * kRowBytes;
+                              (long long)cur.head * geo.dense_head_bytes + blk * kDB * kRowBytes;
                     }
                 }
                 // Lanes arm their own units, S at a time (one stage each); the counter of armed units is
@@ -877,7 +902,7 @@ __global__ void __launch_bounds__(kDecodeThreads, 2) decode_tc_kernel(const __gr
                             } else if (rows > 0) {
                                 mbar_arrive_expect_tx(bar, 2 * rows * kRowBytes);
                                 bulk_g2s(dst, src, rows * kRowBytes, bar);
-                                bulk_g2s(dst + C::kDB * kRowBytes, src + P * kRowBytes, rows * kRowBytes, bar);
+                                bulk_g2s(dst + kDB * kRowBytes, src + P * kRowBytes, rows * kRowBytes, bar);
                             } else {
                                 mbar_arrive(bar);
                             }
@@ -945,7 +970,7 @@ __global__ void __launch_bounds__(kDecodeThreads, 2) decode_tc_kernel(const __gr
                 if (cur_seg < rg.n_local_segs) load_q(a, rg.seg_first + cur_seg, qf, lane);
             }
             if (dsc.kind == kKindEnd) break;
-            dsc.rows = min(dsc.rows, dsc.kind == kKindFactor ? P : C::kDB);
+            dsc.rows = min(dsc.rows, dsc.kind == kKindFactor ? P : kDB);
             if (dsc.rows > 0) {
                 const uint32_t sb = smem_u32(stages + (size_t)s * stage_bytes);
                 if (dsc.kind == kKindFactor) {
@@ -953,8 +978,8 @@ __global__ void __launch_bounds__(kDecodeThreads, 2) decode_tc_kernel(const __gr
                     else factor_unit<P, NT>(sb, geo.ak_off, geo.bk_off, geo.av_off, geo.bv_off, geo.rank_k, geo.rank_v, qf,
                                             geo.scale_log2e, st, lane);
                 } else {
-                    dense_unit<C::kDB>(sb, stages + (size_t)s * stage_bytes, dsc.rows, qf, geo.scale_log2e, st, lane);
-                    if (dsc.rows < C::kDB) asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+                    dense_unit<kDB>(sb, stages + (size_t)s * stage_bytes, dsc.rows, qf, geo.scale_log2e, st, lane);
+                    if (dsc.rows < kDB) asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
                 }
             }
             __syncwarp();
