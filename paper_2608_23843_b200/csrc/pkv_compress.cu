@@ -1,7 +1,7 @@
 // Batched per-page truncated SVD (paper: Eq. 2 and the Gram-matrix route that
 // follows Eq. 3).  One CTA factorizes one P x d page X (K or V of one KV head):
 //   G = X X^T (P x P, fp32, exact bf16 products)        -> shared memory
-//   cyclic Jacobi eigen-solve of G with Q accumulating the rotations (fp32)
+//   cyclic Jacobi eigen-solve of G with Q^T accumulating the rotations (fp32)
 //   A = the r eigenvectors of largest eigenvalue, B = A^T X, both rounded to bf16
 // Pages are independent, so the grid is simply (work-list entries) x (KV heads) x (K|V).
 #include <cuda_bf16.h>
@@ -24,20 +24,28 @@ template <int P>
 struct Shape {
     static constexpr int kThreads = 4 * P;              // 256 / 128 / 64
     static constexpr int kWarps = kThreads / 32;
-    static constexpr int kGs = P + 1;                   // padded row stride of G and Q (floats)
-    static constexpr int kPairsPerWarp = (P / 2) / kWarps;   // = 4 for every P
-    static constexpr int kHalves = (P + 31) / 32;       // 32-row groups a warp walks in the column phase
-    // 2 x 2 block update of G: lanes run over the column pair b, a warp covers kRowPairsPerIter row pairs at once
-    static constexpr int kLanesPerRowPair = (P / 2) < 32 ? (P / 2) : 32;
-    static constexpr int kRowPairsPerIter = 32 / kLanesPerRowPair;
-    static constexpr int kBlockIters = (P / 2) / (kWarps * kRowPairsPerIter);
+    // Row stride of G (floats).  Not padded on purpose: the bank of G[i][j] is then j mod 32 alone, which is what
+    // makes the block update below conflict-free (see there).
+    static constexpr int kGs = P;
+    static constexpr int kPairs = P / 2;
+    // 2 x 2 blocks of G computed per round: one of each mirror-image couple, and the diagonal blocks
+    static constexpr int kBlocks = kPairs * (kPairs / 2) + kPairs / 2;
+    static constexpr int kChunks = P / 4;               // float4 chunks of a row of Q^T
 };
 
+// The page X is needed for the Gram matrix and again for B = A^T X; in between its bytes hold Q^T, and it is
+// fetched a second time (from L2, most likely) into the bytes of G once the eigenvalues are known: two P x P
+// fp32 arrays per page instead of three let more pages share an SM.
 template <int P>
 struct CompressSmem {
-    float G[P * (P + 1)];
-    float Q[P * (P + 1)];
-    __nv_bfloat16 X[P * kXs];
+    union {
+        __nv_bfloat16 X[P * kXs];      // load and Gram phases (padded rows)
+        float QT[P * P];               // Q^T: row j = eigenvector candidate j (16-byte aligned rows)
+    };
+    union {
+        float G[P * P];
+        __nv_bfloat16 X2[P * kHeadDim];    // the page again, rows unpadded (projection phase)
+    };
     float2 cs[P / 2];
     uchar2 pairs[(P - 1) * (P / 2)];   // this page size's rows of c_pairs (lanes index it divergently)
     float lam[P];
@@ -80,7 +88,7 @@ __global__ void __launch_bounds__(Shape<P>::kThreads)
 compress_kernel(Geometry geo, const unsigned char *dense_pool, unsigned char *factor_pool,
                 const int2 *worklist, int *status) {
     using Sh = Shape<P>;
-    constexpr int kGs = Sh::kGs, kThreads = Sh::kThreads, kWarps = Sh::kWarps;
+    constexpr int kGs = Sh::kGs, kThreads = Sh::kThreads, kWarps = Sh::kWarps, kPairs = Sh::kPairs;
     extern __shared__ __align__(16) unsigned char smem_raw[];
     CompressSmem<P> &S = *reinterpret_cast<CompressSmem<P> *>(smem_raw);
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
@@ -127,17 +135,15 @@ compress_kernel(Geometry geo, const unsigned char *dense_pool, unsigned char *fa
 #pragma unroll
         for (int u = 0; u < 4; ++u)
 #pragma unroll
-            for (int w = 0; w < 4; ++w) {
-                S.G[(4 * ti + u) * kGs + 4 * tj + w] = acc[u][w];
-                S.Q[(4 * ti + u) * kGs + 4 * tj + w] = (4 * ti + u == 4 * tj + w) ? 1.f : 0.f;
-            }
+            for (int w = 0; w < 4; ++w) S.G[(4 * ti + u) * kGs + 4 * tj + w] = acc[u][w];
     }
     __syncthreads();
-    // the upper triangle was computed in a different summation order than the lower: symmetrise exactly
-    for (int i = tid; i < P * P; i += kThreads) {
-        const int r = i / P, c = i % P;
-        if (r > c) S.G[r * kGs + c] = S.G[c * kGs + r];
+    for (int i = tid; i < P * P / 4; i += kThreads) {          // Q^T = I, over the bytes of X
+        const int r = i / (P / 4), c4 = (i % (P / 4)) * 4;
+        reinterpret_cast<float4 *>(S.QT)[i] = make_float4(r == c4 ? 1.f : 0.f, r == c4 + 1 ? 1.f : 0.f,
+                                                          r == c4 + 2 ? 1.f : 0.f, r == c4 + 3 ? 1.f : 0.f);
     }
+    // G[i][j] and G[j][i] were accumulated from the same products in the same order: G is bitwise symmetric
     // absolute floor below which an off-diagonal entry is rounding noise of the Gram matrix
     float dmax = 0.f;
     if (tid < P) dmax = fabsf(S.G[tid * kGs + tid]);
@@ -163,18 +169,27 @@ compress_kernel(Geometry geo, const unsigned char *dense_pool, unsigned char *fa
 
     // ---- cyclic Jacobi sweeps ----
     // The P/2 rotations of a round act on disjoint index pairs, so G' = J^T G J splits into (P/2)^2 independent
-    // 2 x 2 blocks: block (a, b) = rows of pair a, columns of pair b, becomes J_a^T . block . J_b.  One thread
-    // owns a block, reads and writes only its four entries, and G passes through shared memory once per round.
-    // Blocks below the diagonal are computed as the transpose of their mirror image (G stays bitwise symmetric).
-    for (int i = tid; i < (P - 1) * (P / 2); i += kThreads) S.pairs[i] = c_pairs[pair_table_offset(P) + i];
+    // 2 x 2 blocks: block (a, b) = rows of pair a, columns of pair b, becomes J_a^T . block . J_b.  G is
+    // symmetric, so one block of every mirror-image couple is computed: a thread reads its block's four entries
+    // and writes them and their mirror images (G stays bitwise symmetric), so G passes through shared memory once
+    // per round.  Lanes walk a wrapped diagonal, block (a, a + delta mod P/2) for lane a: delta = 0 .. P/4 covers
+    // every couple once (delta = P/4 with a < P/4 only).  On a diagonal the lanes' row pairs are all different
+    // and so are their column pairs; the bank of an entry is its column index mod 32 and the oriented pair table
+    // keeps a round's first members (and its second members) in different banks, so neither the block accesses
+    // (bank = a member of the column pair) nor the mirrored stores (bank = a member of the row pair) conflict.
+    // For P < 64 a warp holds several diagonals; every other one takes its pairs in the opposite order, (q, p)
+    // with the rotation (c, -s), which is the same rotation, so that it touches second members while its
+    // neighbour touches first members.
+    // Q^T is stored instead of Q: rotating columns p, q of Q is rotating rows p, q of Q^T, four tokens at a time.
+    for (int i = tid; i < (P - 1) * kPairs; i += kThreads) S.pairs[i] = c_pairs[pair_table_offset(P) + i];
     __syncthreads();
     const uchar2 *pairs = S.pairs;
     bool converged = false;
     for (int sweep = 0; sweep < geo.jacobi_max_sweeps && !converged; ++sweep) {
         int rotated = 0;
         for (int rho = 0; rho < P - 1; ++rho) {
-            const uchar2 *pr = pairs + rho * (P / 2);
-            if (tid < P / 2) {
+            const uchar2 *pr = pairs + rho * kPairs;
+            if (tid < kPairs) {
                 const int p = pr[tid].x, q = pr[tid].y;
                 const float gpp = S.G[p * kGs + p], gqq = S.G[q * kGs + q], gpq = S.G[p * kGs + q];
                 float c = 1.f, s = 0.f;
@@ -188,47 +203,50 @@ compress_kernel(Geometry geo, const unsigned char *dense_pool, unsigned char *fa
                 S.cs[tid] = make_float2(c, s);
             }
             __syncthreads();
-            {
-                const int bb = lane % Sh::kLanesPerRowPair;
-                const uchar2 pb = pr[bb];
-                const float2 cb = S.cs[bb];
 #pragma unroll
-                for (int it = 0; it < Sh::kBlockIters; ++it) {
-                    const int aa = warp * Sh::kRowPairsPerIter + lane / Sh::kLanesPerRowPair +
-                                   it * (kWarps * Sh::kRowPairsPerIter);
-                    const uchar2 pa = pr[aa];
-                    const float2 ca = S.cs[aa];
-                    if (ca.y == 0.f && cb.y == 0.f) continue;
-                    float x00 = S.G[pa.x * kGs + pb.x], x01 = S.G[pa.x * kGs + pb.y];
-                    float x10 = S.G[pa.y * kGs + pb.x], x11 = S.G[pa.y * kGs + pb.y];
-                    const bool lower = aa > bb;
-                    const float cl = lower ? cb.x : ca.x, sl = lower ? cb.y : ca.y;     // applied first
-                    const float cr = lower ? ca.x : cb.x, sr = lower ? ca.y : cb.y;     // applied second
-                    if (lower) { const float t = x01; x01 = x10; x10 = t; }
-                    const float y00 = cl * x00 - sl * x10, y01 = cl * x01 - sl * x11;
-                    const float y10 = sl * x00 + cl * x10, y11 = sl * x01 + cl * x11;
-                    float z00 = cr * y00 - sr * y01, z01 = sr * y00 + cr * y01;
-                    float z10 = cr * y10 - sr * y11, z11 = sr * y10 + cr * y11;
-                    if (lower) { const float t = z01; z01 = z10; z10 = t; }
-                    S.G[pa.x * kGs + pb.x] = z00; S.G[pa.x * kGs + pb.y] = z01;
-                    S.G[pa.y * kGs + pb.x] = z10; S.G[pa.y * kGs + pb.y] = z11;
+            for (int u0 = 0; u0 < Sh::kBlocks; u0 += kThreads) {
+                const int u = u0 + tid;
+                if (u < Sh::kBlocks) {
+                    const int delta = u / kPairs, ia = u % kPairs, ib = (ia + delta) % kPairs;
+                    float2 ca = S.cs[ia], cb = S.cs[ib];
+                    if (ca.y != 0.f || cb.y != 0.f) {
+                        uchar2 pa = pr[ia], pb = pr[ib];
+                        if (kPairs < 32 && (delta & 1)) {
+                            pa = make_uchar2(pa.y, pa.x); ca.y = -ca.y;
+                            pb = make_uchar2(pb.y, pb.x); cb.y = -cb.y;
+                        }
+                        float *g0 = S.G + pa.x * kGs, *g1 = S.G + pa.y * kGs;
+                        const float x00 = g0[pb.x], x01 = g0[pb.y], x10 = g1[pb.x], x11 = g1[pb.y];
+                        const float y00 = ca.x * x00 - ca.y * x10, y01 = ca.x * x01 - ca.y * x11;
+                        const float y10 = ca.y * x00 + ca.x * x10, y11 = ca.y * x01 + ca.x * x11;
+                        const float z00 = cb.x * y00 - cb.y * y01, z01 = cb.y * y00 + cb.x * y01;
+                        const float z10 = cb.x * y10 - cb.y * y11, z11 = cb.y * y10 + cb.x * y11;
+                        if (delta != 0) {
+                            g0[pb.x] = z00; g0[pb.y] = z01; g1[pb.x] = z10; g1[pb.y] = z11;
+                            float *h0 = S.G + pb.x * kGs, *h1 = S.G + pb.y * kGs;
+                            h0[pa.x] = z00; h1[pa.x] = z01; h0[pa.y] = z10; h1[pa.y] = z11;
+                        } else {                       // diagonal block: x01 = x10, and so are their images
+                            g0[pb.x] = z00; g0[pb.y] = z01; g1[pb.x] = z01; g1[pb.y] = z11;
+                        }
+                    }
                 }
             }
-            // columns p, q of Q:  x_p' = c x_p - s x_q,  x_q' = s x_p + c x_q
+            // rows p, q of Q^T:  x_p' = c x_p - s x_q,  x_q' = s x_p + c x_q
 #pragma unroll
-            for (int kk = 0; kk < Sh::kPairsPerWarp; ++kk) {
-                const int k = warp + kk * kWarps;
-                const float2 cs = S.cs[k];
-                if (cs.y != 0.f) {
-                    const int p = pr[k].x, q = pr[k].y;
-#pragma unroll
-                    for (int half = 0; half < Sh::kHalves; ++half) {
-                        const int i = lane + 32 * half;
-                        if (i < P) {
-                            const float qp = S.Q[i * kGs + p], qq = S.Q[i * kGs + q];
-                            S.Q[i * kGs + p] = cs.x * qp - cs.y * qq;
-                            S.Q[i * kGs + q] = cs.y * qp + cs.x * qq;
-                        }
+            for (int i0 = 0; i0 < kPairs * Sh::kChunks; i0 += kThreads) {
+                const int item = i0 + tid;
+                if (item < kPairs * Sh::kChunks) {
+                    const int k = item / Sh::kChunks, ch = item % Sh::kChunks;
+                    const float2 cs = S.cs[k];
+                    if (cs.y != 0.f) {
+                        const uchar2 pq = pr[k];
+                        float4 *rp = reinterpret_cast<float4 *>(S.QT + pq.x * P) + ch;
+                        float4 *rq = reinterpret_cast<float4 *>(S.QT + pq.y * P) + ch;
+                        const float4 xp = *rp, xq = *rq;
+                        *rp = make_float4(cs.x * xp.x - cs.y * xq.x, cs.x * xp.y - cs.y * xq.y,
+                                          cs.x * xp.z - cs.y * xq.z, cs.x * xp.w - cs.y * xq.w);
+                        *rq = make_float4(cs.y * xp.x + cs.x * xq.x, cs.y * xp.y + cs.x * xq.y,
+                                          cs.y * xp.z + cs.x * xq.z, cs.y * xp.w + cs.x * xq.w);
                     }
                 }
             }
@@ -276,6 +294,13 @@ compress_kernel(Geometry geo, const unsigned char *dense_pool, unsigned char *fa
         S.order[r] = tid;       // r < P always; NaN eigenvalues may collide (outputs then unspecified)
     }
     __syncthreads();
+    // ---- the page again (G is no longer needed) ----
+    for (int i = tid; i < P * 16; i += kThreads) {
+        const int row = i >> 4, chunk = i & 15;
+        reinterpret_cast<uint4 *>(S.X2)[i] =
+            *reinterpret_cast<const uint4 *>(src + row * kRowBytes + swz_chunk(row, chunk) * 16);
+    }
+    __syncthreads();
 
     if (geo.factor_bits == 4) {
         // ---- INT4 factors (paper, Section 4.3): A~ = A Sigma^(1/2), B~ = Sigma^(-1/2) B, symmetric 4-bit codes ----
@@ -286,8 +311,8 @@ compress_kernel(Geometry geo, const unsigned char *dense_pool, unsigned char *fa
             float b0 = 0.f, b1 = 0.f;
 #pragma unroll 8
             for (int r = 0; r < P; ++r) {
-                const float a = S.Q[r * kGs + oj];
-                const float2 x = __bfloat1622float2(*reinterpret_cast<const __nv_bfloat162 *>(&S.X[r * kXs + col]));
+                const float a = S.QT[oj * P + r];
+                const float2 x = __bfloat1622float2(*reinterpret_cast<const __nv_bfloat162 *>(&S.X2[r * kHeadDim + col]));
                 b0 = fmaf(a, x.x, b0);
                 b1 = fmaf(a, x.y, b1);
             }
@@ -309,7 +334,7 @@ compress_kernel(Geometry geo, const unsigned char *dense_pool, unsigned char *fa
             if (tid < rank) {
                 const int oj = S.order[tid];
                 float m = 0.f;
-                for (int i = 0; i < P; ++i) m = fmaxf(m, fabsf(S.Q[i * kGs + oj]));
+                for (int i = 0; i < P; ++i) m = fmaxf(m, fabsf(S.QT[oj * P + i]));
                 const float sc = bf16_round(m * Z.root[tid] / 7.f);
                 Z.s_rank[tid] = sc;
                 *reinterpret_cast<__nv_bfloat16 *>(sc_base + geo.sak_off + 2 * tid) = __float2bfloat16_rn(sc);
@@ -318,7 +343,7 @@ compress_kernel(Geometry geo, const unsigned char *dense_pool, unsigned char *fa
             }
         } else if (tid < P) {
             float m = 0.f;
-            for (int j = 0; j < rank; ++j) m = fmaxf(m, fabsf(S.Q[tid * kGs + S.order[j]] * Z.root[j]));
+            for (int j = 0; j < rank; ++j) m = fmaxf(m, fabsf(S.QT[S.order[j] * P + tid] * Z.root[j]));
             const float sc = bf16_round(m / 7.f);
             Z.s_tok[tid] = sc;
             *reinterpret_cast<__nv_bfloat16 *>(sc_base + geo.sav_off + 2 * tid) = __float2bfloat16_rn(sc);
@@ -350,7 +375,7 @@ compress_kernel(Geometry geo, const unsigned char *dense_pool, unsigned char *fa
                 if (is_a) {
                     const bool ok = kv ? int4_b_elem(P, NT, ln, n, h, x, j) : int4_a_elem(P, NT, ln, n, h, x, j);
                     if (ok && j < rank)
-                        code = int4_code(S.Q[x * kGs + S.order[j]] * Z.root[j], kv ? Z.s_tok[x] : Z.s_rank[j]);
+                        code = int4_code(S.QT[S.order[j] * P + x] * Z.root[j], kv ? Z.s_tok[x] : Z.s_rank[j]);
                 } else {
                     const bool ok = kv ? int4_a_elem(kHeadDim, NT, ln, n, h, x, j) : int4_b_elem(kHeadDim, NT, ln, n, h, x, j);
                     if (ok && j < rank) code = int4_code(Z.B[j * kHeadDim + x] * Z.inv[j], Z.s_ch[x]);
@@ -365,7 +390,7 @@ compress_kernel(Geometry geo, const unsigned char *dense_pool, unsigned char *fa
     for (int i = tid; i < rank * (P / 2); i += kThreads) {
         const int j = i / (P / 2), tok = (i % (P / 2)) * 2;
         const int oj = S.order[j];
-        const float a0 = S.Q[tok * kGs + oj], a1 = S.Q[(tok + 1) * kGs + oj];
+        const float a0 = S.QT[oj * P + tok], a1 = S.QT[oj * P + tok + 1];
         *reinterpret_cast<__nv_bfloat162 *>(dstA + a_t_offset(P, j, tok)) = __floats2bfloat162_rn(a0, a1);
     }
     // ---- B = A^T X (fp32 eigenvectors, exact page), rows swizzled like dense rows ----
@@ -375,8 +400,8 @@ compress_kernel(Geometry geo, const unsigned char *dense_pool, unsigned char *fa
         float b0 = 0.f, b1 = 0.f;
 #pragma unroll 8
         for (int r = 0; r < P; ++r) {
-            const float a = S.Q[r * kGs + oj];
-            const float2 x = __bfloat1622float2(*reinterpret_cast<const __nv_bfloat162 *>(&S.X[r * kXs + col]));
+            const float a = S.QT[oj * P + r];
+            const float2 x = __bfloat1622float2(*reinterpret_cast<const __nv_bfloat162 *>(&S.X2[r * kHeadDim + col]));
             b0 = fmaf(a, x.x, b0);
             b1 = fmaf(a, x.y, b1);
         }
