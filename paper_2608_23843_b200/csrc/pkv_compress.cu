@@ -14,11 +14,18 @@ namespace {
 
 constexpr int kXs = kHeadDim + 2;         // padded row stride of X (bf16): 65 words, odd
 
-// Rotation pairs of every round for P = 16, 32, 64 (offsets 0, 15*8, 15*8 + 31*16), written once per device by
-// the host.  A pair is stored as (first, second); for P = 64 the orientation is chosen so that the 32 first
-// members of a round fall into 32 different shared-memory banks (index mod 32), and so do the second members.
-__constant__ uchar2 c_pairs[15 * 8 + 31 * 16 + 63 * 32];
-__host__ __device__ constexpr int pair_table_offset(int P) { return P == 16 ? 0 : (P == 32 ? 15 * 8 : 15 * 8 + 31 * 16); }
+// Rotation pairs of every round of the pair ordering, for P = 16 and 32 (offsets 0 and 15*8), written once per
+// device by the host.  A pair is stored as (first, second) = (smaller, larger index).
+__constant__ uchar2 c_pairs[15 * 8 + 31 * 16];
+
+// P = 64 uses groups of four instead (see the quad ordering in the kernel): the 64 indices are the points of the
+// affine space AG(3, 4), a group is a line, and the 21 parallel classes of 16 lines contain every pair of indices
+// exactly once.  c_quads[class][line] = the line's four members in the order (A, B, A, B): an index and its
+// partner (index ^ 32, the one that shares its shared-memory bank) always get different letters, so the 32
+// A-members of a class lie in 32 different banks, and so do the 32 B-members.
+constexpr int kQuadClasses = 21, kQuadsPerClass = 16;
+__constant__ uchar4 c_quads[kQuadClasses * kQuadsPerClass];
+__host__ __device__ constexpr int pair_table_offset(int P) { return P == 16 ? 0 : 15 * 8; }
 
 template <int P>
 struct Shape {
@@ -28,9 +35,7 @@ struct Shape {
     // makes the block update below conflict-free (see there).
     static constexpr int kGs = P;
     static constexpr int kPairs = P / 2;
-    // 2 x 2 blocks of G computed per round: one of each mirror-image couple, and the diagonal blocks
-    static constexpr int kBlocks = kPairs * (kPairs / 2) + kPairs / 2;
-    static constexpr int kChunks = P / 4;               // float4 chunks of a row of Q^T
+    static constexpr int kMinBlocks = P == 64 ? 4 : 1;  // resident CTAs per SM the register allocation must allow
 };
 
 // The page X is needed for the Gram matrix and again for B = A^T X; in between its bytes hold Q^T, and it is
@@ -47,7 +52,11 @@ struct CompressSmem {
         __nv_bfloat16 X2[P * kHeadDim];    // the page again, rows unpadded (projection phase)
     };
     float2 cs[P / 2];
-    uchar2 pairs[(P - 1) * (P / 2)];   // this page size's rows of c_pairs (lanes index it divergently)
+    uchar2 pairs[P == 64 ? 1 : (P - 1) * (P / 2)];   // this page size's rows of c_pairs (lanes index it divergently)
+    // P = 64 (quad ordering): the 4 x 4 transforms of a class's 16 quads, [variant][row][quad] as float4, and the
+    // member table
+    float4 M[P == 64 ? 2 * 4 * 16 : 1];
+    uchar4 quads[P == 64 ? kQuadClasses * kQuadsPerClass : 1];
     float lam[P];
     int order[P];
     float red[Shape<P>::kWarps];
@@ -83,8 +92,39 @@ inline void pair_of(int P, int rho, int k, int &p, int &q) {
     p = a < b ? a : b; q = a < b ? b : a;
 }
 
+// Early-stopping rule: the energy captured by the r largest diagonal entries of G is ||A^T X||_F^2 of the factors
+// the current Q would give; when it stops growing (relative to the reconstruction error that is left) the
+// remaining rotations only polish eigenvectors inside clusters.  Block-wide; every thread gets the answer.
 template <int P>
-__global__ void __launch_bounds__(Shape<P>::kThreads)
+__device__ __noinline__ bool energy_converged(CompressSmem<P> &S, int rank, float energy_tol, float trace,
+                                              float &captured_prev, int tid, int lane, int warp) {
+    constexpr int kWarps = Shape<P>::kWarps;
+    if (tid < P) S.lam[tid] = S.G[tid * Shape<P>::kGs + tid];
+    __syncthreads();
+    float mine = 0.f;
+    if (tid < P) {
+        const float li = S.lam[tid];
+        int r = 0;
+        for (int j = 0; j < P; ++j) {
+            const float lj = S.lam[j];
+            r += (lj > li) || (lj == li && j < tid);
+        }
+        if (r < rank) mine = li;
+    }
+    for (int o = 16; o; o >>= 1) mine += __shfl_xor_sync(0xffffffffu, mine, o);
+    if (lane == 0) S.red[warp] = mine;
+    __syncthreads();
+    float captured = 0.f;
+#pragma unroll
+    for (int w = 0; w < kWarps; ++w) captured += S.red[w];
+    __syncthreads();
+    const bool done = captured_prev >= 0.f && captured - captured_prev <= energy_tol * fmaxf(trace - captured, 0.f);
+    captured_prev = captured;
+    return done;
+}
+
+template <int P>
+__global__ void __launch_bounds__(Shape<P>::kThreads, Shape<P>::kMinBlocks)
 compress_kernel(Geometry geo, const unsigned char *dense_pool, unsigned char *factor_pool,
                 const int2 *worklist, int *status) {
     using Sh = Shape<P>;
@@ -166,117 +206,241 @@ compress_kernel(Geometry geo, const unsigned char *dense_pool, unsigned char *fa
 #pragma unroll
     for (int w = 0; w < kWarps; ++w) trace += S.red[w];
     float captured_prev = -1.f;
-
-    // ---- cyclic Jacobi sweeps ----
-    // The P/2 rotations of a round act on disjoint index pairs, so G' = J^T G J splits into (P/2)^2 independent
-    // 2 x 2 blocks: block (a, b) = rows of pair a, columns of pair b, becomes J_a^T . block . J_b.  G is
-    // symmetric, so one block of every mirror-image couple is computed: a thread reads its block's four entries
-    // and writes them and their mirror images (G stays bitwise symmetric), so G passes through shared memory once
-    // per round.  Lanes walk a wrapped diagonal, block (a, a + delta mod P/2) for lane a: delta = 0 .. P/4 covers
-    // every couple once (delta = P/4 with a < P/4 only).  On a diagonal the lanes' row pairs are all different
-    // and so are their column pairs; the bank of an entry is its column index mod 32 and the oriented pair table
-    // keeps a round's first members (and its second members) in different banks, so neither the block accesses
-    // (bank = a member of the column pair) nor the mirrored stores (bank = a member of the row pair) conflict.
-    // For P < 64 a warp holds several diagonals; every other one takes its pairs in the opposite order, (q, p)
-    // with the rotation (c, -s), which is the same rotation, so that it touches second members while its
-    // neighbour touches first members.
-    // Q^T is stored instead of Q: rotating columns p, q of Q is rotating rows p, q of Q^T, four tokens at a time.
-    for (int i = tid; i < (P - 1) * kPairs; i += kThreads) S.pairs[i] = c_pairs[pair_table_offset(P) + i];
-    __syncthreads();
-    const uchar2 *pairs = S.pairs;
     bool converged = false;
-    for (int sweep = 0; sweep < geo.jacobi_max_sweeps && !converged; ++sweep) {
-        int rotated = 0;
-        for (int rho = 0; rho < P - 1; ++rho) {
-            const uchar2 *pr = pairs + rho * kPairs;
-            if (tid < kPairs) {
-                const int p = pr[tid].x, q = pr[tid].y;
-                const float gpp = S.G[p * kGs + p], gqq = S.G[q * kGs + q], gpq = S.G[p * kGs + q];
-                float c = 1.f, s = 0.f;
-                if (fabsf(gpq) > fmaxf(tol * sqrtf(fabsf(gpp * gqq)), floor_abs)) {
-                    const float theta = (gqq - gpp) / (2.f * gpq);
-                    const float t = copysignf(1.f, theta) / (fabsf(theta) + sqrtf(1.f + theta * theta));
-                    c = rsqrtf(1.f + t * t);
-                    s = t * c;
-                    rotated = 1;
-                }
-                S.cs[tid] = make_float2(c, s);
-            }
-            __syncthreads();
+    if constexpr (P == 64) {
+        // ---- quad ordering ----
+        // A class partitions the 64 indices into 16 quads.  Inside a quad the six pairs are rotated in three layers,
+        // (0,1)(2,3), (0,2)(1,3), (0,3)(1,2), which needs only the quad's own 4 x 4 diagonal block of G; the product
+        // of the six rotations is a 4 x 4 orthogonal matrix M.  Then G' = M^T G M and Q^T' = M^T Q^T are applied
+        // blockwise with dense 4 x 4 products: one pass over G and Q^T covers what takes three rounds of the pair
+        // ordering, with a third of the shared-memory traffic and instructions, and 21 classes make a sweep in which
+        // every pair is rotated exactly once.
+        //   threads 0-63   four per quad: rotations and M                                        (between barriers)
+        //   warps 0-4      G: a thread owns the 4 x 4 block (quad a, quad b) of a mirror-image couple, lanes walk
+        //                  two wrapped diagonals (b = a + delta mod 16; delta = 0 .. 8, 136 blocks), read 16
+        //                  entries, write 16 and their mirror images
+        //   warps 5-7      Q^T: a thread owns (quad, four tokens): four 128-bit loads, 64 FMAs, four stores
+        // Banks: an entry's bank is its column index mod 32.  Lanes 0-15 take their quads' members in table order,
+        // lanes 16-31 in the order (2, 3, 0, 1) with M permuted to match, so at any step the warp touches either
+        // all A-members or all B-members of the class: 32 different banks, for the block accesses (columns of
+        // quad b) and for the mirrored stores (columns of quad a) alike.
+        for (int i = tid; i < kQuadClasses * kQuadsPerClass; i += kThreads) S.quads[i] = c_quads[i];
+        __syncthreads();
+        float4 *QT4 = reinterpret_cast<float4 *>(S.QT);
+        for (int sweep = 0; sweep < geo.jacobi_max_sweeps && !converged; ++sweep) {
+            int rotated = 0;
+            for (int cls = 0; cls < kQuadClasses && !converged; ++cls) {
+                const uchar4 *quads = S.quads + cls * kQuadsPerClass;
+                if (tid < 4 * kQuadsPerClass) {
+                    // Four lanes per quad; lane t holds row t of the quad's diagonal block D and of M, stored
+                    // "rotated": e[k] = D[t][t ^ k], f[k] = M[t][t ^ k], so that the partner of layer x (t ^ x), the
+                    // pivot (e[x]) and the column pairs (k, k ^ x) have compile-time positions.
+                    const int qd = tid >> 2, t = tid & 3;
+                    const unsigned m4 = reinterpret_cast<const unsigned *>(quads)[qd];
+                    const int mt = (m4 >> (8 * t)) & 0xff;
+                    float e[4], f[4];
 #pragma unroll
-            for (int u0 = 0; u0 < Sh::kBlocks; u0 += kThreads) {
-                const int u = u0 + tid;
-                if (u < Sh::kBlocks) {
-                    const int delta = u / kPairs, ia = u % kPairs, ib = (ia + delta) % kPairs;
-                    float2 ca = S.cs[ia], cb = S.cs[ib];
-                    if (ca.y != 0.f || cb.y != 0.f) {
-                        uchar2 pa = pr[ia], pb = pr[ib];
-                        if (kPairs < 32 && (delta & 1)) {
-                            pa = make_uchar2(pa.y, pa.x); ca.y = -ca.y;
-                            pb = make_uchar2(pb.y, pb.x); cb.y = -cb.y;
+                    for (int k = 0; k < 4; ++k) {
+                        e[k] = S.G[mt * kGs + ((m4 >> (8 * (t ^ k))) & 0xff)];
+                        f[k] = k == 0 ? 1.f : 0.f;
+                    }
+#pragma unroll
+                    for (int x = 1; x <= 3; ++x) {                      // layer x pairs t with t ^ x
+                        const int y = x == 1 ? 2 : 1;                   // t ^ y lies in the layer's other pair
+                        const bool low = t < (t ^ x);                   // this lane is the pair's lower index
+                        const float d_mine = e[0], d_other = __shfl_xor_sync(0xffffffffu, e[0], x);
+                        // both lanes of a pair must arrive at the same rotation: take the pivot from the lower one
+                        const float g_other = __shfl_xor_sync(0xffffffffu, e[x], x), gpq = low ? e[x] : g_other;
+                        const float gpp = low ? d_mine : d_other, gqq = low ? d_other : d_mine;
+                        float c = 1.f, sn = 0.f;
+                        if (fabsf(gpq) > fmaxf(tol * sqrtf(fabsf(gpp * gqq)), floor_abs)) {
+                            const float theta = (gqq - gpp) / (2.f * gpq);
+                            const float tt = copysignf(1.f, theta) / (fabsf(theta) + sqrtf(1.f + theta * theta));
+                            c = rsqrtf(1.f + tt * tt);
+                            sn = tt * c;
+                            rotated = 1;
                         }
-                        float *g0 = S.G + pa.x * kGs, *g1 = S.G + pa.y * kGs;
-                        const float x00 = g0[pb.x], x01 = g0[pb.y], x10 = g1[pb.x], x11 = g1[pb.y];
-                        const float y00 = ca.x * x00 - ca.y * x10, y01 = ca.x * x01 - ca.y * x11;
-                        const float y10 = ca.y * x00 + ca.x * x10, y11 = ca.y * x01 + ca.x * x11;
-                        const float z00 = cb.x * y00 - cb.y * y01, z01 = cb.y * y00 + cb.x * y01;
-                        const float z10 = cb.x * y10 - cb.y * y11, z11 = cb.y * y10 + cb.x * y11;
-                        if (delta != 0) {
-                            g0[pb.x] = z00; g0[pb.y] = z01; g1[pb.x] = z10; g1[pb.y] = z11;
-                            float *h0 = S.G + pb.x * kGs, *h1 = S.G + pb.y * kGs;
-                            h0[pa.x] = z00; h1[pa.x] = z01; h0[pa.y] = z10; h1[pa.y] = z11;
-                        } else {                       // diagonal block: x01 = x10, and so are their images
-                            g0[pb.x] = z00; g0[pb.y] = z01; g1[pb.x] = z01; g1[pb.y] = z11;
+                        const float c2 = __shfl_xor_sync(0xffffffffu, c, y), s2 = __shfl_xor_sync(0xffffffffu, sn, y);
+                        // columns: positions (0, x) belong to this lane's pair, (y, y ^ x) to the other pair; the
+                        // entry at position k is column t ^ k, the lower column of its pair iff (t ^ k) < (t ^ k ^ x)
+                        const float sa = low ? sn : -sn;                                  // position 0 = column t
+                        const float sb = ((t ^ y) < (t ^ y ^ x)) ? s2 : -s2;              // position y
+                        const float e0 = c * e[0] - sa * e[x], ex = c * e[x] + sa * e[0];
+                        const float ey = c2 * e[y] - sb * e[y ^ x], eyx = c2 * e[y ^ x] + sb * e[y];
+                        const float f0 = c * f[0] - sa * f[x], fx = c * f[x] + sa * f[0];
+                        const float fy = c2 * f[y] - sb * f[y ^ x], fyx = c2 * f[y ^ x] + sb * f[y];
+                        f[0] = f0; f[x] = fx; f[y] = fy; f[y ^ x] = fyx;
+                        // rows: new row t = c row t -/+ s row (t ^ x); the partner's entry of the same column sits
+                        // at its position k ^ x
+                        const float p0 = __shfl_xor_sync(0xffffffffu, ex, x), px = __shfl_xor_sync(0xffffffffu, e0, x);
+                        const float py = __shfl_xor_sync(0xffffffffu, eyx, x), pyx = __shfl_xor_sync(0xffffffffu, ey, x);
+                        e[0] = c * e0 - sa * p0; e[x] = c * ex - sa * px;
+                        e[y] = c * ey - sa * py; e[y ^ x] = c * eyx - sa * pyx;
+                    }
+                    // natural column order: M[t][c] = f[t ^ c]
+                    float r0 = f[0], r1 = f[1], r2 = f[2], r3 = f[3];
+                    if (t & 1) { float w = r0; r0 = r1; r1 = w; w = r2; r2 = r3; r3 = w; }
+                    if (t & 2) { float w = r0; r0 = r2; r2 = w; w = r1; r1 = r3; r3 = w; }
+                    S.M[(0 * 4 + t) * 16 + qd] = make_float4(r0, r1, r2, r3);
+                    S.M[(1 * 4 + (t ^ 2)) * 16 + qd] = make_float4(r2, r3, r0, r1);
+                }
+                __syncthreads();
+                if (warp < 5) {
+                    const int h = lane >> 4, ia = lane & 15, delta = 2 * warp + h;
+                    if (delta < 8 || (delta == 8 && ia < 8)) {
+                        const int ib = (ia + delta) & 15;
+                        unsigned ma4 = reinterpret_cast<const unsigned *>(quads)[ia];
+                        unsigned mb4 = reinterpret_cast<const unsigned *>(quads)[ib];
+                        if (h) { ma4 = __byte_perm(ma4, 0u, 0x1032); mb4 = __byte_perm(mb4, 0u, 0x1032); }
+                        int ma[4], mb[4];
+#pragma unroll
+                        for (int i = 0; i < 4; ++i) { ma[i] = (ma4 >> (8 * i)) & 0xff; mb[i] = (mb4 >> (8 * i)) & 0xff; }
+                        const float4 *Ma = S.M + h * 64 + ia, *Mb = S.M + h * 64 + ib;
+                        float T[4][4];
+#pragma unroll
+                        for (int i = 0; i < 4; ++i)
+#pragma unroll
+                            for (int j = 0; j < 4; ++j) T[i][j] = 0.f;
+#pragma unroll
+                        for (int k = 0; k < 4; ++k) {                  // T = M_a^T X
+                            const float4 mk = Ma[k * 16];
+                            const float *row = S.G + ma[k] * kGs;
+#pragma unroll
+                            for (int j = 0; j < 4; ++j) {
+                                const float x = row[mb[j]];
+                                T[0][j] = fmaf(mk.x, x, T[0][j]); T[1][j] = fmaf(mk.y, x, T[1][j]);
+                                T[2][j] = fmaf(mk.z, x, T[2][j]); T[3][j] = fmaf(mk.w, x, T[3][j]);
+                            }
+                        }
+                        const float4 b0 = Mb[0], b1 = Mb[16], b2 = Mb[32], b3 = Mb[48];
+#pragma unroll
+                        for (int i = 0; i < 4; ++i) {                  // Y = T M_b, row i
+                            float y[4];
+                            y[0] = fmaf(T[i][3], b3.x, fmaf(T[i][2], b2.x, fmaf(T[i][1], b1.x, T[i][0] * b0.x)));
+                            y[1] = fmaf(T[i][3], b3.y, fmaf(T[i][2], b2.y, fmaf(T[i][1], b1.y, T[i][0] * b0.y)));
+                            y[2] = fmaf(T[i][3], b3.z, fmaf(T[i][2], b2.z, fmaf(T[i][1], b1.z, T[i][0] * b0.z)));
+                            y[3] = fmaf(T[i][3], b3.w, fmaf(T[i][2], b2.w, fmaf(T[i][1], b1.w, T[i][0] * b0.w)));
+#pragma unroll
+                            for (int j = 0; j < 4; ++j) {
+                                // the diagonal block (a = b) is symmetric: its upper triangle is written to both sides
+                                if (delta != 0 || j >= i) {
+                                    S.G[ma[i] * kGs + mb[j]] = y[j];
+                                    S.G[mb[j] * kGs + ma[i]] = y[j];
+                                }
+                            }
                         }
                     }
-                }
-            }
-            // rows p, q of Q^T:  x_p' = c x_p - s x_q,  x_q' = s x_p + c x_q
-#pragma unroll
-            for (int i0 = 0; i0 < kPairs * Sh::kChunks; i0 += kThreads) {
-                const int item = i0 + tid;
-                if (item < kPairs * Sh::kChunks) {
-                    const int k = item / Sh::kChunks, ch = item % Sh::kChunks;
-                    const float2 cs = S.cs[k];
-                    if (cs.y != 0.f) {
-                        const uchar2 pq = pr[k];
-                        float4 *rp = reinterpret_cast<float4 *>(S.QT + pq.x * P) + ch;
-                        float4 *rq = reinterpret_cast<float4 *>(S.QT + pq.y * P) + ch;
-                        const float4 xp = *rp, xq = *rq;
-                        *rp = make_float4(cs.x * xp.x - cs.y * xq.x, cs.x * xp.y - cs.y * xq.y,
-                                          cs.x * xp.z - cs.y * xq.z, cs.x * xp.w - cs.y * xq.w);
-                        *rq = make_float4(cs.y * xp.x + cs.x * xq.x, cs.y * xp.y + cs.x * xq.y,
-                                          cs.y * xp.z + cs.x * xq.z, cs.y * xp.w + cs.x * xq.w);
+                } else {
+                    for (int itq = (warp - 5) * 3; itq < min(8, (warp - 5) * 3 + 3); ++itq) {
+                        const int v = itq * 32 + lane, k = v >> 4, ch = v & 15;
+                        const uchar4 m4 = quads[k];
+                        float4 *r0 = QT4 + m4.x * (P / 4) + ch, *r1 = QT4 + m4.y * (P / 4) + ch;
+                        float4 *r2 = QT4 + m4.z * (P / 4) + ch, *r3 = QT4 + m4.w * (P / 4) + ch;
+                        const float4 x0 = *r0, x1 = *r1, x2 = *r2, x3 = *r3;
+                        const float4 c0 = S.M[0 * 16 + k], c1 = S.M[1 * 16 + k], c2 = S.M[2 * 16 + k], c3 = S.M[3 * 16 + k];
+#define PKV_MIX(comp) make_float4(fmaf(c3.comp, x3.x, fmaf(c2.comp, x2.x, fmaf(c1.comp, x1.x, c0.comp * x0.x))), \
+                                  fmaf(c3.comp, x3.y, fmaf(c2.comp, x2.y, fmaf(c1.comp, x1.y, c0.comp * x0.y))), \
+                                  fmaf(c3.comp, x3.z, fmaf(c2.comp, x2.z, fmaf(c1.comp, x1.z, c0.comp * x0.z))), \
+                                  fmaf(c3.comp, x3.w, fmaf(c2.comp, x2.w, fmaf(c1.comp, x1.w, c0.comp * x0.w))))
+                        *r0 = PKV_MIX(x); *r1 = PKV_MIX(y); *r2 = PKV_MIX(z); *r3 = PKV_MIX(w);   // row i' = sum_k M[k][i] row k
+#undef PKV_MIX
                     }
                 }
+                __syncthreads();
+                // three checks per sweep
+                if (cls % 7 == 6 && geo.jacobi_energy_tol >= 0.f && energy_converged<P>(S, rank, geo.jacobi_energy_tol, trace, captured_prev, tid, lane, warp)) converged = true;
             }
-            __syncthreads();
+            if (!__syncthreads_or(rotated)) converged = true;
         }
-        converged = !__syncthreads_or(rotated);
-        if (!converged && geo.jacobi_energy_tol >= 0.f) {
-            // energy captured by the r largest diagonal entries after this sweep
-            if (tid < P) S.lam[tid] = S.G[tid * kGs + tid];
-            __syncthreads();
-            float mine = 0.f;
-            if (tid < P) {
-                const float li = S.lam[tid];
-                int r = 0;
-                for (int j = 0; j < P; ++j) {
-                    const float lj = S.lam[j];
-                    r += (lj > li) || (lj == li && j < tid);
+    } else {
+        // ---- cyclic Jacobi sweeps, pair ordering (P = 16, 32) ----
+        // 2 x 2 blocks of G computed per round: one of each mirror-image couple, and the diagonal blocks
+        constexpr int kBlocks = kPairs * (kPairs / 2) + kPairs / 2;
+        constexpr int kChunks = P / 4;               // float4 chunks of a row of Q^T
+        // The P/2 rotations of a round act on disjoint index pairs, so G' = J^T G J splits into (P/2)^2 independent
+        // 2 x 2 blocks: block (a, b) = rows of pair a, columns of pair b, becomes J_a^T . block . J_b.  G is
+        // symmetric, so one block of every mirror-image couple is computed: a thread reads its block's four entries
+        // and writes them and their mirror images (G stays bitwise symmetric), so G passes through shared memory once
+        // per round.  Lanes walk a wrapped diagonal, block (a, a + delta mod P/2) for lane a: delta = 0 .. P/4 covers
+        // every couple once (delta = P/4 with a < P/4 only).  On a diagonal the lanes' row pairs are all different
+        // and so are their column pairs; G's rows are unpadded, so the bank of an entry is its column index (all
+        // below 32 here): neither the block accesses (bank = a member of the column pair) nor the mirrored stores
+        // (bank = a member of the row pair) conflict inside a diagonal.  A warp holds several diagonals; every
+        // other one takes its pairs in the opposite order, (q, p) with the rotation (c, -s), which is the same
+        // rotation, so that it touches second members while its neighbour touches first members.
+        // Q^T is stored instead of Q: rotating columns p, q of Q is rotating rows p, q of Q^T, four tokens at a time.
+        for (int i = tid; i < (P - 1) * kPairs; i += kThreads) S.pairs[i] = c_pairs[pair_table_offset(P) + i];
+        __syncthreads();
+        const uchar2 *pairs = S.pairs;
+        for (int sweep = 0; sweep < geo.jacobi_max_sweeps && !converged; ++sweep) {
+            int rotated = 0;
+            for (int rho = 0; rho < P - 1; ++rho) {
+                const uchar2 *pr = pairs + rho * kPairs;
+                if (tid < kPairs) {
+                    const int p = pr[tid].x, q = pr[tid].y;
+                    const float gpp = S.G[p * kGs + p], gqq = S.G[q * kGs + q], gpq = S.G[p * kGs + q];
+                    float c = 1.f, s = 0.f;
+                    if (fabsf(gpq) > fmaxf(tol * sqrtf(fabsf(gpp * gqq)), floor_abs)) {
+                        const float theta = (gqq - gpp) / (2.f * gpq);
+                        const float t = copysignf(1.f, theta) / (fabsf(theta) + sqrtf(1.f + theta * theta));
+                        c = rsqrtf(1.f + t * t);
+                        s = t * c;
+                        rotated = 1;
+                    }
+                    S.cs[tid] = make_float2(c, s);
                 }
-                if (r < rank) mine = li;
-            }
-            for (int o = 16; o; o >>= 1) mine += __shfl_xor_sync(0xffffffffu, mine, o);
-            if (lane == 0) S.red[warp] = mine;
-            __syncthreads();
-            float captured = 0.f;
+                __syncthreads();
 #pragma unroll
-            for (int w = 0; w < kWarps; ++w) captured += S.red[w];
-            __syncthreads();
-            if (captured_prev >= 0.f && captured - captured_prev <= geo.jacobi_energy_tol * fmaxf(trace - captured, 0.f))
-                converged = true;
-            captured_prev = captured;
+                for (int u0 = 0; u0 < kBlocks; u0 += kThreads) {
+                    const int u = u0 + tid;
+                    if (u < kBlocks) {
+                        const int delta = u / kPairs, ia = u % kPairs, ib = (ia + delta) % kPairs;
+                        float2 ca = S.cs[ia], cb = S.cs[ib];
+                        if (ca.y != 0.f || cb.y != 0.f) {
+                            uchar2 pa = pr[ia], pb = pr[ib];
+                            if (delta & 1) {
+                                pa = make_uchar2(pa.y, pa.x); ca.y = -ca.y;
+                                pb = make_uchar2(pb.y, pb.x); cb.y = -cb.y;
+                            }
+                            float *g0 = S.G + pa.x * kGs, *g1 = S.G + pa.y * kGs;
+                            const float x00 = g0[pb.x], x01 = g0[pb.y], x10 = g1[pb.x], x11 = g1[pb.y];
+                            const float y00 = ca.x * x00 - ca.y * x10, y01 = ca.x * x01 - ca.y * x11;
+                            const float y10 = ca.y * x00 + ca.x * x10, y11 = ca.y * x01 + ca.x * x11;
+                            const float z00 = cb.x * y00 - cb.y * y01, z01 = cb.y * y00 + cb.x * y01;
+                            const float z10 = cb.x * y10 - cb.y * y11, z11 = cb.y * y10 + cb.x * y11;
+                            if (delta != 0) {
+                                g0[pb.x] = z00; g0[pb.y] = z01; g1[pb.x] = z10; g1[pb.y] = z11;
+                                float *h0 = S.G + pb.x * kGs, *h1 = S.G + pb.y * kGs;
+                                h0[pa.x] = z00; h1[pa.x] = z01; h0[pa.y] = z10; h1[pa.y] = z11;
+                            } else {                       // diagonal block: x01 = x10, and so are their images
+                                g0[pb.x] = z00; g0[pb.y] = z01; g1[pb.x] = z01; g1[pb.y] = z11;
+                            }
+                        }
+                    }
+                }
+                // rows p, q of Q^T:  x_p' = c x_p - s x_q,  x_q' = s x_p + c x_q
+#pragma unroll
+                for (int i0 = 0; i0 < kPairs * kChunks; i0 += kThreads) {
+                    const int item = i0 + tid;
+                    if (item < kPairs * kChunks) {
+                        const int k = item / kChunks, ch = item % kChunks;
+                        const float2 cs = S.cs[k];
+                        if (cs.y != 0.f) {
+                            const uchar2 pq = pr[k];
+                            float4 *rp = reinterpret_cast<float4 *>(S.QT + pq.x * P) + ch;
+                            float4 *rq = reinterpret_cast<float4 *>(S.QT + pq.y * P) + ch;
+                            const float4 xp = *rp, xq = *rq;
+                            *rp = make_float4(cs.x * xp.x - cs.y * xq.x, cs.x * xp.y - cs.y * xq.y,
+                                              cs.x * xp.z - cs.y * xq.z, cs.x * xp.w - cs.y * xq.w);
+                            *rq = make_float4(cs.y * xp.x + cs.x * xq.x, cs.y * xp.y + cs.x * xq.y,
+                                              cs.y * xp.z + cs.x * xq.z, cs.y * xp.w + cs.x * xq.w);
+                        }
+                    }
+                }
+                __syncthreads();
+            }
+            converged = !__syncthreads_or(rotated);
+            if (!converged && geo.jacobi_energy_tol >= 0.f && energy_converged<P>(S, rank, geo.jacobi_energy_tol, trace, captured_prev, tid, lane, warp)) converged = true;
         }
     }
     if (!converged && tid == 0) atomicAdd(&status[1], 1);
@@ -410,42 +574,76 @@ compress_kernel(Geometry geo, const unsigned char *dense_pool, unsigned char *fa
     }
 }
 
-// Round-robin pairs of every round.  For P = 64 each pair is oriented (first, second) so that the first members
-// of a round have distinct indices mod 32 (and hence so do the second members): mark x first and its partner y
-// second; y ^ 32 shares y's bank, so it must be a first member; continue from there until the cycle closes.
+// Round-robin pairs of every round (P = 16, 32).
 void fill_pair_table(int P, uchar2 *out) {
     const int B = P / 2;
-    for (int rho = 0; rho < P - 1; ++rho) {
-        int partner[kMaxPage], role[kMaxPage];      // role: 0 unknown, 1 first, 2 second
+    for (int rho = 0; rho < P - 1; ++rho)
         for (int k = 0; k < B; ++k) {
             int p, q;
             pair_of(P, rho, k, p, q);
-            partner[p] = q; partner[q] = p;
-            role[p] = P == 64 ? 0 : 1; role[q] = P == 64 ? 0 : 2;
+            out[rho * B + k] = make_uchar2((unsigned char)p, (unsigned char)q);
         }
-        if (P == 64) {
-            for (int start = 0; start < P; ++start) {
-                int x = start;
-                while (role[x] == 0) {
-                    role[x] = 1;
-                    const int y = partner[x];
-                    role[y] = 2;
-                    x = y ^ 32;
-                }
+}
+
+// The 21 parallel classes of lines of AG(3, 4) over the indices 0..63 (index = x0 + 4 x1 + 16 x2, coordinates in
+// GF(4) = {0, 1, w, w^2} with addition = xor), members ordered (A, B, A, B) as c_quads describes.
+void fill_quad_table(uchar4 *out) {
+    static const int mul[4][4] = {{0, 0, 0, 0}, {0, 1, 2, 3}, {0, 2, 3, 1}, {0, 3, 1, 2}};
+    int dirs[kQuadClasses][3], nd = 0;
+    for (int a = 0; a < 4; ++a) for (int b = 0; b < 4; ++b) { dirs[nd][0] = 1; dirs[nd][1] = a; dirs[nd][2] = b; ++nd; }
+    for (int a = 0; a < 4; ++a) { dirs[nd][0] = 0; dirs[nd][1] = 1; dirs[nd][2] = a; ++nd; }
+    dirs[nd][0] = 0; dirs[nd][1] = 0; dirs[nd][2] = 1; ++nd;
+    for (int c = 0; c < kQuadClasses; ++c) {
+        int line[kQuadsPerClass][4], n_lines = 0, mate[64], colour[64];
+        bool seen[64] = {};
+        for (int x = 0; x < 64; ++x) {
+            if (seen[x]) continue;
+            for (int t = 0; t < 4; ++t) {
+                const int y = (x & 3) ^ mul[t][dirs[c][0]] | (((x >> 2) & 3) ^ mul[t][dirs[c][1]]) << 2 |
+                              (((x >> 4) & 3) ^ mul[t][dirs[c][2]]) << 4;
+                line[n_lines][t] = y;
+                seen[y] = true;
+            }
+            ++n_lines;
+        }
+        // Two-colour the indices so that mates inside a line (members 0-1 and 2-3) differ and so do x and x ^ 32:
+        // the two perfect matchings form even cycles, walked alternately.
+        for (int l = 0; l < kQuadsPerClass; ++l) {
+            mate[line[l][0]] = line[l][1]; mate[line[l][1]] = line[l][0];
+            mate[line[l][2]] = line[l][3]; mate[line[l][3]] = line[l][2];
+        }
+        for (int x = 0; x < 64; ++x) colour[x] = -1;
+        for (int start = 0; start < 64; ++start) {
+            int x = start;
+            while (colour[x] < 0) {
+                colour[x] = 0;
+                const int y = mate[x];
+                colour[y] = 1;
+                x = y ^ 32;
             }
         }
-        int k = 0;
-        for (int x = 0; x < P; ++x)
-            if (role[x] == 1) out[rho * B + k++] = make_uchar2((unsigned char)x, (unsigned char)partner[x]);
+        for (int l = 0; l < kQuadsPerClass; ++l) {
+            int m[4];
+            for (int half = 0; half < 2; ++half) {
+                const int u = line[l][2 * half], v = line[l][2 * half + 1];
+                m[2 * half] = colour[u] == 0 ? u : v;
+                m[2 * half + 1] = colour[u] == 0 ? v : u;
+            }
+            out[c * kQuadsPerClass + l] = make_uchar4((unsigned char)m[0], (unsigned char)m[1], (unsigned char)m[2],
+                                                      (unsigned char)m[3]);
+        }
     }
 }
 
 cudaError_t upload_pair_tables() {
-    static uchar2 host[15 * 8 + 31 * 16 + 63 * 32];
+    static uchar2 host[15 * 8 + 31 * 16];
     fill_pair_table(16, host + pair_table_offset(16));
     fill_pair_table(32, host + pair_table_offset(32));
-    fill_pair_table(64, host + pair_table_offset(64));
-    return cudaMemcpyToSymbol(c_pairs, host, sizeof host);
+    cudaError_t e = cudaMemcpyToSymbol(c_pairs, host, sizeof host);
+    if (e != cudaSuccess) return e;
+    static uchar4 quads[kQuadClasses * kQuadsPerClass];
+    fill_quad_table(quads);
+    return cudaMemcpyToSymbol(c_quads, quads, sizeof quads);
 }
 
 template <int P>
