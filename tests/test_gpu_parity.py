@@ -401,3 +401,47 @@ def test_int4_factors(P, rk, rv, G):
     print("int4 P=%d r=(%d,%d): kernel %.2e, e2e vs int4 oracle %.2e, int4 noise %.2e, storage ratio %.4f"
           % (P, rk, rv, max(g["kernel"]), max(rel_err(got[i], ref4[i]) for i in range(3)),
              max(rel_err(ref4[i], ref16[i]) for i in range(3)), ratio))
+
+
+@pytest.mark.gpu
+@pytest.mark.parametrize("P", [64, 32])
+@pytest.mark.parametrize("energy_tol", [0.0, -1.0])
+def test_prescribed_spectra_with_and_without_the_energy_rule(P, energy_tol):
+    """Pages built as U diag(s) W^T with chosen singular values: a cluster of equal values straddling the rank
+    cut, a sharp gap exactly at the cut, a geometric decay, a flat spectrum.  The stored factors must reach the
+    Eckart-Young error of the (bf16-rounded) page whether the sweeps stop by the energy rule (default) or only when
+    no rotation is left (rule off), and both settings must agree on the error."""
+    r = 16
+    g = torch.Generator().manual_seed(100 + P)
+    spectra = [
+        [4.0] * 8 + [1.0] * 16 + [0.05] * (P - 24),                      # equal values across the cut (r = 16)
+        [3.0] * 16 + [1e-3] * (P - 16),                                  # gap at the cut
+        [0.8 ** i for i in range(P)],                                    # geometric
+        [1.0] * P,                                                       # flat: any 16 directions are optimal
+    ]
+    pages = []
+    for s in spectra:
+        U, _ = torch.linalg.qr(torch.randn(P, P, generator=g, dtype=torch.float64))
+        W, _ = torch.linalg.qr(torch.randn(128, P, generator=g, dtype=torch.float64))
+        pages.append((U * torch.tensor(s, dtype=torch.float64)) @ W.T)
+    x = torch.cat(pages).to(torch.bfloat16)[:, None, :]                  # [4 P, 1, 128]
+    cfg = pkv.make_config(n_layers=1, n_kv_heads=1, n_q_heads=4, rank=r, page_size=P, sink_tokens=0, recent_tokens=0,
+                          max_seqs=1, max_pages_per_seq=8, n_dense_slots=8, n_factor_slots=8,
+                          jacobi_energy_tol=energy_tol)
+    pair = Pair(cfg, seed=3, shuffle=False, oracle=False)
+    pair.gpu.append_kv(0, [0], [4 * P], x.cuda(), x.cuda())
+    assert pair.gpu.compress_eligible_pages(0) == 4
+    torch.cuda.synchronize()
+    assert pair.gpu.stats()["page_svds_not_converged"] == 0
+    X = f64(x[:, 0]).reshape(4, P, 128)
+    _, _, sigma = svd.page_factors(X, r)
+    tail = svd.optimal_tail(sigma, r)
+    _, slots, _ = pair.gpu.page_table(0, 0)
+    for p, slot in enumerate(slots):
+        A_k, B_k, A_v, B_v = [f64(t) for t in pair.gpu.read_factors(slot, 0)]
+        for A, B in ((A_k, B_k), (A_v, B_v)):
+            err = np.linalg.norm(X[p] - A @ B)
+            # bf16 storage of A and B alone costs up to 2^-9 of ||X|| each, which dominates where the tail is tiny
+            assert err <= 1.01 * tail[p] + 4e-3 * np.linalg.norm(X[p]), (P, energy_tol, p, err, tail[p])
+            # columns of A orthonormal up to bf16 rounding
+            assert np.abs(A.T @ A - np.eye(r)).max() <= 2e-2, (P, energy_tol, p)
