@@ -14,18 +14,33 @@ namespace {
 
 constexpr int kXs = kHeadDim + 2;         // padded row stride of X (bf16): 65 words, odd
 
-// Rotation pairs of every round of the pair ordering, for P = 16 and 32 (offsets 0 and 15*8), written once per
-// device by the host.  A pair is stored as (first, second) = (smaller, larger index).
-__constant__ uchar2 c_pairs[15 * 8 + 31 * 16];
+// Rotation pairs of every round of the pair ordering (P = 16), written once per device by the host.  A pair is
+// stored as (first, second) = (smaller, larger index).
+__constant__ uchar2 c_pairs[15 * 8];
 
-// P = 64 uses groups of four instead (see the quad ordering in the kernel): the 64 indices are the points of the
-// affine space AG(3, 4), a group is a line, and the 21 parallel classes of 16 lines contain every pair of indices
-// exactly once.  c_quads[class][line] = the line's four members in the order (A, B, A, B): an index and its
-// partner (index ^ 32, the one that shares its shared-memory bank) always get different letters, so the 32
-// A-members of a class lie in 32 different banks, and so do the 32 B-members.
-constexpr int kQuadClasses = 21, kQuadsPerClass = 16;
-__constant__ uchar4 c_quads[kQuadClasses * kQuadsPerClass];
-__host__ __device__ constexpr int pair_table_offset(int P) { return P == 16 ? 0 : 15 * 8; }
+// P = 64 and P = 32 use groups of four instead (see the quad ordering in the kernel).  A class partitions the P
+// indices into P/4 quads; the classes of a sweep contain every pair of indices at least once.
+//   P = 64: the indices are the points of the affine space AG(3, 4), a quad is a line, and the 21 parallel classes
+//           of 16 lines contain every pair exactly once.  A line's members are stored in the order (A, B, A, B): an
+//           index and its partner (index ^ 32, the one that shares its shared-memory bank) always get different
+//           letters, so the 32 A-members of a class lie in 32 different banks, and so do the 32 B-members.
+//   P = 32: no such design exists for 32 points.  Each half of 16 indices is an affine plane AG(2, 4): its 5
+//           parallel classes of 4 lines give 5 classes of 8 quads with every pair inside a half once; the 256
+//           pairs between the halves come from 8 more classes of quads {x, x ^ u, 16 + (x ^ a), 16 + (x ^ u ^ a)},
+//           which hold the pairs of difference a and u ^ a (the 16 differences are split into 8 couples {a, a ^ u}),
+//           and repeat two pairs inside the halves.  13 classes, 8 of them with two repeated pairs per quad.
+template <int P> struct Quads {
+    static constexpr int kQuads = P / 4;                       // per class
+    static constexpr int kClasses = P == 64 ? 21 : 13;
+    static constexpr int kDiag = 32 / kQuads;                  // wrapped diagonals of quad blocks per warp: 2 or 4
+    static constexpr int kVarStep = 4 / kDiag;                 // lane group g takes its quads' members in the order j ^ (g * kVarStep)
+    static constexpr int kItems = kQuads * (kQuads / 2) + kQuads / 2;   // quad blocks of G computed per class
+    static constexpr int kGWarps = (kItems + 31) / 32;         // 5 or 2; the remaining warps update Q^T
+    static constexpr int kQIters = kQuads * (P / 4) / 32;      // 8 or 2
+    static constexpr int kCheck = (kClasses + 2) / 3;          // the energy rule is evaluated about three times per sweep
+};
+__constant__ uchar4 c_quads64[Quads<64>::kClasses * Quads<64>::kQuads];
+__constant__ uchar4 c_quads32[Quads<32>::kClasses * Quads<32>::kQuads];
 
 template <int P>
 struct Shape {
@@ -35,7 +50,7 @@ struct Shape {
     // makes the block update below conflict-free (see there).
     static constexpr int kGs = P;
     static constexpr int kPairs = P / 2;
-    static constexpr int kMinBlocks = P == 64 ? 4 : 1;  // resident CTAs per SM the register allocation must allow
+    static constexpr int kMinBlocks = P == 64 ? 4 : (P == 32 ? 8 : 1);  // resident CTAs per SM the register allocation must allow
 };
 
 // The page X is needed for the Gram matrix and again for B = A^T X; in between its bytes hold Q^T, and it is
@@ -52,11 +67,11 @@ struct CompressSmem {
         __nv_bfloat16 X2[P * kHeadDim];    // the page again, rows unpadded (projection phase)
     };
     float2 cs[P / 2];
-    uchar2 pairs[P == 64 ? 1 : (P - 1) * (P / 2)];   // this page size's rows of c_pairs (lanes index it divergently)
-    // P = 64 (quad ordering): the 4 x 4 transforms of a class's 16 quads, [variant][row][quad] as float4, and the
-    // member table
-    float4 M[P == 64 ? 2 * 4 * 16 : 1];
-    uchar4 quads[P == 64 ? kQuadClasses * kQuadsPerClass : 1];
+    uchar2 pairs[P >= 32 ? 1 : (P - 1) * (P / 2)];   // pair ordering: the rounds' pairs (lanes index it divergently)
+    // quad ordering: the 4 x 4 transforms of a class's quads, [member order][row][quad] as float4, and the table
+    using Qd = Quads<(P >= 32 ? P : 32)>;
+    float4 M[P >= 32 ? Qd::kDiag * 4 * Qd::kQuads : 1];
+    uchar4 quads[P >= 32 ? Qd::kClasses * Qd::kQuads : 1];
     float lam[P];
     int order[P];
     float red[Shape<P>::kWarps];
@@ -207,31 +222,34 @@ compress_kernel(Geometry geo, const unsigned char *dense_pool, unsigned char *fa
     for (int w = 0; w < kWarps; ++w) trace += S.red[w];
     float captured_prev = -1.f;
     bool converged = false;
-    if constexpr (P == 64) {
+    if constexpr (P >= 32) {
+        using Qd = Quads<P>;
+        constexpr int kQuads = Qd::kQuads;
         // ---- quad ordering ----
-        // A class partitions the 64 indices into 16 quads.  Inside a quad the six pairs are rotated in three layers,
+        // A class partitions the P indices into P/4 quads.  Inside a quad the six pairs are rotated in three layers,
         // (0,1)(2,3), (0,2)(1,3), (0,3)(1,2), which needs only the quad's own 4 x 4 diagonal block of G; the product
         // of the six rotations is a 4 x 4 orthogonal matrix M.  Then G' = M^T G M and Q^T' = M^T Q^T are applied
         // blockwise with dense 4 x 4 products: one pass over G and Q^T covers what takes three rounds of the pair
-        // ordering, with a third of the shared-memory traffic and instructions, and 21 classes make a sweep in which
-        // every pair is rotated exactly once.
-        //   threads 0-63   four per quad: rotations and M                                        (between barriers)
-        //   warps 0-4      G: a thread owns the 4 x 4 block (quad a, quad b) of a mirror-image couple, lanes walk
-        //                  two wrapped diagonals (b = a + delta mod 16; delta = 0 .. 8, 136 blocks), read 16
-        //                  entries, write 16 and their mirror images
-        //   warps 5-7      Q^T: a thread owns (quad, four tokens): four 128-bit loads, 64 FMAs, four stores
-        // Banks: an entry's bank is its column index mod 32.  Lanes 0-15 take their quads' members in table order,
-        // lanes 16-31 in the order (2, 3, 0, 1) with M permuted to match, so at any step the warp touches either
-        // all A-members or all B-members of the class: 32 different banks, for the block accesses (columns of
-        // quad b) and for the mirrored stores (columns of quad a) alike.
-        for (int i = tid; i < kQuadClasses * kQuadsPerClass; i += kThreads) S.quads[i] = c_quads[i];
+        // ordering, with a third of the shared-memory traffic and instructions; 21 classes (P = 64) or 13 (P = 32)
+        // make a sweep in which every pair is rotated (see Quads).
+        //   first P threads     four per quad: rotations and M                                   (between barriers)
+        //   first kGWarps warps G: a thread owns the 4 x 4 block (quad a, quad b) of a mirror-image couple; a group
+        //                       of P/4 lanes walks a wrapped diagonal (b = a + delta mod P/4, delta = 0 .. P/8), reads
+        //                       16 entries, writes 16 and their mirror images
+        //   the other warps     Q^T: a thread owns (quad, four tokens): four 128-bit loads, 64 FMAs, four stores
+        // Banks: an entry's bank is its column index mod 32.  Lane group g of a warp takes its quads' members in
+        // the order j ^ x (x = 0, 2 for the two groups at P = 64; x = 0 .. 3 for the four groups at P = 32) with M
+        // permuted to match.  At P = 64 the warp then touches either all A-members or all B-members of the class at
+        // any step, at P = 32 one member of each kind of every quad, i.e. all 32 indices: 32 different banks, for
+        // the block accesses (columns of quad b) and for the mirrored stores (columns of quad a) alike.
+        for (int i = tid; i < Qd::kClasses * kQuads; i += kThreads) S.quads[i] = P == 64 ? c_quads64[i] : c_quads32[i];
         __syncthreads();
         float4 *QT4 = reinterpret_cast<float4 *>(S.QT);
         for (int sweep = 0; sweep < geo.jacobi_max_sweeps && !converged; ++sweep) {
             int rotated = 0;
-            for (int cls = 0; cls < kQuadClasses && !converged; ++cls) {
-                const uchar4 *quads = S.quads + cls * kQuadsPerClass;
-                if (tid < 4 * kQuadsPerClass) {
+            for (int cls = 0; cls < Qd::kClasses && !converged; ++cls) {
+                const uchar4 *quads = S.quads + cls * kQuads;
+                if (tid < 4 * kQuads) {
                     // Four lanes per quad; lane t holds row t of the quad's diagonal block D and of M, stored
                     // "rotated": e[k] = D[t][t ^ k], f[k] = M[t][t ^ k], so that the partner of layer x (t ^ x), the
                     // pivot (e[x]) and the column pairs (k, k ^ x) have compile-time positions.
@@ -281,21 +299,27 @@ compress_kernel(Geometry geo, const unsigned char *dense_pool, unsigned char *fa
                     float r0 = f[0], r1 = f[1], r2 = f[2], r3 = f[3];
                     if (t & 1) { float w = r0; r0 = r1; r1 = w; w = r2; r2 = r3; r3 = w; }
                     if (t & 2) { float w = r0; r0 = r2; r2 = w; w = r1; r1 = r3; r3 = w; }
-                    S.M[(0 * 4 + t) * 16 + qd] = make_float4(r0, r1, r2, r3);
-                    S.M[(1 * 4 + (t ^ 2)) * 16 + qd] = make_float4(r2, r3, r0, r1);
+                    const float r[4] = {r0, r1, r2, r3};
+#pragma unroll
+                    for (int g = 0; g < Qd::kDiag; ++g) {              // M'[k][j] = M[k ^ x][j ^ x] for member order j ^ x
+                        constexpr int kStep = Qd::kVarStep;
+                        const int x = g * kStep;
+                        S.M[(g * 4 + (t ^ x)) * kQuads + qd] = make_float4(r[0 ^ x], r[1 ^ x], r[2 ^ x], r[3 ^ x]);
+                    }
                 }
                 __syncthreads();
-                if (warp < 5) {
-                    const int h = lane >> 4, ia = lane & 15, delta = 2 * warp + h;
-                    if (delta < 8 || (delta == 8 && ia < 8)) {
-                        const int ib = (ia + delta) & 15;
-                        unsigned ma4 = reinterpret_cast<const unsigned *>(quads)[ia];
-                        unsigned mb4 = reinterpret_cast<const unsigned *>(quads)[ib];
-                        if (h) { ma4 = __byte_perm(ma4, 0u, 0x1032); mb4 = __byte_perm(mb4, 0u, 0x1032); }
+                if (warp < Qd::kGWarps) {
+                    const int h = lane / kQuads, ia = lane % kQuads, delta = Qd::kDiag * warp + h;
+                    if (delta < kQuads / 2 || (delta == kQuads / 2 && ia < kQuads / 2)) {
+                        const int ib = (ia + delta) % kQuads;
+                        // member order j ^ x: byte j of the permuted word is byte j ^ x of the table's
+                        const unsigned sel = 0x3210u ^ (0x1111u * (unsigned)(h * Qd::kVarStep));
+                        const unsigned ma4 = __byte_perm(reinterpret_cast<const unsigned *>(quads)[ia], 0u, sel);
+                        const unsigned mb4 = __byte_perm(reinterpret_cast<const unsigned *>(quads)[ib], 0u, sel);
                         int ma[4], mb[4];
 #pragma unroll
                         for (int i = 0; i < 4; ++i) { ma[i] = (ma4 >> (8 * i)) & 0xff; mb[i] = (mb4 >> (8 * i)) & 0xff; }
-                        const float4 *Ma = S.M + h * 64 + ia, *Mb = S.M + h * 64 + ib;
+                        const float4 *Ma = S.M + h * 4 * kQuads + ia, *Mb = S.M + h * 4 * kQuads + ib;
                         float T[4][4];
 #pragma unroll
                         for (int i = 0; i < 4; ++i)
@@ -303,7 +327,7 @@ compress_kernel(Geometry geo, const unsigned char *dense_pool, unsigned char *fa
                             for (int j = 0; j < 4; ++j) T[i][j] = 0.f;
 #pragma unroll
                         for (int k = 0; k < 4; ++k) {                  // T = M_a^T X
-                            const float4 mk = Ma[k * 16];
+                            const float4 mk = Ma[k * kQuads];
                             const float *row = S.G + ma[k] * kGs;
 #pragma unroll
                             for (int j = 0; j < 4; ++j) {
@@ -312,7 +336,7 @@ compress_kernel(Geometry geo, const unsigned char *dense_pool, unsigned char *fa
                                 T[2][j] = fmaf(mk.z, x, T[2][j]); T[3][j] = fmaf(mk.w, x, T[3][j]);
                             }
                         }
-                        const float4 b0 = Mb[0], b1 = Mb[16], b2 = Mb[32], b3 = Mb[48];
+                        const float4 b0 = Mb[0], b1 = Mb[kQuads], b2 = Mb[2 * kQuads], b3 = Mb[3 * kQuads];
 #pragma unroll
                         for (int i = 0; i < 4; ++i) {                  // Y = T M_b, row i
                             float y[4];
@@ -331,13 +355,13 @@ compress_kernel(Geometry geo, const unsigned char *dense_pool, unsigned char *fa
                         }
                     }
                 } else {
-                    for (int itq = (warp - 5) * 3; itq < min(8, (warp - 5) * 3 + 3); ++itq) {
-                        const int v = itq * 32 + lane, k = v >> 4, ch = v & 15;
+                    for (int itq = warp - Qd::kGWarps; itq < Qd::kQIters; itq += kWarps - Qd::kGWarps) {
+                        const int v = itq * 32 + lane, k = v / (P / 4), ch = v % (P / 4);
                         const uchar4 m4 = quads[k];
                         float4 *r0 = QT4 + m4.x * (P / 4) + ch, *r1 = QT4 + m4.y * (P / 4) + ch;
                         float4 *r2 = QT4 + m4.z * (P / 4) + ch, *r3 = QT4 + m4.w * (P / 4) + ch;
                         const float4 x0 = *r0, x1 = *r1, x2 = *r2, x3 = *r3;
-                        const float4 c0 = S.M[0 * 16 + k], c1 = S.M[1 * 16 + k], c2 = S.M[2 * 16 + k], c3 = S.M[3 * 16 + k];
+                        const float4 c0 = S.M[k], c1 = S.M[kQuads + k], c2 = S.M[2 * kQuads + k], c3 = S.M[3 * kQuads + k];
 #define PKV_MIX(comp) make_float4(fmaf(c3.comp, x3.x, fmaf(c2.comp, x2.x, fmaf(c1.comp, x1.x, c0.comp * x0.x))), \
                                   fmaf(c3.comp, x3.y, fmaf(c2.comp, x2.y, fmaf(c1.comp, x1.y, c0.comp * x0.y))), \
                                   fmaf(c3.comp, x3.z, fmaf(c2.comp, x2.z, fmaf(c1.comp, x1.z, c0.comp * x0.z))), \
@@ -347,13 +371,13 @@ compress_kernel(Geometry geo, const unsigned char *dense_pool, unsigned char *fa
                     }
                 }
                 __syncthreads();
-                // three checks per sweep
-                if (cls % 7 == 6 && geo.jacobi_energy_tol >= 0.f && energy_converged<P>(S, rank, geo.jacobi_energy_tol, trace, captured_prev, tid, lane, warp)) converged = true;
+                // about three checks per sweep
+                if (((cls + 1) % Qd::kCheck == 0 || cls == Qd::kClasses - 1) && geo.jacobi_energy_tol >= 0.f && energy_converged<P>(S, rank, geo.jacobi_energy_tol, trace, captured_prev, tid, lane, warp)) converged = true;
             }
             if (!__syncthreads_or(rotated)) converged = true;
         }
     } else {
-        // ---- cyclic Jacobi sweeps, pair ordering (P = 16, 32) ----
+        // ---- cyclic Jacobi sweeps, pair ordering (P = 16) ----
         // 2 x 2 blocks of G computed per round: one of each mirror-image couple, and the diagonal blocks
         constexpr int kBlocks = kPairs * (kPairs / 2) + kPairs / 2;
         constexpr int kChunks = P / 4;               // float4 chunks of a row of Q^T
@@ -369,7 +393,7 @@ compress_kernel(Geometry geo, const unsigned char *dense_pool, unsigned char *fa
         // other one takes its pairs in the opposite order, (q, p) with the rotation (c, -s), which is the same
         // rotation, so that it touches second members while its neighbour touches first members.
         // Q^T is stored instead of Q: rotating columns p, q of Q is rotating rows p, q of Q^T, four tokens at a time.
-        for (int i = tid; i < (P - 1) * kPairs; i += kThreads) S.pairs[i] = c_pairs[pair_table_offset(P) + i];
+        for (int i = tid; i < (P - 1) * kPairs; i += kThreads) S.pairs[i] = c_pairs[i];
         __syncthreads();
         const uchar2 *pairs = S.pairs;
         for (int sweep = 0; sweep < geo.jacobi_max_sweeps && !converged; ++sweep) {
@@ -574,7 +598,7 @@ compress_kernel(Geometry geo, const unsigned char *dense_pool, unsigned char *fa
     }
 }
 
-// Round-robin pairs of every round (P = 16, 32).
+// Round-robin pairs of every round (P = 16).
 void fill_pair_table(int P, uchar2 *out) {
     const int B = P / 2;
     for (int rho = 0; rho < P - 1; ++rho)
@@ -586,8 +610,9 @@ void fill_pair_table(int P, uchar2 *out) {
 }
 
 // The 21 parallel classes of lines of AG(3, 4) over the indices 0..63 (index = x0 + 4 x1 + 16 x2, coordinates in
-// GF(4) = {0, 1, w, w^2} with addition = xor), members ordered (A, B, A, B) as c_quads describes.
-void fill_quad_table(uchar4 *out) {
+// GF(4) = {0, 1, w, w^2} with addition = xor), members ordered (A, B, A, B) as Quads describes.
+void fill_quad_table64(uchar4 *out) {
+    constexpr int kQuadClasses = Quads<64>::kClasses, kQuadsPerClass = Quads<64>::kQuads;
     static const int mul[4][4] = {{0, 0, 0, 0}, {0, 1, 2, 3}, {0, 2, 3, 1}, {0, 3, 1, 2}};
     int dirs[kQuadClasses][3], nd = 0;
     for (int a = 0; a < 4; ++a) for (int b = 0; b < 4; ++b) { dirs[nd][0] = 1; dirs[nd][1] = a; dirs[nd][2] = b; ++nd; }
@@ -635,15 +660,53 @@ void fill_quad_table(uchar4 *out) {
     }
 }
 
+// The 13 classes of 8 quads for 32 indices (see Quads): GF(4)^2 lines inside each half of 16, then the classes that
+// pair the halves.  Index inside a half = x0 + 4 x1.
+void fill_quad_table32(uchar4 *out) {
+    static const int mul[4][4] = {{0, 0, 0, 0}, {0, 1, 2, 3}, {0, 2, 3, 1}, {0, 3, 1, 2}};
+    static const int dirs[5][2] = {{1, 0}, {1, 1}, {1, 2}, {1, 3}, {0, 1}};
+    int n = 0;
+    for (int c = 0; c < 5; ++c) {
+        bool seen[16] = {};
+        for (int x = 0; x < 16; ++x) {
+            if (seen[x]) continue;
+            int m[4];
+            for (int t = 0; t < 4; ++t) {
+                m[t] = ((x & 3) ^ mul[t][dirs[c][0]]) | (((x >> 2) & 3) ^ mul[t][dirs[c][1]]) << 2;
+                seen[m[t]] = true;
+            }
+            out[n++] = make_uchar4((unsigned char)m[0], (unsigned char)m[1], (unsigned char)m[2], (unsigned char)m[3]);
+        }
+        for (int l = 0; l < 4; ++l) {                       // the same four lines in the other half
+            const uchar4 q = out[n - 4];
+            out[n++] = make_uchar4((unsigned char)(q.x + 16), (unsigned char)(q.y + 16), (unsigned char)(q.z + 16),
+                                   (unsigned char)(q.w + 16));
+        }
+    }
+    // differences 0..15 in couples {a, a ^ u}; u varies so that the repeated pairs inside the halves vary too
+    static const int couple[8][2] = {{0, 1}, {2, 6}, {3, 11}, {4, 5}, {7, 15}, {8, 10}, {9, 13}, {12, 14}};
+    for (int c = 0; c < 8; ++c) {
+        const int a = couple[c][0], u = couple[c][0] ^ couple[c][1];
+        bool seen[16] = {};
+        for (int x = 0; x < 16; ++x) {
+            if (seen[x]) continue;
+            seen[x] = seen[x ^ u] = true;
+            out[n++] = make_uchar4((unsigned char)x, (unsigned char)(16 + (x ^ a)), (unsigned char)(x ^ u),
+                                   (unsigned char)(16 + (x ^ u ^ a)));
+        }
+    }
+}
+
 cudaError_t upload_pair_tables() {
-    static uchar2 host[15 * 8 + 31 * 16];
-    fill_pair_table(16, host + pair_table_offset(16));
-    fill_pair_table(32, host + pair_table_offset(32));
+    static uchar2 host[15 * 8];
+    fill_pair_table(16, host);
     cudaError_t e = cudaMemcpyToSymbol(c_pairs, host, sizeof host);
     if (e != cudaSuccess) return e;
-    static uchar4 quads[kQuadClasses * kQuadsPerClass];
-    fill_quad_table(quads);
-    return cudaMemcpyToSymbol(c_quads, quads, sizeof quads);
+    static uchar4 quads64[Quads<64>::kClasses * Quads<64>::kQuads], quads32[Quads<32>::kClasses * Quads<32>::kQuads];
+    fill_quad_table64(quads64);
+    fill_quad_table32(quads32);
+    if ((e = cudaMemcpyToSymbol(c_quads64, quads64, sizeof quads64)) != cudaSuccess) return e;
+    return cudaMemcpyToSymbol(c_quads32, quads32, sizeof quads32);
 }
 
 template <int P>
