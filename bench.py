@@ -340,7 +340,7 @@ def _config_dict(args, w, rank):
             "overlap": ["0: each launch waits for the previous one",
                         "1: consecutive per-layer launches overlap (programmatic dependent launch) and complete in order",
                         "2: per-layer launches overlap freely (programmatic dependent launch, rotating split-K scratch, "
-                        "a draining launch every 15); valid here because queries are prepared in advance and no "
+                        "a draining launch every 63); valid here because queries are prepared in advance and no "
                         "launch in the step writes the cache"][args.overlap],
             "launch": "one CUDA graph replay per step (%d per-layer launches)" % w.get("layers_per_step", w["n_layers"]) if args.graph else "host launch per layer",
             "parallelism": "replicas x%d" % args.gpus}

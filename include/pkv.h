@@ -103,7 +103,8 @@ typedef struct pkv_config {
                                    2: the same promise for ALL decode launches that may be in flight, and `out`
                                       buffers of consecutive calls must be distinct (or hold the same values).
                                       Launches never wait for one another and may complete out of order; the
-                                      library rotates the split-K scratch over 16 sets and makes every 15th
+                                      library rotates the split-K scratch over n sets (n = 64, fewer where 64 sets
+                                      would exceed 128 MiB of workspace, at least 4) and makes every (n-1)-th
                                       launch an ordinary one, which starts only after all earlier work on the
                                       stream has finished.  Not capturable into a CUDA graph (the call returns
                                       PKV_ERR_UNSUPPORTED while the stream is capturing).

@@ -209,10 +209,16 @@ void derive(const pkv_config &cfg, int n_ctas, Geometry &g, MetaLayout &ml, Work
     wl.n_partials = (long long)n_ctas + (long long)cfg.max_seqs * cfg.n_kv_heads;
     long long w = 0;
     wl.partials_stride = align_up(wl.n_partials * kPartialFloats * 4, 256);
-    wl.partials = w; w += wl.partials_stride * kDecodeBuffers;
-    wl.worklist = w; w = align_up(w + (long long)sizeof(int2) * kCompressChunk, 256);
     wl.tickets_stride = align_up(4LL * cfg.max_seqs * cfg.n_kv_heads, 256);
-    wl.tickets = w;  w += wl.tickets_stride * kDecodeBuffers;
+    // decode_overlap = 2 rotates over several sets of split-K scratch; the more sets, the rarer the draining launch
+    wl.n_sets = 1;
+    if (cfg.decode_overlap == 2) {
+        const long long fit = kDecodeBufferBudget / (wl.partials_stride + wl.tickets_stride);
+        wl.n_sets = (int)std::min<long long>(kMaxDecodeBuffers, std::max<long long>(4, fit));
+    }
+    wl.partials = w; w += wl.partials_stride * wl.n_sets;
+    wl.worklist = w; w = align_up(w + (long long)sizeof(int2) * kCompressChunk, 256);
+    wl.tickets = w;  w += wl.tickets_stride * wl.n_sets;
     wl.trace = w;    w = align_up(w + 64LL * n_ctas, 256);
     wl.total = w;
 }
@@ -667,7 +673,7 @@ pkv_status pkv_decode_attention(pkv_cache *c, int32_t layer, int32_t n_seqs, con
     a.plan_cta = c->ml.plan_cta; a.plan_entry = c->ml.plan_entry; a.plan_seg = c->ml.plan_seg;
     a.q = q; a.out = out; a.out_f32 = out_f32;
     // decode_overlap = 2: launches never wait for one another, so launches in flight must not share split-K
-    // scratch.  The scratch rotates over kDecodeBuffers sets and every (kDecodeBuffers-1)-th launch is a plain
+    // scratch.  The scratch rotates over wl.n_sets sets and every (n_sets-1)-th launch is a plain
     // one (no programmatic serialization: it starts after all earlier work on the stream has finished), so
     // between two users of a set the stream has always drained once.
     int buf = 0;
@@ -680,8 +686,8 @@ pkv_status pkv_decode_attention(pkv_cache *c, int32_t layer, int32_t n_seqs, con
         PKV_CUDA(c, cudaStreamIsCapturing(st, &cap));
         if (cap != cudaStreamCaptureStatusNone)
             return fail(c, PKV_ERR_UNSUPPORTED, "decode_overlap = 2 cannot be captured into a CUDA graph (use 0 or 1)");
-        buf = (int)(c->decode_seq % kDecodeBuffers);
-        if ((c->decode_seq % (kDecodeBuffers - 1)) == 0) a.plain_launch = 1;
+        buf = (int)(c->decode_seq % c->wl.n_sets);
+        if ((c->decode_seq % (c->wl.n_sets - 1)) == 0) a.plain_launch = 1;
         c->decode_seq++;
     }
     a.partials = (float *)(c->workspace + c->wl.partials + c->wl.partials_stride * buf);

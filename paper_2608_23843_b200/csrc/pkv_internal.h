@@ -17,7 +17,8 @@ constexpr int kDecodeThreads = (kConsumerWarps + 1) * 32;
 constexpr int kPartialFloats = kMaxGroup * (kHeadDim + 2);   // o[8][128], m[8], l[8]
 constexpr int kStatusWords = 8;        // [0] device timeouts, [1] page SVDs not converged, [2] slot indices out of range
 constexpr int kCompressChunk = 8192;   // work-list entries per compression launch
-constexpr int kDecodeBuffers = 16;     // decode_overlap = 2: rotating sets of split-K scratch (see pkv_decode_attention)
+constexpr int kMaxDecodeBuffers = 64;  // decode_overlap = 2: at most this many rotating sets of split-K scratch
+constexpr long long kDecodeBufferBudget = 128LL << 20;   // ... and at most this many bytes of them (but at least 4 sets)
 constexpr int kSmemBudget = 227 * 1024;
 
 // Sizes derived from a validated pkv_config.  Plain data: passed to kernels by value.
@@ -69,7 +70,8 @@ struct MetaLayout {                    // byte offsets inside the caller's `meta
 };
 
 struct WorkspaceLayout {
-    long long partials;                // float [kDecodeBuffers][n_partials][kPartialFloats]
+    int n_sets;                        // rotating sets of split-K scratch: 1 unless decode_overlap = 2
+    long long partials;                // float [n_sets][n_partials][kPartialFloats]
     long long n_partials;
     long long partials_stride;         // bytes of one buffer
     long long tickets_stride;

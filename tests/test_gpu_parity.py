@@ -279,7 +279,7 @@ def test_other_page_sizes_and_ranks(P, rk, rv, G):
 @pytest.mark.parametrize("overlap", [1, 2])
 def test_overlapping_launches_give_the_serialised_result(overlap):
     """Many back-to-back decode launches over three layers with decode_overlap 1 and 2 (launches overlap on
-    the GPU; mode 2 rotates the split-K scratch and drains the stream every 15 launches): every launch must
+    the GPU; mode 2 rotates the split-K scratch over 64 sets and drains the stream every 63 launches): every launch must
     reproduce, bit for bit, what a cache with decode_overlap = 0 computes."""
     H, G, L, lengths = 2, 4, 3, [2600, 700]
     outs = {}
@@ -293,7 +293,7 @@ def test_overlapping_launches_give_the_serialised_result(overlap):
                 k, v = gen_kv(17, layer, s, T, cfg)
                 pair.gpu.append_kv(layer, [s], [T], k.cuda(), v.cuda())
         pair.gpu.compress_eligible_pages(-1)
-        qs = [synth.make_q(17, i % L, i, 2, H * G, 128).cuda() for i in range(50)]
+        qs = [synth.make_q(17, i % L, i, 2, H * G, 128).cuda() for i in range(150)]     # wraps around the scratch sets
         res = [torch.empty_like(q) for q in qs]
         torch.cuda.synchronize()
         for i, q in enumerate(qs):
