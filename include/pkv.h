@@ -302,6 +302,20 @@ pkv_status pkv_write_factors(pkv_cache *c, int64_t factor_slot, int32_t kv_head,
 pkv_status pkv_read_dense(pkv_cache *c, int64_t dense_slot, int32_t kv_head, void *K, void *V,
                           void *stream);
 
+/*
+ * The order in which the page-SVD kernel (pkv_compress_eligible_pages) rotates index pairs during one Jacobi sweep,
+ * for inspection and tests.  Host only: no cache, no GPU work.  (The paper fixes the decomposition, Eq. 2, not how the
+ * eigen-solve orders its rotations; this describes this library's kernel.)
+ *   page_size 64 or 32: the indices 0..P-1 are rotated in groups of four.  *n_rounds = 21 (13) classes,
+ *     *groups_per_round = P/4, *group_size = 4; inside a group the six pairs are rotated in the layers
+ *     (0,1)(2,3), (0,2)(1,3), (0,3)(1,2) of the group's member positions.
+ *   page_size 16: pairs.  *n_rounds = 15, *groups_per_round = 8, *group_size = 2.
+ * members [host, out]: n_rounds * groups_per_round * group_size bytes, round-major; `capacity` = its size in bytes.
+ * Returns PKV_ERR_INVALID_ARG for another page size, a NULL pointer or a buffer that is too small (nothing written).
+ */
+pkv_status pkv_get_rotation_schedule(int32_t page_size, uint8_t *members, int64_t capacity, int32_t *n_rounds,
+                                     int32_t *groups_per_round, int32_t *group_size);
+
 #ifdef __cplusplus
 }
 #endif

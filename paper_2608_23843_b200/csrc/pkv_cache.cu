@@ -872,6 +872,14 @@ pkv_status pkv_write_factors(pkv_cache *c, int64_t slot, int32_t head, const voi
     return PKV_OK;
 }
 
+pkv_status pkv_get_rotation_schedule(int32_t page_size, uint8_t *members, int64_t capacity, int32_t *n_rounds,
+                                     int32_t *groups_per_round, int32_t *group_size) {
+    int nr = 0, ng = 0, gs = 0;
+    if (!pkv::rotation_schedule(page_size, members, capacity, &nr, &ng, &gs)) return PKV_ERR_INVALID_ARG;
+    *n_rounds = nr; *groups_per_round = ng; *group_size = gs;
+    return PKV_OK;
+}
+
 pkv_status pkv_read_dense(pkv_cache *c, int64_t slot, int32_t head, void *K, void *V, void *stream) {
     pkv_status r = slot_args(c, slot, c ? c->cfg.n_dense_slots : 0, head);
     if (r != PKV_OK) return r;

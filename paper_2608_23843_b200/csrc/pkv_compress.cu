@@ -731,6 +731,30 @@ cudaError_t launch_p(const Geometry &geo, const unsigned char *dense_pool, unsig
 
 }  // namespace
 
+bool rotation_schedule(int P, unsigned char *out, long long cap, int *n_rounds, int *groups, int *group_size) {
+    if (!out || !n_rounds || !groups || !group_size) return false;
+    if (P == 64 || P == 32) {
+        const int nr = P == 64 ? Quads<64>::kClasses : Quads<32>::kClasses, ng = P / 4;
+        if (cap < (long long)nr * ng * 4) return false;
+        static uchar4 table[Quads<64>::kClasses * Quads<64>::kQuads];
+        if (P == 64) fill_quad_table64(table); else fill_quad_table32(table);
+        for (int i = 0; i < nr * ng; ++i) {
+            out[4 * i] = table[i].x; out[4 * i + 1] = table[i].y; out[4 * i + 2] = table[i].z; out[4 * i + 3] = table[i].w;
+        }
+        *n_rounds = nr; *groups = ng; *group_size = 4;
+        return true;
+    }
+    if (P == 16) {
+        if (cap < 15 * 8 * 2) return false;
+        uchar2 table[15 * 8];
+        fill_pair_table(16, table);
+        for (int i = 0; i < 15 * 8; ++i) { out[2 * i] = table[i].x; out[2 * i + 1] = table[i].y; }
+        *n_rounds = 15; *groups = 8; *group_size = 2;
+        return true;
+    }
+    return false;
+}
+
 cudaError_t launch_compress(const Geometry &geo, const unsigned char *dense_pool, unsigned char *factor_pool,
                             const int2 *worklist, int n_entries, int *status, cudaStream_t st) {
     switch (geo.page) {

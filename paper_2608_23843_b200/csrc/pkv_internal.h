@@ -120,6 +120,9 @@ cudaError_t launch_write_factors(const Geometry &geo, unsigned char *blob, const
 cudaError_t launch_read_dense(const Geometry &geo, const unsigned char *head_base, void *K, void *V,
                               cudaStream_t st);
 cudaError_t decode_kernel_setup();     // raises the dynamic shared-memory limit once per device
+// Rotation order of the compression kernel for page size P (see pkv_get_rotation_schedule); false if P is unsupported
+// or `cap` bytes are too few.
+bool rotation_schedule(int P, unsigned char *out, long long cap, int *n_rounds, int *groups, int *group_size);
 
 // Storage swizzle of a 256-byte row: 16-byte chunk c of row `row` lives at
 // chunk position c ^ (row & 7).  Applied to dense K/V rows and to B factors.

@@ -29,6 +29,7 @@ EXPORTS = [
     "pkv_decode_attention", "pkv_decode_attention_host", "pkv_get_page_table", "pkv_get_stats",
     "pkv_free_seq", "pkv_destroy_cache", "pkv_last_error", "pkv_read_factors", "pkv_write_factors",
     "pkv_read_dense", "pkv_get_decode_plan", "pkv_decode_attention_static_scratch", "pkv_get_decode_trace",
+    "pkv_get_rotation_schedule",
 ]
 
 
@@ -93,6 +94,7 @@ def lib():
         L.pkv_read_dense.argtypes = [vp, i64, i32, vp, vp, vp]
         L.pkv_get_decode_plan.argtypes = [vp, i32, ip, ip, ip, ip]
         L.pkv_get_decode_trace.argtypes = [vp, ctypes.POINTER(ctypes.c_int64), i32, vp]
+        L.pkv_get_rotation_schedule.argtypes = [i32, ctypes.POINTER(ctypes.c_uint8), i64, ip, ip, ip]
         for name in EXPORTS:
             if name != "pkv_last_error":
                 getattr(L, name).restype = ctypes.c_int32
@@ -228,6 +230,18 @@ def pkv_read_factors(handle, slot, kv_head, A_k, B_k, A_v, B_v, stream=None):
 
 def pkv_write_factors(handle, slot, kv_head, A_k, B_k, A_v, B_v, stream=None):
     _check(handle, lib().pkv_write_factors(handle, slot, kv_head, _ptr(A_k), _ptr(B_k), _ptr(A_v), _ptr(B_v), _stream(stream)))
+
+
+def pkv_get_rotation_schedule(page_size):
+    """-> list of rounds, each a list of groups (tuples of member indices)."""
+    buf = (ctypes.c_uint8 * 4096)()
+    nr, ng, gs = ctypes.c_int32(), ctypes.c_int32(), ctypes.c_int32()
+    rc = lib().pkv_get_rotation_schedule(int(page_size), buf, 4096, ctypes.byref(nr), ctypes.byref(ng), ctypes.byref(gs))
+    if rc != PKV_OK:
+        raise PkvError(rc, "pkv_get_rotation_schedule(%r)" % (page_size,))
+    flat = list(buf[:nr.value * ng.value * gs.value])
+    it = iter(flat)
+    return [[tuple(next(it) for _ in range(gs.value)) for _ in range(ng.value)] for _ in range(nr.value)]
 
 
 def pkv_read_dense(handle, slot, kv_head, K, V, stream=None):

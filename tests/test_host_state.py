@@ -242,3 +242,35 @@ def test_decode_plan_covers_every_unit_once_and_is_balanced(lengths, rank):
                     if any(flat[x][0] * H + flat[x][1] == s for x in (a, b - 1)) or
                     (flat[a][0] * H + flat[a][1] < s < flat[b - 1][0] * H + flat[b - 1][1])]
         assert segs[s] == (touching[0], len(touching)), s
+
+
+@pytest.mark.parametrize("P", [64, 32, 16])
+def test_rotation_schedule_of_the_page_svd_kernel(P):
+    """The order in which the compression kernel rotates index pairs within a sweep (host-side table, no GPU):
+    every round partitions the indices; a sweep contains every pair of indices (exactly once for P = 64 and 16;
+    for P = 32, where no such design exists, 64 of the 496 pairs come two or three times); for P = 64 the members
+    at positions {0, 2} of a round's groups fall into 32 different shared-memory banks (index mod 32), and so do
+    the members at positions {1, 3}, which is what keeps the kernel's accesses conflict-free."""
+    rounds = pkv.pkv_get_rotation_schedule(P)
+    expect = {64: (21, 16, 4), 32: (13, 8, 4), 16: (15, 8, 2)}[P]
+    assert (len(rounds), len(rounds[0]), len(rounds[0][0])) == expect
+    seen = np.zeros((P, P), dtype=int)
+    for groups in rounds:
+        assert sorted(m for g in groups for m in g) == list(range(P))          # a partition
+        for g in groups:
+            for i in range(len(g)):
+                for j in range(i + 1, len(g)):
+                    seen[g[i], g[j]] += 1
+                    seen[g[j], g[i]] += 1
+        if P == 64:
+            for positions in ((0, 2), (1, 3)):
+                banks = sorted(g[k] % 32 for g in groups for k in positions)
+                assert banks == list(range(32))
+    off = seen[~np.eye(P, dtype=bool)]
+    assert off.min() >= 1
+    if P == 32:
+        assert off.max() <= 3 and int((off > 1).sum()) // 2 == 64
+    else:
+        assert off.max() == 1
+    with pytest.raises(pkv.PkvError):
+        pkv.pkv_get_rotation_schedule(48)
