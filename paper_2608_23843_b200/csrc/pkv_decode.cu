@@ -411,72 +411,99 @@ __device__ __forceinline__ void factor_unit(uint32_t sb, int ak, int bk, int av,
     const int l7 = lane & 7, mi = lane >> 3, t2 = (lane & 3) * 2;
     const int asw = a_swz<P>(l7);
     // ---- q~^T [G][r] = q [G][d] . B_k^T ----
+    // (the loops run over the independent accumulators innermost, so that consecutive mma do not wait for
+    // one another)
     uint32_t qhi[NT], qlo[NT];
+    {
+        float qt[NT][4];
 #pragma unroll
-    for (int j = 0; j < NT; ++j) {
-        float qt[4] = {0.f, 0.f, 0.f, 0.f};
+        for (int j = 0; j < NT; ++j) qt[j][0] = qt[j][1] = qt[j][2] = qt[j][3] = 0.f;
 #pragma unroll
         for (int qd = 0; qd < 4; ++qd) {
-            uint32_t b[4];
-            ldsm_x4(b, sb + bk + (8 * j + l7) * kRowBytes + (((4 * qd + mi) ^ l7) << 4));
-            mma16816(qt, qf[2 * qd][0], 0u, qf[2 * qd][1], 0u, b[0], b[1]);
-            mma16816(qt, qf[2 * qd + 1][0], 0u, qf[2 * qd + 1][1], 0u, b[2], b[3]);
+            uint32_t b[NT][4];
+#pragma unroll
+            for (int j = 0; j < NT; ++j) ldsm_x4(b[j], sb + bk + (8 * j + l7) * kRowBytes + (((4 * qd + mi) ^ l7) << 4));
+#pragma unroll
+            for (int j = 0; j < NT; ++j) mma16816(qt[j], qf[2 * qd][0], 0u, qf[2 * qd][1], 0u, b[j][0], b[j][1]);
+#pragma unroll
+            for (int j = 0; j < NT; ++j) mma16816(qt[j], qf[2 * qd + 1][0], 0u, qf[2 * qd + 1][1], 0u, b[j][2], b[j][3]);
         }
-        const float x0 = (8 * j + t2 < rk) ? qt[0] * scale : 0.f;
-        const float x1 = (8 * j + t2 + 1 < rk) ? qt[1] * scale : 0.f;
-        qhi[j] = pack_bf16(x0, x1);
-        qlo[j] = pack_bf16(x0 - bf16lo_f(qhi[j]), x1 - bf16hi_f(qhi[j]));
+#pragma unroll
+        for (int j = 0; j < NT; ++j) {
+            const float x0 = (8 * j + t2 < rk) ? qt[j][0] * scale : 0.f;
+            const float x1 = (8 * j + t2 + 1 < rk) ? qt[j][1] * scale : 0.f;
+            qhi[j] = pack_bf16(x0, x1);
+            qlo[j] = pack_bf16(x0 - bf16lo_f(qhi[j]), x1 - bf16hi_f(qhi[j]));
+        }
     }
     // ---- s [P][G] = A_k [P][r] . q~   (A_k^T in shared memory: transposed tile loads) ----
     float s[4][4];
 #pragma unroll
-    for (int i = 0; i < C::kMT; ++i) {
-        s[i][0] = s[i][1] = s[i][2] = s[i][3] = 0.f;
+    for (int i = 0; i < C::kMT; ++i) s[i][0] = s[i][1] = s[i][2] = s[i][3] = 0.f;
 #pragma unroll
-        for (int kk = 0; kk < NT / 2; ++kk) {
-            uint32_t a4[4];
-            ldsm_x4_t(a4, sb + ak + (16 * kk + (mi >> 1) * 8 + l7) * C::kPitchA + (((2 * i + (mi & 1)) ^ asw) << 4));
-            mma16816(s[i], a4[0], a4[1], a4[2], a4[3], qhi[2 * kk], qhi[2 * kk + 1]);
-            mma16816(s[i], a4[0], a4[1], a4[2], a4[3], qlo[2 * kk], qlo[2 * kk + 1]);
-        }
-        if (NT % 2) {
-            uint32_t a2[2];
-            ldsm_x2_t(a2, sb + ak + (8 * (NT - 1) + l7) * C::kPitchA + (((2 * i + (mi & 1)) ^ asw) << 4));
-            mma1688(s[i], a2[0], a2[1], qhi[NT - 1]);
-            mma1688(s[i], a2[0], a2[1], qlo[NT - 1]);
-        }
+    for (int kk = 0; kk < NT / 2; ++kk) {
+        uint32_t a4[C::kMT][4];
+#pragma unroll
+        for (int i = 0; i < C::kMT; ++i)
+            ldsm_x4_t(a4[i], sb + ak + (16 * kk + (mi >> 1) * 8 + l7) * C::kPitchA + (((2 * i + (mi & 1)) ^ asw) << 4));
+#pragma unroll
+        for (int i = 0; i < C::kMT; ++i) mma16816(s[i], a4[i][0], a4[i][1], a4[i][2], a4[i][3], qhi[2 * kk], qhi[2 * kk + 1]);
+#pragma unroll
+        for (int i = 0; i < C::kMT; ++i) mma16816(s[i], a4[i][0], a4[i][1], a4[i][2], a4[i][3], qlo[2 * kk], qlo[2 * kk + 1]);
+    }
+    if (NT % 2) {
+        uint32_t a2[C::kMT][2];
+#pragma unroll
+        for (int i = 0; i < C::kMT; ++i)
+            ldsm_x2_t(a2[i], sb + ak + (8 * (NT - 1) + l7) * C::kPitchA + (((2 * i + (mi & 1)) ^ asw) << 4));
+#pragma unroll
+        for (int i = 0; i < C::kMT; ++i) mma1688(s[i], a2[i][0], a2[i][1], qhi[NT - 1]);
+#pragma unroll
+        for (int i = 0; i < C::kMT; ++i) mma1688(s[i], a2[i][0], a2[i][1], qlo[NT - 1]);
     }
     uint32_t T0[4], T1[4];
     online_softmax<C::kMT>(s, st, T0, T1);
     // ---- w^T [G][r] = p^T [G][P] . A_v [P][r] ----
     uint32_t wh[NT];
+    {
+        float wt[NT][4];
 #pragma unroll
-    for (int j = 0; j < NT; ++j) {
-        float wt[4] = {0.f, 0.f, 0.f, 0.f};
+        for (int j = 0; j < NT; ++j) wt[j][0] = wt[j][1] = wt[j][2] = wt[j][3] = 0.f;
 #pragma unroll
         for (int qd = 0; qd < C::kMT / 2; ++qd) {
-            uint32_t b[4];
-            ldsm_x4(b, sb + av + (8 * j + l7) * C::kPitchA + (((4 * qd + mi) ^ asw) << 4));
-            mma16816(wt, T0[2 * qd], 0u, T1[2 * qd], 0u, b[0], b[1]);
-            mma16816(wt, T0[2 * qd + 1], 0u, T1[2 * qd + 1], 0u, b[2], b[3]);
+            uint32_t b[NT][4];
+#pragma unroll
+            for (int j = 0; j < NT; ++j) ldsm_x4(b[j], sb + av + (8 * j + l7) * C::kPitchA + (((4 * qd + mi) ^ asw) << 4));
+#pragma unroll
+            for (int j = 0; j < NT; ++j) mma16816(wt[j], T0[2 * qd], 0u, T1[2 * qd], 0u, b[j][0], b[j][1]);
+#pragma unroll
+            for (int j = 0; j < NT; ++j) mma16816(wt[j], T0[2 * qd + 1], 0u, T1[2 * qd + 1], 0u, b[j][2], b[j][3]);
         }
         if (C::kMT % 2) {
-            uint32_t b[2];
-            ldsm_x2(b, sb + av + (8 * j + l7) * C::kPitchA + (((2 * (C::kMT - 1) + (mi & 1)) ^ asw) << 4));
-            mma16816(wt, T0[C::kMT - 1], 0u, T1[C::kMT - 1], 0u, b[0], b[1]);
+#pragma unroll
+            for (int j = 0; j < NT; ++j) {
+                uint32_t b[2];
+                ldsm_x2(b, sb + av + (8 * j + l7) * C::kPitchA + (((2 * (C::kMT - 1) + (mi & 1)) ^ asw) << 4));
+                mma16816(wt[j], T0[C::kMT - 1], 0u, T1[C::kMT - 1], 0u, b[0], b[1]);
+            }
         }
-        wh[j] = pack_bf16((8 * j + t2 < rv) ? wt[0] : 0.f, (8 * j + t2 + 1 < rv) ? wt[1] : 0.f);
+#pragma unroll
+        for (int j = 0; j < NT; ++j)
+            wh[j] = pack_bf16((8 * j + t2 < rv) ? wt[j][0] : 0.f, (8 * j + t2 + 1 < rv) ? wt[j][1] : 0.f);
     }
     // ---- o [d][G] += B_v^T [d][r] . w ----
 #pragma unroll
-    for (int i = 0; i < 8; ++i) {
+    for (int kk = 0; kk < NT / 2; ++kk) {
 #pragma unroll
-        for (int kk = 0; kk < NT / 2; ++kk) {
+        for (int i = 0; i < 8; ++i) {
             uint32_t a4[4];
             ldsm_x4_t(a4, sb + bv + (16 * kk + (mi >> 1) * 8 + l7) * kRowBytes + (((2 * i + (mi & 1)) ^ l7) << 4));
             mma16816(st.o[i], a4[0], a4[1], a4[2], a4[3], wh[2 * kk], wh[2 * kk + 1]);
         }
-        if (NT % 2) {
+    }
+    if (NT % 2) {
+#pragma unroll
+        for (int i = 0; i < 8; ++i) {
             uint32_t a2[2];
             ldsm_x2_t(a2, sb + bv + (8 * (NT - 1) + l7) * kRowBytes + (((2 * i + (mi & 1)) ^ l7) << 4));
             mma1688(st.o[i], a2[0], a2[1], wh[NT - 1]);
