@@ -705,6 +705,59 @@ __device__ __forceinline__ void store_out(const DecodeArgs &a, int seg, int hq, 
     if (a.out_f32) *reinterpret_cast<float4 *>(a.out_f32 + off) = acc;
 }
 
+// Eq. 5 across CTAs: the partial states of one segment, summed in CTA order with a running maximum (one pass).
+// A thread owns E items (query head, four dims): ctid, ctid + kThreads, ...; kBatch parts' loads are in flight at a
+// time, because with dozens of parts it is the latency of these loads that the rest of the GPU waits for.
+template <int E, int kBatch>
+__device__ __forceinline__ void merge_parts(const DecodeArgs &a, const float *first, int np, int seg, int ctid) {
+    constexpr int kThreads = kConsumerWarps * 32;
+    const int n_items = a.geo.group * 32;
+    const int d4 = (ctid & 31) * 4;                               // kThreads is a multiple of 32
+    bool has[E];
+    int hq[E];
+    float4 tot[E];
+    float Mr[E], Lr[E];
+#pragma unroll
+    for (int e = 0; e < E; ++e) {
+        has[e] = ctid + e * kThreads < n_items;
+        hq[e] = has[e] ? (ctid + e * kThreads) >> 5 : 0;
+        tot[e] = make_float4(0.f, 0.f, 0.f, 0.f);
+        Mr[e] = kNegInf;
+        Lr[e] = 0.f;
+    }
+    for (int k0 = 0; k0 < np; k0 += kBatch) {
+        float4 o[E][kBatch];
+        float m[E][kBatch], l[E][kBatch];
+#pragma unroll
+        for (int j = 0; j < kBatch; ++j) {
+            const float *pk = first + (long long)min(k0 + j, np - 1) * kPartialFloats;
+#pragma unroll
+            for (int e = 0; e < E; ++e) {
+                o[e][j] = __ldcg(reinterpret_cast<const float4 *>(pk + hq[e] * kHeadDim + d4));
+                m[e][j] = __ldcg(pk + kMaxGroup * kHeadDim + hq[e]);
+                l[e][j] = __ldcg(pk + kMaxGroup * kHeadDim + kMaxGroup + hq[e]);
+            }
+        }
+#pragma unroll
+        for (int j = 0; j < kBatch; ++j) {
+            if (k0 + j < np) {
+#pragma unroll
+                for (int e = 0; e < E; ++e) {
+                    const float Mn = fmaxf(Mr[e], m[e][j]);
+                    const float fa = exp2f(Mr[e] - Mn), fb = exp2f(m[e][j] - Mn);
+                    tot[e].x = tot[e].x * fa + fb * o[e][j].x; tot[e].y = tot[e].y * fa + fb * o[e][j].y;
+                    tot[e].z = tot[e].z * fa + fb * o[e][j].z; tot[e].w = tot[e].w * fa + fb * o[e][j].w;
+                    Lr[e] = Lr[e] * fa + fb * l[e][j];
+                    Mr[e] = Mn;
+                }
+            }
+        }
+    }
+#pragma unroll
+    for (int e = 0; e < E; ++e)
+        if (has[e]) store_out(a, seg, hq[e], d4, tot[e], Lr[e]);
+}
+
 #define PKV_CONSUMER_BARRIER() asm volatile("bar.sync 1, %0;" ::"n"(kConsumerWarps * 32) : "memory")
 
 // All consumer warps combine their states of one segment (Eq. 5 inside the CTA).  If the segment
@@ -773,47 +826,8 @@ __device__ __forceinline__ void flush_segment(const DecodeArgs &a, float *comb, 
         if (*last_flag) {
             __threadfence();
             const float *first = a.partials + ((long long)ps.cta_first + seg) * kPartialFloats;
-            // A thread owns items ctid and ctid + kThreads and walks the parts in CTA order with a running
-            // maximum (one pass); eight parts' loads are in flight at a time, because with dozens of parts
-            // it is the latency of these loads that the rest of the GPU waits for.
-            constexpr int kBatch = 8;
-            const int n_items = a.geo.group * 32, np = ps.n_parts;
-            const bool has[2] = {ctid < n_items, ctid + kThreads < n_items};
-            const int hq[2] = {has[0] ? ctid >> 5 : 0, has[1] ? (ctid + kThreads) >> 5 : 0};
-            const int d4 = (ctid & 31) * 4;                       // kThreads is a multiple of 32
-            float4 tot[2] = {make_float4(0.f, 0.f, 0.f, 0.f), make_float4(0.f, 0.f, 0.f, 0.f)};
-            float Mr[2] = {kNegInf, kNegInf}, Lr[2] = {0.f, 0.f};
-            for (int k0 = 0; k0 < np; k0 += kBatch) {
-                float4 o[2][kBatch];
-                float m[2][kBatch], l[2][kBatch];
-#pragma unroll
-                for (int j = 0; j < kBatch; ++j) {
-                    const float *pk = first + (long long)min(k0 + j, np - 1) * kPartialFloats;
-#pragma unroll
-                    for (int e = 0; e < 2; ++e) {
-                        o[e][j] = __ldcg(reinterpret_cast<const float4 *>(pk + hq[e] * kHeadDim + d4));
-                        m[e][j] = __ldcg(pk + kMaxGroup * kHeadDim + hq[e]);
-                        l[e][j] = __ldcg(pk + kMaxGroup * kHeadDim + kMaxGroup + hq[e]);
-                    }
-                }
-#pragma unroll
-                for (int j = 0; j < kBatch; ++j) {
-                    if (k0 + j < np) {
-#pragma unroll
-                        for (int e = 0; e < 2; ++e) {
-                            const float Mn = fmaxf(Mr[e], m[e][j]);
-                            const float fa = exp2f(Mr[e] - Mn), fb = exp2f(m[e][j] - Mn);
-                            tot[e].x = tot[e].x * fa + fb * o[e][j].x; tot[e].y = tot[e].y * fa + fb * o[e][j].y;
-                            tot[e].z = tot[e].z * fa + fb * o[e][j].z; tot[e].w = tot[e].w * fa + fb * o[e][j].w;
-                            Lr[e] = Lr[e] * fa + fb * l[e][j];
-                            Mr[e] = Mn;
-                        }
-                    }
-                }
-            }
-#pragma unroll
-            for (int e = 0; e < 2; ++e)
-                if (has[e]) store_out(a, seg, hq[e], d4, tot[e], Lr[e]);
+            if (a.geo.group * 32 <= kThreads) merge_parts<1, 16>(a, first, ps.n_parts, seg, ctid);
+            else merge_parts<2, 8>(a, first, ps.n_parts, seg, ctid);
             if (ctid == 0) a.tickets[seg] = 0;          // ready for the next launch
         }
     }
