@@ -341,14 +341,17 @@ pkv_status build_plan(pkv_cache *c, int layer, int n_seqs, const int32_t *seq_id
         total_cost += shapes[i].cost * H;
         total_units += (long long)shapes[i].units * H;
     }
-    // Cut the (entry, head, unit) sequence where the running cost crosses j * total / N.
+    // Cut the (entry, head, unit) sequence where the running cost crosses j * total / n_cut.  A CTA's consumer
+    // warps take units in turn, so ranges shorter than one unit per warp would not finish sooner and only add
+    // partial states to merge: small batches use fewer CTAs.
+    const int n_cut = (int)std::max<long long>(1, std::min<long long>(N, total_units / kConsumerWarps));
     std::vector<PlanCta> ctas;
-    ctas.reserve(N + 1);
+    ctas.reserve(n_cut + 1);
     {
         int i = 0, h = 0;
         long long base = 0;          // cost before (i, h)
-        for (int j = 0; j < N; ++j) {
-            long long b = (total_cost * j) / N;
+        for (int j = 0; j < n_cut; ++j) {
+            long long b = (total_cost * j) / n_cut;
             while (i < n_seqs && base + shapes[i].cost <= b) {
                 base += shapes[i].cost;
                 if (++h == H) { h = 0; ++i; }

@@ -277,11 +277,11 @@ __device__ __forceinline__ int ld_acquire_smem(const volatile int *p) {
 __device__ __forceinline__ void st_release_smem(volatile int *p, int v) {
     asm volatile("st.release.cta.shared.b32 [%0], %1;" ::"r"(smem_u32(const_cast<int *>(p))), "r"(v) : "memory");
 }
-// Bounded spin until the producer has armed unit k.
-__device__ __forceinline__ bool wait_issued(volatile int *issued, int k) {
-    if (ld_acquire_smem(issued) > k) return true;
+// Bounded spin until the producer has armed unit k in its stage (the stage's tag then reads k + 1).
+__device__ __forceinline__ bool wait_armed(volatile int *tag, int k) {
+    if (ld_acquire_smem(tag) == k + 1) return true;
     const long long t0 = clock64();
-    while (ld_acquire_smem(issued) <= k) {
+    while (ld_acquire_smem(tag) != k + 1) {
         if (clock64() - t0 > 2000000000LL) return false;
         __nanosleep(20);
     }
@@ -852,11 +852,11 @@ __global__ void __launch_bounds__(kDecodeThreads, 2) decode_tc_kernel(const __gr
     unsigned long long *empty_bar = full_bar + S;
     StageDesc *descs = reinterpret_cast<StageDesc *>(empty_bar + S);
     volatile int *abort_flag = reinterpret_cast<volatile int *>(descs + S);
-    // Units armed so far.  A parity wait cannot tell phase n from phase n-2, and bulk copies may land out of
-    // order, so a consumer first makes sure that its unit has been armed (which the producer does only after
-    // the stage's previous occupant was consumed) and only then waits on the stage's barrier.
-    volatile int *issued = abort_flag + 1;
-    volatile int *last_flag = abort_flag + 2;
+    volatile int *last_flag = abort_flag + 1;
+    // armed[s] = 1 + the unit last armed in stage s.  A parity wait cannot tell phase n from phase n-2, and bulk
+    // copies may land out of order, so a consumer first makes sure that its own unit has been armed (which the
+    // producer does only after the stage's previous occupant was consumed) and only then waits on the barrier.
+    volatile int *armed = abort_flag + 2;
 
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
     long long *trace = a.trace ? a.trace + 8LL * blockIdx.x : nullptr;
@@ -869,7 +869,7 @@ __global__ void __launch_bounds__(kDecodeThreads, 2) decode_tc_kernel(const __gr
     if (tid == 0) {
         for (int s = 0; s < S; ++s) { mbar_init(smem_u32(full_bar + s), 1); mbar_init(smem_u32(empty_bar + s), 1); }
         *abort_flag = 0;
-        *issued = 0;
+        for (int s = 0; s < S; ++s) armed[s] = 0;
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     }
     if (!I4 && stage_bytes > blob_bytes) {
@@ -924,16 +924,18 @@ __global__ void __launch_bounds__(kDecodeThreads, 2) decode_tc_kernel(const __gr
                               (long long)cur.head * geo.dense_head_bytes + blk * kDB * kRowBytes;
                     }
                 }
-                // Lanes arm their own units, S at a time (one stage each); the counter of armed units is
-                // published after each group so that consumers can free the stages the next group needs.
+                // Lanes arm their own units, S at a time (one stage each).  No lane blocks the others: all lanes
+                // poll together, and a unit is armed and tagged the moment its stage is free.  (Waiting for a
+                // whole group before telling the consumers can deadlock: a consumer may have to see unit k, of a
+                // later segment, to join the flush barrier that another warp must pass before it releases the
+                // stage that unit k + 1 is waiting for.)
                 const int n_here = min(32, u_end - u0);
                 for (int j0 = 0; j0 < n_here && ok; j0 += S) {
-                    const int cnt = min(S, n_here - j0);
-                    bool mine_ok = true;
-                    if (lane >= j0 && lane < j0 + cnt) {
-                        const int kj = k + lane, s = kj % S;
-                        if (kj >= S && !mbar_wait(smem_u32(empty_bar + s), ((kj / S) - 1) & 1)) mine_ok = false;
-                        if (mine_ok) {
+                    const int kj = k + lane, s = kj % S;
+                    bool pending = lane >= j0 && lane < min(j0 + S, n_here);
+                    const long long t0 = clock64();
+                    while (__any_sync(0xffffffffu, pending)) {
+                        if (pending && (kj < S || mbar_try_wait(smem_u32(empty_bar + s), ((kj / S) - 1) & 1))) {
                             descs[s] = StageDesc{kind, rows, seg_local, 0};
                             const uint32_t bar = smem_u32(full_bar + s);
                             const uint32_t dst = smem_u32(stages + (size_t)s * stage_bytes);
@@ -947,11 +949,13 @@ __global__ void __launch_bounds__(kDecodeThreads, 2) decode_tc_kernel(const __gr
                             } else {
                                 mbar_arrive(bar);
                             }
+                            st_release_smem(armed + s, kj + 1);
+                            if (trace && kj == 0) trace[3] = clock64();
+                            pending = false;
                         }
+                        if (clock64() - t0 > 2000000000LL) break;          // about a second: give up
                     }
-                    ok = __all_sync(0xffffffffu, mine_ok);
-                    if (ok && lane == 0) st_release_smem(issued, k + j0 + cnt);
-                    if (trace && lane == 0 && k + j0 == 0) trace[3] = clock64();
+                    ok = !__any_sync(0xffffffffu, pending);
                 }
                 k += n_here;
             }
@@ -968,7 +972,7 @@ __global__ void __launch_bounds__(kDecodeThreads, 2) decode_tc_kernel(const __gr
                 if (ok) {
                     descs[s] = StageDesc{kKindEnd, 0, rg.n_local_segs, 0};
                     mbar_arrive(smem_u32(full_bar + s));
-                    st_release_smem(issued, k + 1);
+                    st_release_smem(armed + s, k + 1);
                 }
             }
             ok = __shfl_sync(0xffffffffu, (int)ok, 0) != 0;
@@ -997,7 +1001,7 @@ __global__ void __launch_bounds__(kDecodeThreads, 2) decode_tc_kernel(const __gr
         bool ok = true;
         for (int k = warp;; k += W) {
             const int s = k % S;
-            if (ok && (*abort_flag || !wait_issued(issued, k) || !mbar_wait(smem_u32(full_bar + s), (k / S) & 1))) {
+            if (ok && (*abort_flag || !wait_armed(armed + s, k) || !mbar_wait(smem_u32(full_bar + s), (k / S) & 1))) {
                 ok = false;
                 if (lane == 0) { *abort_flag = 1; atomicAdd(a.status, 1); }
             }
@@ -1037,7 +1041,7 @@ __global__ void __launch_bounds__(kDecodeThreads, 2) decode_tc_kernel(const __gr
 
 size_t decode_smem_bytes(const Geometry &g) {
     return (size_t)g.n_stages * g.stage_bytes + kConsumerWarps * kPartialFloats * 4 +
-           g.n_stages * (8 + 8 + sizeof(StageDesc)) + 64;
+           g.n_stages * (8 + 8 + sizeof(StageDesc) + 4) + 64;
 }
 
 template <int P, int NT, bool I4>

@@ -445,3 +445,30 @@ def test_prescribed_spectra_with_and_without_the_energy_rule(P, energy_tol):
             assert err <= 1.01 * tail[p] + 4e-3 * np.linalg.norm(X[p]), (P, energy_tol, p, err, tail[p])
             # columns of A orthonormal up to bf16 rounding
             assert np.abs(A.T @ A - np.eye(r)).max() <= 2e-2, (P, energy_tol, p)
+
+
+@pytest.mark.gpu
+@pytest.mark.parametrize("rank,n_ctas", [(32, 3), (32, 8), (24, 2), (8, 5), (32, 0)])
+def test_many_tiny_segments_per_cta(rank, n_ctas):
+    """Sequences of one to seventy tokens, four KV heads, on a handful of CTAs: every CTA walks through many
+    (sequence, KV head) segments of one or two units each, some of them with no valid row, while its warps are at
+    different segments.  (With rank 32 a CTA has as many stages as consumer warps; a producer that told the
+    consumers about armed units only group by group used to deadlock here until its bounded waits gave up.)"""
+    H, G = 4, 4
+    lengths = [1, 2, 33, 64, 65, 70, 1, 31, 3, 64, 1, 1]
+    cfg = pkv.make_config(n_layers=1, n_kv_heads=H, n_q_heads=H * G, rank=rank, sink_tokens=64, recent_tokens=256,
+                          max_seqs=len(lengths), max_pages_per_seq=4, n_dense_slots=40, n_factor_slots=4,
+                          n_ctas=n_ctas)
+    pair = Pair(cfg, seed=rank + n_ctas)
+    for s, T in enumerate(lengths):
+        k, v = gen_kv(9, 0, s, T, cfg)
+        pair.append(0, [s], [k], [v])
+    order = [7, 0, 11, 3, 5, 1, 2, 10, 4, 6, 9, 8]
+    q = synth.make_q(9, 0, 0, len(order), H * G, 128)
+    for _ in range(3):
+        got, got32 = pair.decode(0, order, q)
+    st = pair.gpu.stats()
+    assert st["device_timeouts"] == 0 and st["bad_slot_indices"] == 0
+    assert not np.isnan(got).any() and not np.isnan(got32).any()
+    g = attention_gates(pair, 0, order, q, got, got32)
+    assert_attention_gates(g)
