@@ -114,6 +114,9 @@ template <int P>
 __device__ __noinline__ bool energy_converged(CompressSmem<P> &S, int rank, float energy_tol, float trace,
                                               float &captured_prev, int tid, int lane, int warp) {
     constexpr int kWarps = Shape<P>::kWarps;
+    // At full rank every orthogonal Q captures all of the energy, so the rule says nothing: keep rotating until Q
+    // holds the eigenvectors (they give the factors the smallest entries, hence the least bf16 rounding error).
+    if (rank >= P) return false;
     if (tid < P) S.lam[tid] = S.G[tid * Shape<P>::kGs + tid];
     __syncthreads();
     float mine = 0.f;
