@@ -64,3 +64,55 @@ def test_random_configurations(seed):
         # cases elsewhere keep 4e-3); the bf16 output adds its own 2^-9.
         assert max(g["kernel"]) <= 8e-3 and max(g["kernel_bf16"]) <= 1.2e-2, (what, g["kernel"], g["kernel_bf16"])
         pair.gpu.close()
+
+
+@pytest.mark.parametrize("seed", [1, 2])
+def test_random_schedules(seed):
+    """Random schedules of append (one token up to more than a page, a random subset of the sequences, every layer),
+    compress, free and decode on a random layer in random batch order: page tables bit-exact against the oracle after
+    every step, kernel gate at every decode, in every launch mode and with both factor formats."""
+    rng = random.Random(1000 + seed)
+    for case in range(5):
+        P = rng.choice([16, 32, 64])
+        L, H, G, nseq = rng.choice([1, 2, 3]), rng.choice([1, 2]), rng.choice([1, 4, 8]), rng.choice([2, 4])
+        rk = min(P, rng.choice([8, 16, 24]) if P >= 32 else rng.choice([8, 16]))
+        t_max = 14 * P
+        cfg = pkv.make_config(n_layers=L, n_kv_heads=H, n_q_heads=H * G, rank=rk, page_size=P,
+                              sink_tokens=P * rng.choice([0, 1]), recent_tokens=P * rng.choice([1, 2]), max_seqs=nseq,
+                              max_pages_per_seq=t_max // P + 2, n_dense_slots=L * nseq * 8 + 8,
+                              n_factor_slots=L * nseq * (t_max // P + 2), n_ctas=rng.choice([0, 5, 148]),
+                              decode_overlap=rng.choice([0, 1, 2]), factor_bits=rng.choice([16, 16, 4]))
+        what = (seed, case, P, L, H, G, nseq, rk, cfg.n_ctas, cfg.decode_overlap, cfg.factor_bits)
+        pair = Pair(cfg, seed=case)
+        data = {(ly, s): gen_kv(200 + case, ly, s, t_max, cfg) for ly in range(L) for s in range(nseq)}
+        T = [0] * nseq
+        for step in range(40):
+            ids = [s for s in range(nseq) if rng.random() < 0.7]
+            n_new = [min(rng.choice([1, 1, 1, 2, 5, P, P + 3]), t_max - T[s]) for s in ids]
+            ids, n_new = [s for s, n in zip(ids, n_new) if n > 0], [n for n in n_new if n > 0]
+            if ids:
+                for ly in range(L):
+                    pair.append(ly, ids, [data[(ly, s)][0][T[s]:T[s] + n] for s, n in zip(ids, n_new)],
+                                [data[(ly, s)][1][T[s]:T[s] + n] for s, n in zip(ids, n_new)])
+                for s, n in zip(ids, n_new):
+                    T[s] += n
+            if rng.random() < 0.6:
+                pair.compress(rng.choice([-1] + list(range(L))))
+            if rng.random() < 0.08:
+                s = rng.randrange(nseq)
+                pair.gpu.free_seq(s)
+                pair.orc.free_seq(s)
+                T[s] = 0
+            live = [s for s in range(nseq) if T[s] > 0]
+            if live and rng.random() < 0.7:
+                ly = rng.randrange(L)
+                rng.shuffle(live)
+                q = synth.make_q(200 + case, ly, step, len(live), H * G, 128)
+                got, got32 = pair.decode(ly, live, q)
+                assert not np.isnan(got32).any(), (what, step)
+                g = attention_gates(pair, ly, live, q, got, got32)
+                assert max(g["kernel"]) <= 8e-3 and max(g["kernel_bf16"]) <= 1.2e-2, (what, step, g["kernel"])
+            pair.same_tables()
+        st = pair.gpu.stats()
+        assert st["device_timeouts"] == 0 and st["bad_slot_indices"] == 0, (what, st)
+        pair.gpu.close()
