@@ -213,7 +213,10 @@ void derive(const pkv_config &cfg, int n_ctas, Geometry &g, MetaLayout &ml, Work
     // decode_overlap = 2 rotates over several sets of split-K scratch; the more sets, the rarer the draining launch
     wl.n_sets = 1;
     if (cfg.decode_overlap == 2) {
-        const long long fit = kDecodeBufferBudget / (wl.partials_stride + wl.tickets_stride);
+        // sized for the largest grid pkv_query_sizes() may have assumed (512 CTAs), so that the count does not
+        // depend on the grid actually used and the workspace the caller allocated is always large enough
+        const long long widest = align_up(((long long)std::max(512, n_ctas) + (long long)cfg.max_seqs * cfg.n_kv_heads) * kPartialFloats * 4, 256);
+        const long long fit = kDecodeBufferBudget / (widest + wl.tickets_stride);
         wl.n_sets = (int)std::min<long long>(kMaxDecodeBuffers, std::max<long long>(4, fit));
     }
     wl.partials = w; w += wl.partials_stride * wl.n_sets;
@@ -461,6 +464,15 @@ pkv_status pkv_init_cache(const pkv_config *cfg, void *dense_pool, void *factor_
     int n_ctas = cfg->n_ctas > 0 ? cfg->n_ctas : default_ctas(dry) * (cfg->decode_overlap ? 1 : 2);
     if (cfg->n_ctas == 0 && n_ctas > 512) n_ctas = 512;      // pkv_query_sizes() sized the buffers for <= 512
     derive(*cfg, n_ctas, c->geo, c->ml, c->wl);
+    {
+        // the caller sized meta and workspace with pkv_query_sizes(): never use more than that
+        pkv_sizes promised;
+        if (pkv_query_sizes(cfg, &promised) != PKV_OK || c->ml.total > promised.meta_bytes ||
+            c->wl.total > promised.workspace_bytes) {
+            delete c;
+            return PKV_ERR_INVALID_ARG;
+        }
+    }
     c->dense_pool = (unsigned char *)dense_pool; c->factor_pool = (unsigned char *)factor_pool;
     c->meta = (unsigned char *)meta; c->workspace = (unsigned char *)workspace;
     auto fill = [](FreeList &f, const int32_t *order, int64_t n) -> bool {

@@ -275,3 +275,22 @@ def test_rotation_schedule_of_the_page_svd_kernel(P):
         assert off.max() == 1
     with pytest.raises(pkv.PkvError):
         pkv.pkv_get_rotation_schedule(48)
+
+
+@pytest.mark.parametrize("overlap", [0, 1, 2])
+def test_buffers_promised_by_query_sizes_always_suffice(overlap):
+    """pkv_init_cache lays its metadata and workspace out for the grid it will really launch, which may differ
+    from the one pkv_query_sizes assumed; it must never need more than was promised (it refuses to start
+    otherwise), whatever the batch size, head count or grid."""
+    for max_seqs in (1, 8, 64, 256, 512, 2048, 4096):
+        for H in (1, 8):
+            for n_ctas in (0, 1, 148, 296, 512, 1000):
+                cfg = pkv.make_config(n_layers=2, n_kv_heads=H, n_q_heads=H * 4, rank=24, sink_tokens=64,
+                                      recent_tokens=256, max_seqs=max_seqs, max_pages_per_seq=8, n_dense_slots=64,
+                                      n_factor_slots=64, n_ctas=n_ctas, decode_overlap=overlap)
+                sz = pkv.pkv_query_sizes(cfg)
+                assert sz.workspace_bytes > 0 and sz.meta_bytes > 0
+                if overlap == 2:
+                    assert sz.workspace_bytes <= (192 << 20) + 64 * 4160 * (max(512, n_ctas) + max_seqs * H)
+                handle = pkv.pkv_init_cache(cfg, None, None, None, None, None, None)      # dry run: host logic only
+                pkv.pkv_destroy_cache(handle)
