@@ -568,12 +568,13 @@ pkv_status pkv_append_kv(pkv_cache *c, int32_t layer, int32_t n_seqs, const int3
     }
     if (c->dry) return PKV_OK;
     AppendDesc *ddesc = (AppendDesc *)(c->meta + c->ml.append_desc);
-    if ((r = upload(c, ddesc, desc.data(), sizeof(AppendDesc) * desc.size(), st)) != PKV_OK) return r;
+    const bool inl = (int)desc.size() <= kAppendInline;       // small batch: descriptors ride in the kernel parameters
+    if (!inl && (r = upload(c, ddesc, desc.data(), sizeof(AppendDesc) * desc.size(), st)) != PKV_OK) return r;
     if ((r = stager_flush(c, st)) != PKV_OK) return r;
     c->cache_written = true;
     PKV_CUDA(c, launch_append(c->geo, c->dense_pool, (const int *)(c->meta + c->ml.page_table),
-                              (int *)(c->meta + c->ml.n_tokens), ddesc, (int)desc.size(), n_tok, layer, k, v,
-                              (int *)(c->meta + c->ml.status), st));
+                              (int *)(c->meta + c->ml.n_tokens), ddesc, inl ? desc.data() : nullptr, (int)desc.size(),
+                              n_tok, layer, k, v, (int *)(c->meta + c->ml.status), st));
     return PKV_OK;
 }
 

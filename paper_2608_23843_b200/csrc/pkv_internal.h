@@ -83,6 +83,7 @@ struct WorkspaceLayout {
 };
 
 struct AppendDesc { int seq, t_start, tok_begin, n_new; };
+constexpr int kAppendInline = 64;      // descriptors of up to this many sequences are passed as kernel parameters
 
 struct DecodeArgs {
     Geometry geo;
@@ -106,9 +107,11 @@ struct DecodeArgs {
 };
 
 // Launchers (defined in the .cu files); all return the launch error.
+// desc: device copy of the descriptors; host_desc: if not NULL (and n_seqs <= kAppendInline) the descriptors travel in
+// the kernel's parameters instead and `desc` is not read
 cudaError_t launch_append(const Geometry &geo, unsigned char *dense_pool, const int *page_table,
-                          int *n_tokens, const AppendDesc *desc, int n_seqs, long long n_tok, int layer,
-                          const void *k, const void *v, int *status, cudaStream_t st);
+                          int *n_tokens, const AppendDesc *desc, const AppendDesc *host_desc, int n_seqs,
+                          long long n_tok, int layer, const void *k, const void *v, int *status, cudaStream_t st);
 cudaError_t launch_compress(const Geometry &geo, const unsigned char *dense_pool, unsigned char *factor_pool,
                             const int2 *worklist, int n_entries, int *status, cudaStream_t st);
 cudaError_t launch_decode(const DecodeArgs &a, int n_segs, cudaStream_t st);

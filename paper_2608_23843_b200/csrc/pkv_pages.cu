@@ -8,9 +8,14 @@ namespace {
 
 // One thread moves one 16-byte chunk of one (token, KV head, K|V) row into the
 // swizzled dense page.  Block 0 also publishes the new token counts.
+// The descriptors come either from device memory (`desc_mem`) or, for small batches, inside the kernel's own
+// parameters (`inl`), which saves the host-to-device copy that would otherwise precede every decode step's append.
+struct AppendInline { AppendDesc d[kAppendInline]; };
+
 __global__ void append_kernel(Geometry geo, unsigned char *dense_pool, const int *page_table, int *n_tokens,
-                              const AppendDesc *desc, int n_seqs, long long n_tok, int layer,
-                              const uint4 *k, const uint4 *v, int *status) {
+                              const AppendDesc *desc_mem, const __grid_constant__ AppendInline inl, int n_seqs,
+                              long long n_tok, int layer, const uint4 *k, const uint4 *v, int *status) {
+    const AppendDesc *desc = desc_mem ? desc_mem : inl.d;
     const int H = geo.n_kv_heads;
     const long long total = n_tok * H * 2 * 16;
     for (long long idx = blockIdx.x * (long long)blockDim.x + threadIdx.x; idx < total;
@@ -91,15 +96,20 @@ __global__ void dense_read_kernel(int P, const unsigned char *head_base, unsigne
 }  // namespace
 
 cudaError_t launch_append(const Geometry &geo, unsigned char *dense_pool, const int *page_table,
-                          int *n_tokens, const AppendDesc *desc, int n_seqs, long long n_tok, int layer,
-                          const void *k, const void *v, int *status, cudaStream_t st) {
+                          int *n_tokens, const AppendDesc *desc, const AppendDesc *host_desc, int n_seqs,
+                          long long n_tok, int layer, const void *k, const void *v, int *status, cudaStream_t st) {
     const long long total = n_tok * geo.n_kv_heads * 2 * 16;
     const int threads = 256;
     long long blocks = (total + threads - 1) / threads;
     if (blocks > 148LL * 16) blocks = 148LL * 16;
     if (blocks < 1) blocks = 1;
-    append_kernel<<<(unsigned)blocks, threads, 0, st>>>(geo, dense_pool, page_table, n_tokens, desc, n_seqs, n_tok,
-                                                        layer, (const uint4 *)k, (const uint4 *)v, status);
+    AppendInline inl = {};
+    if (host_desc) {
+        for (int i = 0; i < n_seqs; ++i) inl.d[i] = host_desc[i];
+    }
+    append_kernel<<<(unsigned)blocks, threads, 0, st>>>(geo, dense_pool, page_table, n_tokens, host_desc ? nullptr : desc,
+                                                        inl, n_seqs, n_tok, layer, (const uint4 *)k, (const uint4 *)v,
+                                                        status);
     return cudaGetLastError();
 }
 
