@@ -199,6 +199,15 @@ pkv_status pkv_compress_eligible_pages(pkv_cache *c, int32_t layer, int64_t *n_p
  *   out_f32 [device, may be NULL] the same result before rounding, fp32
  * Scores use softmax_scale; accumulation is fp32.  The result does not depend
  * on physical slot placement and is bit-identical from run to run.
+ *
+ * CUDA graphs: with decode_overlap 0 or 1 the call may be recorded into a graph, provided this layer's plan for
+ * this batch is current, i.e. the same call has been made once outside the capture since the last change of the
+ * batch's page tables (otherwise PKV_ERR_UNSUPPORTED: the plan cannot be uploaded from inside a capture).  A
+ * replay reads token counts, page tables and the plan from device memory when it runs: appends that stay inside a
+ * sequence's current page need nothing; after an append that opens a page, a compression or a free, one such call
+ * outside a capture brings the plan up to date and existing graphs for the same batch are valid again.
+ * pkv_append_kv and pkv_compress_eligible_pages update host-side state and cannot be captured (PKV_ERR_UNSUPPORTED
+ * while the stream is capturing).
  */
 pkv_status pkv_decode_attention(pkv_cache *c, int32_t layer, int32_t n_seqs, const int32_t *seq_ids,
                                 const void *q, void *out, float *out_f32, void *stream);

@@ -521,6 +521,12 @@ pkv_status pkv_destroy_cache(pkv_cache *c) {
 
 const char *pkv_last_error(const pkv_cache *c) { return c ? c->err.c_str() : "cache is NULL"; }
 
+// Calls that change host-side state or copy from the staging ring cannot be recorded into a CUDA graph.
+static bool is_capturing(cudaStream_t st) {
+    cudaStreamCaptureStatus cap = cudaStreamCaptureStatusNone;
+    return cudaStreamIsCapturing(st, &cap) == cudaSuccess && cap != cudaStreamCaptureStatusNone;
+}
+
 pkv_status pkv_append_kv(pkv_cache *c, int32_t layer, int32_t n_seqs, const int32_t *seq_ids,
                          const int32_t *n_new, const void *k, const void *v, void *stream) {
     if (!c) return PKV_ERR_INVALID_ARG;
@@ -544,6 +550,8 @@ pkv_status pkv_append_kv(pkv_cache *c, int32_t layer, int32_t n_seqs, const int3
                     (long long)c->dense_free.available());
     if (!c->dry && n_tok > 0 && (!k || !v)) return fail(c, PKV_ERR_INVALID_ARG, "k or v is NULL");
     if (n_tok == 0) return PKV_OK;
+    if (!c->dry && is_capturing(st))
+        return fail(c, PKV_ERR_UNSUPPORTED, "pkv_append_kv cannot be captured into a CUDA graph");
 
     std::vector<AppendDesc> desc;
     desc.reserve(n_seqs);
@@ -584,6 +592,8 @@ pkv_status pkv_compress_eligible_pages(pkv_cache *c, int32_t layer, int64_t *n_p
     cudaStream_t st = (cudaStream_t)stream;
     if (n_pages_compressed) *n_pages_compressed = 0;
     if (layer < -1 || layer >= c->cfg.n_layers) return fail(c, PKV_ERR_INVALID_ARG, "layer %d out of range", layer);
+    if (!c->dry && is_capturing(st))
+        return fail(c, PKV_ERR_UNSUPPORTED, "pkv_compress_eligible_pages cannot be captured into a CUDA graph");
     const Geometry &g = c->geo;
     const int l0 = layer < 0 ? 0 : layer, l1 = layer < 0 ? c->cfg.n_layers : layer + 1;
     std::vector<int2> work;
@@ -664,6 +674,10 @@ pkv_status pkv_decode_attention(pkv_cache *c, int32_t layer, int32_t n_seqs, con
             return fail(c, PKV_ERR_INVALID_ARG, "sequence %d has no tokens in layer %d", seq_ids[i], layer);
     if (!c->dry && (!q || !out)) return fail(c, PKV_ERR_INVALID_ARG, "q or out is NULL");
     if (!plan_is_current(c, layer, n_seqs, seq_ids)) {
+        // the plan is uploaded through the staging ring: a copy recorded into a graph would replay stale bytes
+        if (!c->dry && is_capturing(st))
+            return fail(c, PKV_ERR_UNSUPPORTED, "the decode plan of layer %d must be rebuilt: call pkv_decode_attention "
+                        "once outside the stream capture for this layer and batch first", layer);
         if ((r = build_plan(c, layer, n_seqs, seq_ids, st)) != PKV_OK) return r;
     }
     const PlanCache &pc = c->plans[layer];

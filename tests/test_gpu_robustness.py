@@ -115,3 +115,108 @@ def test_two_caches_and_a_side_stream():
         pair.load_gpu_factors_into_oracle(0, 0)
         ref = pair.orc.decode_attention(0, [0], f64(qq))
         assert rel_err(got, ref) <= 1e-2
+
+
+@pytest.mark.gpu
+@pytest.mark.parametrize("overlap", [0, 1])
+def test_cuda_graph_replay_sees_appends_and_rebuilt_plans(overlap):
+    """Decode launches recorded into a CUDA graph read token counts, page tables and the plan when they run:
+    a replay after an in-page append equals a fresh eager call; after an append that opens a page plus a
+    compression, one eager call rebuilds the plan and the old graph is valid again.  Calls that cannot be
+    recorded (append, compress, a decode whose plan is stale, mode 2) return PKV_ERR_UNSUPPORTED during capture
+    and leave the capture usable."""
+    L, H, G = 2, 2, 4
+    cfg = pkv.make_config(n_layers=L, n_kv_heads=H, n_q_heads=H * G, rank=16, sink_tokens=64, recent_tokens=128,
+                          max_seqs=2, max_pages_per_seq=40, n_dense_slots=160, n_factor_slots=160,
+                          decode_overlap=overlap)
+    cache = pkv.Cache(cfg, "cuda", None, None)
+    lengths = [700, 1500]
+    data = [[synth.make_kv(21, ly, s, 2200, H, 128, 64, "cuda") for s in range(2)] for ly in range(L)]
+    T = list(lengths)
+    for ly in range(L):
+        for s in range(2):
+            cache.append_kv(ly, [s], [T[s]], data[ly][s][0][:T[s]], data[ly][s][1][:T[s]])
+    cache.compress_eligible_pages(-1)
+    ids = [1, 0]
+    qs = [synth.make_q(21, ly, 0, 2, H * G, 128, "cuda") for ly in range(L)]
+    outs = [torch.empty_like(q) for q in qs]
+
+    def eager():
+        res = [torch.empty_like(q) for q in qs]
+        for ly in range(L):
+            cache.decode_attention(ly, ids, qs[ly], res[ly])
+        torch.cuda.synchronize()
+        return [r.clone() for r in res]
+
+    def grow(n):
+        for ly in range(L):
+            cache.append_kv(ly, [0, 1], [n, n], torch.cat([data[ly][0][0][T[0]:T[0] + n], data[ly][1][0][T[1]:T[1] + n]]),
+                            torch.cat([data[ly][0][1][T[0]:T[0] + n], data[ly][1][1][T[1]:T[1] + n]]))
+        T[0] += n
+        T[1] += n
+
+    ref = eager()                                           # also builds the plans outside any capture
+    side = torch.cuda.Stream()
+    side.wait_stream(torch.cuda.current_stream())
+    graph = torch.cuda.CUDAGraph()
+    with torch.cuda.stream(side):
+        with torch.cuda.graph(graph, stream=side):
+            # not recordable: must refuse without breaking the capture
+            with pytest.raises(pkv.PkvError) as e1:
+                cache.append_kv(0, [0], [1], data[0][0][0][:1], data[0][0][1][:1])
+            assert e1.value.status == pkv.PKV_ERR_UNSUPPORTED
+            with pytest.raises(pkv.PkvError) as e2:
+                cache.compress_eligible_pages(-1)
+            assert e2.value.status == pkv.PKV_ERR_UNSUPPORTED
+            with pytest.raises(pkv.PkvError) as e3:
+                cache.decode_attention(0, [0, 1], qs[0], outs[0])          # another batch order: no current plan
+            assert e3.value.status == pkv.PKV_ERR_UNSUPPORTED
+            for ly in range(L):
+                cache.decode_attention(ly, ids, qs[ly], outs[ly])
+    torch.cuda.current_stream().wait_stream(side)
+    graph.replay()
+    torch.cuda.synchronize()
+    for ly in range(L):
+        assert torch.equal(outs[ly], ref[ly])
+    # three tokens more, same pages (700 -> 703 and 1500 -> 1503 stay inside pages 10 and 23)
+    grow(3)
+    graph.replay()
+    torch.cuda.synchronize()
+    got = [o.clone() for o in outs]
+    ref = eager()
+    for ly in range(L):
+        assert torch.equal(got[ly], ref[ly])
+    # new pages and newly compressed pages: one eager call per layer rebuilds the plan, then the graph is valid again
+    grow(130)
+    cache.compress_eligible_pages(-1)
+    ref = eager()
+    graph.replay()
+    torch.cuda.synchronize()
+    for ly in range(L):
+        assert torch.equal(outs[ly], ref[ly])
+    assert cache.stats()["device_timeouts"] == 0
+    cache.close()
+
+
+@pytest.mark.gpu
+def test_mode_2_refuses_stream_capture():
+    cfg = pkv.make_config(n_layers=1, n_kv_heads=1, n_q_heads=4, rank=16, sink_tokens=64, recent_tokens=128,
+                          max_seqs=1, max_pages_per_seq=8, n_dense_slots=8, n_factor_slots=8, decode_overlap=2)
+    cache = pkv.Cache(cfg, "cuda", None, None)
+    k, v = synth.make_kv(22, 0, 0, 300, 1, 128, 64, "cuda")
+    cache.append_kv(0, [0], [300], k, v)
+    q = synth.make_q(22, 0, 0, 1, 4, 128, "cuda")
+    out = torch.empty_like(q)
+    cache.decode_attention(0, [0], q, out)
+    torch.cuda.synchronize()
+    side = torch.cuda.Stream()
+    side.wait_stream(torch.cuda.current_stream())
+    graph = torch.cuda.CUDAGraph()
+    with torch.cuda.stream(side):
+        with torch.cuda.graph(graph, stream=side):
+            with pytest.raises(pkv.PkvError) as e:
+                cache.decode_attention(0, [0], q, out)
+            assert e.value.status == pkv.PKV_ERR_UNSUPPORTED
+            torch.zeros(4, device="cuda")                    # the capture itself is still alive
+    torch.cuda.current_stream().wait_stream(side)
+    cache.close()
