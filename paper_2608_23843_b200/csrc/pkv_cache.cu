@@ -199,6 +199,7 @@ void derive(const pkv_config &cfg, int n_ctas, Geometry &g, MetaLayout &ml, Work
     long long p = sizeof(PlanHeader);
     ml.plan_cta = p;   p = align_up(p + (long long)sizeof(PlanCta) * (n_ctas + 1), 16);
     ml.plan_entry = p; p = align_up(p + (long long)sizeof(PlanEntry) * cfg.max_seqs, 16);
+    ml.plan_cta_entry = p; p = align_up(p + (long long)sizeof(PlanEntry) * (n_ctas + 1), 16);
     ml.plan_seg = p;   p = align_up(p + (long long)sizeof(PlanSeg) * cfg.max_seqs * cfg.n_kv_heads, 256);
     ml.plan_stride = p;
     ml.plans = off;      off = align_up(off + p * cfg.n_layers, 256);
@@ -404,6 +405,11 @@ pkv_status build_plan(pkv_cache *c, int layer, int n_seqs, const int32_t *seq_id
     pkv_status r;
     if ((r = upload(c, plan, &hdr, sizeof hdr, st)) != PKV_OK) return r;
     if ((r = upload(c, plan + c->ml.plan_cta, ctas.data(), sizeof(PlanCta) * ctas.size(), st)) != PKV_OK) return r;
+    {
+        std::vector<PlanEntry> first(n_used);
+        for (int j = 0; j < n_used; ++j) first[j] = entries[ctas[j].entry];
+        if (n_used > 0 && (r = upload(c, plan + c->ml.plan_cta_entry, first.data(), sizeof(PlanEntry) * n_used, st)) != PKV_OK) return r;
+    }
     if ((r = upload(c, plan + c->ml.plan_entry, entries.data(), sizeof(PlanEntry) * n_seqs, st)) != PKV_OK) return r;
     if ((r = upload(c, plan + c->ml.plan_seg, segs.data(), sizeof(PlanSeg) * n_segs, st)) != PKV_OK) return r;
     return stager_flush(c, st);
@@ -701,6 +707,7 @@ pkv_status pkv_decode_attention(pkv_cache *c, int32_t layer, int32_t n_seqs, con
     a.n_tokens = (const int *)(c->meta + c->ml.n_tokens);
     a.plan = c->meta + c->ml.plans + c->ml.plan_stride * layer;
     a.plan_cta = c->ml.plan_cta; a.plan_entry = c->ml.plan_entry; a.plan_seg = c->ml.plan_seg;
+    a.plan_cta_entry = c->ml.plan_cta_entry;
     a.q = q; a.out = out; a.out_f32 = out_f32;
     // decode_overlap = 2: launches never wait for one another, so launches in flight must not share split-K
     // scratch.  The scratch rotates over wl.n_sets sets and every (n_sets-1)-th launch is a plain
@@ -754,6 +761,7 @@ pkv_status pkv_decode_attention_static_scratch(pkv_cache *c, int32_t layer, int3
     a.n_tokens = (const int *)(c->meta + c->ml.n_tokens);
     a.plan = c->meta + c->ml.plans + c->ml.plan_stride * layer;
     a.plan_cta = c->ml.plan_cta; a.plan_entry = c->ml.plan_entry; a.plan_seg = c->ml.plan_seg;
+    a.plan_cta_entry = c->ml.plan_cta_entry;
     a.q = q; a.out = out; a.out_f32 = out_f32;
     a.partials = nullptr; a.tickets = nullptr;            // set by the launcher from the static scratch
     a.plain_launch = 0;                                   // the launcher's memset already orders it after earlier work

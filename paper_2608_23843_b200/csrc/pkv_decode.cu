@@ -38,6 +38,7 @@ constexpr int kKindDense = 0, kKindFactor = 1, kKindEnd = 2;
 
 struct Range {
     PlanCta start, end;
+    PlanEntry first_entry;             // the entry `start` lies in
     int n_used, seg_first, n_local_segs;
 };
 
@@ -68,6 +69,7 @@ __device__ __forceinline__ bool load_range(const DecodeArgs &a, Range &r) {
     const PlanCta *ctas = reinterpret_cast<const PlanCta *>(a.plan + a.plan_cta);
     r.start = ctas[blockIdx.x];
     r.end = ctas[blockIdx.x + 1];
+    r.first_entry = reinterpret_cast<const PlanEntry *>(a.plan + a.plan_cta_entry)[blockIdx.x];
     const int H = a.geo.n_kv_heads;
     r.seg_first = r.start.entry * H + r.start.head;
     int seg_last = r.end.entry * H + r.end.head;
@@ -897,7 +899,7 @@ __global__ void __launch_bounds__(kDecodeThreads, 2) decode_tc_kernel(const __gr
         bool ok = true;
         PlanCta cur = rg.start;
         while (ok && !(cur.entry == rg.end.entry && cur.head == rg.end.head && cur.unit == rg.end.unit)) {
-            const PlanEntry e = entries[cur.entry];
+            const PlanEntry e = cur.entry == rg.start.entry ? rg.first_entry : entries[cur.entry];
             const HeadUnits hu = head_units(geo, e);
             const bool last_run = cur.entry == rg.end.entry && cur.head == rg.end.head;
             const int u_end = last_run ? rg.end.unit : hu.units;

@@ -64,6 +64,7 @@ struct MetaLayout {                    // byte offsets inside the caller's `meta
     long long plans;                   // n_layers * plan_stride
     long long plan_stride;
     long long plan_cta, plan_entry, plan_seg;   // offsets inside one plan
+    long long plan_cta_entry;          // PlanEntry [n_ctas]: a copy of the entry each CTA's range starts in (saves a dependent load)
     long long append_desc;             // int4 [max_seqs]
     long long status;                  // int32 [kStatusWords]
     long long total;
@@ -91,7 +92,7 @@ struct DecodeArgs {
     const int *page_table;             // whole table
     const int *n_tokens;               // whole array
     const unsigned char *plan;         // this layer's plan
-    long long plan_cta, plan_entry, plan_seg;
+    long long plan_cta, plan_entry, plan_seg, plan_cta_entry;
     const void *q;
     void *out;
     float *out_f32;
