@@ -1010,11 +1010,15 @@ __global__ void __launch_bounds__(kDecodeThreads, 2) decode_tc_kernel(const __gr
             StageDesc dsc = ok ? descs[s] : StageDesc{kKindEnd, 0, rg.n_local_segs, 0};
             if (trace && k == 0 && lane == 0) trace[4] = clock64();
             if (trace && dsc.kind == kKindEnd && warp == 0 && lane == 0) { trace[5] = clock64(); trace[7] = k; }
-            while (cur_seg < dsc.seg) {
-                flush_segment(a, comb, last_flag, st, rg.seg_first + cur_seg, warp, lane, tid, W);
-                ++cur_seg;
-                reset_state(st);
-                if (cur_seg < rg.n_local_segs) load_q(a, rg.seg_first + cur_seg, qf, lane);
+            if (cur_seg < dsc.seg) {
+                // the old segment's queries are no longer needed: fetch the new ones now, so that their latency
+                // hides behind the flush
+                if (dsc.seg < rg.n_local_segs) load_q(a, rg.seg_first + dsc.seg, qf, lane);
+                while (cur_seg < dsc.seg) {
+                    flush_segment(a, comb, last_flag, st, rg.seg_first + cur_seg, warp, lane, tid, W);
+                    ++cur_seg;
+                    reset_state(st);
+                }
             }
             if (dsc.kind == kKindEnd) break;
             dsc.rows = min(dsc.rows, dsc.kind == kKindFactor ? P : kDB);
