@@ -54,7 +54,7 @@ typedef int32_t pkv_status;
 #define PKV_ERR_BAD_SEQ         (-3)  /* sequence id outside [0, max_seqs) or repeated within one call */
 #define PKV_ERR_CUDA            (-4)  /* a CUDA runtime call failed; message holds cudaGetErrorString */
 #define PKV_ERR_NOT_CONVERGED   (-5)  /* reported by pkv_get_stats users: some page hit the Jacobi sweep cap (factors still written) */
-#define PKV_ERR_UNSUPPORTED     (-6)  /* shape outside the supported set */
+#define PKV_ERR_UNSUPPORTED     (-6)  /* shape outside the supported set; or a call that cannot be recorded while its stream is capturing a CUDA graph */
 #define PKV_ERR_DEVICE_TIMEOUT  (-7)  /* a bounded in-kernel wait gave up (seen via pkv_get_stats); results of that call are invalid */
 
 #define PKV_KIND_DENSE  0
@@ -79,12 +79,14 @@ typedef struct pkv_config {
     int32_t n_ctas;             /* decode grid size; 0 => SM count of the current device (148 in dry-run), doubled unless decode_overlap */
     int32_t decode_variant;     /* 0 = tensor-core pipeline kernel (the product path); 1 = scalar fp32 kernel that
                                    evaluates the same equations one unit at a time, kept as a debugging reference */
-    float   jacobi_energy_tol;  /* the sweeps also stop once a sweep raises the energy captured by the r largest
-                                   diagonal entries (= ||A^T X||_F^2 of the factors it would give) by less than this
-                                   fraction of the energy left outside them (= the squared reconstruction error):
-                                   the remaining rotations only polish eigenvectors inside near-degenerate clusters
-                                   and cannot improve A B measurably.  0 => default 1e-4; negative => off (iterate
-                                   until no rotation exceeds jacobi_tol) */
+    float   jacobi_energy_tol;  /* the sweeps also stop once the energy captured by the r largest diagonal entries
+                                   (= ||A^T X||_F^2 of the factors they would give) has grown, since the previous
+                                   check, by less than this fraction of the energy left outside them (= the squared
+                                   reconstruction error): the remaining rotations only polish eigenvectors inside
+                                   near-degenerate clusters and cannot improve A B measurably.  Checked about three
+                                   times per sweep for page sizes 32 and 64, once per sweep for 16; not applied at
+                                   full rank (r = P), where it would say nothing.  0 => default 1e-4; negative => off
+                                   (iterate until no rotation exceeds jacobi_tol) */
     int32_t factor_bits;        /* 0 or 16: factors stored in bf16.  4: INT4 factors (Section 4.3): the singular
                                    values are split evenly, A~ = A Sigma^(1/2), B~ = Sigma^(-1/2) B, and each matrix is
                                    quantized symmetrically to 4 bits with one bf16 scale per column of A~_K, B~_K and
@@ -118,8 +120,10 @@ typedef struct pkv_config {
 typedef struct pkv_sizes {
     int64_t dense_slot_bytes;   /* H_kv * 2 * P * d * 2 */
     int64_t factor_slot_bytes;  /* bf16 factors: H_kv * 2 * (r_k + r_v) * (P + d) bytes, so that Eq. 3 is
-                                   factor_slot_bytes / dense_slot_bytes; INT4 factors: H_kv * ((r_k + r_v)(P + d)/2
-                                   + 2 * (ceil8(r_k) + 2d + P)) bytes rounded up to 16 per KV head */
+                                   factor_slot_bytes / dense_slot_bytes; INT4 factors, with R_k, R_v = the ranks
+                                   rounded up to multiples of 8 (zero codes fill the rest):
+                                   H_kv * ((R_k + R_v)(P + d)/2 + 2 * (R_k + 2d + P)) bytes, each KV head's part
+                                   rounded up to 16 */
     int64_t dense_pool_bytes;   /* n_dense_slots * dense_slot_bytes */
     int64_t factor_pool_bytes;
     int64_t meta_bytes;         /* device page tables, token counts, decode plans, status words */
