@@ -64,43 +64,109 @@ def _peaks():
 
 
 class ClockSampler:
-    """Samples SM clocks and throttle reasons with nvidia-smi while the timed region runs."""
+    """Samples SM clocks and throttle reasons (read-only NVML queries from a thread; nvidia-smi if NVML cannot be
+    loaded) while the timed region runs.  The sampler is started ahead of time, every sample is stamped, and the
+    summary uses the samples that fell between begin() and end(): the timed region of a short workload lasts only
+    tens of milliseconds."""
 
     FIELDS = ("clocks.sm,clocks.max.sm,clocks_event_reasons.hw_slowdown,clocks_event_reasons.hw_thermal_slowdown,"
               "clocks_event_reasons.sw_thermal_slowdown,clocks_event_reasons.sw_power_cap")
+    NAMES = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
 
     def __init__(self, index):
-        self.index, self.rows, self.proc = index, [], None
+        self.index, self.rows, self.proc, self.nvml = index, [], None, None
+        self.t_begin = self.t_end = None
+        self.stop_flag = False
+        self.sm_max = None
+
+    def _nvml_handle(self):
+        import pynvml
+        pynvml.nvmlInit()
+        try:
+            import torch
+            uuid = str(torch.cuda.get_device_properties(self.index).uuid)
+            return pynvml, pynvml.nvmlDeviceGetHandleByUUID(("GPU-" + uuid).encode())
+        except Exception:
+            return pynvml, pynvml.nvmlDeviceGetHandleByIndex(self.index)
 
     def start(self):
         try:
+            self.nvml, self.handle = self._nvml_handle()
+            self.sm_max = float(self.nvml.nvmlDeviceGetMaxClockInfo(self.handle, self.nvml.NVML_CLOCK_SM))
+            self.thread = threading.Thread(target=self._poll, daemon=True)
+            self.thread.start()
+            return
+        except Exception:
+            self.nvml = None
+        try:
             self.proc = subprocess.Popen(["nvidia-smi", "-i", str(self.index), "--query-gpu=" + self.FIELDS,
-                                          "--format=csv,noheader,nounits", "-lms", "20"],
+                                          "--format=csv,noheader,nounits", "-lms", "10"],
                                          stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
             self.thread = threading.Thread(target=self._read, daemon=True)
             self.thread.start()
         except OSError:
             self.proc = None
 
+    def _poll(self):
+        n = self.nvml
+        masks = [n.nvmlClocksEventReasonHwSlowdown, n.nvmlClocksEventReasonHwThermalSlowdown,
+                 n.nvmlClocksEventReasonSwThermalSlowdown, n.nvmlClocksEventReasonSwPowerCap]
+        while not self.stop_flag:
+            try:
+                sm = float(n.nvmlDeviceGetClockInfo(self.handle, n.NVML_CLOCK_SM))
+                why = n.nvmlDeviceGetCurrentClocksEventReasons(self.handle)
+                self.rows.append((time.perf_counter(), sm, [bool(why & m) for m in masks]))
+            except Exception:
+                pass
+            time.sleep(0.002)
+
     def _read(self):
         for line in self.proc.stdout:
-            self.rows.append([x.strip() for x in line.split(",")])
+            r = [x.strip() for x in line.split(",")]
+            if len(r) >= 6 and r[0].replace(".", "").isdigit():
+                if r[1].replace(".", "").isdigit():
+                    self.sm_max = float(r[1])
+                self.rows.append((time.perf_counter(), float(r[0]), [r[2 + i].startswith("Active") for i in range(4)]))
+
+    def begin(self):
+        """Call right before the timed region (waits, briefly, until the sampler is alive)."""
+        if self.nvml is not None or self.proc is not None:
+            t0 = time.perf_counter()
+            while not self.rows and time.perf_counter() - t0 < 2.0:
+                time.sleep(0.002)
+        self.t_begin = time.perf_counter()
+
+    def end(self):
+        self.t_end = time.perf_counter()
 
     def stop(self):
-        if self.proc is None:
-            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["nvidia-smi unavailable"]}
-        time.sleep(0.15)
-        self.proc.terminate()
-        try:
-            self.proc.wait(timeout=5)
-        except subprocess.TimeoutExpired:
-            self.proc.kill()
-        sm = [float(r[0]) for r in self.rows if len(r) >= 6 and r[0].replace(".", "").isdigit()]
-        mx = [float(r[1]) for r in self.rows if len(r) >= 6 and r[1].replace(".", "").isdigit()]
-        names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
-        reasons = sorted({names[i] for r in self.rows if len(r) >= 6 for i in range(4) if r[2 + i].startswith("Active")})
-        return {"sm_mhz": statistics.median(sm) if sm else None, "sm_max_mhz": max(mx) if mx else None,
-                "reasons": reasons, "samples": len(sm)}
+        if self.nvml is None and self.proc is None:
+            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["no clock source (NVML, nvidia-smi) available"], "samples": 0}
+        if self.t_end is None:
+            self.end()
+        time.sleep(0.02)
+        self.stop_flag = True
+        if self.proc is not None:
+            self.proc.terminate()
+            try:
+                self.proc.wait(timeout=5)
+            except subprocess.TimeoutExpired:
+                self.proc.kill()
+        t0 = self.t_begin if self.t_begin is not None else 0.0
+        rows = list(self.rows)
+        inside = [r for r in rows if t0 <= r[0] <= self.t_end + 0.005]
+        note = None
+        if not inside and rows:
+            mid = 0.5 * (t0 + self.t_end)
+            inside = sorted(rows, key=lambda r: abs(r[0] - mid))[:3]
+            note = "no sample fell inside the timed region: the three nearest"
+        sm = [r[1] for r in inside]
+        reasons = sorted({self.NAMES[i] for r in inside for i in range(4) if r[2][i]})
+        out = {"sm_mhz": statistics.median(sm) if sm else None, "sm_max_mhz": self.sm_max, "reasons": reasons,
+               "samples": len(sm), "source": "nvml" if self.nvml is not None else "nvidia-smi"}
+        if note:
+            out["note"] = note
+        return out
 
 
 def build_workload(w, rank, device, overlap=2, n_ctas=0, factor_bits=16, grow=0, keep_kv=False):
@@ -191,19 +257,21 @@ def run_serving(args, w, rank, device, world, rk, local):
             dist.barrier()
         torch.cuda.synchronize()
 
+    sampler = ClockSampler(local)
+    sampler.start()                                       # ahead of the warm-up: nvidia-smi takes a while to start
     for _ in range(warm):
         step(False)
     cache.decode_attention(0, ids, qs[0], out)
     bytes_per_step = cache.stats()["last_decode_bytes"]
-    sampler = ClockSampler(local)
-    sampler.start()
     barrier()
+    sampler.begin()
     e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
     e0.record()
     for _ in range(args.steps):
         step(True)
     e1.record()
     barrier()
+    sampler.end()
     clocks = sampler.stop()
     ms = e0.elapsed_time(e1) / args.steps
     app = [ev[0].elapsed_time(ev[1]) * 1e3 for ev, _ in events]
@@ -419,6 +487,8 @@ def main():
             dist.barrier()
         torch.cuda.synchronize()
 
+    sampler = ClockSampler(local)
+    sampler.start()                                       # ahead of the warm-up: nvidia-smi takes a while to start
     for _ in range(max(3, args.warmup)):
         step()
     torch.cuda.synchronize()
@@ -444,15 +514,15 @@ def main():
     for layer in range(lps):                              # algorithmic bytes, from the library's own accounting
         cache.decode_attention(layer, ids, qs[layer], outs[layer])
         bytes_per_step += cache.stats()["last_decode_bytes"]
-    sampler = ClockSampler(local)
-    sampler.start()
     barrier()
+    sampler.begin()
     e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
     e0.record()
     for _ in range(args.steps):
         step()
     e1.record()
     barrier()
+    sampler.end()
     clocks = sampler.stop()
     ms = e0.elapsed_time(e1) / args.steps
     # average duration of one decode-kernel launch over the timed region: the region holds nothing but
