@@ -102,9 +102,23 @@ def lib():
     return _lib
 
 
+_INT_ARRAYS = {}
+
+
 def _ints(xs):
-    xs = [int(x) for x in xs]
-    return (ctypes.c_int32 * len(xs))(*xs), len(xs)
+    """A ctypes int32 array for a sequence of ints (decode calls pass the same id list every step: remembered)."""
+    if len(xs) > 4096:                                   # e.g. slot orders: built once, not worth remembering
+        vals = [int(x) for x in xs]
+        return (ctypes.c_int32 * len(vals))(*vals), len(vals)
+    key = tuple(xs)
+    hit = _INT_ARRAYS.get(key)
+    if hit is None:
+        vals = [int(x) for x in key]
+        hit = ((ctypes.c_int32 * len(vals))(*vals), len(vals))
+        if len(_INT_ARRAYS) >= 256:
+            _INT_ARRAYS.clear()
+        _INT_ARRAYS[key] = hit
+    return hit
 
 
 def _ptr(t):
