@@ -53,6 +53,8 @@ SEED = 0
 # profiles/decode_tc_kernel_r24_llama3_8b_32k_b8.md: (608.92 MB read + 4.52 MB written) / 608.70 MB.  Every
 # unit is fetched once, so traffic scales with the units a launch processes.
 NCU_TRAFFIC_PER_ALGORITHMIC_BYTE = (608.9216e6 + 4.52096e6) / 608698368.0
+# the same for INT4 factors (profiles/decode_tc_kernel_int4_r24_llama3_8b_32k_b8.md): (183.74 MB + 3.96 MB) / 182.46 MB
+NCU_TRAFFIC_PER_ALGORITHMIC_BYTE_INT4 = (183.737856e6 + 3.961344e6) / 182461440.0
 
 
 def _peaks():
@@ -334,7 +336,7 @@ def run_serving(args, w, rank, device, world, rk, local):
             "pages_factorized_per_s": comp["pages_per_s"], "page_svds_timed": comp["n_page_svds"],
             "roofline": {"bound": "hbm", "kernel": "decode_tc_kernel<P=%d, rank tiles=%d>" % (P, (rank + 7) // 8),
                          "achieved": achieved, "peak": peak, "unit": "GB/s", "frac": achieved / peak,
-                         "peak_source": peak_src, "traffic": bytes_per_step * NCU_TRAFFIC_PER_ALGORITHMIC_BYTE,
+                         "peak_source": peak_src, "traffic": bytes_per_step * (NCU_TRAFFIC_PER_ALGORITHMIC_BYTE_INT4 if args.factor_bits == 4 else NCU_TRAFFIC_PER_ALGORITHMIC_BYTE),
                          "traffic_source": "ncu dram__bytes_read+write of this kernel on the llama3_8b_32k_b8 launch, "
                                            "scaled by algorithmic bytes",
                          "launch_us": att_mean, "algorithmic_bytes_per_launch": bytes_per_step},
@@ -574,7 +576,7 @@ def main():
             "roofline": {"bound": "hbm", "kernel": "decode_tc_kernel<P=%d, rank tiles=%d>" % (w.get("page", 64), (rank + 7) // 8),
                          "achieved": achieved, "peak": peak, "unit": "GB/s", "frac": achieved / peak,
                          "peak_source": peak_src,
-                         "traffic": bytes_per_launch * NCU_TRAFFIC_PER_ALGORITHMIC_BYTE,
+                         "traffic": bytes_per_launch * (NCU_TRAFFIC_PER_ALGORITHMIC_BYTE_INT4 if args.factor_bits == 4 else NCU_TRAFFIC_PER_ALGORITHMIC_BYTE),
                          "traffic_source": "ncu dram__bytes_read+write of this kernel on the llama3_8b_32k_b8 launch, "
                                            "scaled by algorithmic bytes", "launch_us": launch_ms * 1e3,
                          "algorithmic_bytes_per_launch": bytes_per_launch},
