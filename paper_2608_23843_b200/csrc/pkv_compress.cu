@@ -34,8 +34,10 @@ template <int P> struct Quads {
     static constexpr int kClasses = P == 64 ? 21 : 13;
     static constexpr int kDiag = 32 / kQuads;                  // wrapped diagonals of quad blocks per warp: 2 or 4
     static constexpr int kVarStep = 4 / kDiag;                 // lane group g takes its quads' members in the order j ^ (g * kVarStep)
-    static constexpr int kItems = kQuads * (kQuads / 2) + kQuads / 2;   // quad blocks of G computed per class
-    static constexpr int kGWarps = (kItems + 31) / 32;         // 5 or 2; the remaining warps update Q^T
+    // off-diagonal quad blocks of G computed per class, one of every mirror-image couple (the diagonal blocks come
+    // out of the rotation phase)
+    static constexpr int kItems = kQuads * (kQuads / 2 - 1) + kQuads / 2;
+    static constexpr int kGWarps = (kItems + 31) / 32;         // 4 or 1; the remaining warps update Q^T
     static constexpr int kQIters = kQuads * (P / 4) / 32;      // 8 or 2
     static constexpr int kCheck = (kClasses + 2) / 3;          // the energy rule is evaluated about three times per sweep
 };
@@ -105,6 +107,24 @@ inline void pair_of(int P, int rho, int k, int &p, int &q) {
     if (k == 0) { a = m; b = rho; }
     else { a = rho + k; if (a >= m) a -= m; b = rho - k; if (b < 0) b += m; }
     p = a < b ? a : b; q = a < b ? b : a;
+}
+
+// Jacobi rotation (c, s) that zeroes g_pq: t = tan(angle) = 2 g_pq / (d + sign(d) sqrt(d^2 + 4 g_pq^2)), d = g_qq - g_pp
+// (the smaller root, |t| <= 1), c = 1 / sqrt(1 + t^2), s = t c.  Skipped (c = 1, s = 0, returns false) when
+// |g_pq| <= tol sqrt(|g_pp g_qq|) or |g_pq| <= floor_abs.  The reciprocal and the square roots are the hardware
+// approximations (2 ulp): they set the angle, not the orthogonality, which rests on c^2 + s^2 = c^2 (1 + t^2).
+__device__ __forceinline__ bool jacobi_rotation(float gpp, float gqq, float gpq, float tol, float floor_abs, float &c,
+                                                float &s) {
+    c = 1.f;
+    s = 0.f;
+    if (!(fabsf(gpq) > floor_abs && gpq * gpq > tol * tol * fabsf(gpp * gqq))) return false;
+    const float d = gqq - gpp;
+    const float h2 = fmaf(d, d, 4.f * gpq * gpq);
+    const float h = h2 * rsqrtf(h2);
+    const float t = __fdividef(2.f * gpq, d + copysignf(h, d));
+    c = rsqrtf(fmaf(t, t, 1.f));
+    s = t * c;
+    return true;
 }
 
 // Early-stopping rule: the energy captured by the r largest diagonal entries of G is ||A^T X||_F^2 of the factors
@@ -237,7 +257,7 @@ compress_kernel(Geometry geo, const unsigned char *dense_pool, unsigned char *fa
         // make a sweep in which every pair is rotated (see Quads).
         //   first P threads     four per quad: rotations and M                                   (between barriers)
         //   first kGWarps warps G: a thread owns the 4 x 4 block (quad a, quad b) of a mirror-image couple; a group
-        //                       of P/4 lanes walks a wrapped diagonal (b = a + delta mod P/4, delta = 0 .. P/8), reads
+        //                       of P/4 lanes walks a wrapped diagonal (b = a + delta mod P/4, delta = 1 .. P/8), reads
         //                       16 entries, writes 16 and their mirror images
         //   the other warps     Q^T: a thread owns (quad, four tokens): four 128-bit loads, 64 FMAs, four stores
         // Banks: an entry's bank is its column index mod 32.  Lane group g of a warp takes its quads' members in
@@ -273,14 +293,8 @@ compress_kernel(Geometry geo, const unsigned char *dense_pool, unsigned char *fa
                         // both lanes of a pair must arrive at the same rotation: take the pivot from the lower one
                         const float g_other = __shfl_xor_sync(0xffffffffu, e[x], x), gpq = low ? e[x] : g_other;
                         const float gpp = low ? d_mine : d_other, gqq = low ? d_other : d_mine;
-                        float c = 1.f, sn = 0.f;
-                        if (fabsf(gpq) > fmaxf(tol * sqrtf(fabsf(gpp * gqq)), floor_abs)) {
-                            const float theta = (gqq - gpp) / (2.f * gpq);
-                            const float tt = copysignf(1.f, theta) / (fabsf(theta) + sqrtf(1.f + theta * theta));
-                            c = rsqrtf(1.f + tt * tt);
-                            sn = tt * c;
-                            rotated = 1;
-                        }
+                        float c, sn;
+                        if (jacobi_rotation(gpp, gqq, gpq, tol, floor_abs, c, sn)) rotated = 1;
                         const float c2 = __shfl_xor_sync(0xffffffffu, c, y), s2 = __shfl_xor_sync(0xffffffffu, sn, y);
                         // columns: positions (0, x) belong to this lane's pair, (y, y ^ x) to the other pair; the
                         // entry at position k is column t ^ k, the lower column of its pair iff (t ^ k) < (t ^ k ^ x)
@@ -298,6 +312,17 @@ compress_kernel(Geometry geo, const unsigned char *dense_pool, unsigned char *fa
                         e[0] = c * e0 - sa * p0; e[x] = c * ex - sa * px;
                         e[y] = c * ey - sa * py; e[y ^ x] = c * eyx - sa * pyx;
                     }
+                    // e now holds row t of J^T D J over all six rotations = the quad's diagonal block of the new G:
+                    // written here (upper triangle and its mirror image), so the block phase can leave it alone
+#pragma unroll
+                    for (int k = 0; k < 4; ++k) {
+                        const int cc = t ^ k;
+                        if (cc >= t) {
+                            const int mc = (m4 >> (8 * cc)) & 0xff;
+                            S.G[mt * kGs + mc] = e[k];
+                            S.G[mc * kGs + mt] = e[k];
+                        }
+                    }
                     // natural column order: M[t][c] = f[t ^ c]
                     float r0 = f[0], r1 = f[1], r2 = f[2], r3 = f[3];
                     if (t & 1) { float w = r0; r0 = r1; r1 = w; w = r2; r2 = r3; r3 = w; }
@@ -312,7 +337,7 @@ compress_kernel(Geometry geo, const unsigned char *dense_pool, unsigned char *fa
                 }
                 __syncthreads();
                 if (warp < Qd::kGWarps) {
-                    const int h = lane / kQuads, ia = lane % kQuads, delta = Qd::kDiag * warp + h;
+                    const int h = lane / kQuads, ia = lane % kQuads, delta = 1 + Qd::kDiag * warp + h;
                     if (delta < kQuads / 2 || (delta == kQuads / 2 && ia < kQuads / 2)) {
                         const int ib = (ia + delta) % kQuads;
                         // member order j ^ x: byte j of the permuted word is byte j ^ x of the table's
@@ -349,11 +374,8 @@ compress_kernel(Geometry geo, const unsigned char *dense_pool, unsigned char *fa
                             y[3] = fmaf(T[i][3], b3.w, fmaf(T[i][2], b2.w, fmaf(T[i][1], b1.w, T[i][0] * b0.w)));
 #pragma unroll
                             for (int j = 0; j < 4; ++j) {
-                                // the diagonal block (a = b) is symmetric: its upper triangle is written to both sides
-                                if (delta != 0 || j >= i) {
-                                    S.G[ma[i] * kGs + mb[j]] = y[j];
-                                    S.G[mb[j] * kGs + ma[i]] = y[j];
-                                }
+                                S.G[ma[i] * kGs + mb[j]] = y[j];
+                                S.G[mb[j] * kGs + ma[i]] = y[j];
                             }
                         }
                     }
@@ -406,14 +428,8 @@ compress_kernel(Geometry geo, const unsigned char *dense_pool, unsigned char *fa
                 if (tid < kPairs) {
                     const int p = pr[tid].x, q = pr[tid].y;
                     const float gpp = S.G[p * kGs + p], gqq = S.G[q * kGs + q], gpq = S.G[p * kGs + q];
-                    float c = 1.f, s = 0.f;
-                    if (fabsf(gpq) > fmaxf(tol * sqrtf(fabsf(gpp * gqq)), floor_abs)) {
-                        const float theta = (gqq - gpp) / (2.f * gpq);
-                        const float t = copysignf(1.f, theta) / (fabsf(theta) + sqrtf(1.f + theta * theta));
-                        c = rsqrtf(1.f + t * t);
-                        s = t * c;
-                        rotated = 1;
-                    }
+                    float c, s;
+                    if (jacobi_rotation(gpp, gqq, gpq, tol, floor_abs, c, s)) rotated = 1;
                     S.cs[tid] = make_float2(c, s);
                 }
                 __syncthreads();
