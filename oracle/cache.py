@@ -234,6 +234,32 @@ class OracleCache:
                     out[i, h] = _att.attention_plain(q[i, h], K_all, V_all, self.scale)
         return out
 
+    def decode_attention_multi(self, layer, seq_ids, q):
+        """Several queries per sequence (speculative decoding, a chunk of a
+        prefill): q is [n_seqs, q_len, H_q, d] and query j belongs to the
+        position T - q_len + j of its sequence, whose key and value rows are
+        already in the cache.  Eq. 1 is causal: that position attends over the
+        tokens 0 .. T - q_len + j, itself included.  Not spelled out in the
+        paper (its Eq. 4 has one query); q_len = 1 is decode_attention().
+        Returns [n_seqs, q_len, H_q, d] fp64."""
+        c = self.cfg
+        q = np.asarray(q, dtype=np.float64)
+        n, q_len = q.shape[0], q.shape[1]
+        G = c.n_q_heads // c.n_kv_heads
+        out = np.zeros((n, q_len, c.n_q_heads, c.head_dim))
+        for i, seq in enumerate(seq_ids):
+            sl = self.state.get((int(seq), layer))
+            if sl is None or sl.n_tokens < q_len:
+                raise ValueError("fewer tokens in the cache than queries")
+            for kvh in range(c.n_kv_heads):
+                K_all, V_all = self.gather_kv(int(seq), layer, kvh)
+                for j in range(q_len):
+                    visible = sl.n_tokens - q_len + j + 1
+                    for g in range(G):
+                        h = kvh * G + g
+                        out[i, j, h] = _att.attention_plain(q[i, j, h], K_all[:visible], V_all[:visible], self.scale)
+        return out
+
     def decode_attention_pagewise(self, layer, seq_ids, q):
         """Same result through Eq. 4 (factor pages evaluated from factors, never
         materialised) and Eq. 5 (merge).  Used to check the algebra only."""

@@ -105,6 +105,61 @@ def test_pagewise_route_equals_plain_route_and_zero_query_mean():
         assert np.abs(out0[0, h] - V_all.mean(axis=0)).max() <= 1e-14
 
 
+def _causal_block(Q, K, V, scale):
+    """Textbook causal attention for the last len(Q) positions of a sequence of len(K) tokens, written as one
+    masked score matrix (no per-query slicing): independent of how the oracle walks its pages."""
+    n_q, T = Q.shape[0], K.shape[0]
+    S = Q @ K.T * scale
+    pos = np.arange(T)[None, :]
+    own = (T - n_q + np.arange(n_q))[:, None]
+    S = np.where(pos <= own, S, -np.inf)
+    W = np.exp(S - S.max(axis=1, keepdims=True))
+    return (W / W.sum(axis=1, keepdims=True)) @ V
+
+
+def test_multi_query_attention_pins():
+    rng = np.random.default_rng(21)
+    # (a) all-dense cache: the textbook causal block
+    cfg = _cfg(recent_tokens=8 * 100)
+    c = OracleCache(cfg)
+    k, v = _kv(rng, 45, cfg)
+    c.append_kv(0, [0], [45], k, v)
+    for q_len in (1, 3, 8, 11):
+        q = rng.standard_normal((1, q_len, cfg.n_q_heads, cfg.head_dim))
+        out = c.decode_attention_multi(0, [0], q)
+        for h in range(cfg.n_q_heads):
+            ref = _causal_block(q[0, :, h], k[:, h // 2], v[:, h // 2], 0.25)
+            assert np.abs(out[0, :, h] - ref).max() <= 1e-13
+    # (b) mixed cache: the last query is the single-query call; an earlier query equals the single-query call on a
+    #     cache that was fed the same tokens, compressed at the same moment, and then given fewer new tokens
+    cfg = _cfg()
+    c = OracleCache(cfg)
+    k, v = _kv(rng, 77, cfg)
+    c.append_kv(0, [0], [70], k[:70], v[:70])
+    c.compress_eligible_pages()
+    c.append_kv(0, [0], [7], k[70:], v[70:])
+    q = rng.standard_normal((1, 5, cfg.n_q_heads, cfg.head_dim))
+    out = c.decode_attention_multi(0, [0], q)
+    assert np.array_equal(out[:, 4], c.decode_attention(0, [0], q[:, 4]))
+    c2 = OracleCache(cfg)
+    c2.append_kv(0, [0], [70], k[:70], v[:70])
+    c2.compress_eligible_pages()
+    c2.append_kv(0, [0], [4], k[70:74], v[70:74])           # 74 tokens: what query 1 of 5 sees (77 - 5 + 1 + 1)
+    assert np.abs(out[:, 1] - c2.decode_attention(0, [0], q[:, 1])).max() <= 1e-14
+    # (c) the first token's own query returns its value row; zero queries give running means
+    c3 = OracleCache(_cfg(recent_tokens=8 * 100))
+    c3.append_kv(0, [1], [6], k[:6], v[:6])
+    q = rng.standard_normal((1, 6, cfg.n_q_heads, cfg.head_dim))
+    out = c3.decode_attention_multi(0, [1], q)
+    for h in range(cfg.n_q_heads):
+        assert np.abs(out[0, 0, h] - v[0, h // 2]).max() <= 1e-14
+    out0 = c3.decode_attention_multi(0, [1], np.zeros_like(q))
+    for j in range(6):
+        assert np.abs(out0[0, j, 0] - v[:j + 1, 0].mean(axis=0)).max() <= 1e-14
+    with pytest.raises(ValueError):
+        c3.decode_attention_multi(0, [1], np.zeros((1, 7, cfg.n_q_heads, cfg.head_dim)))
+
+
 def test_output_invariant_under_slot_permutation():
     cfg = _cfg()
     rng = np.random.default_rng(3)
