@@ -217,6 +217,26 @@ pkv_status pkv_decode_attention(pkv_cache *c, int32_t layer, int32_t n_seqs, con
                                 const void *q, void *out, float *out_f32, void *stream);
 
 /*
+ * Mixed attention for the q_len newest positions of each sequence at once (a speculative-decoding step, or a
+ * chunk of a prefill after its rows were appended).  The paper's Eq. 4 carries one query; this is the same
+ * operation under the causal rule of Eq. 1: query j (0 <= j < q_len) of a sequence with T tokens in `layer`
+ * belongs to position T - q_len + j and attends over tokens 0 .. T - q_len + j, itself included, factor pages
+ * through their factors and dense pages through their rows exactly as in pkv_decode_attention(); partial states
+ * merge by Eq. 5.  q_len = 1 is pkv_decode_attention().
+ *   q, out  [device] bf16 [n_seqs, q_len, H_q, d];  out_f32 [device, may be NULL] fp32, same shape
+ * Requirements (else PKV_ERR_INVALID_ARG, nothing launched): 1 <= q_len <= T for every listed sequence; no listed
+ * sequence has a factor page that reaches past token T - q_len (so every query sees every factor page whole:
+ * holds whenever q_len <= recent_tokens and compression ran no later than the append of these positions, and it is
+ * checked per call); n_seqs * ceil(q_len / max(1, 8 / (H_q / H_kv))) <= max_seqs, the number of plan entries.
+ * Cost: queries are processed in blocks of 8 / (H_q / H_kv) tokens, and every block walks the sequence's pages
+ * again, so the KV bytes read grow with the number of blocks, not with q_len.
+ * Needs decode_variant 0 (PKV_ERR_UNSUPPORTED otherwise).  CUDA-graph and overlap semantics as for
+ * pkv_decode_attention(); the plan is kept per (layer, batch, q_len).
+ */
+pkv_status pkv_decode_attention_multi(pkv_cache *c, int32_t layer, int32_t n_seqs, const int32_t *seq_ids,
+                                      int32_t q_len, const void *q, void *out, float *out_f32, void *stream);
+
+/*
  * The same call for callers whose queries and results live in host memory.
  *   q_host, out_host [host] bf16 [n_seqs, H_q, d];  q_stage, out_stage [device]
  *   caller-owned staging buffers of the same size.

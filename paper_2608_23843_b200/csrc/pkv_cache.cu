@@ -42,6 +42,7 @@ struct PlanCache {
     bool valid = false;
     std::vector<int32_t> seq_ids;
     std::vector<uint64_t> versions;
+    int q_len = 1;                     // query tokens per sequence the plan was built for
     int n_segs = 0;
     int64_t units = 0;
     std::vector<PlanCta> ctas;         // n_used + 1 entries (last = end sentinel)
@@ -328,19 +329,27 @@ int first_unit_at_or_after(const HeadShape &h, long long rem, long long cf, long
     return h.d0_units + h.nf + (int)std::min<long long>((rem + cd - 1) / cd, h.d1_units);
 }
 
-pkv_status build_plan(pkv_cache *c, int layer, int n_seqs, const int32_t *seq_ids, cudaStream_t st) {
+// Query tokens that share one score tile (eight query columns), and plan entries per sequence.
+int queries_per_tile(const Geometry &g, int q_len) { return std::max(1, std::min(q_len, kMaxGroup / g.group)); }
+int entries_per_seq(const Geometry &g, int q_len) { const int t = queries_per_tile(g, q_len); return (q_len + t - 1) / t; }
+
+// `n_listed` sequences with q_len queries each: every sequence takes entries_per_seq() consecutive plan entries
+// (one per block of query tokens), each of which walks all the sequence's pages.
+pkv_status build_plan(pkv_cache *c, int layer, int n_listed, const int32_t *seq_ids, int q_len, cudaStream_t st) {
     const Geometry &g = c->geo;
     PlanCache &pc = c->plans[layer];
     const int H = g.n_kv_heads, N = g.n_ctas;
     const long long cf = g.blob_bytes + 2048, cd = (long long)g.block_tokens * 2 * kRowBytes + 2048;
+    const int per_seq = entries_per_seq(g, q_len), n_seqs = n_listed * per_seq;
 
     std::vector<PlanEntry> entries(n_seqs);
     std::vector<HeadShape> shapes(n_seqs);
     long long total_cost = 0, total_units = 0;
     for (int i = 0; i < n_seqs; ++i) {
-        const SeqLayer &s = c->at(seq_ids[i], layer);
+        const int32_t seq = seq_ids[i / per_seq];
+        const SeqLayer &s = c->at(seq, layer);
         int n_pages = (s.n_tokens + c->cfg.page_size - 1) / c->cfg.page_size;
-        entries[i] = PlanEntry{seq_ids[i], n_pages, g.sink_pages, s.f_end};
+        entries[i] = PlanEntry{seq, n_pages, g.sink_pages, s.f_end};
         shapes[i] = head_shape(g, n_pages, g.sink_pages, s.f_end, cf, cd);
         total_cost += shapes[i].cost * H;
         total_units += (long long)shapes[i].units * H;
@@ -392,9 +401,10 @@ pkv_status build_plan(pkv_cache *c, int layer, int n_seqs, const int32_t *seq_id
     PlanHeader hdr{n_seqs, n_used, n_segs, (int)std::min<long long>(total_units, INT32_MAX)};
 
     pc.valid = true;
-    pc.seq_ids.assign(seq_ids, seq_ids + n_seqs);
-    pc.versions.resize(n_seqs);
-    for (int i = 0; i < n_seqs; ++i) pc.versions[i] = c->at(seq_ids[i], layer).version;
+    pc.q_len = q_len;
+    pc.seq_ids.assign(seq_ids, seq_ids + n_listed);
+    pc.versions.resize(n_listed);
+    for (int i = 0; i < n_listed; ++i) pc.versions[i] = c->at(seq_ids[i], layer).version;
     pc.n_segs = n_segs;
     pc.units = total_units;
     pc.ctas = ctas;
@@ -415,9 +425,9 @@ pkv_status build_plan(pkv_cache *c, int layer, int n_seqs, const int32_t *seq_id
     return stager_flush(c, st);
 }
 
-bool plan_is_current(pkv_cache *c, int layer, int n_seqs, const int32_t *seq_ids) {
+bool plan_is_current(pkv_cache *c, int layer, int n_seqs, const int32_t *seq_ids, int q_len) {
     const PlanCache &pc = c->plans[layer];
-    if (!pc.valid || (int)pc.seq_ids.size() != n_seqs) return false;
+    if (!pc.valid || (int)pc.seq_ids.size() != n_seqs || pc.q_len != q_len) return false;
     for (int i = 0; i < n_seqs; ++i) {
         if (pc.seq_ids[i] != seq_ids[i]) return false;
         if (pc.versions[i] != c->at(seq_ids[i], layer).version) return false;
@@ -670,6 +680,11 @@ pkv_status pkv_compress_eligible_pages(pkv_cache *c, int32_t layer, int64_t *n_p
 
 pkv_status pkv_decode_attention(pkv_cache *c, int32_t layer, int32_t n_seqs, const int32_t *seq_ids,
                                 const void *q, void *out, float *out_f32, void *stream) {
+    return pkv_decode_attention_multi(c, layer, n_seqs, seq_ids, 1, q, out, out_f32, stream);
+}
+
+pkv_status pkv_decode_attention_multi(pkv_cache *c, int32_t layer, int32_t n_seqs, const int32_t *seq_ids,
+                                      int32_t q_len, const void *q, void *out, float *out_f32, void *stream) {
     if (!c) return PKV_ERR_INVALID_ARG;
     cudaStream_t st = (cudaStream_t)stream;
     if (layer < 0 || layer >= c->cfg.n_layers) return fail(c, PKV_ERR_INVALID_ARG, "layer %d out of range", layer);
@@ -678,16 +693,33 @@ pkv_status pkv_decode_attention(pkv_cache *c, int32_t layer, int32_t n_seqs, con
     for (int i = 0; i < n_seqs; ++i)
         if (c->at(seq_ids[i], layer).n_tokens == 0)
             return fail(c, PKV_ERR_INVALID_ARG, "sequence %d has no tokens in layer %d", seq_ids[i], layer);
+    if (q_len < 1 || q_len > 32767) return fail(c, PKV_ERR_INVALID_ARG, "q_len %d out of range", q_len);
+    if (q_len > 1) {
+        if (c->cfg.decode_variant != 0)
+            return fail(c, PKV_ERR_UNSUPPORTED, "several queries per sequence need the tensor-core kernel (decode_variant 0)");
+        if ((long long)n_seqs * entries_per_seq(c->geo, q_len) > c->cfg.max_seqs)
+            return fail(c, PKV_ERR_INVALID_ARG, "%d sequences x %d query blocks exceed max_seqs = %d plan entries", n_seqs,
+                        entries_per_seq(c->geo, q_len), c->cfg.max_seqs);
+        for (int i = 0; i < n_seqs; ++i) {
+            const SeqLayer &s = c->at(seq_ids[i], layer);
+            // every query must see every factor page whole (and at least its own position)
+            const int first_visible = s.n_tokens - q_len + 1;
+            if (first_visible < 1 || (s.f_end > c->geo.sink_pages && s.f_end * c->cfg.page_size > first_visible))
+                return fail(c, PKV_ERR_INVALID_ARG, "sequence %d: the %d newest positions reach into compressed pages "
+                            "or past the start (%d tokens, factor pages end at token %d)", seq_ids[i], q_len, s.n_tokens,
+                            s.f_end > c->geo.sink_pages ? s.f_end * c->cfg.page_size : 0);
+        }
+    }
     if (!c->dry && (!q || !out)) return fail(c, PKV_ERR_INVALID_ARG, "q or out is NULL");
-    if (!plan_is_current(c, layer, n_seqs, seq_ids)) {
+    if (!plan_is_current(c, layer, n_seqs, seq_ids, q_len)) {
         // the plan is uploaded through the staging ring: a copy recorded into a graph would replay stale bytes
         if (!c->dry && is_capturing(st))
             return fail(c, PKV_ERR_UNSUPPORTED, "the decode plan of layer %d must be rebuilt: call pkv_decode_attention "
                         "once outside the stream capture for this layer and batch first", layer);
-        if ((r = build_plan(c, layer, n_seqs, seq_ids, st)) != PKV_OK) return r;
+        if ((r = build_plan(c, layer, n_seqs, seq_ids, q_len, st)) != PKV_OK) return r;
     }
     const PlanCache &pc = c->plans[layer];
-    int64_t bytes = 2LL * n_seqs * c->cfg.n_q_heads * kRowBytes;          // q and out
+    int64_t bytes = 2LL * n_seqs * q_len * c->cfg.n_q_heads * kRowBytes;  // q and out
     for (int i = 0; i < n_seqs; ++i) {
         const SeqLayer &s = c->at(seq_ids[i], layer);
         const int n_pages = (int)s.slots.size();
@@ -709,6 +741,10 @@ pkv_status pkv_decode_attention(pkv_cache *c, int32_t layer, int32_t n_seqs, con
     a.plan_cta = c->ml.plan_cta; a.plan_entry = c->ml.plan_entry; a.plan_seg = c->ml.plan_seg;
     a.plan_cta_entry = c->ml.plan_cta_entry;
     a.q = q; a.out = out; a.out_f32 = out_f32;
+    a.q_len = q_len;
+    a.q_tpt = queries_per_tile(c->geo, q_len);
+    a.q_nblk = entries_per_seq(c->geo, q_len);
+    a.q_cols = a.q_tpt * c->geo.group;
     // decode_overlap = 2: launches never wait for one another, so launches in flight must not share split-K
     // scratch.  The scratch rotates over wl.n_sets sets and every (n_sets-1)-th launch is a plain
     // one (no programmatic serialization: it starts after all earlier work on the stream has finished), so
@@ -751,8 +787,8 @@ pkv_status pkv_decode_attention_static_scratch(pkv_cache *c, int32_t layer, int3
         if (c->at(seq_ids[i], layer).n_tokens == 0)
             return fail(c, PKV_ERR_INVALID_ARG, "sequence %d has no tokens in layer %d", seq_ids[i], layer);
     if (!q || !out) return fail(c, PKV_ERR_INVALID_ARG, "q or out is NULL");
-    if (!plan_is_current(c, layer, n_seqs, seq_ids)) {
-        if ((r = build_plan(c, layer, n_seqs, seq_ids, st)) != PKV_OK) return r;
+    if (!plan_is_current(c, layer, n_seqs, seq_ids, 1)) {
+        if ((r = build_plan(c, layer, n_seqs, seq_ids, 1, st)) != PKV_OK) return r;
     }
     DecodeArgs a;
     a.geo = c->geo;
@@ -763,6 +799,7 @@ pkv_status pkv_decode_attention_static_scratch(pkv_cache *c, int32_t layer, int3
     a.plan_cta = c->ml.plan_cta; a.plan_entry = c->ml.plan_entry; a.plan_seg = c->ml.plan_seg;
     a.plan_cta_entry = c->ml.plan_cta_entry;
     a.q = q; a.out = out; a.out_f32 = out_f32;
+    a.q_len = 1; a.q_tpt = 1; a.q_nblk = 1; a.q_cols = c->geo.group;
     a.partials = nullptr; a.tickets = nullptr;            // set by the launcher from the static scratch
     a.plain_launch = 0;                                   // the launcher's memset already orders it after earlier work
     c->cache_written = false;

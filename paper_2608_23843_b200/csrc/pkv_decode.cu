@@ -34,6 +34,7 @@ namespace pkv {
 namespace {
 
 constexpr float kNegInf = -1e30f;      // finite stand-in for -inf: exp2(kNegInf - x) == 0, no NaN from inf - inf
+constexpr float kMasked = -2e30f;      // score of a token a query must not see: exp2(kMasked - m) == 0 even while m == kNegInf
 constexpr int kKindDense = 0, kKindFactor = 1, kKindEnd = 2;
 
 struct Range {
@@ -335,7 +336,7 @@ __device__ __forceinline__ uint32_t pack_bf16(float lo, float hi) {
 __device__ __forceinline__ float bf16lo_f(uint32_t x) { return __uint_as_float(x << 16); }
 __device__ __forceinline__ float bf16hi_f(uint32_t x) { return __uint_as_float(x & 0xffff0000u); }
 
-struct StageDesc { int kind, rows, seg, pad; };
+struct StageDesc { int kind, rows, seg, after; };     // after: tokens of the sequence that follow this unit's rows
 
 // Per-warp running state for the query heads 2t, 2t+1 (t = lane & 3) of one KV head.
 struct WarpState {
@@ -635,10 +636,12 @@ __device__ __forceinline__ void factor_unit_int4(uint32_t sb, const Geometry &g,
 #undef PKV_I4
 
 
-// One block of DB rows of a dense page: K rows at sb, V rows at sb + DB*256; `rows` of them are valid.
+// One block of DB rows of a dense page: K rows at sb, V rows at sb + DB*256; `rows` of them are valid.  Query
+// columns 2t and 2t+1 of this lane see the first lim0 and lim1 of them (all `rows` unless the call carries several
+// query tokens per sequence and the block holds positions after the column's own).
 template <int DB>
-__device__ __forceinline__ void dense_unit(uint32_t sb, unsigned char *sp, int rows, const uint32_t (&qf)[8][2],
-                                           float scale, WarpState &st, int lane) {
+__device__ __forceinline__ void dense_unit(uint32_t sb, unsigned char *sp, int rows, int lim0, int lim1,
+                                           const uint32_t (&qf)[8][2], float scale, WarpState &st, int lane) {
     constexpr int NI = DB / 16;
     const int l7 = lane & 7, mi = lane >> 3, g = lane >> 2;
     if (rows < DB) {
@@ -657,9 +660,8 @@ __device__ __forceinline__ void dense_unit(uint32_t sb, unsigned char *sp, int r
             ldsm_x4(a4, sb + (16 * i + (mi & 1) * 8 + l7) * kRowBytes + (((2 * kk + (mi >> 1)) ^ l7) << 4));
             mma16816(s[i], a4[0], a4[1], a4[2], a4[3], qf[kk][0], qf[kk][1]);
         }
-        const bool v0 = 16 * i + g < rows, v1 = 16 * i + 8 + g < rows;
-        s[i][0] = v0 ? s[i][0] * scale : kNegInf; s[i][1] = v0 ? s[i][1] * scale : kNegInf;
-        s[i][2] = v1 ? s[i][2] * scale : kNegInf; s[i][3] = v1 ? s[i][3] * scale : kNegInf;
+        s[i][0] = 16 * i + g < lim0 ? s[i][0] * scale : kMasked;     s[i][1] = 16 * i + g < lim1 ? s[i][1] * scale : kMasked;
+        s[i][2] = 16 * i + 8 + g < lim0 ? s[i][2] * scale : kMasked; s[i][3] = 16 * i + 8 + g < lim1 ? s[i][3] * scale : kMasked;
     }
     uint32_t T0[4], T1[4];
     online_softmax<NI>(s, st, T0, T1);
@@ -682,27 +684,41 @@ __device__ __forceinline__ void reset_state(WarpState &st) {
     st.l[0] = st.l[1] = 0.f;
 }
 
-__device__ __forceinline__ void load_q(const DecodeArgs &a, int seg, uint32_t (&qf)[8][2], int lane) {
+// Query column n of a segment's score tile = query head n % G of the (n / G)-th query token of the plan entry's
+// block; with one query per sequence (q_len = 1) that is query head n.  Row of q / out it maps to, or -1.
+__device__ __forceinline__ long long q_row(const DecodeArgs &a, int seg, int n) {
     const int H = a.geo.n_kv_heads, G = a.geo.group;
-    const int entry = seg / H, head = seg % H, g = lane >> 2, t = lane & 3;
-    if (g < G) {
-        const uint32_t *q = reinterpret_cast<const uint32_t *>(
-            reinterpret_cast<const __nv_bfloat16 *>(a.q) + ((long long)entry * a.geo.n_q_heads + head * G + g) * kHeadDim);
+    const int entry = seg / H, head = seg % H, jl = n / G, j = (entry % a.q_nblk) * a.q_tpt + jl;
+    if (jl >= a.q_tpt || j >= a.q_len) return -1;
+    return ((long long)(entry / a.q_nblk) * a.q_len + j) * a.geo.n_q_heads + head * G + n % G;
+}
+
+// Loads the lane's share of the segment's queries.  Returns, packed in 16-bit halves, how many of the sequence's
+// newest positions the lane's columns 2t and 2t+1 must not see (q_len - 1 - the column's query token).
+__device__ __forceinline__ int load_q(const DecodeArgs &a, int seg, uint32_t (&qf)[8][2], int lane) {
+    const int t = lane & 3;
+    const long long row = q_row(a, seg, lane >> 2);
+    if (row >= 0) {
+        const uint32_t *q = reinterpret_cast<const uint32_t *>(reinterpret_cast<const __nv_bfloat16 *>(a.q) + row * kHeadDim);
 #pragma unroll
         for (int kk = 0; kk < 8; ++kk) { qf[kk][0] = __ldg(q + 8 * kk + t); qf[kk][1] = __ldg(q + 8 * kk + 4 + t); }
     } else {
 #pragma unroll
         for (int kk = 0; kk < 8; ++kk) qf[kk][0] = qf[kk][1] = 0u;
     }
+    if (a.q_len == 1) return 0;
+    const int G = a.geo.group, j0 = ((seg / a.geo.n_kv_heads) % a.q_nblk) * a.q_tpt;
+    const int b0 = max(0, a.q_len - 1 - j0 - (2 * t) / G), b1 = max(0, a.q_len - 1 - j0 - (2 * t + 1) / G);
+    return b0 | (b1 << 16);
 }
 
-// Writes the final result of one (entry, KV head) for query head hq, dims d4..d4+3.
+// Writes the final result of one (entry, KV head) for query column hq, dims d4..d4+3.
 __device__ __forceinline__ void store_out(const DecodeArgs &a, int seg, int hq, int d4, float4 acc, float L) {
-    const Geometry &g = a.geo;
-    const int entry = seg / g.n_kv_heads, head = seg % g.n_kv_heads;
+    const long long row = q_row(a, seg, hq);
+    if (row < 0) return;
     const float inv = 1.f / L;
     acc.x *= inv; acc.y *= inv; acc.z *= inv; acc.w *= inv;
-    const long long off = ((long long)entry * g.n_q_heads + head * g.group + hq) * kHeadDim + d4;
+    const long long off = row * kHeadDim + d4;
     __nv_bfloat162 lo = __floats2bfloat162_rn(acc.x, acc.y), hi = __floats2bfloat162_rn(acc.z, acc.w);
     uint2 packed;
     packed.x = *reinterpret_cast<unsigned *>(&lo);
@@ -717,7 +733,7 @@ __device__ __forceinline__ void store_out(const DecodeArgs &a, int seg, int hq, 
 template <int E, int kBatch>
 __device__ __forceinline__ void merge_parts(const DecodeArgs &a, const float *first, int np, int seg, int ctid) {
     constexpr int kThreads = kConsumerWarps * 32;
-    const int n_items = a.geo.group * 32;
+    const int n_items = a.q_cols * 32;
     const int d4 = (ctid & 31) * 4;                               // kThreads is a multiple of 32
     bool has[E];
     int hq[E];
@@ -815,7 +831,7 @@ __device__ __forceinline__ void flush_segment(const DecodeArgs &a, float *comb, 
             L += f * cw[kMaxGroup * kHeadDim + kMaxGroup + hq];
         }
         if (ps.n_parts <= 1) {
-            if (hq < a.geo.group) store_out(a, seg, hq, d4, acc, L);
+            if (hq < a.q_cols) store_out(a, seg, hq, d4, acc, L);
         } else {
             *reinterpret_cast<float4 *>(part + hq * kHeadDim + d4) = acc;
             if ((item & 31) == 0) {
@@ -832,7 +848,7 @@ __device__ __forceinline__ void flush_segment(const DecodeArgs &a, float *comb, 
         if (*last_flag) {
             __threadfence();
             const float *first = a.partials + ((long long)ps.cta_first + seg) * kPartialFloats;
-            if (a.geo.group * 32 <= kThreads) merge_parts<1, 16>(a, first, ps.n_parts, seg, ctid);
+            if (a.q_cols * 32 <= kThreads) merge_parts<1, 16>(a, first, ps.n_parts, seg, ctid);
             else merge_parts<2, 8>(a, first, ps.n_parts, seg, ctid);
             if (ctid == 0) a.tickets[seg] = 0;          // ready for the next launch
         }
@@ -911,7 +927,7 @@ __global__ void __launch_bounds__(kDecodeThreads, 2) decode_tc_kernel(const __gr
             const int *pt = a.page_table + ((long long)e.seq * geo.n_layers + a.layer) * geo.max_pages;
             for (int u0 = cur.unit; u0 < u_end && ok; u0 += 32) {
                 const int u = u0 + lane;
-                int kind = kKindDense, rows = 0;
+                int kind = kKindDense, rows = 0, after = 0;
                 const unsigned char *src = nullptr;
                 if (u < u_end) {
                     int page, blk;
@@ -926,6 +942,7 @@ __global__ void __launch_bounds__(kDecodeThreads, 2) decode_tc_kernel(const __gr
                         src = a.factor_pool + (long long)slot * geo.factor_slot_bytes + (long long)cur.head * geo.blob_bytes;
                     } else {
                         rows = max(0, min(kDB, T - page * P - blk * kDB));
+                        after = max(0, T - page * P - blk * kDB - rows);
                         src = a.dense_pool + (long long)slot * geo.dense_slot_bytes +
                               (long long)cur.head * geo.dense_head_bytes + blk * kDB * kRowBytes;
                     }
@@ -942,7 +959,7 @@ __global__ void __launch_bounds__(kDecodeThreads, 2) decode_tc_kernel(const __gr
                     const long long t0 = clock64();
                     while (__any_sync(0xffffffffu, pending)) {
                         if (pending && (kj < S || mbar_try_wait(smem_u32(empty_bar + s), ((kj / S) - 1) & 1))) {
-                            descs[s] = StageDesc{kind, rows, seg_local, 0};
+                            descs[s] = StageDesc{kind, rows, seg_local, after};
                             const uint32_t bar = smem_u32(full_bar + s);
                             const uint32_t dst = smem_u32(stages + (size_t)s * stage_bytes);
                             if (kind == kKindFactor) {
@@ -1003,7 +1020,7 @@ __global__ void __launch_bounds__(kDecodeThreads, 2) decode_tc_kernel(const __gr
         }
         uint32_t qf[8][2];
         int cur_seg = 0;
-        load_q(a, rg.seg_first, qf, lane);
+        int hidden = load_q(a, rg.seg_first, qf, lane);
         bool ok = true;
         for (int k = warp;; k += W) {
             const int s = k % S;
@@ -1017,7 +1034,7 @@ __global__ void __launch_bounds__(kDecodeThreads, 2) decode_tc_kernel(const __gr
             if (cur_seg < dsc.seg) {
                 // the old segment's queries are no longer needed: fetch the new ones now, so that their latency
                 // hides behind the flush
-                if (dsc.seg < rg.n_local_segs) load_q(a, rg.seg_first + dsc.seg, qf, lane);
+                if (dsc.seg < rg.n_local_segs) hidden = load_q(a, rg.seg_first + dsc.seg, qf, lane);
                 while (cur_seg < dsc.seg) {
                     flush_segment(a, comb, last_flag, st, rg.seg_first + cur_seg, warp, lane, tid, W);
                     ++cur_seg;
@@ -1033,7 +1050,11 @@ __global__ void __launch_bounds__(kDecodeThreads, 2) decode_tc_kernel(const __gr
                     else factor_unit<P, NT>(sb, geo.ak_off, geo.bk_off, geo.av_off, geo.bv_off, geo.rank_k, geo.rank_v, qf,
                                             geo.scale_log2e, st, lane);
                 } else {
-                    dense_unit<kDB>(sb, stages + (size_t)s * stage_bytes, dsc.rows, qf, geo.scale_log2e, st, lane);
+                    // a column does not see the sequence's last `hidden` positions; `after` of those lie beyond
+                    // this unit's rows
+                    const int lim0 = dsc.rows - max(0, (hidden & 0xffff) - dsc.after);
+                    const int lim1 = dsc.rows - max(0, (hidden >> 16) - dsc.after);
+                    dense_unit<kDB>(sb, stages + (size_t)s * stage_bytes, dsc.rows, lim0, lim1, qf, geo.scale_log2e, st, lane);
                     if (dsc.rows < kDB) asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
                 }
             }

@@ -99,6 +99,10 @@ struct DecodeArgs {
     float *partials;
     int *tickets;                      // one per segment, zero between launches
 
+    // Queries per sequence (1 = decoding).  A score tile has eight query columns: q_tpt = min(q_len, 8 / group)
+    // consecutive query tokens fill q_cols = q_tpt * group of them, so a sequence takes q_nblk = ceil(q_len / q_tpt)
+    // plan entries, each walking the sequence's pages for its own block of query tokens.
+    int q_len, q_tpt, q_nblk, q_cols;
     int *status;
     int layer;
     int variant;                       // 0 = tensor-core pipeline, 1 = scalar reference kernel

@@ -29,6 +29,7 @@ EXPORTS = [
     "pkv_decode_attention", "pkv_decode_attention_host", "pkv_get_page_table", "pkv_get_stats",
     "pkv_free_seq", "pkv_destroy_cache", "pkv_last_error", "pkv_read_factors", "pkv_write_factors",
     "pkv_read_dense", "pkv_get_decode_plan", "pkv_decode_attention_static_scratch", "pkv_get_decode_trace",
+    "pkv_decode_attention_multi",
     "pkv_get_rotation_schedule",
 ]
 
@@ -82,6 +83,7 @@ def lib():
         L.pkv_compress_eligible_pages.argtypes = [vp, i32, ctypes.POINTER(i64), vp]
         L.pkv_decode_attention.argtypes = [vp, i32, i32, ip, vp, vp, vp, vp]
         L.pkv_decode_attention_static_scratch.argtypes = [vp, i32, i32, ip, vp, vp, vp, vp]
+        L.pkv_decode_attention_multi.argtypes = [vp, i32, i32, ip, i32, vp, vp, vp, vp]
         L.pkv_decode_attention_host.argtypes = [vp, i32, i32, ip, vp, vp, vp, vp, vp]
         L.pkv_get_page_table.argtypes = [vp, i32, i32, ip, ip, ip, ip]
         L.pkv_get_stats.argtypes = [vp, ctypes.POINTER(PkvStats), vp]
@@ -178,6 +180,13 @@ def pkv_compress_eligible_pages(handle, layer=-1, stream=None) -> int:
 def pkv_decode_attention(handle, layer, seq_ids, q, out, out_f32=None, stream=None):
     ids, n = _ints(seq_ids)
     _check(handle, lib().pkv_decode_attention(handle, layer, n, ids, _ptr(q), _ptr(out), _ptr(out_f32), _stream(stream)))
+
+
+def pkv_decode_attention_multi(handle, layer, seq_ids, q_len, q, out, out_f32=None, stream=None):
+    """q, out: [n_seqs, q_len, H_q, d]; query j of a sequence belongs to its position T - q_len + j (causal)."""
+    ids, n = _ints(seq_ids)
+    _check(handle, lib().pkv_decode_attention_multi(handle, layer, n, ids, q_len, _ptr(q), _ptr(out), _ptr(out_f32),
+                                                    _stream(stream)))
 
 
 def pkv_decode_attention_static_scratch(handle, layer, seq_ids, q, out, out_f32=None, stream=None):
@@ -303,6 +312,12 @@ class Cache:
         if out is None and q is not None:
             out = torch.empty_like(q)
         pkv_decode_attention(self.handle, layer, seq_ids, q, out, out_f32, self._st())
+        return out
+
+    def decode_attention_multi(self, layer, seq_ids, q_len, q=None, out=None, out_f32=None):
+        if out is None and q is not None:
+            out = torch.empty_like(q)
+        pkv_decode_attention_multi(self.handle, layer, seq_ids, q_len, q, out, out_f32, self._st())
         return out
 
     def decode_attention_host(self, layer, seq_ids, q_host, out_host, q_stage, out_stage):

@@ -472,3 +472,82 @@ def test_many_tiny_segments_per_cta(rank, n_ctas):
     assert not np.isnan(got).any() and not np.isnan(got32).any()
     g = attention_gates(pair, 0, order, q, got, got32)
     assert_attention_gates(g)
+
+
+@pytest.mark.parametrize("P,rk,rv,G,q_len,bits", [
+    (64, 24, 24, 4, 5, 16),       # two query tokens per tile, three blocks, the last one half empty
+    (64, 24, 24, 8, 3, 16),       # one query token per tile
+    (32, 16, 14, 4, 2, 16),       # a single tile; paper-default page shape
+    (16, 8, 8, 1, 11, 16),        # eight query tokens per tile, two blocks; new positions span two pages
+    (64, 16, 16, 2, 7, 16),       # four query tokens per tile
+    (64, 24, 24, 4, 4, 4),        # INT4 factors
+    (64, 32, 32, 4, 64, 16),      # a prefill chunk of one page, 32 blocks
+])
+def test_multi_query_attention(P, rk, rv, G, q_len, bits):
+    """Several new positions per sequence in one call (causal among themselves): every query row against the
+    oracle attending over the GPU's own stored factors (kernel gate) and over its own (end-to-end gate).  Lengths
+    put the new positions across page and dense-block boundaries, at the very start of a sequence (first query
+    sees one token), and behind long runs of factor pages."""
+    H = 2
+    lengths = [40 * P + 5, q_len, P + 1, 23 * P, 10 * P + P // 2 + 1, 3 * P + q_len // 2]
+    lengths = [max(T, q_len) for T in lengths]
+    n = len(lengths)
+    tpt = max(1, min(q_len, 8 // G))
+    nblk = -(-q_len // tpt)
+    W = max(P, -(-q_len // P) * P)
+    cfg = pkv.make_config(n_layers=1, n_kv_heads=H, n_q_heads=H * G, rank=rk, rank_v=rv, page_size=P, sink_tokens=P,
+                          recent_tokens=W, max_seqs=n * nblk, max_pages_per_seq=48, n_dense_slots=200,
+                          n_factor_slots=120, factor_bits=bits)
+    pair = Pair(cfg, seed=P + q_len)
+    for s, T in enumerate(lengths):
+        k, v = gen_kv(5, 0, s, T, cfg, outlier_prob=0.02)
+        cut = T - q_len
+        if cut:
+            pair.append(0, [s], [k[:cut]], [v[:cut]])
+            pair.compress(0)
+        pair.append(0, [s], [k[cut:]], [v[cut:]])
+        if s % 2:
+            pair.compress(0)           # recent_tokens >= q_len: compressing after the append is allowed too
+    pair.same_tables()
+    assert sum(pair.gpu.page_table(0, 0)[0]) >= 36
+    order = [3, 0, 5, 1, 4, 2]
+    g = torch.Generator().manual_seed(1000 + q_len)
+    q = torch.randn((n, q_len, H * G, 128), generator=g).to(torch.bfloat16)
+    qd = q.cuda()
+    out = torch.empty_like(qd)
+    out32 = torch.empty(qd.shape, dtype=torch.float32, device="cuda")
+    pair.gpu.decode_attention_multi(0, order, q_len, qd, out, out32)
+    torch.cuda.synchronize()
+    got, got32 = f64(out), f64(out32)
+    ref = pair.orc.decode_attention_multi(0, order, f64(q))
+    saved = pair.orc.factor
+    pair.orc.factor = dict(saved)
+    for s in order:
+        pair.load_gpu_factors_into_oracle(s, 0)
+    ref_kernel = pair.orc.decode_attention_multi(0, order, f64(q))
+    pair.orc.factor = saved
+    # what storing the factors in bf16 costs on its own (any implementation): the allowance of the end-to-end gate
+    import copy
+    rounded = copy.deepcopy(pair.orc)
+    rounded.round_factors_to_storage_type()
+    ref_rounded = rounded.decode_attention_multi(0, order, f64(q))
+    worst_k = worst_e = 0.0
+    for i in range(n):
+        for j in range(q_len):
+            worst_k = max(worst_k, rel_err(got32[i, j], ref_kernel[i, j]))
+            worst_e = max(worst_e, rel_err(got[i, j], ref[i, j]))
+            assert rel_err(got32[i, j], ref_kernel[i, j]) <= (1e-2 if bits == 4 else 4e-3), (i, j)
+            assert rel_err(got[i, j], ref_kernel[i, j]) <= 1e-2, (i, j)
+            if bits != 4:
+                floor = rel_err(ref_rounded[i, j], ref[i, j])
+                assert rel_err(got[i, j], ref[i, j]) <= 1e-2 + 3.0 * floor, (i, j, floor)
+    # the last query is the single-query call, bit for bit; and the call is reproducible
+    single = torch.empty((n, H * G, 128), dtype=torch.bfloat16, device="cuda")
+    pair.gpu.decode_attention(0, order, qd[:, q_len - 1].contiguous(), single)
+    again = torch.empty_like(out)
+    pair.gpu.decode_attention_multi(0, order, q_len, qd, again)
+    torch.cuda.synchronize()
+    assert torch.equal(single, out[:, q_len - 1]) and torch.equal(again, out)
+    st = pair.gpu.stats()
+    assert st["device_timeouts"] == 0 and st["bad_slot_indices"] == 0
+    print("multi-query P=%d r=(%d,%d) G=%d q_len=%d bits=%d: kernel max %.2e e2e max %.2e" % (P, rk, rv, G, q_len, bits, worst_k, worst_e))

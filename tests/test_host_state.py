@@ -245,6 +245,56 @@ def test_decode_plan_covers_every_unit_once_and_is_balanced(lengths, rank):
         assert segs[s] == (touching[0], len(touching)), s
 
 
+def test_multi_query_call_plan_and_argument_checks():
+    """Several queries per sequence: a sequence takes ceil(q_len / (8 / G)) plan entries that each cover all its
+    units; the call is refused when a query would not see a whole factor page, when it has no token to see, when
+    the plan entries would not fit, or with the scalar kernel variant."""
+    H, G = 2, 4
+    lengths = [1000, 70, 5]
+    kw = dict(n_layers=1, n_kv_heads=H, n_q_heads=H * G, rank=16, sink_tokens=64, recent_tokens=64, max_seqs=9,
+              max_pages_per_seq=32, n_dense_slots=64, n_factor_slots=64)
+    gpu, _, _ = _pair(**kw)
+    gpu.append_kv(0, [0, 1, 2], lengths)
+    gpu.compress_eligible_pages()
+    gpu.decode_attention(0, [0, 1, 2])
+    base = gpu.stats()
+    q_len = 5                                                  # 2 query tokens per tile -> 3 entries per sequence
+    gpu.decode_attention_multi(0, [2, 0, 1], q_len)
+    st = gpu.stats()
+    assert st["last_decode_units"] == 3 * base["last_decode_units"]
+    assert st["last_decode_bytes"] == base["last_decode_bytes"] + 2 * 3 * (q_len - 1) * H * G * 256
+    starts, segs = pkv.pkv_get_decode_plan(gpu.handle, 0, 296, 9, H)
+    assert starts[0] == (0, 0, 0) and starts[-1] == (9, 0, 0) and len(segs) == 9 * H
+    assert all(n_parts >= 1 for _, n_parts in segs)
+    gpu.decode_attention(0, [2, 0, 1])                         # the same batch with one query: its own plan again
+    assert gpu.stats()["last_decode_units"] == base["last_decode_units"]
+    # q_len = 6 on the 5-token sequence: the first query would see nothing
+    with pytest.raises(pkv.PkvError) as e:
+        gpu.decode_attention_multi(0, [2], 6)
+    assert e.value.status == pkv.PKV_ERR_INVALID_ARG
+    gpu.decode_attention_multi(0, [2], 5)
+    # sequence 0 has factor pages up to token 896 = 1000 - 104: 105 queries is the most that see them whole
+    kinds = gpu.page_table(0, 0)[0]
+    assert kinds.index(0, 1) * 64 == 896
+    gpu.decode_attention_multi(0, [0], 8)
+    with pytest.raises(pkv.PkvError) as e:
+        gpu.decode_attention_multi(0, [0], 106)
+    assert e.value.status == pkv.PKV_ERR_INVALID_ARG
+    # 4 sequences' worth of entries do not fit max_seqs = 9 at three entries each
+    gpu2, _, _ = _pair(**dict(kw, max_seqs=4))
+    gpu2.append_kv(0, [0, 1], [100, 100])
+    with pytest.raises(pkv.PkvError) as e:
+        gpu2.decode_attention_multi(0, [0, 1], 5)
+    assert e.value.status == pkv.PKV_ERR_INVALID_ARG
+    gpu2.decode_attention_multi(0, [0, 1], 4)
+    gpu3, _, _ = _pair(**dict(kw, decode_variant=1))
+    gpu3.append_kv(0, [0], [100])
+    gpu3.decode_attention_multi(0, [0], 1)
+    with pytest.raises(pkv.PkvError) as e:
+        gpu3.decode_attention_multi(0, [0], 2)
+    assert e.value.status == pkv.PKV_ERR_UNSUPPORTED
+
+
 @pytest.mark.parametrize("P", [64, 32, 16])
 def test_rotation_schedule_of_the_page_svd_kernel(P):
     """The order in which the compression kernel rotates index pairs within a sweep (host-side table, no GPU):
