@@ -171,7 +171,7 @@ class ClockSampler:
         return out
 
 
-def build_workload(w, rank, device, overlap=2, n_ctas=0, factor_bits=16, grow=0, keep_kv=False):
+def build_workload(w, rank, device, overlap=2, n_ctas=0, factor_bits=16, grow=0, keep_kv=False, plan_entries_per_seq=1):
     """Allocate the cache, generate each (layer, sequence) on the GPU, append and compress layer by layer.
     grow: tokens every sequence may still gain afterwards (sizes the pools and page tables); keep_kv: also
     return the generated K/V of layer 0 including those `grow` tokens (serving loop)."""
@@ -191,7 +191,7 @@ def build_workload(w, rank, device, overlap=2, n_ctas=0, factor_bits=16, grow=0,
     n_dense_slots = sum(pages) + L * sum(p - f for p, f in zip(pages, n_factor)) + 8
     cfg = pkv.make_config(n_layers=L, n_kv_heads=w["n_kv_heads"], n_q_heads=w["n_q_heads"], rank=rank,
                           rank_v=w.get("rank_v", rank), page_size=P,
-                          sink_tokens=w["sink"], recent_tokens=w["recent"], max_seqs=w["batch"],
+                          sink_tokens=w["sink"], recent_tokens=w["recent"], max_seqs=w["batch"] * plan_entries_per_seq,
                           max_pages_per_seq=max(pages), n_dense_slots=n_dense_slots, n_factor_slots=n_factor_slots,
                           decode_overlap=overlap, n_ctas=n_ctas, factor_bits=factor_bits)
     cache = pkv.Cache(cfg, device, synth.slot_permutation(SEED, n_dense_slots, 0).tolist(),
@@ -405,6 +405,7 @@ def run_reference(args, w, rank):
 def _config_dict(args, w, rank):
     return {"workload": args.workload, "n_layers": w["n_layers"], "layers_per_step": w.get("layers_per_step", w["n_layers"]), "n_q_heads": w["n_q_heads"],
             "n_kv_heads": w["n_kv_heads"], "head_dim": 128, "batch": w["batch"], "context": w["T"],
+            "queries_per_sequence": args.q_len,
             "page_size": w.get("page", 64), "rank": rank, "rank_v": w.get("rank_v", rank), "factor_bits": args.factor_bits, "sink_tokens": w["sink"], "recent_tokens": w["recent"],
             "l2": "inputs larger than L2 (no flush)" if args.workload != "tiny" else "L2-resident (latency only)",
             "overlap": ["0: each launch waits for the previous one",
@@ -441,12 +442,17 @@ def main():
                          "overlap but complete in order, 2 = launches never wait for one another (default)")
     ap.add_argument("--n-ctas", type=int, default=0, help="decode grid size (0 = library default)")
     ap.add_argument("--factor-bits", type=int, default=16, choices=[4, 16], help="factor storage: bf16 or INT4 (paper, Section 4.3)")
+    ap.add_argument("--q-len", type=int, default=1,
+                    help="queries per sequence and step (1 = decoding; more = a speculative-decoding or chunked-prefill step "
+                         "over the newest positions, pkv_decode_attention_multi)")
     ap.add_argument("--graph", action="store_true",
                     help="replay one CUDA graph per step instead of launching every layer from the host (overlap 0 or 1)")
     args = ap.parse_args()
     w = WORKLOADS[args.workload]
     rank = args.rank or w["rank"]
     if args.impl == "reference":
+        if args.q_len != 1:
+            raise SystemExit("--impl reference times the single-query path only")
         run_reference(args, w, rank)
         return
 
@@ -469,11 +475,25 @@ def main():
         if world > 1:
             dist.destroy_process_group()
         return
-    cfg, cache, lengths, comp = build_workload(w, rank, device, args.overlap, args.n_ctas, args.factor_bits)
+    QL = args.q_len
+    per_tile = max(1, min(QL, 8 // (w["n_q_heads"] // w["n_kv_heads"])))
+    cfg, cache, lengths, comp = build_workload(w, rank, device, args.overlap, args.n_ctas, args.factor_bits,
+                                               plan_entries_per_seq=-(-QL // per_tile))
     ids = list(range(w["batch"]))
     L, Hq = w["n_layers"], w["n_q_heads"]
-    qs = [synth.make_q(SEED, layer, 0, w["batch"], Hq, 128, device) for layer in range(L)]
+    if QL == 1:
+        qs = [synth.make_q(SEED, layer, 0, w["batch"], Hq, 128, device) for layer in range(L)]
+    else:
+        if QL > w["recent"] or w.get("serving") or args.graph:
+            raise SystemExit("--q-len must not exceed the workload's dense window; not with the serving loop or --graph")
+        qs = [synth.make_q(SEED, layer, 0, w["batch"] * QL, Hq, 128, device).view(w["batch"], QL, Hq, 128) for layer in range(L)]
     outs = [torch.empty_like(q) for q in qs]
+
+    def attend(layer, q, out):
+        if QL == 1:
+            cache.decode_attention(layer, ids, q, out)
+        else:
+            cache.decode_attention_multi(layer, ids, QL, q, out)
 
     lps = w.get("layers_per_step", L)
     cursor = [0]
@@ -482,7 +502,7 @@ def main():
         for _ in range(lps):
             layer = cursor[0] % L
             cursor[0] += 1
-            cache.decode_attention(layer, ids, qs[layer], outs[layer])
+            attend(layer, qs[layer], outs[layer])
 
     def barrier():
         if world > 1:
@@ -514,7 +534,7 @@ def main():
             step()
     bytes_per_step = 0
     for layer in range(lps):                              # algorithmic bytes, from the library's own accounting
-        cache.decode_attention(layer, ids, qs[layer], outs[layer])
+        attend(layer, qs[layer], outs[layer])
         bytes_per_step += cache.stats()["last_decode_bytes"]
     barrier()
     sampler.begin()
@@ -540,7 +560,12 @@ def main():
         for _ in range(lps):
             layer = cursor[0] % L
             cursor[0] += 1
-            cache.decode_attention_host(layer, ids, q_host[layer], out_host[layer], q_stage, out_stage)
+            if QL == 1:
+                cache.decode_attention_host(layer, ids, q_host[layer], out_host[layer], q_stage, out_stage)
+            else:                                         # no host-buffer variant of the multi-query call: copy around it
+                q_stage.copy_(q_host[layer], non_blocking=True)
+                attend(layer, q_stage, out_stage)
+                out_host[layer].copy_(out_stage, non_blocking=True)
         torch.cuda.current_stream().synchronize()        # the caller reads the result on the host
 
     for _ in range(3):
@@ -583,7 +608,7 @@ def main():
             "e2e": {"value": e2e_ms * 1e3, "unit": "us", "h2d_bytes_per_step": qbytes, "d2h_bytes_per_step": qbytes},
             "gpu_launches": lps * args.steps, "clocks": clocks,
         }
-        if not args.no_cpu_baseline and world == 1:
+        if not args.no_cpu_baseline and world == 1 and QL == 1:
             o = oracle_sample(w, rank, 3, args.factor_bits)
             line["cpu_baseline"] = {"value": o["decode_s"] * 1e6 * o["slices_per_step"], "unit": "us",
                                     "cores": o["cores"], "kind": "oracle", "sample": o["sample"],
