@@ -195,6 +195,32 @@ pkv_status pkv_compress_eligible_pages(pkv_cache *c, int32_t layer, int64_t *n_p
                                        void *stream);
 
 /*
+ * The same conversion in two steps, so that the factorization can run on a second stream while the caller's main
+ * stream goes on with other work (the next layer's projections, appends and attention during a chunked prefill).
+ * Not in the paper, which compresses synchronously; the result is the one pkv_compress_eligible_pages() would
+ * give for the same pages.
+ *
+ * pkv_compress_begin(): picks the pages of `layer` (0 <= layer < n_layers) that are eligible now, in ascending
+ * (sequence, page) order, allocates their factor slots, and enqueues the factorization on `side_stream`, ordered
+ * behind everything enqueued on `main_stream` so far (the appends that wrote the pages).  Nothing else changes:
+ * until the commit the pages stay dense pages for every other call - attention keeps reading their rows, appends
+ * and compressions of other layers proceed - and their dense slots stay allocated.
+ *   n_pages_begun [host, may be NULL] pages picked.  PKV_ERR_POOL_EXHAUSTED: the factor pool ran out; the pages
+ *   picked so far are begun and must still be committed.
+ * pkv_compress_commit(): for `layer` (-1 = every layer with a begun compression, ascending) makes `main_stream`
+ * wait for that factorization, then does what pkv_compress_eligible_pages() does per page, in the same order:
+ * the page becomes a factor page, its dense slot is released (so slot reuse stays deterministic: it depends on
+ * the order of calls, never on timing), the page table is updated on `main_stream`.  A layer without a begun
+ * compression is skipped.   n_pages_compressed [host, may be NULL].
+ * Between the two calls, for the layer concerned: pkv_compress_begin and pkv_compress_eligible_pages (also with
+ * layer = -1) return PKV_ERR_UNSUPPORTED, and so does pkv_free_seq for a sequence that has pages in flight.
+ * Neither call can be captured into a CUDA graph.  pkv_destroy_cache waits for factorizations still running.
+ */
+pkv_status pkv_compress_begin(pkv_cache *c, int32_t layer, void *main_stream, void *side_stream,
+                              int64_t *n_pages_begun);
+pkv_status pkv_compress_commit(pkv_cache *c, int32_t layer, void *main_stream, int64_t *n_pages_compressed);
+
+/*
  * Section 3.3 "Attention over Mixed KV Pages", Eq. 4 and Eq. 5: one query per
  * sequence and query head attends over all tokens of that sequence in `layer`.
  *   seq_ids [host] n_seqs distinct ids, each with at least one token in `layer`

@@ -115,6 +115,7 @@ class OracleCache:
         self.sigma = {}      # slot -> (sigma_k [H,P], sigma_v [H,P]) sorted descending
         self.state = {}      # (seq, layer) -> _SeqLayer
         self.pages_compressed = 0
+        self.pending = {}    # layer -> [(seq, page, factor slot, factors, sigma)] begun, not committed
 
     # ------------------------------------------------------------------ append
     def _sl(self, seq, layer):
@@ -170,30 +171,71 @@ class OracleCache:
                     work.append((seq, ly, p))
         if not work:
             return 0
+        factors = self._factorize(work)
+        for (seq, ly, p), (f, sig) in zip(work, factors):
+            fslot = self.factor_free.alloc()
+            self.factor[fslot] = f
+            self.sigma[fslot] = sig
+            self._flip(seq, ly, p, fslot)
+        self.pages_compressed += len(work)
+        return len(work)
+
+    def _factorize(self, work):
+        """Rank-r factors (Eq. 2) of the listed (seq, layer, page) dense pages, every KV head: a list of
+        (dict(A_k, B_k, A_v, B_v), (sigma_k, sigma_v)) in the order of `work`."""
+        c = self.cfg
         Ks = np.stack([self.dense[self.state[(s, ly)].slots[p]][0] for s, ly, p in work])  # [n,H,P,d]
         Vs = np.stack([self.dense[self.state[(s, ly)].slots[p]][1] for s, ly, p in work])
         n, H = Ks.shape[0], c.n_kv_heads
         A_k, B_k, s_k = _svd.page_factors(Ks.reshape(n * H, c.page_size, c.head_dim), c.rank_k)
         A_v, B_v, s_v = _svd.page_factors(Vs.reshape(n * H, c.page_size, c.head_dim), c.rank_v)
-        for i, (seq, ly, p) in enumerate(work):
-            sl = self.state[(seq, ly)]
-            fslot = self.factor_free.alloc()
+        out = []
+        for i in range(n):
             sel = slice(i * H, (i + 1) * H)
-            self.factor[fslot] = dict(A_k=A_k[sel].copy(), B_k=B_k[sel].copy(),
-                                      A_v=A_v[sel].copy(), B_v=B_v[sel].copy())
+            f = dict(A_k=A_k[sel].copy(), B_k=B_k[sel].copy(), A_v=A_v[sel].copy(), B_v=B_v[sel].copy())
             if c.factor_bits == 4:
-                f = self.factor[fslot]
                 for h in range(H):
                     f["A_k"][h], f["B_k"][h], f["A_v"][h], f["B_v"][h] = _quant.quantized_page_factors(
                         f["A_k"][h], f["B_k"][h], f["A_v"][h], f["B_v"][h])
-            self.sigma[fslot] = (s_k[sel].copy(), s_v[sel].copy())
-            dslot = sl.slots[p]
-            del self.dense[dslot]
-            self.dense_free.release(dslot)
-            sl.kinds[p] = FACTOR
-            sl.slots[p] = fslot
-        self.pages_compressed += len(work)
+            out.append((f, (s_k[sel].copy(), s_v[sel].copy())))
+        return out
+
+    def _flip(self, seq, ly, p, fslot):
+        """The page becomes a factor page; its dense slot is released."""
+        sl = self.state[(seq, ly)]
+        dslot = sl.slots[p]
+        del self.dense[dslot]
+        self.dense_free.release(dslot)
+        sl.kinds[p] = FACTOR
+        sl.slots[p] = fslot
+
+    def compress_begin(self, layer):
+        """First half of a two-step compression of one layer (a caller-side arrangement, not in the paper: the
+        factorization may run while other work proceeds).  Picks the pages eligible now, ascending (seq, page),
+        allocates their factor slots and computes their factors; the pages stay dense pages, with their dense
+        slots, until compress_commit().  Returns the number of pages picked."""
+        assert layer not in self.pending, "layer already has an uncommitted compression"
+        c = self.cfg
+        work = [(seq, layer, p) for seq in range(c.max_seqs) for p in self.eligible(seq, layer)]
+        work = work[:len(self.factor_free.order) - self.factor_free.in_use()]      # as many as factor slots are left
+        if not work:
+            return 0
+        self.pending[layer] = [(seq, p, self.factor_free.alloc(), f, sig)
+                               for (seq, _, p), (f, sig) in zip(work, self._factorize(work))]
         return len(work)
+
+    def compress_commit(self, layer=-1):
+        """Second half: per pending page, in the order it was picked, the page becomes a factor page and its
+        dense slot is released.  layer = -1: every layer with a pending compression, ascending."""
+        done = 0
+        for ly in (sorted(self.pending) if layer < 0 else [layer]):
+            for seq, p, fslot, f, sig in self.pending.pop(ly, []):
+                self.factor[fslot] = f
+                self.sigma[fslot] = sig
+                self._flip(seq, ly, p, fslot)
+                done += 1
+        self.pages_compressed += done
+        return done
 
     # ------------------------------------------------------------------ attend
     def gather_kv(self, seq, layer, kv_head):

@@ -49,6 +49,15 @@ struct PlanCache {
     std::vector<PlanSeg> segs;
 };
 
+// Pages whose factorization was started by pkv_compress_begin() and not yet committed: they are still dense pages
+// for every other call (slots, f_end and the device page table are untouched until pkv_compress_commit()).
+struct PendingPage { int32_t seq, page, dense_slot, factor_slot; };
+struct PendingCompress {
+    bool active = false;
+    std::vector<PendingPage> pages;    // ascending (seq, page)
+    cudaEvent_t done = nullptr;        // recorded behind the layer's compression kernels
+};
+
 // Pinned staging ring for host -> device metadata uploads.
 struct Stager {
     static constexpr int kChunks = 32;
@@ -82,6 +91,11 @@ struct pkv_cache {
     int64_t last_decode_bytes = 0, last_decode_units = 0;
     uint64_t decode_seq = 0;           // decode launches so far (decode_overlap = 2: picks the scratch buffer)
     bool cache_written = true;         // an append or compression kernel was enqueued since the last decode launch
+    std::vector<PendingCompress> pending;   // [n_layers]
+    int n_pending = 0;                 // layers with a begun, uncommitted compression
+    cudaEvent_t order_ev = nullptr;    // scratch event: orders a side stream behind the caller's main stream
+    cudaEvent_t worklist_ev = nullptr; // recorded behind the last kernel that reads the device work list
+    bool worklist_busy = false;
 
     SeqLayer &at(int seq, int layer) { return sl[(size_t)seq * cfg.n_layers + layer]; }
     const SeqLayer &at(int seq, int layer) const { return sl[(size_t)seq * cfg.n_layers + layer]; }
@@ -510,6 +524,7 @@ pkv_status pkv_init_cache(const pkv_config *cfg, void *dense_pool, void *factor_
     c->sl.resize((size_t)cfg->max_seqs * cfg->n_layers);
     for (auto &s : c->sl) s.f_end = c->geo.sink_pages;
     c->plans.resize(cfg->n_layers);
+    c->pending.resize(cfg->n_layers);
     c->stamp.assign(cfg->max_seqs, 0);
     if (!dry) {
         cudaError_t e = cudaMemset(c->meta, 0, (size_t)c->ml.total);
@@ -531,6 +546,10 @@ pkv_status pkv_destroy_cache(pkv_cache *c) {
         }
         cudaFreeHost(c->stg.base);
     }
+    for (PendingCompress &pc : c->pending)
+        if (pc.done) { cudaEventSynchronize(pc.done); cudaEventDestroy(pc.done); }
+    if (c->order_ev) cudaEventDestroy(c->order_ev);
+    if (c->worklist_ev) { cudaEventSynchronize(c->worklist_ev); cudaEventDestroy(c->worklist_ev); }
     delete c;
     return PKV_OK;
 }
@@ -602,6 +621,23 @@ pkv_status pkv_append_kv(pkv_cache *c, int32_t layer, int32_t n_seqs, const int3
     return PKV_OK;
 }
 
+// Uploads a work list of (dense slot, factor slot) pairs and launches the compression kernel on it.  The device
+// work list is one buffer: an upload first waits for the last kernel that read it, whatever stream that ran on.
+static pkv_status run_worklist(pkv_cache *c, const std::vector<int2> &work, cudaStream_t st) {
+    int2 *dwl = (int2 *)(c->workspace + c->wl.worklist);
+    if (c->worklist_busy) PKV_CUDA(c, cudaStreamWaitEvent(st, c->worklist_ev, 0));
+    pkv_status rr = upload(c, dwl, work.data(), sizeof(int2) * work.size(), st);
+    if (rr != PKV_OK) return rr;
+    if ((rr = stager_flush(c, st)) != PKV_OK) return rr;
+    c->cache_written = true;
+    PKV_CUDA(c, launch_compress(c->geo, c->dense_pool, c->factor_pool, dwl, (int)work.size(),
+                                (int *)(c->meta + c->ml.status), st));
+    if (!c->worklist_ev) PKV_CUDA(c, cudaEventCreateWithFlags(&c->worklist_ev, cudaEventDisableTiming));
+    PKV_CUDA(c, cudaEventRecord(c->worklist_ev, st));
+    c->worklist_busy = true;
+    return PKV_OK;
+}
+
 pkv_status pkv_compress_eligible_pages(pkv_cache *c, int32_t layer, int64_t *n_pages_compressed,
                                        void *stream) {
     if (!c) return PKV_ERR_INVALID_ARG;
@@ -610,6 +646,8 @@ pkv_status pkv_compress_eligible_pages(pkv_cache *c, int32_t layer, int64_t *n_p
     if (layer < -1 || layer >= c->cfg.n_layers) return fail(c, PKV_ERR_INVALID_ARG, "layer %d out of range", layer);
     if (!c->dry && is_capturing(st))
         return fail(c, PKV_ERR_UNSUPPORTED, "pkv_compress_eligible_pages cannot be captured into a CUDA graph");
+    if (layer < 0 ? c->n_pending > 0 : c->pending[layer].active)
+        return fail(c, PKV_ERR_UNSUPPORTED, "a compression begun with pkv_compress_begin is not committed yet");
     const Geometry &g = c->geo;
     const int l0 = layer < 0 ? 0 : layer, l1 = layer < 0 ? c->cfg.n_layers : layer + 1;
     std::vector<int2> work;
@@ -618,15 +656,9 @@ pkv_status pkv_compress_eligible_pages(pkv_cache *c, int32_t layer, int64_t *n_p
     pkv_status r;
     auto flush_work = [&]() -> pkv_status {
         if (work.empty() || c->dry) { work.clear(); return PKV_OK; }
-        int2 *dwl = (int2 *)(c->workspace + c->wl.worklist);
-        pkv_status rr = upload(c, dwl, work.data(), sizeof(int2) * work.size(), st);
-        if (rr != PKV_OK) return rr;
-        if ((rr = stager_flush(c, st)) != PKV_OK) return rr;
-        c->cache_written = true;
-        PKV_CUDA(c, launch_compress(g, c->dense_pool, c->factor_pool, dwl, (int)work.size(),
-                                    (int *)(c->meta + c->ml.status), st));
+        pkv_status rr = run_worklist(c, work, st);
         work.clear();
-        return PKV_OK;
+        return rr;
     };
     // Page-table uploads of converted pages are queued behind the kernel that reads the dense slots.
     struct Flip { int seq, layer, first, last; };
@@ -675,6 +707,100 @@ pkv_status pkv_compress_eligible_pages(pkv_cache *c, int32_t layer, int64_t *n_p
     c->pages_compressed += done;
     if (n_pages_compressed) *n_pages_compressed = done;
     if (exhausted) return fail(c, PKV_ERR_POOL_EXHAUSTED, "factor pool exhausted after %lld pages", (long long)done);
+    return PKV_OK;
+}
+
+pkv_status pkv_compress_begin(pkv_cache *c, int32_t layer, void *main_stream, void *side_stream,
+                              int64_t *n_pages_begun) {
+    if (!c) return PKV_ERR_INVALID_ARG;
+    cudaStream_t ms = (cudaStream_t)main_stream, ss = (cudaStream_t)side_stream;
+    if (n_pages_begun) *n_pages_begun = 0;
+    if (layer < 0 || layer >= c->cfg.n_layers) return fail(c, PKV_ERR_INVALID_ARG, "layer %d out of range", layer);
+    PendingCompress &pd = c->pending[layer];
+    if (pd.active) return fail(c, PKV_ERR_UNSUPPORTED, "layer %d already has an uncommitted compression", layer);
+    if (!c->dry && (is_capturing(ms) || is_capturing(ss)))
+        return fail(c, PKV_ERR_UNSUPPORTED, "pkv_compress_begin cannot be captured into a CUDA graph");
+    const Geometry &g = c->geo;
+    pd.pages.clear();
+    bool exhausted = false;
+    for (int seq = 0; seq < c->cfg.max_seqs && !exhausted; ++seq) {
+        const SeqLayer &s = c->at(seq, layer);
+        const int hi = std::max(g.sink_pages, s.n_tokens / c->cfg.page_size - g.recent_pages);
+        for (int p = s.f_end; p < hi; ++p) {
+            if (c->factor_free.available() == 0) { exhausted = true; break; }
+            pd.pages.push_back(PendingPage{seq, p, s.slots[p], c->factor_free.alloc()});
+        }
+    }
+    if (n_pages_begun) *n_pages_begun = (int64_t)pd.pages.size();
+    if (!pd.pages.empty()) {
+        pd.active = true;
+        c->n_pending++;
+        if (!c->dry) {
+            // the pages were written by work enqueued on the main stream: the side stream starts behind it
+            if (!c->order_ev) PKV_CUDA(c, cudaEventCreateWithFlags(&c->order_ev, cudaEventDisableTiming));
+            if (!pd.done) PKV_CUDA(c, cudaEventCreateWithFlags(&pd.done, cudaEventDisableTiming));
+            PKV_CUDA(c, cudaEventRecord(c->order_ev, ms));
+            PKV_CUDA(c, cudaStreamWaitEvent(ss, c->order_ev, 0));
+            std::vector<int2> work;
+            pkv_status r;
+            for (size_t i = 0; i < pd.pages.size(); ++i) {
+                work.push_back(make_int2(pd.pages[i].dense_slot, pd.pages[i].factor_slot));
+                if ((int)work.size() == kCompressChunk || i + 1 == pd.pages.size()) {
+                    const bool written = c->cache_written;       // nothing a decode launch reads changes before the commit
+                    r = run_worklist(c, work, ss);
+                    c->cache_written = written;
+                    if (r != PKV_OK) return r;
+                    work.clear();
+                }
+            }
+            PKV_CUDA(c, cudaEventRecord(pd.done, ss));
+        }
+    }
+    if (exhausted)
+        return fail(c, PKV_ERR_POOL_EXHAUSTED, "factor pool exhausted after %lld pages", (long long)pd.pages.size());
+    return PKV_OK;
+}
+
+pkv_status pkv_compress_commit(pkv_cache *c, int32_t layer, void *main_stream, int64_t *n_pages_compressed) {
+    if (!c) return PKV_ERR_INVALID_ARG;
+    cudaStream_t ms = (cudaStream_t)main_stream;
+    if (n_pages_compressed) *n_pages_compressed = 0;
+    if (layer < -1 || layer >= c->cfg.n_layers) return fail(c, PKV_ERR_INVALID_ARG, "layer %d out of range", layer);
+    if (!c->dry && is_capturing(ms))
+        return fail(c, PKV_ERR_UNSUPPORTED, "pkv_compress_commit cannot be captured into a CUDA graph");
+    const int l0 = layer < 0 ? 0 : layer, l1 = layer < 0 ? c->cfg.n_layers : layer + 1;
+    int64_t done = 0;
+    for (int ly = l0; ly < l1; ++ly) {
+        PendingCompress &pd = c->pending[ly];
+        if (!pd.active) continue;
+        if (!c->dry) PKV_CUDA(c, cudaStreamWaitEvent(ms, pd.done, 0));
+        // the same state changes, in the same order, as pkv_compress_eligible_pages makes page by page
+        for (size_t i = 0; i < pd.pages.size();) {
+            const int seq = pd.pages[i].seq;
+            SeqLayer &s = c->at(seq, ly);
+            const int first = pd.pages[i].page;
+            for (; i < pd.pages.size() && pd.pages[i].seq == seq; ++i) {
+                const PendingPage &pp = pd.pages[i];
+                s.slots[pp.page] = pp.factor_slot;
+                c->dense_free.release(pp.dense_slot);
+                s.f_end = pp.page + 1;
+                ++done;
+            }
+            s.version++;
+            if (!c->dry) {
+                pkv_status r = upload(c, dev_page_table_row(c, seq, ly) + first, s.slots.data() + first,
+                                      sizeof(int32_t) * (s.f_end - first), ms);
+                if (r != PKV_OK) return r;
+            }
+        }
+        pd.pages.clear();
+        pd.active = false;
+        c->n_pending--;
+        c->cache_written = true;
+    }
+    if (!c->dry) { pkv_status r = stager_flush(c, ms); if (r != PKV_OK) return r; }
+    c->pages_compressed += done;
+    if (n_pages_compressed) *n_pages_compressed = done;
     return PKV_OK;
 }
 
@@ -904,6 +1030,10 @@ pkv_status pkv_get_stats(pkv_cache *c, pkv_stats *out, void *stream) {
 pkv_status pkv_free_seq(pkv_cache *c, int32_t seq) {
     if (!c) return PKV_ERR_INVALID_ARG;
     if (seq < 0 || seq >= c->cfg.max_seqs) return fail(c, PKV_ERR_BAD_SEQ, "sequence id %d out of range", seq);
+    for (int ly = 0; ly < c->cfg.n_layers && c->n_pending > 0; ++ly)
+        for (const PendingPage &pp : c->pending[ly].pages)
+            if (pp.seq == seq)
+                return fail(c, PKV_ERR_UNSUPPORTED, "sequence %d has pages in an uncommitted compression (layer %d)", seq, ly);
     for (int ly = 0; ly < c->cfg.n_layers; ++ly) {
         SeqLayer &s = c->at(seq, ly);
         for (size_t p = 0; p < s.slots.size(); ++p) {

@@ -29,7 +29,7 @@ EXPORTS = [
     "pkv_decode_attention", "pkv_decode_attention_host", "pkv_get_page_table", "pkv_get_stats",
     "pkv_free_seq", "pkv_destroy_cache", "pkv_last_error", "pkv_read_factors", "pkv_write_factors",
     "pkv_read_dense", "pkv_get_decode_plan", "pkv_decode_attention_static_scratch", "pkv_get_decode_trace",
-    "pkv_decode_attention_multi",
+    "pkv_decode_attention_multi", "pkv_compress_begin", "pkv_compress_commit",
     "pkv_get_rotation_schedule",
 ]
 
@@ -84,6 +84,8 @@ def lib():
         L.pkv_decode_attention.argtypes = [vp, i32, i32, ip, vp, vp, vp, vp]
         L.pkv_decode_attention_static_scratch.argtypes = [vp, i32, i32, ip, vp, vp, vp, vp]
         L.pkv_decode_attention_multi.argtypes = [vp, i32, i32, ip, i32, vp, vp, vp, vp]
+        L.pkv_compress_begin.argtypes = [vp, i32, vp, vp, ctypes.POINTER(i64)]
+        L.pkv_compress_commit.argtypes = [vp, i32, vp, ctypes.POINTER(i64)]
         L.pkv_decode_attention_host.argtypes = [vp, i32, i32, ip, vp, vp, vp, vp, vp]
         L.pkv_get_page_table.argtypes = [vp, i32, i32, ip, ip, ip, ip]
         L.pkv_get_stats.argtypes = [vp, ctypes.POINTER(PkvStats), vp]
@@ -174,6 +176,25 @@ def pkv_compress_eligible_pages(handle, layer=-1, stream=None) -> int:
     n = ctypes.c_int64(0)
     st = lib().pkv_compress_eligible_pages(handle, layer, ctypes.byref(n), _stream(stream))
     _check(handle, st)
+    return int(n.value)
+
+
+def pkv_compress_begin(handle, layer, main_stream=None, side_stream=None) -> int:
+    """Starts factorizing the layer's eligible pages on side_stream; returns how many.  The pages stay dense until
+    pkv_compress_commit.  If the factor pool runs out, PkvError carries the status and `begun` the pages begun."""
+    n = ctypes.c_int64(0)
+    st = lib().pkv_compress_begin(handle, layer, _stream(main_stream), _stream(side_stream), ctypes.byref(n))
+    if st != PKV_OK:
+        msg = lib().pkv_last_error(handle)
+        e = PkvError(st, msg.decode() if msg else "")
+        e.begun = int(n.value)
+        raise e
+    return int(n.value)
+
+
+def pkv_compress_commit(handle, layer=-1, main_stream=None) -> int:
+    n = ctypes.c_int64(0)
+    _check(handle, lib().pkv_compress_commit(handle, layer, _stream(main_stream), ctypes.byref(n)))
     return int(n.value)
 
 
@@ -307,6 +328,12 @@ class Cache:
 
     def compress_eligible_pages(self, layer=-1):
         return pkv_compress_eligible_pages(self.handle, layer, self._st())
+
+    def compress_begin(self, layer, side_stream=None):
+        return pkv_compress_begin(self.handle, layer, self._st(), side_stream)
+
+    def compress_commit(self, layer=-1):
+        return pkv_compress_commit(self.handle, layer, self._st())
 
     def decode_attention(self, layer, seq_ids, q=None, out=None, out_f32=None):
         if out is None and q is not None:

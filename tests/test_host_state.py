@@ -109,6 +109,63 @@ def test_random_schedule_matches_oracle_bit_exact(seed, shape):
         _same_tables(gpu, orc, base)
 
 
+@pytest.mark.parametrize("seed", [1, 2, 3])
+def test_two_step_compression_schedule_matches_oracle_bit_exact(seed):
+    """pkv_compress_begin / pkv_compress_commit interleaved with appends, one-step compressions of other layers and
+    frees: page tables (kinds, slots, token counts) stay bit-equal to the oracle's two-step form after every call;
+    calls that would touch a layer with a begun compression are refused and change nothing."""
+    gpu, orc, base = _pair(seed=seed, n_layers=3, max_seqs=3, n_dense_slots=160, n_factor_slots=120)
+    rng = np.random.default_rng(500 + seed)
+    H, L = base["n_kv_heads"], base["n_layers"]
+    pending = {}                                           # layer -> set of sequences with pages in flight
+    for step in range(90):
+        op = rng.integers(0, 12)
+        layer = int(rng.integers(0, L))
+        if op < 5:
+            seqs = [int(x) for x in rng.choice(base["max_seqs"], size=int(rng.integers(1, 4)), replace=False)]
+            n_new = [int(rng.choice([1, 1, 7, 64, 65, 200])) for _ in seqs]
+            _oracle_append(orc, layer, seqs, n_new, H)
+            gpu.append_kv(layer, seqs, n_new)
+        elif op < 8:
+            if layer in pending:
+                with pytest.raises(pkv.PkvError) as e:
+                    gpu.compress_begin(layer)
+                assert e.value.status == pkv.PKV_ERR_UNSUPPORTED
+            else:
+                before = [orc.page_table(s, layer) for s in range(base["max_seqs"])]
+                n = orc.compress_begin(layer)
+                assert gpu.compress_begin(layer) == n
+                assert before == [orc.page_table(s, layer) for s in range(base["max_seqs"])]     # nothing visible yet
+                if n:
+                    pending[layer] = {seq for seq, *_ in orc.pending[layer]}
+        elif op < 10:
+            which = int(rng.integers(-1, L))
+            assert gpu.compress_commit(which) == orc.compress_commit(which)
+            for ly in ([which] if which >= 0 else list(pending)):
+                pending.pop(ly, None)
+        elif op < 11:
+            which = int(rng.integers(-1, L))
+            if (which < 0 and pending) or which in pending:
+                with pytest.raises(pkv.PkvError) as e:
+                    gpu.compress_eligible_pages(which)
+                assert e.value.status == pkv.PKV_ERR_UNSUPPORTED
+            else:
+                assert gpu.compress_eligible_pages(which) == orc.compress_eligible_pages(which)
+        else:
+            s_ = int(rng.integers(0, base["max_seqs"]))
+            if any(s_ in seqs for seqs in pending.values()):
+                with pytest.raises(pkv.PkvError) as e:
+                    gpu.free_seq(s_)
+                assert e.value.status == pkv.PKV_ERR_UNSUPPORTED
+            else:
+                orc.free_seq(s_)
+                gpu.free_seq(s_)
+        _same_tables(gpu, orc, base)
+    assert gpu.compress_commit() == orc.compress_commit()
+    _same_tables(gpu, orc, base)
+    assert gpu.stats()["pages_compressed"] == orc.pages_compressed > 0
+
+
 def test_incremental_conversion_is_one_page_per_boundary_step():
     gpu, orc, base = _pair(n_layers=1, max_seqs=2, sink_tokens=64, recent_tokens=256)
     gpu.append_kv(0, [0, 1], [8192 // 16, 8192 // 16])

@@ -160,6 +160,50 @@ def test_multi_query_attention_pins():
         c3.decode_attention_multi(0, [1], np.zeros((1, 7, cfg.n_q_heads, cfg.head_dim)))
 
 
+def test_two_step_compression_pins():
+    """compress_begin + compress_commit: back to back it is compress_eligible_pages (tables, factors, free lists);
+    between the two the cache reads as before the begin; pages appended in between do not join the set."""
+    rng = np.random.default_rng(31)
+    cfg = _cfg(n_layers=2, max_seqs=2)
+    k, v = _kv(rng, 90, cfg)
+
+    def fed():
+        c = OracleCache(cfg)
+        c.append_kv(0, [0, 1], [60, 30], k, v)
+        c.append_kv(1, [1], [50], k[:50], v[:50])
+        return c
+    a, b = fed(), fed()
+    n = a.compress_eligible_pages(0)
+    assert b.compress_begin(0) == n == (60 // 8 - 2 - 1)
+    assert b.compress_commit(0) == n and b.pending == {}
+    for s in (0, 1):
+        assert a.page_table(s, 0) == b.page_table(s, 0)
+    assert sorted(a.factor) == sorted(b.factor)
+    for slot in a.factor:
+        for name in ("A_k", "B_k", "A_v", "B_v"):
+            assert np.array_equal(a.factor[slot][name], b.factor[slot][name])
+    assert [a.dense_free.alloc() for _ in range(4)] == [b.dense_free.alloc() for _ in range(4)]
+    assert a.factor_free.alloc() == b.factor_free.alloc()
+    # in between: attention and tables as before the begin; later appends stay out of the begun set
+    c = fed()
+    q = rng.standard_normal((1, cfg.n_q_heads, cfg.head_dim))
+    before, table = c.decode_attention(0, [0], q), c.page_table(0, 0)
+    assert c.compress_begin(0) == n
+    assert np.array_equal(c.decode_attention(0, [0], q), before) and c.page_table(0, 0) == table
+    k2, v2 = _kv(rng, 16, cfg)
+    c.append_kv(0, [0], [16], k2, v2)                          # two more pages become eligible
+    assert len(c.eligible(0, 0)) == n + 2
+    assert c.compress_commit() == n
+    assert sum(kd == FACTOR for kd in c.page_table(0, 0)[0]) == n and len(c.eligible(0, 0)) == 2
+    # the committed factors are those of the pages as they were (complete pages never change)
+    d = fed()
+    d.compress_eligible_pages(0)
+    for p in range(1, 1 + n):
+        fa, fb = c.factor[c.page_table(0, 0)[1][p]], d.factor[d.page_table(0, 0)[1][p]]
+        assert np.array_equal(fa["A_k"], fb["A_k"]) and np.array_equal(fa["B_v"], fb["B_v"])
+    assert c.compress_commit() == 0
+
+
 def test_output_invariant_under_slot_permutation():
     cfg = _cfg()
     rng = np.random.default_rng(3)
