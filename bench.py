@@ -236,6 +236,24 @@ def run_serving(args, w, rank, device, world, rk, local):
     cursor = [0]
     events = []
 
+    side = torch.cuda.Stream() if args.two_step > 0 else None
+    begun_at = [None]
+
+    def compress_step(t):
+        """One-step: factorize what left the window now, on this stream.  Two-step (--two-step K): start it on a side
+        stream and make the pages factor pages K steps later (they stay dense, and readable, meanwhile)."""
+        if side is None:
+            return cache.compress_eligible_pages(0)
+        if begun_at[0] is not None and t - begun_at[0] >= args.two_step:
+            cache.compress_commit(0)
+            begun_at[0] = None
+        n = 0
+        if begun_at[0] is None:
+            n = cache.compress_begin(0, side)
+            if n:
+                begun_at[0] = t
+        return n
+
     def step(record):
         t = cursor[0]
         cursor[0] += 1
@@ -248,7 +266,7 @@ def run_serving(args, w, rank, device, world, rk, local):
         cache.decode_attention(0, ids, qs[t % 8], out)
         if record:
             ev[2].record()
-        n = cache.compress_eligible_pages(0)
+        n = compress_step(t)
         if record:
             ev[3].record()
             events.append((ev, n))
@@ -299,7 +317,7 @@ def run_serving(args, w, rank, device, world, rk, local):
         dv.copy_(hv[t], non_blocking=True)
         cache.append_kv(0, ids, [1] * B, dk, dv)
         cache.decode_attention_host(0, ids, hq[t % 8], hout, q_stage, out_stage)
-        cache.compress_eligible_pages(0)
+        compress_step(t)
         torch.cuda.current_stream().synchronize()
 
     for _ in range(3):
@@ -324,7 +342,9 @@ def run_serving(args, w, rank, device, world, rk, local):
             "metric": "decode_us_per_step", "value": ms * 1e3, "unit": "us", "n_gpus": world, "steps": args.steps,
             "warmup": warm, "ms_per_step": ms, "higher_is_better": False, "scaling": "weak", "vs_baseline": None,
             "dtype": "bf16", "data": "synthetic", "config": dict(_config_dict(args, w, rank),
-                step="append (1 token per sequence) + decode + compress_eligible on one layer", overlap="0"),
+                step="append (1 token per sequence) + decode + compress_eligible on one layer" if args.two_step <= 0 else
+                     "append (1 token per sequence) + decode + compress_commit %d steps after compress_begin on a side stream" % args.two_step,
+                overlap="0"),
             "append_us": {"mean": statistics.mean(app), "p99": pct(app, 0.99)},
             "attention_us": {"mean": statistics.mean(att), "p99": pct(att, 0.99)},
             "compress_us": {"mean_no_event": statistics.mean([us for us, n in cmp_all if n == 0] or [0.0]),
@@ -445,6 +465,9 @@ def main():
     ap.add_argument("--q-len", type=int, default=1,
                     help="queries per sequence and step (1 = decoding; more = a speculative-decoding or chunked-prefill step "
                          "over the newest positions, pkv_decode_attention_multi)")
+    ap.add_argument("--two-step", type=int, default=0,
+                    help="serving loop only: factorize on a side stream (pkv_compress_begin) and commit K steps later, "
+                         "instead of the one-step call inside the step")
     ap.add_argument("--graph", action="store_true",
                     help="replay one CUDA graph per step instead of launching every layer from the host (overlap 0 or 1)")
     args = ap.parse_args()

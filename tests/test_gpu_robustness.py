@@ -220,3 +220,81 @@ def test_mode_2_refuses_stream_capture():
             torch.zeros(4, device="cuda")                    # the capture itself is still alive
     torch.cuda.current_stream().wait_stream(side)
     cache.close()
+
+
+@pytest.mark.parametrize("bits", [16, 4])
+def test_two_step_compression_on_a_side_stream(bits):
+    """A chunked prefill with the factorization on a second stream: per chunk and layer, append the chunk, attend
+    with all the chunk's positions as queries, begin the layer's compression on the side stream, and commit it one
+    chunk later.  Checked: between begin and commit the cache reads as dense (kernel gate against the oracle in
+    the same state); page tables equal the oracle's two-step form after every commit; at the end every factor
+    page holds bit for bit the factors that the one-step call produces on a second cache fed the same tokens, and
+    both caches give the same attention output bit for bit."""
+    L, H, G, P, chunk, n_chunks = 2, 2, 4, 64, 192, 6
+    cfg = pkv.make_config(n_layers=L, n_kv_heads=H, n_q_heads=H * G, rank=16, sink_tokens=P, recent_tokens=4 * P,
+                          max_seqs=2 * (chunk // 2), max_pages_per_seq=32, n_dense_slots=160, n_factor_slots=120,
+                          factor_bits=bits)
+    pair = Pair(cfg, seed=9)
+    sync = pkv.Cache(cfg, "cuda")                      # one-step path, its own slot numbering
+    side = torch.cuda.Stream()
+    seqs = [0, 1]
+    kv = {(ly, s): gen_kv(9, ly, s, chunk * n_chunks, cfg, outlier_prob=0.01) for ly in range(L) for s in seqs}
+    gq = torch.Generator().manual_seed(77)
+    worst = 0.0
+    for ci in range(n_chunks):
+        lo, hi = ci * chunk, (ci + 1) * chunk
+        for ly in range(L):
+            if ci > 0:
+                n = pair.gpu.compress_commit(ly)
+                assert pair.orc.compress_commit(ly) == n
+                pair.same_tables()
+            ks = [kv[(ly, s)][0][lo:hi] for s in seqs]
+            vs = [kv[(ly, s)][1][lo:hi] for s in seqs]
+            pair.append(ly, seqs, ks, vs)
+            sync.append_kv(ly, seqs, [chunk] * 2, torch.cat(ks).cuda(), torch.cat(vs).cuda())
+            q = torch.randn((2, chunk, H * G, 128), generator=gq).to(torch.bfloat16)
+            out32 = torch.empty(q.shape, dtype=torch.float32, device="cuda")
+            out = torch.empty(q.shape, dtype=torch.bfloat16, device="cuda")
+            # begin now, then attend while the side stream factorizes: the attention must still see these pages dense
+            n_b = pair.gpu.compress_begin(ly, side)
+            assert pair.orc.compress_begin(ly) == n_b == (0 if ci == 0 else 2 if ci == 1 else 6)
+            pair.gpu.decode_attention_multi(ly, seqs, chunk, q.cuda(), out, out32)
+            sync.compress_eligible_pages(ly)
+            if ci in (2, n_chunks - 1) and ly == 1:
+                torch.cuda.synchronize()
+                saved = pair.orc.factor
+                pair.orc.factor = dict(saved)
+                for s in seqs:
+                    pair.load_gpu_factors_into_oracle(s, ly)
+                ref = pair.orc.decode_attention_multi(ly, seqs, f64(q))
+                pair.orc.factor = saved
+                got = f64(out32)
+                for i in range(2):
+                    for j in range(0, chunk, 13):
+                        worst = max(worst, rel_err(got[i, j], ref[i, j]))
+                        assert rel_err(got[i, j], ref[i, j]) <= (1e-2 if bits == 4 else 4e-3), (ci, i, j)
+    assert pair.gpu.compress_commit() == pair.orc.compress_commit() > 0
+    pair.same_tables()
+    assert pair.gpu.compress_commit() == 0
+    torch.cuda.synchronize()
+    # logical pages of both caches: same kinds, same bytes
+    for ly in range(L):
+        for s in seqs:
+            ka, sa, Ta = pair.gpu.page_table(s, ly)
+            kb, sb, Tb = sync.page_table(s, ly)
+            assert ka == kb and Ta == Tb and sum(ka) > 0
+            for p, kind in enumerate(ka):
+                if kind == 1:
+                    for h in range(H):
+                        fa, fb = pair.gpu.read_factors(sa[p], h), sync.read_factors(sb[p], h)
+                        assert all(torch.equal(x, y) for x, y in zip(fa, fb)), (ly, s, p, h)
+        q1 = synth.make_q(9, ly, 0, 2, H * G, 128, "cuda")
+        oa, ob = torch.empty_like(q1), torch.empty_like(q1)
+        pair.gpu.decode_attention(ly, seqs, q1, oa)
+        sync.decode_attention(ly, seqs, q1, ob)
+        torch.cuda.synchronize()
+        assert torch.equal(oa, ob)
+    st = pair.gpu.stats()
+    assert st["device_timeouts"] == 0 and st["page_svds_not_converged"] == 0 and st["bad_slot_indices"] == 0
+    print("two-step compression bits=%d: kernel gate max %.2e, %d pages" % (bits, worst, st["pages_compressed"]))
+    sync.close()
