@@ -434,7 +434,8 @@ def _config_dict(args, w, rank):
                         "a draining launch every 63); valid here because queries are prepared in advance and no "
                         "launch in the step writes the cache"][args.overlap],
             "launch": "one CUDA graph replay per step (%d per-layer launches)" % w.get("layers_per_step", w["n_layers"]) if args.graph else "host launch per layer",
-            "parallelism": "replicas x%d" % args.gpus}
+            "parallelism": ("sequence-sharded x%d (per layer: local softmax states, all-gather, Eq. 5 merge)" % args.gpus
+                            if getattr(args, "seq_sharded", False) else "replicas x%d" % args.gpus)}
 
 
 def max_over_ranks(values, world, device="cpu"):
@@ -468,6 +469,10 @@ def main():
     ap.add_argument("--two-step", type=int, default=0,
                     help="serving loop only: factorize on a side stream (pkv_compress_begin) and commit K steps later, "
                          "instead of the one-step call inside the step")
+    ap.add_argument("--seq-sharded", action="store_true",
+                    help="strong scaling of one step: every rank's cache holds 1/N of each sequence's tokens (rank 0 the "
+                         "sink, the last rank the dense window); per layer each rank computes its softmax state, the states "
+                         "are all-gathered (NCCL) and merged by Eq. 5.  Not the default: the driver's scaling runs are replicas")
     ap.add_argument("--graph", action="store_true",
                     help="replay one CUDA graph per step instead of launching every layer from the host (overlap 0 or 1)")
     args = ap.parse_args()
@@ -498,6 +503,10 @@ def main():
         if world > 1:
             dist.destroy_process_group()
         return
+    if args.seq_sharded:
+        if w["ragged"] or w.get("serving") or args.q_len != 1 or args.graph or w["T"] % (64 * world):
+            raise SystemExit("--seq-sharded needs a uniform, non-serving workload whose context divides into whole pages per rank")
+        w = dict(w, T=w["T"] // world, sink=w["sink"] if rk == 0 else 0, recent=w["recent"] if rk == world - 1 else 0)
     QL = args.q_len
     per_tile = max(1, min(QL, 8 // (w["n_q_heads"] // w["n_kv_heads"])))
     cfg, cache, lengths, comp = build_workload(w, rank, device, args.overlap, args.n_ctas, args.factor_bits,
@@ -512,8 +521,15 @@ def main():
         qs = [synth.make_q(SEED, layer, 0, w["batch"] * QL, Hq, 128, device).view(w["batch"], QL, Hq, 128) for layer in range(L)]
     outs = [torch.empty_like(q) for q in qs]
 
+    if args.seq_sharded:
+        from paper_2608_23843_b200 import sharded
+        sh_state = [torch.empty((w["batch"], Hq, 130), dtype=torch.float32, device=device) for _ in range(L)]
+        sh_all = [torch.empty((world, w["batch"], Hq, 130), dtype=torch.float32, device=device) for _ in range(L)]
+
     def attend(layer, q, out):
-        if QL == 1:
+        if args.seq_sharded:
+            sharded.sequence_sharded_decode(cache, layer, ids, q, out, state=sh_state[layer], gathered=sh_all[layer])
+        elif QL == 1:
             cache.decode_attention(layer, ids, q, out)
         else:
             cache.decode_attention_multi(layer, ids, QL, q, out)
@@ -583,7 +599,7 @@ def main():
         for _ in range(lps):
             layer = cursor[0] % L
             cursor[0] += 1
-            if QL == 1:
+            if QL == 1 and not args.seq_sharded:
                 cache.decode_attention_host(layer, ids, q_host[layer], out_host[layer], q_stage, out_stage)
             else:                                         # no host-buffer variant of the multi-query call: copy around it
                 q_stage.copy_(q_host[layer], non_blocking=True)
@@ -615,7 +631,8 @@ def main():
         qbytes = sum(q.numel() * 2 for q in qs[:lps])
         line = {
             "metric": "decode_us_per_step", "value": ms * 1e3, "unit": "us", "n_gpus": world, "steps": args.steps,
-            "warmup": max(3, args.warmup), "ms_per_step": ms, "higher_is_better": False, "scaling": "weak",
+            "warmup": max(3, args.warmup), "ms_per_step": ms, "higher_is_better": False,
+            "scaling": "strong" if args.seq_sharded else "weak",
             "vs_baseline": None, "dtype": "bf16", "data": "synthetic", "config": _config_dict(args, w, rank),
             "hbm_gbs": bytes_per_step / (ms * 1e-3) / 1e9 * world,
             "frac_of_8tbs": bytes_per_step / (ms * 1e-3) / 8e12,
@@ -629,7 +646,7 @@ def main():
                                            "scaled by algorithmic bytes", "launch_us": launch_ms * 1e3,
                          "algorithmic_bytes_per_launch": bytes_per_launch},
             "e2e": {"value": e2e_ms * 1e3, "unit": "us", "h2d_bytes_per_step": qbytes, "d2h_bytes_per_step": qbytes},
-            "gpu_launches": lps * args.steps, "clocks": clocks,
+            "gpu_launches": lps * args.steps * (2 if args.seq_sharded else 1), "clocks": clocks,
         }
         if not args.no_cpu_baseline and world == 1 and QL == 1:
             o = oracle_sample(w, rank, 3, args.factor_bits)

@@ -263,6 +263,29 @@ pkv_status pkv_decode_attention_multi(pkv_cache *c, int32_t layer, int32_t n_seq
                                       int32_t q_len, const void *q, void *out, float *out_f32, void *stream);
 
 /*
+ * One sequence spread over several caches (sequence sharding: each cache, e.g. one per GPU, holds a contiguous
+ * range of the sequence's tokens with its own pages and factors).  Eq. 5 merges per-page softmax states; the same
+ * rule merges per-cache states, so each cache returns its state instead of a normalised output and one more
+ * application of Eq. 5 gives the attention over all tokens.  The paper runs on one GPU; this is the exchange step
+ * its page-wise formulation allows.
+ *
+ * pkv_decode_attention_partial(): as pkv_decode_attention(), but writes
+ *   state [device] fp32 [n_seqs, H_q, d + 2]: per query head o (d values, not divided by l), then m, then l, where
+ *   with s_t = (q . k_t) * softmax_scale * log2(e) over this cache's tokens: m = max_t s_t, l = sum_t 2^(s_t - m),
+ *   o = sum_t 2^(s_t - m) v_t  (factor pages contribute through their factors as in Eq. 4).
+ * pkv_merge_attention_states(): Eq. 5 over n_shards such arrays stored back to back,
+ *   states [device] fp32 [n_shards, n_rows, d + 2] (n_rows = n_seqs * H_q; e.g. the result of an all-gather),
+ *   out [device, may be NULL] bf16 [n_rows, d];  out_f32 [device, may be NULL] fp32 [n_rows, d]; not both NULL.
+ * Shards are summed in index order, so every holder of the same gathered array computes the same bits.  Needs no
+ * cache handle; returns PKV_ERR_INVALID_ARG for NULL / misaligned pointers (states and out 8 bytes, out_f32 16),
+ * PKV_ERR_CUDA if the launch fails.
+ */
+pkv_status pkv_decode_attention_partial(pkv_cache *c, int32_t layer, int32_t n_seqs, const int32_t *seq_ids,
+                                        const void *q, float *state, void *stream);
+pkv_status pkv_merge_attention_states(const float *states, int32_t n_shards, int64_t n_rows, void *out,
+                                      float *out_f32, void *stream);
+
+/*
  * The same call for callers whose queries and results live in host memory.
  *   q_host, out_host [host] bf16 [n_seqs, H_q, d];  q_stage, out_stage [device]
  *   caller-owned staging buffers of the same size.

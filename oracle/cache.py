@@ -302,6 +302,24 @@ class OracleCache:
                         out[i, j, h] = _att.attention_plain(q[i, j, h], K_all[:visible], V_all[:visible], self.scale)
         return out
 
+    def attention_state(self, layer, seq_ids, q):
+        """The softmax state of this cache's tokens for each query (the quantities Eq. 5 merges), for a sequence
+        whose tokens are spread over several caches: m [n, H_q] = max_t s_t with s_t = q . k_t * scale (natural
+        units), l [n, H_q] = sum_t exp(s_t - m), o [n, H_q, d] = sum_t exp(s_t - m) v_t.  Factor pages enter as A B.
+        Merging the states of all caches with attention.merge_page_states gives Eq. 1 over all tokens."""
+        c = self.cfg
+        q = np.asarray(q, dtype=np.float64)
+        G = c.n_q_heads // c.n_kv_heads
+        n = len(seq_ids)
+        m, l, o = np.zeros((n, c.n_q_heads)), np.zeros((n, c.n_q_heads)), np.zeros((n, c.n_q_heads, c.head_dim))
+        for i, seq in enumerate(seq_ids):
+            for kvh in range(c.n_kv_heads):
+                K_all, V_all = self.gather_kv(int(seq), layer, kvh)
+                for g in range(G):
+                    h = kvh * G + g
+                    m[i, h], l[i, h], o[i, h] = _att.page_state_dense(q[i, h], K_all, V_all, self.scale)
+        return m, l, o
+
     def decode_attention_pagewise(self, layer, seq_ids, q):
         """Same result through Eq. 4 (factor pages evaluated from factors, never
         materialised) and Eq. 5 (merge).  Used to check the algebra only."""

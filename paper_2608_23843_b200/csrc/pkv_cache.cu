@@ -804,13 +804,38 @@ pkv_status pkv_compress_commit(pkv_cache *c, int32_t layer, void *main_stream, i
     return PKV_OK;
 }
 
+static pkv_status decode_impl(pkv_cache *c, int32_t layer, int32_t n_seqs, const int32_t *seq_ids, int32_t q_len,
+                              const void *q, void *out, float *out_f32, float *state, void *stream);
+
 pkv_status pkv_decode_attention(pkv_cache *c, int32_t layer, int32_t n_seqs, const int32_t *seq_ids,
                                 const void *q, void *out, float *out_f32, void *stream) {
-    return pkv_decode_attention_multi(c, layer, n_seqs, seq_ids, 1, q, out, out_f32, stream);
+    return decode_impl(c, layer, n_seqs, seq_ids, 1, q, out, out_f32, nullptr, stream);
 }
 
 pkv_status pkv_decode_attention_multi(pkv_cache *c, int32_t layer, int32_t n_seqs, const int32_t *seq_ids,
                                       int32_t q_len, const void *q, void *out, float *out_f32, void *stream) {
+    return decode_impl(c, layer, n_seqs, seq_ids, q_len, q, out, out_f32, nullptr, stream);
+}
+
+pkv_status pkv_decode_attention_partial(pkv_cache *c, int32_t layer, int32_t n_seqs, const int32_t *seq_ids,
+                                        const void *q, float *state, void *stream) {
+    if (!c) return PKV_ERR_INVALID_ARG;
+    if (c->cfg.decode_variant != 0)
+        return fail(c, PKV_ERR_UNSUPPORTED, "pkv_decode_attention_partial needs the tensor-core kernel (decode_variant 0)");
+    if (!c->dry && !state) return fail(c, PKV_ERR_INVALID_ARG, "state is NULL");
+    return decode_impl(c, layer, n_seqs, seq_ids, 1, q, nullptr, nullptr, state, stream);
+}
+
+pkv_status pkv_merge_attention_states(const float *states, int32_t n_shards, int64_t n_rows, void *out, float *out_f32,
+                                      void *stream) {
+    if (!states || n_shards < 1 || n_rows < 0 || (!out && !out_f32)) return PKV_ERR_INVALID_ARG;
+    if (((uintptr_t)states & 7) || ((uintptr_t)out & 7) || ((uintptr_t)out_f32 & 15)) return PKV_ERR_INVALID_ARG;
+    return launch_merge_states(states, n_shards, n_rows, out, out_f32, (cudaStream_t)stream) == cudaSuccess
+               ? PKV_OK : PKV_ERR_CUDA;
+}
+
+static pkv_status decode_impl(pkv_cache *c, int32_t layer, int32_t n_seqs, const int32_t *seq_ids, int32_t q_len,
+                              const void *q, void *out, float *out_f32, float *state, void *stream) {
     if (!c) return PKV_ERR_INVALID_ARG;
     cudaStream_t st = (cudaStream_t)stream;
     if (layer < 0 || layer >= c->cfg.n_layers) return fail(c, PKV_ERR_INVALID_ARG, "layer %d out of range", layer);
@@ -836,7 +861,7 @@ pkv_status pkv_decode_attention_multi(pkv_cache *c, int32_t layer, int32_t n_seq
                             s.f_end > c->geo.sink_pages ? s.f_end * c->cfg.page_size : 0);
         }
     }
-    if (!c->dry && (!q || !out)) return fail(c, PKV_ERR_INVALID_ARG, "q or out is NULL");
+    if (!c->dry && (!q || (!out && !state))) return fail(c, PKV_ERR_INVALID_ARG, "q or out is NULL");
     if (!plan_is_current(c, layer, n_seqs, seq_ids, q_len)) {
         // the plan is uploaded through the staging ring: a copy recorded into a graph would replay stale bytes
         if (!c->dry && is_capturing(st))
@@ -867,6 +892,7 @@ pkv_status pkv_decode_attention_multi(pkv_cache *c, int32_t layer, int32_t n_seq
     a.plan_cta = c->ml.plan_cta; a.plan_entry = c->ml.plan_entry; a.plan_seg = c->ml.plan_seg;
     a.plan_cta_entry = c->ml.plan_cta_entry;
     a.q = q; a.out = out; a.out_f32 = out_f32;
+    a.state = state;
     a.q_len = q_len;
     a.q_tpt = queries_per_tile(c->geo, q_len);
     a.q_nblk = entries_per_seq(c->geo, q_len);
@@ -925,6 +951,7 @@ pkv_status pkv_decode_attention_static_scratch(pkv_cache *c, int32_t layer, int3
     a.plan_cta = c->ml.plan_cta; a.plan_entry = c->ml.plan_entry; a.plan_seg = c->ml.plan_seg;
     a.plan_cta_entry = c->ml.plan_cta_entry;
     a.q = q; a.out = out; a.out_f32 = out_f32;
+    a.state = nullptr;
     a.q_len = 1; a.q_tpt = 1; a.q_nblk = 1; a.q_cols = c->geo.group;
     a.partials = nullptr; a.tickets = nullptr;            // set by the launcher from the static scratch
     a.plain_launch = 0;                                   // the launcher's memset already orders it after earlier work

@@ -713,9 +713,19 @@ __device__ __forceinline__ int load_q(const DecodeArgs &a, int seg, uint32_t (&q
 }
 
 // Writes the final result of one (entry, KV head) for query column hq, dims d4..d4+3.
-__device__ __forceinline__ void store_out(const DecodeArgs &a, int seg, int hq, int d4, float4 acc, float L) {
+// With a.state set the call returns the softmax state instead (Eq. 5's inputs, for a merge across caches that
+// hold different token ranges of the sequence): row = o[0..d) unnormalised, then m (the running maximum of the
+// scaled scores in base-2 units, i.e. of s * softmax_scale * log2 e), then l.
+__device__ __forceinline__ void store_out(const DecodeArgs &a, int seg, int hq, int d4, float4 acc, float M, float L) {
     const long long row = q_row(a, seg, hq);
     if (row < 0) return;
+    if (a.state) {
+        float *st = a.state + row * (kHeadDim + 2);
+        *reinterpret_cast<float2 *>(st + d4) = make_float2(acc.x, acc.y);     // rows are 8-byte aligned only
+        *reinterpret_cast<float2 *>(st + d4 + 2) = make_float2(acc.z, acc.w);
+        if (d4 == 0) { st[kHeadDim] = M; st[kHeadDim + 1] = L; }
+        return;
+    }
     const float inv = 1.f / L;
     acc.x *= inv; acc.y *= inv; acc.z *= inv; acc.w *= inv;
     const long long off = row * kHeadDim + d4;
@@ -777,7 +787,7 @@ __device__ __forceinline__ void merge_parts(const DecodeArgs &a, const float *fi
     }
 #pragma unroll
     for (int e = 0; e < E; ++e)
-        if (has[e]) store_out(a, seg, hq[e], d4, tot[e], Lr[e]);
+        if (has[e]) store_out(a, seg, hq[e], d4, tot[e], Mr[e], Lr[e]);
 }
 
 #define PKV_CONSUMER_BARRIER() asm volatile("bar.sync 1, %0;" ::"n"(kConsumerWarps * 32) : "memory")
@@ -831,7 +841,7 @@ __device__ __forceinline__ void flush_segment(const DecodeArgs &a, float *comb, 
             L += f * cw[kMaxGroup * kHeadDim + kMaxGroup + hq];
         }
         if (ps.n_parts <= 1) {
-            if (hq < a.q_cols) store_out(a, seg, hq, d4, acc, L);
+            if (hq < a.q_cols) store_out(a, seg, hq, d4, acc, M, L);
         } else {
             *reinterpret_cast<float4 *>(part + hq * kHeadDim + d4) = acc;
             if ((item & 31) == 0) {
@@ -1124,6 +1134,46 @@ cudaError_t launch_decode(const DecodeArgs &a, int n_segs, cudaStream_t st) {
     }
     if (e != cudaSuccess || a.variant != 1) return e;
     merge_kernel<<<n_segs, 256, 0, st>>>(a);
+    return cudaGetLastError();
+}
+
+// Eq. 5 across caches: states [n_shards][n_rows][d + 2] as written by store_out; one warp per row.
+__global__ void __launch_bounds__(128) merge_states_kernel(const float *states, int n_shards, long long n_rows,
+                                                           __nv_bfloat16 *out, float *out_f32) {
+    const long long row = (long long)blockIdx.x * 4 + (threadIdx.x >> 5);
+    if (row >= n_rows) return;
+    const int d4 = (threadIdx.x & 31) * 4;
+    const long long stride = n_rows * (kHeadDim + 2);
+    const float *base = states + row * (kHeadDim + 2);
+    float M = kNegInf;
+    for (int k = 0; k < n_shards; ++k) M = fmaxf(M, base[k * stride + kHeadDim]);
+    float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
+    float L = 0.f;
+    for (int k = 0; k < n_shards; ++k) {                    // shard order: the result does not depend on who merges
+        const float *pk = base + k * stride;
+        const float w = exp2f(pk[kHeadDim] - M);
+        const float2 a0 = *reinterpret_cast<const float2 *>(pk + d4), a1 = *reinterpret_cast<const float2 *>(pk + d4 + 2);
+        acc.x += w * a0.x; acc.y += w * a0.y; acc.z += w * a1.x; acc.w += w * a1.y;
+        L += w * pk[kHeadDim + 1];
+    }
+    const float inv = 1.f / L;
+    acc.x *= inv; acc.y *= inv; acc.z *= inv; acc.w *= inv;
+    const long long off = row * kHeadDim + d4;
+    if (out) {
+        __nv_bfloat162 lo = __floats2bfloat162_rn(acc.x, acc.y), hi = __floats2bfloat162_rn(acc.z, acc.w);
+        uint2 packed;
+        packed.x = *reinterpret_cast<unsigned *>(&lo);
+        packed.y = *reinterpret_cast<unsigned *>(&hi);
+        *reinterpret_cast<uint2 *>(out + off) = packed;
+    }
+    if (out_f32) *reinterpret_cast<float4 *>(out_f32 + off) = acc;
+}
+
+cudaError_t launch_merge_states(const float *states, int n_shards, long long n_rows, void *out, float *out_f32,
+                                cudaStream_t st) {
+    if (n_rows <= 0) return cudaSuccess;
+    merge_states_kernel<<<(unsigned)((n_rows + 3) / 4), 128, 0, st>>>(states, n_shards, n_rows,
+                                                                      reinterpret_cast<__nv_bfloat16 *>(out), out_f32);
     return cudaGetLastError();
 }
 

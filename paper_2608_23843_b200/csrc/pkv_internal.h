@@ -96,6 +96,7 @@ struct DecodeArgs {
     const void *q;
     void *out;
     float *out_f32;
+    float *state;                      // not NULL: write (o unnormalised, m, l) rows of d + 2 floats instead of out / out_f32
     float *partials;
     int *tickets;                      // one per segment, zero between launches
 
@@ -120,6 +121,8 @@ cudaError_t launch_append(const Geometry &geo, unsigned char *dense_pool, const 
 cudaError_t launch_compress(const Geometry &geo, const unsigned char *dense_pool, unsigned char *factor_pool,
                             const int2 *worklist, int n_entries, int *status, cudaStream_t st);
 cudaError_t launch_decode(const DecodeArgs &a, int n_segs, cudaStream_t st);
+cudaError_t launch_merge_states(const float *states, int n_shards, long long n_rows, void *out, float *out_f32,
+                                cudaStream_t st);
 cudaError_t launch_decode_static_scratch(const DecodeArgs &a, int n_segs, cudaStream_t st, const char **why);
 cudaError_t launch_read_factors(const Geometry &geo, const unsigned char *blob, void *A_k, void *B_k,
                                 void *A_v, void *B_v, cudaStream_t st);

@@ -30,6 +30,7 @@ EXPORTS = [
     "pkv_free_seq", "pkv_destroy_cache", "pkv_last_error", "pkv_read_factors", "pkv_write_factors",
     "pkv_read_dense", "pkv_get_decode_plan", "pkv_decode_attention_static_scratch", "pkv_get_decode_trace",
     "pkv_decode_attention_multi", "pkv_compress_begin", "pkv_compress_commit",
+    "pkv_decode_attention_partial", "pkv_merge_attention_states",
     "pkv_get_rotation_schedule",
 ]
 
@@ -85,6 +86,8 @@ def lib():
         L.pkv_decode_attention_static_scratch.argtypes = [vp, i32, i32, ip, vp, vp, vp, vp]
         L.pkv_decode_attention_multi.argtypes = [vp, i32, i32, ip, i32, vp, vp, vp, vp]
         L.pkv_compress_begin.argtypes = [vp, i32, vp, vp, ctypes.POINTER(i64)]
+        L.pkv_decode_attention_partial.argtypes = [vp, i32, i32, ip, vp, vp, vp]
+        L.pkv_merge_attention_states.argtypes = [vp, i32, i64, vp, vp, vp]
         L.pkv_compress_commit.argtypes = [vp, i32, vp, ctypes.POINTER(i64)]
         L.pkv_decode_attention_host.argtypes = [vp, i32, i32, ip, vp, vp, vp, vp, vp]
         L.pkv_get_page_table.argtypes = [vp, i32, i32, ip, ip, ip, ip]
@@ -208,6 +211,19 @@ def pkv_decode_attention_multi(handle, layer, seq_ids, q_len, q, out, out_f32=No
     ids, n = _ints(seq_ids)
     _check(handle, lib().pkv_decode_attention_multi(handle, layer, n, ids, q_len, _ptr(q), _ptr(out), _ptr(out_f32),
                                                     _stream(stream)))
+
+
+def pkv_decode_attention_partial(handle, layer, seq_ids, q, state, stream=None):
+    """state: fp32 [n_seqs, H_q, d + 2] = (o unnormalised, m in base-2 units, l) over this cache's tokens."""
+    ids, n = _ints(seq_ids)
+    _check(handle, lib().pkv_decode_attention_partial(handle, layer, n, ids, _ptr(q), _ptr(state), _stream(stream)))
+
+
+def pkv_merge_attention_states(states, n_shards, n_rows, out=None, out_f32=None, stream=None):
+    """Eq. 5 over n_shards state arrays stored back to back ([n_shards, n_rows, d + 2] fp32)."""
+    st = lib().pkv_merge_attention_states(_ptr(states), n_shards, n_rows, _ptr(out), _ptr(out_f32), _stream(stream))
+    if st != PKV_OK:
+        raise PkvError(st, "pkv_merge_attention_states")
 
 
 def pkv_decode_attention_static_scratch(handle, layer, seq_ids, q, out, out_f32=None, stream=None):
@@ -346,6 +362,12 @@ class Cache:
             out = torch.empty_like(q)
         pkv_decode_attention_multi(self.handle, layer, seq_ids, q_len, q, out, out_f32, self._st())
         return out
+
+    def decode_attention_partial(self, layer, seq_ids, q, state=None):
+        if state is None:
+            state = torch.empty((q.shape[0], q.shape[1], q.shape[2] + 2), dtype=torch.float32, device=q.device)
+        pkv_decode_attention_partial(self.handle, layer, seq_ids, q, state, self._st())
+        return state
 
     def decode_attention_host(self, layer, seq_ids, q_host, out_host, q_stage, out_stage):
         pkv_decode_attention_host(self.handle, layer, seq_ids, q_host, out_host, q_stage, out_stage, self._st())

@@ -43,3 +43,42 @@ def test_reference_arm_under_torchrun_prints_once():
     assert d["impl"] == "reference" and d["n_gpus"] == 2 and d["unit"] == "us" and d["higher_is_better"] is False
     assert d["cpu_baseline"]["kind"] == "oracle" and d["e2e"]["h2d_bytes_per_step"] == 0
     assert d["config"]["workload"] == "tiny" and d["value"] > 0
+
+
+def _shard_worker(rank, world, port, out):
+    """Each rank owns a token range of one sequence, computes its softmax state with the oracle, and gathers the
+    states with the package's helper (gloo, CPU tensors)."""
+    os.environ.update(MASTER_ADDR="127.0.0.1", MASTER_PORT=str(port), RANK=str(rank), WORLD_SIZE=str(world))
+    sys.path.insert(0, ROOT)
+    import numpy as np
+    from oracle import attention as att
+    from paper_2608_23843_b200 import sharded
+    dist.init_process_group("gloo", rank=rank, world_size=world)
+    rng = np.random.default_rng(7)                        # the same stream on both ranks
+    T, d, Hq = 90, 128, 4
+    K, V, q = rng.standard_normal((T, d)), rng.standard_normal((T, d)), rng.standard_normal((1, Hq, d))
+    lo, hi = (0, 53) if rank == 0 else (53, T)
+    state = torch.zeros((1, Hq, d + 2), dtype=torch.float64)
+    for h in range(Hq):
+        m, l, o = att.page_state_dense(q[0, h], K[lo:hi], V[lo:hi], d ** -0.5)
+        state[0, h, :d] = torch.from_numpy(o)
+        state[0, h, d], state[0, h, d + 1] = m, l
+    gathered = sharded.gather_states(state)
+    dist.barrier()
+    dist.destroy_process_group()
+    merged = []
+    for h in range(Hq):
+        sts = [(float(gathered[r, 0, h, d]), float(gathered[r, 0, h, d + 1]), gathered[r, 0, h, :d].numpy()) for r in range(world)]
+        merged.append(att.merge_page_states(sts))
+    ref = [att.attention_plain(q[0, h], K, V, d ** -0.5) for h in range(Hq)]
+    out[rank] = (tuple(gathered.shape), float(max(np.abs(a - b).max() for a, b in zip(merged, ref))),
+                 float(gathered[rank, 0, 0, d + 1] - state[0, 0, d + 1]))
+
+
+def test_gathered_shard_states_merge_to_full_attention_gloo_world2():
+    mgr = mp.Manager()
+    out = mgr.dict()
+    mp.spawn(_shard_worker, args=(2, 29613, out), nprocs=2, join=True)
+    for rank in (0, 1):
+        shape, err, own = out[rank]
+        assert shape == (2, 1, 4, 130) and err <= 1e-13 and own == 0.0     # slot `rank` of the result is the rank's own state

@@ -551,3 +551,74 @@ def test_multi_query_attention(P, rk, rv, G, q_len, bits):
     st = pair.gpu.stats()
     assert st["device_timeouts"] == 0 and st["bad_slot_indices"] == 0
     print("multi-query P=%d r=(%d,%d) G=%d q_len=%d bits=%d: kernel max %.2e e2e max %.2e" % (P, rk, rv, G, q_len, bits, worst_k, worst_e))
+
+
+@pytest.mark.parametrize("bits", [16, 4])
+def test_sequence_sharded_attention_states(bits):
+    """Sequences split over three caches on one GPU (token ranges; the first keeps the sink, the middle one
+    compresses every complete page, the last keeps the window): each cache's state from
+    pkv_decode_attention_partial against the oracle's state of the same cache (normalised output and
+    log-sum-exp), and the Eq. 5 merge of the three (pkv_merge_attention_states) against the oracle's attention
+    over all tokens - kernel gate, the oracle reading the GPU's stored factors."""
+    import math
+    from oracle import attention as att
+    H, G, P = 2, 4, 64
+    splits = {0: (1500, 2100, 777), 1: (64, 1, 130), 2: (70, 640, 5)}     # tokens per (sequence, shard)
+    shard_cfg = [dict(sink_tokens=P, recent_tokens=0), dict(sink_tokens=0, recent_tokens=0),
+                 dict(sink_tokens=0, recent_tokens=2 * P)]
+    pairs = []
+    for r, kw in enumerate(shard_cfg):
+        cfg = pkv.make_config(n_layers=1, n_kv_heads=H, n_q_heads=H * G, rank=24, max_seqs=3, max_pages_per_seq=40,
+                              n_dense_slots=80, n_factor_slots=80, factor_bits=bits, **kw)
+        pair = Pair(cfg, seed=20 + r)
+        for s, lens in splits.items():
+            k, v = gen_kv(6, 0, 10 * s + r, lens[r], cfg, outlier_prob=0.02)
+            pair.append(0, [s], [k], [v])
+        pair.compress(0)
+        pair.same_tables()
+        pairs.append(pair)
+    assert sum(pairs[1].gpu.page_table(0, 0)[0]) == 2100 // P
+    order = [2, 0, 1]
+    q = synth.make_q(6, 0, 0, 3, H * G, 128)
+    qd = q.cuda()
+    states = torch.empty((3, 3, H * G, 130), dtype=torch.float32, device="cuda")
+    ref_states = []
+    for r, pair in enumerate(pairs):
+        pair.gpu.decode_attention_partial(0, order, qd, states[r])
+        for s in order:
+            pair.load_gpu_factors_into_oracle(s, 0)
+        ref_states.append(pair.orc.attention_state(0, order, f64(q)))
+    out = torch.empty_like(qd)
+    out32 = torch.empty(qd.shape, dtype=torch.float32, device="cuda")
+    pkv.pkv_merge_attention_states(states, 3, 3 * H * G, out, out32, torch.cuda.current_stream())
+    only32 = torch.empty_like(out32)
+    pkv.pkv_merge_attention_states(states, 3, 3 * H * G, None, only32, torch.cuda.current_stream())
+    torch.cuda.synchronize()
+    got_states, got, got32 = f64(states), f64(out), f64(out32)
+    assert torch.equal(only32, out32)
+    worst = worst_lse = 0.0
+    tol32 = 1e-2 if bits == 4 else 8e-3                # tiny shards (1 and 5 tokens): nothing averages the bf16 rounding of p
+    for i in range(3):
+        for h in range(H * G):
+            merged = att.merge_page_states([(m[i, h], l[i, h], o[i, h]) for m, l, o in ref_states])
+            scale = np.abs(merged).max()
+            worst = max(worst, np.abs(got32[i, h] - merged).max() / scale)
+            assert np.abs(got[i, h] - merged).max() <= 1.2e-2 * scale
+            for r in range(3):
+                m, l, o = ref_states[r]
+                st = got_states[r, i, h]
+                lse = st[128] * math.log(2.0) + math.log(st[129])
+                worst_lse = max(worst_lse, abs(lse - (m[i, h] + math.log(l[i, h]))))
+                ref_o = o[i, h] / l[i, h]
+                assert np.abs(st[:128] / st[129] - ref_o).max() <= tol32 * np.abs(ref_o).max(), (r, i, h)
+    assert worst <= tol32 and worst_lse <= 2e-2
+    # a single shard merged with itself alone is the ordinary call, bit for bit
+    single = torch.empty_like(qd)
+    pairs[0].gpu.decode_attention(0, order, qd, single)
+    alone = torch.empty_like(qd)
+    pkv.pkv_merge_attention_states(states[0], 1, 3 * H * G, alone, None, torch.cuda.current_stream())
+    torch.cuda.synchronize()
+    assert torch.equal(single, alone)
+    with pytest.raises(pkv.PkvError):
+        pkv.pkv_merge_attention_states(states, 0, 3 * H * G, out, None, torch.cuda.current_stream())
+    print("sharded states bits=%d: merged kernel gate max %.2e, log-sum-exp max abs %.2e" % (bits, worst, worst_lse))

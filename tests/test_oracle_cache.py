@@ -204,6 +204,35 @@ def test_two_step_compression_pins():
     assert c.compress_commit() == 0
 
 
+def test_states_of_token_ranges_merge_to_attention_over_all_tokens():
+    """A sequence split over three caches (first with the sink, middle all compressed, last with the window): the
+    per-cache states merged by Eq. 5 equal Eq. 1 over the concatenated (partly reconstructed) tokens, and each
+    state on its own normalises to that cache's attention with the expected log-sum-exp."""
+    rng = np.random.default_rng(41)
+    parts = [(_cfg(sink_tokens=8, recent_tokens=0), 50), (_cfg(sink_tokens=0, recent_tokens=0), 41),
+             (_cfg(sink_tokens=0, recent_tokens=16), 37)]
+    caches, Ks, Vs = [], [], []
+    for cfg, T in parts:
+        c = OracleCache(cfg)
+        k, v = _kv(rng, T, cfg)
+        c.append_kv(0, [1], [T], k, v)
+        assert c.compress_eligible_pages() > 0
+        caches.append(c)
+    cfg = parts[0][0]
+    q = rng.standard_normal((1, cfg.n_q_heads, cfg.head_dim))
+    states = [c.attention_state(0, [1], q) for c in caches]
+    for h in range(cfg.n_q_heads):
+        K = np.concatenate([c.gather_kv(1, 0, h // 2)[0] for c in caches])
+        V = np.concatenate([c.gather_kv(1, 0, h // 2)[1] for c in caches])
+        assert K.shape[0] == 50 + 41 + 37
+        merged = att.merge_page_states([(m[0, h], l[0, h], o[0, h]) for m, l, o in states])
+        assert np.abs(merged - att.attention_plain(q[0, h], K, V, 0.25)).max() <= 1e-13
+        for c, (m, l, o) in zip(caches, states):
+            assert np.abs(o[0, h] / l[0, h] - c.decode_attention(0, [1], q)[0, h]).max() <= 1e-13
+            s = c.gather_kv(1, 0, h // 2)[0] @ q[0, h] * 0.25
+            assert abs(m[0, h] + np.log(l[0, h]) - np.log(np.exp(s).sum())) <= 1e-12
+
+
 def test_output_invariant_under_slot_permutation():
     cfg = _cfg()
     rng = np.random.default_rng(3)
