@@ -504,7 +504,7 @@ def main():
             dist.destroy_process_group()
         return
     if args.seq_sharded:
-        if w["ragged"] or w.get("serving") or args.q_len != 1 or args.graph or w["T"] % (64 * world):
+        if w["ragged"] or w.get("serving") or args.q_len != 1 or args.graph or w["T"] % (w.get("page", 64) * world):
             raise SystemExit("--seq-sharded needs a uniform, non-serving workload whose context divides into whole pages per rank")
         w = dict(w, T=w["T"] // world, sink=w["sink"] if rk == 0 else 0, recent=w["recent"] if rk == world - 1 else 0)
     QL = args.q_len

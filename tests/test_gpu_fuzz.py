@@ -116,3 +116,110 @@ def test_random_schedules(seed):
         st = pair.gpu.stats()
         assert st["device_timeouts"] == 0 and st["bad_slot_indices"] == 0, (what, st)
         pair.gpu.close()
+
+
+@pytest.mark.parametrize("seed", [1, 2])
+def test_random_schedules_with_two_step_compression_multi_query_and_states(seed):
+    """The schedule test again with the other entry points mixed in: compression either in one step or begun on a
+    side stream and committed some steps later; attention either for one query per sequence, for the q_len newest
+    positions (kernel gate against the oracle's causal form), or as a softmax state that, merged alone, must
+    reproduce the ordinary call bit for bit.  Page tables bit-exact after every step."""
+    import torch
+    from gpu_helpers import f64, rel_err
+    rng = random.Random(3000 + seed)
+    side = torch.cuda.Stream()
+    for case in range(4):
+        P = rng.choice([16, 32, 64])
+        L, H, G, nseq = rng.choice([1, 2]), rng.choice([1, 2]), rng.choice([1, 2, 4, 8]), rng.choice([2, 3])
+        rk = min(P, rng.choice([8, 16, 24]) if P >= 32 else rng.choice([8, 16]))
+        t_max = 14 * P
+        cfg = pkv.make_config(n_layers=L, n_kv_heads=H, n_q_heads=H * G, rank=rk, page_size=P,
+                              sink_tokens=P * rng.choice([0, 1]), recent_tokens=P * rng.choice([1, 2]), max_seqs=nseq * 6,
+                              max_pages_per_seq=t_max // P + 2, n_dense_slots=L * nseq * 12 + 8,
+                              n_factor_slots=L * nseq * (t_max // P + 2), n_ctas=rng.choice([0, 5, 148]),
+                              decode_overlap=rng.choice([0, 1, 2]), factor_bits=rng.choice([16, 16, 4]))
+        what = (seed, case, P, L, H, G, nseq, rk, cfg.n_ctas, cfg.decode_overlap, cfg.factor_bits)
+        pair = Pair(cfg, seed=case)
+        data = {(ly, s): gen_kv(300 + case, ly, s, t_max, cfg) for ly in range(L) for s in range(nseq)}
+        T = [0] * nseq
+        begun = {}                                         # layer -> (step begun, sequences with pages in flight)
+        for step in range(40):
+            ids = [s for s in range(nseq) if rng.random() < 0.7]
+            n_new = [min(rng.choice([1, 1, 1, 2, 5, P, P + 3]), t_max - T[s]) for s in ids]
+            ids, n_new = [s for s, n in zip(ids, n_new) if n > 0], [n for n in n_new if n > 0]
+            if ids:
+                for ly in range(L):
+                    pair.append(ly, ids, [data[(ly, s)][0][T[s]:T[s] + n] for s, n in zip(ids, n_new)],
+                                [data[(ly, s)][1][T[s]:T[s] + n] for s, n in zip(ids, n_new)])
+                for s, n in zip(ids, n_new):
+                    T[s] += n
+            for ly in list(begun):
+                if step - begun[ly][0] >= 2 and rng.random() < 0.6:
+                    assert pair.gpu.compress_commit(ly) == pair.orc.compress_commit(ly) > 0
+                    del begun[ly]
+            ly = rng.randrange(L)
+            r = rng.random()
+            if r < 0.35 and ly not in begun:
+                n = pair.gpu.compress_begin(ly, side)
+                assert pair.orc.compress_begin(ly) == n
+                if n:
+                    begun[ly] = (step, {s_ for s_, *_ in pair.orc.pending[ly]})
+            elif r < 0.6 and ly not in begun:
+                pair.compress(ly)
+            if rng.random() < 0.06:
+                s = rng.randrange(nseq)
+                if not any(s in seqs for _, seqs in begun.values()):
+                    pair.gpu.free_seq(s)
+                    pair.orc.free_seq(s)
+                    T[s] = 0
+            live = [s for s in range(nseq) if T[s] > 0]
+            if live and rng.random() < 0.8:
+                ly = rng.randrange(L)
+                rng.shuffle(live)
+                mode = rng.choice(["one", "multi", "state"])
+                if mode == "multi":
+                    q_len = rng.choice([2, 3, 5, 8 // G + 1])
+
+                    def fits(s):
+                        kinds = pair.gpu.page_table(s, ly)[0]
+                        f_end = max([p + 1 for p, kd in enumerate(kinds) if kd == 1], default=0)
+                        return q_len <= T[s] and f_end * P <= T[s] - q_len + 1
+                    batch = [s for s in live if fits(s)]
+                    per_tile = max(1, min(q_len, 8 // G))
+                    if batch and len(batch) * -(-q_len // per_tile) <= cfg.max_seqs:
+                        g = torch.Generator().manual_seed(step * 17 + case)
+                        q = torch.randn((len(batch), q_len, H * G, 128), generator=g).to(torch.bfloat16)
+                        out32 = torch.empty(q.shape, dtype=torch.float32, device="cuda")
+                        pair.gpu.decode_attention_multi(ly, batch, q_len, q.cuda(), None, out32)
+                        torch.cuda.synchronize()
+                        saved = pair.orc.factor
+                        pair.orc.factor = dict(saved)
+                        for s in batch:
+                            pair.load_gpu_factors_into_oracle(s, ly)
+                        ref = pair.orc.decode_attention_multi(ly, batch, f64(q))
+                        pair.orc.factor = saved
+                        got = f64(out32)
+                        assert not np.isnan(got).any(), (what, step)
+                        for i in range(len(batch)):
+                            for j in range(q_len):
+                                assert rel_err(got[i, j], ref[i, j]) <= 8e-3, (what, step, i, j)
+                else:
+                    q = synth.make_q(300 + case, ly, step, len(live), H * G, 128)
+                    got, got32 = pair.decode(ly, live, q)
+                    assert not np.isnan(got32).any(), (what, step)
+                    if mode == "one":
+                        g = attention_gates(pair, ly, live, q, got, got32)
+                        assert max(g["kernel"]) <= 8e-3 and max(g["kernel_bf16"]) <= 1.2e-2, (what, step, g["kernel"])
+                    else:
+                        qd = q.cuda()
+                        state = pair.gpu.decode_attention_partial(ly, live, qd)
+                        alone = torch.empty_like(qd)
+                        pkv.pkv_merge_attention_states(state, 1, len(live) * H * G, alone, None, torch.cuda.current_stream())
+                        torch.cuda.synchronize()
+                        assert np.array_equal(f64(alone), got), (what, step)
+            pair.same_tables()
+        assert pair.gpu.compress_commit() == pair.orc.compress_commit()
+        pair.same_tables()
+        st = pair.gpu.stats()
+        assert st["device_timeouts"] == 0 and st["bad_slot_indices"] == 0, (what, st)
+        pair.gpu.close()
