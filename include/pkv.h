@@ -10,6 +10,16 @@
  * evaluates factor pages straight from the factors and merges all pages with an
  * online softmax; historical K/V is never rebuilt.
  *
+ * Entry points: the paper's path is pkv_init_cache, pkv_append_kv,
+ * pkv_compress_eligible_pages, pkv_decode_attention.  Around it: the same attention
+ * for several new positions per sequence (pkv_decode_attention_multi), from host
+ * buffers (pkv_decode_attention_host), without a workspace
+ * (pkv_decode_attention_static_scratch), as a softmax state for sequences sharded
+ * over caches (pkv_decode_attention_partial, pkv_merge_attention_states); the
+ * compression in two steps on a side stream (pkv_compress_begin,
+ * pkv_compress_commit); inspection and test access (pkv_get_*, pkv_read_*,
+ * pkv_write_factors).
+ *
  * Conventions
  *  - Every function returns a pkv_status (0 = PKV_OK, negative = error).  No
  *    exception or abort crosses this boundary.  pkv_last_error() gives a
@@ -23,7 +33,8 @@
  *    [host] are ordinary host addresses.  bf16 = IEEE bfloat16 bit pattern.
  *  - All device work is enqueued on the `stream` argument (a cudaStream_t passed
  *    as void*); calls are asynchronous unless stated.  Operations on one cache
- *    must be issued on one stream (or the caller orders the streams).
+ *    must be issued on one stream (or the caller orders the streams); the one
+ *    exception is pkv_compress_begin(), which takes a second stream by design.
  *  - One cache object is not thread-safe; use one host thread per cache.
  *  - Supported shapes: head_dim = 128; page_size 16, 32 or 64; 1 <= rank_k,
  *    rank_v <= min(32, page_size) with ceil(rank_k / 8) == ceil(rank_v / 8)
@@ -54,7 +65,7 @@ typedef int32_t pkv_status;
 #define PKV_ERR_BAD_SEQ         (-3)  /* sequence id outside [0, max_seqs) or repeated within one call */
 #define PKV_ERR_CUDA            (-4)  /* a CUDA runtime call failed; message holds cudaGetErrorString */
 #define PKV_ERR_NOT_CONVERGED   (-5)  /* reported by pkv_get_stats users: some page hit the Jacobi sweep cap (factors still written) */
-#define PKV_ERR_UNSUPPORTED     (-6)  /* shape outside the supported set; or a call that cannot be recorded while its stream is capturing a CUDA graph */
+#define PKV_ERR_UNSUPPORTED     (-6)  /* shape outside the supported set; a call that cannot be recorded while its stream is capturing a CUDA graph; or a call that would interfere with a compression begun and not yet committed */
 #define PKV_ERR_DEVICE_TIMEOUT  (-7)  /* a bounded in-kernel wait gave up (seen via pkv_get_stats); results of that call are invalid */
 
 #define PKV_KIND_DENSE  0
