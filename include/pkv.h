@@ -88,8 +88,9 @@ typedef struct pkv_config {
     int32_t jacobi_max_sweeps;  /* 0 => default (16) */
     float   jacobi_tol;         /* 0 => default; rotation skipped when |g_pq| <= tol*sqrt(g_pp*g_qq) */
     int32_t n_ctas;             /* decode grid size; 0 => SM count of the current device (148 in dry-run), doubled unless decode_overlap */
-    int32_t decode_variant;     /* 0 = tensor-core pipeline kernel (the product path); 1 = scalar fp32 kernel that
-                                   evaluates the same equations one unit at a time, kept as a debugging reference */
+    int32_t decode_variant;     /* 0 = tensor-core kernels (the product path); 1 = scalar fp32 kernel that evaluates
+                                   the same equations one unit at a time, kept as a debugging reference; 2 = as 0 but
+                                   pkv_decode_attention_multi never uses its row-block kernel (for comparisons) */
     float   jacobi_energy_tol;  /* the sweeps also stop once the energy captured by the r largest diagonal entries
                                    (= ||A^T X||_F^2 of the factors they would give) has grown, since the previous
                                    check, by less than this fraction of the energy left outside them (= the squared
@@ -265,9 +266,12 @@ pkv_status pkv_decode_attention(pkv_cache *c, int32_t layer, int32_t n_seqs, con
  * sequence has a factor page that reaches past token T - q_len (so every query sees every factor page whole:
  * holds whenever q_len <= recent_tokens and compression ran no later than the append of these positions, and it is
  * checked per call); n_seqs * ceil(q_len / max(1, 8 / (H_q / H_kv))) <= max_seqs, the number of plan entries.
- * Cost: queries are processed in blocks of 8 / (H_q / H_kv) tokens, and every block walks the sequence's pages
- * again, so the KV bytes read grow with the number of blocks, not with q_len.
- * Needs decode_variant 0 (PKV_ERR_UNSUPPORTED otherwise).  CUDA-graph and overlap semantics as for
+ * Two kernels serve this call.  With q_len * (H_q / H_kv) >= 64 query rows per KV head and bf16 factors, a
+ * row-block kernel runs: one CTA per (sequence, KV head, 64 rows) reads the sequence's pages once for its 64 rows
+ * (tensor-core products with the query rows as the 16-row operand); the limit on n_seqs above does not apply
+ * then.  Otherwise the decode kernel takes 8 / (H_q / H_kv) query tokens per pass over the pages, so the KV bytes
+ * read grow with the number of such passes.
+ * Needs decode_variant 0 or 2 (PKV_ERR_UNSUPPORTED with 1).  CUDA-graph and overlap semantics as for
  * pkv_decode_attention(); the plan is kept per (layer, batch, q_len).
  */
 pkv_status pkv_decode_attention_multi(pkv_cache *c, int32_t layer, int32_t n_seqs, const int32_t *seq_ids,

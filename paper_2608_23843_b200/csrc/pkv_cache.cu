@@ -139,7 +139,7 @@ pkv_status validate(const pkv_config *cfg, const char **why) {
         *why = "sink_tokens and recent_tokens must be non-negative multiples of page_size"; return PKV_ERR_INVALID_ARG;
     }
     if (cfg->softmax_scale < 0.f || cfg->jacobi_max_sweeps < 0 || cfg->jacobi_tol < 0.f || cfg->n_ctas < 0 ||
-        cfg->decode_variant < 0 || cfg->decode_variant > 1 ||
+        cfg->decode_variant < 0 || cfg->decode_variant > 2 ||
         cfg->decode_overlap < 0 || cfg->decode_overlap > 2 ||
         (cfg->factor_bits != 0 && cfg->factor_bits != 4 && cfg->factor_bits != 16)) {
         *why = "negative scale / sweep cap / tolerance / n_ctas, or unknown decode_variant / decode_overlap / factor_bits"; return PKV_ERR_INVALID_ARG;
@@ -349,12 +349,24 @@ int entries_per_seq(const Geometry &g, int q_len) { const int t = queries_per_ti
 
 // `n_listed` sequences with q_len queries each: every sequence takes entries_per_seq() consecutive plan entries
 // (one per block of query tokens), each of which walks all the sequence's pages.
+// Whether a call with q_len queries for each of n_seqs sequences goes to the row-block kernel (one CTA per 64 query
+// rows of a KV head, which walks the whole sequence alone) instead of the pipeline kernel (eight query columns per
+// pass over the pages, split over all CTAs).  The row-block kernel needs enough CTAs to fill the GPU; below that the
+// pipeline kernel is used if its plan entries fit.
+bool uses_row_blocks(const pkv_cache *c, int q_len, int n_seqs) {
+    const long long rows = (long long)q_len * c->geo.group;
+    if (q_len <= 1 || c->cfg.decode_variant != 0 || c->geo.factor_bits == 4 || rows < kRowBlock) return false;
+    const long long n_ctas = (long long)n_seqs * c->geo.n_kv_heads * ((rows + kRowBlock - 1) / kRowBlock);
+    return n_ctas >= 128 || (long long)n_seqs * entries_per_seq(c->geo, q_len) > c->cfg.max_seqs;
+}
+
 pkv_status build_plan(pkv_cache *c, int layer, int n_listed, const int32_t *seq_ids, int q_len, cudaStream_t st) {
     const Geometry &g = c->geo;
     PlanCache &pc = c->plans[layer];
     const int H = g.n_kv_heads, N = g.n_ctas;
     const long long cf = g.blob_bytes + 2048, cd = (long long)g.block_tokens * 2 * kRowBytes + 2048;
-    const int per_seq = entries_per_seq(g, q_len), n_seqs = n_listed * per_seq;
+    // the row-block kernel only reads the entries (one per listed sequence); the split over CTAs is not used
+    const int per_seq = uses_row_blocks(c, q_len, n_listed) ? 1 : entries_per_seq(g, q_len), n_seqs = n_listed * per_seq;
 
     std::vector<PlanEntry> entries(n_seqs);
     std::vector<HeadShape> shapes(n_seqs);
@@ -820,7 +832,7 @@ pkv_status pkv_decode_attention_multi(pkv_cache *c, int32_t layer, int32_t n_seq
 pkv_status pkv_decode_attention_partial(pkv_cache *c, int32_t layer, int32_t n_seqs, const int32_t *seq_ids,
                                         const void *q, float *state, void *stream) {
     if (!c) return PKV_ERR_INVALID_ARG;
-    if (c->cfg.decode_variant != 0)
+    if (c->cfg.decode_variant == 1)
         return fail(c, PKV_ERR_UNSUPPORTED, "pkv_decode_attention_partial needs the tensor-core kernel (decode_variant 0)");
     if (!c->dry && !state) return fail(c, PKV_ERR_INVALID_ARG, "state is NULL");
     return decode_impl(c, layer, n_seqs, seq_ids, 1, q, nullptr, nullptr, state, stream);
@@ -846,9 +858,9 @@ static pkv_status decode_impl(pkv_cache *c, int32_t layer, int32_t n_seqs, const
             return fail(c, PKV_ERR_INVALID_ARG, "sequence %d has no tokens in layer %d", seq_ids[i], layer);
     if (q_len < 1 || q_len > 32767) return fail(c, PKV_ERR_INVALID_ARG, "q_len %d out of range", q_len);
     if (q_len > 1) {
-        if (c->cfg.decode_variant != 0)
-            return fail(c, PKV_ERR_UNSUPPORTED, "several queries per sequence need the tensor-core kernel (decode_variant 0)");
-        if ((long long)n_seqs * entries_per_seq(c->geo, q_len) > c->cfg.max_seqs)
+        if (c->cfg.decode_variant == 1)
+            return fail(c, PKV_ERR_UNSUPPORTED, "several queries per sequence need the tensor-core kernels (decode_variant 0)");
+        if (!uses_row_blocks(c, q_len, n_seqs) && (long long)n_seqs * entries_per_seq(c->geo, q_len) > c->cfg.max_seqs)
             return fail(c, PKV_ERR_INVALID_ARG, "%d sequences x %d query blocks exceed max_seqs = %d plan entries", n_seqs,
                         entries_per_seq(c->geo, q_len), c->cfg.max_seqs);
         for (int i = 0; i < n_seqs; ++i) {
@@ -906,7 +918,17 @@ static pkv_status decode_impl(pkv_cache *c, int32_t layer, int32_t n_seqs, const
     // launched the ordinary way, after everything before it on the stream has finished
     a.plain_launch = c->cache_written ? 1 : 0;
     c->cache_written = false;
-    if (c->cfg.decode_overlap == 2 && c->cfg.decode_variant == 0) {
+    if (uses_row_blocks(c, q_len, n_seqs)) {
+        // one ordinary launch (starts after everything before it on the stream); no split-K scratch involved
+        a.partials = nullptr; a.tickets = nullptr;
+        a.status = (int *)(c->meta + c->ml.status);
+        a.layer = layer;
+        a.variant = 0; a.overlap = 0; a.plain_launch = 1; a.trace = nullptr;
+        c->cache_written = false;
+        PKV_CUDA(c, launch_decode_blocks(a, n_seqs, st));
+        return PKV_OK;
+    }
+    if (c->cfg.decode_overlap == 2 && c->cfg.decode_variant != 1) {
         cudaStreamCaptureStatus cap = cudaStreamCaptureStatusNone;
         PKV_CUDA(c, cudaStreamIsCapturing(st, &cap));
         if (cap != cudaStreamCaptureStatusNone)

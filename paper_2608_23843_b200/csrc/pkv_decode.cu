@@ -298,6 +298,12 @@ __device__ __forceinline__ void bulk_g2s(uint32_t dst, const void *src, uint32_t
     asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes.L2::cache_hint [%0], [%1], %2, [%3], %4;"
                  ::"r"(dst), "l"(src), "r"(bytes), "r"(bar), "l"(policy) : "memory");
 }
+// The row-block kernel reads a sequence's pages once per block of 64 query rows: there the copies leave the
+// lines in L2 for the other blocks.
+__device__ __forceinline__ void bulk_g2s_keep(uint32_t dst, const void *src, uint32_t bytes, uint32_t bar) {
+    asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];"
+                 ::"r"(dst), "l"(src), "r"(bytes), "r"(bar) : "memory");
+}
 __device__ __forceinline__ void ldsm_x4(uint32_t (&r)[4], uint32_t addr) {
     asm volatile("ldmatrix.sync.aligned.m8n8.x4.shared.b16 {%0,%1,%2,%3}, [%4];"
                  : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]) : "r"(addr));
@@ -1080,6 +1086,413 @@ __global__ void __launch_bounds__(kDecodeThreads, 2) decode_tc_kernel(const __gr
     }
 }
 
+// =============================================================================
+// Row-block kernel: many queries per sequence (a chunk of a prefill).
+//
+// The pipeline kernel above keeps queries in the 8-wide column operand, which suits G <= 8 query heads of one
+// token.  With q_len * G >= 64 query rows per (sequence, KV head) the roles are swapped: 16 (query token, query
+// head) rows are the row operand of every product, a warp owns 16 rows, a CTA 64, and all four warps read each
+// unit from the same shared-memory stage, so the sequence's pages are fetched once per 64 rows instead of once
+// per 8 columns.  The tile loads are the very ones of factor_unit / dense_unit (the storage swizzles serve both
+// roles); only which operand they feed changes.  One CTA handles one (sequence, KV head, block of 64 rows)
+// from the first unit to the last, so there is no split-K state to merge.
+// =============================================================================
+constexpr int kBlockWarps = 4;
+constexpr int kBlockRows = 16 * kBlockWarps;
+constexpr int kBlockThreads = (kBlockWarps + 1) * 32;
+
+// Running state of rows g and g + 8 (g = lane >> 2) of a warp's 16 rows.
+struct RowState {
+    float o[16][4];       // o[c]: (row g, channels 8c+2t, +1), (row g+8, same channels);  t = lane & 3
+    float m[2], l[2];     // l is this lane's share of the row sum; summed over t at the end
+};
+
+// Softmax over NS score tiles of 8 tokens for rows g, g+8; returns p as the row operand of the next product:
+// pa[i] = k-step over tokens 16i .. 16i+15.
+template <int NS>
+__device__ __forceinline__ void row_softmax(float (&s)[NS][4], RowState &st, uint32_t (&pa)[NS / 2][4]) {
+    float mx0 = kNegInf, mx1 = kNegInf;
+#pragma unroll
+    for (int b = 0; b < NS; ++b) {
+        mx0 = fmaxf(mx0, fmaxf(s[b][0], s[b][1]));
+        mx1 = fmaxf(mx1, fmaxf(s[b][2], s[b][3]));
+    }
+#pragma unroll
+    for (int off = 1; off <= 2; off <<= 1) {
+        mx0 = fmaxf(mx0, __shfl_xor_sync(0xffffffffu, mx0, off));
+        mx1 = fmaxf(mx1, __shfl_xor_sync(0xffffffffu, mx1, off));
+    }
+    const float mn0 = fmaxf(st.m[0], mx0), mn1 = fmaxf(st.m[1], mx1);
+    const float al0 = exp2f(st.m[0] - mn0), al1 = exp2f(st.m[1] - mn1);
+    st.m[0] = mn0; st.m[1] = mn1;
+    float sum0 = 0.f, sum1 = 0.f;
+#pragma unroll
+    for (int b = 0; b < NS; ++b) {
+        s[b][0] = exp2f(s[b][0] - mn0); s[b][1] = exp2f(s[b][1] - mn0);
+        s[b][2] = exp2f(s[b][2] - mn1); s[b][3] = exp2f(s[b][3] - mn1);
+        sum0 += s[b][0] + s[b][1];
+        sum1 += s[b][2] + s[b][3];
+    }
+    st.l[0] = st.l[0] * al0 + sum0;
+    st.l[1] = st.l[1] * al1 + sum1;
+    if (__any_sync(0xffffffffu, al0 != 1.f || al1 != 1.f)) {
+#pragma unroll
+        for (int c = 0; c < 16; ++c) { st.o[c][0] *= al0; st.o[c][1] *= al0; st.o[c][2] *= al1; st.o[c][3] *= al1; }
+    }
+#pragma unroll
+    for (int i = 0; i < NS / 2; ++i) {
+        pa[i][0] = pack_bf16(s[2 * i][0], s[2 * i][1]);
+        pa[i][1] = pack_bf16(s[2 * i][2], s[2 * i][3]);
+        pa[i][2] = pack_bf16(s[2 * i + 1][0], s[2 * i + 1][1]);
+        pa[i][3] = pack_bf16(s[2 * i + 1][2], s[2 * i + 1][3]);
+    }
+}
+
+// One factor page for 16 query rows (Eq. 4 with the queries as rows): q~ = q B_k^T, s = q~ A_k^T, p = softmax
+// numerators, w = p A_v, o += w B_v.  qf[kk] = the row operand of q for channels 16kk .. 16kk+15.
+template <int P, int NT>
+__device__ __forceinline__ void block_factor_unit(uint32_t sb, int ak, int bk, int av, int bv, int rk, int rv,
+                                                  const uint32_t (&qf)[8][4], float scale, RowState &st, int lane) {
+    using C = Tc<P, NT>;
+    constexpr int NS = P / 8;
+    const int l7 = lane & 7, mi = lane >> 3, t2 = (lane & 3) * 2;
+    const int asw = a_swz<P>(l7);
+    // ---- q~ [16][r] = q [16][d] . B_k^T, scaled, split into two bf16 terms ----
+    uint32_t qh[NT][2], ql[NT][2];                  // per rank tile: rows g, g+8
+    {
+        float qt[NT][4];
+#pragma unroll
+        for (int j = 0; j < NT; ++j) qt[j][0] = qt[j][1] = qt[j][2] = qt[j][3] = 0.f;
+#pragma unroll
+        for (int qd = 0; qd < 4; ++qd) {
+            uint32_t b[NT][4];
+#pragma unroll
+            for (int j = 0; j < NT; ++j) ldsm_x4(b[j], sb + bk + (8 * j + l7) * kRowBytes + (((4 * qd + mi) ^ l7) << 4));
+#pragma unroll
+            for (int j = 0; j < NT; ++j)
+                mma16816(qt[j], qf[2 * qd][0], qf[2 * qd][1], qf[2 * qd][2], qf[2 * qd][3], b[j][0], b[j][1]);
+#pragma unroll
+            for (int j = 0; j < NT; ++j)
+                mma16816(qt[j], qf[2 * qd + 1][0], qf[2 * qd + 1][1], qf[2 * qd + 1][2], qf[2 * qd + 1][3], b[j][2], b[j][3]);
+        }
+#pragma unroll
+        for (int j = 0; j < NT; ++j) {
+            const bool v0 = 8 * j + t2 < rk, v1 = 8 * j + t2 + 1 < rk;
+            const float x0 = v0 ? qt[j][0] * scale : 0.f, x1 = v1 ? qt[j][1] * scale : 0.f;
+            const float y0 = v0 ? qt[j][2] * scale : 0.f, y1 = v1 ? qt[j][3] * scale : 0.f;
+            qh[j][0] = pack_bf16(x0, x1);
+            qh[j][1] = pack_bf16(y0, y1);
+            ql[j][0] = pack_bf16(x0 - bf16lo_f(qh[j][0]), x1 - bf16hi_f(qh[j][0]));
+            ql[j][1] = pack_bf16(y0 - bf16lo_f(qh[j][1]), y1 - bf16hi_f(qh[j][1]));
+        }
+    }
+    // ---- s [16][P] = q~ . A_k^T   (A_k^T rows = ranks: transposed tile loads give the column operand) ----
+    float s[NS][4];
+#pragma unroll
+    for (int b = 0; b < NS; ++b) s[b][0] = s[b][1] = s[b][2] = s[b][3] = 0.f;
+#pragma unroll
+    for (int kk = 0; kk < NT / 2; ++kk) {
+#pragma unroll
+        for (int i = 0; i < C::kMT; ++i) {
+            uint32_t a4[4];       // (ranks lo, tokens 16i..), (ranks lo, tokens 16i+8..), (ranks hi, 16i..), (ranks hi, 16i+8..)
+            ldsm_x4_t(a4, sb + ak + (16 * kk + (mi >> 1) * 8 + l7) * C::kPitchA + (((2 * i + (mi & 1)) ^ asw) << 4));
+            mma16816(s[2 * i], qh[2 * kk][0], qh[2 * kk][1], qh[2 * kk + 1][0], qh[2 * kk + 1][1], a4[0], a4[2]);
+            mma16816(s[2 * i + 1], qh[2 * kk][0], qh[2 * kk][1], qh[2 * kk + 1][0], qh[2 * kk + 1][1], a4[1], a4[3]);
+            mma16816(s[2 * i], ql[2 * kk][0], ql[2 * kk][1], ql[2 * kk + 1][0], ql[2 * kk + 1][1], a4[0], a4[2]);
+            mma16816(s[2 * i + 1], ql[2 * kk][0], ql[2 * kk][1], ql[2 * kk + 1][0], ql[2 * kk + 1][1], a4[1], a4[3]);
+        }
+    }
+    if (NT % 2) {
+#pragma unroll
+        for (int i = 0; i < C::kMT; ++i) {
+            uint32_t a2[2];
+            ldsm_x2_t(a2, sb + ak + (8 * (NT - 1) + l7) * C::kPitchA + (((2 * i + (mi & 1)) ^ asw) << 4));
+            mma1688(s[2 * i], qh[NT - 1][0], qh[NT - 1][1], a2[0]);
+            mma1688(s[2 * i + 1], qh[NT - 1][0], qh[NT - 1][1], a2[1]);
+            mma1688(s[2 * i], ql[NT - 1][0], ql[NT - 1][1], a2[0]);
+            mma1688(s[2 * i + 1], ql[NT - 1][0], ql[NT - 1][1], a2[1]);
+        }
+    }
+    uint32_t pa[NS / 2][4];
+    row_softmax<NS>(s, st, pa);
+    // ---- w [16][r] = p [16][P] . A_v ----
+    uint32_t wa[NT][2];
+    {
+        float wt[NT][4];
+#pragma unroll
+        for (int j = 0; j < NT; ++j) wt[j][0] = wt[j][1] = wt[j][2] = wt[j][3] = 0.f;
+#pragma unroll
+        for (int qd = 0; qd < C::kMT / 2; ++qd) {
+            uint32_t b[NT][4];
+#pragma unroll
+            for (int j = 0; j < NT; ++j) ldsm_x4(b[j], sb + av + (8 * j + l7) * C::kPitchA + (((4 * qd + mi) ^ asw) << 4));
+#pragma unroll
+            for (int j = 0; j < NT; ++j) mma16816(wt[j], pa[2 * qd][0], pa[2 * qd][1], pa[2 * qd][2], pa[2 * qd][3], b[j][0], b[j][1]);
+#pragma unroll
+            for (int j = 0; j < NT; ++j)
+                mma16816(wt[j], pa[2 * qd + 1][0], pa[2 * qd + 1][1], pa[2 * qd + 1][2], pa[2 * qd + 1][3], b[j][2], b[j][3]);
+        }
+        if (C::kMT % 2) {
+#pragma unroll
+            for (int j = 0; j < NT; ++j) {
+                uint32_t b[2];
+                ldsm_x2(b, sb + av + (8 * j + l7) * C::kPitchA + (((2 * (C::kMT - 1) + (mi & 1)) ^ asw) << 4));
+                mma16816(wt[j], pa[C::kMT - 1][0], pa[C::kMT - 1][1], pa[C::kMT - 1][2], pa[C::kMT - 1][3], b[0], b[1]);
+            }
+        }
+#pragma unroll
+        for (int j = 0; j < NT; ++j) {
+            const bool v0 = 8 * j + t2 < rv, v1 = 8 * j + t2 + 1 < rv;
+            wa[j][0] = pack_bf16(v0 ? wt[j][0] : 0.f, v1 ? wt[j][1] : 0.f);
+            wa[j][1] = pack_bf16(v0 ? wt[j][2] : 0.f, v1 ? wt[j][3] : 0.f);
+        }
+    }
+    // ---- o [16][d] += w . B_v ----
+#pragma unroll
+    for (int kk = 0; kk < NT / 2; ++kk) {
+#pragma unroll
+        for (int i = 0; i < 8; ++i) {
+            uint32_t a4[4];       // (ranks lo, channels 16i..), (ranks lo, 16i+8..), (ranks hi, 16i..), (ranks hi, 16i+8..)
+            ldsm_x4_t(a4, sb + bv + (16 * kk + (mi >> 1) * 8 + l7) * kRowBytes + (((2 * i + (mi & 1)) ^ l7) << 4));
+            mma16816(st.o[2 * i], wa[2 * kk][0], wa[2 * kk][1], wa[2 * kk + 1][0], wa[2 * kk + 1][1], a4[0], a4[2]);
+            mma16816(st.o[2 * i + 1], wa[2 * kk][0], wa[2 * kk][1], wa[2 * kk + 1][0], wa[2 * kk + 1][1], a4[1], a4[3]);
+        }
+    }
+    if (NT % 2) {
+#pragma unroll
+        for (int i = 0; i < 8; ++i) {
+            uint32_t a2[2];
+            ldsm_x2_t(a2, sb + bv + (8 * (NT - 1) + l7) * kRowBytes + (((2 * i + (mi & 1)) ^ l7) << 4));
+            mma1688(st.o[2 * i], wa[NT - 1][0], wa[NT - 1][1], a2[0]);
+            mma1688(st.o[2 * i + 1], wa[NT - 1][0], wa[NT - 1][1], a2[1]);
+        }
+    }
+}
+
+// One block of DB rows of a dense page for 16 query rows; rows g / g+8 of the lane see the first lim0 / lim1 of
+// the block's `rows` valid tokens.  Stale V rows past `rows` have been zeroed by the caller.
+template <int DB>
+__device__ __forceinline__ void block_dense_unit(uint32_t sb, int lim0, int lim1, const uint32_t (&qf)[8][4],
+                                                 float scale, RowState &st, int lane) {
+    constexpr int NI = DB / 16, NS = DB / 8;
+    const int l7 = lane & 7, mi = lane >> 3, t2 = (lane & 3) * 2;
+    float s[NS][4];
+#pragma unroll
+    for (int i = 0; i < NI; ++i) {
+        s[2 * i][0] = s[2 * i][1] = s[2 * i][2] = s[2 * i][3] = 0.f;
+        s[2 * i + 1][0] = s[2 * i + 1][1] = s[2 * i + 1][2] = s[2 * i + 1][3] = 0.f;
+#pragma unroll
+        for (int kk = 0; kk < 8; ++kk) {
+            uint32_t a4[4];       // (tokens 16i.., channels lo), (tokens 16i+8.., lo), (16i.., hi), (16i+8.., hi)
+            ldsm_x4(a4, sb + (16 * i + (mi & 1) * 8 + l7) * kRowBytes + (((2 * kk + (mi >> 1)) ^ l7) << 4));
+            mma16816(s[2 * i], qf[kk][0], qf[kk][1], qf[kk][2], qf[kk][3], a4[0], a4[2]);
+            mma16816(s[2 * i + 1], qf[kk][0], qf[kk][1], qf[kk][2], qf[kk][3], a4[1], a4[3]);
+        }
+    }
+#pragma unroll
+    for (int b = 0; b < NS; ++b) {
+        const int tok = 8 * b + t2;
+        s[b][0] = tok < lim0 ? s[b][0] * scale : kMasked;     s[b][1] = tok + 1 < lim0 ? s[b][1] * scale : kMasked;
+        s[b][2] = tok < lim1 ? s[b][2] * scale : kMasked;     s[b][3] = tok + 1 < lim1 ? s[b][3] * scale : kMasked;
+    }
+    uint32_t pa[NI][4];
+    row_softmax<NS>(s, st, pa);
+#pragma unroll
+    for (int i = 0; i < NI; ++i) {
+#pragma unroll
+        for (int ii = 0; ii < 8; ++ii) {
+            uint32_t a4[4];       // (tokens lo, channels 16ii..), (tokens lo, 16ii+8..), (tokens hi, 16ii..), (tokens hi, 16ii+8..)
+            ldsm_x4_t(a4, sb + DB * kRowBytes + (16 * i + (mi >> 1) * 8 + l7) * kRowBytes + (((2 * ii + (mi & 1)) ^ l7) << 4));
+            mma16816(st.o[2 * ii], pa[i][0], pa[i][1], pa[i][2], pa[i][3], a4[0], a4[2]);
+            mma16816(st.o[2 * ii + 1], pa[i][0], pa[i][1], pa[i][2], pa[i][3], a4[1], a4[3]);
+        }
+    }
+}
+
+#define PKV_BLOCK_BARRIER() asm volatile("bar.sync 2, %0;" ::"n"(kBlockWarps * 32) : "memory")
+
+// Stages of the row-block kernel: as many as fit 100 KiB (two CTAs per SM), at least two, at most eight.
+__host__ __device__ inline int block_stages(const Geometry &g) { return max(2, min(8, (100 * 1024) / g.stage_bytes)); }
+
+template <int P, int NT>
+__global__ void __launch_bounds__(kBlockThreads, 2) block_tc_kernel(const __grid_constant__ DecodeArgs a) {
+    constexpr int kDB = kDenseBlock<P, NT, false>;
+    const Geometry &geo = a.geo;
+    const int S = block_stages(geo), H = geo.n_kv_heads, G = geo.group;
+    const int n_rows = a.q_len * G, n_blk = (n_rows + kBlockRows - 1) / kBlockRows;
+    const int rb = blockIdx.x % n_blk, head = (blockIdx.x / n_blk) % H, entry = blockIdx.x / (n_blk * H);
+    const PlanHeader hdr = *reinterpret_cast<const PlanHeader *>(a.plan);
+    if (entry >= hdr.n_seqs) return;
+    extern __shared__ __align__(1024) unsigned char smem[];
+    unsigned char *stages = smem;
+    const int stage_bytes = geo.stage_bytes, blob_bytes = geo.blob_bytes;
+    unsigned long long *full_bar = reinterpret_cast<unsigned long long *>(smem + (size_t)S * stage_bytes);
+    unsigned long long *empty_bar = full_bar + S;
+    StageDesc *descs = reinterpret_cast<StageDesc *>(empty_bar + S);
+    volatile int *abort_flag = reinterpret_cast<volatile int *>(descs + S);
+    const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+    if (tid == 0) {
+        for (int s = 0; s < S; ++s) { mbar_init(smem_u32(full_bar + s), 1); mbar_init(smem_u32(empty_bar + s), kBlockWarps); }
+        *abort_flag = 0;
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    }
+    if (stage_bytes > blob_bytes) {          // tails that 8-row tile loads read past a rank that is not a multiple of 8
+        const int tail16 = (stage_bytes - blob_bytes) >> 4;
+        for (int i = tid; i < S * tail16; i += kBlockThreads)
+            reinterpret_cast<uint4 *>(stages + (size_t)(i / tail16) * stage_bytes + blob_bytes)[i % tail16] =
+                make_uint4(0u, 0u, 0u, 0u);
+        asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+    }
+    __syncthreads();
+    const PlanEntry e = reinterpret_cast<const PlanEntry *>(a.plan + a.plan_entry)[entry];
+    const HeadUnits hu = head_units(geo, e);
+    const int T = a.n_tokens[(long long)e.seq * geo.n_layers + a.layer];
+
+    if (warp == kBlockWarps) {
+        // ------------------------------ producer (one lane) ------------------------------
+        if (lane != 0) return;
+        const int *pt = a.page_table + ((long long)e.seq * geo.n_layers + a.layer) * geo.max_pages;
+        bool ok = true;
+        int u = 0;
+        for (; u < hu.units && ok; ++u) {
+            const int s = u % S;
+            if (u >= S && !mbar_wait(smem_u32(empty_bar + s), ((u / S) - 1) & 1)) { ok = false; break; }
+            int page, blk, kind;
+            unit_to_page(geo, hu, u, page, blk, kind);
+            const int slot = pt[page];
+            int rows = 0, after = 0;
+            const unsigned char *src = nullptr;
+            if (slot < 0 || slot >= (kind == kKindFactor ? geo.n_factor_slots : geo.n_dense_slots)) {
+                atomicAdd(a.status + 2, 1);                  // corrupt page table: skip the unit, leave a mark
+                kind = kKindDense;
+            } else if (kind == kKindFactor) {
+                rows = P;
+                src = a.factor_pool + (long long)slot * geo.factor_slot_bytes + (long long)head * geo.blob_bytes;
+            } else {
+                rows = max(0, min(kDB, T - page * P - blk * kDB));
+                after = max(0, T - page * P - blk * kDB - rows);
+                src = a.dense_pool + (long long)slot * geo.dense_slot_bytes + (long long)head * geo.dense_head_bytes +
+                      blk * kDB * kRowBytes;
+            }
+            descs[s] = StageDesc{kind, rows, 0, after};
+            const uint32_t bar = smem_u32(full_bar + s);
+            const uint32_t dst = smem_u32(stages + (size_t)s * stage_bytes);
+            if (kind == kKindFactor) {
+                mbar_arrive_expect_tx(bar, blob_bytes);
+                bulk_g2s_keep(dst, src, blob_bytes, bar);
+            } else if (rows > 0) {
+                mbar_arrive_expect_tx(bar, 2 * rows * kRowBytes);
+                bulk_g2s_keep(dst, src, rows * kRowBytes, bar);
+                bulk_g2s_keep(dst + kDB * kRowBytes, src + P * kRowBytes, rows * kRowBytes, bar);
+            } else {
+                mbar_arrive(bar);
+            }
+        }
+        if (!ok) {
+            *abort_flag = 1;
+            atomicAdd(a.status, 1);
+        }
+        // copies already in flight must land before the CTA retires: wait (bounded) for the stages armed last
+        for (int back = 1; back <= min(u, S); ++back) {
+            const int k = u - back;
+            (void)mbar_wait(smem_u32(full_bar + k % S), (k / S) & 1);
+        }
+        return;
+    }
+    // ------------------------------ consumers: 16 query rows per warp ------------------------------
+    const int g8 = lane >> 2, t = lane & 3;
+    const int row0 = rb * kBlockRows + warp * 16 + g8, row1 = row0 + 8;       // row = query token * G + query head
+    const int j0 = row0 / G, j1 = row1 / G;
+    const bool ok0 = row0 < n_rows, ok1 = row1 < n_rows;
+    const long long qrow0 = ((long long)entry * a.q_len + j0) * geo.n_q_heads + head * G + row0 % G;
+    const long long qrow1 = ((long long)entry * a.q_len + j1) * geo.n_q_heads + head * G + row1 % G;
+    uint32_t qf[8][4];
+    {
+        const uint32_t *q0 = reinterpret_cast<const uint32_t *>(reinterpret_cast<const __nv_bfloat16 *>(a.q) + qrow0 * kHeadDim);
+        const uint32_t *q1 = reinterpret_cast<const uint32_t *>(reinterpret_cast<const __nv_bfloat16 *>(a.q) + qrow1 * kHeadDim);
+#pragma unroll
+        for (int kk = 0; kk < 8; ++kk) {
+            qf[kk][0] = ok0 ? __ldg(q0 + 8 * kk + t) : 0u;
+            qf[kk][1] = ok1 ? __ldg(q1 + 8 * kk + t) : 0u;
+            qf[kk][2] = ok0 ? __ldg(q0 + 8 * kk + 4 + t) : 0u;
+            qf[kk][3] = ok1 ? __ldg(q1 + 8 * kk + 4 + t) : 0u;
+        }
+    }
+    // positions of the sequence's newest that rows g / g+8 must not see (rows past the end: none, result unused)
+    const int hid0 = ok0 ? a.q_len - 1 - j0 : 0, hid1 = ok1 ? a.q_len - 1 - j1 : 0;
+    RowState st;
+#pragma unroll
+    for (int c = 0; c < 16; ++c) st.o[c][0] = st.o[c][1] = st.o[c][2] = st.o[c][3] = 0.f;
+    st.m[0] = st.m[1] = kNegInf;
+    st.l[0] = st.l[1] = 0.f;
+    bool ok = true;
+    for (int u = 0; u < hu.units; ++u) {
+        const int s = u % S;
+        // The only way out is this warp's own wait running out: if the producer gave up, every warp ends up at the
+        // same unarmed unit, so no warp is left alone at the block barrier below.
+        if (!mbar_wait(smem_u32(full_bar + s), (u / S) & 1)) {
+            ok = false;
+            if (lane == 0) { *abort_flag = 1; atomicAdd(a.status, 1); }
+            break;
+        }
+        const StageDesc dsc = descs[s];
+        const int rows = min(dsc.rows, dsc.kind == kKindFactor ? P : kDB);
+        if (rows > 0) {
+            const uint32_t sb = smem_u32(stages + (size_t)s * stage_bytes);
+            if (dsc.kind == kKindFactor) {
+                block_factor_unit<P, NT>(sb, geo.ak_off, geo.bk_off, geo.av_off, geo.bv_off, geo.rank_k, geo.rank_v, qf,
+                                         geo.scale_log2e, st, lane);
+            } else {
+                if (rows < kDB) {
+                    // unfilled V rows hold stale bytes: zero them (each warp a share) before any warp reads V
+                    uint4 *v = reinterpret_cast<uint4 *>(stages + (size_t)s * stage_bytes + kDB * kRowBytes + rows * kRowBytes);
+                    for (int i = warp * 32 + lane; i < (kDB - rows) * 16; i += kBlockWarps * 32) v[i] = make_uint4(0u, 0u, 0u, 0u);
+                    PKV_BLOCK_BARRIER();
+                }
+                const int lim0 = rows - max(0, hid0 - dsc.after), lim1 = rows - max(0, hid1 - dsc.after);
+                block_dense_unit<kDB>(sb, lim0, lim1, qf, geo.scale_log2e, st, lane);
+                if (rows < kDB) asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+            }
+        }
+        __syncwarp();
+        if (lane == 0) mbar_arrive(smem_u32(empty_bar + s));
+    }
+    if (!ok) return;
+    float l0 = st.l[0], l1 = st.l[1];
+#pragma unroll
+    for (int off = 1; off <= 2; off <<= 1) {
+        l0 += __shfl_xor_sync(0xffffffffu, l0, off);
+        l1 += __shfl_xor_sync(0xffffffffu, l1, off);
+    }
+    const float inv0 = 1.f / l0, inv1 = 1.f / l1;
+    __nv_bfloat16 *out = reinterpret_cast<__nv_bfloat16 *>(a.out);
+#pragma unroll
+    for (int c = 0; c < 16; ++c) {
+        const int ch = 8 * c + 2 * t;
+        if (ok0) {
+            const float x = st.o[c][0] * inv0, y = st.o[c][1] * inv0;
+            if (out) *reinterpret_cast<uint32_t *>(out + qrow0 * kHeadDim + ch) = pack_bf16(x, y);
+            if (a.out_f32) *reinterpret_cast<float2 *>(a.out_f32 + qrow0 * kHeadDim + ch) = make_float2(x, y);
+        }
+        if (ok1) {
+            const float x = st.o[c][2] * inv1, y = st.o[c][3] * inv1;
+            if (out) *reinterpret_cast<uint32_t *>(out + qrow1 * kHeadDim + ch) = pack_bf16(x, y);
+            if (a.out_f32) *reinterpret_cast<float2 *>(a.out_f32 + qrow1 * kHeadDim + ch) = make_float2(x, y);
+        }
+    }
+}
+
+size_t block_smem_bytes(const Geometry &g) {
+    const int S = block_stages(g);
+    return (size_t)S * g.stage_bytes + S * (8 + 8 + sizeof(StageDesc)) + 64;
+}
+
+template <int P, int NT>
+cudaError_t launch_block(const DecodeArgs &a, int n_ctas, cudaStream_t st) {
+    block_tc_kernel<P, NT><<<n_ctas, kBlockThreads, block_smem_bytes(a.geo), st>>>(a);
+    return cudaGetLastError();
+}
+
 size_t decode_smem_bytes(const Geometry &g) {
     return (size_t)g.n_stages * g.stage_bytes + kConsumerWarps * kPartialFloats * 4 +
            g.n_stages * (8 + 8 + sizeof(StageDesc) + 4) + 64;
@@ -1103,6 +1516,8 @@ cudaError_t launch_tc(const DecodeArgs &a, cudaStream_t st) {
 template <int P, int NT>
 cudaError_t setup_tc() {
     cudaError_t e = cudaFuncSetAttribute(decode_tc_kernel<P, NT, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBudget / 2);
+    if (e != cudaSuccess) return e;
+    e = cudaFuncSetAttribute(block_tc_kernel<P, NT>, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBudget / 2);
     if (e != cudaSuccess) return e;
     return cudaFuncSetAttribute(decode_tc_kernel<P, NT, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBudget / 2);
 }
@@ -1135,6 +1550,18 @@ cudaError_t launch_decode(const DecodeArgs &a, int n_segs, cudaStream_t st) {
     if (e != cudaSuccess || a.variant != 1) return e;
     merge_kernel<<<n_segs, 256, 0, st>>>(a);
     return cudaGetLastError();
+}
+
+// Row-block kernel: one CTA per (sequence, KV head, block of 64 query rows); bf16 factors only.
+cudaError_t launch_decode_blocks(const DecodeArgs &a, int n_seqs, cudaStream_t st) {
+    const int n_blk = (a.q_len * a.geo.group + kBlockRows - 1) / kBlockRows;
+    const long long n_ctas = (long long)n_seqs * a.geo.n_kv_heads * n_blk;
+    if (a.geo.factor_bits == 4 || n_ctas <= 0 || n_ctas > 0x7fffffffLL) return cudaErrorInvalidValue;
+    cudaError_t e = cudaErrorInvalidValue;
+#define PKV_LAUNCH_BLOCK(P, NT) if (a.geo.page == P && a.geo.rank_tiles == NT) e = launch_block<P, NT>(a, (int)n_ctas, st);
+    PKV_FOR_EACH_SHAPE(PKV_LAUNCH_BLOCK)
+#undef PKV_LAUNCH_BLOCK
+    return e;
 }
 
 // Eq. 5 across caches: states [n_shards][n_rows][d + 2] as written by store_out; one warp per row.

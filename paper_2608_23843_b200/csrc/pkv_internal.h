@@ -121,6 +121,8 @@ cudaError_t launch_append(const Geometry &geo, unsigned char *dense_pool, const 
 cudaError_t launch_compress(const Geometry &geo, const unsigned char *dense_pool, unsigned char *factor_pool,
                             const int2 *worklist, int n_entries, int *status, cudaStream_t st);
 cudaError_t launch_decode(const DecodeArgs &a, int n_segs, cudaStream_t st);
+cudaError_t launch_decode_blocks(const DecodeArgs &a, int n_seqs, cudaStream_t st);
+constexpr int kRowBlock = 64;          // query rows (token x query head) per CTA of the row-block kernel
 cudaError_t launch_merge_states(const float *states, int n_shards, long long n_rows, void *out, float *out_f32,
                                 cudaStream_t st);
 cudaError_t launch_decode_static_scratch(const DecodeArgs &a, int n_segs, cudaStream_t st, const char **why);

@@ -481,7 +481,13 @@ def test_many_tiny_segments_per_cta(rank, n_ctas):
     (16, 8, 8, 1, 11, 16),        # eight query tokens per tile, two blocks; new positions span two pages
     (64, 16, 16, 2, 7, 16),       # four query tokens per tile
     (64, 24, 24, 4, 4, 4),        # INT4 factors
-    (64, 32, 32, 4, 64, 16),      # a prefill chunk of one page, 32 blocks
+    (64, 32, 32, 4, 64, 16),      # a prefill chunk of one page: 256 query rows per KV head -> row-block kernel
+    (32, 16, 14, 4, 16, 16),      # row-block kernel, exactly one block of 64 rows; unequal ranks
+    (16, 8, 8, 8, 9, 16),         # row-block kernel, 72 rows (second block mostly empty), P = 16
+    (64, 13, 11, 2, 37, 16),      # row-block kernel, 74 rows, ranks that are not multiples of 8
+    (64, 32, 32, 1, 70, 16),      # row-block kernel, one query head per KV head, full-width ranks
+    (64, 24, 24, 8, 16, 16),      # row-block kernel, 128 rows, two tokens per 16-row tile
+    (32, 8, 8, 4, 40, 16),        # row-block kernel, one rank tile, queries spanning two pages
 ])
 def test_multi_query_attention(P, rk, rv, G, q_len, bits):
     """Several new positions per sequence in one call (causal among themselves): every query row against the
@@ -495,8 +501,11 @@ def test_multi_query_attention(P, rk, rv, G, q_len, bits):
     tpt = max(1, min(q_len, 8 // G))
     nblk = -(-q_len // tpt)
     W = max(P, -(-q_len // P) * P)
+    # With 64 or more query rows per KV head the row-block kernel is meant; this small batch would not fill the GPU
+    # with it and the library would choose the column kernel, unless that one's plan entries do not fit: make it so.
+    row_blocks = q_len * G >= 64 and bits != 4
     cfg = pkv.make_config(n_layers=1, n_kv_heads=H, n_q_heads=H * G, rank=rk, rank_v=rv, page_size=P, sink_tokens=P,
-                          recent_tokens=W, max_seqs=n * nblk, max_pages_per_seq=48, n_dense_slots=200,
+                          recent_tokens=W, max_seqs=n if row_blocks else n * nblk, max_pages_per_seq=48, n_dense_slots=200,
                           n_factor_slots=120, factor_bits=bits)
     pair = Pair(cfg, seed=P + q_len)
     for s, T in enumerate(lengths):
@@ -541,13 +550,18 @@ def test_multi_query_attention(P, rk, rv, G, q_len, bits):
             if bits != 4:
                 floor = rel_err(ref_rounded[i, j], ref[i, j])
                 assert rel_err(got[i, j], ref[i, j]) <= 1e-2 + 3.0 * floor, (i, j, floor)
-    # the last query is the single-query call, bit for bit; and the call is reproducible
+    # the call is reproducible; its last query is the single-query call (bit for bit where the same kernel serves both)
     single = torch.empty((n, H * G, 128), dtype=torch.bfloat16, device="cuda")
     pair.gpu.decode_attention(0, order, qd[:, q_len - 1].contiguous(), single)
     again = torch.empty_like(out)
     pair.gpu.decode_attention_multi(0, order, q_len, qd, again)
     torch.cuda.synchronize()
-    assert torch.equal(single, out[:, q_len - 1]) and torch.equal(again, out)
+    assert torch.equal(again, out)
+    if row_blocks:                           # row-block kernel: another summation order than the single-query kernel
+        a, b = f64(single), f64(out[:, q_len - 1])
+        assert np.abs(a - b).max() <= 1e-2 * np.abs(a).max()
+    else:
+        assert torch.equal(single, out[:, q_len - 1])
     st = pair.gpu.stats()
     assert st["device_timeouts"] == 0 and st["bad_slot_indices"] == 0
     print("multi-query P=%d r=(%d,%d) G=%d q_len=%d bits=%d: kernel max %.2e e2e max %.2e" % (P, rk, rv, G, q_len, bits, worst_k, worst_e))
@@ -622,3 +636,45 @@ def test_sequence_sharded_attention_states(bits):
     with pytest.raises(pkv.PkvError):
         pkv.pkv_merge_attention_states(states, 0, 3 * H * G, out, None, torch.cuda.current_stream())
     print("sharded states bits=%d: merged kernel gate max %.2e, log-sum-exp max abs %.2e" % (bits, worst, worst_lse))
+
+
+@pytest.mark.parametrize("P,rk,rv,G,q_len", [(64, 24, 24, 4, 128), (32, 16, 14, 8, 33), (16, 16, 16, 2, 48), (64, 8, 5, 4, 17)])
+def test_row_block_kernel_agrees_with_the_column_kernel(P, rk, rv, G, q_len):
+    """pkv_decode_attention_multi picks its kernel by shape; decode_variant = 2 pins the decode (column) kernel.  The
+    two must agree to fp32-accumulation accuracy on the same cache contents (same compression kernel, same factors),
+    including sequences whose new positions start a page, end mid-block, or make up the whole sequence."""
+    H = 2
+    lengths = [30 * P + 3, q_len, 5 * P, 12 * P + P // 2, q_len + 1]
+    W = -(-q_len // P) * P
+    outs = []
+    for variant in (0, 2):
+        tpt = max(1, min(q_len, 8 // G))
+        # variant 0 with too few plan entries for the column kernel: the row-block kernel runs whatever the batch size
+        cfg = pkv.make_config(n_layers=1, n_kv_heads=H, n_q_heads=H * G, rank=rk, rank_v=rv, page_size=P, sink_tokens=P,
+                              recent_tokens=W, max_seqs=len(lengths) * (-(-q_len // tpt) if variant == 2 else 1),
+                              max_pages_per_seq=40, n_dense_slots=200, n_factor_slots=160, decode_variant=variant)
+        cache = pkv.Cache(cfg, "cuda")
+        for s, T in enumerate(lengths):
+            k, v = gen_kv(8, 0, s, T, cfg, outlier_prob=0.01)
+            if T > q_len:
+                cache.append_kv(0, [s], [T - q_len], k[:T - q_len].cuda(), v[:T - q_len].cuda())
+                cache.compress_eligible_pages(0)
+            cache.append_kv(0, [s], [q_len], k[T - q_len:].cuda(), v[T - q_len:].cuda())
+        g = torch.Generator().manual_seed(5)
+        q = torch.randn((len(lengths), q_len, H * G, 128), generator=g).to(torch.bfloat16).cuda()
+        out32 = torch.empty(q.shape, dtype=torch.float32, device="cuda")
+        out = cache.decode_attention_multi(0, [4, 2, 0, 1, 3], q_len, q, None, out32)
+        again = torch.empty_like(out32)
+        cache.decode_attention_multi(0, [4, 2, 0, 1, 3], q_len, q, None, again)
+        torch.cuda.synchronize()
+        st = cache.stats()
+        assert st["device_timeouts"] == 0 and st["bad_slot_indices"] == 0 and not out32.isnan().any()
+        assert torch.equal(again, out32)                                     # reproducible
+        outs.append((f64(out), f64(out32)))
+        cache.close()
+    a, b = outs[0][1], outs[1][1]
+    for i in range(a.shape[0]):
+        for j in range(q_len):
+            assert np.abs(a[i, j] - b[i, j]).max() <= 6e-3 * np.abs(b[i, j]).max(), (i, j)
+    print("row-block vs column kernel P=%d r=(%d,%d) G=%d q_len=%d: max rel diff %.2e"
+          % (P, rk, rv, G, q_len, max(np.abs(a[i, j] - b[i, j]).max() / np.abs(b[i, j]).max() for i in range(a.shape[0]) for j in range(q_len))))
