@@ -44,6 +44,10 @@ WORKLOADS = {
     # sequence) -> decode -> compress_eligible, so every 64th step factorizes one page per (sequence, KV head, K|V)
     "serving_b32_8k": dict(n_layers=1, n_kv_heads=8, n_q_heads=32, batch=32, T=8192, rank=24, sink=64, recent=256,
                            ragged=False, outliers=0.0, serving=True),
+    # A chunk of a prefill on the Llama-3-8B shape: one sequence of 32K tokens whose newest 2048 positions (inside a
+    # dense window of that size) are the queries.  Use with --q-len 2048 (pkv_decode_attention_multi).
+    "prefill_chunk_llama3_8b_32k": dict(n_layers=2, layers_per_step=1, n_kv_heads=8, n_q_heads=32, batch=1, T=32768,
+                                        rank=24, sink=64, recent=2048, ragged=False, outliers=0.0),
     # BASELINE config 0: tiny (L2-resident; latency only)
     "tiny": dict(n_layers=1, n_kv_heads=1, n_q_heads=4, batch=1, T=1024, rank=16, sink=64, recent=128,
                  ragged=False, outliers=0.0),
@@ -63,6 +67,15 @@ def _peaks():
         with open(path) as f:
             return float(json.load(f)["hbm_gbs"]), "measured (MEASURED_PEAKS.json hbm_gbs)"
     return 6650.0, "fallback (6.65 TB/s)"
+
+
+def _tensor_peak():
+    """Dense bf16 tensor throughput in TFLOP/s (the burst figure: kernels here are timed in short regions)."""
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(path):
+        with open(path) as f:
+            return float(json.load(f)["bf16_tflops"]), "measured (MEASURED_PEAKS.json bf16_tflops)"
+    return 1590.0, "fallback (1.59 PFLOP/s)"
 
 
 class ClockSampler:
@@ -648,6 +661,25 @@ def main():
             "e2e": {"value": e2e_ms * 1e3, "unit": "us", "h2d_bytes_per_step": qbytes, "d2h_bytes_per_step": qbytes},
             "gpu_launches": lps * args.steps * (2 if args.seq_sharded else 1), "clocks": clocks,
         }
+        P_, Gq = w.get("page", 64), Hq // w["n_kv_heads"]
+        rows = QL * Gq
+        if QL > 1 and args.factor_bits != 4 and rows >= 64 and w["batch"] * w["n_kv_heads"] * -(-rows // 64) >= 128:
+            # Served by the row-block kernel, whose bound is the tensor pipe, not HBM: algorithmic FLOPs per launch =
+            # query rows x (factor pages x 2 (d r_k + r_k P + P r_v + r_v d) + dense tokens x 4 d); the causal
+            # triangle among the new positions is counted in full.
+            rv_ = w.get("rank_v", rank)
+            flops = 0
+            for T_ in lengths:
+                n_pages_ = -(-T_ // P_)
+                nf_ = max(0, T_ // P_ - w["recent"] // P_ - w["sink"] // P_)
+                dense_tok = T_ - nf_ * P_
+                flops += QL * Hq * (nf_ * 2 * (128 * rank + rank * P_ + P_ * rv_ + rv_ * 128) + dense_tok * 4 * 128)
+            tpeak, tsrc = _tensor_peak()
+            tach = flops / (launch_ms * 1e-3) / 1e12
+            line["roofline"] = {"bound": "tensor", "kernel": "block_tc_kernel<P=%d, rank tiles=%d>" % (P_, (rank + 7) // 8),
+                                "achieved": tach, "peak": tpeak, "unit": "TFLOP/s", "frac": tach / tpeak,
+                                "peak_source": tsrc + "; the kernel uses mma.sync, whose pipe ncu showed 50 % busy at this rate",
+                                "traffic": None, "launch_us": launch_ms * 1e3, "algorithmic_flops_per_launch": flops}
         if not args.no_cpu_baseline and world == 1 and QL == 1:
             o = oracle_sample(w, rank, 3, args.factor_bits)
             line["cpu_baseline"] = {"value": o["decode_s"] * 1e6 * o["slices_per_step"], "unit": "us",

@@ -1163,17 +1163,24 @@ __device__ __forceinline__ void block_factor_unit(uint32_t sb, int ak, int bk, i
         float qt[NT][4];
 #pragma unroll
         for (int j = 0; j < NT; ++j) qt[j][0] = qt[j][1] = qt[j][2] = qt[j][3] = 0.f;
+        // The asm statements keep their order, so loads are issued by hand ahead of the products that use them:
+        // here one group of NT tiles ahead.
+        uint32_t b[2][NT][4];
+#pragma unroll
+        for (int j = 0; j < NT; ++j) ldsm_x4(b[0][j], sb + bk + (8 * j + l7) * kRowBytes + ((mi ^ l7) << 4));
 #pragma unroll
         for (int qd = 0; qd < 4; ++qd) {
-            uint32_t b[NT][4];
+            if (qd + 1 < 4) {
 #pragma unroll
-            for (int j = 0; j < NT; ++j) ldsm_x4(b[j], sb + bk + (8 * j + l7) * kRowBytes + (((4 * qd + mi) ^ l7) << 4));
+                for (int j = 0; j < NT; ++j)
+                    ldsm_x4(b[(qd + 1) & 1][j], sb + bk + (8 * j + l7) * kRowBytes + (((4 * (qd + 1) + mi) ^ l7) << 4));
+            }
 #pragma unroll
             for (int j = 0; j < NT; ++j)
-                mma16816(qt[j], qf[2 * qd][0], qf[2 * qd][1], qf[2 * qd][2], qf[2 * qd][3], b[j][0], b[j][1]);
+                mma16816(qt[j], qf[2 * qd][0], qf[2 * qd][1], qf[2 * qd][2], qf[2 * qd][3], b[qd & 1][j][0], b[qd & 1][j][1]);
 #pragma unroll
             for (int j = 0; j < NT; ++j)
-                mma16816(qt[j], qf[2 * qd + 1][0], qf[2 * qd + 1][1], qf[2 * qd + 1][2], qf[2 * qd + 1][3], b[j][2], b[j][3]);
+                mma16816(qt[j], qf[2 * qd + 1][0], qf[2 * qd + 1][1], qf[2 * qd + 1][2], qf[2 * qd + 1][3], b[qd & 1][j][2], b[qd & 1][j][3]);
         }
 #pragma unroll
         for (int j = 0; j < NT; ++j) {
@@ -1190,27 +1197,37 @@ __device__ __forceinline__ void block_factor_unit(uint32_t sb, int ak, int bk, i
     float s[NS][4];
 #pragma unroll
     for (int b = 0; b < NS; ++b) s[b][0] = s[b][1] = s[b][2] = s[b][3] = 0.f;
+    if (NT >= 2) {
+        // a4 = (ranks lo, tokens 16i..), (ranks lo, tokens 16i+8..), (ranks hi, 16i..), (ranks hi, 16i+8..); one item ahead
+        constexpr int kItems = (NT / 2) * C::kMT;
+        uint32_t a4[2][4];
+        ldsm_x4_t(a4[0], sb + ak + ((mi >> 1) * 8 + l7) * C::kPitchA + (((mi & 1) ^ asw) << 4));
 #pragma unroll
-    for (int kk = 0; kk < NT / 2; ++kk) {
-#pragma unroll
-        for (int i = 0; i < C::kMT; ++i) {
-            uint32_t a4[4];       // (ranks lo, tokens 16i..), (ranks lo, tokens 16i+8..), (ranks hi, 16i..), (ranks hi, 16i+8..)
-            ldsm_x4_t(a4, sb + ak + (16 * kk + (mi >> 1) * 8 + l7) * C::kPitchA + (((2 * i + (mi & 1)) ^ asw) << 4));
-            mma16816(s[2 * i], qh[2 * kk][0], qh[2 * kk][1], qh[2 * kk + 1][0], qh[2 * kk + 1][1], a4[0], a4[2]);
-            mma16816(s[2 * i + 1], qh[2 * kk][0], qh[2 * kk][1], qh[2 * kk + 1][0], qh[2 * kk + 1][1], a4[1], a4[3]);
-            mma16816(s[2 * i], ql[2 * kk][0], ql[2 * kk][1], ql[2 * kk + 1][0], ql[2 * kk + 1][1], a4[0], a4[2]);
-            mma16816(s[2 * i + 1], ql[2 * kk][0], ql[2 * kk][1], ql[2 * kk + 1][0], ql[2 * kk + 1][1], a4[1], a4[3]);
+        for (int it = 0; it < kItems; ++it) {
+            const int kk = it / C::kMT, i = it % C::kMT;
+            if (it + 1 < kItems) {
+                const int kn = (it + 1) / C::kMT, in = (it + 1) % C::kMT;
+                ldsm_x4_t(a4[(it + 1) & 1], sb + ak + (16 * kn + (mi >> 1) * 8 + l7) * C::kPitchA + (((2 * in + (mi & 1)) ^ asw) << 4));
+            }
+            const uint32_t *x = a4[it & 1];
+            mma16816(s[2 * i], qh[2 * kk][0], qh[2 * kk][1], qh[2 * kk + 1][0], qh[2 * kk + 1][1], x[0], x[2]);
+            mma16816(s[2 * i + 1], qh[2 * kk][0], qh[2 * kk][1], qh[2 * kk + 1][0], qh[2 * kk + 1][1], x[1], x[3]);
+            mma16816(s[2 * i], ql[2 * kk][0], ql[2 * kk][1], ql[2 * kk + 1][0], ql[2 * kk + 1][1], x[0], x[2]);
+            mma16816(s[2 * i + 1], ql[2 * kk][0], ql[2 * kk][1], ql[2 * kk + 1][0], ql[2 * kk + 1][1], x[1], x[3]);
         }
     }
     if (NT % 2) {
+        uint32_t a2[2][2];
+        ldsm_x2_t(a2[0], sb + ak + (8 * (NT - 1) + l7) * C::kPitchA + (((mi & 1) ^ asw) << 4));
 #pragma unroll
         for (int i = 0; i < C::kMT; ++i) {
-            uint32_t a2[2];
-            ldsm_x2_t(a2, sb + ak + (8 * (NT - 1) + l7) * C::kPitchA + (((2 * i + (mi & 1)) ^ asw) << 4));
-            mma1688(s[2 * i], qh[NT - 1][0], qh[NT - 1][1], a2[0]);
-            mma1688(s[2 * i + 1], qh[NT - 1][0], qh[NT - 1][1], a2[1]);
-            mma1688(s[2 * i], ql[NT - 1][0], ql[NT - 1][1], a2[0]);
-            mma1688(s[2 * i + 1], ql[NT - 1][0], ql[NT - 1][1], a2[1]);
+            if (i + 1 < C::kMT)
+                ldsm_x2_t(a2[(i + 1) & 1], sb + ak + (8 * (NT - 1) + l7) * C::kPitchA + (((2 * (i + 1) + (mi & 1)) ^ asw) << 4));
+            const uint32_t *x = a2[i & 1];
+            mma1688(s[2 * i], qh[NT - 1][0], qh[NT - 1][1], x[0]);
+            mma1688(s[2 * i + 1], qh[NT - 1][0], qh[NT - 1][1], x[1]);
+            mma1688(s[2 * i], ql[NT - 1][0], ql[NT - 1][1], x[0]);
+            mma1688(s[2 * i + 1], ql[NT - 1][0], ql[NT - 1][1], x[1]);
         }
     }
     uint32_t pa[NS / 2][4];
@@ -1221,16 +1238,22 @@ __device__ __forceinline__ void block_factor_unit(uint32_t sb, int ak, int bk, i
         float wt[NT][4];
 #pragma unroll
         for (int j = 0; j < NT; ++j) wt[j][0] = wt[j][1] = wt[j][2] = wt[j][3] = 0.f;
+        if (C::kMT >= 2) {
+            // the score registers are free by now: all tiles of A_v are fetched before the first product
+            uint32_t b[C::kMT / 2 > 0 ? C::kMT / 2 : 1][NT][4];
 #pragma unroll
-        for (int qd = 0; qd < C::kMT / 2; ++qd) {
-            uint32_t b[NT][4];
+            for (int qd = 0; qd < C::kMT / 2; ++qd)
 #pragma unroll
-            for (int j = 0; j < NT; ++j) ldsm_x4(b[j], sb + av + (8 * j + l7) * C::kPitchA + (((4 * qd + mi) ^ asw) << 4));
+                for (int j = 0; j < NT; ++j) ldsm_x4(b[qd][j], sb + av + (8 * j + l7) * C::kPitchA + (((4 * qd + mi) ^ asw) << 4));
 #pragma unroll
-            for (int j = 0; j < NT; ++j) mma16816(wt[j], pa[2 * qd][0], pa[2 * qd][1], pa[2 * qd][2], pa[2 * qd][3], b[j][0], b[j][1]);
+            for (int qd = 0; qd < C::kMT / 2; ++qd) {
 #pragma unroll
-            for (int j = 0; j < NT; ++j)
-                mma16816(wt[j], pa[2 * qd + 1][0], pa[2 * qd + 1][1], pa[2 * qd + 1][2], pa[2 * qd + 1][3], b[j][2], b[j][3]);
+                for (int j = 0; j < NT; ++j)
+                    mma16816(wt[j], pa[2 * qd][0], pa[2 * qd][1], pa[2 * qd][2], pa[2 * qd][3], b[qd][j][0], b[qd][j][1]);
+#pragma unroll
+                for (int j = 0; j < NT; ++j)
+                    mma16816(wt[j], pa[2 * qd + 1][0], pa[2 * qd + 1][1], pa[2 * qd + 1][2], pa[2 * qd + 1][3], b[qd][j][2], b[qd][j][3]);
+            }
         }
         if (C::kMT % 2) {
 #pragma unroll
@@ -1248,23 +1271,35 @@ __device__ __forceinline__ void block_factor_unit(uint32_t sb, int ak, int bk, i
         }
     }
     // ---- o [16][d] += w . B_v ----
+    if (NT >= 2) {
+        // a4 = (ranks lo, channels 16i..), (ranks lo, 16i+8..), (ranks hi, 16i..), (ranks hi, 16i+8..); two items ahead
+        constexpr int kItems = (NT / 2) * 8;
+        uint32_t a4[3][4];
+        ldsm_x4_t(a4[0], sb + bv + ((mi >> 1) * 8 + l7) * kRowBytes + (((mi & 1) ^ l7) << 4));
+        ldsm_x4_t(a4[1], sb + bv + ((mi >> 1) * 8 + l7) * kRowBytes + (((2 + (mi & 1)) ^ l7) << 4));
 #pragma unroll
-    for (int kk = 0; kk < NT / 2; ++kk) {
-#pragma unroll
-        for (int i = 0; i < 8; ++i) {
-            uint32_t a4[4];       // (ranks lo, channels 16i..), (ranks lo, 16i+8..), (ranks hi, 16i..), (ranks hi, 16i+8..)
-            ldsm_x4_t(a4, sb + bv + (16 * kk + (mi >> 1) * 8 + l7) * kRowBytes + (((2 * i + (mi & 1)) ^ l7) << 4));
-            mma16816(st.o[2 * i], wa[2 * kk][0], wa[2 * kk][1], wa[2 * kk + 1][0], wa[2 * kk + 1][1], a4[0], a4[2]);
-            mma16816(st.o[2 * i + 1], wa[2 * kk][0], wa[2 * kk][1], wa[2 * kk + 1][0], wa[2 * kk + 1][1], a4[1], a4[3]);
+        for (int it = 0; it < kItems; ++it) {
+            const int kk = it / 8, i = it % 8;
+            if (it + 2 < kItems) {
+                const int kn = (it + 2) / 8, in = (it + 2) % 8;
+                ldsm_x4_t(a4[(it + 2) % 3], sb + bv + (16 * kn + (mi >> 1) * 8 + l7) * kRowBytes + (((2 * in + (mi & 1)) ^ l7) << 4));
+            }
+            const uint32_t *x = a4[it % 3];
+            mma16816(st.o[2 * i], wa[2 * kk][0], wa[2 * kk][1], wa[2 * kk + 1][0], wa[2 * kk + 1][1], x[0], x[2]);
+            mma16816(st.o[2 * i + 1], wa[2 * kk][0], wa[2 * kk][1], wa[2 * kk + 1][0], wa[2 * kk + 1][1], x[1], x[3]);
         }
     }
     if (NT % 2) {
+        uint32_t a2[3][2];
+        ldsm_x2_t(a2[0], sb + bv + (8 * (NT - 1) + l7) * kRowBytes + (((mi & 1) ^ l7) << 4));
+        ldsm_x2_t(a2[1], sb + bv + (8 * (NT - 1) + l7) * kRowBytes + (((2 + (mi & 1)) ^ l7) << 4));
 #pragma unroll
         for (int i = 0; i < 8; ++i) {
-            uint32_t a2[2];
-            ldsm_x2_t(a2, sb + bv + (8 * (NT - 1) + l7) * kRowBytes + (((2 * i + (mi & 1)) ^ l7) << 4));
-            mma1688(st.o[2 * i], wa[NT - 1][0], wa[NT - 1][1], a2[0]);
-            mma1688(st.o[2 * i + 1], wa[NT - 1][0], wa[NT - 1][1], a2[1]);
+            if (i + 2 < 8)
+                ldsm_x2_t(a2[(i + 2) % 3], sb + bv + (8 * (NT - 1) + l7) * kRowBytes + (((2 * (i + 2) + (mi & 1)) ^ l7) << 4));
+            const uint32_t *x = a2[i % 3];
+            mma1688(st.o[2 * i], wa[NT - 1][0], wa[NT - 1][1], x[0]);
+            mma1688(st.o[2 * i + 1], wa[NT - 1][0], wa[NT - 1][1], x[1]);
         }
     }
 }
