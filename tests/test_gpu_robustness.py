@@ -298,3 +298,74 @@ def test_two_step_compression_on_a_side_stream(bits):
     assert st["device_timeouts"] == 0 and st["page_svds_not_converged"] == 0 and st["bad_slot_indices"] == 0
     print("two-step compression bits=%d: kernel gate max %.2e, %d pages" % (bits, worst, st["pages_compressed"]))
     sync.close()
+
+
+@pytest.mark.gpu
+@pytest.mark.parametrize("q_len,max_seqs", [(3, 4), (40, 2)])
+def test_cuda_graph_replay_of_multi_query_and_state_calls(q_len, max_seqs):
+    """pkv_decode_attention_multi (decode kernel with query columns at q_len = 3; row-block kernel at q_len = 40,
+    forced by max_seqs) and pkv_decode_attention_partial + pkv_merge_attention_states recorded into one CUDA graph:
+    replays equal eager calls, also after appends that stay inside the current pages."""
+    H, G = 2, 2
+    cfg = pkv.make_config(n_layers=1, n_kv_heads=H, n_q_heads=H * G, rank=16, sink_tokens=64, recent_tokens=128,
+                          max_seqs=max_seqs, max_pages_per_seq=40, n_dense_slots=100, n_factor_slots=100, decode_overlap=1)
+    cache = pkv.Cache(cfg, "cuda", None, None)
+    T = [900, 1410]
+    data = [synth.make_kv(31, 0, s, 2000, H, 128, 64, "cuda") for s in range(2)]
+    for s in range(2):
+        cache.append_kv(0, [s], [T[s]], data[s][0][:T[s]], data[s][1][:T[s]])
+    cache.compress_eligible_pages(0)
+    ids = [1, 0]
+    g = torch.Generator(device="cuda").manual_seed(3)
+    qm = torch.randn((2, q_len, H * G, 128), generator=g, device="cuda").to(torch.bfloat16)
+    q1 = qm[:, -1].contiguous()
+    out_m, out_1 = torch.empty_like(qm), torch.empty_like(q1)
+    state = torch.empty((2, H * G, 130), dtype=torch.float32, device="cuda")
+
+    def eager():
+        a, b = torch.empty_like(qm), torch.empty_like(q1)
+        cache.decode_attention_multi(0, ids, q_len, qm, a)
+        st = cache.decode_attention_partial(0, ids, q1)
+        pkv.pkv_merge_attention_states(st, 1, 2 * H * G, b, None, torch.cuda.current_stream())
+        torch.cuda.synchronize()
+        return a, b
+
+    ref_m, ref_1 = eager()                                  # builds both plans outside the capture
+    cache.decode_attention_multi(0, ids, q_len, qm, out_m)  # the multi-query plan is the current one again
+    side = torch.cuda.Stream()
+    side.wait_stream(torch.cuda.current_stream())
+    graph = torch.cuda.CUDAGraph()
+    with torch.cuda.stream(side):
+        with torch.cuda.graph(graph, stream=side):
+            cache.decode_attention_multi(0, ids, q_len, qm, out_m)
+            with pytest.raises(pkv.PkvError) as e:         # one plan per layer: the single-query plan is stale now
+                cache.decode_attention_partial(0, ids, q1, state)
+            assert e.value.status == pkv.PKV_ERR_UNSUPPORTED
+    torch.cuda.current_stream().wait_stream(side)
+    for n in (0, 2):
+        if n:
+            cache.append_kv(0, [0, 1], [n, n], torch.cat([data[0][0][T[0]:T[0] + n], data[1][0][T[1]:T[1] + n]]),
+                            torch.cat([data[0][1][T[0]:T[0] + n], data[1][1][T[1]:T[1] + n]]))
+            T[0] += n
+            T[1] += n
+            cache.decode_attention_multi(0, ids, q_len, qm, out_m)         # same pages: nothing to rebuild
+            ref_m, ref_1 = eager()
+            cache.decode_attention_multi(0, ids, q_len, qm, torch.empty_like(qm))
+        out_m.zero_()
+        graph.replay()
+        torch.cuda.synchronize()
+        assert torch.equal(out_m, ref_m)
+    # the state call in a graph of its own, with its plan current
+    cache.decode_attention_partial(0, ids, q1, state)
+    graph2 = torch.cuda.CUDAGraph()
+    side.wait_stream(torch.cuda.current_stream())
+    with torch.cuda.stream(side):
+        with torch.cuda.graph(graph2, stream=side):
+            cache.decode_attention_partial(0, ids, q1, state)
+            pkv.pkv_merge_attention_states(state, 1, 2 * H * G, out_1, None, side)
+    torch.cuda.current_stream().wait_stream(side)
+    graph2.replay()
+    torch.cuda.synchronize()
+    assert torch.equal(out_1, ref_1)
+    assert cache.stats()["device_timeouts"] == 0
+    cache.close()
