@@ -1382,6 +1382,19 @@ __global__ void __launch_bounds__(kBlockThreads, 2) block_tc_kernel(const __grid
     const PlanEntry e = reinterpret_cast<const PlanEntry *>(a.plan + a.plan_entry)[entry];
     const HeadUnits hu = head_units(geo, e);
     const int T = a.n_tokens[(long long)e.seq * geo.n_layers + a.layer];
+    // Units are in token order and the block's last row sees the most: units that start after what it sees are
+    // hidden from every row of the block and are left out (producer and consumers agree on the count).
+    int n_units = hu.units;
+    {
+        const int last_row = min(n_rows, (rb + 1) * kBlockRows) - 1;
+        const int vis = T - (a.q_len - 1 - last_row / G);                 // tokens the last row sees (>= 1)
+        const int page = (vis - 1) / P, blk = ((vis - 1) % P) / kDB;
+        int need;
+        if (page < hu.fb) need = page * geo.blocks_per_page + blk + 1;
+        else if (page < hu.fe) need = hu.d0 + hu.nf;
+        else need = hu.d0 + hu.nf + (page - hu.fe) * geo.blocks_per_page + blk + 1;
+        n_units = max(1, min(need, hu.units));
+    }
 
     if (warp == kBlockWarps) {
         // ------------------------------ producer (one lane) ------------------------------
@@ -1389,7 +1402,7 @@ __global__ void __launch_bounds__(kBlockThreads, 2) block_tc_kernel(const __grid
         const int *pt = a.page_table + ((long long)e.seq * geo.n_layers + a.layer) * geo.max_pages;
         bool ok = true;
         int u = 0;
-        for (; u < hu.units && ok; ++u) {
+        for (; u < n_units && ok; ++u) {
             const int s = u % S;
             if (u >= S && !mbar_wait(smem_u32(empty_bar + s), ((u / S) - 1) & 1)) { ok = false; break; }
             int page, blk, kind;
@@ -1461,7 +1474,7 @@ __global__ void __launch_bounds__(kBlockThreads, 2) block_tc_kernel(const __grid
     st.m[0] = st.m[1] = kNegInf;
     st.l[0] = st.l[1] = 0.f;
     bool ok = true;
-    for (int u = 0; u < hu.units; ++u) {
+    for (int u = 0; u < n_units; ++u) {
         const int s = u % S;
         // The only way out is this warp's own wait running out: if the producer gave up, every warp ends up at the
         // same unarmed unit, so no warp is left alone at the block barrier below.
