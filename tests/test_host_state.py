@@ -166,6 +166,37 @@ def test_two_step_compression_schedule_matches_oracle_bit_exact(seed):
     assert gpu.stats()["pages_compressed"] == orc.pages_compressed > 0
 
 
+def test_two_step_compression_when_the_factor_pool_runs_out():
+    """pkv_compress_begin with fewer free factor slots than eligible pages: the pages that got a slot are begun (and
+    reported), the call returns PKV_ERR_POOL_EXHAUSTED, the commit converts exactly those, and a later begin picks up
+    the rest once slots are free again.  Same tables as the oracle throughout."""
+    gpu, orc, base = _pair(n_layers=1, max_seqs=2, n_dense_slots=64, n_factor_slots=5, sink_tokens=64, recent_tokens=64)
+    H = base["n_kv_heads"]
+    _oracle_append(orc, 0, [0, 1], [64 * 6, 64 * 7], H)
+    gpu.append_kv(0, [0, 1], [64 * 6, 64 * 7])             # eligible: pages 1..4 of sequence 0, 1..5 of sequence 1
+    with pytest.raises(pkv.PkvError) as e:
+        gpu.compress_begin(0)
+    assert e.value.status == pkv.PKV_ERR_POOL_EXHAUSTED and e.value.begun == 5
+    assert orc.compress_begin(0) == 5
+    _same_tables(gpu, orc, base)                            # nothing visible yet
+    with pytest.raises(pkv.PkvError) as e:
+        gpu.compress_begin(0)                               # still uncommitted
+    assert e.value.status == pkv.PKV_ERR_UNSUPPORTED
+    assert gpu.compress_commit(0) == orc.compress_commit(0) == 5
+    _same_tables(gpu, orc, base)
+    assert gpu.page_table(0, 0)[0][:6] == [0, 1, 1, 1, 1, 0] and gpu.page_table(1, 0)[0][:3] == [0, 1, 0]
+    with pytest.raises(pkv.PkvError) as e:
+        gpu.compress_begin(0)                               # no factor slot left at all
+    assert e.value.status == pkv.PKV_ERR_POOL_EXHAUSTED and e.value.begun == 0
+    assert gpu.compress_commit(0) == 0
+    orc.free_seq(0)
+    gpu.free_seq(0)                                         # four factor slots come back
+    assert gpu.compress_begin(0) == orc.compress_begin(0) == 4
+    assert gpu.compress_commit() == orc.compress_commit() == 4
+    _same_tables(gpu, orc, base)
+    assert gpu.page_table(1, 0)[0][:7] == [0, 1, 1, 1, 1, 1, 0]
+
+
 def test_incremental_conversion_is_one_page_per_boundary_step():
     gpu, orc, base = _pair(n_layers=1, max_seqs=2, sink_tokens=64, recent_tokens=256)
     gpu.append_kv(0, [0, 1], [8192 // 16, 8192 // 16])
