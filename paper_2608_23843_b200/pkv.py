@@ -129,15 +129,21 @@ def _ints(xs):
 
 
 def _ptr(t):
-    return None if t is None else ctypes.c_void_p(t.data_ptr())
+    """Device (or host) address of a tensor as a plain int: ctypes converts it for a void* parameter, and building
+    a c_void_p object per argument is a measurable part of a 5 us call."""
+    return None if t is None else t.data_ptr()
 
 
 def _stream(stream):
-    if stream is None:
-        return None
-    if isinstance(stream, int):
-        return ctypes.c_void_p(stream)
-    return ctypes.c_void_p(stream.cuda_stream)
+    if stream is None or isinstance(stream, int):
+        return stream
+    return stream.cuda_stream
+
+
+try:                                                     # raw handle of the current stream without a Stream object (2 us less per call)
+    _raw_current_stream = torch._C._cuda_getCurrentRawStream
+except AttributeError:                                   # pragma: no cover
+    _raw_current_stream = None
 
 
 # ---- functions with the C names -------------------------------------------------
@@ -330,14 +336,23 @@ class Cache:
             self.stream = None
         else:
             self.device = torch.device(device)
+            self._device_index = self.dense_pool_device_index(self.device)
             mk = lambda n: torch.empty(max(int(n), 256), dtype=torch.uint8, device=self.device)
             self.dense_pool, self.factor_pool = mk(self.sizes.dense_pool_bytes), mk(self.sizes.factor_pool_bytes)
             self.meta, self.workspace = mk(self.sizes.meta_bytes), mk(self.sizes.workspace_bytes)
         self.handle = pkv_init_cache(cfg, self.dense_pool, self.factor_pool, self.meta, self.workspace,
                                      dense_slot_order, factor_slot_order)
 
+    @staticmethod
+    def dense_pool_device_index(device):
+        return device.index if device.index is not None else torch.cuda.current_device()
+
     def _st(self):
-        return None if self.dry_run else torch.cuda.current_stream(self.device)
+        if self.dry_run:
+            return None
+        if _raw_current_stream is not None:
+            return _raw_current_stream(self._device_index)
+        return torch.cuda.current_stream(self.device)
 
     def append_kv(self, layer, seq_ids, n_new, k=None, v=None):
         pkv_append_kv(self.handle, layer, seq_ids, n_new, k, v, self._st())
