@@ -64,13 +64,15 @@ __device__ __forceinline__ void unit_to_page(const Geometry &g, const HeadUnits 
 }
 
 __device__ __forceinline__ bool load_range(const DecodeArgs &a, Range &r) {
-    const PlanHeader hdr = *reinterpret_cast<const PlanHeader *>(a.plan);
-    r.n_used = hdr.n_used_ctas;
-    if ((int)blockIdx.x >= hdr.n_used_ctas) return false;
+    // All four loads are issued together (the arrays have an element for every CTA of the grid, used or not), so
+    // that the header's latency is not paid a second time before the CTA knows its range.
     const PlanCta *ctas = reinterpret_cast<const PlanCta *>(a.plan + a.plan_cta);
+    const PlanHeader hdr = *reinterpret_cast<const PlanHeader *>(a.plan);
     r.start = ctas[blockIdx.x];
     r.end = ctas[blockIdx.x + 1];
     r.first_entry = reinterpret_cast<const PlanEntry *>(a.plan + a.plan_cta_entry)[blockIdx.x];
+    r.n_used = hdr.n_used_ctas;
+    if ((int)blockIdx.x >= hdr.n_used_ctas) return false;
     const int H = a.geo.n_kv_heads;
     r.seg_first = r.start.entry * H + r.start.head;
     int seg_last = r.end.entry * H + r.end.head;
