@@ -120,8 +120,8 @@ typedef struct pkv_config {
                                       library rotates the split-K scratch over n sets (n = 64, fewer where 64 sets
                                       would exceed 128 MiB of workspace, at least 4) and makes every (n-1)-th
                                       launch an ordinary one, which starts only after all earlier work on the
-                                      stream has finished.  Not capturable into a CUDA graph (the call returns
-                                      PKV_ERR_UNSUPPORTED while the stream is capturing).
+                                      stream has finished.  May be recorded into CUDA graphs (see
+                                      pkv_decode_attention).
                                    Work enqueued after a decode call by any other means (another kernel, a copy)
                                    still starts only after that call has completed, in every mode, and a decode
                                    call that follows a pkv_append_kv or pkv_compress_eligible_pages call on this
@@ -242,14 +242,16 @@ pkv_status pkv_compress_commit(pkv_cache *c, int32_t layer, void *main_stream, i
  * Scores use softmax_scale; accumulation is fp32.  The result does not depend
  * on physical slot placement and is bit-identical from run to run.
  *
- * CUDA graphs: with decode_overlap 0 or 1 the call may be recorded into a graph, provided this layer's plan for
+ * CUDA graphs: the call may be recorded into a graph (any decode_overlap), provided this layer's plan for
  * this batch is current, i.e. the same call has been made once outside the capture since the last change of the
  * batch's page tables (otherwise PKV_ERR_UNSUPPORTED: the plan cannot be uploaded from inside a capture).  A
  * replay reads token counts, page tables and the plan from device memory when it runs: appends that stay inside a
  * sequence's current page need nothing; after an append that opens a page, a compression or a free, one such call
  * outside a capture brings the plan up to date and existing graphs for the same batch are valid again.
  * pkv_append_kv and pkv_compress_eligible_pages update host-side state and cannot be captured (PKV_ERR_UNSUPPORTED
- * while the stream is capturing).
+ * while the stream is capturing).  With decode_overlap = 2 a recorded launch keeps its scratch set in every replay:
+ * launches inside a graph overlap as they do outside, consecutive graph launches are ordered by the stream, and
+ * from the first capture on, this cache's launches outside a graph are ordinary (non-overlapping) ones.
  */
 pkv_status pkv_decode_attention(pkv_cache *c, int32_t layer, int32_t n_seqs, const int32_t *seq_ids,
                                 const void *q, void *out, float *out_f32, void *stream);

@@ -91,6 +91,7 @@ struct pkv_cache {
     int64_t last_decode_bytes = 0, last_decode_units = 0;
     uint64_t decode_seq = 0;           // decode launches so far (decode_overlap = 2: picks the scratch buffer)
     bool cache_written = true;         // an append or compression kernel was enqueued since the last decode launch
+    bool captured_mode2 = false;       // a decode_overlap = 2 launch has been recorded into a CUDA graph
     std::vector<PendingCompress> pending;   // [n_layers]
     int n_pending = 0;                 // layers with a begun, uncommitted compression
     cudaEvent_t order_ev = nullptr;    // scratch event: orders a side stream behind the caller's main stream
@@ -929,10 +930,14 @@ static pkv_status decode_impl(pkv_cache *c, int32_t layer, int32_t n_seqs, const
         return PKV_OK;
     }
     if (c->cfg.decode_overlap == 2 && c->cfg.decode_variant != 1) {
+        // Recorded into a CUDA graph, a launch keeps the set chosen here in every replay.  That is sound inside a
+        // graph (same rotation, same draining launches) and between graph launches (each starts after the previous
+        // one has finished); a launch outside a graph could however meet a set that a graph's last launches still
+        // use, so once this cache has been captured its launches outside a graph are ordinary ones.
         cudaStreamCaptureStatus cap = cudaStreamCaptureStatusNone;
         PKV_CUDA(c, cudaStreamIsCapturing(st, &cap));
-        if (cap != cudaStreamCaptureStatusNone)
-            return fail(c, PKV_ERR_UNSUPPORTED, "decode_overlap = 2 cannot be captured into a CUDA graph (use 0 or 1)");
+        if (cap != cudaStreamCaptureStatusNone) c->captured_mode2 = true;
+        else if (c->captured_mode2) a.plain_launch = 1;
         buf = (int)(c->decode_seq % c->wl.n_sets);
         if ((c->decode_seq % (c->wl.n_sets - 1)) == 0) a.plain_launch = 1;
         c->decode_seq++;

@@ -123,7 +123,7 @@ def test_cuda_graph_replay_sees_appends_and_rebuilt_plans(overlap):
     """Decode launches recorded into a CUDA graph read token counts, page tables and the plan when they run:
     a replay after an in-page append equals a fresh eager call; after an append that opens a page plus a
     compression, one eager call rebuilds the plan and the old graph is valid again.  Calls that cannot be
-    recorded (append, compress, a decode whose plan is stale, mode 2) return PKV_ERR_UNSUPPORTED during capture
+    recorded (append, compress, a decode whose plan is stale) return PKV_ERR_UNSUPPORTED during capture
     and leave the capture usable."""
     L, H, G = 2, 2, 4
     cfg = pkv.make_config(n_layers=L, n_kv_heads=H, n_q_heads=H * G, rank=16, sink_tokens=64, recent_tokens=128,
@@ -199,27 +199,57 @@ def test_cuda_graph_replay_sees_appends_and_rebuilt_plans(overlap):
 
 
 @pytest.mark.gpu
-def test_mode_2_refuses_stream_capture():
-    cfg = pkv.make_config(n_layers=1, n_kv_heads=1, n_q_heads=4, rank=16, sink_tokens=64, recent_tokens=128,
-                          max_seqs=1, max_pages_per_seq=8, n_dense_slots=8, n_factor_slots=8, decode_overlap=2)
-    cache = pkv.Cache(cfg, "cuda", None, None)
-    k, v = synth.make_kv(22, 0, 0, 300, 1, 128, 64, "cuda")
-    cache.append_kv(0, [0], [300], k, v)
-    q = synth.make_q(22, 0, 0, 1, 4, 128, "cuda")
-    out = torch.empty_like(q)
-    cache.decode_attention(0, [0], q, out)
+def test_mode_2_launches_in_a_cuda_graph():
+    """decode_overlap = 2 recorded into a graph: 70 launches over three layers (more than the 64 scratch sets, so the
+    graph contains a draining launch) reproduce, in every replay and bit for bit, what a cache with decode_overlap = 0
+    computes; launches outside a graph still work afterwards (as ordinary launches), also between replays."""
+    L, H, G = 3, 2, 4
+    kw = dict(n_layers=L, n_kv_heads=H, n_q_heads=H * G, rank=24, sink_tokens=64, recent_tokens=128, max_seqs=3,
+              max_pages_per_seq=40, n_dense_slots=300, n_factor_slots=300)
+    fast, slow = pkv.Cache(pkv.make_config(decode_overlap=2, **kw), "cuda"), pkv.Cache(pkv.make_config(decode_overlap=0, **kw), "cuda")
+    lengths = [2100, 130, 900]
+    for ly in range(L):
+        for s_, T in enumerate(lengths):
+            k, v = synth.make_kv(23, ly, s_, T, H, 128, 64, "cuda")
+            for c in (fast, slow):
+                c.append_kv(ly, [s_], [T], k, v)
+    for c in (fast, slow):
+        c.compress_eligible_pages(-1)
+    ids = [2, 0, 1]
+    n_launch = 70
+    qs = [synth.make_q(23, i % L, i, 3, H * G, 128, "cuda") for i in range(n_launch)]
+    ref = [torch.empty_like(q) for q in qs]
+    for i in range(n_launch):
+        slow.decode_attention(i % L, ids, qs[i], ref[i])
+    outs = [torch.empty_like(q) for q in qs]
+    for ly in range(L):
+        fast.decode_attention(ly, ids, qs[ly], outs[ly])    # plans built outside the capture
     torch.cuda.synchronize()
     side = torch.cuda.Stream()
     side.wait_stream(torch.cuda.current_stream())
     graph = torch.cuda.CUDAGraph()
     with torch.cuda.stream(side):
         with torch.cuda.graph(graph, stream=side):
-            with pytest.raises(pkv.PkvError) as e:
-                cache.decode_attention(0, [0], q, out)
-            assert e.value.status == pkv.PKV_ERR_UNSUPPORTED
-            torch.zeros(4, device="cuda")                    # the capture itself is still alive
+            for i in range(n_launch):
+                fast.decode_attention(i % L, ids, qs[i], outs[i])
     torch.cuda.current_stream().wait_stream(side)
-    cache.close()
+    for rep in range(3):
+        for o in outs:
+            o.zero_()
+        graph.replay()
+        if rep == 1:                                            # a launch outside the graph right behind a replay
+            extra = torch.empty_like(qs[0])
+            fast.decode_attention(0, ids, qs[0], extra)
+        graph.replay()
+        torch.cuda.synchronize()
+        for i in range(n_launch):
+            assert torch.equal(outs[i], ref[i]), (rep, i)
+        if rep == 1:
+            assert torch.equal(extra, ref[0])
+    st = fast.stats()
+    assert st["device_timeouts"] == 0 and st["bad_slot_indices"] == 0
+    fast.close()
+    slow.close()
 
 
 @pytest.mark.parametrize("bits", [16, 4])
