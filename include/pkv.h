@@ -267,13 +267,16 @@ pkv_status pkv_decode_attention(pkv_cache *c, int32_t layer, int32_t n_seqs, con
  * Requirements (else PKV_ERR_INVALID_ARG, nothing launched): 1 <= q_len <= T for every listed sequence; no listed
  * sequence has a factor page that reaches past token T - q_len (so every query sees every factor page whole:
  * holds whenever q_len <= recent_tokens and compression ran no later than the append of these positions, and it is
- * checked per call); n_seqs * ceil(q_len / max(1, 8 / (H_q / H_kv))) <= max_seqs, the number of plan entries.
+ * checked per call); n_seqs * ceil(q_len / max(1, 8 / (H_q / H_kv))) <= max_seqs (split-K partial states and
+ * tickets are kept per sequence and block of query tokens).
  * Two kernels serve this call.  A row-block kernel - one CTA per (sequence, KV head, 64 query rows), which reads the
  * sequence's pages once for its 64 rows (tensor-core products with the query rows as the 16-row operand) - runs
  * when q_len * (H_q / H_kv) >= 64, the factors are bf16, and the call makes at least 128 such CTAs (enough to fill
- * the GPU) or would exceed the plan-entry limit above, which does not apply to this kernel.  Otherwise the decode
- * kernel takes 8 / (H_q / H_kv) query tokens per pass over the pages, so the KV bytes read grow with the number of
- * such passes.  Both give the same result up to fp32 summation order.
+ * the GPU) or would exceed the limit above, which does not apply to this kernel.  Otherwise the decode kernel runs
+ * with its CTAs in groups of b = ceil(q_len / max(1, 8 / (H_q / H_kv))): the CTAs of a group walk the same pages at
+ * the same time, one block of 8 / (H_q / H_kv) query tokens each, so HBM delivers a page once and L2 delivers it b
+ * times (q_len = 2 at H_q / H_kv = 8 costs 1.3 single-query launches, q_len = 2 at H_q / H_kv = 4 costs one).
+ * Both kernels give the same result up to fp32 summation order.
  * Needs decode_variant 0 or 2 (PKV_ERR_UNSUPPORTED with 1).  CUDA-graph and overlap semantics as for
  * pkv_decode_attention(); a layer keeps one plan, that of its most recent (batch, q_len), so calls that
  * alternate between shapes on one layer rebuild it each time (host work and a small upload; not capturable).

@@ -348,8 +348,11 @@ int first_unit_at_or_after(const HeadShape &h, long long rem, long long cf, long
 int queries_per_tile(const Geometry &g, int q_len) { return std::max(1, std::min(q_len, kMaxGroup / g.group)); }
 int entries_per_seq(const Geometry &g, int q_len) { const int t = queries_per_tile(g, q_len); return (q_len + t - 1) / t; }
 
-// `n_listed` sequences with q_len queries each: every sequence takes entries_per_seq() consecutive plan entries
-// (one per block of query tokens), each of which walks all the sequence's pages.
+// `n_listed` sequences with q_len queries each.  The plan always covers the sequences once: with
+// entries_per_seq() = b > 1 query blocks per sequence, the (sequence, KV head, unit) order is cut into at most
+// n_ctas / b ranges and the launch's CTAs work in groups of b on one range each, one query block per CTA.  The
+// partial states and tickets are then counted per (sequence, query block, KV head), which is why
+// n_listed * b <= max_seqs is required.
 // Whether a call with q_len queries for each of n_seqs sequences goes to the row-block kernel (one CTA per 64 query
 // rows of a KV head, which walks the whole sequence alone) instead of the pipeline kernel (eight query columns per
 // pass over the pages, split over all CTAs).  The row-block kernel needs enough CTAs to fill the GPU; below that the
@@ -364,16 +367,17 @@ bool uses_row_blocks(const pkv_cache *c, int q_len, int n_seqs) {
 pkv_status build_plan(pkv_cache *c, int layer, int n_listed, const int32_t *seq_ids, int q_len, cudaStream_t st) {
     const Geometry &g = c->geo;
     PlanCache &pc = c->plans[layer];
-    const int H = g.n_kv_heads, N = g.n_ctas;
+    const int H = g.n_kv_heads;
     const long long cf = g.blob_bytes + 2048, cd = (long long)g.block_tokens * 2 * kRowBytes + 2048;
-    // the row-block kernel only reads the entries (one per listed sequence); the split over CTAs is not used
-    const int per_seq = uses_row_blocks(c, q_len, n_listed) ? 1 : entries_per_seq(g, q_len), n_seqs = n_listed * per_seq;
+    // (the row-block kernel only reads the entries; the split over CTAs is not used by it)
+    const int groups = uses_row_blocks(c, q_len, n_listed) ? 1 : entries_per_seq(g, q_len);
+    const int N = std::max(1, g.n_ctas / groups), n_seqs = n_listed;
 
     std::vector<PlanEntry> entries(n_seqs);
     std::vector<HeadShape> shapes(n_seqs);
     long long total_cost = 0, total_units = 0;
     for (int i = 0; i < n_seqs; ++i) {
-        const int32_t seq = seq_ids[i / per_seq];
+        const int32_t seq = seq_ids[i];
         const SeqLayer &s = c->at(seq, layer);
         int n_pages = (s.n_tokens + c->cfg.page_size - 1) / c->cfg.page_size;
         entries[i] = PlanEntry{seq, n_pages, g.sink_pages, s.f_end};
@@ -861,9 +865,10 @@ static pkv_status decode_impl(pkv_cache *c, int32_t layer, int32_t n_seqs, const
     if (q_len > 1) {
         if (c->cfg.decode_variant == 1)
             return fail(c, PKV_ERR_UNSUPPORTED, "several queries per sequence need the tensor-core kernels (decode_variant 0)");
-        if (!uses_row_blocks(c, q_len, n_seqs) && (long long)n_seqs * entries_per_seq(c->geo, q_len) > c->cfg.max_seqs)
-            return fail(c, PKV_ERR_INVALID_ARG, "%d sequences x %d query blocks exceed max_seqs = %d plan entries", n_seqs,
-                        entries_per_seq(c->geo, q_len), c->cfg.max_seqs);
+        if (!uses_row_blocks(c, q_len, n_seqs) && ((long long)n_seqs * entries_per_seq(c->geo, q_len) > c->cfg.max_seqs ||
+                                                   entries_per_seq(c->geo, q_len) > c->geo.n_ctas))
+            return fail(c, PKV_ERR_INVALID_ARG, "%d sequences x %d query blocks exceed max_seqs = %d (or the blocks the %d CTAs)",
+                        n_seqs, entries_per_seq(c->geo, q_len), c->cfg.max_seqs, c->geo.n_ctas);
         for (int i = 0; i < n_seqs; ++i) {
             const SeqLayer &s = c->at(seq_ids[i], layer);
             // every query must see every factor page whole (and at least its own position)

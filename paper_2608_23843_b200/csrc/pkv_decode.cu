@@ -66,13 +66,17 @@ __device__ __forceinline__ void unit_to_page(const Geometry &g, const HeadUnits 
 __device__ __forceinline__ bool load_range(const DecodeArgs &a, Range &r) {
     // All four loads are issued together (the arrays have an element for every CTA of the grid, used or not), so
     // that the header's latency is not paid a second time before the CTA knows its range.
+    // With several query blocks per sequence (q_nblk > 1) the CTAs come in groups of q_nblk that share a range:
+    // CTA b walks range b / q_nblk for query block b % q_nblk.  The siblings start together and read the same
+    // pages in the same order, so all but the first find them in L2.
+    const int range = blockIdx.x / a.q_nblk;
     const PlanCta *ctas = reinterpret_cast<const PlanCta *>(a.plan + a.plan_cta);
     const PlanHeader hdr = *reinterpret_cast<const PlanHeader *>(a.plan);
-    r.start = ctas[blockIdx.x];
-    r.end = ctas[blockIdx.x + 1];
-    r.first_entry = reinterpret_cast<const PlanEntry *>(a.plan + a.plan_cta_entry)[blockIdx.x];
+    r.start = ctas[range];
+    r.end = ctas[range + 1];
+    r.first_entry = reinterpret_cast<const PlanEntry *>(a.plan + a.plan_cta_entry)[range];
     r.n_used = hdr.n_used_ctas;
-    if ((int)blockIdx.x >= hdr.n_used_ctas) return false;
+    if (range >= hdr.n_used_ctas) return false;
     const int H = a.geo.n_kv_heads;
     r.seg_first = r.start.entry * H + r.start.head;
     int seg_last = r.end.entry * H + r.end.head;
@@ -692,8 +696,22 @@ __device__ __forceinline__ void reset_state(WarpState &st) {
     st.l[0] = st.l[1] = 0.f;
 }
 
+// Index of (sequence, query block, KV head) - what q, out and the tickets are indexed by - for segment `seg` of the
+// plan, which is (sequence, KV head); the query block is this CTA's.
+__device__ __forceinline__ int query_seg(const DecodeArgs &a, int seg) {
+    if (a.q_nblk == 1) return seg;
+    const int H = a.geo.n_kv_heads;
+    return ((seg / H) * a.q_nblk + (int)(blockIdx.x % a.q_nblk)) * H + seg % H;
+}
+// This CTA's partial state of segment `seg`, or with `cta` = the segment's first range, the first of its partial
+// states; consecutive ranges' states of one query block are q_nblk slots apart.
+__device__ __forceinline__ float *partial_slot(const DecodeArgs &a, int cta_range, int seg) {
+    return a.partials + (((long long)cta_range + seg) * a.q_nblk + blockIdx.x % a.q_nblk) * kPartialFloats;
+}
+
 // Query column n of a segment's score tile = query head n % G of the (n / G)-th query token of the plan entry's
 // block; with one query per sequence (q_len = 1) that is query head n.  Row of q / out it maps to, or -1.
+// (`seg` here is a query_seg() index.)
 __device__ __forceinline__ long long q_row(const DecodeArgs &a, int seg, int n) {
     const int H = a.geo.n_kv_heads, G = a.geo.group;
     const int entry = seg / H, head = seg % H, jl = n / G, j = (entry % a.q_nblk) * a.q_tpt + jl;
@@ -750,6 +768,7 @@ __device__ __forceinline__ void store_out(const DecodeArgs &a, int seg, int hq, 
 // time, because with dozens of parts it is the latency of these loads that the rest of the GPU waits for.
 template <int E, int kBatch>
 __device__ __forceinline__ void merge_parts(const DecodeArgs &a, const float *first, int np, int seg, int ctid) {
+    const long long stride = (long long)a.q_nblk * kPartialFloats;      // between the states of consecutive ranges
     constexpr int kThreads = kConsumerWarps * 32;
     const int n_items = a.q_cols * 32;
     const int d4 = (ctid & 31) * 4;                               // kThreads is a multiple of 32
@@ -770,7 +789,7 @@ __device__ __forceinline__ void merge_parts(const DecodeArgs &a, const float *fi
         float m[E][kBatch], l[E][kBatch];
 #pragma unroll
         for (int j = 0; j < kBatch; ++j) {
-            const float *pk = first + (long long)min(k0 + j, np - 1) * kPartialFloats;
+            const float *pk = first + (long long)min(k0 + j, np - 1) * stride;
 #pragma unroll
             for (int e = 0; e < E; ++e) {
                 o[e][j] = __ldcg(reinterpret_cast<const float4 *>(pk + hq[e] * kHeadDim + d4));
@@ -834,7 +853,8 @@ __device__ __forceinline__ void flush_segment(const DecodeArgs &a, float *comb, 
     // overlap mode 1: partial states, tickets and `out` may still be in use by the preceding launch
     if (a.overlap == 1) asm volatile("griddepcontrol.wait;" ::: "memory");
     const PlanSeg ps = reinterpret_cast<const PlanSeg *>(a.plan + a.plan_seg)[seg];
-    float *part = a.partials + ((long long)blockIdx.x + seg) * kPartialFloats;
+    const int qseg = query_seg(a, seg);
+    float *part = partial_slot(a, blockIdx.x / a.q_nblk, seg);
     for (int item = ctid; item < kItems; item += kThreads) {
         const int hq = item >> 5, d4 = (item & 31) * 4;
         float M = kNegInf;
@@ -849,7 +869,7 @@ __device__ __forceinline__ void flush_segment(const DecodeArgs &a, float *comb, 
             L += f * cw[kMaxGroup * kHeadDim + kMaxGroup + hq];
         }
         if (ps.n_parts <= 1) {
-            if (hq < a.q_cols) store_out(a, seg, hq, d4, acc, M, L);
+            if (hq < a.q_cols) store_out(a, qseg, hq, d4, acc, M, L);
         } else {
             *reinterpret_cast<float4 *>(part + hq * kHeadDim + d4) = acc;
             if ((item & 31) == 0) {
@@ -861,14 +881,14 @@ __device__ __forceinline__ void flush_segment(const DecodeArgs &a, float *comb, 
     if (ps.n_parts > 1) {
         __threadfence();
         PKV_CONSUMER_BARRIER();
-        if (ctid == 0) *last_flag = (atomicAdd(a.tickets + seg, 1) == ps.n_parts - 1);
+        if (ctid == 0) *last_flag = (atomicAdd(a.tickets + qseg, 1) == ps.n_parts - 1);
         PKV_CONSUMER_BARRIER();
         if (*last_flag) {
             __threadfence();
-            const float *first = a.partials + ((long long)ps.cta_first + seg) * kPartialFloats;
-            if (a.q_cols * 32 <= kThreads) merge_parts<1, 16>(a, first, ps.n_parts, seg, ctid);
-            else merge_parts<2, 8>(a, first, ps.n_parts, seg, ctid);
-            if (ctid == 0) a.tickets[seg] = 0;          // ready for the next launch
+            const float *first = partial_slot(a, ps.cta_first, seg);
+            if (a.q_cols * 32 <= kThreads) merge_parts<1, 16>(a, first, ps.n_parts, qseg, ctid);
+            else merge_parts<2, 8>(a, first, ps.n_parts, qseg, ctid);
+            if (ctid == 0) a.tickets[qseg] = 0;         // ready for the next launch
         }
     }
     PKV_CONSUMER_BARRIER();
@@ -935,6 +955,7 @@ __global__ void __launch_bounds__(kDecodeThreads, 2) decode_tc_kernel(const __gr
         const PlanEntry *entries = reinterpret_cast<const PlanEntry *>(a.plan + a.plan_entry);
         int k = 0, seg_local = 0;
         bool ok = true;
+        const bool keep = a.q_nblk > 1;      // sibling CTAs read the same pages: leave them in L2 for one another
         PlanCta cur = rg.start;
         while (ok && !(cur.entry == rg.end.entry && cur.head == rg.end.head && cur.unit == rg.end.unit)) {
             const PlanEntry e = cur.entry == rg.start.entry ? rg.first_entry : entries[cur.entry];
@@ -982,11 +1003,17 @@ __global__ void __launch_bounds__(kDecodeThreads, 2) decode_tc_kernel(const __gr
                             const uint32_t dst = smem_u32(stages + (size_t)s * stage_bytes);
                             if (kind == kKindFactor) {
                                 mbar_arrive_expect_tx(bar, blob_bytes);
-                                bulk_g2s(dst, src, blob_bytes, bar);
+                                if (keep) bulk_g2s_keep(dst, src, blob_bytes, bar);
+                                else bulk_g2s(dst, src, blob_bytes, bar);
                             } else if (rows > 0) {
                                 mbar_arrive_expect_tx(bar, 2 * rows * kRowBytes);
-                                bulk_g2s(dst, src, rows * kRowBytes, bar);
-                                bulk_g2s(dst + kDB * kRowBytes, src + P * kRowBytes, rows * kRowBytes, bar);
+                                if (keep) {
+                                    bulk_g2s_keep(dst, src, rows * kRowBytes, bar);
+                                    bulk_g2s_keep(dst + kDB * kRowBytes, src + P * kRowBytes, rows * kRowBytes, bar);
+                                } else {
+                                    bulk_g2s(dst, src, rows * kRowBytes, bar);
+                                    bulk_g2s(dst + kDB * kRowBytes, src + P * kRowBytes, rows * kRowBytes, bar);
+                                }
                             } else {
                                 mbar_arrive(bar);
                             }
@@ -1038,7 +1065,7 @@ __global__ void __launch_bounds__(kDecodeThreads, 2) decode_tc_kernel(const __gr
         }
         uint32_t qf[8][2];
         int cur_seg = 0;
-        int hidden = load_q(a, rg.seg_first, qf, lane);
+        int hidden = load_q(a, query_seg(a, rg.seg_first), qf, lane);
         bool ok = true;
         for (int k = warp;; k += W) {
             const int s = k % S;
@@ -1052,7 +1079,7 @@ __global__ void __launch_bounds__(kDecodeThreads, 2) decode_tc_kernel(const __gr
             if (cur_seg < dsc.seg) {
                 // the old segment's queries are no longer needed: fetch the new ones now, so that their latency
                 // hides behind the flush
-                if (dsc.seg < rg.n_local_segs) hidden = load_q(a, rg.seg_first + dsc.seg, qf, lane);
+                if (dsc.seg < rg.n_local_segs) hidden = load_q(a, query_seg(a, rg.seg_first + dsc.seg), qf, lane);
                 while (cur_seg < dsc.seg) {
                     flush_segment(a, comb, last_flag, st, rg.seg_first + cur_seg, warp, lane, tid, W);
                     ++cur_seg;
