@@ -184,7 +184,8 @@ class ClockSampler:
         return out
 
 
-def build_workload(w, rank, device, overlap=2, n_ctas=0, factor_bits=16, grow=0, keep_kv=False, plan_entries_per_seq=1):
+def build_workload(w, rank, device, overlap=2, n_ctas=0, factor_bits=16, grow=0, keep_kv=False, plan_entries_per_seq=1,
+                   decode_variant=0):
     """Allocate the cache, generate each (layer, sequence) on the GPU, append and compress layer by layer.
     grow: tokens every sequence may still gain afterwards (sizes the pools and page tables); keep_kv: also
     return the generated K/V of layer 0 including those `grow` tokens (serving loop)."""
@@ -206,7 +207,8 @@ def build_workload(w, rank, device, overlap=2, n_ctas=0, factor_bits=16, grow=0,
                           rank_v=w.get("rank_v", rank), page_size=P,
                           sink_tokens=w["sink"], recent_tokens=w["recent"], max_seqs=w["batch"] * plan_entries_per_seq,
                           max_pages_per_seq=max(pages), n_dense_slots=n_dense_slots, n_factor_slots=n_factor_slots,
-                          decode_overlap=overlap, n_ctas=n_ctas, factor_bits=factor_bits)
+                          decode_overlap=overlap, n_ctas=n_ctas, factor_bits=factor_bits,
+                          decode_variant=decode_variant)
     cache = pkv.Cache(cfg, device, synth.slot_permutation(SEED, n_dense_slots, 0).tolist(),
                       synth.slot_permutation(SEED, n_factor_slots, 1).tolist())
     ids = list(range(w["batch"]))
@@ -486,6 +488,8 @@ def main():
                     help="strong scaling of one step: every rank's cache holds 1/N of each sequence's tokens (rank 0 the "
                          "sink, the last rank the dense window); per layer each rank computes its softmax state, the states "
                          "are all-gathered (NCCL) and merged by Eq. 5.  Not the default: the driver's scaling runs are replicas")
+    ap.add_argument("--decode-variant", type=int, default=0, choices=[0, 2],
+                    help="2 = pkv_decode_attention_multi never uses its row-block kernel (comparisons)")
     ap.add_argument("--graph", action="store_true",
                     help="replay one CUDA graph per step instead of launching every layer from the host")
     args = ap.parse_args()
@@ -523,7 +527,7 @@ def main():
     QL = args.q_len
     per_tile = max(1, min(QL, 8 // (w["n_q_heads"] // w["n_kv_heads"])))
     cfg, cache, lengths, comp = build_workload(w, rank, device, args.overlap, args.n_ctas, args.factor_bits,
-                                               plan_entries_per_seq=-(-QL // per_tile))
+                                               plan_entries_per_seq=-(-QL // per_tile), decode_variant=args.decode_variant)
     ids = list(range(w["batch"]))
     L, Hq = w["n_layers"], w["n_q_heads"]
     if QL == 1:
@@ -661,7 +665,7 @@ def main():
         }
         P_, Gq = w.get("page", 64), Hq // w["n_kv_heads"]
         rows = QL * Gq
-        if QL > 1 and args.factor_bits != 4 and rows >= 64 and w["batch"] * w["n_kv_heads"] * -(-rows // 64) >= 128:
+        if QL > 1 and args.decode_variant == 0 and args.factor_bits != 4 and rows >= 64 and w["batch"] * w["n_kv_heads"] * -(-rows // 64) >= 128:
             # Served by the row-block kernel, whose bound is the tensor pipe, not HBM: algorithmic FLOPs per launch =
             # query rows x (factor pages x 2 (d r_k + r_k P + P r_v + r_v d) + dense tokens x 4 d); the causal
             # triangle among the new positions is counted in full.
