@@ -347,12 +347,18 @@ int first_unit_at_or_after(const HeadShape &h, long long rem, long long cf, long
 // Query tokens that share one score tile (eight query columns), and plan entries per sequence.
 int queries_per_tile(const Geometry &g, int q_len) { return std::max(1, std::min(q_len, kMaxGroup / g.group)); }
 int entries_per_seq(const Geometry &g, int q_len) { const int t = queries_per_tile(g, q_len); return (q_len + t - 1) / t; }
+// Sibling CTAs per plan range (at most the grid), and plan entries ("passes") per sequence that this leaves.
+int sibling_group(const Geometry &g, int q_len) { return std::max(1, std::min(entries_per_seq(g, q_len), g.n_ctas)); }
+int passes_per_seq(const Geometry &g, int q_len) { const int s = sibling_group(g, q_len); return (entries_per_seq(g, q_len) + s - 1) / s; }
+// Block numbers per sequence, including the empty ones of the last pass: what partial states and tickets are sized by.
+int block_slots_per_seq(const Geometry &g, int q_len) { return passes_per_seq(g, q_len) * sibling_group(g, q_len); }
 
-// `n_listed` sequences with q_len queries each.  The plan always covers the sequences once: with
-// entries_per_seq() = b > 1 query blocks per sequence, the (sequence, KV head, unit) order is cut into at most
-// n_ctas / b ranges and the launch's CTAs work in groups of b on one range each, one query block per CTA.  The
-// partial states and tickets are then counted per (sequence, query block, KV head), which is why
-// n_listed * b <= max_seqs is required.
+// `n_listed` sequences with q_len queries each.  With entries_per_seq() = b > 1 query blocks per sequence, the
+// (sequence, KV head, unit) order is cut into at most n_ctas / s ranges, s = sibling_group(), and the launch's
+// CTAs work in groups of s on one range each, one query block per CTA; a sequence appears once in the plan unless
+// b exceeds the grid, in which case it appears passes_per_seq() times, each pass for the next s blocks.  The
+// partial states and tickets are counted per (sequence, block number, KV head), which is why
+// n_listed * block_slots_per_seq() <= max_seqs is required.
 // Whether a call with q_len queries for each of n_seqs sequences goes to the row-block kernel (one CTA per 64 query
 // rows of a KV head, which walks the whole sequence alone) instead of the pipeline kernel (eight query columns per
 // pass over the pages, split over all CTAs).  The row-block kernel needs enough CTAs to fill the GPU; below that the
@@ -361,7 +367,7 @@ bool uses_row_blocks(const pkv_cache *c, int q_len, int n_seqs) {
     const long long rows = (long long)q_len * c->geo.group;
     if (q_len <= 1 || c->cfg.decode_variant != 0 || c->geo.factor_bits == 4 || rows < kRowBlock) return false;
     const long long n_ctas = (long long)n_seqs * c->geo.n_kv_heads * ((rows + kRowBlock - 1) / kRowBlock);
-    return n_ctas >= 128 || (long long)n_seqs * entries_per_seq(c->geo, q_len) > c->cfg.max_seqs;
+    return n_ctas >= 128 || (long long)n_seqs * block_slots_per_seq(c->geo, q_len) > c->cfg.max_seqs;
 }
 
 pkv_status build_plan(pkv_cache *c, int layer, int n_listed, const int32_t *seq_ids, int q_len, cudaStream_t st) {
@@ -370,14 +376,15 @@ pkv_status build_plan(pkv_cache *c, int layer, int n_listed, const int32_t *seq_
     const int H = g.n_kv_heads;
     const long long cf = g.blob_bytes + 2048, cd = (long long)g.block_tokens * 2 * kRowBytes + 2048;
     // (the row-block kernel only reads the entries; the split over CTAs is not used by it)
-    const int groups = uses_row_blocks(c, q_len, n_listed) ? 1 : entries_per_seq(g, q_len);
-    const int N = std::max(1, g.n_ctas / groups), n_seqs = n_listed;
+    const bool blocks = uses_row_blocks(c, q_len, n_listed);
+    const int groups = blocks ? 1 : sibling_group(g, q_len), per_seq = blocks ? 1 : passes_per_seq(g, q_len);
+    const int N = std::max(1, g.n_ctas / groups), n_seqs = n_listed * per_seq;
 
     std::vector<PlanEntry> entries(n_seqs);
     std::vector<HeadShape> shapes(n_seqs);
     long long total_cost = 0, total_units = 0;
     for (int i = 0; i < n_seqs; ++i) {
-        const int32_t seq = seq_ids[i];
+        const int32_t seq = seq_ids[i / per_seq];
         const SeqLayer &s = c->at(seq, layer);
         int n_pages = (s.n_tokens + c->cfg.page_size - 1) / c->cfg.page_size;
         entries[i] = PlanEntry{seq, n_pages, g.sink_pages, s.f_end};
@@ -865,10 +872,9 @@ static pkv_status decode_impl(pkv_cache *c, int32_t layer, int32_t n_seqs, const
     if (q_len > 1) {
         if (c->cfg.decode_variant == 1)
             return fail(c, PKV_ERR_UNSUPPORTED, "several queries per sequence need the tensor-core kernels (decode_variant 0)");
-        if (!uses_row_blocks(c, q_len, n_seqs) && ((long long)n_seqs * entries_per_seq(c->geo, q_len) > c->cfg.max_seqs ||
-                                                   entries_per_seq(c->geo, q_len) > c->geo.n_ctas))
-            return fail(c, PKV_ERR_INVALID_ARG, "%d sequences x %d query blocks exceed max_seqs = %d (or the blocks the %d CTAs)",
-                        n_seqs, entries_per_seq(c->geo, q_len), c->cfg.max_seqs, c->geo.n_ctas);
+        if (!uses_row_blocks(c, q_len, n_seqs) && (long long)n_seqs * block_slots_per_seq(c->geo, q_len) > c->cfg.max_seqs)
+            return fail(c, PKV_ERR_INVALID_ARG, "%d sequences x %d query blocks exceed max_seqs = %d", n_seqs,
+                        block_slots_per_seq(c->geo, q_len), c->cfg.max_seqs);
         for (int i = 0; i < n_seqs; ++i) {
             const SeqLayer &s = c->at(seq_ids[i], layer);
             // every query must see every factor page whole (and at least its own position)
@@ -913,7 +919,8 @@ static pkv_status decode_impl(pkv_cache *c, int32_t layer, int32_t n_seqs, const
     a.state = state;
     a.q_len = q_len;
     a.q_tpt = queries_per_tile(c->geo, q_len);
-    a.q_nblk = entries_per_seq(c->geo, q_len);
+    a.q_group = sibling_group(c->geo, q_len);
+    a.q_nblk = block_slots_per_seq(c->geo, q_len);
     a.q_cols = a.q_tpt * c->geo.group;
     // decode_overlap = 2: launches never wait for one another, so launches in flight must not share split-K
     // scratch.  The scratch rotates over wl.n_sets sets and every (n_sets-1)-th launch is a plain
@@ -984,7 +991,7 @@ pkv_status pkv_decode_attention_static_scratch(pkv_cache *c, int32_t layer, int3
     a.plan_cta_entry = c->ml.plan_cta_entry;
     a.q = q; a.out = out; a.out_f32 = out_f32;
     a.state = nullptr;
-    a.q_len = 1; a.q_tpt = 1; a.q_nblk = 1; a.q_cols = c->geo.group;
+    a.q_len = 1; a.q_tpt = 1; a.q_nblk = 1; a.q_group = 1; a.q_cols = c->geo.group;
     a.partials = nullptr; a.tickets = nullptr;            // set by the launcher from the static scratch
     a.plain_launch = 0;                                   // the launcher's memset already orders it after earlier work
     c->cache_written = false;

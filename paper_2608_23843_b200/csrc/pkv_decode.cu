@@ -66,10 +66,10 @@ __device__ __forceinline__ void unit_to_page(const Geometry &g, const HeadUnits 
 __device__ __forceinline__ bool load_range(const DecodeArgs &a, Range &r) {
     // All four loads are issued together (the arrays have an element for every CTA of the grid, used or not), so
     // that the header's latency is not paid a second time before the CTA knows its range.
-    // With several query blocks per sequence (q_nblk > 1) the CTAs come in groups of q_nblk that share a range:
-    // CTA b walks range b / q_nblk for query block b % q_nblk.  The siblings start together and read the same
-    // pages in the same order, so all but the first find them in L2.
-    const int range = blockIdx.x / a.q_nblk;
+    // With several query blocks per sequence the CTAs come in groups of q_group that share a range: CTA b walks
+    // range b / q_group for the (b % q_group)-th query block of the range's plan entry.  The siblings start
+    // together and read the same pages in the same order, so all but the first find them in L2.
+    const int range = blockIdx.x / a.q_group;
     const PlanCta *ctas = reinterpret_cast<const PlanCta *>(a.plan + a.plan_cta);
     const PlanHeader hdr = *reinterpret_cast<const PlanHeader *>(a.plan);
     r.start = ctas[range];
@@ -699,14 +699,14 @@ __device__ __forceinline__ void reset_state(WarpState &st) {
 // Index of (sequence, query block, KV head) - what q, out and the tickets are indexed by - for segment `seg` of the
 // plan, which is (sequence, KV head); the query block is this CTA's.
 __device__ __forceinline__ int query_seg(const DecodeArgs &a, int seg) {
-    if (a.q_nblk == 1) return seg;
+    if (a.q_group == 1) return seg;
     const int H = a.geo.n_kv_heads;
-    return ((seg / H) * a.q_nblk + (int)(blockIdx.x % a.q_nblk)) * H + seg % H;
+    return ((seg / H) * a.q_group + (int)(blockIdx.x % a.q_group)) * H + seg % H;
 }
 // This CTA's partial state of segment `seg`, or with `cta` = the segment's first range, the first of its partial
-// states; consecutive ranges' states of one query block are q_nblk slots apart.
+// states; consecutive ranges' states of one query block are q_group slots apart.
 __device__ __forceinline__ float *partial_slot(const DecodeArgs &a, int cta_range, int seg) {
-    return a.partials + (((long long)cta_range + seg) * a.q_nblk + blockIdx.x % a.q_nblk) * kPartialFloats;
+    return a.partials + (((long long)cta_range + seg) * a.q_group + blockIdx.x % a.q_group) * kPartialFloats;
 }
 
 // Query column n of a segment's score tile = query head n % G of the (n / G)-th query token of the plan entry's
@@ -768,7 +768,7 @@ __device__ __forceinline__ void store_out(const DecodeArgs &a, int seg, int hq, 
 // time, because with dozens of parts it is the latency of these loads that the rest of the GPU waits for.
 template <int E, int kBatch>
 __device__ __forceinline__ void merge_parts(const DecodeArgs &a, const float *first, int np, int seg, int ctid) {
-    const long long stride = (long long)a.q_nblk * kPartialFloats;      // between the states of consecutive ranges
+    const long long stride = (long long)a.q_group * kPartialFloats;     // between the states of consecutive ranges
     constexpr int kThreads = kConsumerWarps * 32;
     const int n_items = a.q_cols * 32;
     const int d4 = (ctid & 31) * 4;                               // kThreads is a multiple of 32
@@ -854,7 +854,7 @@ __device__ __forceinline__ void flush_segment(const DecodeArgs &a, float *comb, 
     if (a.overlap == 1) asm volatile("griddepcontrol.wait;" ::: "memory");
     const PlanSeg ps = reinterpret_cast<const PlanSeg *>(a.plan + a.plan_seg)[seg];
     const int qseg = query_seg(a, seg);
-    float *part = partial_slot(a, blockIdx.x / a.q_nblk, seg);
+    float *part = partial_slot(a, blockIdx.x / a.q_group, seg);
     for (int item = ctid; item < kItems; item += kThreads) {
         const int hq = item >> 5, d4 = (item & 31) * 4;
         float M = kNegInf;
@@ -955,7 +955,7 @@ __global__ void __launch_bounds__(kDecodeThreads, 2) decode_tc_kernel(const __gr
         const PlanEntry *entries = reinterpret_cast<const PlanEntry *>(a.plan + a.plan_entry);
         int k = 0, seg_local = 0;
         bool ok = true;
-        const bool keep = a.q_nblk > 1;      // sibling CTAs read the same pages: leave them in L2 for one another
+        const bool keep = a.q_group > 1;     // sibling CTAs read the same pages: leave them in L2 for one another
         PlanCta cur = rg.start;
         while (ok && !(cur.entry == rg.end.entry && cur.head == rg.end.head && cur.unit == rg.end.unit)) {
             const PlanEntry e = cur.entry == rg.start.entry ? rg.first_entry : entries[cur.entry];

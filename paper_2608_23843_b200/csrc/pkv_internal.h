@@ -101,9 +101,11 @@ struct DecodeArgs {
     int *tickets;                      // one per segment, zero between launches
 
     // Queries per sequence (1 = decoding).  A score tile has eight query columns: q_tpt = min(q_len, 8 / group)
-    // consecutive query tokens fill q_cols = q_tpt * group of them, so a sequence takes q_nblk = ceil(q_len / q_tpt)
-    // plan entries, each walking the sequence's pages for its own block of query tokens.
-    int q_len, q_tpt, q_nblk, q_cols;
+    // consecutive query tokens fill q_cols = q_tpt * group of them, so a sequence has b = ceil(q_len / q_tpt) blocks of
+    // query tokens.  The CTAs of a launch work in groups of q_group siblings on one plan range, one block each; a
+    // sequence has ceil(b / q_group) plan entries (more than one only if b exceeds the grid), so block numbers run
+    // over q_nblk = entries x q_group per sequence (those past b are empty).
+    int q_len, q_tpt, q_nblk, q_group, q_cols;
     int *status;
     int layer;
     int variant;                       // 0 = tensor-core pipeline, 1 = scalar reference kernel

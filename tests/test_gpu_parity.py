@@ -678,3 +678,39 @@ def test_row_block_kernel_agrees_with_the_column_kernel(P, rk, rv, G, q_len):
             assert np.abs(a[i, j] - b[i, j]).max() <= 6e-3 * np.abs(b[i, j]).max(), (i, j)
     print("row-block vs column kernel P=%d r=(%d,%d) G=%d q_len=%d: max rel diff %.2e"
           % (P, rk, rv, G, q_len, max(np.abs(a[i, j] - b[i, j]).max() / np.abs(b[i, j]).max() for i in range(a.shape[0]) for j in range(q_len))))
+
+
+def test_more_query_blocks_than_ctas():
+    """Twelve blocks of query tokens per sequence on a grid of five CTAs (decode kernel route pinned by
+    decode_variant = 2): the blocks are served in three passes of five sibling CTAs (the last pass has two empty
+    ones).  Kernel gate against the oracle, and agreement with the same call on the default grid."""
+    H, G, P, q_len = 2, 4, 64, 24
+    lengths = [20 * P + 7, q_len + 3, 6 * P]
+    outs = []
+    for n_ctas in (5, 0):
+        cfg = pkv.make_config(n_layers=1, n_kv_heads=H, n_q_heads=H * G, rank=16, sink_tokens=P, recent_tokens=P,
+                              max_seqs=3 * 15, max_pages_per_seq=24, n_dense_slots=80, n_factor_slots=80,
+                              decode_variant=2, n_ctas=n_ctas)
+        pair = Pair(cfg, seed=4)
+        for s, T in enumerate(lengths):
+            k, v = gen_kv(12, 0, s, T, cfg, outlier_prob=0.01)
+            pair.append(0, [s], [k[:T - q_len]], [v[:T - q_len]])
+            pair.compress(0)
+            pair.append(0, [s], [k[T - q_len:]], [v[T - q_len:]])
+        g = torch.Generator().manual_seed(9)
+        q = torch.randn((3, q_len, H * G, 128), generator=g).to(torch.bfloat16)
+        out32 = torch.empty(q.shape, dtype=torch.float32, device="cuda")
+        order = [1, 2, 0]
+        pair.gpu.decode_attention_multi(0, order, q_len, q.cuda(), None, out32)
+        torch.cuda.synchronize()
+        st = pair.gpu.stats()
+        assert st["device_timeouts"] == 0 and st["bad_slot_indices"] == 0
+        got = f64(out32)
+        for s in order:
+            pair.load_gpu_factors_into_oracle(s, 0)
+        ref = pair.orc.decode_attention_multi(0, order, f64(q))
+        for i in range(3):
+            assert np.abs(got[i] - ref[i]).max() <= 4e-3 * np.abs(ref[i]).max(), (n_ctas, i)
+        outs.append(got)
+        pair.gpu.close()
+    assert np.abs(outs[0] - outs[1]).max() <= 2e-3 * np.abs(outs[1]).max()
