@@ -267,8 +267,9 @@ pkv_status pkv_decode_attention(pkv_cache *c, int32_t layer, int32_t n_seqs, con
  * Requirements (else PKV_ERR_INVALID_ARG, nothing launched): 1 <= q_len <= T for every listed sequence; no listed
  * sequence has a factor page that reaches past token T - q_len (so every query sees every factor page whole:
  * holds whenever q_len <= recent_tokens and compression ran no later than the append of these positions, and it is
- * checked per call); n_seqs * ceil(q_len / max(1, 8 / (H_q / H_kv))) <= max_seqs (split-K partial states and
- * tickets are kept per sequence and block of query tokens).
+ * checked per call); n_seqs * b <= max_seqs with b = ceil(q_len / max(1, 8 / (H_q / H_kv))) blocks of query tokens
+ * per sequence, b rounded up to a multiple of the grid size if it exceeds it (split-K partial states and tickets
+ * are kept per sequence and block).
  * Two kernels serve this call.  A row-block kernel - one CTA per (sequence, KV head, 64 query rows), which reads the
  * sequence's pages once for its 64 rows (tensor-core products with the query rows as the 16-row operand) - runs
  * when q_len * (H_q / H_kv) >= 64, the factors are bf16, and the call makes at least 128 such CTAs (enough to fill
