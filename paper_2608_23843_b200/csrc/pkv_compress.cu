@@ -40,11 +40,11 @@ template <int P> struct Quads {
     static constexpr int kGWarps = (kItems + 31) / 32;         // 4 or 1; the remaining warps update Q^T
     static constexpr int kQIters = kQuads * (P / 4) / 32;      // 8 or 2
     static constexpr int kCheck = (kClasses + 2) / 3;          // the energy rule is evaluated about three times per sweep
-    // Column of quad q's row k inside row k of M.  At P = 32 every rotation lane stores four variants of its row, and
-    // with the plain column the eight lanes of a quarter warp (two quads x four rows) hit two 16-byte bank groups;
-    // q ^ 2k spreads them over eight (+10 % throughput).  At P = 64 (two variants) the extra index arithmetic costs
-    // more than the conflicts.
-    __host__ __device__ static constexpr int mcol(int q, int k) { return P == 32 ? (q ^ (2 * k)) : q; }
+    // Where row k of quad q's 4 x 4 transform lives in M (variant g): quad-major with a stride of five float4.  The
+    // eight lanes of a quarter warp that store rows (two quads x four rows: slots 5q + k) and the eight that load one
+    // row of eight consecutive quads (slots 5q + k, q = 8j .. 8j+7) both cover all eight 16-byte bank groups.
+    static constexpr int kMStride = 5;
+    __host__ __device__ static constexpr int mslot(int g, int q, int k) { return (g * kQuads + q) * kMStride + k; }
 };
 __constant__ uchar4 c_quads64[Quads<64>::kClasses * Quads<64>::kQuads];
 __constant__ uchar4 c_quads32[Quads<32>::kClasses * Quads<32>::kQuads];
@@ -77,7 +77,7 @@ struct CompressSmem {
     uchar2 pairs[P >= 32 ? 1 : (P - 1) * (P / 2)];   // pair ordering: the rounds' pairs (lanes index it divergently)
     // quad ordering: the 4 x 4 transforms of a class's quads, [member order][row][quad] as float4, and the table
     using Qd = Quads<(P >= 32 ? P : 32)>;
-    float4 M[P >= 32 ? Qd::kDiag * 4 * Qd::kQuads : 1];
+    float4 M[P >= 32 ? Qd::kDiag * Qd::kMStride * Qd::kQuads : 1];
     uchar4 quads[P >= 32 ? Qd::kClasses * Qd::kQuads : 1];
     float lam[P];
     int order[P];
@@ -337,7 +337,7 @@ compress_kernel(Geometry geo, const unsigned char *dense_pool, unsigned char *fa
                     for (int g = 0; g < Qd::kDiag; ++g) {              // M'[k][j] = M[k ^ x][j ^ x] for member order j ^ x
                         constexpr int kStep = Qd::kVarStep;
                         const int x = g * kStep;
-                        S.M[(g * 4 + (t ^ x)) * kQuads + Qd::mcol(qd, t ^ x)] = make_float4(r[0 ^ x], r[1 ^ x], r[2 ^ x], r[3 ^ x]);
+                        S.M[Qd::mslot(g, qd, t ^ x)] = make_float4(r[0 ^ x], r[1 ^ x], r[2 ^ x], r[3 ^ x]);
                     }
                 }
                 __syncthreads();
@@ -352,7 +352,7 @@ compress_kernel(Geometry geo, const unsigned char *dense_pool, unsigned char *fa
                         int ma[4], mb[4];
 #pragma unroll
                         for (int i = 0; i < 4; ++i) { ma[i] = (ma4 >> (8 * i)) & 0xff; mb[i] = (mb4 >> (8 * i)) & 0xff; }
-                        const float4 *Ma = S.M + h * 4 * kQuads, *Mb = S.M + h * 4 * kQuads;       // row k of quad q: [k * kQuads + mcol(q, k)]
+                        const float4 *Ma = S.M + Qd::mslot(h, ia, 0), *Mb = S.M + Qd::mslot(h, ib, 0);    // rows 0..3 of the quad
                         float T[4][4];
 #pragma unroll
                         for (int i = 0; i < 4; ++i)
@@ -360,7 +360,7 @@ compress_kernel(Geometry geo, const unsigned char *dense_pool, unsigned char *fa
                             for (int j = 0; j < 4; ++j) T[i][j] = 0.f;
 #pragma unroll
                         for (int k = 0; k < 4; ++k) {                  // T = M_a^T X
-                            const float4 mk = Ma[k * kQuads + Qd::mcol(ia, k)];
+                            const float4 mk = Ma[k];
                             const float *row = S.G + ma[k] * kGs;
 #pragma unroll
                             for (int j = 0; j < 4; ++j) {
@@ -369,7 +369,7 @@ compress_kernel(Geometry geo, const unsigned char *dense_pool, unsigned char *fa
                                 T[2][j] = fmaf(mk.z, x, T[2][j]); T[3][j] = fmaf(mk.w, x, T[3][j]);
                             }
                         }
-                        const float4 b0 = Mb[ib], b1 = Mb[kQuads + Qd::mcol(ib, 1)], b2 = Mb[2 * kQuads + Qd::mcol(ib, 2)], b3 = Mb[3 * kQuads + Qd::mcol(ib, 3)];
+                        const float4 b0 = Mb[0], b1 = Mb[1], b2 = Mb[2], b3 = Mb[3];
 #pragma unroll
                         for (int i = 0; i < 4; ++i) {                  // Y = T M_b, row i
                             float y[4];
@@ -391,7 +391,8 @@ compress_kernel(Geometry geo, const unsigned char *dense_pool, unsigned char *fa
                         float4 *r0 = QT4 + m4.x * (P / 4) + ch, *r1 = QT4 + m4.y * (P / 4) + ch;
                         float4 *r2 = QT4 + m4.z * (P / 4) + ch, *r3 = QT4 + m4.w * (P / 4) + ch;
                         const float4 x0 = *r0, x1 = *r1, x2 = *r2, x3 = *r3;
-                        const float4 c0 = S.M[k], c1 = S.M[kQuads + Qd::mcol(k, 1)], c2 = S.M[2 * kQuads + Qd::mcol(k, 2)], c3 = S.M[3 * kQuads + Qd::mcol(k, 3)];
+                        const float4 *Mk = S.M + Qd::mslot(0, k, 0);
+                        const float4 c0 = Mk[0], c1 = Mk[1], c2 = Mk[2], c3 = Mk[3];
 #define PKV_MIX(comp) make_float4(fmaf(c3.comp, x3.x, fmaf(c2.comp, x2.x, fmaf(c1.comp, x1.x, c0.comp * x0.x))), \
                                   fmaf(c3.comp, x3.y, fmaf(c2.comp, x2.y, fmaf(c1.comp, x1.y, c0.comp * x0.y))), \
                                   fmaf(c3.comp, x3.z, fmaf(c2.comp, x2.z, fmaf(c1.comp, x1.z, c0.comp * x0.z))), \
