@@ -25,22 +25,22 @@ ROOT = os.path.dirname(os.path.abspath(__file__))
 sys.path.insert(0, ROOT)
 
 WORKLOADS = {
-    # BASELINE config 2: Qwen3-32B-shaped long context
+    # Qwen3-32B-shaped long context (the headline workload): 64 layers, one 128K-token sequence
     "qwen3_32b_128k": dict(n_layers=64, n_kv_heads=8, n_q_heads=64, batch=1, T=131072, rank=24,
                            sink=64, recent=512, ragged=False, outliers=0.0),
-    # BASELINE config 1: Llama-3-8B-shaped decode layer
+    # Llama-3-8B-shaped decode layer, batch 8, 32K tokens each
     # (four independent layers of that shape are built and a step decodes one of them in turn, so that
     # overlapping launches never stream the same bytes and cannot feed each other through L2)
     "llama3_8b_32k_b8": dict(n_layers=4, layers_per_step=1, n_kv_heads=8, n_q_heads=32, batch=8, T=32768, rank=24,
                              sink=64, recent=256, ragged=False, outliers=0.0),
-    # BASELINE config 4: ragged serving batch (rank chosen with --rank)
+    # ragged serving batch: 64 requests of 2K..64K tokens, outlier key tokens (rank chosen with --rank)
     "ragged_b64": dict(n_layers=2, layers_per_step=1, n_kv_heads=8, n_q_heads=32, batch=64, T=(2048, 65536), rank=24,
                        sink=64, recent=256, ragged=True, outliers=0.02),
     # The paper's own setting: Qwen3-8B shape (36 layers, 32q/8kv), 16K context, P=32, ranks (16,14),
     # one sink page, last completed page + incomplete page dense
     "qwen3_8b_16k_paper_default": dict(n_layers=36, n_kv_heads=8, n_q_heads=32, batch=1, T=16384 + 17, rank=16,
                                        rank_v=14, page=32, sink=32, recent=32, ragged=False, outliers=0.0),
-    # BASELINE config 3: serving loop.  Prompts are prefilled and compressed; a step is append (one token per
+    # serving loop: incremental compression during decoding.  Prompts are prefilled and compressed; a step is append (one token per
     # sequence) -> decode -> compress_eligible, so every 64th step factorizes one page per (sequence, KV head, K|V)
     "serving_b32_8k": dict(n_layers=1, n_kv_heads=8, n_q_heads=32, batch=32, T=8192, rank=24, sink=64, recent=256,
                            ragged=False, outliers=0.0, serving=True),
@@ -48,7 +48,7 @@ WORKLOADS = {
     # dense window of that size) are the queries.  Use with --q-len 2048 (pkv_decode_attention_multi).
     "prefill_chunk_llama3_8b_32k": dict(n_layers=2, layers_per_step=1, n_kv_heads=8, n_q_heads=32, batch=1, T=32768,
                                         rank=24, sink=64, recent=2048, ragged=False, outliers=0.0),
-    # BASELINE config 0: tiny (L2-resident; latency only)
+    # tiny single decode step (L2-resident; latency only)
     "tiny": dict(n_layers=1, n_kv_heads=1, n_q_heads=4, batch=1, T=1024, rank=16, sink=64, recent=128,
                  ragged=False, outliers=0.0),
 }
@@ -143,6 +143,11 @@ class ClockSampler:
                     self.sm_max = float(r[1])
                 self.rows.append((time.perf_counter(), float(r[0]), [r[2 + i].startswith("Active") for i in range(4)]))
 
+    def median_mhz(self, spans):
+        """Median SM clock of the samples stamped inside any of the (t0, t1) wall-clock spans, or None."""
+        sm = [r[1] for r in list(self.rows) if any(t0 <= r[0] <= t1 for t0, t1 in spans)]
+        return statistics.median(sm) if sm else None
+
     def begin(self):
         """Call right before the timed region (waits, briefly, until the sampler is alive)."""
         if self.nvml is not None or self.proc is not None:
@@ -214,6 +219,7 @@ def build_workload(w, rank, device, overlap=2, n_ctas=0, factor_bits=16, grow=0,
     ids = list(range(w["batch"]))
     svd_ms, n_svds = 0.0, 0
     kept = []
+    spans = []                                            # wall-clock spans of the compression calls (for the clock samples)
     for layer in range(L):
         for s in ids:
             k, v = synth.make_kv(SEED, layer, s, lengths[s] + grow, w["n_kv_heads"], 128, P, device, w["outliers"])
@@ -222,27 +228,91 @@ def build_workload(w, rank, device, overlap=2, n_ctas=0, factor_bits=16, grow=0,
                 kept.append((k[lengths[s]:].clone(), v[lengths[s]:].clone()))
             del k, v
         e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        torch.cuda.synchronize()
+        t0 = time.perf_counter()
         e0.record()
         n = cache.compress_eligible_pages(layer)
         e1.record()
         torch.cuda.synchronize()
+        spans.append((t0, time.perf_counter()))
         svd_ms += e0.elapsed_time(e1)
         n_svds += n * w["n_kv_heads"] * 2
-    comp = dict(pages_per_s=(n_svds / (svd_ms * 1e-3) if svd_ms > 0 else None), n_page_svds=n_svds, svd_ms=svd_ms)
+    st = cache.stats()
+    comp = dict(pages_per_s=(n_svds / (svd_ms * 1e-3) if svd_ms > 0 else None), n_page_svds=n_svds, svd_ms=svd_ms,
+                spans=spans, jacobi_rounds=st["jacobi_rounds"], page_svds_counted=st["page_svds"],
+                not_converged=st["page_svds_not_converged"], page=P, rank=rank, rank_v=w.get("rank_v", rank))
     if keep_kv:
         comp["new_k"] = torch.stack([k for k, _ in kept], 1).contiguous()      # [grow][batch][H_kv][d]
         comp["new_v"] = torch.stack([v for _, v in kept], 1).contiguous()
     return cfg, cache, lengths, comp
 
 
+N_SMS, FP32_LANES_PER_SM = 148, 128
+
+
+def hbm_roofline(kernel, bytes_per_launch, launch_us, factor_bits):
+    """Roofline record of the decode kernel (bound: HBM).  achieved = algorithmic bytes per launch / average launch
+    duration.  The peak is the measured copy bandwidth: a STREAM-style copy reads and writes, this kernel only
+    reads, so a fraction a little above 1 is possible and is flagged; `frac_of_8tbs` is the same figure against the
+    nominal 8 TB/s.  `traffic` scales the DRAM bytes ncu counted on the llama3_8b_32k_b8 launch (every unit is read
+    once, so traffic grows with the units processed); it is not a capture of this workload."""
+    peak, peak_src = _peaks()
+    achieved = bytes_per_launch / (launch_us * 1e-6) / 1e9
+    ratio = NCU_TRAFFIC_PER_ALGORITHMIC_BYTE_INT4 if factor_bits == 4 else NCU_TRAFFIC_PER_ALGORITHMIC_BYTE
+    rec = {"bound": "hbm", "kernel": kernel, "achieved": achieved, "peak": peak, "unit": "GB/s", "frac": achieved / peak,
+           "frac_of_8tbs": achieved / 8000.0, "peak_source": peak_src,
+           "peak_kind": "read+write copy bandwidth (not an upper bound for a read-only stream)",
+           "traffic": bytes_per_launch * ratio,
+           "traffic_source": "ncu dram__bytes_read+write of this kernel captured on the llama3_8b_32k_b8 launch "
+                             "(%.4f DRAM bytes per algorithmic byte), scaled by this launch's algorithmic bytes" % ratio,
+           "launch_us": launch_us, "algorithmic_bytes_per_launch": bytes_per_launch}
+    if rec["frac"] > 1.0:
+        rec["note"] = "above 1.0 of the copy-based peak: the kernel reads only; see frac_of_8tbs"
+    return rec
+
+
+def compress_record(comp, sampler):
+    """Throughput of the page-SVD kernel against the bound that applies to it: plain fp32 FMAs (the Gram matrix and
+    the projection are 7 % of the work; the rest is 4 x 4 rotations in shared memory, no tensor-core shape).
+    Flops per page SVD, counted from what the algorithm needs with the measured number of rotation rounds:
+      Gram matrix, one triangle      P^2 d
+      per round, page size 64 / 32   16 P^2   (G' = M^T G M on one triangle: 8 P^2; Q^T' = M^T Q^T: 8 P^2)
+      per round, page size 16        8 P^2    (2 x 2 rotations)
+      B = A^T X                      2 r P d
+    Peak = SMs x 128 FMA lanes x 2 x SM clock sampled while the kernel ran (the maximum clock if no sample fell
+    inside)."""
+    n = comp["page_svds_counted"]
+    if not n or not comp["pages_per_s"]:
+        return None
+    P, d = comp["page"], 128
+    rounds = comp["jacobi_rounds"] / n
+    per_sweep = {64: 21, 32: 13, 16: 15}[P]
+    per_round = (16 if P >= 32 else 8) * P * P
+    r_mean = 0.5 * (comp["rank"] + comp["rank_v"])
+    flops = P * P * d + rounds * per_round + 2 * r_mean * P * d
+    mhz = sampler.median_mhz(comp["spans"]) if sampler is not None else None
+    clock_src = "sampled during the compression launches"
+    if mhz is None:
+        mhz, clock_src = (sampler.sm_max if sampler is not None and sampler.sm_max else 1965.0), "maximum SM clock (no sample fell inside)"
+    peak = N_SMS * FP32_LANES_PER_SM * 2 * mhz * 1e6 / 1e12
+    achieved = comp["pages_per_s"] * flops / 1e12
+    return {"pages_per_s": comp["pages_per_s"], "page_svds": n, "rounds_per_page": rounds,
+            "sweeps_per_page": rounds / per_sweep, "not_converged": comp["not_converged"],
+            "flops_per_page": flops, "bound": "alu", "achieved": achieved, "peak": peak, "unit": "TFLOP/s",
+            "frac": achieved / peak, "sm_mhz": mhz, "clock_source": clock_src,
+            "peak_source": "148 SMs x 128 fp32 FMA lanes x 2 x SM clock"}
+
+
 def run_serving(args, w, rank, device, world, rk, local):
-    """BASELINE config 3: `steps` iterations of append (one token per sequence) -> decode -> compress on one
+    """Serving loop: `steps` iterations of append (one token per sequence) -> decode -> compress on one
     layer, timed as a whole and call by call with CUDA events on the launching stream."""
     import torch
     from paper_2608_23843_b200 import synth
     B, Hq, P = w["batch"], w["n_q_heads"], w.get("page", 64)
     warm = max(3, args.warmup)
     total = warm + 2 * args.steps + 3           # device-resident pass, host-buffer pass, warm-ups
+    sampler = ClockSampler(local)
+    sampler.start()                                       # ahead of the cache build: its compression launches are sampled too
     cfg, cache, lengths, comp = build_workload(w, rank, device, 0, args.n_ctas, args.factor_bits, grow=total, keep_kv=True)
     ids = list(range(B))
     new_k, new_v = comp["new_k"], comp["new_v"]
@@ -292,8 +362,6 @@ def run_serving(args, w, rank, device, world, rk, local):
             dist.barrier()
         torch.cuda.synchronize()
 
-    sampler = ClockSampler(local)
-    sampler.start()                                       # ahead of the warm-up: nvidia-smi takes a while to start
     for _ in range(warm):
         step(False)
     cache.decode_attention(0, ids, qs[0], out)
@@ -349,8 +417,6 @@ def run_serving(args, w, rank, device, world, rk, local):
     att_mean = statistics.mean(att)
     ms, e2e_ms, att_mean = max_over_ranks([ms, e2e_ms, att_mean], world, device)
     if rk == 0:
-        peak, peak_src = _peaks()
-        achieved = bytes_per_step / (att_mean * 1e-6) / 1e9
         n_event_svds = sum(n for _, n in cmp_event) * w["n_kv_heads"] * 2
         step_bytes = 2 * B * w["n_kv_heads"] * 128 * 2 + 2 * B * Hq * 128 * 2
         line = {
@@ -369,12 +435,9 @@ def run_serving(args, w, rank, device, world, rk, local):
             "step_us_p99": pct([a + b + c for a, b, (c, _) in zip(app, att, cmp_all)], 0.99),
             "algorithmic_bytes_per_step": bytes_per_step,
             "pages_factorized_per_s": comp["pages_per_s"], "page_svds_timed": comp["n_page_svds"],
-            "roofline": {"bound": "hbm", "kernel": "decode_tc_kernel<P=%d, rank tiles=%d>" % (P, (rank + 7) // 8),
-                         "achieved": achieved, "peak": peak, "unit": "GB/s", "frac": achieved / peak,
-                         "peak_source": peak_src, "traffic": bytes_per_step * (NCU_TRAFFIC_PER_ALGORITHMIC_BYTE_INT4 if args.factor_bits == 4 else NCU_TRAFFIC_PER_ALGORITHMIC_BYTE),
-                         "traffic_source": "ncu dram__bytes_read+write of this kernel on the llama3_8b_32k_b8 launch, "
-                                           "scaled by algorithmic bytes",
-                         "launch_us": att_mean, "algorithmic_bytes_per_launch": bytes_per_step},
+            "compress": compress_record(comp, sampler),
+            "roofline": hbm_roofline("decode_tc_kernel<P=%d, rank tiles=%d>" % (P, (rank + 7) // 8), bytes_per_step,
+                                     att_mean, args.factor_bits),
             "e2e": {"value": e2e_ms * 1e3, "unit": "us", "h2d_bytes_per_step": step_bytes - B * Hq * 128 * 2,
                     "d2h_bytes_per_step": B * Hq * 128 * 2},
             "gpu_launches": args.steps * 2 + len(cmp_event), "clocks": clocks,
@@ -423,6 +486,8 @@ def oracle_sample(w, rank, steps, factor_bits=16):
 
 def run_reference(args, w, rank):
     rank0 = int(os.environ.get("RANK", "0")) == 0
+    if os.environ.get("PKV_BENCH_RANK_MARKER"):           # lets a test see that every rank was started
+        print("rank %s of %s present" % (os.environ.get("RANK", "0"), os.environ.get("WORLD_SIZE", "1")), file=sys.stderr)
     if not rank0:
         return
     o = oracle_sample(w, rank, args.steps + args.warmup, args.factor_bits)
@@ -473,6 +538,8 @@ def main():
     ap.add_argument("--rank", type=int, default=0, help="override the workload's rank (8, 16, 24, 32)")
     ap.add_argument("--impl", default="pkv", choices=["pkv", "reference"])
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--no-standalone", action="store_true",
+                    help="skip the second measurement with decode_overlap = 0 (the `standalone` record)")
     ap.add_argument("--overlap", type=int, default=2, choices=[0, 1, 2],
                     help="decode_overlap mode of the cache: 0 = every launch waits for the previous one, 1 = launches "
                          "overlap but complete in order, 2 = launches never wait for one another (default)")
@@ -493,6 +560,15 @@ def main():
     ap.add_argument("--graph", action="store_true",
                     help="replay one CUDA graph per step instead of launching every layer from the host")
     args = ap.parse_args()
+    if args.gpus > 1 and "WORLD_SIZE" not in os.environ:
+        # launched plainly: start one rank per GPU ourselves (what the torchrun command line would do)
+        import socket
+        with socket.socket() as sk:
+            sk.bind(("127.0.0.1", 0))
+            port = sk.getsockname()[1]
+        cmd = [sys.executable, "-m", "torch.distributed.run", "--nnodes=1", "--nproc-per-node", str(args.gpus),
+               "--master-addr", "127.0.0.1", "--master-port", str(port), os.path.abspath(__file__)] + sys.argv[1:]
+        raise SystemExit(subprocess.call(cmd))
     w = WORKLOADS[args.workload]
     rank = args.rank or w["rank"]
     if args.impl == "reference":
@@ -513,6 +589,7 @@ def main():
     device = torch.device("cuda", local)
     if world > 1:
         dist.init_process_group("nccl", device_id=device)
+        print("bench.py: rank %d of %d on cuda:%d (%s)" % (rk, world, local, torch.cuda.get_device_name(local)), file=sys.stderr)
     pkv.lib()                                             # fail loudly if the CUDA library is missing
 
     if w.get("serving"):
@@ -526,6 +603,8 @@ def main():
         w = dict(w, T=w["T"] // world, sink=w["sink"] if rk == 0 else 0, recent=w["recent"] if rk == world - 1 else 0)
     QL = args.q_len
     per_tile = max(1, min(QL, 8 // (w["n_q_heads"] // w["n_kv_heads"])))
+    sampler = ClockSampler(local)
+    sampler.start()                                       # ahead of the cache build: its compression launches are sampled too
     cfg, cache, lengths, comp = build_workload(w, rank, device, args.overlap, args.n_ctas, args.factor_bits,
                                                plan_entries_per_seq=-(-QL // per_tile), decode_variant=args.decode_variant)
     ids = list(range(w["batch"]))
@@ -565,8 +644,6 @@ def main():
             dist.barrier()
         torch.cuda.synchronize()
 
-    sampler = ClockSampler(local)
-    sampler.start()                                       # ahead of the warm-up: nvidia-smi takes a while to start
     for _ in range(max(3, args.warmup)):
         step()
     torch.cuda.synchronize()
@@ -637,12 +714,35 @@ def main():
     if st["device_timeouts"] or st["bad_slot_indices"] or (outs[0].float().isnan().any().item()):
         raise SystemExit("decode produced timeouts or NaNs: %r" % st)
 
+    # The same step with every launch standing alone (decode_overlap = 0: a launch starts computing only when the
+    # kernel before it has finished, as in a decoder whose queries come from the layer before): a second cache of
+    # the same workload, timed the same way in this run.
+    standalone_ms = None
+    if args.overlap != 0 and QL == 1 and not args.seq_sharded and not args.graph and not args.no_standalone:
+        cache.close()
+        cache = None
+        torch.cuda.empty_cache()
+        _, cache, _, _ = build_workload(w, rank, device, 0, args.n_ctas, args.factor_bits, decode_variant=args.decode_variant)
+        for _ in range(max(3, args.warmup)):
+            eager_step()
+        barrier()
+        s0, s1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        s0.record()
+        for _ in range(args.steps):
+            eager_step()
+        s1.record()
+        barrier()
+        standalone_ms = s0.elapsed_time(s1) / args.steps
+        st = cache.stats()
+        if st["device_timeouts"] or st["bad_slot_indices"]:
+            raise SystemExit("decode produced timeouts: %r" % st)
+
     ms, e2e_ms, launch_ms = max_over_ranks([ms, e2e_ms, launch_ms], world, device)
+    if standalone_ms is not None:
+        standalone_ms = max_over_ranks([standalone_ms], world, device)[0]
 
     if rk == 0:
-        peak, peak_src = _peaks()
         bytes_per_launch = bytes_per_step / lps
-        achieved = bytes_per_launch / (launch_ms * 1e-3) / 1e9
         qbytes = sum(q.numel() * 2 for q in qs[:lps])
         line = {
             "metric": "decode_us_per_step", "value": ms * 1e3, "unit": "us", "n_gpus": world, "steps": args.steps,
@@ -653,16 +753,20 @@ def main():
             "frac_of_8tbs": bytes_per_step / (ms * 1e-3) / 8e12,
             "algorithmic_bytes_per_step": bytes_per_step,
             "pages_factorized_per_s": comp["pages_per_s"], "page_svds_timed": comp["n_page_svds"],
-            "roofline": {"bound": "hbm", "kernel": "decode_tc_kernel<P=%d, rank tiles=%d>" % (w.get("page", 64), (rank + 7) // 8),
-                         "achieved": achieved, "peak": peak, "unit": "GB/s", "frac": achieved / peak,
-                         "peak_source": peak_src,
-                         "traffic": bytes_per_launch * (NCU_TRAFFIC_PER_ALGORITHMIC_BYTE_INT4 if args.factor_bits == 4 else NCU_TRAFFIC_PER_ALGORITHMIC_BYTE),
-                         "traffic_source": "ncu dram__bytes_read+write of this kernel on the llama3_8b_32k_b8 launch, "
-                                           "scaled by algorithmic bytes", "launch_us": launch_ms * 1e3,
-                         "algorithmic_bytes_per_launch": bytes_per_launch},
+            "compress": compress_record(comp, sampler),
+            "roofline": hbm_roofline("decode_tc_kernel<P=%d, rank tiles=%d>" % (w.get("page", 64), (rank + 7) // 8),
+                                     bytes_per_launch, launch_ms * 1e3, args.factor_bits),
             "e2e": {"value": e2e_ms * 1e3, "unit": "us", "h2d_bytes_per_step": qbytes, "d2h_bytes_per_step": qbytes},
             "gpu_launches": lps * args.steps * (2 if args.seq_sharded else 1), "clocks": clocks,
         }
+        if standalone_ms is not None:
+            r0 = hbm_roofline(line["roofline"]["kernel"], bytes_per_launch, standalone_ms * 1e3 / lps, args.factor_bits)
+            line["standalone"] = {"mode": "decode_overlap=0: each launch waits for the kernel before it before it reads q "
+                                          "or writes anything (cache pages are prefetched into shared memory meanwhile)",
+                                  "value": standalone_ms * 1e3, "unit": "us", "steps": args.steps,
+                                  "hbm_gbs": bytes_per_step / (standalone_ms * 1e-3) / 1e9 * world,
+                                  "frac_of_8tbs": r0["frac_of_8tbs"], "frac": r0["frac"], "launch_us": r0["launch_us"],
+                                  "gpu_launches": lps * args.steps}
         P_, Gq = w.get("page", 64), Hq // w["n_kv_heads"]
         rows = QL * Gq
         if QL > 1 and args.decode_variant == 0 and args.factor_bits != 4 and rows >= 64 and w["batch"] * w["n_kv_heads"] * -(-rows // 64) >= 128:

@@ -31,6 +31,9 @@
  *    pkv_destroy_cache().
  *  - Pointers marked [device] are device addresses on the current CUDA device,
  *    [host] are ordinary host addresses.  bf16 = IEEE bfloat16 bit pattern.
+ *  - Alignment of caller buffers (checked on the host; PKV_ERR_INVALID_ARG, nothing
+ *    launched): k and v 16 bytes, q 4, out 8, out_f32 16, state 8.  Contiguous
+ *    tensors from any allocator satisfy this; a view at an odd element offset may not.
  *  - All device work is enqueued on the `stream` argument (a cudaStream_t passed
  *    as void*); calls are asynchronous unless stated.  Operations on one cache
  *    must be issued on one stream (or the caller orders the streams); the one
@@ -108,7 +111,10 @@ typedef struct pkv_config {
     int32_t decode_overlap;     /* pkv_decode_attention is launched with programmatic stream serialization, so its
                                    CTAs start as SMs free up.
                                    0 (default): the kernel waits for the preceding kernel on the stream to finish
-                                      before it reads the cache or q.
+                                      before it reads q or writes anything.  Pages of the cache are already
+                                      streamed into shared memory while that kernel finishes: only this library's
+                                      own calls write the pools, and a decode call that follows one of them is
+                                      launched the ordinary way (see the last paragraph).
                                    1: the caller promises that the kernel enqueued just before each
                                       pkv_decode_attention call writes neither this cache's pools nor q (typical:
                                       the previous layer's decode with queries prepared in advance).  The kernel
@@ -124,9 +130,11 @@ typedef struct pkv_config {
                                       pkv_decode_attention).
                                    Work enqueued after a decode call by any other means (another kernel, a copy)
                                    still starts only after that call has completed, in every mode, and a decode
-                                   call that follows a pkv_append_kv or pkv_compress_eligible_pages call on this
-                                   cache always waits for it: the promise concerns other writers (of q, or of the
-                                   pools through their raw pointers) only. */
+                                   call that follows a pkv_append_kv, pkv_compress_eligible_pages,
+                                   pkv_compress_commit or pkv_write_factors call on this cache always waits for
+                                   it, in every mode: the promise concerns other writers (of q, or of the pools
+                                   through their raw pointers, which no mode allows while decode calls are in
+                                   flight) only. */
 } pkv_config;
 
 typedef struct pkv_sizes {
@@ -152,6 +160,11 @@ typedef struct pkv_stats {
     int64_t last_decode_bytes;       /* algorithmic HBM bytes of the most recent pkv_decode_attention call:
                                         factor blobs + valid dense rows + q + out */
     int64_t last_decode_units;       /* work units (factor pages + dense blocks) of that call */
+    int64_t page_svds;               /* K or V pages of one KV head factorized so far (Eq. 2, one SVD each) */
+    int64_t jacobi_rounds;           /* rotation rounds those SVDs took in total.  A round rotates P/2 disjoint pairs
+                                        (page size 16: P - 1 rounds per sweep) or P/4 disjoint groups of four indices,
+                                        six pairs each (page size 64: 21 rounds per sweep, 32: 13); see
+                                        pkv_get_rotation_schedule() */
 } pkv_stats;
 
 /* Sizes of the caller-allocated buffers for a configuration.  Validates cfg. */
@@ -336,12 +349,17 @@ pkv_status pkv_decode_attention_host(pkv_cache *c, int32_t layer, int32_t n_seqs
  * cache's own workspace buffer is not touched.
  *
  * Limits and rules
- *  - Capacity: n_ctas + n_seqs * n_kv_heads <= 1024 partial states.  A larger call is rejected
- *    with PKV_ERR_INVALID_ARG and a message; nothing is launched.
+ *  - Capacity: 1024 partial states: F + F / 8 + S + 2 <= 1024 with S = n_seqs * n_kv_heads and
+ *    F = n_ctas + S (one state per CTA and segment, plus the states of groups of eight CTAs that a
+ *    segment spread over many CTAs is summed through).  The default grid (296 CTAs) leaves room for
+ *    about 280 (sequence, KV head) pairs.  A larger call is rejected with PKV_ERR_INVALID_ARG and a
+ *    message; nothing is launched.
  *  - Cost: the array (about 4.1 MiB) is part of the library image, so every GPU on which the
  *    library is loaded holds it until the process exits, whether or not this function is called.
  *  - The first call on each device looks up the array's device address (the device must be
- *    current).  Make that first call outside any CUDA stream capture.
+ *    current).  Make that first call outside any CUDA stream capture.  As with
+ *    pkv_decode_attention(), a call whose plan must be rebuilt (new batch, or a page table
+ *    changed) returns PKV_ERR_UNSUPPORTED while `stream` is capturing.
  *  - All calls on a device share the one array, which keeps the previous call's contents; the
  *    function clears the part that must start at zero (the tickets) on `stream` before each
  *    launch.  Two calls that may run on the GPU at the same time (different streams without an
@@ -375,10 +393,13 @@ pkv_status pkv_get_decode_plan(const pkv_cache *c, int32_t layer, int32_t *n_use
 
 /*
  * Debugging aid.  When the environment variable PKV_DECODE_TRACE=1 is set at pkv_init_cache() time, every
- * CTA of a decode launch records eight 64-bit time stamps in the workspace: [0] globaltimer (ns) at entry,
+ * CTA of a decode launch records sixteen 64-bit values in the workspace: [0] globaltimer (ns) at entry,
  * [1] at exit, then SM clock counts: [2] entry, [3] first copy issued, [4] first unit's data arrived,
- * [5] last unit of the CTA consumed, [6] exit, [7] units processed.  This call synchronises `stream` and
- * copies the stamps of the most recent launch to out [host, n_ctas * 8 values].
+ * [5] last unit of the CTA consumed, [6] exit, [7] units processed (a count), [8] consumers released (mode 0:
+ * the preceding kernel has finished), and for the CTA's last segment [9] flush begun, [10] partial state and
+ * ticket done, [11] cross-CTA merge: copies issued, [12] first round landed, [13] result stored ([11]-[13] are 0
+ * unless this CTA merged); [14], [15] unused.  This call synchronises `stream` and copies the stamps of the most
+ * recent launch to out [host, n_ctas * 16 values].
  */
 pkv_status pkv_get_decode_trace(pkv_cache *c, int64_t *out, int32_t n_ctas, void *stream);
 

@@ -44,6 +44,7 @@ struct PlanCache {
     std::vector<uint64_t> versions;
     int q_len = 1;                     // query tokens per sequence the plan was built for
     int n_segs = 0;
+    int max_parts = 0;                 // most CTAs any segment is split over
     int64_t units = 0;
     std::vector<PlanCta> ctas;         // n_used + 1 entries (last = end sentinel)
     std::vector<PlanSeg> segs;
@@ -223,23 +224,27 @@ void derive(const pkv_config &cfg, int n_ctas, Geometry &g, MetaLayout &ml, Work
     ml.status = off;     off = align_up(off + 4LL * kStatusWords, 256);
     ml.total = off;
 
-    wl.n_partials = (long long)n_ctas + (long long)cfg.max_seqs * cfg.n_kv_heads;
+    wl.n_seg_tickets = (long long)cfg.max_seqs * cfg.n_kv_heads;
+    wl.n_flat = (long long)n_ctas + wl.n_seg_tickets;
+    wl.n_group = merge_group_slots(wl.n_flat, wl.n_seg_tickets);
+    wl.n_partials = wl.n_flat + wl.n_group;
     long long w = 0;
     wl.partials_stride = align_up(wl.n_partials * kPartialFloats * 4, 256);
-    wl.tickets_stride = align_up(4LL * cfg.max_seqs * cfg.n_kv_heads, 256);
+    wl.tickets_stride = align_up(4LL * (wl.n_seg_tickets + wl.n_group), 256);
     // decode_overlap = 2 rotates over several sets of split-K scratch; the more sets, the rarer the draining launch
     wl.n_sets = 1;
     if (cfg.decode_overlap == 2) {
         // sized for the largest grid pkv_query_sizes() may have assumed (512 CTAs), so that the count does not
         // depend on the grid actually used and the workspace the caller allocated is always large enough
-        const long long widest = align_up(((long long)std::max(512, n_ctas) + (long long)cfg.max_seqs * cfg.n_kv_heads) * kPartialFloats * 4, 256);
+        const long long widest_flat = (long long)std::max(512, n_ctas) + wl.n_seg_tickets;
+        const long long widest = align_up((widest_flat + merge_group_slots(widest_flat, wl.n_seg_tickets)) * kPartialFloats * 4, 256);
         const long long fit = kDecodeBufferBudget / (widest + wl.tickets_stride);
         wl.n_sets = (int)std::min<long long>(kMaxDecodeBuffers, std::max<long long>(4, fit));
     }
     wl.partials = w; w += wl.partials_stride * wl.n_sets;
     wl.worklist = w; w = align_up(w + (long long)sizeof(int2) * kCompressChunk, 256);
     wl.tickets = w;  w += wl.tickets_stride * wl.n_sets;
-    wl.trace = w;    w = align_up(w + 64LL * n_ctas, 256);
+    wl.trace = w;    w = align_up(w + 8LL * kTraceSlots * n_ctas, 256);
     wl.total = w;
 }
 
@@ -444,6 +449,8 @@ pkv_status build_plan(pkv_cache *c, int layer, int n_listed, const int32_t *seq_
     pc.versions.resize(n_listed);
     for (int i = 0; i < n_listed; ++i) pc.versions[i] = c->at(seq_ids[i], layer).version;
     pc.n_segs = n_segs;
+    pc.max_parts = 0;
+    for (const PlanSeg &sg : segs) pc.max_parts = std::max(pc.max_parts, sg.n_parts);
     pc.units = total_units;
     pc.ctas = ctas;
     pc.segs = segs;
@@ -608,6 +615,7 @@ pkv_status pkv_append_kv(pkv_cache *c, int32_t layer, int32_t n_seqs, const int3
         return fail(c, PKV_ERR_POOL_EXHAUSTED, "dense pool exhausted: need %lld slots, %lld free", need,
                     (long long)c->dense_free.available());
     if (!c->dry && n_tok > 0 && (!k || !v)) return fail(c, PKV_ERR_INVALID_ARG, "k or v is NULL");
+    if (((uintptr_t)k | (uintptr_t)v) & 15) return fail(c, PKV_ERR_INVALID_ARG, "k and v must be 16-byte aligned");
     if (n_tok == 0) return PKV_OK;
     if (!c->dry && is_capturing(st))
         return fail(c, PKV_ERR_UNSUPPORTED, "pkv_append_kv cannot be captured into a CUDA graph");
@@ -829,7 +837,8 @@ pkv_status pkv_compress_commit(pkv_cache *c, int32_t layer, void *main_stream, i
 }
 
 static pkv_status decode_impl(pkv_cache *c, int32_t layer, int32_t n_seqs, const int32_t *seq_ids, int32_t q_len,
-                              const void *q, void *out, float *out_f32, float *state, void *stream);
+                              const void *q, void *out, float *out_f32, float *state, void *stream,
+                              bool static_scratch = false);
 
 pkv_status pkv_decode_attention(pkv_cache *c, int32_t layer, int32_t n_seqs, const int32_t *seq_ids,
                                 const void *q, void *out, float *out_f32, void *stream) {
@@ -839,6 +848,16 @@ pkv_status pkv_decode_attention(pkv_cache *c, int32_t layer, int32_t n_seqs, con
 pkv_status pkv_decode_attention_multi(pkv_cache *c, int32_t layer, int32_t n_seqs, const int32_t *seq_ids,
                                       int32_t q_len, const void *q, void *out, float *out_f32, void *stream) {
     return decode_impl(c, layer, n_seqs, seq_ids, q_len, q, out, out_f32, nullptr, stream);
+}
+
+// Same validation, plan and accounting as pkv_decode_attention(); only the split-K scratch differs.
+pkv_status pkv_decode_attention_static_scratch(pkv_cache *c, int32_t layer, int32_t n_seqs,
+                                               const int32_t *seq_ids, const void *q, void *out, float *out_f32,
+                                               void *stream) {
+    if (!c) return PKV_ERR_INVALID_ARG;
+    if (c->dry) return fail(c, PKV_ERR_INVALID_ARG, "no device buffers in dry-run mode");
+    if (!out) return fail(c, PKV_ERR_INVALID_ARG, "q or out is NULL");
+    return decode_impl(c, layer, n_seqs, seq_ids, 1, q, out, out_f32, nullptr, stream, true);
 }
 
 pkv_status pkv_decode_attention_partial(pkv_cache *c, int32_t layer, int32_t n_seqs, const int32_t *seq_ids,
@@ -858,8 +877,13 @@ pkv_status pkv_merge_attention_states(const float *states, int32_t n_shards, int
                ? PKV_OK : PKV_ERR_CUDA;
 }
 
+// Alignment the kernels rely on: q rows are read as 32-bit words, out is written 8 bytes at a time, out_f32 16,
+// state rows (d + 2 floats) 8.
+static bool misaligned(const void *p, uintptr_t a) { return p && ((uintptr_t)p & (a - 1)) != 0; }
+
 static pkv_status decode_impl(pkv_cache *c, int32_t layer, int32_t n_seqs, const int32_t *seq_ids, int32_t q_len,
-                              const void *q, void *out, float *out_f32, float *state, void *stream) {
+                              const void *q, void *out, float *out_f32, float *state, void *stream,
+                              bool static_scratch) {
     if (!c) return PKV_ERR_INVALID_ARG;
     cudaStream_t st = (cudaStream_t)stream;
     if (layer < 0 || layer >= c->cfg.n_layers) return fail(c, PKV_ERR_INVALID_ARG, "layer %d out of range", layer);
@@ -886,6 +910,8 @@ static pkv_status decode_impl(pkv_cache *c, int32_t layer, int32_t n_seqs, const
         }
     }
     if (!c->dry && (!q || (!out && !state))) return fail(c, PKV_ERR_INVALID_ARG, "q or out is NULL");
+    if (misaligned(q, 4) || misaligned(out, 8) || misaligned(out_f32, 16) || misaligned(state, 8))
+        return fail(c, PKV_ERR_INVALID_ARG, "misaligned pointer: q needs 4-byte, out 8-byte, out_f32 16-byte, state 8-byte alignment");
     if (!plan_is_current(c, layer, n_seqs, seq_ids, q_len)) {
         // the plan is uploaded through the staging ring: a copy recorded into a graph would replay stale bytes
         if (!c->dry && is_capturing(st))
@@ -933,12 +959,30 @@ static pkv_status decode_impl(pkv_cache *c, int32_t layer, int32_t n_seqs, const
     c->cache_written = false;
     if (uses_row_blocks(c, q_len, n_seqs)) {
         // one ordinary launch (starts after everything before it on the stream); no split-K scratch involved
-        a.partials = nullptr; a.tickets = nullptr;
+        a.partials = nullptr; a.tickets = nullptr; a.gpartials = nullptr; a.gtickets = nullptr;
         a.status = (int *)(c->meta + c->ml.status);
         a.layer = layer;
         a.variant = 0; a.overlap = 0; a.plain_launch = 1; a.trace = nullptr;
         c->cache_written = false;
         PKV_CUDA(c, launch_decode_blocks(a, n_seqs, st));
+        return PKV_OK;
+    }
+    if (static_scratch) {
+        // partial states and tickets live in the library's own array (set by the launcher); the memset that clears
+        // the tickets already orders the launch behind all earlier work on the stream
+        a.partials = nullptr; a.tickets = nullptr; a.gpartials = nullptr; a.gtickets = nullptr;
+        a.plain_launch = 0;
+        a.status = (int *)(c->meta + c->ml.status);
+        a.layer = layer;
+        a.variant = c->cfg.decode_variant;
+        a.overlap = c->cfg.decode_overlap;
+        a.trace = nullptr;
+        const char *why = "";
+        cudaError_t e = launch_decode_static_scratch(a, pc.n_segs, st, &why);
+        if (e == cudaErrorInvalidValue && why[0])
+            return fail(c, PKV_ERR_INVALID_ARG, "pkv_decode_attention_static_scratch: %s", why);
+        if (e != cudaSuccess)
+            return fail(c, PKV_ERR_CUDA, "pkv_decode_attention_static_scratch: %s: %s", why, cudaGetErrorString(e));
         return PKV_OK;
     }
     if (c->cfg.decode_overlap == 2 && c->cfg.decode_variant != 1) {
@@ -956,56 +1000,14 @@ static pkv_status decode_impl(pkv_cache *c, int32_t layer, int32_t n_seqs, const
     }
     a.partials = (float *)(c->workspace + c->wl.partials + c->wl.partials_stride * buf);
     a.tickets = (int *)(c->workspace + c->wl.tickets + c->wl.tickets_stride * buf);
+    a.gpartials = a.partials + c->wl.n_flat * kPartialFloats;
+    a.gtickets = a.tickets + c->wl.n_seg_tickets;
     a.status = (int *)(c->meta + c->ml.status);
     a.layer = layer;
     a.variant = c->cfg.decode_variant;
     a.overlap = c->cfg.decode_overlap;
     a.trace = c->trace ? (long long *)(c->workspace + c->wl.trace) : nullptr;
     PKV_CUDA(c, launch_decode(a, pc.n_segs, st));
-    return PKV_OK;
-}
-
-pkv_status pkv_decode_attention_static_scratch(pkv_cache *c, int32_t layer, int32_t n_seqs,
-                                               const int32_t *seq_ids, const void *q, void *out, float *out_f32,
-                                               void *stream) {
-    if (!c) return PKV_ERR_INVALID_ARG;
-    if (c->dry) return fail(c, PKV_ERR_INVALID_ARG, "no device buffers in dry-run mode");
-    cudaStream_t st = (cudaStream_t)stream;
-    if (layer < 0 || layer >= c->cfg.n_layers) return fail(c, PKV_ERR_INVALID_ARG, "layer %d out of range", layer);
-    pkv_status r = check_seq_list(c, n_seqs, seq_ids);
-    if (r != PKV_OK) return r;
-    for (int i = 0; i < n_seqs; ++i)
-        if (c->at(seq_ids[i], layer).n_tokens == 0)
-            return fail(c, PKV_ERR_INVALID_ARG, "sequence %d has no tokens in layer %d", seq_ids[i], layer);
-    if (!q || !out) return fail(c, PKV_ERR_INVALID_ARG, "q or out is NULL");
-    if (!plan_is_current(c, layer, n_seqs, seq_ids, 1)) {
-        if ((r = build_plan(c, layer, n_seqs, seq_ids, 1, st)) != PKV_OK) return r;
-    }
-    DecodeArgs a;
-    a.geo = c->geo;
-    a.dense_pool = c->dense_pool; a.factor_pool = c->factor_pool;
-    a.page_table = (const int *)(c->meta + c->ml.page_table);
-    a.n_tokens = (const int *)(c->meta + c->ml.n_tokens);
-    a.plan = c->meta + c->ml.plans + c->ml.plan_stride * layer;
-    a.plan_cta = c->ml.plan_cta; a.plan_entry = c->ml.plan_entry; a.plan_seg = c->ml.plan_seg;
-    a.plan_cta_entry = c->ml.plan_cta_entry;
-    a.q = q; a.out = out; a.out_f32 = out_f32;
-    a.state = nullptr;
-    a.q_len = 1; a.q_tpt = 1; a.q_nblk = 1; a.q_group = 1; a.q_cols = c->geo.group;
-    a.partials = nullptr; a.tickets = nullptr;            // set by the launcher from the static scratch
-    a.plain_launch = 0;                                   // the launcher's memset already orders it after earlier work
-    c->cache_written = false;
-    a.status = (int *)(c->meta + c->ml.status);
-    a.layer = layer;
-    a.variant = c->cfg.decode_variant;
-    a.overlap = c->cfg.decode_overlap;
-    a.trace = nullptr;
-    const char *why = "";
-    cudaError_t e = launch_decode_static_scratch(a, c->plans[layer].n_segs, st, &why);
-    if (e == cudaErrorInvalidValue && why[0])
-        return fail(c, PKV_ERR_INVALID_ARG, "pkv_decode_attention_static_scratch: %s", why);
-    if (e != cudaSuccess)
-        return fail(c, PKV_ERR_CUDA, "pkv_decode_attention_static_scratch: %s: %s", why, cudaGetErrorString(e));
     return PKV_OK;
 }
 
@@ -1070,7 +1072,7 @@ pkv_status pkv_get_decode_trace(pkv_cache *c, int64_t *out, int32_t n_ctas, void
     if (!c || !out || c->dry || n_ctas <= 0 || n_ctas > c->geo.n_ctas) return PKV_ERR_INVALID_ARG;
     if (!c->trace) return fail(c, PKV_ERR_INVALID_ARG, "tracing is off: set PKV_DECODE_TRACE=1 before pkv_init_cache");
     PKV_CUDA(c, cudaStreamSynchronize((cudaStream_t)stream));
-    PKV_CUDA(c, cudaMemcpy(out, c->workspace + c->wl.trace, 64 * (size_t)n_ctas, cudaMemcpyDeviceToHost));
+    PKV_CUDA(c, cudaMemcpy(out, c->workspace + c->wl.trace, 8 * (size_t)kTraceSlots * n_ctas, cudaMemcpyDeviceToHost));
     return PKV_OK;
 }
 
@@ -1089,6 +1091,10 @@ pkv_status pkv_get_stats(pkv_cache *c, pkv_stats *out, void *stream) {
         out->device_timeouts = st[0];
         out->page_svds_not_converged = st[1];
         out->bad_slot_indices = st[2];
+        uint64_t wide[2];
+        memcpy(wide, st + 4, sizeof wide);
+        out->jacobi_rounds = (int64_t)wide[0];
+        out->page_svds = (int64_t)wide[1];
     }
     return PKV_OK;
 }
@@ -1139,6 +1145,7 @@ pkv_status pkv_write_factors(pkv_cache *c, int64_t slot, int32_t head, const voi
     if (!A_k || !B_k || !A_v || !B_v) return fail(c, PKV_ERR_INVALID_ARG, "input pointer is NULL");
     if (c->geo.factor_bits == 4) return fail(c, PKV_ERR_UNSUPPORTED, "pkv_write_factors is not available with INT4 factors");
     unsigned char *blob = c->factor_pool + slot * c->geo.factor_slot_bytes + (int64_t)head * c->geo.blob_bytes;
+    c->cache_written = true;                     // the next decode launch must not start ahead of this kernel
     PKV_CUDA(c, launch_write_factors(c->geo, blob, A_k, B_k, A_v, B_v, (cudaStream_t)stream));
     return PKV_OK;
 }

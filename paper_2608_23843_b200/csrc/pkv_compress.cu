@@ -250,6 +250,7 @@ compress_kernel(Geometry geo, const unsigned char *dense_pool, unsigned char *fa
     for (int w = 0; w < kWarps; ++w) trace += S.red[w];
     float captured_prev = -1.f;
     bool converged = false;
+    int n_rounds = 0;                 // rotation rounds (classes of quads, or rounds of pairs) this page went through
     if constexpr (P >= 32) {
         using Qd = Quads<P>;
         constexpr int kQuads = Qd::kQuads;
@@ -277,6 +278,7 @@ compress_kernel(Geometry geo, const unsigned char *dense_pool, unsigned char *fa
             int rotated = 0;
             for (int cls = 0; cls < Qd::kClasses && !converged; ++cls) {
                 const uchar4 *quads = S.quads + cls * kQuads;
+                ++n_rounds;
                 if (tid < 4 * kQuads) {
                     // Four lanes per quad; lane t holds row t of the quad's diagonal block D and of M, stored
                     // "rotated": e[k] = D[t][t ^ k], f[k] = M[t][t ^ k], so that the partner of layer x (t ^ x), the
@@ -431,6 +433,7 @@ compress_kernel(Geometry geo, const unsigned char *dense_pool, unsigned char *fa
             int rotated = 0;
             for (int rho = 0; rho < P - 1; ++rho) {
                 const uchar2 *pr = pairs + rho * kPairs;
+                ++n_rounds;
                 if (tid < kPairs) {
                     const int p = pr[tid].x, q = pr[tid].y;
                     const float gpp = S.G[p * kGs + p], gqq = S.G[q * kGs + q], gpq = S.G[p * kGs + q];
@@ -492,7 +495,12 @@ compress_kernel(Geometry geo, const unsigned char *dense_pool, unsigned char *fa
             if (!converged && geo.jacobi_energy_tol >= 0.f && energy_converged<P>(S, rank, geo.jacobi_energy_tol, trace, captured_prev, tid, lane, warp)) converged = true;
         }
     }
-    if (!converged && tid == 0) atomicAdd(&status[1], 1);
+    if (tid == 0) {
+        if (!converged) atomicAdd(&status[1], 1);
+        // 64-bit totals for the throughput report: rounds and page SVDs
+        atomicAdd(reinterpret_cast<unsigned long long *>(status + 4), (unsigned long long)n_rounds);
+        atomicAdd(reinterpret_cast<unsigned long long *>(status + 6), 1ull);
+    }
 
     // ---- order eigenvalues: descending, ties by lower index ----
     if (tid < P) { S.lam[tid] = S.G[tid * kGs + tid]; S.order[tid] = tid; }

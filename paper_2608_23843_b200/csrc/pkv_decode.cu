@@ -4,7 +4,7 @@
 // host into byte-balanced contiguous ranges, one per persistent CTA.  Inside a
 // CTA a producer warp walks the page table and streams whole factor blobs / dense
 // row blocks into a shared-memory ring with bulk async copies (TMA, mbarrier
-// completion); eight consumer warps each take one unit at a time and evaluate
+// completion); five consumer warps each take one unit at a time and evaluate
 //     q~ = B_k q          (tensor cores, bf16 x bf16 -> fp32)
 //     s  = A_k q~ * scale (q~ split into two bf16 terms so the exponent sees ~fp32)
 //     online softmax      (fp32, exp2 with the scale folded in)
@@ -348,7 +348,7 @@ __device__ __forceinline__ uint32_t pack_bf16(float lo, float hi) {
 __device__ __forceinline__ float bf16lo_f(uint32_t x) { return __uint_as_float(x << 16); }
 __device__ __forceinline__ float bf16hi_f(uint32_t x) { return __uint_as_float(x & 0xffff0000u); }
 
-struct StageDesc { int kind, rows, seg, after; };     // after: tokens of the sequence that follow this unit's rows
+struct StageDesc { int kind, rows, seg, after; };
 
 // Per-warp running state for the query heads 2t, 2t+1 (t = lane & 3) of one KV head.
 struct WarpState {
@@ -763,11 +763,23 @@ __device__ __forceinline__ void store_out(const DecodeArgs &a, int seg, int hq, 
     if (a.out_f32) *reinterpret_cast<float4 *>(a.out_f32 + off) = acc;
 }
 
-// Eq. 5 across CTAs: the partial states of one segment, summed in CTA order with a running maximum (one pass).
+// One step of Eq. 5: folds the state (o, m, l) into the running (tot, Mr, Lr).  Spelled with explicit roundings so
+// that every caller (the merge inside the decode kernel, the separate merge kernel) produces the same bits.
+__device__ __forceinline__ void fold_state(float4 &tot, float &Mr, float &Lr, const float4 o, float m, float l) {
+    const float Mn = fmaxf(Mr, m);
+    const float fa = exp2f(Mr - Mn), fb = exp2f(m - Mn);
+    tot.x = __fmaf_rn(fb, o.x, __fmul_rn(tot.x, fa)); tot.y = __fmaf_rn(fb, o.y, __fmul_rn(tot.y, fa));
+    tot.z = __fmaf_rn(fb, o.z, __fmul_rn(tot.z, fa)); tot.w = __fmaf_rn(fb, o.w, __fmul_rn(tot.w, fa));
+    Lr = __fmaf_rn(fb, l, __fmul_rn(Lr, fa));
+    Mr = Mn;
+}
+
+// Eq. 5 across CTAs: partial states summed in CTA order with a running maximum (one pass).
 // A thread owns E items (query head, four dims): ctid, ctid + kThreads, ...; kBatch parts' loads are in flight at a
 // time, because with dozens of parts it is the latency of these loads that the rest of the GPU waits for.
 template <int E, int kBatch>
-__device__ __forceinline__ void merge_parts(const DecodeArgs &a, const float *first, int np, int seg, int ctid) {
+__device__ __forceinline__ void merge_parts(const DecodeArgs &a, const float *first, int np, int seg, int ctid,
+                                            float *dst) {
     const long long stride = (long long)a.q_group * kPartialFloats;     // between the states of consecutive ranges
     constexpr int kThreads = kConsumerWarps * 32;
     const int n_items = a.q_cols * 32;
@@ -801,20 +813,20 @@ __device__ __forceinline__ void merge_parts(const DecodeArgs &a, const float *fi
         for (int j = 0; j < kBatch; ++j) {
             if (k0 + j < np) {
 #pragma unroll
-                for (int e = 0; e < E; ++e) {
-                    const float Mn = fmaxf(Mr[e], m[e][j]);
-                    const float fa = exp2f(Mr[e] - Mn), fb = exp2f(m[e][j] - Mn);
-                    tot[e].x = tot[e].x * fa + fb * o[e][j].x; tot[e].y = tot[e].y * fa + fb * o[e][j].y;
-                    tot[e].z = tot[e].z * fa + fb * o[e][j].z; tot[e].w = tot[e].w * fa + fb * o[e][j].w;
-                    Lr[e] = Lr[e] * fa + fb * l[e][j];
-                    Mr[e] = Mn;
-                }
+                for (int e = 0; e < E; ++e) fold_state(tot[e], Mr[e], Lr[e], o[e][j], m[e][j], l[e][j]);
             }
         }
     }
 #pragma unroll
-    for (int e = 0; e < E; ++e)
-        if (has[e]) store_out(a, seg, hq[e], d4, tot[e], Mr[e], Lr[e]);
+    for (int e = 0; e < E; ++e) {
+        if (!has[e]) continue;
+        if (dst) {                                                    // the sum is itself a partial state (of a group)
+            *reinterpret_cast<float4 *>(dst + hq[e] * kHeadDim + d4) = tot[e];
+            if (d4 == 0) { dst[kMaxGroup * kHeadDim + hq[e]] = Mr[e]; dst[kMaxGroup * kHeadDim + kMaxGroup + hq[e]] = Lr[e]; }
+        } else {
+            store_out(a, seg, hq[e], d4, tot[e], Mr[e], Lr[e]);
+        }
+    }
 }
 
 #define PKV_CONSUMER_BARRIER() asm volatile("bar.sync 1, %0;" ::"n"(kConsumerWarps * 32) : "memory")
@@ -824,9 +836,11 @@ __device__ __forceinline__ void merge_parts(const DecodeArgs &a, const float *fi
 // ticket, and the CTA that draws the last ticket of the segment applies Eq. 5 across CTAs.  Partials
 // are always summed in CTA order, so the result does not depend on which CTA arrives last.
 __device__ __forceinline__ void flush_segment(const DecodeArgs &a, float *comb, volatile int *last_flag, WarpState &st,
-                                              int seg, int warp, int lane, int ctid, int n_active) {
+                                              int seg, const PlanSeg ps, int warp, int lane, int ctid, int n_active,
+                                              long long *trace) {
     constexpr int kThreads = kConsumerWarps * 32, kItems = kMaxGroup * 32;   // item = (query head, 4 dims)
     const int g = lane >> 2, t = lane & 3;
+    if (trace && ctid == 0) trace[9] = clock64();
     if (warp < n_active) {
         float l0 = st.l[0], l1 = st.l[1];
 #pragma unroll
@@ -852,7 +866,6 @@ __device__ __forceinline__ void flush_segment(const DecodeArgs &a, float *comb, 
     PKV_CONSUMER_BARRIER();
     // overlap mode 1: partial states, tickets and `out` may still be in use by the preceding launch
     if (a.overlap == 1) asm volatile("griddepcontrol.wait;" ::: "memory");
-    const PlanSeg ps = reinterpret_cast<const PlanSeg *>(a.plan + a.plan_seg)[seg];
     const int qseg = query_seg(a, seg);
     float *part = partial_slot(a, blockIdx.x / a.q_group, seg);
     for (int item = ctid; item < kItems; item += kThreads) {
@@ -879,16 +892,54 @@ __device__ __forceinline__ void flush_segment(const DecodeArgs &a, float *comb, 
         }
     }
     if (ps.n_parts > 1) {
-        __threadfence();
-        PKV_CONSUMER_BARRIER();
-        if (ctid == 0) *last_flag = (atomicAdd(a.tickets + qseg, 1) == ps.n_parts - 1);
-        PKV_CONSUMER_BARRIER();
-        if (*last_flag) {
-            __threadfence();
-            const float *first = partial_slot(a, ps.cta_first, seg);
-            if (a.q_cols * 32 <= kThreads) merge_parts<1, 16>(a, first, ps.n_parts, qseg, ctid);
-            else merge_parts<2, 8>(a, first, ps.n_parts, qseg, ctid);
-            if (ctid == 0) a.tickets[qseg] = 0;         // ready for the next launch
+        // Drawing a ticket: the barrier orders every thread's stores of the state before thread 0's fence, which
+        // makes them visible device-wide before the ticket is drawn; on the way back thread 0's second fence and the
+        // barrier order the other CTAs' states (whose tickets this one has seen) before every thread's reads of them.
+        // A segment held by more than kMergeFan CTAs is summed in two levels: the CTAs form groups of kMergeFan
+        // consecutive ranges; the last of a group to arrive sums the group's states into a group state, and the last
+        // group to arrive sums the group states.  The slowest CTA of the launch then has one short sum of its
+        // group and one of the groups ahead of it instead of one long sum of everything, and the other groups'
+        // sums are over before it arrives.  The grouping is fixed, so the bits do not depend on who arrives when.
+        const float *first = partial_slot(a, ps.cta_first, seg);
+        int np = ps.n_parts;
+        bool mine = true;                                  // this CTA still carries the sum upwards
+        if (a.q_group == 1 && ps.n_parts > kMergeFan) {
+            const int k = blockIdx.x - ps.cta_first, g = k / kMergeFan;
+            const int gsize = min(kMergeFan, ps.n_parts - g * kMergeFan);
+            const int gslot0 = (ps.cta_first + seg) / kMergeFan + seg;     // group slots of consecutive groups and segments never collide
+            PKV_CONSUMER_BARRIER();
+            if (ctid == 0) {
+                __threadfence();
+                *last_flag = (atomicAdd(a.gtickets + gslot0 + g, 1) == gsize - 1);
+                __threadfence();
+            }
+            PKV_CONSUMER_BARRIER();
+            mine = *last_flag != 0;
+            if (mine) {
+                float *dst = a.gpartials + (long long)(gslot0 + g) * kPartialFloats;
+                const float *gfirst = first + (long long)g * kMergeFan * kPartialFloats;
+                if (a.q_cols * 32 <= kThreads) merge_parts<1, 16>(a, gfirst, gsize, qseg, ctid, dst);
+                else merge_parts<2, 8>(a, gfirst, gsize, qseg, ctid, dst);
+                if (ctid == 0) a.gtickets[gslot0 + g] = 0;     // ready for the next launch
+                first = a.gpartials + (long long)gslot0 * kPartialFloats;
+                np = (ps.n_parts + kMergeFan - 1) / kMergeFan;
+            }
+        }
+        if (mine) {
+            PKV_CONSUMER_BARRIER();
+            if (ctid == 0) {
+                __threadfence();
+                *last_flag = (atomicAdd(a.tickets + qseg, 1) == np - 1);
+                __threadfence();
+            }
+            PKV_CONSUMER_BARRIER();
+            if (trace && ctid == 0) trace[10] = clock64();
+            if (*last_flag) {
+                if (a.q_cols * 32 <= kThreads) merge_parts<1, 16>(a, first, np, qseg, ctid, nullptr);
+                else merge_parts<2, 8>(a, first, np, qseg, ctid, nullptr);
+                if (ctid == 0) a.tickets[qseg] = 0;         // ready for the next launch
+                if (trace && ctid == 0) trace[13] = clock64();
+            }
         }
     }
     PKV_CONSUMER_BARRIER();
@@ -919,12 +970,13 @@ __global__ void __launch_bounds__(kDecodeThreads, 2) decode_tc_kernel(const __gr
     volatile int *armed = abort_flag + 2;
 
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
-    long long *trace = a.trace ? a.trace + 8LL * blockIdx.x : nullptr;
+    long long *trace = a.trace ? a.trace + (long long)kTraceSlots * blockIdx.x : nullptr;
     if (trace && tid == 0) {
         unsigned long long gt;
         asm volatile("mov.u64 %0, %globaltimer;" : "=l"(gt));
         trace[0] = (long long)gt;
         trace[2] = clock64();
+        for (int i = 8; i < kTraceSlots; ++i) trace[i] = 0;
     }
     if (tid == 0) {
         for (int s = 0; s < S; ++s) { mbar_init(smem_u32(full_bar + s), 1); mbar_init(smem_u32(empty_bar + s), 1); }
@@ -943,11 +995,14 @@ __global__ void __launch_bounds__(kDecodeThreads, 2) decode_tc_kernel(const __gr
         asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
     }
     __syncthreads();
-    // Programmatic dependent launch: let the next kernel on the stream begin as SMs free up.  Unless the caller
-    // vouched that the preceding kernel writes neither this cache nor q (overlap mode), wait for it to finish
-    // before reading anything it may have produced.  Mode 1 waits later, before the shared split-K scratch is
-    // touched (flush_segment); mode 2 never waits: the host rotates the scratch and drains the stream in time.
-    if (!a.overlap) asm volatile("griddepcontrol.wait;" ::: "memory");
+    // Programmatic dependent launch: let the next kernel on the stream begin as SMs free up.  What the producer
+    // reads - plan, page table, token counts, pages - is written only by this library's own uploads and kernels
+    // (append, compression, pkv_write_factors), and the host makes the first decode launch after any of those an
+    // ordinary one, which starts when they are done; so the producer never has to wait for the kernel before this
+    // one and fills the ring while that kernel is still finishing.  The queries may come from that kernel:
+    // mode 0 (no promise from the caller) makes every consumer warp wait for it before it reads q.  Mode 1 waits
+    // later, before the shared split-K scratch is touched (flush_segment); mode 2 never waits: the host rotates
+    // the scratch and drains the stream in time.
     asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
 
     if (warp == kConsumerWarps) {
@@ -1058,9 +1113,22 @@ __global__ void __launch_bounds__(kDecodeThreads, 2) decode_tc_kernel(const __gr
         // ------------------------------ consumers ------------------------------
         WarpState st;
         reset_state(st);
+        // Only the first and the last segment of a range can be shared with other CTAs.  What their flushes need
+        // from global memory - the segment's place in the plan, its ticket - is fetched now, while the warp would
+        // otherwise just wait for the kernel before this one (the plan is host-written, the tickets are zero
+        // between launches).
+        const PlanSeg *plan_segs = reinterpret_cast<const PlanSeg *>(a.plan + a.plan_seg);
+        const PlanSeg ps_first = plan_segs[rg.seg_first], ps_last = plan_segs[rg.seg_first + rg.n_local_segs - 1];
+        if (lane == 0 && a.q_group == 1) {
+            asm volatile("prefetch.global.L2 [%0];" ::"l"(a.tickets + rg.seg_first));
+            asm volatile("prefetch.global.L2 [%0];" ::"l"(a.tickets + rg.seg_first + rg.n_local_segs - 1));
+        }
+        auto seg_info = [&](int sg) { return sg == 0 ? ps_first : (sg == rg.n_local_segs - 1 ? ps_last : PlanSeg{(int)(blockIdx.x / a.q_group), 1}); };
+        if (!a.overlap) asm volatile("griddepcontrol.wait;" ::: "memory");
+        if (trace && tid == 0) trace[8] = clock64();
         if (warp >= W) {
             for (int sg = 0; sg < rg.n_local_segs; ++sg)
-                flush_segment(a, comb, last_flag, st, rg.seg_first + sg, warp, lane, tid, W);
+                flush_segment(a, comb, last_flag, st, rg.seg_first + sg, seg_info(sg), warp, lane, tid, W, nullptr);
             return;
         }
         uint32_t qf[8][2];
@@ -1081,7 +1149,7 @@ __global__ void __launch_bounds__(kDecodeThreads, 2) decode_tc_kernel(const __gr
                 // hides behind the flush
                 if (dsc.seg < rg.n_local_segs) hidden = load_q(a, query_seg(a, rg.seg_first + dsc.seg), qf, lane);
                 while (cur_seg < dsc.seg) {
-                    flush_segment(a, comb, last_flag, st, rg.seg_first + cur_seg, warp, lane, tid, W);
+                    flush_segment(a, comb, last_flag, st, rg.seg_first + cur_seg, seg_info(cur_seg), warp, lane, tid, W, trace);
                     ++cur_seg;
                     reset_state(st);
                 }
@@ -1687,9 +1755,11 @@ cudaError_t launch_merge_states(const float *states, int n_shards, long long n_r
 cudaError_t launch_decode_static_scratch(const DecodeArgs &a, int n_segs, cudaStream_t st, const char **why) {
     static unsigned char *scratch_of_device[64] = {};
     *why = "";
-    if ((long long)a.geo.n_ctas + n_segs > kStaticPartialStates || n_segs > kStaticTickets) {
+    // per-CTA states, then the states of groups of CTAs; tickets per segment, then per group
+    const long long n_flat = (long long)a.geo.n_ctas + n_segs, n_group = merge_group_slots(n_flat, n_segs);
+    if (n_flat + n_group > kStaticPartialStates || n_segs + n_group > kStaticTickets) {
         *why = "call needs more split-K partial states than the static scratch holds "
-               "(n_ctas + n_seqs * n_kv_heads must be <= 1024)";
+               "(F + F / 8 + S + 2 must be <= 1024, with S = n_seqs * n_kv_heads and F = n_ctas + S)";
         return cudaErrorInvalidValue;
     }
     int dev = -1;
@@ -1706,8 +1776,10 @@ cudaError_t launch_decode_static_scratch(const DecodeArgs &a, int n_segs, cudaSt
     DecodeArgs b = a;
     b.partials = reinterpret_cast<float *>(base);
     b.tickets = reinterpret_cast<int *>(base + kStaticTicketOffset);
+    b.gpartials = b.partials + n_flat * kPartialFloats;
+    b.gtickets = b.tickets + n_segs;
     // the array keeps whatever the previous call (or an aborted one) left: tickets must start at zero
-    e = cudaMemsetAsync(b.tickets, 0, (size_t)n_segs * sizeof(int), st);
+    e = cudaMemsetAsync(b.tickets, 0, (size_t)(n_segs + n_group) * sizeof(int), st);
     if (e != cudaSuccess) { *why = "clearing the tickets failed"; return e; }
     e = launch_decode(b, n_segs, st);
     if (e != cudaSuccess) *why = "kernel launch failed";

@@ -15,11 +15,16 @@ constexpr int kMaxGroup = 8;           // query heads per KV head handled by the
 constexpr int kConsumerWarps = 5;      // decode kernel: warps that compute (two CTAs share an SM; 6 warps x 168 regs x 2 fit the register file)
 constexpr int kDecodeThreads = (kConsumerWarps + 1) * 32;
 constexpr int kPartialFloats = kMaxGroup * (kHeadDim + 2);   // o[8][128], m[8], l[8]
-constexpr int kStatusWords = 8;        // [0] device timeouts, [1] page SVDs not converged, [2] slot indices out of range
+constexpr int kStatusWords = 8;        // [0] device timeouts, [1] page SVDs not converged, [2] slot indices out of range,
+                                       // [4..5] Jacobi rounds executed (64-bit), [6..7] page SVDs run (64-bit)
 constexpr int kCompressChunk = 8192;   // work-list entries per compression launch
 constexpr int kMaxDecodeBuffers = 64;  // decode_overlap = 2: at most this many rotating sets of split-K scratch
 constexpr long long kDecodeBufferBudget = 128LL << 20;   // ... and at most this many bytes of them (but at least 4 sets)
 constexpr int kSmemBudget = 227 * 1024;
+constexpr int kMergeFan = 8;           // partial states summed at a time by the cross-CTA merge (see flush_segment)
+// Group states and tickets a launch with `n_flat` per-CTA state slots and `n_segs` segments may index.
+inline long long merge_group_slots(long long n_flat, long long n_segs) { return n_flat / kMergeFan + n_segs + 2; }
+constexpr int kTraceSlots = 16;        // 64-bit time stamps per CTA of a traced decode launch
 
 // Sizes derived from a validated pkv_config.  Plain data: passed to kernels by value.
 struct Geometry {
@@ -72,14 +77,15 @@ struct MetaLayout {                    // byte offsets inside the caller's `meta
 
 struct WorkspaceLayout {
     int n_sets;                        // rotating sets of split-K scratch: 1 unless decode_overlap = 2
-    long long partials;                // float [n_sets][n_partials][kPartialFloats]
-    long long n_partials;
+    long long partials;                // float [n_sets][n_partials][kPartialFloats]: per-CTA states, then group states
+    long long n_partials;              // = n_flat + n_group
+    long long n_flat, n_group, n_seg_tickets;
     long long partials_stride;         // bytes of one buffer
     long long tickets_stride;
 
     long long worklist;                // int2 [kCompressChunk]
-    long long tickets;                 // int [max_seqs * n_kv_heads]
-    long long trace;                   // long long [n_ctas][8]
+    long long tickets;                 // int [n_sets][n_seg_tickets + n_group]: per segment, then per group
+    long long trace;                   // long long [n_ctas][kTraceSlots]
     long long total;
 };
 
@@ -99,6 +105,8 @@ struct DecodeArgs {
     float *state;                      // not NULL: write (o unnormalised, m, l) rows of d + 2 floats instead of out / out_f32
     float *partials;
     int *tickets;                      // one per segment, zero between launches
+    float *gpartials;                  // states of groups of kMergeFan CTAs (segments split over more CTAs than that)
+    int *gtickets;                     // one per group, zero between launches
 
     // Queries per sequence (1 = decoding).  A score tile has eight query columns: q_tpt = min(q_len, 8 / group)
     // consecutive query tokens fill q_cols = q_tpt * group of them, so a sequence has b = ceil(q_len / q_tpt) blocks of
@@ -111,7 +119,7 @@ struct DecodeArgs {
     int variant;                       // 0 = tensor-core pipeline, 1 = scalar reference kernel
     int overlap;                       // 0 wait at entry, 1 wait before the first partial state is written, 2 never wait
     int plain_launch;                  // launch without programmatic serialization (drains the stream first)
-    long long *trace;                  // NULL, or [n_ctas][8] time stamps written by each CTA (debugging)
+    long long *trace;                  // NULL, or [n_ctas][kTraceSlots] time stamps written by each CTA (debugging)
 };
 
 // Launchers (defined in the .cu files); all return the launch error.

@@ -35,9 +35,11 @@ __global__ void append_kernel(Geometry geo, unsigned char *dense_pool, const int
         const AppendDesc e = desc[lo];
         const int t = e.t_start + (int)(tok - e.tok_begin);
         const int page = t / geo.page, row = t % geo.page;
-        const int slot = page_table[((long long)e.seq * geo.n_layers + layer) * geo.max_pages + page];
-        if (slot < 0 || slot >= geo.n_dense_slots || page >= geo.max_pages) {
-            if (chunk == 0 && kv == 0 && h == 0) atomicAdd(status + 2, 1);   // corrupt page table: skip the row
+        // a corrupt descriptor or page table: skip the row, leave a mark (checked before the table is indexed)
+        const bool in_table = t >= 0 && page < geo.max_pages && e.seq >= 0 && e.seq < geo.max_seqs;
+        const int slot = in_table ? page_table[((long long)e.seq * geo.n_layers + layer) * geo.max_pages + page] : -1;
+        if (slot < 0 || slot >= geo.n_dense_slots) {
+            if (chunk == 0 && kv == 0 && h == 0) atomicAdd(status + 2, 1);
             continue;
         }
         const uint4 val = (kv ? v : k)[(tok * H + h) * 16 + chunk];

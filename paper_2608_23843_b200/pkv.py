@@ -56,7 +56,7 @@ class PkvSizes(ctypes.Structure):
 class PkvStats(ctypes.Structure):
     _fields_ = [(n, ctypes.c_int64) for n in ("dense_slots_in_use", "factor_slots_in_use", "pages_compressed",
                                               "page_svds_not_converged", "device_timeouts", "bad_slot_indices",
-                                              "last_decode_bytes", "last_decode_units")]
+                                              "last_decode_bytes", "last_decode_units", "page_svds", "jacobi_rounds")]
 
 
 class PkvError(RuntimeError):
@@ -276,10 +276,10 @@ def pkv_get_decode_plan(handle, layer, n_ctas, n_seqs, n_kv_heads):
 
 
 def pkv_get_decode_trace(handle, n_ctas, stream=None):
-    """Per-CTA time stamps of the last decode launch (needs PKV_DECODE_TRACE=1 at init): list of 8-tuples."""
-    buf = (ctypes.c_int64 * (8 * n_ctas))()
+    """Per-CTA time stamps of the last decode launch (needs PKV_DECODE_TRACE=1 at init): list of 16-tuples."""
+    buf = (ctypes.c_int64 * (16 * n_ctas))()
     _check(handle, lib().pkv_get_decode_trace(handle, buf, n_ctas, _stream(stream)))
-    return [tuple(buf[8 * i:8 * i + 8]) for i in range(n_ctas)]
+    return [tuple(buf[16 * i:16 * i + 16]) for i in range(n_ctas)]
 
 
 def pkv_free_seq(handle, seq):

@@ -45,6 +45,20 @@ def test_reference_arm_under_torchrun_prints_once():
     assert d["config"]["workload"] == "tiny" and d["value"] > 0
 
 
+def test_plain_launch_with_gpus_2_starts_two_ranks_itself():
+    """`python bench.py --gpus 2` without a launcher around it must start one rank per GPU on its own (here the
+    reference arm, which needs no GPU): one JSON line, n_gpus 2, and both ranks ran (rank 1 leaves a marker)."""
+    cmd = [sys.executable, os.path.join(ROOT, "bench.py"), "--impl", "reference", "--gpus", "2", "--workload", "tiny",
+           "--steps", "1", "--warmup", "0"]
+    env = {k: v for k, v in os.environ.items() if k not in ("WORLD_SIZE", "RANK", "LOCAL_RANK")}
+    env.update(OMP_NUM_THREADS="2", PKV_BENCH_RANK_MARKER="1")
+    r = subprocess.run(cmd, capture_output=True, text=True, timeout=300, env=env, cwd=ROOT)
+    assert r.returncode == 0, r.stderr[-2000:]
+    lines = [json.loads(l) for l in r.stdout.splitlines() if l.startswith("{")]
+    assert len(lines) == 1 and lines[0]["n_gpus"] == 2 and lines[0]["impl"] == "reference"
+    assert "rank 1 of 2 present" in r.stderr
+
+
 def _shard_worker(rank, world, port, out):
     """Each rank owns a token range of one sequence, computes its softmax state with the oracle, and gathers the
     states with the package's helper (gloo, CPU tensors)."""

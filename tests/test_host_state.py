@@ -238,6 +238,27 @@ def test_error_codes_and_unchanged_state_on_failure():
     assert gpu2.page_table(0, 0)[0] == [1, 0, 0]                      # the page converted before exhaustion stays converted
 
 
+def test_misaligned_caller_pointers_are_refused_before_any_launch():
+    """The kernels read k/v 16 bytes at a time and q as 32-bit words, and write out 8 and out_f32 16 bytes at a
+    time: a pointer that breaks this is an argument error, not a device fault.  Checked on the host, so a dry-run
+    cache (which never dereferences anything) can show it with made-up addresses."""
+    gpu, _, _ = _pair(n_dense_slots=8, n_factor_slots=4, n_layers=1)
+    L, h = pkv.lib(), gpu.handle
+    ids, cnt = (ctypes.c_int32 * 1)(0), (ctypes.c_int32 * 1)(3)
+    assert L.pkv_append_kv(h, 0, 1, ids, cnt, 0x10008, 0x20000, None) == pkv.PKV_ERR_INVALID_ARG
+    assert L.pkv_append_kv(h, 0, 1, ids, cnt, 0x10000, 0x20004, None) == pkv.PKV_ERR_INVALID_ARG
+    assert gpu.page_table(0, 0) == ([], [], 0)                         # nothing was appended
+    assert L.pkv_append_kv(h, 0, 1, ids, cnt, 0x10000, 0x20000, None) == pkv.PKV_OK
+    good = dict(q=0x1000, out=0x2000, f32=0x3000)
+    for bad in (dict(q=0x1002), dict(out=0x2004), dict(f32=0x3008)):
+        a = dict(good, **bad)
+        st = L.pkv_decode_attention(h, 0, 1, ids, a["q"], a["out"], a["f32"], None)
+        assert st == pkv.PKV_ERR_INVALID_ARG, (bad, st)
+        assert L.pkv_decode_attention_multi(h, 0, 1, ids, 2, a["q"], a["out"], a["f32"], None) == pkv.PKV_ERR_INVALID_ARG
+    assert L.pkv_decode_attention_partial(h, 0, 1, ids, 0x1000, 0x5004, None) == pkv.PKV_ERR_INVALID_ARG
+    assert L.pkv_decode_attention(h, 0, 1, ids, good["q"], good["out"], good["f32"], None) == pkv.PKV_OK
+
+
 def test_config_validation():
     ok = dict(n_layers=1, n_kv_heads=1, n_q_heads=4, rank=16, sink_tokens=64, recent_tokens=64, max_seqs=1,
               max_pages_per_seq=4, n_dense_slots=4, n_factor_slots=4)
