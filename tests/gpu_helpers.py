@@ -95,19 +95,64 @@ def attention_gates(pair, layer, order, q, got, got32):
     for s in order:
         pair.load_gpu_factors_into_oracle(s, layer)
     ref_kernel = pair.orc.decode_attention(layer, order, qd)
+    vmax = [entry_vmax(pair.orc, s, layer) for s in order]      # (the oracle holds the GPU's factors at this point)
     pair.orc.factor = saved
     n = len(order)
     return dict(kernel=[rel_err(got32[i], ref_kernel[i]) for i in range(n)],
                 kernel_bf16=[rel_err(got[i], ref_kernel[i]) for i in range(n)],
                 e2e=[rel_err(got[i], ref[i]) for i in range(n)],
-                floor=[rel_err(ref_rounded[i], ref[i]) for i in range(n)])
+                floor=[rel_err(ref_rounded[i], ref[i]) for i in range(n)],
+                abs32=[float(np.abs(got32[i] - ref_kernel[i]).max()) for i in range(n)],
+                abs16=[float(np.abs(got[i] - ref_kernel[i]).max()) for i in range(n)],
+                norm=[float(np.abs(ref_kernel[i]).max()) for i in range(n)], vmax=vmax)
+
+
+E2E_FLOOR_FACTOR, E2E_FLOOR_CAP = 2.0, 0.10
 
 
 def assert_attention_gates(g, tol=1e-2, kernel_f32_tol=4e-3):
+    """Kernel gate: the stated tolerance as is.  End-to-end gate: the stated 1e-2 plus 2 x floor, where floor is what
+    storing the factors in bf16 costs the oracle itself on this query (no implementation that stores bf16 factors
+    can do better than its floor).  The GPU's rounding is an independent draw of that noise, and its factors may be
+    a different, equally optimal set near the rank cut, so its max-abs error is another sample of the floor's
+    distribution, not the floor itself: measured ratios (e2e - 1e-2) / floor run from below 0 to 1.7 (the full-size
+    workloads: e2e / floor between 0.85 and 1.4, see tests/results/parity_fullsize.jsonl); 1.5 x was tried and
+    failed one small ragged case at 1.7.  A floor above 10 % would mean the inputs, not the kernel, decide the
+    comparison: the test then fails."""
     for i in range(len(g["e2e"])):
         assert g["kernel"][i] <= kernel_f32_tol, ("kernel gate (fp32 out)", i, g["kernel"][i])
         assert g["kernel_bf16"][i] <= tol, ("kernel gate", i, g["kernel_bf16"][i])
-        assert g["e2e"][i] <= tol + 3.0 * g["floor"][i], ("end-to-end gate", i, g["e2e"][i], g["floor"][i])
+        assert g["floor"][i] <= E2E_FLOOR_CAP, ("bf16-storage floor of the oracle itself", i, g["floor"][i])
+        assert g["e2e"][i] <= tol + E2E_FLOOR_FACTOR * g["floor"][i], ("end-to-end gate", i, g["e2e"][i], g["floor"][i])
+
+
+def entry_vmax(orc, seq, layer):
+    """max |v| over the tokens of one sequence as attention reads them (factor pages through their factors)."""
+    return float(max(np.abs(orc.gather_kv(seq, layer, h)[1]).max() for h in range(orc.cfg.n_kv_heads)))
+
+
+def kernel_tolerances(ref_norm, vmax):
+    """Absolute tolerances (fp32 output, bf16 output) of the kernel gate for arbitrary shapes - one rule, from the
+    kernel's arithmetic: the stated fraction of ||out||_inf (4e-3 for the fp32 output, 1e-2 for the bf16 output), or
+    one bf16 unit (2^-9) of the largest value the query reads, whichever is larger.
+    Why the second term: the kernel rounds the softmax numerators p to bf16 before the tensor-core product with V, an
+    error of at most 2^-9 sum_t p_t |v_t| / l <= 2^-9 max|v| whatever the size of the result (the rounding of
+    w = A_v^T p adds a similar term).  Where attention averages over many tokens the errors average too and the
+    stated fraction of ||out||_inf holds with room (the fixed-shape and full-size tests assert exactly that); where a
+    query sees a handful of tokens whose values nearly cancel, ||out||_inf can be a few percent of max|v| and no
+    fraction of it bounds a rounding error that is relative to max|v|.  (A split rule - the stated tolerance
+    wherever ||out||_inf >= max|v| / 4, the arithmetic bound below - was tried first and failed on a committed seed
+    at ||out||_inf = 0.30 max|v| with an error of 0.67 x 2^-9 max|v|: the switch point has no basis in the
+    arithmetic, the maximum of the two bounds has.)  The bf16 output adds its own rounding, 2^-9 ||out||_inf."""
+    unit = 2.0 ** -9 * vmax
+    return max(4e-3 * ref_norm, unit), max(1e-2 * ref_norm, unit + 2.0 ** -8 * ref_norm)
+
+
+def assert_kernel_gate_any_shape(g, what=None):
+    for i in range(len(g["norm"])):
+        tol32, tol16 = kernel_tolerances(g["norm"][i], g["vmax"][i])
+        assert g["abs32"][i] <= tol32, ("kernel gate (fp32 out)", what, i, g["abs32"][i], tol32, g["norm"][i], g["vmax"][i])
+        assert g["abs16"][i] <= tol16, ("kernel gate (bf16 out)", what, i, g["abs16"][i], tol16, g["norm"][i], g["vmax"][i])
 
 
 def gen_kv(seed, layer, seq, n_tokens, cfg, outlier_prob=0.0):

@@ -4,20 +4,29 @@ so it checks sampled (sequence, layer, KV head) slices: heads are independent, s
 query heads of one KV head needs only that head's pages.
 
   kernel gate      the oracle attends over the slice's pages exactly as stored on the GPU (bf16 factors
-                   and dense rows read back): max-abs <= 1e-2 * ||out||_inf
-  factor gate      every factor page of the slice: ||X - A B||_F <= 1.01 * tail + 1e-3 * ||X||_F, tail
-                   from the oracle's fp64 SVD of the regenerated page
+                   and dense rows read back): max-abs <= 1e-2 * ||out||_inf.  Every sequence of the batch x
+                   at least three (layer, KV head) samples per workload.
+  factor gate      every factor page of the sampled slices, at least 4096 page SVDs per workload:
+                   ||X - A B||_F <= 1.01 * tail + 1e-3 * ||X||_F, tail from the oracle's fp64 SVD of the
+                   regenerated page.  A page that misses this (tail small against ||X||, where bf16 storage of the
+                   factors alone costs more than the allowance) is judged against the error of the oracle's own
+                   optimal factors rounded to bf16 instead, and counted (pages_judged_by_storage_floor)
   end-to-end gate  oracle append + compress + attend on the regenerated slice (fp64 factors):
-                   <= 1e-2 + 3 x (the oracle's own bf16-storage error)
+                   <= 1e-2 + 2 x (the oracle's own bf16-storage error, itself capped at 10 %)
+
+The measured figures of every workload are appended, as one JSON object per line, to the file named by the
+environment variable PKV_PARITY_RESULTS when it is set (tests/results/parity_fullsize.jsonl is such a run).
 """
 import copy
+import json
+import os
 
 import numpy as np
 import pytest
 import torch
 
 import bench
-from gpu_helpers import f64, rel_err
+from gpu_helpers import E2E_FLOOR_CAP, E2E_FLOOR_FACTOR, f64, rel_err
 from oracle import attention as oatt
 from oracle import svd as osvd
 from oracle.cache import FACTOR, OracleCache, OracleConfig
@@ -25,6 +34,14 @@ from paper_2608_23843_b200 import pkv, synth
 
 pytestmark = pytest.mark.gpu
 ATT_TOL = 1e-2
+MIN_PAGE_SVDS = 4096
+
+
+def record(workload, **figures):
+    path = os.environ.get("PKV_PARITY_RESULTS")
+    if path:
+        with open(path, "a") as f:
+            f.write(json.dumps(dict(workload=workload, **figures)) + "\n")
 
 
 def stored_kv(cache, seq, layer, head):
@@ -76,30 +93,66 @@ def oracle_slice(w, rank, seq, layer, head, T, device, steps_kv=None):
     return orc, k, v
 
 
-def factor_and_e2e_gates(cache, w, rank, seq, layer, head, T, q_row, out_row, device):
-    """q_row/out_row: [G, d] of this KV head's query heads."""
-    orc, k, v = oracle_slice(w, rank, seq, layer, head, T, device)
+def factor_gate(cache, w, rank, seq, layer, head, T, device, orc=None, k=None, v=None):
+    """Every factor page (K and V) of one slice against the oracle's singular values.  Returns the oracle slice,
+    the number of page SVDs checked and the worst err / bound."""
+    if orc is None:
+        orc, k, v = oracle_slice(w, rank, seq, layer, head, T, device)
     _, _, gpu_factors = stored_kv(cache, seq, layer, head)
     okinds, oslots, _ = orc.page_table(0, 0)
     assert sorted(gpu_factors) == [p for p, kd in enumerate(okinds) if kd == FACTOR]
-    worst = 0.0
+    from oracle.bf16 import round_to_bf16
+    worst, n, n_floor = 0.0, 0, 0
     P, rank_v = w.get("page", 64), w.get("rank_v", rank)
     for p, (A_k, B_k, A_v, B_v) in gpu_factors.items():
         sig_k, sig_v = orc.sigma[oslots[p]]
-        for X, A, B, sig, r in ((k[p * P:(p + 1) * P, 0], A_k, B_k, sig_k[0], rank), (v[p * P:(p + 1) * P, 0], A_v, B_v, sig_v[0], rank_v)):
+        opt = orc.factor[oslots[p]]
+        for X, A, B, sig, r, oa, ob in ((k[p * P:(p + 1) * P, 0], A_k, B_k, sig_k[0], rank, opt["A_k"][0], opt["B_k"][0]),
+                                        (v[p * P:(p + 1) * P, 0], A_v, B_v, sig_v[0], rank_v, opt["A_v"][0], opt["B_v"][0])):
             err = np.linalg.norm(X - A @ B)
             bound = 1.01 * float(np.sqrt((sig[r:] ** 2).sum())) + 1e-3 * np.linalg.norm(X)
+            if err > bound:
+                # Pages whose tail is small against ||X|| (a x10 outlier row at a high rank): storing the factors in
+                # bf16 alone costs about 2.3e-3 ||X||, in quadrature with the tail, for any implementation.  The
+                # yardstick is then what the oracle's own optimal factors give once rounded to the storage type.
+                n_floor += 1
+                bound = 1.01 * float(np.linalg.norm(X - round_to_bf16(oa) @ round_to_bf16(ob))) + 1e-3 * np.linalg.norm(X)
             assert err <= bound, (seq, layer, head, p, err, bound)
             worst = max(worst, err / bound)
             assert np.abs(A.T @ A - np.eye(r)).max() <= 1e-2
+            n += 1
+    return orc, n, worst, n_floor
+
+
+def e2e_gate(orc, q_row, out_row, what):
+    """q_row / out_row: [G, d] of the slice's query heads.  Returns (e2e, floor)."""
     qd = f64(q_row)[None]
     ref = orc.decode_attention(0, [0], qd)[0]
     rounded = copy.deepcopy(orc)
     rounded.round_factors_to_storage_type()
     floor = rel_err(rounded.decode_attention(0, [0], qd)[0], ref)
     e2e = rel_err(f64(out_row), ref)
-    assert e2e <= ATT_TOL + 3.0 * floor, (seq, layer, head, e2e, floor)
-    return worst, e2e, floor
+    assert floor <= E2E_FLOOR_CAP, (what, floor)
+    assert e2e <= ATT_TOL + E2E_FLOOR_FACTOR * floor, (what, e2e, floor)
+    return e2e, floor
+
+
+def check_slices(cache, w, rank, slices, lengths, qs, outs, device, n_e2e=1):
+    """Factor gate over the listed (sequence, layer, KV head) slices and the end-to-end gate over the first n_e2e of
+    them.  Returns dict(page_svds, factor_worst, e2e=[...], floor=[...])."""
+    G = w["n_q_heads"] // w["n_kv_heads"]
+    res = dict(page_svds=0, pages_judged_by_storage_floor=0, factor_worst=0.0, e2e=[], floor=[])
+    for i, (seq, layer, head) in enumerate(slices):
+        orc, n, worst, n_floor = factor_gate(cache, w, rank, seq, layer, head, lengths[seq], device)
+        res["page_svds"] += n
+        res["pages_judged_by_storage_floor"] += n_floor
+        res["factor_worst"] = max(res["factor_worst"], worst)
+        if i < n_e2e:
+            e2e, floor = e2e_gate(orc, qs[layer][seq, head * G:(head + 1) * G], outs[layer][seq, head * G:(head + 1) * G],
+                                  (seq, layer, head))
+            res["e2e"].append(e2e)
+            res["floor"].append(floor)
+    return res
 
 
 def _decode_all(cache, w, ids, device):
@@ -118,40 +171,41 @@ def _finish(cache):
 
 
 def test_llama3_8b_layer_batch8_context_32k():
-    """BASELINE config 1: 32q/8kv, batch 8, T=32768, r=24, 64 sink + 256 recent, shuffled pools."""
+    """Llama-3-8B-shaped layer: 32q/8kv, batch 8, T=32768, r=24, 64 sink + 256 recent, shuffled pools."""
     w, device = bench.WORKLOADS["llama3_8b_32k_b8"], torch.device("cuda", 0)
     cfg, cache, lengths, comp = bench.build_workload(w, w["rank"], device)
     assert comp["n_page_svds"] == 64896 * w["n_layers"]
     ids = list(range(w["batch"]))
     assert cache.page_table(3, 0)[0] == [0] + [1] * 507 + [0] * 4
     qs, outs = _decode_all(cache, w, ids, device)
-    G = 4
-    worst = kernel_gate(cache, cfg, 0, ids, qs[0], outs[0], [(0, 0), (5, 7), (7, 3)])
-    fw, e2e, floor = factor_and_e2e_gates(cache, w, w["rank"], 5, 0, 7, lengths[5], qs[0][5, 7 * G:8 * G], outs[0][5, 7 * G:8 * G], device)
+    # kernel gate: every sequence x three KV heads of one layer, and one more layer for two sequences
+    worst = kernel_gate(cache, cfg, 0, ids, qs[0], outs[0], [(i, h) for i in ids for h in (0, 3, 7)])
+    worst = max(worst, kernel_gate(cache, cfg, 2, ids, qs[2], outs[2], [(1, 5), (6, 2)]))
+    res = check_slices(cache, w, w["rank"], [(5, 0, 7), (0, 0, 0), (7, 0, 3), (2, 2, 5), (4, 1, 1)], lengths, qs, outs, device, n_e2e=2)
+    assert res["page_svds"] >= MIN_PAGE_SVDS
     again = torch.empty_like(outs[0])
     cache.decode_attention(0, ids, qs[0], again)
     torch.cuda.synchronize()
     assert torch.equal(again, outs[0])
-    print("config 1: kernel gate %.2e, factor err/bound %.3f, e2e %.2e (floor %.2e)" % (worst, fw, e2e, floor))
+    record("llama3_8b_32k_b8", kernel_gate_worst=worst, kernel_gate_slices=26, **res)
     _finish(cache)
 
 
 def test_qwen3_32b_64_layers_context_128k():
-    """BASELINE config 2: 64 layers, 64q/8kv, batch 1, T=131072, r=24, 64 sink + 512 recent."""
+    """Qwen3-32B-shaped long context: 64 layers, 64q/8kv, batch 1, T=131072, r=24, 64 sink + 512 recent."""
     w, device = bench.WORKLOADS["qwen3_32b_128k"], torch.device("cuda", 0)
     cfg, cache, lengths, comp = bench.build_workload(w, w["rank"], device)
     assert comp["n_page_svds"] == 2087936
     kinds = cache.page_table(0, 63)[0]
     assert kinds == [0] + [1] * 2039 + [0] * 8
     qs, outs = _decode_all(cache, w, [0], device)
-    G = 8
     worst = 0.0
-    for layer, head in ((0, 0), (31, 5), (63, 7)):
+    samples = ((0, 0), (31, 5), (63, 7), (17, 2))
+    for layer, head in samples:
         worst = max(worst, kernel_gate(cache, cfg, layer, [0], qs[layer], outs[layer], [(0, head)]))
-    fw, e2e, floor = factor_and_e2e_gates(cache, w, w["rank"], 0, 31, 5, lengths[0], qs[31][0, 5 * G:6 * G],
-                                          outs[31][0, 5 * G:6 * G], device)
-    print("config 2: kernel gate %.2e, factor err/bound %.3f, e2e %.2e (floor %.2e), %.0f page SVDs/s"
-          % (worst, fw, e2e, floor, comp["pages_per_s"]))
+    res = check_slices(cache, w, w["rank"], [(0, 31, 5), (0, 63, 7)], lengths, qs, outs, device, n_e2e=2)
+    assert res["page_svds"] >= MIN_PAGE_SVDS
+    record("qwen3_32b_128k", kernel_gate_worst=worst, kernel_gate_slices=len(samples), pages_per_s=comp["pages_per_s"], **res)
     _finish(cache)
 
 
@@ -164,39 +218,48 @@ def test_paper_default_shape_qwen3_8b_16k():
     sz = cache.sizes
     assert sz.factor_slot_bytes / sz.dense_slot_bytes == 0.5859375             # Eq. 3 at (16,14), P=32, d=128
     qs, outs = _decode_all(cache, w, [0], device)
-    G = 4
     worst = 0.0
-    for layer, head in ((0, 0), (17, 3), (35, 7)):
+    samples = ((0, 0), (17, 3), (35, 7), (8, 5))
+    for layer, head in samples:
         worst = max(worst, kernel_gate(cache, cfg, layer, [0], qs[layer], outs[layer], [(0, head)]))
-    fw, e2e, floor = factor_and_e2e_gates(cache, w, w["rank"], 0, 17, 3, lengths[0], qs[17][0, 3 * G:4 * G],
-                                          outs[17][0, 3 * G:4 * G], device)
-    print("paper default: kernel gate %.2e, factor err/bound %.3f, e2e %.2e (floor %.2e), %.0f page SVDs/s"
-          % (worst, fw, e2e, floor, comp["pages_per_s"]))
+    res = check_slices(cache, w, w["rank"], [(0, 17, 3), (0, 0, 0), (0, 35, 7), (0, 8, 5), (0, 26, 1)], lengths, qs, outs,
+                       device, n_e2e=2)
+    assert res["page_svds"] >= MIN_PAGE_SVDS
+    record("qwen3_8b_16k_paper_default", kernel_gate_worst=worst, kernel_gate_slices=len(samples),
+           pages_per_s=comp["pages_per_s"], **res)
     _finish(cache)
 
 
 @pytest.mark.parametrize("rank", [8, 16, 24, 32])
 def test_ragged_serving_batch_rank_sweep(rank):
-    """BASELINE config 4: 64 requests, lengths log-uniform in [2048, 65536], 2% outlier key tokens (x10)."""
+    """Ragged serving batch: 64 requests, lengths log-uniform in [2048, 65536], 2% outlier key tokens (x10)."""
     w, device = bench.WORKLOADS["ragged_b64"], torch.device("cuda", 0)
     cfg, cache, lengths, comp = bench.build_workload(w, rank, device)
     ids = list(range(w["batch"]))
     qs, outs = _decode_all(cache, w, ids, device)
-    short, long_ = int(np.argmin(lengths)), int(np.argmax(lengths))
-    worst = kernel_gate(cache, cfg, 0, ids, qs[0], outs[0], [(short, 1), (long_, 6), (17, 0)])
-    G = 4
-    fw, e2e, floor = factor_and_e2e_gates(cache, w, rank, short, 0, 1, lengths[short], qs[0][short, G:2 * G],
-                                          outs[0][short, G:2 * G], device)
+    # kernel gate: every sequence, three KV heads in rotation
+    worst = kernel_gate(cache, cfg, 0, ids, qs[0], outs[0], [(i, (i + j) % 8) for i in ids for j in (0, 3, 6)])
+    # factor and end-to-end gates: the shortest and the longest sequence, then further long ones until enough pages
+    by_len = sorted(ids, key=lambda i: lengths[i])
+    slices, n = [(by_len[0], 0, 1), (by_len[-1], 0, 6)], 0
+    for rank_pos, i in enumerate(reversed(by_len[:-1])):
+        if sum(2 * max(0, lengths[s] // 64 - 5) for s, _, _ in slices) >= MIN_PAGE_SVDS:
+            break
+        slices.append((i, 0, rank_pos % 8))
+    res = check_slices(cache, w, rank, slices, lengths, qs, outs, device, n_e2e=2)
+    assert res["page_svds"] >= MIN_PAGE_SVDS
     assert any(t % 64 for t in lengths)                     # partial last pages are present
-    print("config 4 r=%d: kernel gate %.2e, factor err/bound %.3f, e2e %.2e (floor %.2e)" % (rank, worst, fw, e2e, floor))
+    record("ragged_b64", rank=rank, kernel_gate_worst=worst, kernel_gate_slices=3 * len(ids), **res)
     _finish(cache)
 
 
 def test_incremental_compression_during_decoding():
-    """BASELINE config 3: batch 32, prompts of 8192 tokens prefilled and compressed, then 512 steps of
-    append -> attend -> compress; a page per (sequence, KV head, K|V) leaves the 256-token window every
-    64 steps.  Page tables are checked bit-exact against the oracle's state machine at every step; the
-    kernel gate runs at sampled steps; one slice is followed end to end by a single-head oracle."""
+    """Incremental compression during decoding: batch 32, prompts of 8192 tokens prefilled and compressed, then
+    512 steps of append -> attend -> compress; a page per (sequence, KV head, K|V) leaves the 256-token window
+    every 64 steps.  Page tables are checked bit-exact against the oracle's state machine at every step; the
+    kernel gate runs at sampled steps over every sequence; one slice is followed end to end by a single-head
+    oracle; at the end the factor gate covers sixteen slices (pages factorized at the prefill and during the
+    steps alike)."""
     device = torch.device("cuda", 0)
     H, Hq, B, T0, steps, rank = 8, 32, 32, 8192, 512, 24
     n_pages = (T0 + steps) // 64 + 1
@@ -226,6 +289,7 @@ def test_incremental_compression_during_decoding():
     orc.compress_eligible_pages(0)
     z1 = np.zeros((B, 1, 128))
     n_events = 0
+    worst, e2es, floors = 0.0, [], []
     for t in range(steps):
         knew = torch.cat([k[T0 + t:T0 + t + 1] for k, _ in kv])
         vnew = torch.cat([v[T0 + t:T0 + t + 1] for _, v in kv])
@@ -236,14 +300,10 @@ def test_incremental_compression_during_decoding():
             q = synth.make_q(3, 0, t, B, Hq, 128, device)
             out = cache.decode_attention(0, ids, q)
             torch.cuda.synchronize()
-            kernel_gate(cache, cfg, 0, ids, q, out, [(seq_s, head_s), (0, 7)])
-            qd = f64(q[seq_s, head_s * G:(head_s + 1) * G])[None]
-            ref = orc.decode_attention(0, [0], qd)[0]
-            rounded = copy.deepcopy(orc)
-            rounded.round_factors_to_storage_type()
-            floor = rel_err(rounded.decode_attention(0, [0], qd)[0], ref)
-            e2e = rel_err(f64(out[seq_s, head_s * G:(head_s + 1) * G]), ref)
-            assert e2e <= ATT_TOL + 3.0 * floor, (t, e2e, floor)
+            worst = max(worst, kernel_gate(cache, cfg, 0, ids, q, out, [(seq_s, head_s)] + [(i, (i + t) % H) for i in ids]))
+            e2e, floor = e2e_gate(orc, q[seq_s, head_s * G:(head_s + 1) * G], out[seq_s, head_s * G:(head_s + 1) * G], t)
+            e2es.append(e2e)
+            floors.append(floor)
         n = cache.compress_eligible_pages(0)
         assert n == mirror.compress_eligible_pages(0) == (B if (T0 + t + 1) % 64 == 0 else 0)
         orc.compress_eligible_pages(0)
@@ -252,4 +312,21 @@ def test_incremental_compression_during_decoding():
     for s in (0, seq_s, B - 1):
         assert cache.page_table(s, 0) == mirror.page_table(s, 0)
     assert cache.page_table(seq_s, 0)[0] == orc.page_table(0, 0)[0]
+    # factor gate: the slice followed step by step, then fifteen more (their oracle factorizes the final context in
+    # one go: every page is factorized once, from the same rows, whenever that happens)
+    wl = dict(n_kv_heads=H, n_q_heads=Hq, sink=64, recent=256)
+    _, n_svds, fworst, n_floor = factor_gate(cache, wl, rank, seq_s, 0, head_s, T0 + steps, device, orc=orc, k=ks, v=vs)
+    for i in range(15):
+        s, h = (2 * i + 1) % B, i % H
+        kk, vv = f64(kv[s][0][:, h:h + 1]), f64(kv[s][1][:, h:h + 1])
+        o2 = OracleCache(OracleConfig(n_layers=1, n_kv_heads=1, n_q_heads=G, head_dim=128, page_size=64, rank_k=rank,
+                                      rank_v=rank, sink_tokens=64, recent_tokens=256, max_seqs=1, n_dense_slots=n_pages,
+                                      n_factor_slots=n_pages))
+        o2.append_kv(0, [0], [T0 + steps], kk, vv)
+        o2.compress_eligible_pages(0)
+        _, n, fw, nf = factor_gate(cache, wl, rank, s, 0, h, T0 + steps, device, orc=o2, k=kk, v=vv)
+        n_svds, fworst, n_floor = n_svds + n, max(fworst, fw), n_floor + nf
+    assert n_svds >= MIN_PAGE_SVDS
+    record("serving_b32_8k (512 steps)", kernel_gate_worst=worst, kernel_gate_slices=4 * (B + 1), page_svds=n_svds,
+           pages_judged_by_storage_floor=n_floor, factor_worst=fworst, e2e=e2es, floor=floors, steps_checked=[1, 64, 65, 512])
     _finish(cache)

@@ -8,15 +8,17 @@ stored bf16 factors, so both sides read identical inputs; the 1e-2 tolerance
 applies as stated.  End-to-end gate: the oracle uses its own unrounded fp64
 factors; storing factors in bf16 perturbs scores by ~0.2% of their magnitude
 for ANY implementation, which on these inputs (scores up to +-80) moves outputs
-by 1-7% on its own, so the bound is 1e-2 plus 3x that storage-noise floor (the
+by 1-7% on its own, so the bound is 1e-2 plus 2x that storage-noise floor (the
 GPU's rounding is an independent draw of the same noise, and near the rank cut
 fp32 and fp64 may keep different, equally good directions), the floor being
-measured inside the oracle (fp64 factors rounded to bf16 vs unrounded)."""
+measured inside the oracle (fp64 factors rounded to bf16 vs unrounded) and
+itself capped at 10 % (see gpu_helpers.assert_attention_gates)."""
 import numpy as np
 import pytest
 import torch
 
-from gpu_helpers import Pair, assert_attention_gates, attention_gates, f64, gen_kv, rel_err
+from gpu_helpers import (E2E_FLOOR_FACTOR, Pair, assert_attention_gates, attention_gates, entry_vmax, f64, gen_kv, kernel_tolerances,
+                         rel_err)
 from oracle import svd
 from oracle.cache import FACTOR
 from paper_2608_23843_b200 import pkv, synth
@@ -24,6 +26,14 @@ from paper_2608_23843_b200 import pkv, synth
 pytestmark = pytest.mark.gpu
 
 ATT_TOL = 1e-2
+
+
+def stored_optimum_error(X, r):
+    """||X - bf16(A) bf16(B)||_F for the oracle's optimal rank-r factors of X: what the best factorization costs once
+    its factors are stored in bf16 (equal to the Eckart-Young tail where the tail dominates the rounding)."""
+    from oracle.bf16 import round_to_bf16
+    A, B, _ = svd.page_factors(X[None], r)
+    return float(np.linalg.norm(X - round_to_bf16(A[0]) @ round_to_bf16(B[0])))
 
 
 def _check_reconstruction(pair, seq, layer, heads=None):
@@ -44,9 +54,10 @@ def _check_reconstruction(pair, seq, layer, heads=None):
                 tail = float(np.sqrt((sig[r:] ** 2).sum()))
                 bound = 1.01 * tail + 1e-3 * np.linalg.norm(X)
                 if r == cfg.page_size:
-                    # full rank: the optimal tail is zero and what is left is the bf16 rounding of the two
-                    # factors (about 0.0023 ||X|| rms), which the 1e-3 ||X|| allowance does not cover
-                    bound = 4e-3 * np.linalg.norm(X)
+                    # full rank: the optimal tail is zero and what is left is the bf16 rounding of the two factors,
+                    # which the 1e-3 ||X|| allowance does not cover for any implementation that stores bf16: the
+                    # oracle's own optimal factors, rounded to the storage type, take the tail's place
+                    bound = 1.01 * stored_optimum_error(X, r) + 1e-3 * np.linalg.norm(X)
                 assert err <= bound, (seq, p, h, name, err, bound)
                 worst = max(worst, err / bound)
                 assert np.abs(A.T @ A - np.eye(r)).max() <= 1e-2
@@ -338,7 +349,8 @@ def test_int4_factors(P, rk, rv, G):
     """INT4 factor storage (Section 4.3): the GPU quantizes in the compression kernel and dequantises in the
     decode kernel's registers.  Kernel gate: the oracle attends over the GPU's own dequantised factors (<= 1e-2).  Factor gate: the
     GPU's quantized reconstruction error is no worse than the oracle's INT4 error for the same page (x1.15).
-    End to end against the oracle's INT4 cache: 1e-2 + 3 x the error INT4 causes inside the oracle."""
+    End to end against the oracle's INT4 cache: 1e-2 + a tenth of the error INT4 itself causes inside the oracle
+    (20-26 % on these inputs): the two INT4 caches must agree ten times better than either agrees with bf16."""
     import copy
     from oracle import quant
     from oracle.cache import OracleCache
@@ -392,7 +404,7 @@ def test_int4_factors(P, rk, rv, G):
     for i in range(3):
         assert g["kernel"][i] <= 4e-3 and g["kernel_bf16"][i] <= ATT_TOL, (i, g["kernel"][i])
         floor4 = rel_err(ref4[i], ref16[i])
-        assert rel_err(got[i], ref4[i]) <= ATT_TOL + 3.0 * floor4, (i, rel_err(got[i], ref4[i]), floor4)
+        assert rel_err(got[i], ref4[i]) <= ATT_TOL + 0.1 * floor4, (i, rel_err(got[i], ref4[i]), floor4)
     with pytest.raises(pkv.PkvError) as e:
         pair.gpu.write_factors(slots[1], 0, *pair.gpu.read_factors(slots[1], 0))
     assert e.value.status == pkv.PKV_ERR_UNSUPPORTED
@@ -441,8 +453,10 @@ def test_prescribed_spectra_with_and_without_the_energy_rule(P, energy_tol):
         A_k, B_k, A_v, B_v = [f64(t) for t in pair.gpu.read_factors(slot, 0)]
         for A, B in ((A_k, B_k), (A_v, B_v)):
             err = np.linalg.norm(X[p] - A @ B)
-            # bf16 storage of A and B alone costs up to 2^-9 of ||X|| each, which dominates where the tail is tiny
-            assert err <= 1.01 * tail[p] + 4e-3 * np.linalg.norm(X[p]), (P, energy_tol, p, err, tail[p])
+            # where the tail is tiny (a gap of 3000 at the cut) the bf16 storage of A and B dominates: the yardstick
+            # is what the oracle's own optimal factors give once rounded to the storage type, if that is larger
+            best = max(tail[p], stored_optimum_error(X[p], r))
+            assert err <= 1.01 * best + 1e-3 * np.linalg.norm(X[p]), (P, energy_tol, p, err, tail[p], best)
             # columns of A orthonormal up to bf16 rounding
             assert np.abs(A.T @ A - np.eye(r)).max() <= 2e-2, (P, energy_tol, p)
 
@@ -549,7 +563,7 @@ def test_multi_query_attention(P, rk, rv, G, q_len, bits):
             assert rel_err(got[i, j], ref_kernel[i, j]) <= 1e-2, (i, j)
             if bits != 4:
                 floor = rel_err(ref_rounded[i, j], ref[i, j])
-                assert rel_err(got[i, j], ref[i, j]) <= 1e-2 + 3.0 * floor, (i, j, floor)
+                assert rel_err(got[i, j], ref[i, j]) <= 1e-2 + E2E_FLOOR_FACTOR * floor, (i, j, floor)   # (per single query the floor belongs to that query's few dominant tokens: no cap)
     # the call is reproducible; its last query is the single-query call (bit for bit where the same kernel serves both)
     single = torch.empty((n, H * G, 128), dtype=torch.bfloat16, device="cuda")
     pair.gpu.decode_attention(0, order, qd[:, q_len - 1].contiguous(), single)
@@ -596,12 +610,13 @@ def test_sequence_sharded_attention_states(bits):
     q = synth.make_q(6, 0, 0, 3, H * G, 128)
     qd = q.cuda()
     states = torch.empty((3, 3, H * G, 130), dtype=torch.float32, device="cuda")
-    ref_states = []
+    ref_states, shard_vmax = [], []
     for r, pair in enumerate(pairs):
         pair.gpu.decode_attention_partial(0, order, qd, states[r])
         for s in order:
             pair.load_gpu_factors_into_oracle(s, 0)
         ref_states.append(pair.orc.attention_state(0, order, f64(q)))
+        shard_vmax.append([entry_vmax(pair.orc, s, 0) for s in order])
     out = torch.empty_like(qd)
     out32 = torch.empty(qd.shape, dtype=torch.float32, device="cuda")
     pkv.pkv_merge_attention_states(states, 3, 3 * H * G, out, out32, torch.cuda.current_stream())
@@ -611,21 +626,29 @@ def test_sequence_sharded_attention_states(bits):
     got_states, got, got32 = f64(states), f64(out), f64(out32)
     assert torch.equal(only32, out32)
     worst = worst_lse = 0.0
-    tol32 = 1e-2 if bits == 4 else 8e-3                # tiny shards (1 and 5 tokens): nothing averages the bf16 rounding of p
+    # tolerances per query head from the rule for arbitrary shapes (some shards hold 1 and 5 tokens: nothing averages
+    # the bf16 rounding of p there); INT4 factors: 1e-2 for the fp32 output as in the other INT4 tests
     for i in range(3):
         for h in range(H * G):
             merged = att.merge_page_states([(m[i, h], l[i, h], o[i, h]) for m, l, o in ref_states])
-            scale = np.abs(merged).max()
+            scale = float(np.abs(merged).max())
+            tol32, tol16 = kernel_tolerances(scale, max(shard_vmax[r][i] for r in range(3)))
+            if bits == 4:
+                tol32 = max(tol32, 1e-2 * scale)
             worst = max(worst, np.abs(got32[i, h] - merged).max() / scale)
-            assert np.abs(got[i, h] - merged).max() <= 1.2e-2 * scale
+            assert np.abs(got32[i, h] - merged).max() <= tol32, (i, h)
+            assert np.abs(got[i, h] - merged).max() <= tol16, (i, h)
             for r in range(3):
                 m, l, o = ref_states[r]
                 st = got_states[r, i, h]
                 lse = st[128] * math.log(2.0) + math.log(st[129])
                 worst_lse = max(worst_lse, abs(lse - (m[i, h] + math.log(l[i, h]))))
                 ref_o = o[i, h] / l[i, h]
-                assert np.abs(st[:128] / st[129] - ref_o).max() <= tol32 * np.abs(ref_o).max(), (r, i, h)
-    assert worst <= tol32 and worst_lse <= 2e-2
+                t32, _ = kernel_tolerances(float(np.abs(ref_o).max()), shard_vmax[r][i])
+                if bits == 4:
+                    t32 = max(t32, 1e-2 * float(np.abs(ref_o).max()))
+                assert np.abs(st[:128] / st[129] - ref_o).max() <= t32, (r, i, h)
+    assert worst_lse <= 2e-2
     # a single shard merged with itself alone is the ordinary call, bit for bit
     single = torch.empty_like(qd)
     pairs[0].gpu.decode_attention(0, order, qd, single)
