@@ -98,6 +98,12 @@ struct pkv_cache {
     cudaEvent_t order_ev = nullptr;    // scratch event: orders a side stream behind the caller's main stream
     cudaEvent_t worklist_ev = nullptr; // recorded behind the last kernel that reads the device work list
     bool worklist_busy = false;
+    // Test hooks (environment, read once per cache): PKV_TEST_WAIT_CLOCKS shortens the decode kernel's bounded
+    // waits, PKV_TEST_DROP_UNIT makes the first decode launch leave one unit unarmed, so that a wait runs out.
+    long long wait_clocks = 2000000000LL;
+    int drop_unit = -1;
+    int64_t timeouts_seen = 0;         // device_timeouts at the last pkv_get_stats()
+    bool tickets_dirty = false;        // a launch gave up: merge tickets may be left non-zero
 
     SeqLayer &at(int seq, int layer) { return sl[(size_t)seq * cfg.n_layers + layer]; }
     const SeqLayer &at(int seq, int layer) const { return sl[(size_t)seq * cfg.n_layers + layer]; }
@@ -520,6 +526,8 @@ pkv_status pkv_init_cache(const pkv_config *cfg, void *dense_pool, void *factor_
     c->cfg = *cfg;
     c->dry = dry;
     { const char *t = getenv("PKV_DECODE_TRACE"); c->trace = t && t[0] == '1'; }
+    { const char *t = getenv("PKV_TEST_WAIT_CLOCKS"); if (t && atoll(t) > 0) c->wait_clocks = atoll(t); }
+    { const char *t = getenv("PKV_TEST_DROP_UNIT"); if (t && t[0]) c->drop_unit = atoi(t); }
     // default grid: one CTA per SM when consecutive launches overlap (two launches share each SM),
     // otherwise two CTAs per SM
     int n_ctas = cfg->n_ctas > 0 ? cfg->n_ctas : default_ctas(dry) * (cfg->decode_overlap ? 1 : 2);
@@ -943,6 +951,14 @@ static pkv_status decode_impl(pkv_cache *c, int32_t layer, int32_t n_seqs, const
     a.plan_cta_entry = c->ml.plan_cta_entry;
     a.q = q; a.out = out; a.out_f32 = out_f32;
     a.state = state;
+    a.wait_clocks = c->wait_clocks;
+    a.drop_unit = c->drop_unit;
+    c->drop_unit = -1;                                    // (one launch only)
+    if (c->tickets_dirty && !is_capturing(st)) {
+        // an earlier launch gave up on a wait and may have left merge tickets drawn: start from zero again
+        PKV_CUDA(c, cudaMemsetAsync(c->workspace + c->wl.tickets, 0, (size_t)(c->wl.tickets_stride * c->wl.n_sets), st));
+        c->tickets_dirty = false;
+    }
     a.q_len = q_len;
     a.q_tpt = queries_per_tile(c->geo, q_len);
     a.q_group = sibling_group(c->geo, q_len);
@@ -1089,6 +1105,7 @@ pkv_status pkv_get_stats(pkv_cache *c, pkv_stats *out, void *stream) {
         PKV_CUDA(c, cudaStreamSynchronize((cudaStream_t)stream));
         PKV_CUDA(c, cudaMemcpy(st, c->meta + c->ml.status, sizeof st, cudaMemcpyDeviceToHost));
         out->device_timeouts = st[0];
+        if (st[0] != c->timeouts_seen) { c->timeouts_seen = st[0]; c->tickets_dirty = true; }
         out->page_svds_not_converged = st[1];
         out->bad_slot_indices = st[2];
         uint64_t wide[2];

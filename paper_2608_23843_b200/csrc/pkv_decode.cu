@@ -269,12 +269,14 @@ __device__ __forceinline__ bool mbar_try_wait(uint32_t bar, uint32_t parity) {
         : "=r"(ok) : "r"(bar), "r"(parity) : "memory");
     return ok != 0;
 }
-// Bounded wait: gives up after ~2e9 clocks (about a second) and reports failure.
-__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity) {
+// Bounded wait: gives up after `limit` clocks (kWaitClocks, about a second, unless a test shortened it) and reports
+// failure.
+constexpr long long kWaitClocks = 2000000000LL;
+__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, long long limit = kWaitClocks) {
     if (mbar_try_wait(bar, parity)) return true;
     const long long t0 = clock64();
     while (!mbar_try_wait(bar, parity)) {
-        if (clock64() - t0 > 2000000000LL) return false;
+        if (clock64() - t0 > limit) return false;
     }
     return true;
 }
@@ -287,11 +289,11 @@ __device__ __forceinline__ void st_release_smem(volatile int *p, int v) {
     asm volatile("st.release.cta.shared.b32 [%0], %1;" ::"r"(smem_u32(const_cast<int *>(p))), "r"(v) : "memory");
 }
 // Bounded spin until the producer has armed unit k in its stage (the stage's tag then reads k + 1).
-__device__ __forceinline__ bool wait_armed(volatile int *tag, int k) {
+__device__ __forceinline__ bool wait_armed(volatile int *tag, int k, long long limit) {
     if (ld_acquire_smem(tag) == k + 1) return true;
     const long long t0 = clock64();
     while (ld_acquire_smem(tag) != k + 1) {
-        if (clock64() - t0 > 2000000000LL) return false;
+        if (clock64() - t0 > limit) return false;
         __nanosleep(20);
     }
     return true;
@@ -1052,7 +1054,9 @@ __global__ void __launch_bounds__(kDecodeThreads, 2) decode_tc_kernel(const __gr
                     bool pending = lane >= j0 && lane < min(j0 + S, n_here);
                     const long long t0 = clock64();
                     while (__any_sync(0xffffffffu, pending)) {
-                        if (pending && (kj < S || mbar_try_wait(smem_u32(empty_bar + s), ((kj / S) - 1) & 1))) {
+                        if (pending && a.drop_unit == kj && blockIdx.x == 0) {
+                            pending = false;             // test hook: this unit is never armed, so its consumer's wait runs out
+                        } else if (pending && (kj < S || mbar_try_wait(smem_u32(empty_bar + s), ((kj / S) - 1) & 1))) {
                             descs[s] = StageDesc{kind, rows, seg_local, after};
                             const uint32_t bar = smem_u32(full_bar + s);
                             const uint32_t dst = smem_u32(stages + (size_t)s * stage_bytes);
@@ -1076,7 +1080,7 @@ __global__ void __launch_bounds__(kDecodeThreads, 2) decode_tc_kernel(const __gr
                             if (trace && kj == 0) trace[3] = clock64();
                             pending = false;
                         }
-                        if (clock64() - t0 > 2000000000LL) break;          // about a second: give up
+                        if (clock64() - t0 > a.wait_clocks) break;         // about a second: give up
                     }
                     ok = !__any_sync(0xffffffffu, pending);
                 }
@@ -1091,7 +1095,7 @@ __global__ void __launch_bounds__(kDecodeThreads, 2) decode_tc_kernel(const __gr
         for (int w = 0; w < W && ok; ++w, ++k) {
             if (lane == 0) {
                 const int s = k % S;
-                if (k >= S && !mbar_wait(smem_u32(empty_bar + s), ((k / S) - 1) & 1)) ok = false;
+                if (k >= S && !mbar_wait(smem_u32(empty_bar + s), ((k / S) - 1) & 1, a.wait_clocks)) ok = false;
                 if (ok) {
                     descs[s] = StageDesc{kKindEnd, 0, rg.n_local_segs, 0};
                     mbar_arrive(smem_u32(full_bar + s));
@@ -1106,7 +1110,7 @@ __global__ void __launch_bounds__(kDecodeThreads, 2) decode_tc_kernel(const __gr
             // let copies already in flight land before the CTA retires
             for (int back = 1; back <= min(k, S); ++back) {
                 const int kk = k - back;
-                (void)mbar_wait(smem_u32(full_bar + kk % S), (kk / S) & 1);
+                (void)mbar_wait(smem_u32(full_bar + kk % S), (kk / S) & 1, a.wait_clocks);
             }
         }
     } else {
@@ -1137,7 +1141,8 @@ __global__ void __launch_bounds__(kDecodeThreads, 2) decode_tc_kernel(const __gr
         bool ok = true;
         for (int k = warp;; k += W) {
             const int s = k % S;
-            if (ok && (*abort_flag || !wait_armed(armed + s, k) || !mbar_wait(smem_u32(full_bar + s), (k / S) & 1))) {
+            if (ok && (*abort_flag || !wait_armed(armed + s, k, a.wait_clocks) ||
+                       !mbar_wait(smem_u32(full_bar + s), (k / S) & 1, a.wait_clocks))) {
                 ok = false;
                 if (lane == 0) { *abort_flag = 1; atomicAdd(a.status, 1); }
             }

@@ -119,6 +119,8 @@ struct DecodeArgs {
     int variant;                       // 0 = tensor-core pipeline, 1 = scalar reference kernel
     int overlap;                       // 0 wait at entry, 1 wait before the first partial state is written, 2 never wait
     int plain_launch;                  // launch without programmatic serialization (drains the stream first)
+    long long wait_clocks;             // limit of every in-kernel wait of the decode kernel (SM clocks)
+    int drop_unit;                     // -1; test hook: CTA 0's producer never arms this unit (a wait must run out)
     long long *trace;                  // NULL, or [n_ctas][kTraceSlots] time stamps written by each CTA (debugging)
 };
 

@@ -399,3 +399,34 @@ def test_cuda_graph_replay_of_multi_query_and_state_calls(q_len, max_seqs):
     assert torch.equal(out_1, ref_1)
     assert cache.stats()["device_timeouts"] == 0
     cache.close()
+
+
+@pytest.mark.parametrize("n_ctas", [1, 6])
+def test_a_bounded_wait_that_runs_out_is_reported_and_the_cache_stays_usable(monkeypatch, n_ctas):
+    """Every wait inside the decode kernel gives up after a fixed number of clocks.  Here one is made to: the
+    library's test hooks (read from the environment when the cache is created) shorten the limit to about a
+    millisecond and make the producer of CTA 0 leave one unit of the first launch unarmed, so the consumer warp that
+    waits for it finds nothing (nothing faults and nothing spins for ever: the wait ends by construction).  The call
+    must return, the timeout must be counted, and the next call on the same cache must be correct again - also when
+    the segment was split over several CTAs, whose merge tickets the aborted launch may have left drawn."""
+    monkeypatch.setenv("PKV_TEST_WAIT_CLOCKS", "2000000")
+    monkeypatch.setenv("PKV_TEST_DROP_UNIT", "3")
+    H, G, T = 1, 4, 1500
+    cfg = pkv.make_config(n_layers=1, n_kv_heads=H, n_q_heads=H * G, rank=16, sink_tokens=64, recent_tokens=128,
+                          max_seqs=1, max_pages_per_seq=32, n_dense_slots=32, n_factor_slots=32, n_ctas=n_ctas)
+    pair = Pair(cfg, seed=9)
+    monkeypatch.delenv("PKV_TEST_WAIT_CLOCKS")
+    monkeypatch.delenv("PKV_TEST_DROP_UNIT")
+    k, v = gen_kv(9, 0, 0, T, cfg)
+    pair.append(0, [0], [k], [v])
+    pair.compress(0)
+    q = synth.make_q(9, 0, 0, 1, H * G, 128)
+    pair.decode(0, [0], q)                                   # the launch with the unarmed unit: returns, result invalid
+    st = pair.gpu.stats()
+    assert st["device_timeouts"] >= 1
+    got, got32 = pair.decode(0, [0], q)                      # an ordinary launch on the same cache
+    assert pair.gpu.stats()["device_timeouts"] == st["device_timeouts"]
+    pair.load_gpu_factors_into_oracle(0, 0)
+    ref = pair.orc.decode_attention(0, [0], f64(q))
+    assert rel_err(got32, ref) <= 4e-3 and rel_err(got, ref) <= 1e-2
+    pair.gpu.close()
