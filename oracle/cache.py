@@ -25,6 +25,7 @@ import numpy as np
 
 from . import attention as _att
 from . import bf16 as _bf16
+from . import global_svd as _global
 from . import quant as _quant
 from . import svd as _svd
 
@@ -47,6 +48,8 @@ class OracleConfig:
     n_factor_slots: int
     softmax_scale: float = 0.0          # 0 => 1/sqrt(head_dim)  (Eq. 1)
     factor_bits: int = 16               # 4 => factors are INT4-quantized when a page is converted (Section 4.3)
+    global_rank: int = 0                # > 0 => the Global SVD form (Section 4.2): one basis per (sequence, layer, KV
+                                        # head), fixed by the pages of the first conversion; rank_k, rank_v unused
 
 
 class PoolExhausted(RuntimeError):
@@ -116,6 +119,7 @@ class OracleCache:
         self.state = {}      # (seq, layer) -> _SeqLayer
         self.pages_compressed = 0
         self.pending = {}    # layer -> [(seq, page, factor slot, factors, sigma)] begun, not committed
+        self.basis = {}      # Global SVD form: (seq, layer) -> dict(B_k [H,r,d], B_v [H,r,d], sigma_k, sigma_v, pages)
 
     # ------------------------------------------------------------------ append
     def _sl(self, seq, layer):
@@ -184,6 +188,8 @@ class OracleCache:
         """Rank-r factors (Eq. 2) of the listed (seq, layer, page) dense pages, every KV head: a list of
         (dict(A_k, B_k, A_v, B_v), (sigma_k, sigma_v)) in the order of `work`."""
         c = self.cfg
+        if c.global_rank > 0:
+            return self._factorize_global(work)
         Ks = np.stack([self.dense[self.state[(s, ly)].slots[p]][0] for s, ly, p in work])  # [n,H,P,d]
         Vs = np.stack([self.dense[self.state[(s, ly)].slots[p]][1] for s, ly, p in work])
         n, H = Ks.shape[0], c.n_kv_heads
@@ -198,6 +204,33 @@ class OracleCache:
                     f["A_k"][h], f["B_k"][h], f["A_v"][h], f["B_v"][h] = _quant.quantized_page_factors(
                         f["A_k"][h], f["B_k"][h], f["A_v"][h], f["B_v"][h])
             out.append((f, (s_k[sel].copy(), s_v[sel].copy())))
+        return out
+
+    def _factorize_global(self, work):
+        """Global SVD form.  The pages of the first conversion of a (sequence, layer) are its region: their rows,
+        stacked in page order, give the basis of every KV head (K and V separately); every page - of the region or
+        converted later - stores A = X_page B^T and shares B."""
+        c, r = self.cfg, self.cfg.global_rank
+        H = c.n_kv_heads
+        by_sl = {}
+        for s, ly, p in work:
+            by_sl.setdefault((s, ly), []).append(p)
+        for (s, ly), pages in by_sl.items():
+            if (s, ly) in self.basis:
+                continue
+            Kr = np.concatenate([self.dense[self.state[(s, ly)].slots[p]][0] for p in pages], axis=1)   # [H, T, d]
+            Vr = np.concatenate([self.dense[self.state[(s, ly)].slots[p]][1] for p in pages], axis=1)
+            fk = [_global.region_factors(Kr[h], r) for h in range(H)]
+            fv = [_global.region_factors(Vr[h], r) for h in range(H)]
+            self.basis[(s, ly)] = dict(B_k=np.stack([f[1] for f in fk]), B_v=np.stack([f[1] for f in fv]),
+                                       sigma_k=[f[2] for f in fk], sigma_v=[f[2] for f in fv], pages=list(pages))
+        out = []
+        for s, ly, p in work:
+            b = self.basis[(s, ly)]
+            Kp, Vp = self.dense[self.state[(s, ly)].slots[p]]
+            f = dict(A_k=np.stack([_global.project_page(Kp[h], b["B_k"][h]) for h in range(H)]), B_k=b["B_k"],
+                     A_v=np.stack([_global.project_page(Vp[h], b["B_v"][h]) for h in range(H)]), B_v=b["B_v"])
+            out.append((f, None))
         return out
 
     def _flip(self, seq, ly, p, fslot):
@@ -362,10 +395,13 @@ class OracleCache:
         type).  Attention afterwards reads the stored values, still in fp64."""
         for slot, f in self.factor.items():
             self.factor[slot] = {k: _bf16.round_to_bf16(v) for k, v in f.items()}
+        for b in self.basis.values():
+            b["B_k"], b["B_v"] = _bf16.round_to_bf16(b["B_k"]), _bf16.round_to_bf16(b["B_v"])
 
     def free_seq(self, seq):
         """Release every slot of a sequence, layers ascending, pages ascending."""
         for ly in range(self.cfg.n_layers):
+            self.basis.pop((seq, ly), None)
             sl = self.state.pop((seq, ly), None)
             if sl is None:
                 continue
