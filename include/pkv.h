@@ -135,6 +135,19 @@ typedef struct pkv_config {
                                    it, in every mode: the promise concerns other writers (of q, or of the pools
                                    through their raw pointers, which no mode allows while decode calls are in
                                    flight) only. */
+    int32_t global_rank;        /* 0: the paper's page-wise factors.  64, 80 or 96: the Global SVD form the paper
+                                   compares with (Section 4.1 "Baselines", Section 4.2), as a second workload of
+                                   the same decode kernel: each (sequence, layer, KV head) gets ONE basis B_k and
+                                   one B_v (global_rank x d, orthonormal rows: the leading right singular vectors
+                                   of the rows of all pages converted by the first compression of that sequence
+                                   and layer - its region), and every factor page stores only its token rows
+                                   A = X_page B^T (P x global_rank, for K and for V); pages converted later are
+                                   projected on the same basis.  Attention computes q~ = B_k q once per (sequence,
+                                   KV head) and CTA instead of once per page, streams only the A rows, keeps the
+                                   weighted sum in rank space and applies B_v once at the end.  rank_k and rank_v
+                                   are ignored (the paper's 76-78 rounds up to 80).  Needs page_size 32 or 64,
+                                   bf16 factors, decode_variant 0; pkv_decode_attention_multi,
+                                   pkv_compress_begin and pkv_write_factors return PKV_ERR_UNSUPPORTED. */
 } pkv_config;
 
 typedef struct pkv_sizes {
@@ -146,7 +159,8 @@ typedef struct pkv_sizes {
                                    rounded up to 16 */
     int64_t dense_pool_bytes;   /* n_dense_slots * dense_slot_bytes */
     int64_t factor_pool_bytes;
-    int64_t meta_bytes;         /* device page tables, token counts, decode plans, status words */
+    int64_t meta_bytes;         /* device page tables, token counts, decode plans, status words; with global_rank
+                                   also the bases: max_seqs * n_layers * H_kv * 2 * global_rank * d * 2 bytes */
     int64_t workspace_bytes;    /* split-K partial states, merge tickets, compression work list */
 } pkv_sizes;
 
@@ -426,6 +440,14 @@ pkv_status pkv_read_factors(pkv_cache *c, int64_t factor_slot, int32_t kv_head, 
 pkv_status pkv_write_factors(pkv_cache *c, int64_t factor_slot, int32_t kv_head, const void *A_k,
                              const void *B_k, const void *A_v, const void *B_v, void *stream);
 pkv_status pkv_read_dense(pkv_cache *c, int64_t dense_slot, int32_t kv_head, void *K, void *V,
+                          void *stream);
+/*
+ * Global SVD form only (global_rank > 0; Section 4.2): the shared basis of one (sequence, layer, KV head) as plain
+ * row-major bf16, B_k [global_rank, d] and B_v [global_rank, d] ([device], caller-owned).  In that form
+ * pkv_read_factors() returns A_k [P, global_rank] and A_v [P, global_rank] only (its B_k, B_v may be NULL), and a
+ * page's K^ is A_k B_k with this B_k.  PKV_ERR_INVALID_ARG if the sequence has no basis yet (nothing compressed).
+ */
+pkv_status pkv_read_basis(pkv_cache *c, int32_t seq, int32_t layer, int32_t kv_head, void *B_k, void *B_v,
                           void *stream);
 
 /*

@@ -35,6 +35,7 @@ struct SeqLayer {
     int32_t n_tokens = 0;
     int32_t f_end = 0;                 // pages [sink_pages, f_end) are factor pages
     uint64_t version = 0;              // bumped whenever the page list changes
+    bool has_basis = false;            // Global SVD form: the region's basis has been computed
     std::vector<int32_t> slots;
 };
 
@@ -138,8 +139,9 @@ pkv_status validate(const pkv_config *cfg, const char **why) {
         *why = "counts must be positive"; return PKV_ERR_INVALID_ARG;
     }
     if (cfg->n_q_heads % cfg->n_kv_heads) { *why = "n_q_heads must be a multiple of n_kv_heads"; return PKV_ERR_INVALID_ARG; }
-    if (cfg->page_size <= 0 || cfg->rank_k <= 0 || cfg->rank_v <= 0 || cfg->rank_k > cfg->page_size ||
-        cfg->rank_v > cfg->page_size || cfg->page_size > cfg->head_dim) {
+    if (cfg->global_rank <= 0 &&
+        (cfg->page_size <= 0 || cfg->rank_k <= 0 || cfg->rank_v <= 0 || cfg->rank_k > cfg->page_size ||
+         cfg->rank_v > cfg->page_size || cfg->page_size > cfg->head_dim)) {
         *why = "need 0 < rank <= page_size <= head_dim"; return PKV_ERR_INVALID_ARG;
     }
     if (cfg->sink_tokens < 0 || cfg->recent_tokens < 0 || cfg->sink_tokens % cfg->page_size ||
@@ -154,6 +156,17 @@ pkv_status validate(const pkv_config *cfg, const char **why) {
     }
     if (cfg->n_dense_slots > INT32_MAX || cfg->n_factor_slots > INT32_MAX) {
         *why = "slot counts must fit in int32"; return PKV_ERR_INVALID_ARG;
+    }
+    if (cfg->global_rank < 0) { *why = "global_rank is negative"; return PKV_ERR_INVALID_ARG; }
+    if (cfg->global_rank > 0) {
+        if (cfg->head_dim != kHeadDim) { *why = "only head_dim = 128 is supported"; return PKV_ERR_UNSUPPORTED; }
+        if ((cfg->global_rank != 64 && cfg->global_rank != 80 && cfg->global_rank != 96) ||
+            (cfg->page_size != 32 && cfg->page_size != 64) || cfg->factor_bits == 4 || cfg->decode_variant == 1) {
+            *why = "the Global SVD form needs global_rank 64, 80 or 96, page_size 32 or 64, bf16 factors, decode_variant 0 or 2";
+            return PKV_ERR_UNSUPPORTED;
+        }
+        if (cfg->n_q_heads / cfg->n_kv_heads > kMaxGroup) { *why = "only n_q_heads/n_kv_heads <= 8 is supported"; return PKV_ERR_UNSUPPORTED; }
+        return PKV_OK;
     }
     if (cfg->head_dim != kHeadDim) { *why = "only head_dim = 128 is supported"; return PKV_ERR_UNSUPPORTED; }
     if (cfg->page_size != 16 && cfg->page_size != 32 && cfg->page_size != 64) {
@@ -173,16 +186,19 @@ void derive(const pkv_config &cfg, int n_ctas, Geometry &g, MetaLayout &ml, Work
     g.n_layers = cfg.n_layers; g.n_kv_heads = cfg.n_kv_heads; g.n_q_heads = cfg.n_q_heads;
     g.group = cfg.n_q_heads / cfg.n_kv_heads;
     g.page = P;
-    g.rank_k = cfg.rank_k; g.rank_v = cfg.rank_v;
-    g.rank_tiles = (cfg.rank_k + 7) / 8;
+    g.global_rank = cfg.global_rank;
+    g.rank_k = cfg.global_rank > 0 ? cfg.global_rank : cfg.rank_k;
+    g.rank_v = cfg.global_rank > 0 ? cfg.global_rank : cfg.rank_v;
+    g.rank_tiles = (g.rank_k + 7) / 8;
+    g.basis_head_bytes = 2 * cfg.global_rank * kRowBytes;
     g.max_seqs = cfg.max_seqs; g.max_pages = cfg.max_pages_per_seq;
     g.n_dense_slots = (int)cfg.n_dense_slots; g.n_factor_slots = (int)cfg.n_factor_slots;
     g.sink_pages = cfg.sink_tokens / P; g.recent_pages = cfg.recent_tokens / P;
     g.ak_off = 0;
-    g.bk_off = g.ak_off + P * cfg.rank_k * 2;
-    g.av_off = g.bk_off + cfg.rank_k * d * 2;
-    g.bv_off = g.av_off + P * cfg.rank_v * 2;
-    g.blob16_bytes = g.bv_off + cfg.rank_v * d * 2;
+    g.bk_off = g.ak_off + P * g.rank_k * 2;
+    g.av_off = g.bk_off + (cfg.global_rank > 0 ? 0 : g.rank_k * d * 2);
+    g.bv_off = g.av_off + P * g.rank_v * 2;
+    g.blob16_bytes = g.bv_off + (cfg.global_rank > 0 ? 0 : g.rank_v * d * 2);
     g.factor_bits = cfg.factor_bits == 4 ? 4 : 16;
     g.cak_off = 0;
     g.cbk_off = g.cak_off + 4 * int4_a_words(P, g.rank_tiles);
@@ -190,7 +206,7 @@ void derive(const pkv_config &cfg, int n_ctas, Geometry &g, MetaLayout &ml, Work
     g.cbv_off = g.cav_off + 4 * int4_b_words(P, g.rank_tiles);
     g.codes_bytes = g.cbv_off + 4 * int4_a_words(d, g.rank_tiles);
     g.sak_off = 0;
-    g.sbk_off = g.sak_off + 2 * (int)align_up(cfg.rank_k, 8);
+    g.sbk_off = g.sak_off + 2 * (int)align_up(g.rank_k, 8);
     g.sav_off = g.sbk_off + 2 * d;
     g.sbv_off = g.sav_off + 2 * P;
     const int scales_bytes = g.sbv_off + 2 * d;
@@ -202,8 +218,9 @@ void derive(const pkv_config &cfg, int n_ctas, Geometry &g, MetaLayout &ml, Work
     // the rows that 8-row tile loads read past the last matrix when rank_v is not a multiple of 8.
     g.block_tokens = (g.factor_bits != 4 && P >= 32 && g.rank_tiles >= 3) ? 32 : 16;
     g.blocks_per_page = P / g.block_tokens;
-    const int overread = (8 * g.rank_tiles - cfg.rank_v) * kRowBytes;
-    const int factor_stage = g.factor_bits == 4 ? g.blob_bytes : (int)align_up(g.blob16_bytes + overread, 16);
+    const int overread = (8 * g.rank_tiles - g.rank_v) * kRowBytes;
+    int factor_stage = g.factor_bits == 4 ? g.blob_bytes : (int)align_up(g.blob16_bytes + overread, 16);
+    if (cfg.global_rank > 0) factor_stage = std::max(g.blob16_bytes, cfg.global_rank * kRowBytes);   // a page's rows, or one basis matrix
     g.stage_bytes = (int)align_up(std::max(factor_stage, g.block_tokens * 2 * kRowBytes), 128);
     // two CTAs are resident per SM (consecutive launches overlap, or the grid holds two CTAs per SM),
     // so that one streams while the other is in its prologue or merging
@@ -228,6 +245,7 @@ void derive(const pkv_config &cfg, int n_ctas, Geometry &g, MetaLayout &ml, Work
     ml.plans = off;      off = align_up(off + p * cfg.n_layers, 256);
     ml.append_desc = off; off = align_up(off + (long long)sizeof(AppendDesc) * cfg.max_seqs, 256);
     ml.status = off;     off = align_up(off + 4LL * kStatusWords, 256);
+    ml.basis = off;      off = align_up(off + (long long)cfg.max_seqs * cfg.n_layers * cfg.n_kv_heads * g.basis_head_bytes, 256);
     ml.total = off;
 
     wl.n_seg_tickets = (long long)cfg.max_seqs * cfg.n_kv_heads;
@@ -250,6 +268,7 @@ void derive(const pkv_config &cfg, int n_ctas, Geometry &g, MetaLayout &ml, Work
     wl.partials = w; w += wl.partials_stride * wl.n_sets;
     wl.worklist = w; w = align_up(w + (long long)sizeof(int2) * kCompressChunk, 256);
     wl.tickets = w;  w += wl.tickets_stride * wl.n_sets;
+    wl.gram = w;     w = align_up(w + (cfg.global_rank > 0 ? 4LL * cfg.n_kv_heads * 2 * d * d : 0), 256);
     wl.trace = w;    w = align_up(w + 8LL * kTraceSlots * n_ctas, 256);
     wl.total = w;
 }
@@ -678,6 +697,63 @@ static pkv_status run_worklist(pkv_cache *c, const std::vector<int2> &work, cuda
     return PKV_OK;
 }
 
+// Global SVD form (Section 4.2): per (sequence, layer) the eligible pages are converted together.  The first
+// conversion fixes the bases of the sequence's KV heads from exactly those pages (region Gram matrix, Jacobi
+// eigen-solve, leading eigenvectors); then, and at every later conversion, each page stores A = X_page B^T.  Same
+// page order, slot allocation and page-table updates as the page-wise path.
+static pkv_status compress_global(pkv_cache *c, int l0, int l1, int64_t *n_pages_compressed, cudaStream_t st) {
+    const Geometry &g = c->geo;
+    int64_t done = 0;
+    bool exhausted = false;
+    for (int seq = 0; seq < c->cfg.max_seqs && !exhausted; ++seq) {
+        for (int ly = l0; ly < l1 && !exhausted; ++ly) {
+            SeqLayer &s = c->at(seq, ly);
+            const int hi = std::max(g.sink_pages, s.n_tokens / c->cfg.page_size - g.recent_pages);
+            if (s.f_end >= hi) continue;
+            const int first = s.f_end;
+            std::vector<int2> work;
+            for (int p = s.f_end; p < hi && (int)work.size() < kCompressChunk; ++p) {
+                if (c->factor_free.available() == 0) { exhausted = true; break; }
+                const int32_t fs = c->factor_free.alloc(), ds = s.slots[p];
+                work.push_back(make_int2(ds, fs));
+                s.slots[p] = fs;
+                c->dense_free.release(ds);
+                s.f_end = p + 1;
+                ++done;
+            }
+            if (work.empty()) continue;
+            s.version++;
+            if (c->dry) { s.has_basis = true; continue; }
+            int2 *dwl = (int2 *)(c->workspace + c->wl.worklist);
+            if (c->worklist_busy) PKV_CUDA(c, cudaStreamWaitEvent(st, c->worklist_ev, 0));
+            pkv_status r = upload(c, dwl, work.data(), sizeof(int2) * work.size(), st);
+            if (r != PKV_OK) return r;
+            if ((r = stager_flush(c, st)) != PKV_OK) return r;
+            c->cache_written = true;
+            unsigned char *basis = c->meta + c->ml.basis +
+                                   ((long long)seq * c->cfg.n_layers + ly) * g.n_kv_heads * g.basis_head_bytes;
+            int *status = (int *)(c->meta + c->ml.status);
+            if (!s.has_basis) {
+                PKV_CUDA(c, launch_region_basis(g, c->dense_pool, dwl, (int)work.size(), (float *)(c->workspace + c->wl.gram),
+                                                basis, status, st));
+                s.has_basis = true;
+            }
+            PKV_CUDA(c, launch_project_pages(g, c->dense_pool, c->factor_pool, dwl, (int)work.size(), basis, status, st));
+            if (!c->worklist_ev) PKV_CUDA(c, cudaEventCreateWithFlags(&c->worklist_ev, cudaEventDisableTiming));
+            PKV_CUDA(c, cudaEventRecord(c->worklist_ev, st));
+            c->worklist_busy = true;
+            // the page-table rows of the converted pages, behind the kernels that read their dense slots
+            if ((r = upload(c, dev_page_table_row(c, seq, ly) + first, s.slots.data() + first,
+                            sizeof(int32_t) * (s.f_end - first), st)) != PKV_OK) return r;
+            if ((r = stager_flush(c, st)) != PKV_OK) return r;
+        }
+    }
+    c->pages_compressed += done;
+    if (n_pages_compressed) *n_pages_compressed = done;
+    if (exhausted) return fail(c, PKV_ERR_POOL_EXHAUSTED, "factor pool exhausted after %lld pages", (long long)done);
+    return PKV_OK;
+}
+
 pkv_status pkv_compress_eligible_pages(pkv_cache *c, int32_t layer, int64_t *n_pages_compressed,
                                        void *stream) {
     if (!c) return PKV_ERR_INVALID_ARG;
@@ -690,6 +766,7 @@ pkv_status pkv_compress_eligible_pages(pkv_cache *c, int32_t layer, int64_t *n_p
         return fail(c, PKV_ERR_UNSUPPORTED, "a compression begun with pkv_compress_begin is not committed yet");
     const Geometry &g = c->geo;
     const int l0 = layer < 0 ? 0 : layer, l1 = layer < 0 ? c->cfg.n_layers : layer + 1;
+    if (g.global_rank > 0) return compress_global(c, l0, l1, n_pages_compressed, st);
     std::vector<int2> work;
     int64_t done = 0;
     bool exhausted = false;
@@ -757,6 +834,7 @@ pkv_status pkv_compress_begin(pkv_cache *c, int32_t layer, void *main_stream, vo
     if (n_pages_begun) *n_pages_begun = 0;
     if (layer < 0 || layer >= c->cfg.n_layers) return fail(c, PKV_ERR_INVALID_ARG, "layer %d out of range", layer);
     PendingCompress &pd = c->pending[layer];
+    if (c->geo.global_rank > 0) return fail(c, PKV_ERR_UNSUPPORTED, "pkv_compress_begin is not available in the Global SVD form");
     if (pd.active) return fail(c, PKV_ERR_UNSUPPORTED, "layer %d already has an uncommitted compression", layer);
     if (!c->dry && (is_capturing(ms) || is_capturing(ss)))
         return fail(c, PKV_ERR_UNSUPPORTED, "pkv_compress_begin cannot be captured into a CUDA graph");
@@ -902,6 +980,8 @@ static pkv_status decode_impl(pkv_cache *c, int32_t layer, int32_t n_seqs, const
             return fail(c, PKV_ERR_INVALID_ARG, "sequence %d has no tokens in layer %d", seq_ids[i], layer);
     if (q_len < 1 || q_len > 32767) return fail(c, PKV_ERR_INVALID_ARG, "q_len %d out of range", q_len);
     if (q_len > 1) {
+        if (c->geo.global_rank > 0)
+            return fail(c, PKV_ERR_UNSUPPORTED, "several queries per sequence are not available in the Global SVD form");
         if (c->cfg.decode_variant == 1)
             return fail(c, PKV_ERR_UNSUPPORTED, "several queries per sequence need the tensor-core kernels (decode_variant 0)");
         if (!uses_row_blocks(c, q_len, n_seqs) && (long long)n_seqs * block_slots_per_seq(c->geo, q_len) > c->cfg.max_seqs)
@@ -937,6 +1017,7 @@ static pkv_status decode_impl(pkv_cache *c, int32_t layer, int32_t n_seqs, const
         int64_t rows = (int64_t)(n_pages - nf) * c->cfg.page_size;
         if (last_dense) rows -= (int64_t)n_pages * c->cfg.page_size - s.n_tokens;  // unfilled rows of the last page are not read
         bytes += (int64_t)c->geo.n_kv_heads * ((int64_t)nf * c->geo.blob_bytes + rows * 2 * kRowBytes);
+        if (nf > 0) bytes += (int64_t)c->geo.n_kv_heads * c->geo.basis_head_bytes;     // Global SVD form: the shared bases, once
     }
     c->last_decode_bytes = bytes;
     c->last_decode_units = pc.units;
@@ -946,6 +1027,7 @@ static pkv_status decode_impl(pkv_cache *c, int32_t layer, int32_t n_seqs, const
     a.dense_pool = c->dense_pool; a.factor_pool = c->factor_pool;
     a.page_table = (const int *)(c->meta + c->ml.page_table);
     a.n_tokens = (const int *)(c->meta + c->ml.n_tokens);
+    a.basis = c->meta + c->ml.basis;
     a.plan = c->meta + c->ml.plans + c->ml.plan_stride * layer;
     a.plan_cta = c->ml.plan_cta; a.plan_entry = c->ml.plan_entry; a.plan_seg = c->ml.plan_seg;
     a.plan_cta_entry = c->ml.plan_cta_entry;
@@ -1132,6 +1214,7 @@ pkv_status pkv_free_seq(pkv_cache *c, int32_t seq) {
         s.slots.clear();
         s.n_tokens = 0;
         s.f_end = c->geo.sink_pages;
+        s.has_basis = false;
         s.version++;
     }
     return PKV_OK;
@@ -1149,7 +1232,7 @@ pkv_status pkv_read_factors(pkv_cache *c, int64_t slot, int32_t head, void *A_k,
                             void *B_v, void *stream) {
     pkv_status r = slot_args(c, slot, c ? c->cfg.n_factor_slots : 0, head);
     if (r != PKV_OK) return r;
-    if (!A_k || !B_k || !A_v || !B_v) return fail(c, PKV_ERR_INVALID_ARG, "output pointer is NULL");
+    if (!A_k || !A_v || (c->geo.global_rank == 0 && (!B_k || !B_v))) return fail(c, PKV_ERR_INVALID_ARG, "output pointer is NULL");
     const unsigned char *blob = c->factor_pool + slot * c->geo.factor_slot_bytes + (int64_t)head * c->geo.blob_bytes;
     PKV_CUDA(c, launch_read_factors(c->geo, blob, A_k, B_k, A_v, B_v, (cudaStream_t)stream));
     return PKV_OK;
@@ -1161,6 +1244,7 @@ pkv_status pkv_write_factors(pkv_cache *c, int64_t slot, int32_t head, const voi
     if (r != PKV_OK) return r;
     if (!A_k || !B_k || !A_v || !B_v) return fail(c, PKV_ERR_INVALID_ARG, "input pointer is NULL");
     if (c->geo.factor_bits == 4) return fail(c, PKV_ERR_UNSUPPORTED, "pkv_write_factors is not available with INT4 factors");
+    if (c->geo.global_rank > 0) return fail(c, PKV_ERR_UNSUPPORTED, "pkv_write_factors is not available in the Global SVD form");
     unsigned char *blob = c->factor_pool + slot * c->geo.factor_slot_bytes + (int64_t)head * c->geo.blob_bytes;
     c->cache_written = true;                     // the next decode launch must not start ahead of this kernel
     PKV_CUDA(c, launch_write_factors(c->geo, blob, A_k, B_k, A_v, B_v, (cudaStream_t)stream));
@@ -1172,6 +1256,20 @@ pkv_status pkv_get_rotation_schedule(int32_t page_size, uint8_t *members, int64_
     int nr = 0, ng = 0, gs = 0;
     if (!pkv::rotation_schedule(page_size, members, capacity, &nr, &ng, &gs)) return PKV_ERR_INVALID_ARG;
     *n_rounds = nr; *groups_per_round = ng; *group_size = gs;
+    return PKV_OK;
+}
+
+pkv_status pkv_read_basis(pkv_cache *c, int32_t seq, int32_t layer, int32_t head, void *B_k, void *B_v, void *stream) {
+    if (!c) return PKV_ERR_INVALID_ARG;
+    if (c->dry) return fail(c, PKV_ERR_INVALID_ARG, "no device buffers in dry-run mode");
+    if (c->geo.global_rank == 0) return fail(c, PKV_ERR_INVALID_ARG, "the cache does not use the Global SVD form");
+    if (seq < 0 || seq >= c->cfg.max_seqs) return fail(c, PKV_ERR_BAD_SEQ, "sequence id %d out of range", seq);
+    if (layer < 0 || layer >= c->cfg.n_layers || head < 0 || head >= c->cfg.n_kv_heads || !B_k || !B_v)
+        return fail(c, PKV_ERR_INVALID_ARG, "layer or head out of range, or an output pointer is NULL");
+    if (!c->at(seq, layer).has_basis) return fail(c, PKV_ERR_INVALID_ARG, "sequence %d has no basis in layer %d yet", seq, layer);
+    const unsigned char *b = c->meta + c->ml.basis +
+                             (((long long)seq * c->cfg.n_layers + layer) * c->geo.n_kv_heads + head) * c->geo.basis_head_bytes;
+    PKV_CUDA(c, launch_read_basis(c->geo, b, B_k, B_v, (cudaStream_t)stream));
     return PKV_OK;
 }
 

@@ -36,6 +36,8 @@ namespace {
 constexpr float kNegInf = -1e30f;      // finite stand-in for -inf: exp2(kNegInf - x) == 0, no NaN from inf - inf
 constexpr float kMasked = -2e30f;      // score of a token a query must not see: exp2(kMasked - m) == 0 even while m == kNegInf
 constexpr int kKindDense = 0, kKindFactor = 1, kKindEnd = 2;
+// Global SVD form: a region's shared basis travels through the ring like a page, once per consumer warp
+constexpr int kKindBasisK = 3, kKindBasisV = 4;
 
 struct Range {
     PlanCta start, end;
@@ -361,8 +363,10 @@ struct WarpState {
 // Shapes fixed at compile time: P tokens per page, NT = ceil(rank / 8) rank tiles (K and V alike), I4 = factors
 // stored as INT4 codes.
 // rows per dense block: 32 where a stage has to be that large for a bf16 factor page anyway
-template <int P, int NT, bool I4>
-constexpr int kDenseBlock = (!I4 && P >= 32 && NT >= 3) ? 32 : 16;
+// F = storage form of the factors: 0 = bf16 page-wise (Eq. 2), 1 = INT4 page-wise (Section 4.3), 2 = Global SVD form
+// (Section 4.2: pages hold A rows only, the basis is shared by the region)
+template <int P, int NT, int F>
+constexpr int kDenseBlock = (F != 1 && P >= 32 && NT >= 3) ? 32 : 16;
 
 template <int P, int NT>
 struct Tc {
@@ -375,7 +379,8 @@ template <int P>
 __device__ __forceinline__ int a_swz(int l7) { return P == 64 ? l7 : (P == 32 ? (l7 >> 1) : (l7 >> 2)); }
 
 template <int NI>         // softmax over NI score tiles of 16 tokens; leaves p in place and its bf16, transposed copies
-__device__ __forceinline__ void online_softmax(float (&s)[4][4], WarpState &st, uint32_t (&T0)[4], uint32_t (&T1)[4]) {
+__device__ __forceinline__ void online_softmax(float (&s)[4][4], WarpState &st, uint32_t (&T0)[4], uint32_t (&T1)[4],
+                                               float &al0_out, float &al1_out) {
     float mx0 = kNegInf, mx1 = kNegInf;
 #pragma unroll
     for (int i = 0; i < NI; ++i) {
@@ -389,6 +394,7 @@ __device__ __forceinline__ void online_softmax(float (&s)[4][4], WarpState &st, 
     }
     const float mn0 = fmaxf(st.m[0], mx0), mn1 = fmaxf(st.m[1], mx1);
     const float al0 = exp2f(st.m[0] - mn0), al1 = exp2f(st.m[1] - mn1);
+    al0_out = al0; al1_out = al1;                       // (for accumulators the caller keeps besides st.o)
     st.m[0] = mn0; st.m[1] = mn1;
     float sum0 = 0.f, sum1 = 0.f;
 #pragma unroll
@@ -409,6 +415,12 @@ __device__ __forceinline__ void online_softmax(float (&s)[4][4], WarpState &st, 
         T0[i] = movm_t(pack_bf16(s[i][0], s[i][1]));   // (head g; tokens 16i+2t, +1)
         T1[i] = movm_t(pack_bf16(s[i][2], s[i][3]));   // (head g; tokens 16i+8+2t, +1)
     }
+}
+
+template <int NI>
+__device__ __forceinline__ void online_softmax(float (&s)[4][4], WarpState &st, uint32_t (&T0)[4], uint32_t (&T1)[4]) {
+    float a0, a1;
+    online_softmax<NI>(s, st, T0, T1, a0, a1);
 }
 
 __device__ __forceinline__ uint32_t lds32(uint32_t addr) {
@@ -655,7 +667,8 @@ __device__ __forceinline__ void factor_unit_int4(uint32_t sb, const Geometry &g,
 // query tokens per sequence and the block holds positions after the column's own).
 template <int DB>
 __device__ __forceinline__ void dense_unit(uint32_t sb, unsigned char *sp, int rows, int lim0, int lim1,
-                                           const uint32_t (&qf)[8][2], float scale, WarpState &st, int lane) {
+                                           const uint32_t (&qf)[8][2], float scale, WarpState &st, int lane,
+                                           float *alphas = nullptr) {
     constexpr int NI = DB / 16;
     const int l7 = lane & 7, mi = lane >> 3, g = lane >> 2;
     if (rows < DB) {
@@ -678,7 +691,9 @@ __device__ __forceinline__ void dense_unit(uint32_t sb, unsigned char *sp, int r
         s[i][2] = 16 * i + 8 + g < lim0 ? s[i][2] * scale : kMasked; s[i][3] = 16 * i + 8 + g < lim1 ? s[i][3] * scale : kMasked;
     }
     uint32_t T0[4], T1[4];
-    online_softmax<NI>(s, st, T0, T1);
+    float al0, al1;
+    online_softmax<NI>(s, st, T0, T1, al0, al1);
+    if (alphas) { alphas[0] = al0; alphas[1] = al1; }
 #pragma unroll
     for (int ii = 0; ii < 8; ++ii) {
 #pragma unroll
@@ -687,6 +702,142 @@ __device__ __forceinline__ void dense_unit(uint32_t sb, unsigned char *sp, int r
             ldsm_x4_t(a4, sb + DB * kRowBytes + (16 * i + (mi >> 1) * 8 + l7) * kRowBytes +
                               (((2 * ii + (mi & 1)) ^ l7) << 4));
             mma16816(st.o[ii], a4[0], a4[1], a4[2], a4[3], T0[i], T1[i]);
+        }
+    }
+}
+
+// ---- Global SVD form (Section 4.2) ------------------------------------------------------------------------
+// A region shares its bases; a page holds A_k^T and A_v^T (r x P each).  Per CTA and segment every consumer warp
+// gets one copy of B_k before the pages (it computes q~ = B_k q once and keeps it, as two bf16 terms, in its own part
+// of the combine area) and one copy of B_v after them (it turns its rank-space sum w = sum_pages A_v^T p into
+// o += B_v^T w).  Between the two a page costs s = A_k q~, the softmax, and w += A_v^T p.
+// w lives in registers as the mma accumulator of w^T [heads][ranks]: wacc[j] = (head lane >> 2; ranks 8j + 2t, +1).
+
+// The factor that a rescaling of query head lane >> 2 applies to this lane's wacc (the softmax keeps its factors by
+// column pair: head 2t in al0, head 2t + 1 in al1, t = lane & 3).
+__device__ __forceinline__ float alpha_of_row_head(float al0, float al1, int lane) {
+    const int g = lane >> 2;
+    const float a0 = __shfl_sync(0xffffffffu, al0, g >> 1), a1 = __shfl_sync(0xffffffffu, al1, g >> 1);
+    return (g & 1) ? a1 : a0;
+}
+
+template <int NT>
+__device__ __forceinline__ void scale_wacc(float (&wacc)[NT][2], float al0, float al1, int lane) {
+    if (__any_sync(0xffffffffu, al0 != 1.f || al1 != 1.f)) {
+        const float aw = alpha_of_row_head(al0, al1, lane);
+#pragma unroll
+        for (int j = 0; j < NT; ++j) { wacc[j][0] *= aw; wacc[j][1] *= aw; }
+    }
+}
+
+// B_k (r x d, at sb): q~^T [G][r] = q . B_k^T, scaled, split into two bf16 terms, stored for this lane at
+// qts + (2j, 2j + 1) * 128 bytes + lane * 4.
+template <int NT>
+__device__ __forceinline__ void global_basis_k(uint32_t sb, const uint32_t (&qf)[8][2], float scale, uint32_t qts, int lane) {
+    const int l7 = lane & 7, mi = lane >> 3;
+#pragma unroll
+    for (int jc = 0; jc < NT; jc += 4) {
+        float qt[4][4];
+#pragma unroll
+        for (int j = 0; j < 4; ++j) qt[j][0] = qt[j][1] = qt[j][2] = qt[j][3] = 0.f;
+#pragma unroll
+        for (int qd = 0; qd < 4; ++qd) {
+            uint32_t b[4][4];
+#pragma unroll
+            for (int j = 0; j < 4; ++j)
+                if (jc + j < NT) ldsm_x4(b[j], sb + (8 * (jc + j) + l7) * kRowBytes + (((4 * qd + mi) ^ l7) << 4));
+#pragma unroll
+            for (int j = 0; j < 4; ++j)
+                if (jc + j < NT) mma16816(qt[j], qf[2 * qd][0], 0u, qf[2 * qd][1], 0u, b[j][0], b[j][1]);
+#pragma unroll
+            for (int j = 0; j < 4; ++j)
+                if (jc + j < NT) mma16816(qt[j], qf[2 * qd + 1][0], 0u, qf[2 * qd + 1][1], 0u, b[j][2], b[j][3]);
+        }
+#pragma unroll
+        for (int j = 0; j < 4; ++j) {
+            if (jc + j < NT) {
+                const float x0 = qt[j][0] * scale, x1 = qt[j][1] * scale;
+                const uint32_t hi = pack_bf16(x0, x1);
+                const uint32_t lo = pack_bf16(x0 - bf16lo_f(hi), x1 - bf16hi_f(hi));
+                asm volatile("st.shared.b32 [%0], %1;" ::"r"(qts + (2 * (jc + j)) * 128 + lane * 4), "r"(hi) : "memory");
+                asm volatile("st.shared.b32 [%0], %1;" ::"r"(qts + (2 * (jc + j) + 1) * 128 + lane * 4), "r"(lo) : "memory");
+            }
+        }
+    }
+    __syncwarp();
+}
+
+// One page: A_k^T at sb, A_v^T at sb + av.
+template <int P, int NT>
+__device__ __forceinline__ void global_page_unit(uint32_t sb, int av, uint32_t qts, WarpState &st, float (&wacc)[NT][2],
+                                                 int lane) {
+    using C = Tc<P, NT>;
+    static_assert(NT % 2 == 0, "the Global SVD form uses ranks that are multiples of 16");
+    const int l7 = lane & 7, mi = lane >> 3;
+    const int asw = a_swz<P>(l7);
+    float s[4][4];
+#pragma unroll
+    for (int i = 0; i < C::kMT; ++i) s[i][0] = s[i][1] = s[i][2] = s[i][3] = 0.f;
+#pragma unroll
+    for (int kk = 0; kk < NT / 2; ++kk) {
+        uint32_t a4[C::kMT][4];
+#pragma unroll
+        for (int i = 0; i < C::kMT; ++i)
+            ldsm_x4_t(a4[i], sb + (16 * kk + (mi >> 1) * 8 + l7) * C::kPitchA + (((2 * i + (mi & 1)) ^ asw) << 4));
+        const uint32_t h0 = lds32(qts + (4 * kk) * 128 + lane * 4), l0 = lds32(qts + (4 * kk + 1) * 128 + lane * 4);
+        const uint32_t h1 = lds32(qts + (4 * kk + 2) * 128 + lane * 4), l1 = lds32(qts + (4 * kk + 3) * 128 + lane * 4);
+#pragma unroll
+        for (int i = 0; i < C::kMT; ++i) mma16816(s[i], a4[i][0], a4[i][1], a4[i][2], a4[i][3], h0, h1);
+#pragma unroll
+        for (int i = 0; i < C::kMT; ++i) mma16816(s[i], a4[i][0], a4[i][1], a4[i][2], a4[i][3], l0, l1);
+    }
+    uint32_t T0[4], T1[4];
+    float al0, al1;
+    online_softmax<C::kMT>(s, st, T0, T1, al0, al1);
+    scale_wacc<NT>(wacc, al0, al1, lane);
+    // ---- w^T [G][r] += p^T [G][P] . A_v [P][r] ----
+#pragma unroll
+    for (int jc = 0; jc < NT; jc += 4) {
+        float wt[4][4];
+#pragma unroll
+        for (int j = 0; j < 4; ++j) {
+            wt[j][0] = jc + j < NT ? wacc[jc + j < NT ? jc + j : 0][0] : 0.f;
+            wt[j][1] = jc + j < NT ? wacc[jc + j < NT ? jc + j : 0][1] : 0.f;
+            wt[j][2] = wt[j][3] = 0.f;
+        }
+#pragma unroll
+        for (int qd = 0; qd < C::kMT / 2; ++qd) {
+            uint32_t b[4][4];
+#pragma unroll
+            for (int j = 0; j < 4; ++j)
+                if (jc + j < NT) ldsm_x4(b[j], sb + av + (8 * (jc + j) + l7) * C::kPitchA + (((4 * qd + mi) ^ asw) << 4));
+#pragma unroll
+            for (int j = 0; j < 4; ++j)
+                if (jc + j < NT) mma16816(wt[j], T0[2 * qd], 0u, T1[2 * qd], 0u, b[j][0], b[j][1]);
+#pragma unroll
+            for (int j = 0; j < 4; ++j)
+                if (jc + j < NT) mma16816(wt[j], T0[2 * qd + 1], 0u, T1[2 * qd + 1], 0u, b[j][2], b[j][3]);
+        }
+#pragma unroll
+        for (int j = 0; j < 4; ++j)
+            if (jc + j < NT) { wacc[jc + j < NT ? jc + j : 0][0] = wt[j][0]; wacc[jc + j < NT ? jc + j : 0][1] = wt[j][1]; }
+    }
+}
+
+// B_v (r x d, at sb): o [d][G] += B_v^T . w, then w = 0.
+template <int NT>
+__device__ __forceinline__ void global_basis_v(uint32_t sb, float (&wacc)[NT][2], WarpState &st, int lane) {
+    const int l7 = lane & 7, mi = lane >> 3;
+    uint32_t wh[NT];
+#pragma unroll
+    for (int j = 0; j < NT; ++j) { wh[j] = pack_bf16(wacc[j][0], wacc[j][1]); wacc[j][0] = wacc[j][1] = 0.f; }
+#pragma unroll
+    for (int kk = 0; kk < NT / 2; ++kk) {
+#pragma unroll
+        for (int i = 0; i < 8; ++i) {
+            uint32_t a4[4];
+            ldsm_x4_t(a4, sb + (16 * kk + (mi >> 1) * 8 + l7) * kRowBytes + (((2 * i + (mi & 1)) ^ l7) << 4));
+            mma16816(st.o[i], a4[0], a4[1], a4[2], a4[3], wh[2 * kk], wh[2 * kk + 1]);
         }
     }
 }
@@ -947,9 +1098,10 @@ __device__ __forceinline__ void flush_segment(const DecodeArgs &a, float *comb, 
     PKV_CONSUMER_BARRIER();
 }
 
-template <int P, int NT, bool I4>
+template <int P, int NT, int F>
 __global__ void __launch_bounds__(kDecodeThreads, 2) decode_tc_kernel(const __grid_constant__ DecodeArgs a) {
-    constexpr int kDB = kDenseBlock<P, NT, I4>;
+    constexpr int kDB = kDenseBlock<P, NT, F>;
+    constexpr bool I4 = F == 1, kGlobal = F == 2;
     Range rg;
     if (!load_range(a, rg)) return;
     const Geometry &geo = a.geo;
@@ -986,7 +1138,7 @@ __global__ void __launch_bounds__(kDecodeThreads, 2) decode_tc_kernel(const __gr
         for (int s = 0; s < S; ++s) armed[s] = 0;
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     }
-    if (!I4 && stage_bytes > blob_bytes) {
+    if (F == 0 && stage_bytes > blob_bytes) {
         // Tile loads of 8 rows read past a rank that is not a multiple of 8; past the last matrix that is the
         // tail of the stage, which no copy of a factor page ever writes.  Those values are multiplied by exact
         // zeros, so they only have to be finite: clear the tails once.
@@ -1013,6 +1165,53 @@ __global__ void __launch_bounds__(kDecodeThreads, 2) decode_tc_kernel(const __gr
         int k = 0, seg_local = 0;
         bool ok = true;
         const bool keep = a.q_group > 1;     // sibling CTAs read the same pages: leave them in L2 for one another
+        // Lanes 0 .. n_here-1 arm their own units (kind, rows, after, src are per lane), S at a time (one stage
+        // each).  No lane blocks the others: all lanes poll together, and a unit is armed and tagged the moment its
+        // stage is free.  (Waiting for a whole group before telling the consumers can deadlock: a consumer may have
+        // to see unit k, of a later segment, to join the flush barrier that another warp must pass before it
+        // releases the stage that unit k + 1 is waiting for.)
+        auto arm = [&](int n_here, int kind, int rows, int after, const unsigned char *src) {
+            for (int j0 = 0; j0 < n_here && ok; j0 += S) {
+                const int kj = k + lane, s = kj % S;
+                bool pending = lane >= j0 && lane < min(j0 + S, n_here);
+                const long long t0 = clock64();
+                while (__any_sync(0xffffffffu, pending)) {
+                    if (pending && a.drop_unit == kj && blockIdx.x == 0) {
+                        pending = false;             // test hook: this unit is never armed, so its consumer's wait runs out
+                    } else if (pending && (kj < S || mbar_try_wait(smem_u32(empty_bar + s), ((kj / S) - 1) & 1))) {
+                        descs[s] = StageDesc{kind, rows, seg_local, after};
+                        const uint32_t bar = smem_u32(full_bar + s);
+                        const uint32_t dst = smem_u32(stages + (size_t)s * stage_bytes);
+                        if (kind == kKindFactor) {
+                            mbar_arrive_expect_tx(bar, blob_bytes);
+                            if (keep) bulk_g2s_keep(dst, src, blob_bytes, bar);
+                            else bulk_g2s(dst, src, blob_bytes, bar);
+                        } else if (kind == kKindBasisK || kind == kKindBasisV) {
+                            // (every CTA of the segment reads the same basis: leave it in L2)
+                            mbar_arrive_expect_tx(bar, geo.global_rank * kRowBytes);
+                            bulk_g2s_keep(dst, src, geo.global_rank * kRowBytes, bar);
+                        } else if (rows > 0) {
+                            mbar_arrive_expect_tx(bar, 2 * rows * kRowBytes);
+                            if (keep) {
+                                bulk_g2s_keep(dst, src, rows * kRowBytes, bar);
+                                bulk_g2s_keep(dst + kDB * kRowBytes, src + P * kRowBytes, rows * kRowBytes, bar);
+                            } else {
+                                bulk_g2s(dst, src, rows * kRowBytes, bar);
+                                bulk_g2s(dst + kDB * kRowBytes, src + P * kRowBytes, rows * kRowBytes, bar);
+                            }
+                        } else {
+                            mbar_arrive(bar);
+                        }
+                        st_release_smem(armed + s, kj + 1);
+                        if (trace && kj == 0) trace[3] = clock64();
+                        pending = false;
+                    }
+                    if (clock64() - t0 > a.wait_clocks) break;         // about a second: give up
+                }
+                ok = !__any_sync(0xffffffffu, pending);
+            }
+            k += n_here;
+        };
         PlanCta cur = rg.start;
         while (ok && !(cur.entry == rg.end.entry && cur.head == rg.end.head && cur.unit == rg.end.unit)) {
             const PlanEntry e = cur.entry == rg.start.entry ? rg.first_entry : entries[cur.entry];
@@ -1021,6 +1220,12 @@ __global__ void __launch_bounds__(kDecodeThreads, 2) decode_tc_kernel(const __gr
             const int u_end = last_run ? rg.end.unit : hu.units;
             const int T = a.n_tokens[(long long)e.seq * geo.n_layers + a.layer];
             const int *pt = a.page_table + ((long long)e.seq * geo.n_layers + a.layer) * geo.max_pages;
+            // Global SVD form: if this run holds factor pages, every consumer warp gets the region's B_k ahead of
+            // them and its B_v behind them (W consecutive units go to W different warps)
+            const bool run_global = kGlobal && max(cur.unit, hu.d0) < min(u_end, hu.d0 + hu.nf);
+            const unsigned char *bsrc = kGlobal ? a.basis + (((long long)e.seq * geo.n_layers + a.layer) * geo.n_kv_heads + cur.head) *
+                                                                geo.basis_head_bytes : nullptr;
+            if (run_global) arm(W, kKindBasisK, 1, 0, bsrc);
             for (int u0 = cur.unit; u0 < u_end && ok; u0 += 32) {
                 const int u = u0 + lane;
                 int kind = kKindDense, rows = 0, after = 0;
@@ -1043,49 +1248,9 @@ __global__ void __launch_bounds__(kDecodeThreads, 2) decode_tc_kernel(const __gr
                               (long long)cur.head * geo.dense_head_bytes + blk * kDB * kRowBytes;
                     }
                 }
-                // Lanes arm their own units, S at a time (one stage each).  No lane blocks the others: all lanes
-                // poll together, and a unit is armed and tagged the moment its stage is free.  (Waiting for a
-                // whole group before telling the consumers can deadlock: a consumer may have to see unit k, of a
-                // later segment, to join the flush barrier that another warp must pass before it releases the
-                // stage that unit k + 1 is waiting for.)
-                const int n_here = min(32, u_end - u0);
-                for (int j0 = 0; j0 < n_here && ok; j0 += S) {
-                    const int kj = k + lane, s = kj % S;
-                    bool pending = lane >= j0 && lane < min(j0 + S, n_here);
-                    const long long t0 = clock64();
-                    while (__any_sync(0xffffffffu, pending)) {
-                        if (pending && a.drop_unit == kj && blockIdx.x == 0) {
-                            pending = false;             // test hook: this unit is never armed, so its consumer's wait runs out
-                        } else if (pending && (kj < S || mbar_try_wait(smem_u32(empty_bar + s), ((kj / S) - 1) & 1))) {
-                            descs[s] = StageDesc{kind, rows, seg_local, after};
-                            const uint32_t bar = smem_u32(full_bar + s);
-                            const uint32_t dst = smem_u32(stages + (size_t)s * stage_bytes);
-                            if (kind == kKindFactor) {
-                                mbar_arrive_expect_tx(bar, blob_bytes);
-                                if (keep) bulk_g2s_keep(dst, src, blob_bytes, bar);
-                                else bulk_g2s(dst, src, blob_bytes, bar);
-                            } else if (rows > 0) {
-                                mbar_arrive_expect_tx(bar, 2 * rows * kRowBytes);
-                                if (keep) {
-                                    bulk_g2s_keep(dst, src, rows * kRowBytes, bar);
-                                    bulk_g2s_keep(dst + kDB * kRowBytes, src + P * kRowBytes, rows * kRowBytes, bar);
-                                } else {
-                                    bulk_g2s(dst, src, rows * kRowBytes, bar);
-                                    bulk_g2s(dst + kDB * kRowBytes, src + P * kRowBytes, rows * kRowBytes, bar);
-                                }
-                            } else {
-                                mbar_arrive(bar);
-                            }
-                            st_release_smem(armed + s, kj + 1);
-                            if (trace && kj == 0) trace[3] = clock64();
-                            pending = false;
-                        }
-                        if (clock64() - t0 > a.wait_clocks) break;         // about a second: give up
-                    }
-                    ok = !__any_sync(0xffffffffu, pending);
-                }
-                k += n_here;
+                arm(min(32, u_end - u0), kind, rows, after, src);
             }
+            if (run_global && ok) arm(W, kKindBasisV, 1, 0, bsrc + geo.global_rank * kRowBytes);
             if (last_run) break;
             cur.unit = 0;
             if (++cur.head == geo.n_kv_heads) { cur.head = 0; ++cur.entry; }
@@ -1138,6 +1303,12 @@ __global__ void __launch_bounds__(kDecodeThreads, 2) decode_tc_kernel(const __gr
         uint32_t qf[8][2];
         int cur_seg = 0;
         int hidden = load_q(a, query_seg(a, rg.seg_first), qf, lane);
+        // Global SVD form: this warp's rank-space sum, and where it keeps q~ (its own part of the combine area, which it
+        // overwrites with its state only at a flush, when q~ of that segment is no longer needed)
+        float wacc[kGlobal ? NT : 1][2];
+#pragma unroll
+        for (int j = 0; j < (kGlobal ? NT : 1); ++j) wacc[j][0] = wacc[j][1] = 0.f;
+        const uint32_t qts = smem_u32(comb + warp * kPartialFloats);
         bool ok = true;
         for (int k = warp;; k += W) {
             const int s = k % S;
@@ -1163,7 +1334,18 @@ __global__ void __launch_bounds__(kDecodeThreads, 2) decode_tc_kernel(const __gr
             dsc.rows = min(dsc.rows, dsc.kind == kKindFactor ? P : kDB);
             if (dsc.rows > 0) {
                 const uint32_t sb = smem_u32(stages + (size_t)s * stage_bytes);
-                if (dsc.kind == kKindFactor) {
+                if constexpr (kGlobal) {
+                    if (dsc.kind == kKindBasisK) global_basis_k<NT>(sb, qf, geo.scale_log2e, qts, lane);
+                    else if (dsc.kind == kKindBasisV) global_basis_v<NT>(sb, wacc, st, lane);
+                    else if (dsc.kind == kKindFactor) global_page_unit<P, NT>(sb, geo.av_off, qts, st, wacc, lane);
+                    else {
+                        float al[2];
+                        dense_unit<kDB>(sb, stages + (size_t)s * stage_bytes, dsc.rows, dsc.rows, dsc.rows, qf, geo.scale_log2e, st,
+                                        lane, al);
+                        scale_wacc<NT>(wacc, al[0], al[1], lane);
+                        if (dsc.rows < kDB) asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+                    }
+                } else if (dsc.kind == kKindFactor) {
                     if (I4) factor_unit_int4<P, NT>(sb, geo, qf, st, lane);
                     else factor_unit<P, NT>(sb, geo.ak_off, geo.bk_off, geo.av_off, geo.bv_off, geo.rank_k, geo.rank_v, qf,
                                             geo.scale_log2e, st, lane);
@@ -1648,7 +1830,7 @@ size_t decode_smem_bytes(const Geometry &g) {
            g.n_stages * (8 + 8 + sizeof(StageDesc) + 4) + 64;
 }
 
-template <int P, int NT, bool I4>
+template <int P, int NT, int F>
 cudaError_t launch_tc(const DecodeArgs &a, cudaStream_t st) {
     cudaLaunchConfig_t cfg = {};
     cfg.gridDim = dim3(a.geo.n_ctas);
@@ -1660,17 +1842,20 @@ cudaError_t launch_tc(const DecodeArgs &a, cudaStream_t st) {
     attr[0].val.programmaticStreamSerializationAllowed = 1;
     cfg.attrs = attr;
     cfg.numAttrs = a.plain_launch ? 0 : 1;
-    return cudaLaunchKernelEx(&cfg, decode_tc_kernel<P, NT, I4>, a);
+    return cudaLaunchKernelEx(&cfg, decode_tc_kernel<P, NT, F>, a);
 }
 
 template <int P, int NT>
 cudaError_t setup_tc() {
-    cudaError_t e = cudaFuncSetAttribute(decode_tc_kernel<P, NT, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBudget / 2);
+    cudaError_t e = cudaFuncSetAttribute(decode_tc_kernel<P, NT, 0>, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBudget / 2);
     if (e != cudaSuccess) return e;
     e = cudaFuncSetAttribute(block_tc_kernel<P, NT>, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBudget / 2);
     if (e != cudaSuccess) return e;
-    return cudaFuncSetAttribute(decode_tc_kernel<P, NT, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBudget / 2);
+    return cudaFuncSetAttribute(decode_tc_kernel<P, NT, 1>, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBudget / 2);
 }
+
+// the Global SVD form: P in {32, 64}, ranks 64, 80, 96
+#define PKV_FOR_EACH_GLOBAL_SHAPE(X) X(32, 8) X(32, 10) X(32, 12) X(64, 8) X(64, 10) X(64, 12)
 
 // the instantiated shapes: P in {16, 32, 64}, rank tiles 1..4 (1..2 for P = 16)
 #define PKV_FOR_EACH_SHAPE(X) \
@@ -1683,6 +1868,10 @@ cudaError_t decode_kernel_setup() {
 #define PKV_SETUP(P, NT) if ((e = setup_tc<P, NT>()) != cudaSuccess) return e;
     PKV_FOR_EACH_SHAPE(PKV_SETUP)
 #undef PKV_SETUP
+#define PKV_SETUP_G(P, NT) \
+    if ((e = cudaFuncSetAttribute(decode_tc_kernel<P, NT, 2>, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBudget / 2)) != cudaSuccess) return e;
+    PKV_FOR_EACH_GLOBAL_SHAPE(PKV_SETUP_G)
+#undef PKV_SETUP_G
     return cudaSuccess;
 }
 
@@ -1692,10 +1881,16 @@ cudaError_t launch_decode(const DecodeArgs &a, int n_segs, cudaStream_t st) {
         decode_scalar_kernel<<<a.geo.n_ctas, 128, 0, st>>>(a);
         e = cudaGetLastError();
     } else {
+        if (a.geo.global_rank > 0) {
+#define PKV_LAUNCH_G(P, NT) if (a.geo.page == P && a.geo.rank_tiles == NT) e = launch_tc<P, NT, 2>(a, st);
+            PKV_FOR_EACH_GLOBAL_SHAPE(PKV_LAUNCH_G)
+#undef PKV_LAUNCH_G
+        } else {
 #define PKV_LAUNCH(P, NT) if (a.geo.page == P && a.geo.rank_tiles == NT) \
-            e = a.geo.factor_bits == 4 ? launch_tc<P, NT, true>(a, st) : launch_tc<P, NT, false>(a, st);
-        PKV_FOR_EACH_SHAPE(PKV_LAUNCH)
+            e = a.geo.factor_bits == 4 ? launch_tc<P, NT, 1>(a, st) : launch_tc<P, NT, 0>(a, st);
+            PKV_FOR_EACH_SHAPE(PKV_LAUNCH)
 #undef PKV_LAUNCH
+        }
     }
     if (e != cudaSuccess || a.variant != 1) return e;
     merge_kernel<<<n_segs, 256, 0, st>>>(a);

@@ -40,6 +40,10 @@ struct Geometry {
     int blob16_bytes;                  // size of the bf16 form
     int blob_bytes;                    // stored size of a blob in the factor pool (= blob16_bytes for bf16 factors)
     int factor_bits;                   // 16 or 4
+    // Global SVD form (global_rank > 0): rank_k = rank_v = global_rank; a page's blob is [A_k^T r x P][A_v^T r x P]
+    // (bk_off, bv_off unused); the basis of a (sequence, layer, KV head) is [B_k r x d][B_v r x d] bf16 with the
+    // dense-row swizzle, basis_head_bytes in all, kept in the meta buffer.
+    int global_rank, basis_head_bytes;
     // INT4 blobs: [codes of A~_K][codes of B~_K][codes of A~_V][codes of B~_V][bf16 scales: A~_K per rank column
     // (padded to 8), B~_K per channel, A~_V per token, B~_V per channel].  Codes are stored in the register order
     // of the mma operand each matrix is read as (see int4_a_pos / int4_b_pos).
@@ -72,6 +76,7 @@ struct MetaLayout {                    // byte offsets inside the caller's `meta
     long long plan_cta_entry;          // PlanEntry [n_ctas]: a copy of the entry each CTA's range starts in (saves a dependent load)
     long long append_desc;             // int4 [max_seqs]
     long long status;                  // int32 [kStatusWords]
+    long long basis;                   // Global SVD form: bytes [max_seqs][n_layers][H_kv][basis_head_bytes]
     long long total;
 };
 
@@ -85,6 +90,7 @@ struct WorkspaceLayout {
 
     long long worklist;                // int2 [kCompressChunk]
     long long tickets;                 // int [n_sets][n_seg_tickets + n_group]: per segment, then per group
+    long long gram;                    // Global SVD form: float [H_kv][2][d][d], the region Gram matrices of one (sequence, layer)
     long long trace;                   // long long [n_ctas][kTraceSlots]
     long long total;
 };
@@ -97,6 +103,7 @@ struct DecodeArgs {
     const unsigned char *dense_pool, *factor_pool;
     const int *page_table;             // whole table
     const int *n_tokens;               // whole array
+    const unsigned char *basis;        // Global SVD form: all bases (see MetaLayout::basis)
     const unsigned char *plan;         // this layer's plan
     long long plan_cta, plan_entry, plan_seg, plan_cta_entry;
     const void *q;
@@ -144,6 +151,13 @@ cudaError_t launch_write_factors(const Geometry &geo, unsigned char *blob, const
                                  const void *A_v, const void *B_v, cudaStream_t st);
 cudaError_t launch_read_dense(const Geometry &geo, const unsigned char *head_base, void *K, void *V,
                               cudaStream_t st);
+// Global SVD form (pkv_global.cu).  worklist: (dense slot, factor slot) of the pages of ONE (sequence, layer).
+cudaError_t launch_region_basis(const Geometry &geo, const unsigned char *dense_pool, const int2 *worklist, int n_pages,
+                                float *gram, unsigned char *basis_seq_layer, int *status, cudaStream_t st);
+cudaError_t launch_project_pages(const Geometry &geo, const unsigned char *dense_pool, unsigned char *factor_pool,
+                                 const int2 *worklist, int n_pages, const unsigned char *basis_seq_layer, int *status,
+                                 cudaStream_t st);
+cudaError_t launch_read_basis(const Geometry &geo, const unsigned char *basis_head, void *B_k, void *B_v, cudaStream_t st);
 cudaError_t decode_kernel_setup();     // raises the dynamic shared-memory limit once per device
 // Rotation order of the compression kernel for page size P (see pkv_get_rotation_schedule); false if P is unsupported
 // or `cap` bytes are too few.

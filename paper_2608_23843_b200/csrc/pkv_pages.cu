@@ -60,7 +60,8 @@ __global__ void append_kernel(Geometry geo, unsigned char *dense_pool, const int
 __global__ void factor_io_kernel(Geometry geo, unsigned char *blob, unsigned short *A_k, unsigned short *B_k,
                                  unsigned short *A_v, unsigned short *B_v, int dir) {
     const int P = geo.page, rk = geo.rank_k, rv = geo.rank_v;
-    const int nAk = P * rk, nBk = rk * kHeadDim, nAv = P * rv, nBv = rv * kHeadDim;
+    // (Global SVD form: a page stores only its A rows)
+    const int nAk = P * rk, nBk = geo.global_rank ? 0 : rk * kHeadDim, nAv = P * rv, nBv = geo.global_rank ? 0 : rv * kHeadDim;
     for (int i = blockIdx.x * blockDim.x + threadIdx.x; i < nAk + nBk + nAv + nBv; i += gridDim.x * blockDim.x) {
         unsigned short *plain;
         int which, r, e, off;

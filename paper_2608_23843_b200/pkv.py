@@ -31,7 +31,7 @@ EXPORTS = [
     "pkv_read_dense", "pkv_get_decode_plan", "pkv_decode_attention_static_scratch", "pkv_get_decode_trace",
     "pkv_decode_attention_multi", "pkv_compress_begin", "pkv_compress_commit",
     "pkv_decode_attention_partial", "pkv_merge_attention_states",
-    "pkv_get_rotation_schedule",
+    "pkv_get_rotation_schedule", "pkv_read_basis",
 ]
 
 
@@ -45,6 +45,7 @@ class PkvConfig(ctypes.Structure):
         ("softmax_scale", ctypes.c_float), ("jacobi_max_sweeps", ctypes.c_int32),
         ("jacobi_tol", ctypes.c_float), ("n_ctas", ctypes.c_int32), ("decode_variant", ctypes.c_int32),
         ("jacobi_energy_tol", ctypes.c_float), ("factor_bits", ctypes.c_int32), ("decode_overlap", ctypes.c_int32),
+        ("global_rank", ctypes.c_int32),
     ]
 
 
@@ -99,6 +100,7 @@ def lib():
         L.pkv_read_factors.argtypes = [vp, i64, i32, vp, vp, vp, vp, vp]
         L.pkv_write_factors.argtypes = [vp, i64, i32, vp, vp, vp, vp, vp]
         L.pkv_read_dense.argtypes = [vp, i64, i32, vp, vp, vp]
+        L.pkv_read_basis.argtypes = [vp, i32, i32, i32, vp, vp, vp]
         L.pkv_get_decode_plan.argtypes = [vp, i32, ip, ip, ip, ip]
         L.pkv_get_decode_trace.argtypes = [vp, ctypes.POINTER(ctypes.c_int64), i32, vp]
         L.pkv_get_rotation_schedule.argtypes = [i32, ctypes.POINTER(ctypes.c_uint8), i64, ip, ip, ip]
@@ -314,14 +316,19 @@ def pkv_read_dense(handle, slot, kv_head, K, V, stream=None):
     _check(handle, lib().pkv_read_dense(handle, slot, kv_head, _ptr(K), _ptr(V), _stream(stream)))
 
 
+def pkv_read_basis(handle, seq, layer, kv_head, B_k, B_v, stream=None):
+    _check(handle, lib().pkv_read_basis(handle, seq, layer, kv_head, _ptr(B_k), _ptr(B_v), _stream(stream)))
+
+
 # ---- convenience wrapper ----------------------------------------------------------
 def make_config(n_layers, n_kv_heads, n_q_heads, rank, sink_tokens, recent_tokens, max_seqs, max_pages_per_seq,
                 n_dense_slots, n_factor_slots, head_dim=128, page_size=64, rank_v=None, softmax_scale=0.0,
                 jacobi_max_sweeps=0, jacobi_tol=0.0, n_ctas=0, decode_variant=0, decode_overlap=0,
-                jacobi_energy_tol=0.0, factor_bits=0) -> PkvConfig:
+                jacobi_energy_tol=0.0, factor_bits=0, global_rank=0) -> PkvConfig:
     return PkvConfig(n_layers, n_kv_heads, n_q_heads, head_dim, page_size, rank, rank if rank_v is None else rank_v,
                      sink_tokens, recent_tokens, max_seqs, max_pages_per_seq, n_dense_slots, n_factor_slots,
-                     softmax_scale, jacobi_max_sweeps, jacobi_tol, n_ctas, decode_variant, jacobi_energy_tol, factor_bits, decode_overlap)
+                     softmax_scale, jacobi_max_sweeps, jacobi_tol, n_ctas, decode_variant, jacobi_energy_tol, factor_bits, decode_overlap,
+                     global_rank)
 
 
 class Cache:
@@ -396,9 +403,21 @@ class Cache:
     def free_seq(self, seq):
         pkv_free_seq(self.handle, seq)
 
+    def read_basis(self, seq, layer, kv_head):
+        """Global SVD form: (B_k, B_v), each [global_rank, d] bf16."""
+        c = self.cfg
+        B_k = torch.empty((c.global_rank, c.head_dim), dtype=torch.bfloat16, device=self.device)
+        B_v = torch.empty_like(B_k)
+        pkv_read_basis(self.handle, seq, layer, kv_head, B_k, B_v, self._st())
+        return B_k, B_v
+
     def read_factors(self, slot, kv_head):
         c = self.cfg
         mk = lambda *s: torch.empty(s, dtype=torch.bfloat16, device=self.device)
+        if c.global_rank > 0:                               # only the token rows are stored per page
+            A_k, A_v = mk(c.page_size, c.global_rank), mk(c.page_size, c.global_rank)
+            pkv_read_factors(self.handle, slot, kv_head, A_k, None, A_v, None, self._st())
+            return A_k, None, A_v, None
         A_k, B_k = mk(c.page_size, c.rank_k), mk(c.rank_k, c.head_dim)
         A_v, B_v = mk(c.page_size, c.rank_v), mk(c.rank_v, c.head_dim)
         pkv_read_factors(self.handle, slot, kv_head, A_k, B_k, A_v, B_v, self._st())

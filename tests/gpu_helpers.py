@@ -17,7 +17,8 @@ def oracle_config(cfg: pkv.PkvConfig) -> OracleConfig:
                         head_dim=cfg.head_dim, page_size=cfg.page_size, rank_k=cfg.rank_k, rank_v=cfg.rank_v,
                         sink_tokens=cfg.sink_tokens, recent_tokens=cfg.recent_tokens, max_seqs=cfg.max_seqs,
                         n_dense_slots=cfg.n_dense_slots, n_factor_slots=cfg.n_factor_slots,
-                        softmax_scale=cfg.softmax_scale, factor_bits=4 if cfg.factor_bits == 4 else 16)
+                        softmax_scale=cfg.softmax_scale, factor_bits=4 if cfg.factor_bits == 4 else 16,
+                        global_rank=cfg.global_rank)
 
 
 class Pair:
@@ -63,12 +64,21 @@ class Pair:
     def load_gpu_factors_into_oracle(self, seq, layer):
         """Kernel gate: make the oracle attend over the GPU's own bf16 factors."""
         kinds, slots, _ = self.gpu.page_table(seq, layer)
+        H = self.cfg.n_kv_heads
+        basis = None
+        if self.cfg.global_rank > 0 and FACTOR in kinds:      # Global SVD form: pages hold A rows, the basis is shared
+            bs = [self.gpu.read_basis(seq, layer, h) for h in range(H)]
+            basis = [np.stack([f64(b[i]) for b in bs]) for i in range(2)]
         for kd, slot in zip(kinds, slots):
             if kd != FACTOR:
                 continue
-            parts = [self.gpu.read_factors(slot, h) for h in range(self.cfg.n_kv_heads)]
+            parts = [self.gpu.read_factors(slot, h) for h in range(H)]
             torch.cuda.synchronize()
-            self.orc.set_factors(slot, *[np.stack([f64(p[i]) for p in parts]) for i in range(4)])
+            if basis is not None:
+                self.orc.set_factors(slot, np.stack([f64(p[0]) for p in parts]), basis[0],
+                                     np.stack([f64(p[2]) for p in parts]), basis[1])
+            else:
+                self.orc.set_factors(slot, *[np.stack([f64(p[i]) for p in parts]) for i in range(4)])
 
     def dense_page_gpu(self, slot, head):
         K, V = self.gpu.read_dense(slot, head)
