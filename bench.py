@@ -54,9 +54,9 @@ WORKLOADS = {
 }
 SEED = 0
 # DRAM bytes (read + write) per algorithmic byte of a decode launch, from the ncu capture summarised in
-# profiles/decode_tc_kernel_r24_llama3_8b_32k_b8.md: (608.92 MB read + 4.52 MB written) / 608.70 MB.  Every
+# profiles/decode_tc_kernel_r24_llama3_8b_32k_b8.md: (608.78 MB read + 3.38 MB written) / 608.70 MB.  Every
 # unit is fetched once, so traffic scales with the units a launch processes.
-NCU_TRAFFIC_PER_ALGORITHMIC_BYTE = (608.9216e6 + 4.52096e6) / 608698368.0
+NCU_TRAFFIC_PER_ALGORITHMIC_BYTE = (608.780544e6 + 3.382016e6) / 608698368.0
 # the same for INT4 factors (profiles/decode_tc_kernel_int4_r24_llama3_8b_32k_b8.md): (183.74 MB + 3.96 MB) / 182.46 MB
 NCU_TRAFFIC_PER_ALGORITHMIC_BYTE_INT4 = (183.737856e6 + 3.961344e6) / 182461440.0
 
@@ -190,7 +190,7 @@ class ClockSampler:
 
 
 def build_workload(w, rank, device, overlap=2, n_ctas=0, factor_bits=16, grow=0, keep_kv=False, plan_entries_per_seq=1,
-                   decode_variant=0):
+                   decode_variant=0, global_rank=0):
     """Allocate the cache, generate each (layer, sequence) on the GPU, append and compress layer by layer.
     grow: tokens every sequence may still gain afterwards (sizes the pools and page tables); keep_kv: also
     return the generated K/V of layer 0 including those `grow` tokens (serving loop)."""
@@ -213,7 +213,7 @@ def build_workload(w, rank, device, overlap=2, n_ctas=0, factor_bits=16, grow=0,
                           sink_tokens=w["sink"], recent_tokens=w["recent"], max_seqs=w["batch"] * plan_entries_per_seq,
                           max_pages_per_seq=max(pages), n_dense_slots=n_dense_slots, n_factor_slots=n_factor_slots,
                           decode_overlap=overlap, n_ctas=n_ctas, factor_bits=factor_bits,
-                          decode_variant=decode_variant)
+                          decode_variant=decode_variant, global_rank=global_rank)
     cache = pkv.Cache(cfg, device, synth.slot_permutation(SEED, n_dense_slots, 0).tolist(),
                       synth.slot_permutation(SEED, n_factor_slots, 1).tolist())
     ids = list(range(w["batch"]))
@@ -240,7 +240,8 @@ def build_workload(w, rank, device, overlap=2, n_ctas=0, factor_bits=16, grow=0,
     st = cache.stats()
     comp = dict(pages_per_s=(n_svds / (svd_ms * 1e-3) if svd_ms > 0 else None), n_page_svds=n_svds, svd_ms=svd_ms,
                 spans=spans, jacobi_rounds=st["jacobi_rounds"], page_svds_counted=st["page_svds"],
-                not_converged=st["page_svds_not_converged"], page=P, rank=rank, rank_v=w.get("rank_v", rank))
+                not_converged=st["page_svds_not_converged"], page=P, rank=rank, rank_v=w.get("rank_v", rank),
+                global_rank=global_rank)
     if keep_kv:
         comp["new_k"] = torch.stack([k for k, _ in kept], 1).contiguous()      # [grow][batch][H_kv][d]
         comp["new_v"] = torch.stack([v for _, v in kept], 1).contiguous()
@@ -282,7 +283,7 @@ def compress_record(comp, sampler):
     Peak = SMs x 128 FMA lanes x 2 x SM clock sampled while the kernel ran (the maximum clock if no sample fell
     inside)."""
     n = comp["page_svds_counted"]
-    if not n or not comp["pages_per_s"]:
+    if not n or not comp["pages_per_s"] or comp.get("global_rank"):
         return None
     P, d = comp["page"], 128
     rounds = comp["jacobi_rounds"] / n
@@ -506,7 +507,8 @@ def _config_dict(args, w, rank):
     return {"workload": args.workload, "n_layers": w["n_layers"], "layers_per_step": w.get("layers_per_step", w["n_layers"]), "n_q_heads": w["n_q_heads"],
             "n_kv_heads": w["n_kv_heads"], "head_dim": 128, "batch": w["batch"], "context": w["T"],
             "queries_per_sequence": args.q_len,
-            "page_size": w.get("page", 64), "rank": rank, "rank_v": w.get("rank_v", rank), "factor_bits": args.factor_bits, "sink_tokens": w["sink"], "recent_tokens": w["recent"],
+            "page_size": w.get("page", 64), "rank": rank, "rank_v": w.get("rank_v", rank), "factor_bits": args.factor_bits,
+            "global_rank": getattr(args, "global_rank", 0), "sink_tokens": w["sink"], "recent_tokens": w["recent"],
             "l2": "inputs larger than L2 (no flush)" if args.workload != "tiny" else "L2-resident (latency only)",
             "overlap": ["0: each launch waits for the previous one",
                         "1: consecutive per-layer launches overlap (programmatic dependent launch) and complete in order",
@@ -545,6 +547,9 @@ def main():
                          "overlap but complete in order, 2 = launches never wait for one another (default)")
     ap.add_argument("--n-ctas", type=int, default=0, help="decode grid size (0 = library default)")
     ap.add_argument("--factor-bits", type=int, default=16, choices=[4, 16], help="factor storage: bf16 or INT4 (paper, Section 4.3)")
+    ap.add_argument("--global-rank", type=int, default=0, choices=[0, 64, 80, 96],
+                    help="the Global SVD form the paper compares with (Section 4.2): one basis of this rank per (sequence, layer, "
+                         "KV head) instead of page-wise factors")
     ap.add_argument("--q-len", type=int, default=1,
                     help="queries per sequence and step (1 = decoding; more = a speculative-decoding or chunked-prefill step "
                          "over the newest positions, pkv_decode_attention_multi)")
@@ -606,7 +611,8 @@ def main():
     sampler = ClockSampler(local)
     sampler.start()                                       # ahead of the cache build: its compression launches are sampled too
     cfg, cache, lengths, comp = build_workload(w, rank, device, args.overlap, args.n_ctas, args.factor_bits,
-                                               plan_entries_per_seq=-(-QL // per_tile), decode_variant=args.decode_variant)
+                                               plan_entries_per_seq=-(-QL // per_tile), decode_variant=args.decode_variant,
+                                               global_rank=args.global_rank)
     ids = list(range(w["batch"]))
     L, Hq = w["n_layers"], w["n_q_heads"]
     if QL == 1:
@@ -722,7 +728,8 @@ def main():
         cache.close()
         cache = None
         torch.cuda.empty_cache()
-        _, cache, _, _ = build_workload(w, rank, device, 0, args.n_ctas, args.factor_bits, decode_variant=args.decode_variant)
+        _, cache, _, _ = build_workload(w, rank, device, 0, args.n_ctas, args.factor_bits, decode_variant=args.decode_variant,
+                                        global_rank=args.global_rank)
         for _ in range(max(3, args.warmup)):
             eager_step()
         barrier()
@@ -754,7 +761,8 @@ def main():
             "algorithmic_bytes_per_step": bytes_per_step,
             "pages_factorized_per_s": comp["pages_per_s"], "page_svds_timed": comp["n_page_svds"],
             "compress": compress_record(comp, sampler),
-            "roofline": hbm_roofline("decode_tc_kernel<P=%d, rank tiles=%d>" % (w.get("page", 64), (rank + 7) // 8),
+            "roofline": hbm_roofline("decode_tc_kernel<P=%d, rank tiles=%d%s>" % (w.get("page", 64), ((args.global_rank or rank) + 7) // 8,
+                                                                                 ", Global SVD form" if args.global_rank else ""),
                                      bytes_per_launch, launch_ms * 1e3, args.factor_bits),
             "e2e": {"value": e2e_ms * 1e3, "unit": "us", "h2d_bytes_per_step": qbytes, "d2h_bytes_per_step": qbytes},
             "gpu_launches": lps * args.steps * (2 if args.seq_sharded else 1), "clocks": clocks,
@@ -786,7 +794,7 @@ def main():
                                 "achieved": tach, "peak": tpeak, "unit": "TFLOP/s", "frac": tach / tpeak,
                                 "peak_source": tsrc + "; the kernel uses mma.sync, whose pipe ncu showed 50 % busy at this rate",
                                 "traffic": None, "launch_us": launch_ms * 1e3, "algorithmic_flops_per_launch": flops}
-        if not args.no_cpu_baseline and world == 1 and QL == 1:
+        if not args.no_cpu_baseline and world == 1 and QL == 1 and not args.global_rank:
             o = oracle_sample(w, rank, 3, args.factor_bits)
             line["cpu_baseline"] = {"value": o["decode_s"] * 1e6 * o["slices_per_step"], "unit": "us",
                                     "cores": o["cores"], "kind": "oracle", "sample": o["sample"],
