@@ -731,37 +731,33 @@ __device__ __forceinline__ void scale_wacc(float (&wacc)[NT][2], float al0, floa
 }
 
 // B_k (r x d, at sb): q~^T [G][r] = q . B_k^T, scaled, split into two bf16 terms, stored for this lane at
-// qts + (2j, 2j + 1) * 128 bytes + lane * 4.
+// qts + (2j, 2j + 1) * 128 bytes + lane * 4.  (Rank tiles are taken two at a time: NT is even in this form.)
 template <int NT>
 __device__ __forceinline__ void global_basis_k(uint32_t sb, const uint32_t (&qf)[8][2], float scale, uint32_t qts, int lane) {
+    static_assert(NT % 2 == 0, "the Global SVD form uses ranks that are multiples of 16");
     const int l7 = lane & 7, mi = lane >> 3;
 #pragma unroll
-    for (int jc = 0; jc < NT; jc += 4) {
-        float qt[4][4];
+    for (int jc = 0; jc < NT; jc += 2) {
+        float qt[2][4];
 #pragma unroll
-        for (int j = 0; j < 4; ++j) qt[j][0] = qt[j][1] = qt[j][2] = qt[j][3] = 0.f;
+        for (int j = 0; j < 2; ++j) qt[j][0] = qt[j][1] = qt[j][2] = qt[j][3] = 0.f;
 #pragma unroll
         for (int qd = 0; qd < 4; ++qd) {
-            uint32_t b[4][4];
+            uint32_t b[2][4];
 #pragma unroll
-            for (int j = 0; j < 4; ++j)
-                if (jc + j < NT) ldsm_x4(b[j], sb + (8 * (jc + j) + l7) * kRowBytes + (((4 * qd + mi) ^ l7) << 4));
+            for (int j = 0; j < 2; ++j) ldsm_x4(b[j], sb + (8 * (jc + j) + l7) * kRowBytes + (((4 * qd + mi) ^ l7) << 4));
 #pragma unroll
-            for (int j = 0; j < 4; ++j)
-                if (jc + j < NT) mma16816(qt[j], qf[2 * qd][0], 0u, qf[2 * qd][1], 0u, b[j][0], b[j][1]);
+            for (int j = 0; j < 2; ++j) mma16816(qt[j], qf[2 * qd][0], 0u, qf[2 * qd][1], 0u, b[j][0], b[j][1]);
 #pragma unroll
-            for (int j = 0; j < 4; ++j)
-                if (jc + j < NT) mma16816(qt[j], qf[2 * qd + 1][0], 0u, qf[2 * qd + 1][1], 0u, b[j][2], b[j][3]);
+            for (int j = 0; j < 2; ++j) mma16816(qt[j], qf[2 * qd + 1][0], 0u, qf[2 * qd + 1][1], 0u, b[j][2], b[j][3]);
         }
 #pragma unroll
-        for (int j = 0; j < 4; ++j) {
-            if (jc + j < NT) {
-                const float x0 = qt[j][0] * scale, x1 = qt[j][1] * scale;
-                const uint32_t hi = pack_bf16(x0, x1);
-                const uint32_t lo = pack_bf16(x0 - bf16lo_f(hi), x1 - bf16hi_f(hi));
-                asm volatile("st.shared.b32 [%0], %1;" ::"r"(qts + (2 * (jc + j)) * 128 + lane * 4), "r"(hi) : "memory");
-                asm volatile("st.shared.b32 [%0], %1;" ::"r"(qts + (2 * (jc + j) + 1) * 128 + lane * 4), "r"(lo) : "memory");
-            }
+        for (int j = 0; j < 2; ++j) {
+            const float x0 = qt[j][0] * scale, x1 = qt[j][1] * scale;
+            const uint32_t hi = pack_bf16(x0, x1);
+            const uint32_t lo = pack_bf16(x0 - bf16lo_f(hi), x1 - bf16hi_f(hi));
+            asm volatile("st.shared.b32 [%0], %1;" ::"r"(qts + (2 * (jc + j)) * 128 + lane * 4), "r"(hi) : "memory");
+            asm volatile("st.shared.b32 [%0], %1;" ::"r"(qts + (2 * (jc + j) + 1) * 128 + lane * 4), "r"(lo) : "memory");
         }
     }
     __syncwarp();
@@ -797,30 +793,22 @@ __device__ __forceinline__ void global_page_unit(uint32_t sb, int av, uint32_t q
     scale_wacc<NT>(wacc, al0, al1, lane);
     // ---- w^T [G][r] += p^T [G][P] . A_v [P][r] ----
 #pragma unroll
-    for (int jc = 0; jc < NT; jc += 4) {
-        float wt[4][4];
+    for (int jc = 0; jc < NT; jc += 2) {
+        float wt[2][4];
 #pragma unroll
-        for (int j = 0; j < 4; ++j) {
-            wt[j][0] = jc + j < NT ? wacc[jc + j < NT ? jc + j : 0][0] : 0.f;
-            wt[j][1] = jc + j < NT ? wacc[jc + j < NT ? jc + j : 0][1] : 0.f;
-            wt[j][2] = wt[j][3] = 0.f;
-        }
+        for (int j = 0; j < 2; ++j) { wt[j][0] = wacc[jc + j][0]; wt[j][1] = wacc[jc + j][1]; wt[j][2] = wt[j][3] = 0.f; }
 #pragma unroll
         for (int qd = 0; qd < C::kMT / 2; ++qd) {
-            uint32_t b[4][4];
+            uint32_t b[2][4];
 #pragma unroll
-            for (int j = 0; j < 4; ++j)
-                if (jc + j < NT) ldsm_x4(b[j], sb + av + (8 * (jc + j) + l7) * C::kPitchA + (((4 * qd + mi) ^ asw) << 4));
+            for (int j = 0; j < 2; ++j) ldsm_x4(b[j], sb + av + (8 * (jc + j) + l7) * C::kPitchA + (((4 * qd + mi) ^ asw) << 4));
 #pragma unroll
-            for (int j = 0; j < 4; ++j)
-                if (jc + j < NT) mma16816(wt[j], T0[2 * qd], 0u, T1[2 * qd], 0u, b[j][0], b[j][1]);
+            for (int j = 0; j < 2; ++j) mma16816(wt[j], T0[2 * qd], 0u, T1[2 * qd], 0u, b[j][0], b[j][1]);
 #pragma unroll
-            for (int j = 0; j < 4; ++j)
-                if (jc + j < NT) mma16816(wt[j], T0[2 * qd + 1], 0u, T1[2 * qd + 1], 0u, b[j][2], b[j][3]);
+            for (int j = 0; j < 2; ++j) mma16816(wt[j], T0[2 * qd + 1], 0u, T1[2 * qd + 1], 0u, b[j][2], b[j][3]);
         }
 #pragma unroll
-        for (int j = 0; j < 4; ++j)
-            if (jc + j < NT) { wacc[jc + j < NT ? jc + j : 0][0] = wt[j][0]; wacc[jc + j < NT ? jc + j : 0][1] = wt[j][1]; }
+        for (int j = 0; j < 2; ++j) { wacc[jc + j][0] = wt[j][0]; wacc[jc + j][1] = wt[j][1]; }
     }
 }
 
