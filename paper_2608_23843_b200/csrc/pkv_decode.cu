@@ -970,6 +970,13 @@ __device__ __forceinline__ void merge_parts(const DecodeArgs &a, const float *fi
     }
 }
 
+// One ticket of a counter in global memory, with release and acquire semantics at device scope.
+__device__ __forceinline__ int draw_ticket(int *counter) {
+    int old;
+    asm volatile("atom.acq_rel.gpu.global.add.s32 %0, [%1], 1;" : "=r"(old) : "l"(counter) : "memory");
+    return old;
+}
+
 #define PKV_CONSUMER_BARRIER() asm volatile("bar.sync 1, %0;" ::"n"(kConsumerWarps * 32) : "memory")
 
 // All consumer warps combine their states of one segment (Eq. 5 inside the CTA).  If the segment
@@ -1033,9 +1040,10 @@ __device__ __forceinline__ void flush_segment(const DecodeArgs &a, float *comb, 
         }
     }
     if (ps.n_parts > 1) {
-        // Drawing a ticket: the barrier orders every thread's stores of the state before thread 0's fence, which
-        // makes them visible device-wide before the ticket is drawn; on the way back thread 0's second fence and the
-        // barrier order the other CTAs' states (whose tickets this one has seen) before every thread's reads of them.
+        // Drawing a ticket: the barrier orders every thread's stores of the state before thread 0's atomic, whose
+        // release half makes them visible device-wide before the ticket is drawn; on the way back its acquire half
+        // and the barrier order the other CTAs' states (whose tickets this one has seen) before every thread's reads
+        // of them (the pattern of a cooperative grid sync, with the two fences folded into the atomic).
         // A segment held by more than kMergeFan CTAs is summed in two levels: the CTAs form groups of kMergeFan
         // consecutive ranges; the last of a group to arrive sums the group's states into a group state, and the last
         // group to arrive sums the group states.  The slowest CTA of the launch then has one short sum of its
@@ -1049,11 +1057,7 @@ __device__ __forceinline__ void flush_segment(const DecodeArgs &a, float *comb, 
             const int gsize = min(kMergeFan, ps.n_parts - g * kMergeFan);
             const int gslot0 = (ps.cta_first + seg) / kMergeFan + seg;     // group slots of consecutive groups and segments never collide
             PKV_CONSUMER_BARRIER();
-            if (ctid == 0) {
-                __threadfence();
-                *last_flag = (atomicAdd(a.gtickets + gslot0 + g, 1) == gsize - 1);
-                __threadfence();
-            }
+            if (ctid == 0) *last_flag = (draw_ticket(a.gtickets + gslot0 + g) == gsize - 1);
             PKV_CONSUMER_BARRIER();
             mine = *last_flag != 0;
             if (mine) {
@@ -1068,11 +1072,7 @@ __device__ __forceinline__ void flush_segment(const DecodeArgs &a, float *comb, 
         }
         if (mine) {
             PKV_CONSUMER_BARRIER();
-            if (ctid == 0) {
-                __threadfence();
-                *last_flag = (atomicAdd(a.tickets + qseg, 1) == np - 1);
-                __threadfence();
-            }
+            if (ctid == 0) *last_flag = (draw_ticket(a.tickets + qseg) == np - 1);
             PKV_CONSUMER_BARRIER();
             if (trace && ctid == 0) trace[10] = clock64();
             if (*last_flag) {
