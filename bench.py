@@ -560,8 +560,8 @@ def main():
                     help="strong scaling of one step: every rank's cache holds 1/N of each sequence's tokens (rank 0 the "
                          "sink, the last rank the dense window); per layer each rank computes its softmax state, the states "
                          "are all-gathered (NCCL) and merged by Eq. 5.  Not the default: the driver's scaling runs are replicas")
-    ap.add_argument("--decode-variant", type=int, default=0, choices=[0, 2],
-                    help="2 = pkv_decode_attention_multi never uses its row-block kernel (comparisons)")
+    ap.add_argument("--decode-variant", type=int, default=0, choices=[0, 2, 3],
+                    help="2 = pkv_decode_attention_multi never uses its row-block kernels; 3 = its row-block kernel is the mma.sync one (comparisons)")
     ap.add_argument("--graph", action="store_true",
                     help="replay one CUDA graph per step instead of launching every layer from the host")
     args = ap.parse_args()
@@ -777,7 +777,7 @@ def main():
                                   "gpu_launches": lps * args.steps}
         P_, Gq = w.get("page", 64), Hq // w["n_kv_heads"]
         rows = QL * Gq
-        if QL > 1 and args.decode_variant == 0 and args.factor_bits != 4 and rows >= 64 and w["batch"] * w["n_kv_heads"] * -(-rows // 64) >= 128:
+        if QL > 1 and args.decode_variant in (0, 3) and args.factor_bits != 4 and rows >= 64 and w["batch"] * w["n_kv_heads"] * -(-rows // 64) >= 128:
             # Served by the row-block kernel, whose bound is the tensor pipe, not HBM: algorithmic FLOPs per launch =
             # query rows x (factor pages x 2 (d r_k + r_k P + P r_v + r_v d) + dense tokens x 4 d); the causal
             # triangle among the new positions is counted in full.

@@ -93,7 +93,8 @@ typedef struct pkv_config {
     int32_t n_ctas;             /* decode grid size; 0 => SM count of the current device (148 in dry-run), doubled unless decode_overlap */
     int32_t decode_variant;     /* 0 = tensor-core kernels (the product path); 1 = scalar fp32 kernel that evaluates
                                    the same equations one unit at a time, kept as a debugging reference; 2 = as 0 but
-                                   pkv_decode_attention_multi never uses its row-block kernel (for comparisons) */
+                                   pkv_decode_attention_multi never uses its row-block kernels; 3 = as 0 but the
+                                   row-block kernel is the mma.sync one for every shape (2, 3: for comparisons) */
     float   jacobi_energy_tol;  /* the sweeps also stop once the energy captured by the r largest diagonal entries
                                    (= ||A^T X||_F^2 of the factors they would give) has grown, since the previous
                                    check, by less than this fraction of the energy left outside them (= the squared

@@ -82,6 +82,7 @@ struct pkv_cache {
     bool dry = false;
     bool trace = false;                // PKV_DECODE_TRACE=1: CTAs write time stamps into the workspace
     unsigned char *dense_pool = nullptr, *factor_pool = nullptr, *meta = nullptr, *workspace = nullptr;
+    RowBlockMaps row_maps = {};        // TMA descriptors of the pools (tcgen05 row-block kernel)
     FreeList dense_free, factor_free;
     std::vector<SeqLayer> sl;          // [max_seqs * n_layers]
     std::vector<PlanCache> plans;      // [n_layers]
@@ -149,7 +150,7 @@ pkv_status validate(const pkv_config *cfg, const char **why) {
         *why = "sink_tokens and recent_tokens must be non-negative multiples of page_size"; return PKV_ERR_INVALID_ARG;
     }
     if (cfg->softmax_scale < 0.f || cfg->jacobi_max_sweeps < 0 || cfg->jacobi_tol < 0.f || cfg->n_ctas < 0 ||
-        cfg->decode_variant < 0 || cfg->decode_variant > 2 ||
+        cfg->decode_variant < 0 || cfg->decode_variant > 3 ||
         cfg->decode_overlap < 0 || cfg->decode_overlap > 2 ||
         (cfg->factor_bits != 0 && cfg->factor_bits != 4 && cfg->factor_bits != 16)) {
         *why = "negative scale / sweep cap / tolerance / n_ctas, or unknown decode_variant / decode_overlap / factor_bits"; return PKV_ERR_INVALID_ARG;
@@ -395,7 +396,7 @@ int block_slots_per_seq(const Geometry &g, int q_len) { return passes_per_seq(g,
 // pipeline kernel is used if its plan entries fit.
 bool uses_row_blocks(const pkv_cache *c, int q_len, int n_seqs) {
     const long long rows = (long long)q_len * c->geo.group;
-    if (q_len <= 1 || c->cfg.decode_variant != 0 || c->geo.factor_bits == 4 || rows < kRowBlock) return false;
+    if (q_len <= 1 || (c->cfg.decode_variant != 0 && c->cfg.decode_variant != 3) || c->geo.factor_bits == 4 || rows < kRowBlock) return false;
     const long long n_ctas = (long long)n_seqs * c->geo.n_kv_heads * ((rows + kRowBlock - 1) / kRowBlock);
     return n_ctas >= 128 || (long long)n_seqs * block_slots_per_seq(c->geo, q_len) > c->cfg.max_seqs;
 }
@@ -588,6 +589,7 @@ pkv_status pkv_init_cache(const pkv_config *cfg, void *dense_pool, void *factor_
         cudaError_t e = cudaMemset(c->meta, 0, (size_t)c->ml.total);
         if (e == cudaSuccess) e = cudaMemset(c->workspace, 0, (size_t)c->wl.total);
         if (e == cudaSuccess) e = decode_kernel_setup();
+        if (e == cudaSuccess) row_block_make_maps(c->geo, c->factor_pool, c->dense_pool, &c->row_maps);
         if (e == cudaSuccess) e = cudaDeviceSynchronize();
         if (e != cudaSuccess || stager_init(c) != PKV_OK) { delete c; return PKV_ERR_CUDA; }
     }
@@ -1060,9 +1062,9 @@ static pkv_status decode_impl(pkv_cache *c, int32_t layer, int32_t n_seqs, const
         a.partials = nullptr; a.tickets = nullptr; a.gpartials = nullptr; a.gtickets = nullptr;
         a.status = (int *)(c->meta + c->ml.status);
         a.layer = layer;
-        a.variant = 0; a.overlap = 0; a.plain_launch = 1; a.trace = nullptr;
+        a.variant = c->cfg.decode_variant == 3 ? 3 : 0; a.overlap = 0; a.plain_launch = 1; a.trace = nullptr;
         c->cache_written = false;
-        PKV_CUDA(c, launch_decode_blocks(a, n_seqs, st));
+        PKV_CUDA(c, launch_decode_blocks(a, n_seqs, c->row_maps, st));
         return PKV_OK;
     }
     if (static_scratch) {

@@ -18,6 +18,7 @@
 // reference (decode_variant = 1).
 #include <cuda_bf16.h>
 
+#include "pkv_device.cuh"
 #include "pkv_internal.h"
 
 // Scratch of pkv_decode_attention_static_scratch(): split-K partial states followed by the merge
@@ -33,37 +34,11 @@ namespace pkv {
 
 namespace {
 
-constexpr float kNegInf = -1e30f;      // finite stand-in for -inf: exp2(kNegInf - x) == 0, no NaN from inf - inf
-constexpr float kMasked = -2e30f;      // score of a token a query must not see: exp2(kMasked - m) == 0 even while m == kNegInf
-constexpr int kKindDense = 0, kKindFactor = 1, kKindEnd = 2;
-// Global SVD form: a region's shared basis travels through the ring like a page, once per consumer warp
-constexpr int kKindBasisK = 3, kKindBasisV = 4;
-
 struct Range {
     PlanCta start, end;
     PlanEntry first_entry;             // the entry `start` lies in
     int n_used, seg_first, n_local_segs;
 };
-
-struct HeadUnits { int d0, nf, units, fb, fe; };
-
-__device__ __forceinline__ HeadUnits head_units(const Geometry &g, const PlanEntry &e) {
-    HeadUnits h;
-    h.fb = min(e.f_begin, e.n_pages);
-    h.fe = min(max(e.f_end, h.fb), e.n_pages);
-    h.d0 = h.fb * g.blocks_per_page;
-    h.nf = h.fe - h.fb;
-    h.units = h.d0 + h.nf + (e.n_pages - h.fe) * g.blocks_per_page;
-    return h;
-}
-
-// unit index within an (entry, head) run -> logical page, block inside the page, kind
-__device__ __forceinline__ void unit_to_page(const Geometry &g, const HeadUnits &h, int u, int &page, int &blk,
-                                             int &kind) {
-    if (u < h.d0) { page = u / g.blocks_per_page; blk = u % g.blocks_per_page; kind = kKindDense; }
-    else if (u < h.d0 + h.nf) { page = h.fb + (u - h.d0); blk = 0; kind = kKindFactor; }
-    else { int v = u - h.d0 - h.nf; page = h.fe + v / g.blocks_per_page; blk = v % g.blocks_per_page; kind = kKindDense; }
-}
 
 __device__ __forceinline__ bool load_range(const DecodeArgs &a, Range &r) {
     // All four loads are issued together (the arrays have an element for every CTA of the grid, used or not), so
@@ -251,37 +226,6 @@ __global__ void __launch_bounds__(256) merge_kernel(const __grid_constant__ Deco
 // =============================================================================
 // Tensor-core pipeline kernel.
 // =============================================================================
-__device__ __forceinline__ uint32_t smem_u32(const void *p) { return (uint32_t)__cvta_generic_to_shared(p); }
-
-__device__ __forceinline__ void mbar_init(uint32_t bar, uint32_t count) {
-    asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(bar), "r"(count));
-}
-__device__ __forceinline__ void mbar_arrive(uint32_t bar) {
-    asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(bar) : "memory");
-}
-__device__ __forceinline__ void mbar_arrive_expect_tx(uint32_t bar, uint32_t bytes) {
-    asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(bytes) : "memory");
-}
-__device__ __forceinline__ bool mbar_try_wait(uint32_t bar, uint32_t parity) {
-    uint32_t ok;
-    asm volatile(
-        "{\n\t.reg .pred p;\n\t"
-        "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
-        "selp.u32 %0, 1, 0, p;\n\t}"
-        : "=r"(ok) : "r"(bar), "r"(parity) : "memory");
-    return ok != 0;
-}
-// Bounded wait: gives up after `limit` clocks (kWaitClocks, about a second, unless a test shortened it) and reports
-// failure.
-constexpr long long kWaitClocks = 2000000000LL;
-__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, long long limit = kWaitClocks) {
-    if (mbar_try_wait(bar, parity)) return true;
-    const long long t0 = clock64();
-    while (!mbar_try_wait(bar, parity)) {
-        if (clock64() - t0 > limit) return false;
-    }
-    return true;
-}
 __device__ __forceinline__ int ld_acquire_smem(const volatile int *p) {
     int v;
     asm volatile("ld.acquire.cta.shared.b32 %0, [%1];" : "=r"(v) : "r"(smem_u32(const_cast<const int *>(p))) : "memory");
@@ -299,20 +243,6 @@ __device__ __forceinline__ bool wait_armed(volatile int *tag, int k, long long l
         __nanosleep(20);
     }
     return true;
-}
-// Pages are read once per launch: ask L2 to drop them first, so that the plan, the queries and the split-K partial
-// states stay resident.
-__device__ __forceinline__ void bulk_g2s(uint32_t dst, const void *src, uint32_t bytes, uint32_t bar) {
-    unsigned long long policy;
-    asm volatile("createpolicy.fractional.L2::evict_first.b64 %0, 1.0;" : "=l"(policy));
-    asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes.L2::cache_hint [%0], [%1], %2, [%3], %4;"
-                 ::"r"(dst), "l"(src), "r"(bytes), "r"(bar), "l"(policy) : "memory");
-}
-// The row-block kernel reads a sequence's pages once per block of 64 query rows: there the copies leave the
-// lines in L2 for the other blocks.
-__device__ __forceinline__ void bulk_g2s_keep(uint32_t dst, const void *src, uint32_t bytes, uint32_t bar) {
-    asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];"
-                 ::"r"(dst), "l"(src), "r"(bytes), "r"(bar) : "memory");
 }
 __device__ __forceinline__ void ldsm_x4(uint32_t (&r)[4], uint32_t addr) {
     asm volatile("ldmatrix.sync.aligned.m8n8.x4.shared.b16 {%0,%1,%2,%3}, [%4];"
@@ -343,30 +273,11 @@ __device__ __forceinline__ uint32_t movm_t(uint32_t x) {
     asm volatile("movmatrix.sync.aligned.m8n8.trans.b16 %0, %1;" : "=r"(y) : "r"(x));
     return y;
 }
-// two floats -> packed bf16x2 (lo in the low half), round to nearest even
-__device__ __forceinline__ uint32_t pack_bf16(float lo, float hi) {
-    uint32_t r;
-    asm("cvt.rn.bf16x2.f32 %0, %1, %2;" : "=r"(r) : "f"(hi), "f"(lo));
-    return r;
-}
-__device__ __forceinline__ float bf16lo_f(uint32_t x) { return __uint_as_float(x << 16); }
-__device__ __forceinline__ float bf16hi_f(uint32_t x) { return __uint_as_float(x & 0xffff0000u); }
-
-struct StageDesc { int kind, rows, seg, after; };
-
 // Per-warp running state for the query heads 2t, 2t+1 (t = lane & 3) of one KV head.
 struct WarpState {
     float o[8][4];        // o[i]: (d = 16i+g, heads 2t,2t+1), (d = 16i+8+g, heads 2t,2t+1);  g = lane >> 2
     float m[2], l[2];     // l is this lane's share; summed over g at flush time
 };
-
-// Shapes fixed at compile time: P tokens per page, NT = ceil(rank / 8) rank tiles (K and V alike), I4 = factors
-// stored as INT4 codes.
-// rows per dense block: 32 where a stage has to be that large for a bf16 factor page anyway
-// F = storage form of the factors: 0 = bf16 page-wise (Eq. 2), 1 = INT4 page-wise (Section 4.3), 2 = Global SVD form
-// (Section 4.2: pages hold A rows only, the basis is shared by the region)
-template <int P, int NT, int F>
-constexpr int kDenseBlock = (F != 1 && P >= 32 && NT >= 3) ? 32 : 16;
 
 template <int P, int NT>
 struct Tc {
@@ -1860,7 +1771,7 @@ cudaError_t decode_kernel_setup() {
     if ((e = cudaFuncSetAttribute(decode_tc_kernel<P, NT, 2>, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBudget / 2)) != cudaSuccess) return e;
     PKV_FOR_EACH_GLOBAL_SHAPE(PKV_SETUP_G)
 #undef PKV_SETUP_G
-    return cudaSuccess;
+    return row_block_umma_setup();
 }
 
 cudaError_t launch_decode(const DecodeArgs &a, int n_segs, cudaStream_t st) {
@@ -1885,8 +1796,11 @@ cudaError_t launch_decode(const DecodeArgs &a, int n_segs, cudaStream_t st) {
     return cudaGetLastError();
 }
 
-// Row-block kernel: one CTA per (sequence, KV head, block of 64 query rows); bf16 factors only.
-cudaError_t launch_decode_blocks(const DecodeArgs &a, int n_seqs, cudaStream_t st) {
+// Row-block kernels; bf16 factors only.  Shapes the tcgen05 kernel covers go to it (one CTA per 128 query rows of a
+// (sequence, KV head)) unless the caller pinned the mma.sync kernel (decode_variant 3); the rest to the latter (one
+// CTA per 64 rows).
+cudaError_t launch_decode_blocks(const DecodeArgs &a, int n_seqs, const RowBlockMaps &maps, cudaStream_t st) {
+    if (a.variant != 3 && maps.valid) return launch_decode_blocks_umma(a, n_seqs, maps, st);
     const int n_blk = (a.q_len * a.geo.group + kBlockRows - 1) / kBlockRows;
     const long long n_ctas = (long long)n_seqs * a.geo.n_kv_heads * n_blk;
     if (a.geo.factor_bits == 4 || n_ctas <= 0 || n_ctas > 0x7fffffffLL) return cudaErrorInvalidValue;

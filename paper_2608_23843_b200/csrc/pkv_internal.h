@@ -1,6 +1,7 @@
 // Internal declarations shared by the host cache manager and the CUDA kernels.
 #pragma once
 
+#include <cuda.h>            // CUtensorMap (the type only: no driver call is linked)
 #include <cuda_runtime.h>
 #include <stdint.h>
 
@@ -140,8 +141,16 @@ cudaError_t launch_append(const Geometry &geo, unsigned char *dense_pool, const 
 cudaError_t launch_compress(const Geometry &geo, const unsigned char *dense_pool, unsigned char *factor_pool,
                             const int2 *worklist, int n_entries, int *status, cudaStream_t st);
 cudaError_t launch_decode(const DecodeArgs &a, int n_segs, cudaStream_t st);
-cudaError_t launch_decode_blocks(const DecodeArgs &a, int n_seqs, cudaStream_t st);
-constexpr int kRowBlock = 64;          // query rows (token x query head) per CTA of the row-block kernel
+constexpr int kRowBlock = 64;          // query rows (token x query head) per CTA of the mma.sync row-block kernel
+// tcgen05 row-block kernel (pkv_rowblock.cu): 128 query rows per CTA; P = 64, bf16 page-wise factors, rank_k a multiple of 8
+bool row_block_umma_supported(const Geometry &geo);
+cudaError_t row_block_umma_setup();
+// TMA descriptors of the pools for that kernel (B factors; dense K / V); valid = 0 where the shape is not covered or
+// the driver offers no encoder, and the mma.sync kernel is used instead
+struct RowBlockMaps { CUtensorMap bk, bv, dense; int valid; };
+void row_block_make_maps(const Geometry &geo, const void *factor_pool, const void *dense_pool, RowBlockMaps *maps);
+cudaError_t launch_decode_blocks_umma(const DecodeArgs &a, int n_seqs, const RowBlockMaps &maps, cudaStream_t st);
+cudaError_t launch_decode_blocks(const DecodeArgs &a, int n_seqs, const RowBlockMaps &maps, cudaStream_t st);
 cudaError_t launch_merge_states(const float *states, int n_shards, long long n_rows, void *out, float *out_f32,
                                 cudaStream_t st);
 cudaError_t launch_decode_static_scratch(const DecodeArgs &a, int n_segs, cudaStream_t st, const char **why);

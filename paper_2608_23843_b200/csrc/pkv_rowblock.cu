@@ -1,0 +1,619 @@
+// Row-block attention on the fifth-generation tensor cores (tcgen05.mma, accumulators and row operands in tensor
+// memory).
+//
+// Same job as the mma.sync row-block kernel of pkv_decode.cu — many queries per sequence (a chunk of a prefill), one
+// CTA per (sequence, KV head, block of query rows), Eq. 4 for factor pages and plain attention for dense ones, the
+// pages in token order so that no split-K state is left to merge — but with 128 query rows per CTA as the M
+// dimension of every product:
+//     G1: q~ [128 x r] = Q [128 x d] . B_k^T        G2: s [128 x P] = (q~_hi + q~_lo) . A_k^T
+//     G3: w  [128 x r] = p [128 x P] . A_v          G4: o [128 x d] += w . B_v
+//     dense pages:  Ga: s = Q . K^T                 Gb: o += p . V
+// One thread owns one query row (= one lane of tensor memory): it reads its row of q~, s, w back from tensor memory,
+// does the scaling, the two-term bf16 split, the masking and the online softmax alone (no shuffles), and writes the
+// row of the next product's A operand over the columns it has just read (tcgen05.mma takes A from tensor memory).
+// A^T factors are used where the bulk copy put them: the storage swizzle of a 128-byte A^T row is the tensor core's
+// 128-byte swizzle (A_k^T as an MN-major B operand, A_v^T as a K-major one).  Rows of 256 bytes (B factors, dense
+// K / V) are split by the row threads into two panels of 128-byte rows first, which is the same swizzle again.
+//
+// Warps 0-3: the 128 query rows.  Warp 4, one lane: bulk copies into the ring.  Warp 5, one lane: issues every
+// tcgen05.mma.  Rows -> issuer: an mbarrier all 128 row threads arrive on; issuer -> rows: tcgen05.commit on a second
+// mbarrier.  The four products of a factor page depend on one another through the row threads, so consecutive units
+// are skewed: a unit costs two exchanges, each carrying one product of the unit and one of the next,
+//     exchange 1 of unit u:  rows: softmax of s(u), panels V(u) and K(u+1)   then issuer: G3(u) | Gb(u), G1(u+1)
+//     exchange 2 of unit u:  rows: w(u) and q~(u+1) to bf16                  then issuer: G4(u), G2(u+1) | Ga(u+1)
+// and two CTAs per SM overlap one another's chains.  Every wait is bounded; tensor memory is released on every path
+// out.
+#include <cstdio>
+
+#include "pkv_device.cuh"
+
+namespace pkv {
+
+namespace {
+
+constexpr int kURows = 128;
+constexpr int kUThreads = 192;
+constexpr int kUQBytes = 2 * kURows * 128;       // Q: two panels [128 rows][64 channels], 128-byte swizzle
+constexpr uint32_t kColQt = 0, kColS = 32, kColW = 96, kColO = 128, kTmemCols = 256;
+
+// A stage holds one unit the way the products read it, RB = 16 or 32 rows of 128 bytes per part:
+//     [A_k^T][K side, channels 0-63][K side, channels 64-127][A_v^T][V side, channels 0-63][V side, channels 64-127]
+// K side = B_k or a block of dense K, V side = B_v or a block of dense V.  The sides are written by tiled TMA
+// copies (box = 64 channels x rows) straight from the pools' 256-byte rows: 16-byte chunk c of row j is stored at
+// chunk c ^ (j & 7), so each half of a row is a 128-byte row in the tensor core's 128-byte swizzle.
+__host__ __device__ inline int umma_part_rows(const Geometry &g) { return g.rank_tiles <= 2 ? 16 : 32; }
+__host__ __device__ inline int umma_stage_bytes(const Geometry &g) { return 6 * umma_part_rows(g) * 128; }
+// stages: the units u and u + 1 are in use at any time; the rest is the copies' lead
+__host__ __device__ inline int umma_stages(const Geometry &g) {
+    const int room = 113 * 1024 - kUQBytes - 512;
+    return max(3, min(6, room / umma_stage_bytes(g)));
+}
+
+// ---- tcgen05 wrappers --------------------------------------------------------------------------------------
+// Shared-memory matrix descriptor: start address, leading / stride byte offsets (all in 16-byte units), descriptor
+// version 1, layout 0 = no swizzle, 2 = 128-byte swizzle.
+__device__ __forceinline__ uint64_t umma_desc(uint32_t saddr, uint32_t lbo, uint32_t sbo, uint32_t layout) {
+    return (uint64_t)((saddr >> 4) & 0x3FFF) | (uint64_t)((lbo >> 4) & 0x3FFF) << 16 | (uint64_t)((sbo >> 4) & 0x3FFF) << 32 |
+           (uint64_t)1 << 46 | (uint64_t)layout << 61;
+}
+// Instruction descriptor: bf16 x bf16 -> fp32, M x N, B operand K-major (0) or MN-major (1); A always K-major.
+__host__ __device__ constexpr uint32_t umma_idesc(int M, int N, int b_mn_major) {
+    return (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)b_mn_major << 16) | ((uint32_t)(N >> 3) << 17) | ((uint32_t)(M >> 4) << 24);
+}
+// d (+)= a . b with a in shared memory / in tensor memory (row = lane, two bf16 per 32-bit column, 8 columns per
+// step of 16 along the contraction)
+__device__ __forceinline__ void umma_ss(uint32_t d_tmem, uint64_t adesc, uint64_t bdesc, uint32_t idesc, uint32_t accumulate) {
+    asm volatile("{\n\t.reg .pred p;\n\tsetp.ne.b32 p, %4, 0;\n\ttcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n\t}"
+                 ::"r"(d_tmem), "l"(adesc), "l"(bdesc), "r"(idesc), "r"(accumulate) : "memory");
+}
+__device__ __forceinline__ void umma_ts(uint32_t d_tmem, uint32_t a_tmem, uint64_t bdesc, uint32_t idesc, uint32_t accumulate) {
+    asm volatile("{\n\t.reg .pred p;\n\tsetp.ne.b32 p, %4, 0;\n\ttcgen05.mma.cta_group::1.kind::f16 [%0], [%1], %2, %3, p;\n\t}"
+                 ::"r"(d_tmem), "r"(a_tmem), "l"(bdesc), "r"(idesc), "r"(accumulate) : "memory");
+}
+__device__ __forceinline__ void umma_commit(uint32_t bar) {
+    asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(bar) : "memory");
+}
+__device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
+__device__ __forceinline__ void tc_fence_after() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
+__device__ __forceinline__ void fence_async_smem() { asm volatile("fence.proxy.async.shared::cta;" ::: "memory"); }
+// Tiled copy of one box (64 channels x the map's rows) starting at channel x of pool row y; completes on `bar`.
+__device__ __forceinline__ void tma_box(uint32_t dst, const CUtensorMap *map, int x, int y, uint32_t bar) {
+    asm volatile("cp.async.bulk.tensor.2d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3}], [%4];"
+                 ::"r"(dst), "l"(map), "r"(x), "r"(y), "r"(bar) : "memory");
+}
+
+#define PKV_R8(r, o) "=r"(r[o]), "=r"(r[o + 1]), "=r"(r[o + 2]), "=r"(r[o + 3]), "=r"(r[o + 4]), "=r"(r[o + 5]), "=r"(r[o + 6]), "=r"(r[o + 7])
+#define PKV_W8(r, o) "r"(r[o]), "r"(r[o + 1]), "r"(r[o + 2]), "r"(r[o + 3]), "r"(r[o + 4]), "r"(r[o + 5]), "r"(r[o + 6]), "r"(r[o + 7])
+// consecutive 32-bit columns of this thread's lane
+__device__ __forceinline__ void tmem_ld32(uint32_t taddr, uint32_t *r) {
+    asm volatile("tcgen05.ld.sync.aligned.32x32b.x32.b32 {%0,%1,%2,%3,%4,%5,%6,%7,%8,%9,%10,%11,%12,%13,%14,%15,"
+                 "%16,%17,%18,%19,%20,%21,%22,%23,%24,%25,%26,%27,%28,%29,%30,%31}, [%32];"
+                 : PKV_R8(r, 0), PKV_R8(r, 8), PKV_R8(r, 16), PKV_R8(r, 24) : "r"(taddr));
+}
+__device__ __forceinline__ void tmem_ld16(uint32_t taddr, uint32_t *r) {
+    asm volatile("tcgen05.ld.sync.aligned.32x32b.x16.b32 {%0,%1,%2,%3,%4,%5,%6,%7,%8,%9,%10,%11,%12,%13,%14,%15}, [%16];"
+                 : PKV_R8(r, 0), PKV_R8(r, 8) : "r"(taddr));
+}
+__device__ __forceinline__ void tmem_ld_wait() { asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory"); }
+__device__ __forceinline__ void tmem_st32(uint32_t taddr, const uint32_t *r) {
+    asm volatile("tcgen05.st.sync.aligned.32x32b.x32.b32 [%0], {%1,%2,%3,%4,%5,%6,%7,%8,%9,%10,%11,%12,%13,%14,%15,%16,"
+                 "%17,%18,%19,%20,%21,%22,%23,%24,%25,%26,%27,%28,%29,%30,%31,%32};"
+                 ::"r"(taddr), PKV_W8(r, 0), PKV_W8(r, 8), PKV_W8(r, 16), PKV_W8(r, 24) : "memory");
+}
+__device__ __forceinline__ void tmem_st16(uint32_t taddr, const uint32_t *r) {
+    asm volatile("tcgen05.st.sync.aligned.32x32b.x16.b32 [%0], {%1,%2,%3,%4,%5,%6,%7,%8,%9,%10,%11,%12,%13,%14,%15,%16};"
+                 ::"r"(taddr), PKV_W8(r, 0), PKV_W8(r, 8) : "memory");
+}
+__device__ __forceinline__ void tmem_st8(uint32_t taddr, const uint32_t *r) {
+    asm volatile("tcgen05.st.sync.aligned.32x32b.x8.b32 [%0], {%1,%2,%3,%4,%5,%6,%7,%8};" ::"r"(taddr), PKV_W8(r, 0) : "memory");
+}
+__device__ __forceinline__ void tmem_st_wait() { asm volatile("tcgen05.wait::st.sync.aligned;" ::: "memory"); }
+template <int N>
+__device__ __forceinline__ void tmem_ld(uint32_t taddr, uint32_t *r) {
+    static_assert(N == 16 || N == 32 || N == 64, "16, 32 or 64 columns");
+    if (N == 16) tmem_ld16(taddr, r);
+    else { tmem_ld32(taddr, r); if (N == 64) tmem_ld32(taddr + 32, r + 32); }
+    tmem_ld_wait();
+}
+template <int N>
+__device__ __forceinline__ void tmem_st(uint32_t taddr, const uint32_t *r) {
+    static_assert(N == 8 || N == 16 || N == 32, "8, 16 or 32 columns");
+    if (N == 8) tmem_st8(taddr, r);
+    else if (N == 16) tmem_st16(taddr, r);
+    else tmem_st32(taddr, r);
+}
+// True in exactly one lane of a converged warp.  The single-lane roles are entered through this rather than through
+// `lane == 0`: the compiler then knows that one lane runs the code, and issues tcgen05.mma (whose operands are
+// warp-uniform registers) directly; behind a plain lane test each issue measured 230 clocks instead of 40.
+__device__ __forceinline__ bool elect_one() {
+    uint32_t leader;
+    asm volatile("{\n\t.reg .pred P;\n\telect.sync _|P, 0xffffffff;\n\tselp.u32 %0, 1, 0, P;\n\t}" : "=r"(leader));
+    return leader != 0;
+}
+// 2^x for x <= 0 (and the large negative stand-ins for -inf, which give 0)
+__device__ __forceinline__ float exp2_fast(float x) {
+    float y;
+    asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
+    return y;
+}
+
+// Bounded waits.  One lane (producer, issuer): gives up when the clock limit passes or another role has given up.
+__device__ __forceinline__ bool wait_lane(uint32_t bar, uint32_t parity, volatile int *abort_flag) {
+    if (mbar_try_wait(bar, parity)) return true;
+    const long long t0 = clock64();
+    while (!mbar_try_wait(bar, parity)) {
+        if (clock64() - t0 > kWaitClocks || *abort_flag) return false;
+    }
+    return true;
+}
+// A whole warp (the row threads run warp-collective tensor-memory loads right after): the outcome is the same for
+// all 32 lanes.
+__device__ __forceinline__ bool wait_warp(uint32_t bar, uint32_t parity, volatile int *abort_flag) {
+    if (__all_sync(0xffffffffu, mbar_try_wait(bar, parity))) return true;
+    const long long t0 = clock64();
+    for (;;) {
+        if (__all_sync(0xffffffffu, mbar_try_wait(bar, parity))) return true;
+        if (__any_sync(0xffffffffu, clock64() - t0 > kWaitClocks || *abort_flag)) return false;
+    }
+}
+
+struct RowSoftmax {
+    float m, l;           // running maximum (log2 units) and sum of this thread's row
+};
+
+// Online softmax of one row over N scores held in sv (already scaled and masked): updates (m, l), rescales o in
+// tensor memory when some row of the warp has a new maximum, and writes p as bf16 pairs over the first N / 2 columns
+// the scores were read from.  o_valid: some product has already written o.
+template <int N>
+__device__ __forceinline__ void softmax_row(float *sv, RowSoftmax &st, bool o_valid, uint32_t t_s, uint32_t t_o) {
+    float mx = sv[0];
+#pragma unroll
+    for (int i = 1; i < N; ++i) mx = fmaxf(mx, sv[i]);
+    const bool grow = mx > st.m;
+    float alpha = 1.f;
+    if (grow) { alpha = exp2_fast(st.m - mx); st.m = mx; st.l *= alpha; }
+    if (o_valid && __any_sync(0xffffffffu, grow)) {
+        uint32_t r[32];
+#pragma unroll 1
+        for (int c = 0; c < 4; ++c) {
+            tmem_ld32(t_o + 32 * c, r);
+            tmem_ld_wait();
+#pragma unroll
+            for (int i = 0; i < 32; ++i) r[i] = __float_as_uint(__uint_as_float(r[i]) * alpha);
+            tmem_st32(t_o + 32 * c, r);
+        }
+    }
+    float sum = 0.f;
+    const float m = st.m;
+    uint32_t pk[N / 2];
+#pragma unroll
+    for (int e = 0; e < N / 2; ++e) {
+        pk[e] = pack_bf16(exp2_fast(sv[2 * e] - m), exp2_fast(sv[2 * e + 1] - m));
+        sum += bf16lo_f(pk[e]) + bf16hi_f(pk[e]);          // l sums the weights as the product sees them
+    }
+    tmem_st<N / 2>(t_s, pk);
+    tmem_st_wait();
+    st.l += sum;
+}
+
+template <int NT>
+__global__ void __launch_bounds__(kUThreads, 2) block_umma_kernel(const __grid_constant__ DecodeArgs a,
+                                                                  const __grid_constant__ CUtensorMap map_bk,
+                                                                  const __grid_constant__ CUtensorMap map_bv,
+                                                                  const __grid_constant__ CUtensorMap map_dense) {
+    constexpr int P = 64, RP = NT <= 2 ? 16 : 32, kDB = kDenseBlock<P, NT, 0>;
+    static_assert(kDB == RP, "dense blocks and padded ranks share the stage layout");
+    constexpr int kPart = RP * 128;                   // bytes of one part of a stage
+    constexpr int oAk = 0, oK = kPart, oAv = 3 * kPart, oV = 4 * kPart;
+    const Geometry &geo = a.geo;
+    const int S = umma_stages(geo), ustage = umma_stage_bytes(geo), H = geo.n_kv_heads, G = geo.group;
+    const int n_rows = a.q_len * G, n_blk = (n_rows + kURows - 1) / kURows;
+    const int rb = blockIdx.x % n_blk, head = (blockIdx.x / n_blk) % H, entry = blockIdx.x / (n_blk * H);
+    const PlanHeader hdr = *reinterpret_cast<const PlanHeader *>(a.plan);
+    if (entry >= hdr.n_seqs) return;
+    extern __shared__ __align__(1024) unsigned char smem[];
+    unsigned char *sq = smem, *stages = smem + kUQBytes;
+    unsigned long long *full_bar = reinterpret_cast<unsigned long long *>(stages + (size_t)S * ustage);
+    unsigned long long *empty_bar = full_bar + S;
+    unsigned long long *c2m_bar = empty_bar + S, *m2c_bar = c2m_bar + 1, *drain_bar = m2c_bar + 1;
+    StageDesc *descs = reinterpret_cast<StageDesc *>(drain_bar + 1);
+    volatile int *abort_flag = reinterpret_cast<volatile int *>(descs + S);
+    uint32_t *tmem_slot = reinterpret_cast<uint32_t *>(const_cast<int *>(abort_flag) + 1);
+    const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+    if (tid == 0) {
+        for (int s = 0; s < S; ++s) { mbar_init(smem_u32(full_bar + s), 1); mbar_init(smem_u32(empty_bar + s), 1); }
+        mbar_init(smem_u32(c2m_bar), kURows);
+        mbar_init(smem_u32(m2c_bar), 1);
+        mbar_init(smem_u32(drain_bar), 1);
+        *abort_flag = 0;
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    }
+    // Rows past the rank are never written by the copies and are multiplied by exact zeros: they must hold finite
+    // values from the start.
+    for (int i = tid; i < S * ustage / 16; i += kUThreads) reinterpret_cast<uint4 *>(stages)[i] = make_uint4(0u, 0u, 0u, 0u);
+    fence_async_smem();
+    if (warp == 0) {
+        asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(tmem_slot)), "r"(kTmemCols) : "memory");
+        asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+    }
+    tc_fence_before();
+    __syncthreads();
+    tc_fence_after();
+    const uint32_t tm = *tmem_slot;
+    const PlanEntry e = reinterpret_cast<const PlanEntry *>(a.plan + a.plan_entry)[entry];
+    const HeadUnits hu = head_units(geo, e);
+    const int T = a.n_tokens[(long long)e.seq * geo.n_layers + a.layer];
+    // Units are in token order and the block's last row sees the most: units that start after what it sees are
+    // hidden from every row of the block and are left out (all roles agree on the count).
+    int n_units = hu.units;
+    {
+        const int last_row = min(n_rows, (rb + 1) * kURows) - 1;
+        const int vis = T - (a.q_len - 1 - last_row / G);                 // tokens the last row sees (>= 1)
+        const int page = (vis - 1) / P, blk = ((vis - 1) % P) / kDB;
+        int need;
+        if (page < hu.fb) need = page * geo.blocks_per_page + blk + 1;
+        else if (page < hu.fe) need = hu.d0 + hu.nf;
+        else need = hu.d0 + hu.nf + (page - hu.fe) * geo.blocks_per_page + blk + 1;
+        n_units = max(1, min(need, hu.units));
+    }
+    const uint32_t c2m = smem_u32(c2m_bar), m2c = smem_u32(m2c_bar);
+
+    if (warp == 4) {
+        // ------------------------------ copies (one lane) ------------------------------
+        if (elect_one()) {
+            const int *pt = a.page_table + ((long long)e.seq * geo.n_layers + a.layer) * geo.max_pages;
+            bool ok = true;
+            int u = 0;
+            for (; u < n_units; ++u) {
+                const int s = u % S;
+                if (u >= S && !wait_lane(smem_u32(empty_bar + s), ((u / S) - 1) & 1, abort_flag)) { ok = false; break; }
+                int page, blk, kind;
+                unit_to_page(geo, hu, u, page, blk, kind);
+                const int slot = pt[page];
+                int rows = 0, after = 0;
+                const bool bad = slot < 0 || slot >= (kind == kKindFactor ? geo.n_factor_slots : geo.n_dense_slots);
+                if (bad) {
+                    atomicAdd(a.status + 2, 1);                  // corrupt page table: an empty unit, and a mark
+                    kind = kKindDense;
+                } else if (kind == kKindFactor) {
+                    rows = P;
+                } else {
+                    rows = max(0, min(kDB, T - page * P - blk * kDB));
+                    after = max(0, T - page * P - blk * kDB - rows);
+                }
+                descs[s] = StageDesc{kind, rows, 0, after};
+                const uint32_t bar = smem_u32(full_bar + s);
+                const uint32_t dst = smem_u32(stages + (size_t)s * ustage);
+                if (kind == kKindFactor) {
+                    const long long off = (long long)slot * geo.factor_slot_bytes + (long long)head * geo.blob_bytes;
+                    const unsigned char *src = a.factor_pool + off;
+                    const int yk = (int)((off + geo.bk_off) >> 8), yv = (int)((off + geo.bv_off) >> 8);     // pool rows of 256 bytes
+                    mbar_arrive_expect_tx(bar, geo.blob_bytes);
+                    bulk_g2s_keep(dst + oAk, src + geo.ak_off, geo.rank_k * 128, bar);
+                    bulk_g2s_keep(dst + oAv, src + geo.av_off, geo.rank_v * 128, bar);
+                    tma_box(dst + oK, &map_bk, 0, yk, bar);
+                    tma_box(dst + oK + kPart, &map_bk, 64, yk, bar);
+                    tma_box(dst + oV, &map_bv, 0, yv, bar);
+                    tma_box(dst + oV + kPart, &map_bv, 64, yv, bar);
+                } else if (rows > 0) {
+                    // whole blocks: rows past the sequence's end hold whatever the pool holds; the scores there are
+                    // masked and the row threads clear those rows of V
+                    const int y = (int)(((long long)slot * geo.dense_slot_bytes + (long long)head * geo.dense_head_bytes) >> 8) + blk * kDB;
+                    mbar_arrive_expect_tx(bar, 4 * kPart);
+                    tma_box(dst + oK, &map_dense, 0, y, bar);
+                    tma_box(dst + oK + kPart, &map_dense, 64, y, bar);
+                    tma_box(dst + oV, &map_dense, 0, y + P, bar);
+                    tma_box(dst + oV + kPart, &map_dense, 64, y + P, bar);
+                } else {
+                    mbar_arrive(bar);
+                }
+            }
+            if (!ok && !*abort_flag) { *abort_flag = 1; atomicAdd(a.status, 1); }
+            // copies already in flight must land before the CTA retires: wait (bounded) for the stages armed last
+            for (int back = 1; back <= min(u, S); ++back) {
+                const int k = u - back;
+                (void)mbar_wait(smem_u32(full_bar + k % S), (k / S) & 1);
+            }
+        }
+    } else if (warp == 5) {
+        // ------------------------------ products (one lane) ------------------------------
+        if (elect_one()) {
+            const uint32_t sq_a = smem_u32(sq);
+            const uint32_t t_qt = tm + kColQt, t_s = tm + kColS, t_w = tm + kColW, t_o = tm + kColO;
+            uint32_t xph = 0;
+            bool ok = true, o_valid = false;
+            // [128 x n] = Q . (K side)^T: 8 steps of 16 channels; both operands K-major, 128-byte swizzle
+            auto qk = [&](uint32_t t_dst, uint32_t sb) {
+                const uint32_t idesc = umma_idesc(128, RP, 0);
+#pragma unroll
+                for (int ks = 0; ks < 8; ++ks)
+                    umma_ss(t_dst, umma_desc(sq_a + (ks >> 2) * (kURows * 128) + (ks & 3) * 32, 16, 1024, 2),
+                            umma_desc(sb + oK + (ks >> 2) * kPart + (ks & 3) * 32, 16, 1024, 2), idesc, ks > 0);
+            };
+            // o [128 x d] (+)= (rows of n bf16 at t_src) . (V side): the V side is MN-major, two panels of 64 channels
+            auto pv = [&](uint32_t t_src, uint32_t sb) {
+#pragma unroll
+                for (int ks = 0; ks < RP / 16; ++ks)
+                    umma_ts(t_o, t_src + ks * 8, umma_desc(sb + oV + ks * 2048, kPart, 1024, 2), umma_idesc(128, 128, 1),
+                            o_valid || ks > 0);
+                o_valid = true;
+            };
+            // s = (q~_hi + q~_lo) . A_k^T, A_k^T in place (MN-major)
+            auto g2 = [&](uint32_t sb) {
+#pragma unroll
+                for (int t = 0; t < 2; ++t)
+#pragma unroll
+                    for (int ks = 0; ks < RP / 16; ++ks)
+                        umma_ts(t_s, t_qt + t * (RP / 2) + ks * 8, umma_desc(sb + oAk + ks * 2048, 16, 1024, 2),
+                                umma_idesc(128, P, 1), (t | ks) > 0);
+            };
+            // kind of a unit as the products see it: units without tokens run as dense units with every score masked
+            auto unit_kind = [&](int u, bool &good) -> int {
+                const int s = u % S;
+                if (!wait_lane(smem_u32(full_bar + s), (u / S) & 1, abort_flag)) { good = false; return kKindDense; }
+                const StageDesc d = descs[s];
+                return d.kind == kKindFactor && d.rows > 0 ? kKindFactor : kKindDense;
+            };
+#ifdef PKV_UMMA_PROFILE
+            long long tw = 0, ti = 0, tx = 0, t0 = clock64(), t1;
+#define PKV_EXCHANGE_BEGIN() if (!wait_lane(c2m, xph, abort_flag)) { ok = false; break; } tc_fence_after(); t1 = clock64(); tw += t1 - t0; t0 = t1;
+#define PKV_EXCHANGE_END() umma_commit(m2c); t1 = clock64(); ti += t1 - t0; t0 = t1; (void)wait_lane(m2c, xph, abort_flag); t1 = clock64(); tx += t1 - t0; t0 = t1; xph ^= 1;
+#else
+#define PKV_EXCHANGE_BEGIN() if (!wait_lane(c2m, xph, abort_flag)) { ok = false; break; } tc_fence_after();
+#define PKV_EXCHANGE_END() umma_commit(m2c); xph ^= 1;
+#endif
+            int kind_cur = kKindDense, kind_nxt = kKindDense;
+            for (int u = -1; u < n_units; ++u) {
+                const uint32_t sb = smem_u32(stages + (size_t)((u + S) % S) * ustage);
+                const uint32_t sb_nxt = smem_u32(stages + (size_t)((u + 1) % S) * ustage);
+                // exchange 1: G3(u) | Gb(u), then G1(u+1)
+                PKV_EXCHANGE_BEGIN()
+                if (u + 1 < n_units) { kind_nxt = unit_kind(u + 1, ok); if (!ok) break; }
+                if (u >= 0) {
+                    if (kind_cur == kKindFactor) {
+#pragma unroll
+                        for (int ks = 0; ks < P / 16; ++ks)      // w = p . A_v, A_v^T in place (K-major)
+                            umma_ts(t_w, t_s + ks * 8, umma_desc(sb + oAv + ks * 32, 16, 1024, 2), umma_idesc(128, RP, 0), ks > 0);
+                    } else {
+                        pv(t_s, sb);
+                        umma_commit(smem_u32(empty_bar + u % S));      // a dense unit's stage is free after Gb
+                    }
+                }
+                if (u + 1 < n_units && kind_nxt == kKindFactor) qk(t_qt, sb_nxt);
+                PKV_EXCHANGE_END()
+                // exchange 2: G4(u), then G2(u+1) | Ga(u+1)
+                PKV_EXCHANGE_BEGIN()
+                if (u >= 0 && kind_cur == kKindFactor) {
+                    pv(t_w, sb);
+                    umma_commit(smem_u32(empty_bar + u % S));          // a factor unit's stage is free after G4
+                }
+                if (u + 1 < n_units) {
+                    if (kind_nxt == kKindFactor) g2(sb_nxt);
+                    else qk(t_s, sb_nxt);
+                }
+                PKV_EXCHANGE_END()
+                kind_cur = kind_nxt;
+            }
+#undef PKV_EXCHANGE_BEGIN
+#undef PKV_EXCHANGE_END
+#ifdef PKV_UMMA_PROFILE
+            if (blockIdx.x == 0 || blockIdx.x == 300)
+                printf("cta %d issuer units %d: wait rows %lld, issue %lld, products %lld (cycles per unit, two exchanges)\n", blockIdx.x, n_units, tw / n_units, ti / n_units, tx / n_units);
+#endif
+            if (!ok && !*abort_flag) { *abort_flag = 1; atomicAdd(a.status, 1); }
+            // nothing of this CTA's may still be running on the tensor cores when tensor memory is given back
+            umma_commit(smem_u32(drain_bar));
+            (void)mbar_wait(smem_u32(drain_bar), 0);
+        }
+    } else {
+        // ------------------------------ rows: one query row per thread ------------------------------
+        const int row = rb * kURows + tid, j = row / G;
+        const bool row_ok = row < n_rows;
+        const long long qrow = ((long long)entry * a.q_len + j) * geo.n_q_heads + head * G + row % G;
+        {
+            const uint4 *qg = reinterpret_cast<const uint4 *>(reinterpret_cast<const __nv_bfloat16 *>(a.q) + qrow * kHeadDim);
+#pragma unroll
+            for (int c = 0; c < 16; ++c) {
+                const uint4 v = row_ok ? __ldg(qg + c) : make_uint4(0u, 0u, 0u, 0u);
+                *reinterpret_cast<uint4 *>(sq + (c >> 3) * (kURows * 128) + tid * 128 + (((c & 7) ^ (tid & 7)) << 4)) = v;
+            }
+            fence_async_smem();          // the products read Q through the async proxy
+        }
+        const int hid = row_ok ? a.q_len - 1 - j : 0;       // newest positions this row must not see
+        const uint32_t t_lane = tm + ((uint32_t)(warp * 32) << 16);
+        const uint32_t t_qt = t_lane + kColQt, t_s = t_lane + kColS, t_w = t_lane + kColW, t_o = t_lane + kColO;
+        RowSoftmax st{kNegInf, 0.f};
+        uint32_t xph = 0;
+        bool ok = true;
+        const float scale = geo.scale_log2e;
+        StageDesc cur{kKindDense, 0, 0, 0}, nxt{kKindDense, 0, 0, 0};
+#ifdef PKV_UMMA_PROFILE
+        long long tp[6] = {0, 0, 0, 0, 0, 0}, tc0 = clock64(), tc1;
+#define PKV_TICK(i) tc1 = clock64(); tp[i] += tc1 - tc0; tc0 = tc1;
+#else
+#define PKV_TICK(i)
+#endif
+#define PKV_HAND_OVER() tc_fence_before(); mbar_arrive(c2m);
+#define PKV_TAKE_BACK() if (!wait_warp(m2c, xph, abort_flag)) { ok = false; break; } xph ^= 1; tc_fence_after();
+        for (int u = -1; u < n_units; ++u) {
+            // ---- before exchange 1: softmax of s(u) ----
+            if (u >= 0) {
+                if (cur.kind == kKindFactor) {
+                    float sv[P];
+                    tmem_ld<P>(t_s, reinterpret_cast<uint32_t *>(sv));
+                    softmax_row<P>(sv, st, u > 0, t_s, t_o);
+                } else {
+                    float sv[kDB];
+                    tmem_ld<kDB>(t_s, reinterpret_cast<uint32_t *>(sv));
+                    const int lim = cur.rows - max(0, hid - cur.after);
+#pragma unroll
+                    for (int i = 0; i < kDB; ++i) sv[i] = i < lim ? sv[i] * scale : kMasked;
+                    softmax_row<kDB>(sv, st, u > 0, t_s, t_o);
+                    if (cur.rows < kDB) {          // V rows past the sequence's end: p is 0 there, the rows must be finite
+                        unsigned char *v = stages + (size_t)(u % S) * ustage + oV;
+                        for (int i = tid; i < (kDB - cur.rows) * 16; i += kURows)
+                            *reinterpret_cast<uint4 *>(v + (i & 1) * kPart + (cur.rows + (i >> 4)) * 128 + ((i >> 1) & 7) * 16) = make_uint4(0u, 0u, 0u, 0u);
+                        fence_async_smem();
+                    }
+                }
+            }
+            PKV_TICK(0)
+            if (u + 1 < n_units) {
+                const int s = (u + 1) % S;
+                if (!wait_warp(smem_u32(full_bar + s), ((u + 1) / S) & 1, abort_flag)) { ok = false; break; }
+                PKV_TICK(1)
+                nxt = descs[s];
+                if (nxt.rows <= 0 || nxt.kind != kKindFactor) { nxt.kind = kKindDense; nxt.rows = max(0, min(nxt.rows, kDB)); }
+            }
+            PKV_TICK(2)
+            PKV_HAND_OVER()
+            PKV_TAKE_BACK()
+            PKV_TICK(3)
+            // ---- before exchange 2: w(u) and q~(u+1) as bf16 rows ----
+            if (u >= 0 && cur.kind == kKindFactor) {       // w: columns past the rank are exact zeros
+                uint32_t r[RP], pk[RP / 2];
+                tmem_ld<RP>(t_w, r);
+#pragma unroll
+                for (int k = 0; k < RP / 2; ++k)
+                    pk[k] = pack_bf16(2 * k < geo.rank_v ? __uint_as_float(r[2 * k]) : 0.f, 2 * k + 1 < geo.rank_v ? __uint_as_float(r[2 * k + 1]) : 0.f);
+                tmem_st<RP / 2>(t_w, pk);
+            }
+            if (u + 1 < n_units && nxt.kind == kKindFactor) {   // q~: scaled, two bf16 terms, columns past the rank exact zeros
+                uint32_t r[RP], hi[RP / 2], lo[RP / 2];
+                tmem_ld<RP>(t_qt, r);
+#pragma unroll
+                for (int k = 0; k < RP / 2; ++k) {
+                    const float x0 = 2 * k < geo.rank_k ? __uint_as_float(r[2 * k]) * scale : 0.f;
+                    const float x1 = 2 * k + 1 < geo.rank_k ? __uint_as_float(r[2 * k + 1]) * scale : 0.f;
+                    hi[k] = pack_bf16(x0, x1);
+                    lo[k] = pack_bf16(x0 - bf16lo_f(hi[k]), x1 - bf16hi_f(hi[k]));
+                }
+                tmem_st<RP / 2>(t_qt, hi);
+                tmem_st<RP / 2>(t_qt + RP / 2, lo);
+            }
+            tmem_st_wait();
+            PKV_TICK(4)
+            PKV_HAND_OVER()
+            PKV_TAKE_BACK()
+            PKV_TICK(5)
+            cur = nxt;
+        }
+#ifdef PKV_UMMA_PROFILE
+        if ((blockIdx.x == 0 || blockIdx.x == 300) && (tid == 0 || tid == 64))
+            printf("cta %d tid %d units %d: softmax+Vpanel %lld, wait full %lld, Kpanel %lld, exch1 %lld, convert %lld, exch2 %lld (cycles per unit)\n", blockIdx.x, tid, n_units,
+                   tp[0] / n_units, tp[1] / n_units, tp[2] / n_units, tp[3] / n_units, tp[4] / n_units, tp[5] / n_units);
+#endif
+#undef PKV_HAND_OVER
+#undef PKV_TAKE_BACK
+        if (!ok && lane == 0 && !*abort_flag) { *abort_flag = 1; atomicAdd(a.status, 1); }
+        if (ok) {
+            const float inv = st.l > 0.f ? 1.f / st.l : 0.f;
+            __nv_bfloat16 *out = reinterpret_cast<__nv_bfloat16 *>(a.out);
+#pragma unroll 1
+            for (int c = 0; c < 4; ++c) {
+                uint32_t r[32];
+                tmem_ld32(t_o + 32 * c, r);
+                tmem_ld_wait();
+#pragma unroll
+                for (int i = 0; i < 32; ++i) r[i] = __float_as_uint(__uint_as_float(r[i]) * inv);
+                if (row_ok) {
+                    if (out) {
+#pragma unroll
+                        for (int k = 0; k < 4; ++k)
+                            *reinterpret_cast<uint4 *>(out + qrow * kHeadDim + 32 * c + 8 * k) =
+                                make_uint4(pack_bf16(__uint_as_float(r[8 * k]), __uint_as_float(r[8 * k + 1])),
+                                           pack_bf16(__uint_as_float(r[8 * k + 2]), __uint_as_float(r[8 * k + 3])),
+                                           pack_bf16(__uint_as_float(r[8 * k + 4]), __uint_as_float(r[8 * k + 5])),
+                                           pack_bf16(__uint_as_float(r[8 * k + 6]), __uint_as_float(r[8 * k + 7])));
+                    }
+                    if (a.out_f32) {
+#pragma unroll
+                        for (int k = 0; k < 8; ++k)
+                            *reinterpret_cast<uint4 *>(a.out_f32 + qrow * kHeadDim + 32 * c + 4 * k) = make_uint4(r[4 * k], r[4 * k + 1], r[4 * k + 2], r[4 * k + 3]);
+                    }
+                }
+            }
+        }
+    }
+    // ------------------------------ every thread: give tensor memory back ------------------------------
+    tc_fence_before();
+    __syncthreads();
+    if (warp == 0) asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tm), "r"(kTmemCols) : "memory");
+}
+
+size_t umma_smem_bytes(const Geometry &g) {
+    const int S = umma_stages(g);
+    return (size_t)kUQBytes + (size_t)S * umma_stage_bytes(g) + (2 * S + 3) * 8 + S * sizeof(StageDesc) + 64;
+}
+
+}  // namespace
+
+bool row_block_umma_supported(const Geometry &g) {
+    // A^T rows of 128 bytes (P = 64); every part of a blob on a 256-byte row of the pool (ranks even), A_v^T on a
+    // 1024-byte boundary of its own (the swizzle pattern repeats every 8 rows)
+    return g.page == 64 && g.factor_bits == 16 && g.global_rank == 0 && g.rank_k % 8 == 0 && g.rank_v % 2 == 0 &&
+           g.rank_v <= g.rank_k && g.rank_tiles >= 1 && g.rank_tiles <= 4 && g.bk_off % 256 == 0 && g.bv_off % 256 == 0 &&
+           g.blob_bytes % 256 == 0 && umma_smem_bytes(g) <= (size_t)kSmemBudget / 2;
+}
+
+cudaError_t row_block_umma_setup() {
+    cudaError_t e;
+    if ((e = cudaFuncSetAttribute(block_umma_kernel<1>, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBudget / 2)) != cudaSuccess) return e;
+    if ((e = cudaFuncSetAttribute(block_umma_kernel<2>, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBudget / 2)) != cudaSuccess) return e;
+    if ((e = cudaFuncSetAttribute(block_umma_kernel<3>, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBudget / 2)) != cudaSuccess) return e;
+    return cudaFuncSetAttribute(block_umma_kernel<4>, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBudget / 2);
+}
+
+// Tensor maps of the two pools seen as matrices of 256-byte rows (128 bf16), box = 64 channels x `rows`.  The
+// encoder is a driver entry point; it is looked up at run time so that the library does not link against the driver.
+void row_block_make_maps(const Geometry &g, const void *factor_pool, const void *dense_pool, RowBlockMaps *maps) {
+    typedef CUresult (*EncodeTiled)(CUtensorMap *, CUtensorMapDataType, cuuint32_t, void *, const cuuint64_t *, const cuuint64_t *,
+                                    const cuuint32_t *, const cuuint32_t *, CUtensorMapInterleave, CUtensorMapSwizzle,
+                                    CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+    maps->valid = 0;
+    if (!row_block_umma_supported(g) || !dense_pool) return;
+    void *fn = nullptr;
+    cudaDriverEntryPointQueryResult found = cudaDriverEntryPointSymbolNotFound;
+    if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &fn, cudaEnableDefault, &found) != cudaSuccess || !fn ||
+        found != cudaDriverEntryPointSuccess) {
+        (void)cudaGetLastError();
+        return;
+    }
+    const EncodeTiled encode = reinterpret_cast<EncodeTiled>(fn);
+    auto make = [&](CUtensorMap *m, const void *base, long long bytes, int rows) -> bool {
+        const cuuint64_t dims[2] = {(cuuint64_t)kHeadDim, (cuuint64_t)(bytes / kRowBytes)};
+        const cuuint64_t strides[1] = {(cuuint64_t)kRowBytes};
+        const cuuint32_t box[2] = {64u, (cuuint32_t)rows}, elem[2] = {1u, 1u};
+        return dims[1] > 0 && dims[1] < (1ull << 31) &&
+               encode(m, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void *>(base), dims, strides, box, elem,
+                      CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_NONE, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+                      CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+    };
+    const int rb = umma_part_rows(g);
+    if (!make(&maps->dense, dense_pool, (long long)g.n_dense_slots * g.dense_slot_bytes, rb)) return;
+    if (factor_pool && g.n_factor_slots > 0) {
+        const long long bytes = (long long)g.n_factor_slots * g.factor_slot_bytes;
+        if (!make(&maps->bk, factor_pool, bytes, g.rank_k) || !make(&maps->bv, factor_pool, bytes, g.rank_v)) return;
+    } else {
+        maps->bk = maps->dense;          // no factor pages: never used
+        maps->bv = maps->dense;
+    }
+    maps->valid = 1;
+}
+
+// One CTA per (sequence, KV head, block of 128 query rows).
+cudaError_t launch_decode_blocks_umma(const DecodeArgs &a, int n_seqs, const RowBlockMaps &maps, cudaStream_t st) {
+    const int n_blk = (a.q_len * a.geo.group + kURows - 1) / kURows;
+    const long long n_ctas = (long long)n_seqs * a.geo.n_kv_heads * n_blk;
+    if (!maps.valid || !row_block_umma_supported(a.geo) || n_ctas <= 0 || n_ctas > 0x7fffffffLL) return cudaErrorInvalidValue;
+    const size_t smem = umma_smem_bytes(a.geo);
+    switch (a.geo.rank_tiles) {
+        case 1: block_umma_kernel<1><<<(unsigned)n_ctas, kUThreads, smem, st>>>(a, maps.bk, maps.bv, maps.dense); break;
+        case 2: block_umma_kernel<2><<<(unsigned)n_ctas, kUThreads, smem, st>>>(a, maps.bk, maps.bv, maps.dense); break;
+        case 3: block_umma_kernel<3><<<(unsigned)n_ctas, kUThreads, smem, st>>>(a, maps.bk, maps.bv, maps.dense); break;
+        default: block_umma_kernel<4><<<(unsigned)n_ctas, kUThreads, smem, st>>>(a, maps.bk, maps.bv, maps.dense); break;
+    }
+    return cudaGetLastError();
+}
+
+}  // namespace pkv
