@@ -13,18 +13,16 @@
 // row of the next product's A operand over the columns it has just read (tcgen05.mma takes A from tensor memory).
 // A^T factors are used where the bulk copy put them: the storage swizzle of a 128-byte A^T row is the tensor core's
 // 128-byte swizzle (A_k^T as an MN-major B operand, A_v^T as a K-major one).  Rows of 256 bytes (B factors, dense
-// K / V) are split by the row threads into two panels of 128-byte rows first, which is the same swizzle again.
+// K / V) arrive as two panels of 128-byte rows (tiled TMA copies, 64 channels each), which is the same swizzle again.
 //
 // Warps 0-3: the 128 query rows.  Warp 4, one lane: bulk copies into the ring.  Warp 5, one lane: issues every
 // tcgen05.mma.  Rows -> issuer: an mbarrier all 128 row threads arrive on; issuer -> rows: tcgen05.commit on a second
 // mbarrier.  The four products of a factor page depend on one another through the row threads, so consecutive units
 // are skewed: a unit costs two exchanges, each carrying one product of the unit and one of the next,
-//     exchange 1 of unit u:  rows: softmax of s(u), panels V(u) and K(u+1)   then issuer: G3(u) | Gb(u), G1(u+1)
-//     exchange 2 of unit u:  rows: w(u) and q~(u+1) to bf16                  then issuer: G4(u), G2(u+1) | Ga(u+1)
+//     exchange 1 of unit u:  rows: softmax of s(u)               then issuer: G3(u) | Gb(u)
+//     exchange 2 of unit u:  rows: w(u) and q~(u+1) to bf16      then issuer: G4(u), G2(u+1) | Ga(u+1); behind it G1(u+2)
 // and two CTAs per SM overlap one another's chains.  Every wait is bounded; tensor memory is released on every path
 // out.
-#include <cstdio>
-
 #include "pkv_device.cuh"
 
 namespace pkv {
@@ -109,6 +107,12 @@ __device__ __forceinline__ void tmem_st8(uint32_t taddr, const uint32_t *r) {
 }
 __device__ __forceinline__ void tmem_st_wait() { asm volatile("tcgen05.wait::st.sync.aligned;" ::: "memory"); }
 template <int N>
+__device__ __forceinline__ void tmem_ld_nowait(uint32_t taddr, uint32_t *r) {
+    static_assert(N == 16 || N == 32, "16 or 32 columns");
+    if (N == 16) tmem_ld16(taddr, r);
+    else tmem_ld32(taddr, r);
+}
+template <int N>
 __device__ __forceinline__ void tmem_ld(uint32_t taddr, uint32_t *r) {
     static_assert(N == 16 || N == 32 || N == 64, "16, 32 or 64 columns");
     if (N == 16) tmem_ld16(taddr, r);
@@ -166,9 +170,10 @@ struct RowSoftmax {
 // the scores were read from.  o_valid: some product has already written o.
 template <int N>
 __device__ __forceinline__ void softmax_row(float *sv, RowSoftmax &st, bool o_valid, uint32_t t_s, uint32_t t_o) {
-    float mx = sv[0];
+    float mx4[4] = {sv[0], sv[1], sv[2], sv[3]};           // four chains: a thread has no other work to hide latencies with
 #pragma unroll
-    for (int i = 1; i < N; ++i) mx = fmaxf(mx, sv[i]);
+    for (int i = 4; i < N; ++i) mx4[i & 3] = fmaxf(mx4[i & 3], sv[i]);
+    const float mx = fmaxf(fmaxf(mx4[0], mx4[1]), fmaxf(mx4[2], mx4[3]));
     const bool grow = mx > st.m;
     float alpha = 1.f;
     if (grow) { alpha = exp2_fast(st.m - mx); st.m = mx; st.l *= alpha; }
@@ -183,17 +188,18 @@ __device__ __forceinline__ void softmax_row(float *sv, RowSoftmax &st, bool o_va
             tmem_st32(t_o + 32 * c, r);
         }
     }
-    float sum = 0.f;
+    float sum4[4] = {0.f, 0.f, 0.f, 0.f};
     const float m = st.m;
     uint32_t pk[N / 2];
 #pragma unroll
     for (int e = 0; e < N / 2; ++e) {
-        pk[e] = pack_bf16(exp2_fast(sv[2 * e] - m), exp2_fast(sv[2 * e + 1] - m));
-        sum += bf16lo_f(pk[e]) + bf16hi_f(pk[e]);          // l sums the weights as the product sees them
+        const float p0 = exp2_fast(sv[2 * e] - m), p1 = exp2_fast(sv[2 * e + 1] - m);
+        sum4[e & 3] += p0 + p1;
+        pk[e] = pack_bf16(p0, p1);
     }
     tmem_st<N / 2>(t_s, pk);
     tmem_st_wait();
-    st.l += sum;
+    st.l += (sum4[0] + sum4[1]) + (sum4[2] + sum4[3]);
 }
 
 template <int NT>
@@ -354,22 +360,19 @@ __global__ void __launch_bounds__(kUThreads, 2) block_umma_kernel(const __grid_c
                 const StageDesc d = descs[s];
                 return d.kind == kKindFactor && d.rows > 0 ? kKindFactor : kKindDense;
             };
-#ifdef PKV_UMMA_PROFILE
-            long long tw = 0, ti = 0, tx = 0, t0 = clock64(), t1;
-#define PKV_EXCHANGE_BEGIN() if (!wait_lane(c2m, xph, abort_flag)) { ok = false; break; } tc_fence_after(); t1 = clock64(); tw += t1 - t0; t0 = t1;
-#define PKV_EXCHANGE_END() umma_commit(m2c); t1 = clock64(); ti += t1 - t0; t0 = t1; (void)wait_lane(m2c, xph, abort_flag); t1 = clock64(); tx += t1 - t0; t0 = t1; xph ^= 1;
-#else
 #define PKV_EXCHANGE_BEGIN() if (!wait_lane(c2m, xph, abort_flag)) { ok = false; break; } tc_fence_after();
 #define PKV_EXCHANGE_END() umma_commit(m2c); xph ^= 1;
-#endif
             int kind_cur = kKindDense, kind_nxt = kKindDense;
             for (int u = -1; u < n_units; ++u) {
                 const uint32_t sb = smem_u32(stages + (size_t)((u + S) % S) * ustage);
                 const uint32_t sb_nxt = smem_u32(stages + (size_t)((u + 1) % S) * ustage);
-                // exchange 1: G3(u) | Gb(u), then G1(u+1)
+                // exchange 1: G3(u) | Gb(u)  (before the first unit: G1(0))
                 PKV_EXCHANGE_BEGIN()
-                if (u + 1 < n_units) { kind_nxt = unit_kind(u + 1, ok); if (!ok) break; }
-                if (u >= 0) {
+                if (u < 0) {
+                    kind_nxt = unit_kind(0, ok);
+                    if (!ok) break;
+                    if (kind_nxt == kKindFactor) qk(t_qt, sb_nxt);
+                } else {
                     if (kind_cur == kKindFactor) {
 #pragma unroll
                         for (int ks = 0; ks < P / 16; ++ks)      // w = p . A_v, A_v^T in place (K-major)
@@ -379,7 +382,6 @@ __global__ void __launch_bounds__(kUThreads, 2) block_umma_kernel(const __grid_c
                         umma_commit(smem_u32(empty_bar + u % S));      // a dense unit's stage is free after Gb
                     }
                 }
-                if (u + 1 < n_units && kind_nxt == kKindFactor) qk(t_qt, sb_nxt);
                 PKV_EXCHANGE_END()
                 // exchange 2: G4(u), then G2(u+1) | Ga(u+1)
                 PKV_EXCHANGE_BEGIN()
@@ -392,14 +394,17 @@ __global__ void __launch_bounds__(kUThreads, 2) block_umma_kernel(const __grid_c
                     else qk(t_s, sb_nxt);
                 }
                 PKV_EXCHANGE_END()
+                // Behind the exchange, off the rows' path: G1(u+2).  It overwrites the q~ columns G2(u+1) has just been
+                // issued on (products run in issue order); the rows meet its result after exchange 1 of unit u + 1.
                 kind_cur = kind_nxt;
+                if (u + 2 < n_units) {
+                    kind_nxt = unit_kind(u + 2, ok);
+                    if (!ok) break;
+                    if (kind_nxt == kKindFactor) qk(t_qt, smem_u32(stages + (size_t)((u + 2) % S) * ustage));
+                }
             }
 #undef PKV_EXCHANGE_BEGIN
 #undef PKV_EXCHANGE_END
-#ifdef PKV_UMMA_PROFILE
-            if (blockIdx.x == 0 || blockIdx.x == 300)
-                printf("cta %d issuer units %d: wait rows %lld, issue %lld, products %lld (cycles per unit, two exchanges)\n", blockIdx.x, n_units, tw / n_units, ti / n_units, tx / n_units);
-#endif
             if (!ok && !*abort_flag) { *abort_flag = 1; atomicAdd(a.status, 1); }
             // nothing of this CTA's may still be running on the tensor cores when tensor memory is given back
             umma_commit(smem_u32(drain_bar));
@@ -427,12 +432,6 @@ __global__ void __launch_bounds__(kUThreads, 2) block_umma_kernel(const __grid_c
         bool ok = true;
         const float scale = geo.scale_log2e;
         StageDesc cur{kKindDense, 0, 0, 0}, nxt{kKindDense, 0, 0, 0};
-#ifdef PKV_UMMA_PROFILE
-        long long tp[6] = {0, 0, 0, 0, 0, 0}, tc0 = clock64(), tc1;
-#define PKV_TICK(i) tc1 = clock64(); tp[i] += tc1 - tc0; tc0 = tc1;
-#else
-#define PKV_TICK(i)
-#endif
 #define PKV_HAND_OVER() tc_fence_before(); mbar_arrive(c2m);
 #define PKV_TAKE_BACK() if (!wait_warp(m2c, xph, abort_flag)) { ok = false; break; } xph ^= 1; tc_fence_after();
         for (int u = -1; u < n_units; ++u) {
@@ -457,52 +456,47 @@ __global__ void __launch_bounds__(kUThreads, 2) block_umma_kernel(const __grid_c
                     }
                 }
             }
-            PKV_TICK(0)
             if (u + 1 < n_units) {
                 const int s = (u + 1) % S;
                 if (!wait_warp(smem_u32(full_bar + s), ((u + 1) / S) & 1, abort_flag)) { ok = false; break; }
-                PKV_TICK(1)
                 nxt = descs[s];
                 if (nxt.rows <= 0 || nxt.kind != kKindFactor) { nxt.kind = kKindDense; nxt.rows = max(0, min(nxt.rows, kDB)); }
             }
-            PKV_TICK(2)
             PKV_HAND_OVER()
             PKV_TAKE_BACK()
-            PKV_TICK(3)
             // ---- before exchange 2: w(u) and q~(u+1) as bf16 rows ----
-            if (u >= 0 && cur.kind == kKindFactor) {       // w: columns past the rank are exact zeros
-                uint32_t r[RP], pk[RP / 2];
-                tmem_ld<RP>(t_w, r);
+            {
+                // both loads first: their latencies overlap, and a thread has nothing else to fill them with
+                const bool do_w = u >= 0 && cur.kind == kKindFactor, do_q = u + 1 < n_units && nxt.kind == kKindFactor;
+                uint32_t rw[RP], rq[RP];
+                if (do_w) tmem_ld_nowait<RP>(t_w, rw);
+                if (do_q) tmem_ld_nowait<RP>(t_qt, rq);
+                tmem_ld_wait();
+                if (do_w) {                                   // w: columns past the rank are exact zeros
+                    uint32_t pk[RP / 2];
 #pragma unroll
-                for (int k = 0; k < RP / 2; ++k)
-                    pk[k] = pack_bf16(2 * k < geo.rank_v ? __uint_as_float(r[2 * k]) : 0.f, 2 * k + 1 < geo.rank_v ? __uint_as_float(r[2 * k + 1]) : 0.f);
-                tmem_st<RP / 2>(t_w, pk);
-            }
-            if (u + 1 < n_units && nxt.kind == kKindFactor) {   // q~: scaled, two bf16 terms, columns past the rank exact zeros
-                uint32_t r[RP], hi[RP / 2], lo[RP / 2];
-                tmem_ld<RP>(t_qt, r);
-#pragma unroll
-                for (int k = 0; k < RP / 2; ++k) {
-                    const float x0 = 2 * k < geo.rank_k ? __uint_as_float(r[2 * k]) * scale : 0.f;
-                    const float x1 = 2 * k + 1 < geo.rank_k ? __uint_as_float(r[2 * k + 1]) * scale : 0.f;
-                    hi[k] = pack_bf16(x0, x1);
-                    lo[k] = pack_bf16(x0 - bf16lo_f(hi[k]), x1 - bf16hi_f(hi[k]));
+                    for (int k = 0; k < RP / 2; ++k)
+                        pk[k] = pack_bf16(2 * k < geo.rank_v ? __uint_as_float(rw[2 * k]) : 0.f, 2 * k + 1 < geo.rank_v ? __uint_as_float(rw[2 * k + 1]) : 0.f);
+                    tmem_st<RP / 2>(t_w, pk);
                 }
-                tmem_st<RP / 2>(t_qt, hi);
-                tmem_st<RP / 2>(t_qt + RP / 2, lo);
+                if (do_q) {                                   // q~: scaled, two bf16 terms, columns past the rank exact zeros
+                    uint32_t hi[RP / 2], lo[RP / 2];
+#pragma unroll
+                    for (int k = 0; k < RP / 2; ++k) {
+                        const float x0 = 2 * k < geo.rank_k ? __uint_as_float(rq[2 * k]) * scale : 0.f;
+                        const float x1 = 2 * k + 1 < geo.rank_k ? __uint_as_float(rq[2 * k + 1]) * scale : 0.f;
+                        hi[k] = pack_bf16(x0, x1);
+                        lo[k] = pack_bf16(x0 - bf16lo_f(hi[k]), x1 - bf16hi_f(hi[k]));
+                    }
+                    tmem_st<RP / 2>(t_qt, hi);
+                    tmem_st<RP / 2>(t_qt + RP / 2, lo);
+                }
             }
             tmem_st_wait();
-            PKV_TICK(4)
             PKV_HAND_OVER()
             PKV_TAKE_BACK()
-            PKV_TICK(5)
             cur = nxt;
         }
-#ifdef PKV_UMMA_PROFILE
-        if ((blockIdx.x == 0 || blockIdx.x == 300) && (tid == 0 || tid == 64))
-            printf("cta %d tid %d units %d: softmax+Vpanel %lld, wait full %lld, Kpanel %lld, exch1 %lld, convert %lld, exch2 %lld (cycles per unit)\n", blockIdx.x, tid, n_units,
-                   tp[0] / n_units, tp[1] / n_units, tp[2] / n_units, tp[3] / n_units, tp[4] / n_units, tp[5] / n_units);
-#endif
 #undef PKV_HAND_OVER
 #undef PKV_TAKE_BACK
         if (!ok && lane == 0 && !*abort_flag) { *abort_flag = 1; atomicAdd(a.status, 1); }
