@@ -142,22 +142,22 @@ __device__ __forceinline__ float exp2_fast(float x) {
 }
 
 // Bounded waits.  One lane (producer, issuer): gives up when the clock limit passes or another role has given up.
-__device__ __forceinline__ bool wait_lane(uint32_t bar, uint32_t parity, volatile int *abort_flag) {
+__device__ __forceinline__ bool wait_lane(uint32_t bar, uint32_t parity, volatile int *abort_flag, long long limit) {
     if (mbar_try_wait(bar, parity)) return true;
     const long long t0 = clock64();
     while (!mbar_try_wait(bar, parity)) {
-        if (clock64() - t0 > kWaitClocks || *abort_flag) return false;
+        if (clock64() - t0 > limit || *abort_flag) return false;
     }
     return true;
 }
 // A whole warp (the row threads run warp-collective tensor-memory loads right after): the outcome is the same for
 // all 32 lanes.
-__device__ __forceinline__ bool wait_warp(uint32_t bar, uint32_t parity, volatile int *abort_flag) {
+__device__ __forceinline__ bool wait_warp(uint32_t bar, uint32_t parity, volatile int *abort_flag, long long limit) {
     if (__all_sync(0xffffffffu, mbar_try_wait(bar, parity))) return true;
     const long long t0 = clock64();
     for (;;) {
         if (__all_sync(0xffffffffu, mbar_try_wait(bar, parity))) return true;
-        if (__any_sync(0xffffffffu, clock64() - t0 > kWaitClocks || *abort_flag)) return false;
+        if (__any_sync(0xffffffffu, clock64() - t0 > limit || *abort_flag)) return false;
     }
 }
 
@@ -272,7 +272,7 @@ __global__ void __launch_bounds__(kUThreads, 2) block_umma_kernel(const __grid_c
             int u = 0;
             for (; u < n_units; ++u) {
                 const int s = u % S;
-                if (u >= S && !wait_lane(smem_u32(empty_bar + s), ((u / S) - 1) & 1, abort_flag)) { ok = false; break; }
+                if (u >= S && !wait_lane(smem_u32(empty_bar + s), ((u / S) - 1) & 1, abort_flag, a.wait_clocks)) { ok = false; break; }
                 int page, blk, kind;
                 unit_to_page(geo, hu, u, page, blk, kind);
                 const int slot = pt[page];
@@ -287,6 +287,7 @@ __global__ void __launch_bounds__(kUThreads, 2) block_umma_kernel(const __grid_c
                     rows = max(0, min(kDB, T - page * P - blk * kDB));
                     after = max(0, T - page * P - blk * kDB - rows);
                 }
+                if (a.drop_unit == u && blockIdx.x == 0) continue;          // test hook: the unit is never armed, a wait must run out
                 descs[s] = StageDesc{kind, rows, 0, after};
                 const uint32_t bar = smem_u32(full_bar + s);
                 const uint32_t dst = smem_u32(stages + (size_t)s * ustage);
@@ -318,7 +319,7 @@ __global__ void __launch_bounds__(kUThreads, 2) block_umma_kernel(const __grid_c
             // copies already in flight must land before the CTA retires: wait (bounded) for the stages armed last
             for (int back = 1; back <= min(u, S); ++back) {
                 const int k = u - back;
-                (void)mbar_wait(smem_u32(full_bar + k % S), (k / S) & 1);
+                (void)mbar_wait(smem_u32(full_bar + k % S), (k / S) & 1, a.wait_clocks);
             }
         }
     } else if (warp == 5) {
@@ -356,11 +357,11 @@ __global__ void __launch_bounds__(kUThreads, 2) block_umma_kernel(const __grid_c
             // kind of a unit as the products see it: units without tokens run as dense units with every score masked
             auto unit_kind = [&](int u, bool &good) -> int {
                 const int s = u % S;
-                if (!wait_lane(smem_u32(full_bar + s), (u / S) & 1, abort_flag)) { good = false; return kKindDense; }
+                if (!wait_lane(smem_u32(full_bar + s), (u / S) & 1, abort_flag, a.wait_clocks)) { good = false; return kKindDense; }
                 const StageDesc d = descs[s];
                 return d.kind == kKindFactor && d.rows > 0 ? kKindFactor : kKindDense;
             };
-#define PKV_EXCHANGE_BEGIN() if (!wait_lane(c2m, xph, abort_flag)) { ok = false; break; } tc_fence_after();
+#define PKV_EXCHANGE_BEGIN() if (!wait_lane(c2m, xph, abort_flag, a.wait_clocks)) { ok = false; break; } tc_fence_after();
 #define PKV_EXCHANGE_END() umma_commit(m2c); xph ^= 1;
             int kind_cur = kKindDense, kind_nxt = kKindDense;
             for (int u = -1; u < n_units; ++u) {
@@ -408,7 +409,7 @@ __global__ void __launch_bounds__(kUThreads, 2) block_umma_kernel(const __grid_c
             if (!ok && !*abort_flag) { *abort_flag = 1; atomicAdd(a.status, 1); }
             // nothing of this CTA's may still be running on the tensor cores when tensor memory is given back
             umma_commit(smem_u32(drain_bar));
-            (void)mbar_wait(smem_u32(drain_bar), 0);
+            (void)mbar_wait(smem_u32(drain_bar), 0, a.wait_clocks);
         }
     } else {
         // ------------------------------ rows: one query row per thread ------------------------------
@@ -433,7 +434,7 @@ __global__ void __launch_bounds__(kUThreads, 2) block_umma_kernel(const __grid_c
         const float scale = geo.scale_log2e;
         StageDesc cur{kKindDense, 0, 0, 0}, nxt{kKindDense, 0, 0, 0};
 #define PKV_HAND_OVER() tc_fence_before(); mbar_arrive(c2m);
-#define PKV_TAKE_BACK() if (!wait_warp(m2c, xph, abort_flag)) { ok = false; break; } xph ^= 1; tc_fence_after();
+#define PKV_TAKE_BACK() if (!wait_warp(m2c, xph, abort_flag, a.wait_clocks)) { ok = false; break; } xph ^= 1; tc_fence_after();
         for (int u = -1; u < n_units; ++u) {
             // ---- before exchange 1: softmax of s(u) ----
             if (u >= 0) {
@@ -458,7 +459,7 @@ __global__ void __launch_bounds__(kUThreads, 2) block_umma_kernel(const __grid_c
             }
             if (u + 1 < n_units) {
                 const int s = (u + 1) % S;
-                if (!wait_warp(smem_u32(full_bar + s), ((u + 1) / S) & 1, abort_flag)) { ok = false; break; }
+                if (!wait_warp(smem_u32(full_bar + s), ((u + 1) / S) & 1, abort_flag, a.wait_clocks)) { ok = false; break; }
                 nxt = descs[s];
                 if (nxt.rows <= 0 || nxt.kind != kKindFactor) { nxt.kind = kKindDense; nxt.rows = max(0, min(nxt.rows, kDB)); }
             }

@@ -430,3 +430,40 @@ def test_a_bounded_wait_that_runs_out_is_reported_and_the_cache_stays_usable(mon
     ref = pair.orc.decode_attention(0, [0], f64(q))
     assert rel_err(got32, ref) <= 4e-3 and rel_err(got, ref) <= 1e-2
     pair.gpu.close()
+
+
+@pytest.mark.gpu
+def test_a_wait_that_runs_out_in_the_tcgen05_row_block_kernel(monkeypatch):
+    """The same for the tcgen05 row-block kernel, whose CTAs allocate tensor memory: the copy lane of CTA 0 leaves one
+    unit unarmed, the row threads' wait for it runs out, every role of the CTA leaves through the common exit (which
+    gives tensor memory back), the call returns with the timeout counted, and the next call on the same cache - whose
+    CTAs allocate tensor memory again - is correct."""
+    monkeypatch.setenv("PKV_TEST_WAIT_CLOCKS", "4000000")
+    monkeypatch.setenv("PKV_TEST_DROP_UNIT", "5")
+    H, G, q_len, T = 1, 4, 64, 1500
+    cfg = pkv.make_config(n_layers=1, n_kv_heads=H, n_q_heads=H * G, rank=24, sink_tokens=64, recent_tokens=128,
+                          max_seqs=1, max_pages_per_seq=32, n_dense_slots=32, n_factor_slots=32)
+    pair = Pair(cfg, seed=11)
+    monkeypatch.delenv("PKV_TEST_WAIT_CLOCKS")
+    monkeypatch.delenv("PKV_TEST_DROP_UNIT")
+    k, v = gen_kv(11, 0, 0, T, cfg)
+    pair.append(0, [0], [k[:T - q_len]], [v[:T - q_len]])
+    pair.compress(0)
+    pair.append(0, [0], [k[T - q_len:]], [v[T - q_len:]])
+    g = torch.Generator().manual_seed(12)
+    q = torch.randn((1, q_len, H * G, 128), generator=g).to(torch.bfloat16)
+    qd = q.cuda()
+    out32 = torch.empty(qd.shape, dtype=torch.float32, device="cuda")
+    pair.gpu.decode_attention_multi(0, [0], q_len, qd, None, out32)       # the launch with the unarmed unit
+    torch.cuda.synchronize()
+    st = pair.gpu.stats()
+    assert st["device_timeouts"] >= 1
+    pair.gpu.decode_attention_multi(0, [0], q_len, qd, None, out32)       # an ordinary launch on the same cache
+    torch.cuda.synchronize()
+    assert pair.gpu.stats()["device_timeouts"] == st["device_timeouts"]
+    pair.load_gpu_factors_into_oracle(0, 0)
+    ref = pair.orc.decode_attention_multi(0, [0], f64(q))
+    got32 = f64(out32)
+    for j in range(q_len):
+        assert rel_err(got32[0, j], ref[0, j]) <= 4e-3, j
+    pair.gpu.close()
