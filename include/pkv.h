@@ -300,15 +300,18 @@ pkv_status pkv_decode_attention(pkv_cache *c, int32_t layer, int32_t n_seqs, con
  * checked per call); n_seqs * b <= max_seqs with b = ceil(q_len / max(1, 8 / (H_q / H_kv))) blocks of query tokens
  * per sequence, b rounded up to a multiple of the grid size if it exceeds it (split-K partial states and tickets
  * are kept per sequence and block).
- * Two kernels serve this call.  A row-block kernel - one CTA per (sequence, KV head, 64 query rows), which reads the
- * sequence's pages once for its 64 rows (tensor-core products with the query rows as the 16-row operand) - runs
- * when q_len * (H_q / H_kv) >= 64, the factors are bf16, and the call makes at least 128 such CTAs (enough to fill
- * the GPU) or would exceed the limit above, which does not apply to this kernel.  Otherwise the decode kernel runs
+ * Two kinds of kernel serve this call.  A row-block kernel - one CTA per (sequence, KV head, block of query rows),
+ * which reads the sequence's pages once for its block, the query rows being the row operand of every product of
+ * Eq. 4 - runs when q_len * (H_q / H_kv) >= 64, the factors are bf16, and the call makes at least 128 blocks of 64
+ * rows (enough to fill the GPU) or would exceed the limit above, which does not apply to this kernel.  For
+ * page_size 64, rank a multiple of 8 and rank_v even it is the tcgen05 kernel (128 rows per CTA, accumulators and
+ * row operands in tensor memory, pages brought in by TMA in the layout the tensor cores read); for other shapes,
+ * or with decode_variant 3, the mma.sync kernel (64 rows per CTA).  Otherwise the decode kernel runs
  * with its CTAs in groups of b = ceil(q_len / max(1, 8 / (H_q / H_kv))): the CTAs of a group walk the same pages at
  * the same time, one block of 8 / (H_q / H_kv) query tokens each, so HBM delivers a page once and L2 delivers it b
  * times (q_len = 2 at H_q / H_kv = 8 costs 1.3 single-query launches, q_len = 2 at H_q / H_kv = 4 costs one).
- * Both kernels give the same result up to fp32 summation order.
- * Needs decode_variant 0 or 2 (PKV_ERR_UNSUPPORTED with 1).  CUDA-graph and overlap semantics as for
+ * All of them give the same result up to fp32 summation order.
+ * Needs decode_variant 0, 2 or 3 (PKV_ERR_UNSUPPORTED with 1).  CUDA-graph and overlap semantics as for
  * pkv_decode_attention(); a layer keeps one plan, that of its most recent (batch, q_len), so calls that
  * alternate between shapes on one layer rebuild it each time (host work and a small upload; not capturable).
  */
