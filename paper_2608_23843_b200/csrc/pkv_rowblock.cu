@@ -15,14 +15,17 @@
 // 128-byte swizzle (A_k^T as an MN-major B operand, A_v^T as a K-major one).  Rows of 256 bytes (B factors, dense
 // K / V) arrive as two panels of 128-byte rows (tiled TMA copies, 64 channels each), which is the same swizzle again.
 //
-// Warps 0-3: the 128 query rows.  Warp 4, one lane: bulk copies into the ring.  Warp 5, one lane: issues every
-// tcgen05.mma.  Rows -> issuer: an mbarrier all 128 row threads arrive on; issuer -> rows: tcgen05.commit on a second
-// mbarrier.  The four products of a factor page depend on one another through the row threads, so consecutive units
-// are skewed: a unit costs two exchanges, each carrying one product of the unit and one of the next,
-//     exchange 1 of unit u:  rows: softmax of s(u)               then issuer: G3(u) | Gb(u)
-//     exchange 2 of unit u:  rows: w(u) and q~(u+1) to bf16      then issuer: G4(u), G2(u+1) | Ga(u+1); behind it G1(u+2)
-// and two CTAs per SM overlap one another's chains.  Every wait is bounded; tensor memory is released on every path
-// out.
+// Warps 0-3: the 128 query rows.  Warp 4, one lane: copies into the ring.  Warp 5, one lane: issues every
+// tcgen05.mma.  The four products of a factor page depend on one another through the row threads; the schedule
+// keeps the row threads waiting for as few of them as it can.  Per unit u the rows hand over three times (an
+// mbarrier of 128 arrivals each) and the issuer answers with tcgen05.commit on four mbarriers:
+//     rows: wait S(u); softmax -> p(u)                      hand-over A -> issuer: G3(u) | Gb(u); commit "G3"
+//     rows: wait "Q"; q~(u+1) to two bf16 terms             hand-over B -> issuer: G2(u+1) | Ga(u+1); commit "S"
+//     rows: wait "G3"; w(u) to bf16                         hand-over C -> issuer: G4(u); commit "O"; G1(u+2); commit "Q"
+// so the conversion of q~(u+1) runs while G3(u) does, s(u+1) is being computed while w(u) is converted, and the rows
+// never wait for G4 or G1 unless o has to be rescaled (they meet commit "O" later in the unit, when it has long
+// arrived).  Two CTAs per SM overlap one another's remaining waits.  Every wait is bounded; tensor memory is
+// released on every path out.
 #include "pkv_device.cuh"
 
 namespace pkv {
@@ -34,16 +37,20 @@ constexpr int kUThreads = 192;
 constexpr int kUQBytes = 2 * kURows * 128;       // Q: two panels [128 rows][64 channels], 128-byte swizzle
 constexpr uint32_t kColQt = 0, kColS = 32, kColW = 96, kColO = 128, kTmemCols = 256;
 
-// A stage holds one unit the way the products read it, RB = 16 or 32 rows of 128 bytes per part:
-//     [A_k^T][K side, channels 0-63][K side, channels 64-127][A_v^T][V side, channels 0-63][V side, channels 64-127]
-// K side = B_k or a block of dense K, V side = B_v or a block of dense V.  The sides are written by tiled TMA
+// A stage holds one unit the way the products read it, in parts of 128-byte rows (see StageLayout).  K side = B_k or
+// a block of dense K, V side = B_v or a block of dense V; a side is two panels of 64 channels, written by tiled TMA
 // copies (box = 64 channels x rows) straight from the pools' 256-byte rows: 16-byte chunk c of row j is stored at
 // chunk c ^ (j & 7), so each half of a row is a 128-byte row in the tensor core's 128-byte swizzle.
+// Rows of a dense block, and what a rank is padded to in the products (16 or 32):
 __host__ __device__ inline int umma_part_rows(const Geometry &g) { return g.rank_tiles <= 2 ? 16 : 32; }
-__host__ __device__ inline int umma_stage_bytes(const Geometry &g) { return 6 * umma_part_rows(g) * 128; }
-// stages: the units u and u + 1 are in use at any time; the rest is the copies' lead
+constexpr int kUStagePad = 1024;
+__host__ __device__ inline int umma_stage_bytes(const Geometry &g) {
+    const int factor = 3 * 128 * (g.rank_k + g.rank_v), dense = 4 * umma_part_rows(g) * 128;
+    return ((factor > dense ? factor : dense) + 1023) & ~1023;
+}
+// stages: the units u, u + 1 and u + 2 are in use at any time; the rest is the copies' lead
 __host__ __device__ inline int umma_stages(const Geometry &g) {
-    const int room = 113 * 1024 - kUQBytes - 512;
+    const int room = 113 * 1024 - kUQBytes - kUStagePad - 512;
     return max(3, min(6, room / umma_stage_bytes(g)));
 }
 
@@ -165,11 +172,29 @@ struct RowSoftmax {
     float m, l;           // running maximum (log2 units) and sum of this thread's row
 };
 
-// Online softmax of one row over N scores held in sv (already scaled and masked): updates (m, l), rescales o in
-// tensor memory when some row of the warp has a new maximum, and writes p as bf16 pairs over the first N / 2 columns
-// the scores were read from.  o_valid: some product has already written o.
+// Byte offsets of a unit's parts inside its stage.  A factor unit fills the stage without gaps,
+//     [A_k^T: r_k rows][K side: 2 panels of r_k rows][A_v^T: r_v rows][V side: 2 panels of r_v rows]    (128-byte rows)
+// so a product that reads a rank padded to 16 or 32 rows runs into the next part: real data, multiplied by exact
+// zeros (or producing columns that are replaced by exact zeros).  A dense unit is [K side: 2 x RB rows][V side: 2 x RB rows].
+struct StageLayout {
+    int ak, k, k_panel, av, v, v_panel;         // factor units
+    int dk, dv, d_panel;                        // dense units
+};
+__host__ __device__ inline StageLayout umma_layout(const Geometry &g) {
+    StageLayout L;
+    L.ak = 0; L.k = g.rank_k * 128; L.k_panel = g.rank_k * 128;
+    L.av = 3 * g.rank_k * 128; L.v = L.av + g.rank_v * 128; L.v_panel = g.rank_v * 128;
+    L.d_panel = umma_part_rows(g) * 128; L.dk = 0; L.dv = 2 * L.d_panel;
+    return L;
+}
+
+// Online softmax of one row over N scores held in sv (already scaled and masked): updates (m, l); when some row of the
+// warp has a new maximum, waits (once per unit: o_seen) for the product of the unit before that adds to o and
+// rescales o in tensor memory; writes p as bf16 pairs over the first N / 2 columns the scores were read from.
+// o_valid: some product has already written o.  False if the wait ran out.
 template <int N>
-__device__ __forceinline__ void softmax_row(float *sv, RowSoftmax &st, bool o_valid, uint32_t t_s, uint32_t t_o) {
+__device__ __forceinline__ bool softmax_row(float *sv, RowSoftmax &st, bool o_valid, uint32_t t_s, uint32_t t_o, uint32_t bar_O,
+                                            uint32_t &ph_O, bool &o_seen, volatile int *abort_flag, long long limit) {
     float mx4[4] = {sv[0], sv[1], sv[2], sv[3]};           // four chains: a thread has no other work to hide latencies with
 #pragma unroll
     for (int i = 4; i < N; ++i) mx4[i & 3] = fmaxf(mx4[i & 3], sv[i]);
@@ -178,6 +203,10 @@ __device__ __forceinline__ void softmax_row(float *sv, RowSoftmax &st, bool o_va
     float alpha = 1.f;
     if (grow) { alpha = exp2_fast(st.m - mx); st.m = mx; st.l *= alpha; }
     if (o_valid && __any_sync(0xffffffffu, grow)) {
+        if (!wait_warp(bar_O, ph_O, abort_flag, limit)) return false;
+        ph_O ^= 1;
+        o_seen = true;
+        tc_fence_after();
         uint32_t r[32];
 #pragma unroll 1
         for (int c = 0; c < 4; ++c) {
@@ -200,6 +229,7 @@ __device__ __forceinline__ void softmax_row(float *sv, RowSoftmax &st, bool o_va
     tmem_st<N / 2>(t_s, pk);
     tmem_st_wait();
     st.l += (sum4[0] + sum4[1]) + (sum4[2] + sum4[3]);
+    return true;
 }
 
 template <int NT>
@@ -208,10 +238,9 @@ __global__ void __launch_bounds__(kUThreads, 2) block_umma_kernel(const __grid_c
                                                                   const __grid_constant__ CUtensorMap map_bv,
                                                                   const __grid_constant__ CUtensorMap map_dense) {
     constexpr int P = 64, RP = NT <= 2 ? 16 : 32, kDB = kDenseBlock<P, NT, 0>;
-    static_assert(kDB == RP, "dense blocks and padded ranks share the stage layout");
-    constexpr int kPart = RP * 128;                   // bytes of one part of a stage
-    constexpr int oAk = 0, oK = kPart, oAv = 3 * kPart, oV = 4 * kPart;
+    static_assert(kDB == RP, "dense blocks and padded ranks have the same number of rows");
     const Geometry &geo = a.geo;
+    const StageLayout L = umma_layout(geo);
     const int S = umma_stages(geo), ustage = umma_stage_bytes(geo), H = geo.n_kv_heads, G = geo.group;
     const int n_rows = a.q_len * G, n_blk = (n_rows + kURows - 1) / kURows;
     const int rb = blockIdx.x % n_blk, head = (blockIdx.x / n_blk) % H, entry = blockIdx.x / (n_blk * H);
@@ -219,24 +248,26 @@ __global__ void __launch_bounds__(kUThreads, 2) block_umma_kernel(const __grid_c
     if (entry >= hdr.n_seqs) return;
     extern __shared__ __align__(1024) unsigned char smem[];
     unsigned char *sq = smem, *stages = smem + kUQBytes;
-    unsigned long long *full_bar = reinterpret_cast<unsigned long long *>(stages + (size_t)S * ustage);
+    // (one more KiB behind the last stage: a padded product of the last stage's last part reads it)
+    unsigned long long *full_bar = reinterpret_cast<unsigned long long *>(stages + (size_t)S * ustage + kUStagePad);
     unsigned long long *empty_bar = full_bar + S;
-    unsigned long long *c2m_bar = empty_bar + S, *m2c_bar = c2m_bar + 1, *drain_bar = m2c_bar + 1;
-    StageDesc *descs = reinterpret_cast<StageDesc *>(drain_bar + 1);
+    unsigned long long *bars = empty_bar + S;          // rows -> issuer: A, B, C; issuer -> rows: G3, S, O, Q; drain
+    StageDesc *descs = reinterpret_cast<StageDesc *>(bars + 8);
     volatile int *abort_flag = reinterpret_cast<volatile int *>(descs + S);
     uint32_t *tmem_slot = reinterpret_cast<uint32_t *>(const_cast<int *>(abort_flag) + 1);
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+    const uint32_t bar_A = smem_u32(bars + 0), bar_B = smem_u32(bars + 1), bar_C = smem_u32(bars + 2);
+    const uint32_t bar_G3 = smem_u32(bars + 3), bar_S = smem_u32(bars + 4), bar_O = smem_u32(bars + 5), bar_Q = smem_u32(bars + 6);
+    const uint32_t bar_drain = smem_u32(bars + 7);
     if (tid == 0) {
         for (int s = 0; s < S; ++s) { mbar_init(smem_u32(full_bar + s), 1); mbar_init(smem_u32(empty_bar + s), 1); }
-        mbar_init(smem_u32(c2m_bar), kURows);
-        mbar_init(smem_u32(m2c_bar), 1);
-        mbar_init(smem_u32(drain_bar), 1);
+        mbar_init(bar_A, kURows); mbar_init(bar_B, kURows); mbar_init(bar_C, kURows);
+        mbar_init(bar_G3, 1); mbar_init(bar_S, 1); mbar_init(bar_O, 1); mbar_init(bar_Q, 1); mbar_init(bar_drain, 1);
         *abort_flag = 0;
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     }
-    // Rows past the rank are never written by the copies and are multiplied by exact zeros: they must hold finite
-    // values from the start.
-    for (int i = tid; i < S * ustage / 16; i += kUThreads) reinterpret_cast<uint4 *>(stages)[i] = make_uint4(0u, 0u, 0u, 0u);
+    // What a padded product reads past a unit's own rows must be finite from the start.
+    for (int i = tid; i < (S * ustage + kUStagePad) / 16; i += kUThreads) reinterpret_cast<uint4 *>(stages)[i] = make_uint4(0u, 0u, 0u, 0u);
     fence_async_smem();
     if (warp == 0) {
         asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(tmem_slot)), "r"(kTmemCols) : "memory");
@@ -262,7 +293,7 @@ __global__ void __launch_bounds__(kUThreads, 2) block_umma_kernel(const __grid_c
         else need = hu.d0 + hu.nf + (page - hu.fe) * geo.blocks_per_page + blk + 1;
         n_units = max(1, min(need, hu.units));
     }
-    const uint32_t c2m = smem_u32(c2m_bar), m2c = smem_u32(m2c_bar);
+    const long long limit = a.wait_clocks;
 
     if (warp == 4) {
         // ------------------------------ copies (one lane) ------------------------------
@@ -272,7 +303,7 @@ __global__ void __launch_bounds__(kUThreads, 2) block_umma_kernel(const __grid_c
             int u = 0;
             for (; u < n_units; ++u) {
                 const int s = u % S;
-                if (u >= S && !wait_lane(smem_u32(empty_bar + s), ((u / S) - 1) & 1, abort_flag, a.wait_clocks)) { ok = false; break; }
+                if (u >= S && !wait_lane(smem_u32(empty_bar + s), ((u / S) - 1) & 1, abort_flag, limit)) { ok = false; break; }
                 int page, blk, kind;
                 unit_to_page(geo, hu, u, page, blk, kind);
                 const int slot = pt[page];
@@ -296,21 +327,21 @@ __global__ void __launch_bounds__(kUThreads, 2) block_umma_kernel(const __grid_c
                     const unsigned char *src = a.factor_pool + off;
                     const int yk = (int)((off + geo.bk_off) >> 8), yv = (int)((off + geo.bv_off) >> 8);     // pool rows of 256 bytes
                     mbar_arrive_expect_tx(bar, geo.blob_bytes);
-                    bulk_g2s_keep(dst + oAk, src + geo.ak_off, geo.rank_k * 128, bar);
-                    bulk_g2s_keep(dst + oAv, src + geo.av_off, geo.rank_v * 128, bar);
-                    tma_box(dst + oK, &map_bk, 0, yk, bar);
-                    tma_box(dst + oK + kPart, &map_bk, 64, yk, bar);
-                    tma_box(dst + oV, &map_bv, 0, yv, bar);
-                    tma_box(dst + oV + kPart, &map_bv, 64, yv, bar);
+                    bulk_g2s_keep(dst + L.ak, src + geo.ak_off, geo.rank_k * 128, bar);
+                    bulk_g2s_keep(dst + L.av, src + geo.av_off, geo.rank_v * 128, bar);
+                    tma_box(dst + L.k, &map_bk, 0, yk, bar);
+                    tma_box(dst + L.k + L.k_panel, &map_bk, 64, yk, bar);
+                    tma_box(dst + L.v, &map_bv, 0, yv, bar);
+                    tma_box(dst + L.v + L.v_panel, &map_bv, 64, yv, bar);
                 } else if (rows > 0) {
                     // whole blocks: rows past the sequence's end hold whatever the pool holds; the scores there are
-                    // masked and the row threads clear those rows of V
+                    // masked and the row threads clear those rows
                     const int y = (int)(((long long)slot * geo.dense_slot_bytes + (long long)head * geo.dense_head_bytes) >> 8) + blk * kDB;
-                    mbar_arrive_expect_tx(bar, 4 * kPart);
-                    tma_box(dst + oK, &map_dense, 0, y, bar);
-                    tma_box(dst + oK + kPart, &map_dense, 64, y, bar);
-                    tma_box(dst + oV, &map_dense, 0, y + P, bar);
-                    tma_box(dst + oV + kPart, &map_dense, 64, y + P, bar);
+                    mbar_arrive_expect_tx(bar, 4 * L.d_panel);
+                    tma_box(dst + L.dk, &map_dense, 0, y, bar);
+                    tma_box(dst + L.dk + L.d_panel, &map_dense, 64, y, bar);
+                    tma_box(dst + L.dv, &map_dense, 0, y + P, bar);
+                    tma_box(dst + L.dv + L.d_panel, &map_dense, 64, y + P, bar);
                 } else {
                     mbar_arrive(bar);
                 }
@@ -319,7 +350,7 @@ __global__ void __launch_bounds__(kUThreads, 2) block_umma_kernel(const __grid_c
             // copies already in flight must land before the CTA retires: wait (bounded) for the stages armed last
             for (int back = 1; back <= min(u, S); ++back) {
                 const int k = u - back;
-                (void)mbar_wait(smem_u32(full_bar + k % S), (k / S) & 1, a.wait_clocks);
+                (void)mbar_wait(smem_u32(full_bar + k % S), (k / S) & 1, limit);
             }
         }
     } else if (warp == 5) {
@@ -327,89 +358,88 @@ __global__ void __launch_bounds__(kUThreads, 2) block_umma_kernel(const __grid_c
         if (elect_one()) {
             const uint32_t sq_a = smem_u32(sq);
             const uint32_t t_qt = tm + kColQt, t_s = tm + kColS, t_w = tm + kColW, t_o = tm + kColO;
-            uint32_t xph = 0;
+            uint32_t ph_A = 0, ph_B = 0, ph_C = 0;
             bool ok = true, o_valid = false;
-            // [128 x n] = Q . (K side)^T: 8 steps of 16 channels; both operands K-major, 128-byte swizzle
-            auto qk = [&](uint32_t t_dst, uint32_t sb) {
+            auto stage_of = [&](int u) { return smem_u32(stages + (size_t)(u % S) * ustage); };
+            // [128 x RP] = Q . (K side)^T: 8 steps of 16 channels; both operands K-major, 128-byte swizzle
+            auto qk = [&](uint32_t t_dst, uint32_t kside, int panel) {
                 const uint32_t idesc = umma_idesc(128, RP, 0);
 #pragma unroll
                 for (int ks = 0; ks < 8; ++ks)
                     umma_ss(t_dst, umma_desc(sq_a + (ks >> 2) * (kURows * 128) + (ks & 3) * 32, 16, 1024, 2),
-                            umma_desc(sb + oK + (ks >> 2) * kPart + (ks & 3) * 32, 16, 1024, 2), idesc, ks > 0);
+                            umma_desc(kside + (ks >> 2) * panel + (ks & 3) * 32, 16, 1024, 2), idesc, ks > 0);
             };
-            // o [128 x d] (+)= (rows of n bf16 at t_src) . (V side): the V side is MN-major, two panels of 64 channels
-            auto pv = [&](uint32_t t_src, uint32_t sb) {
+            // o [128 x d] (+)= (rows of RP bf16 at t_src) . (V side): MN-major, two panels of 64 channels
+            auto pv = [&](uint32_t t_src, uint32_t vside, int panel) {
 #pragma unroll
                 for (int ks = 0; ks < RP / 16; ++ks)
-                    umma_ts(t_o, t_src + ks * 8, umma_desc(sb + oV + ks * 2048, kPart, 1024, 2), umma_idesc(128, 128, 1),
-                            o_valid || ks > 0);
+                    umma_ts(t_o, t_src + ks * 8, umma_desc(vside + ks * 2048, panel, 1024, 2), umma_idesc(128, 128, 1), o_valid || ks > 0);
                 o_valid = true;
-            };
-            // s = (q~_hi + q~_lo) . A_k^T, A_k^T in place (MN-major)
-            auto g2 = [&](uint32_t sb) {
-#pragma unroll
-                for (int t = 0; t < 2; ++t)
-#pragma unroll
-                    for (int ks = 0; ks < RP / 16; ++ks)
-                        umma_ts(t_s, t_qt + t * (RP / 2) + ks * 8, umma_desc(sb + oAk + ks * 2048, 16, 1024, 2),
-                                umma_idesc(128, P, 1), (t | ks) > 0);
             };
             // kind of a unit as the products see it: units without tokens run as dense units with every score masked
             auto unit_kind = [&](int u, bool &good) -> int {
                 const int s = u % S;
-                if (!wait_lane(smem_u32(full_bar + s), (u / S) & 1, abort_flag, a.wait_clocks)) { good = false; return kKindDense; }
+                if (!wait_lane(smem_u32(full_bar + s), (u / S) & 1, abort_flag, limit)) { good = false; return kKindDense; }
                 const StageDesc d = descs[s];
                 return d.kind == kKindFactor && d.rows > 0 ? kKindFactor : kKindDense;
             };
-#define PKV_EXCHANGE_BEGIN() if (!wait_lane(c2m, xph, abort_flag, a.wait_clocks)) { ok = false; break; } tc_fence_after();
-#define PKV_EXCHANGE_END() umma_commit(m2c); xph ^= 1;
-            int kind_cur = kKindDense, kind_nxt = kKindDense;
-            for (int u = -1; u < n_units; ++u) {
-                const uint32_t sb = smem_u32(stages + (size_t)((u + S) % S) * ustage);
-                const uint32_t sb_nxt = smem_u32(stages + (size_t)((u + 1) % S) * ustage);
-                // exchange 1: G3(u) | Gb(u)  (before the first unit: G1(0))
-                PKV_EXCHANGE_BEGIN()
-                if (u < 0) {
-                    kind_nxt = unit_kind(0, ok);
-                    if (!ok) break;
-                    if (kind_nxt == kKindFactor) qk(t_qt, sb_nxt);
-                } else {
-                    if (kind_cur == kKindFactor) {
+            int k0 = kKindDense, k1 = kKindDense, k2 = kKindDense;       // kinds of the units u, u + 1, u + 2
+            for (int u = -2; u < n_units; ++u) {
+                if (u >= 0) {
+                    // hand-over A: p(u) is in tensor memory -> G3(u) | Gb(u)
+                    if (!wait_lane(bar_A, ph_A, abort_flag, limit)) { ok = false; break; }
+                    ph_A ^= 1;
+                    tc_fence_after();
+                    const uint32_t sb = stage_of(u);
+                    if (k0 == kKindFactor) {
 #pragma unroll
                         for (int ks = 0; ks < P / 16; ++ks)      // w = p . A_v, A_v^T in place (K-major)
-                            umma_ts(t_w, t_s + ks * 8, umma_desc(sb + oAv + ks * 32, 16, 1024, 2), umma_idesc(128, RP, 0), ks > 0);
+                            umma_ts(t_w, t_s + ks * 8, umma_desc(sb + L.av + ks * 32, 16, 1024, 2), umma_idesc(128, RP, 0), ks > 0);
                     } else {
-                        pv(t_s, sb);
+                        pv(t_s, sb + L.dv, L.d_panel);
                         umma_commit(smem_u32(empty_bar + u % S));      // a dense unit's stage is free after Gb
                     }
+                    umma_commit(bar_G3);
                 }
-                PKV_EXCHANGE_END()
-                // exchange 2: G4(u), then G2(u+1) | Ga(u+1)
-                PKV_EXCHANGE_BEGIN()
-                if (u >= 0 && kind_cur == kKindFactor) {
-                    pv(t_w, sb);
+                if (u >= -1 && u + 1 < n_units) {
+                    // hand-over B: q~(u+1) is in tensor memory -> G2(u+1) | Ga(u+1)
+                    if (!wait_lane(bar_B, ph_B, abort_flag, limit)) { ok = false; break; }
+                    ph_B ^= 1;
+                    tc_fence_after();
+                    const uint32_t sb = stage_of(u + 1);
+                    if (k1 == kKindFactor) {
+#pragma unroll
+                        for (int t = 0; t < 2; ++t)              // s = (q~_hi + q~_lo) . A_k^T, A_k^T in place (MN-major)
+#pragma unroll
+                            for (int ks = 0; ks < RP / 16; ++ks)
+                                umma_ts(t_s, t_qt + t * (RP / 2) + ks * 8, umma_desc(sb + L.ak + ks * 2048, 16, 1024, 2),
+                                        umma_idesc(128, P, 1), (t | ks) > 0);
+                    } else {
+                        qk(t_s, sb + L.dk, L.d_panel);
+                    }
+                    umma_commit(bar_S);
+                }
+                // hand-over C: w(u) is in tensor memory -> G4(u); then, off the rows' path, G1(u+2)
+                if (!wait_lane(bar_C, ph_C, abort_flag, limit)) { ok = false; break; }
+                ph_C ^= 1;
+                tc_fence_after();
+                if (u >= 0 && k0 == kKindFactor) {
+                    pv(t_w, stage_of(u) + L.v, L.v_panel);
                     umma_commit(smem_u32(empty_bar + u % S));          // a factor unit's stage is free after G4
                 }
-                if (u + 1 < n_units) {
-                    if (kind_nxt == kKindFactor) g2(sb_nxt);
-                    else qk(t_s, sb_nxt);
-                }
-                PKV_EXCHANGE_END()
-                // Behind the exchange, off the rows' path: G1(u+2).  It overwrites the q~ columns G2(u+1) has just been
-                // issued on (products run in issue order); the rows meet its result after exchange 1 of unit u + 1.
-                kind_cur = kind_nxt;
+                umma_commit(bar_O);
                 if (u + 2 < n_units) {
-                    kind_nxt = unit_kind(u + 2, ok);
+                    k2 = unit_kind(u + 2, ok);
                     if (!ok) break;
-                    if (kind_nxt == kKindFactor) qk(t_qt, smem_u32(stages + (size_t)((u + 2) % S) * ustage));
+                    if (k2 == kKindFactor) qk(t_qt, stage_of(u + 2) + L.k, L.k_panel);
                 }
+                umma_commit(bar_Q);
+                k0 = k1; k1 = k2;
             }
-#undef PKV_EXCHANGE_BEGIN
-#undef PKV_EXCHANGE_END
             if (!ok && !*abort_flag) { *abort_flag = 1; atomicAdd(a.status, 1); }
             // nothing of this CTA's may still be running on the tensor cores when tensor memory is given back
-            umma_commit(smem_u32(drain_bar));
-            (void)mbar_wait(smem_u32(drain_bar), 0, a.wait_clocks);
+            umma_commit(bar_drain);
+            (void)mbar_wait(bar_drain, 0, limit);
         }
     } else {
         // ------------------------------ rows: one query row per thread ------------------------------
@@ -429,59 +459,46 @@ __global__ void __launch_bounds__(kUThreads, 2) block_umma_kernel(const __grid_c
         const uint32_t t_lane = tm + ((uint32_t)(warp * 32) << 16);
         const uint32_t t_qt = t_lane + kColQt, t_s = t_lane + kColS, t_w = t_lane + kColW, t_o = t_lane + kColO;
         RowSoftmax st{kNegInf, 0.f};
-        uint32_t xph = 0;
+        uint32_t ph_G3 = 0, ph_S = 0, ph_O = 0, ph_Q = 0;
         bool ok = true;
         const float scale = geo.scale_log2e;
         StageDesc cur{kKindDense, 0, 0, 0}, nxt{kKindDense, 0, 0, 0};
-#define PKV_HAND_OVER() tc_fence_before(); mbar_arrive(c2m);
-#define PKV_TAKE_BACK() if (!wait_warp(m2c, xph, abort_flag, a.wait_clocks)) { ok = false; break; } xph ^= 1; tc_fence_after();
-        for (int u = -1; u < n_units; ++u) {
-            // ---- before exchange 1: softmax of s(u) ----
+#define PKV_ROWS_WAIT(bar, ph) { if (!wait_warp(bar, ph, abort_flag, limit)) { ok = false; break; } ph ^= 1; tc_fence_after(); }
+#define PKV_ROWS_ARRIVE(bar) { tc_fence_before(); mbar_arrive(bar); }
+        for (int u = -2; u < n_units; ++u) {
+            bool o_seen = false;          // whether this iteration has waited for the o of the unit before
             if (u >= 0) {
+                // ---- softmax of s(u); p(u) -> hand-over A ----
+                PKV_ROWS_WAIT(bar_S, ph_S)
+                bool fine;
                 if (cur.kind == kKindFactor) {
                     float sv[P];
                     tmem_ld<P>(t_s, reinterpret_cast<uint32_t *>(sv));
-                    softmax_row<P>(sv, st, u > 0, t_s, t_o);
+                    fine = softmax_row<P>(sv, st, u > 0, t_s, t_o, bar_O, ph_O, o_seen, abort_flag, limit);
                 } else {
                     float sv[kDB];
                     tmem_ld<kDB>(t_s, reinterpret_cast<uint32_t *>(sv));
                     const int lim = cur.rows - max(0, hid - cur.after);
 #pragma unroll
                     for (int i = 0; i < kDB; ++i) sv[i] = i < lim ? sv[i] * scale : kMasked;
-                    softmax_row<kDB>(sv, st, u > 0, t_s, t_o);
-                    if (cur.rows < kDB) {          // V rows past the sequence's end: p is 0 there, the rows must be finite
-                        unsigned char *v = stages + (size_t)(u % S) * ustage + oV;
-                        for (int i = tid; i < (kDB - cur.rows) * 16; i += kURows)
-                            *reinterpret_cast<uint4 *>(v + (i & 1) * kPart + (cur.rows + (i >> 4)) * 128 + ((i >> 1) & 7) * 16) = make_uint4(0u, 0u, 0u, 0u);
-                        fence_async_smem();
-                    }
+                    fine = softmax_row<kDB>(sv, st, u > 0, t_s, t_o, bar_O, ph_O, o_seen, abort_flag, limit);
                 }
+                if (!fine) { ok = false; break; }
+                PKV_ROWS_ARRIVE(bar_A)
             }
-            if (u + 1 < n_units) {
+            if (u >= -1) {
+                if (!o_seen) PKV_ROWS_WAIT(bar_O, ph_O)          // (one wait per commit keeps the phases in step)
+                PKV_ROWS_WAIT(bar_Q, ph_Q)                       // G1(u+1) has written q~
+            }
+            if (u >= -1 && u + 1 < n_units) {
+                // ---- the next unit's descriptor; q~(u+1) as two bf16 terms -> hand-over B ----
                 const int s = (u + 1) % S;
-                if (!wait_warp(smem_u32(full_bar + s), ((u + 1) / S) & 1, abort_flag, a.wait_clocks)) { ok = false; break; }
+                if (!wait_warp(smem_u32(full_bar + s), ((u + 1) / S) & 1, abort_flag, limit)) { ok = false; break; }
                 nxt = descs[s];
                 if (nxt.rows <= 0 || nxt.kind != kKindFactor) { nxt.kind = kKindDense; nxt.rows = max(0, min(nxt.rows, kDB)); }
-            }
-            PKV_HAND_OVER()
-            PKV_TAKE_BACK()
-            // ---- before exchange 2: w(u) and q~(u+1) as bf16 rows ----
-            {
-                // both loads first: their latencies overlap, and a thread has nothing else to fill them with
-                const bool do_w = u >= 0 && cur.kind == kKindFactor, do_q = u + 1 < n_units && nxt.kind == kKindFactor;
-                uint32_t rw[RP], rq[RP];
-                if (do_w) tmem_ld_nowait<RP>(t_w, rw);
-                if (do_q) tmem_ld_nowait<RP>(t_qt, rq);
-                tmem_ld_wait();
-                if (do_w) {                                   // w: columns past the rank are exact zeros
-                    uint32_t pk[RP / 2];
-#pragma unroll
-                    for (int k = 0; k < RP / 2; ++k)
-                        pk[k] = pack_bf16(2 * k < geo.rank_v ? __uint_as_float(rw[2 * k]) : 0.f, 2 * k + 1 < geo.rank_v ? __uint_as_float(rw[2 * k + 1]) : 0.f);
-                    tmem_st<RP / 2>(t_w, pk);
-                }
-                if (do_q) {                                   // q~: scaled, two bf16 terms, columns past the rank exact zeros
-                    uint32_t hi[RP / 2], lo[RP / 2];
+                if (nxt.kind == kKindFactor) {      // columns past the rank are exact zeros
+                    uint32_t rq[RP], hi[RP / 2], lo[RP / 2];
+                    tmem_ld<RP>(t_qt, rq);
 #pragma unroll
                     for (int k = 0; k < RP / 2; ++k) {
                         const float x0 = 2 * k < geo.rank_k ? __uint_as_float(rq[2 * k]) * scale : 0.f;
@@ -491,15 +508,41 @@ __global__ void __launch_bounds__(kUThreads, 2) block_umma_kernel(const __grid_c
                     }
                     tmem_st<RP / 2>(t_qt, hi);
                     tmem_st<RP / 2>(t_qt + RP / 2, lo);
+                    tmem_st_wait();
+                } else if (nxt.rows < kDB) {
+                    // rows past the sequence's end hold whatever the pool held: p is 0 there, but the rows must be
+                    // finite (V), also for a padded product of the stage before this one (K)
+                    unsigned char *st_base = stages + (size_t)s * ustage;
+                    for (int i = tid; i < (kDB - nxt.rows) * 32; i += kURows) {
+                        const int side = i & 1, panel = (i >> 1) & 1, chunk = (i >> 2) & 7, r = nxt.rows + (i >> 5);
+                        *reinterpret_cast<uint4 *>(st_base + (side ? L.dv : L.dk) + panel * L.d_panel + r * 128 + chunk * 16) = make_uint4(0u, 0u, 0u, 0u);
+                    }
+                    fence_async_smem();
+                }
+                PKV_ROWS_ARRIVE(bar_B)
+            }
+            if (u >= 0) {
+                // ---- w(u) as bf16 -> hand-over C ----
+                PKV_ROWS_WAIT(bar_G3, ph_G3)
+                if (cur.kind == kKindFactor) {       // columns past the rank are exact zeros
+                    uint32_t rw[RP], pk[RP / 2];
+                    tmem_ld<RP>(t_w, rw);
+#pragma unroll
+                    for (int k = 0; k < RP / 2; ++k)
+                        pk[k] = pack_bf16(2 * k < geo.rank_v ? __uint_as_float(rw[2 * k]) : 0.f, 2 * k + 1 < geo.rank_v ? __uint_as_float(rw[2 * k + 1]) : 0.f);
+                    tmem_st<RP / 2>(t_w, pk);
+                    tmem_st_wait();
                 }
             }
-            tmem_st_wait();
-            PKV_HAND_OVER()
-            PKV_TAKE_BACK()
+            PKV_ROWS_ARRIVE(bar_C)
             cur = nxt;
         }
-#undef PKV_HAND_OVER
-#undef PKV_TAKE_BACK
+        if (ok) {                                                       // the last G4 | Gb
+            ok = wait_warp(bar_O, ph_O, abort_flag, limit);
+            tc_fence_after();
+        }
+#undef PKV_ROWS_WAIT
+#undef PKV_ROWS_ARRIVE
         if (!ok && lane == 0 && !*abort_flag) { *abort_flag = 1; atomicAdd(a.status, 1); }
         if (ok) {
             const float inv = st.l > 0.f ? 1.f / st.l : 0.f;
@@ -538,15 +581,15 @@ __global__ void __launch_bounds__(kUThreads, 2) block_umma_kernel(const __grid_c
 
 size_t umma_smem_bytes(const Geometry &g) {
     const int S = umma_stages(g);
-    return (size_t)kUQBytes + (size_t)S * umma_stage_bytes(g) + (2 * S + 3) * 8 + S * sizeof(StageDesc) + 64;
+    return (size_t)kUQBytes + (size_t)S * umma_stage_bytes(g) + kUStagePad + (2 * S + 8) * 8 + S * sizeof(StageDesc) + 64;
 }
 
 }  // namespace
 
 bool row_block_umma_supported(const Geometry &g) {
-    // A^T rows of 128 bytes (P = 64); every part of a blob on a 256-byte row of the pool (ranks even), A_v^T on a
-    // 1024-byte boundary of its own (the swizzle pattern repeats every 8 rows)
-    return g.page == 64 && g.factor_bits == 16 && g.global_rank == 0 && g.rank_k % 8 == 0 && g.rank_v % 2 == 0 &&
+    // A^T rows of 128 bytes (P = 64); every part of a blob on a 256-byte row of the pool, every part of a stage on a
+    // 1024-byte boundary (the swizzle pattern repeats every 8 rows): ranks that are multiples of 8
+    return g.page == 64 && g.factor_bits == 16 && g.global_rank == 0 && g.rank_k % 8 == 0 && g.rank_v % 8 == 0 &&
            g.rank_v <= g.rank_k && g.rank_tiles >= 1 && g.rank_tiles <= 4 && g.bk_off % 256 == 0 && g.bv_off % 256 == 0 &&
            g.blob_bytes % 256 == 0 && umma_smem_bytes(g) <= (size_t)kSmemBudget / 2;
 }
