@@ -168,9 +168,16 @@ __device__ __forceinline__ bool wait_warp(uint32_t bar, uint32_t parity, volatil
     }
 }
 
+// Softmax state of this thread's row.  p and l are always taken against the true running maximum m, so the largest
+// weight is exactly 1 and its bf16 rounding costs nothing.  o, which lives in tensor memory, is kept against an
+// older maximum m_ref <= m instead of being rescaled every time m grows: a factor page's contribution enters o
+// through w, an fp32 row that this thread rounds to bf16 itself, so it multiplies w by 2^(m - m_ref) first - the
+// rounding is relative and does not care.  o is rescaled for real only when that factor would pass 2^kFrameLag, or
+// before a dense block, whose p goes to the product as it is.
 struct RowSoftmax {
-    float m, l;           // running maximum (log2 units) and sum of this thread's row
+    float m, l, m_ref;
 };
+constexpr float kFrameLag = 8.f;
 
 // Byte offsets of a unit's parts inside its stage.  A factor unit fills the stage without gaps,
 //     [A_k^T: r_k rows][K side: 2 panels of r_k rows][A_v^T: r_v rows][V side: 2 panels of r_v rows]    (128-byte rows)
@@ -188,32 +195,37 @@ __host__ __device__ inline StageLayout umma_layout(const Geometry &g) {
     return L;
 }
 
-// Online softmax of one row over N scores held in sv (already scaled and masked): updates (m, l); when some row of the
-// warp has a new maximum, waits (once per unit: o_seen) for the product of the unit before that adds to o and
-// rescales o in tensor memory; writes p as bf16 pairs over the first N / 2 columns the scores were read from.
-// o_valid: some product has already written o.  False if the wait ran out.
-template <int N>
+// Online softmax of one row over N scores held in sv (already scaled and masked): updates (m, l), brings o to a
+// frame it may stay in (see RowSoftmax) - which, when some row of the warp needs it, means waiting (once per unit:
+// o_seen) for the product of the unit before that adds to o and rescaling o in tensor memory - and writes p as bf16
+// pairs over the first N / 2 columns the scores were read from.  o_valid: some product has already written o.
+// False if the wait ran out.
+template <int N, bool kDense>
 __device__ __forceinline__ bool softmax_row(float *sv, RowSoftmax &st, bool o_valid, uint32_t t_s, uint32_t t_o, uint32_t bar_O,
                                             uint32_t &ph_O, bool &o_seen, volatile int *abort_flag, long long limit) {
     float mx4[4] = {sv[0], sv[1], sv[2], sv[3]};           // four chains: a thread has no other work to hide latencies with
 #pragma unroll
     for (int i = 4; i < N; ++i) mx4[i & 3] = fmaxf(mx4[i & 3], sv[i]);
     const float mx = fmaxf(fmaxf(mx4[0], mx4[1]), fmaxf(mx4[2], mx4[3]));
-    const bool grow = mx > st.m;
-    float alpha = 1.f;
-    if (grow) { alpha = exp2_fast(st.m - mx); st.m = mx; st.l *= alpha; }
-    if (o_valid && __any_sync(0xffffffffu, grow)) {
-        if (!wait_warp(bar_O, ph_O, abort_flag, limit)) return false;
-        ph_O ^= 1;
-        o_seen = true;
-        tc_fence_after();
+    if (mx > st.m) { st.l *= exp2_fast(st.m - mx); st.m = mx; }
+    if (!o_valid) {
+        st.m_ref = st.m;
+    } else if (__any_sync(0xffffffffu, kDense ? st.m != st.m_ref : st.m - st.m_ref > kFrameLag)) {
+        if (!o_seen) {
+            if (!wait_warp(bar_O, ph_O, abort_flag, limit)) return false;
+            ph_O ^= 1;
+            o_seen = true;
+            tc_fence_after();
+        }
+        const float f = exp2_fast(st.m_ref - st.m);
+        st.m_ref = st.m;
         uint32_t r[32];
 #pragma unroll 1
         for (int c = 0; c < 4; ++c) {
             tmem_ld32(t_o + 32 * c, r);
             tmem_ld_wait();
 #pragma unroll
-            for (int i = 0; i < 32; ++i) r[i] = __float_as_uint(__uint_as_float(r[i]) * alpha);
+            for (int i = 0; i < 32; ++i) r[i] = __float_as_uint(__uint_as_float(r[i]) * f);
             tmem_st32(t_o + 32 * c, r);
         }
     }
@@ -458,7 +470,7 @@ __global__ void __launch_bounds__(kUThreads, 2) block_umma_kernel(const __grid_c
         const int hid = row_ok ? a.q_len - 1 - j : 0;       // newest positions this row must not see
         const uint32_t t_lane = tm + ((uint32_t)(warp * 32) << 16);
         const uint32_t t_qt = t_lane + kColQt, t_s = t_lane + kColS, t_w = t_lane + kColW, t_o = t_lane + kColO;
-        RowSoftmax st{kNegInf, 0.f};
+        RowSoftmax st{kNegInf, 0.f, kNegInf};
         uint32_t ph_G3 = 0, ph_S = 0, ph_O = 0, ph_Q = 0;
         bool ok = true;
         const float scale = geo.scale_log2e;
@@ -474,14 +486,14 @@ __global__ void __launch_bounds__(kUThreads, 2) block_umma_kernel(const __grid_c
                 if (cur.kind == kKindFactor) {
                     float sv[P];
                     tmem_ld<P>(t_s, reinterpret_cast<uint32_t *>(sv));
-                    fine = softmax_row<P>(sv, st, u > 0, t_s, t_o, bar_O, ph_O, o_seen, abort_flag, limit);
+                    fine = softmax_row<P, false>(sv, st, u > 0, t_s, t_o, bar_O, ph_O, o_seen, abort_flag, limit);
                 } else {
                     float sv[kDB];
                     tmem_ld<kDB>(t_s, reinterpret_cast<uint32_t *>(sv));
                     const int lim = cur.rows - max(0, hid - cur.after);
 #pragma unroll
                     for (int i = 0; i < kDB; ++i) sv[i] = i < lim ? sv[i] * scale : kMasked;
-                    fine = softmax_row<kDB>(sv, st, u > 0, t_s, t_o, bar_O, ph_O, o_seen, abort_flag, limit);
+                    fine = softmax_row<kDB, true>(sv, st, u > 0, t_s, t_o, bar_O, ph_O, o_seen, abort_flag, limit);
                 }
                 if (!fine) { ok = false; break; }
                 PKV_ROWS_ARRIVE(bar_A)
@@ -524,12 +536,13 @@ __global__ void __launch_bounds__(kUThreads, 2) block_umma_kernel(const __grid_c
             if (u >= 0) {
                 // ---- w(u) as bf16 -> hand-over C ----
                 PKV_ROWS_WAIT(bar_G3, ph_G3)
-                if (cur.kind == kKindFactor) {       // columns past the rank are exact zeros
+                if (cur.kind == kKindFactor) {       // into the frame o is kept in; columns past the rank are exact zeros
                     uint32_t rw[RP], pk[RP / 2];
                     tmem_ld<RP>(t_w, rw);
+                    const float c = exp2_fast(st.m - st.m_ref);
 #pragma unroll
                     for (int k = 0; k < RP / 2; ++k)
-                        pk[k] = pack_bf16(2 * k < geo.rank_v ? __uint_as_float(rw[2 * k]) : 0.f, 2 * k + 1 < geo.rank_v ? __uint_as_float(rw[2 * k + 1]) : 0.f);
+                        pk[k] = pack_bf16(2 * k < geo.rank_v ? __uint_as_float(rw[2 * k]) * c : 0.f, 2 * k + 1 < geo.rank_v ? __uint_as_float(rw[2 * k + 1]) * c : 0.f);
                     tmem_st<RP / 2>(t_w, pk);
                     tmem_st_wait();
                 }
@@ -545,7 +558,7 @@ __global__ void __launch_bounds__(kUThreads, 2) block_umma_kernel(const __grid_c
 #undef PKV_ROWS_ARRIVE
         if (!ok && lane == 0 && !*abort_flag) { *abort_flag = 1; atomicAdd(a.status, 1); }
         if (ok) {
-            const float inv = st.l > 0.f ? 1.f / st.l : 0.f;
+            const float inv = st.l > 0.f ? exp2_fast(st.m_ref - st.m) / st.l : 0.f;          // o is in the frame of m_ref
             __nv_bfloat16 *out = reinterpret_cast<__nv_bfloat16 *>(a.out);
 #pragma unroll 1
             for (int c = 0; c < 4; ++c) {
