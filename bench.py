@@ -790,15 +790,15 @@ def main():
                 flops += QL * Hq * (nf_ * 2 * (128 * rank + rank * P_ + P_ * rv_ + rv_ * 128) + dense_tok * 4 * 128)
             tpeak, tsrc = _tensor_peak()
             tach = flops / (launch_ms * 1e-3) / 1e12
-            # the library's own rule (row_block_umma_supported): tcgen05 kernel for P = 64, bf16 factors, rank_k a
-            # multiple of 8, rank_v even; the mma.sync kernel otherwise or when decode_variant 3 pins it
-            umma = args.decode_variant == 0 and P_ == 64 and rank % 8 == 0 and rv_ % 2 == 0 and rv_ <= rank
+            # the library's own rule (row_block_umma_supported): tcgen05 kernel for P = 64, bf16 factors, ranks that are
+            # multiples of 8; the mma.sync kernel otherwise or when decode_variant 3 pins it
+            umma = args.decode_variant == 0 and P_ == 64 and rank % 8 == 0 and rv_ % 8 == 0 and rv_ <= rank
             line["roofline"] = {"bound": "tensor",
                                 "kernel": ("block_umma_kernel<rank tiles=%d> (tcgen05, 128 query rows per CTA)" if umma else
                                            "block_tc_kernel<P=%d, rank tiles=%%d> (mma.sync, 64 query rows per CTA)" % P_) % ((rank + 7) // 8),
                                 "achieved": tach, "peak": tpeak, "unit": "TFLOP/s", "frac": tach / tpeak,
                                 "peak_source": tsrc + ("; the products are small (N = 32 to 128 per instruction, four dependent products per "
-                                                       "page through the row threads): ncu shows the tensor pipe about 20 % busy" if umma else
+                                                       "page through the row threads): ncu shows the tensor pipe about 25 % busy" if umma else
                                                        "; ncu showed the mma.sync pipe 50 % busy at this rate"),
                                 "traffic": None, "launch_us": launch_ms * 1e3, "algorithmic_flops_per_launch": flops}
         if not args.no_cpu_baseline and world == 1 and QL == 1 and not args.global_rank:
