@@ -230,6 +230,59 @@ def test_paper_default_shape_qwen3_8b_16k():
     _finish(cache)
 
 
+@pytest.mark.parametrize("variant", [0, 3])
+def test_prefill_chunk_2048_positions_against_32k(variant):
+    """The bench's prefill-chunk launch (`--workload prefill_chunk_llama3_8b_32k --q-len 2048`): one sequence of
+    32768 tokens whose last 2048 positions are the queries, 8192 query rows per KV head, served by the row-block
+    kernels (variant 0: tcgen05, 512 CTAs of 128 rows; 3: mma.sync, 1024 CTAs of 64 rows).  Sampled query rows -
+    the first and last positions of the chunk, positions on either side of page and block boundaries, a row from every
+    128-row block parity - against plain attention over the pages exactly as the GPU stores them (kernel gate; the
+    causal limit is part of what is checked), the two kernels against one another on every row, and a rerun bit for
+    bit."""
+    w, device = bench.WORKLOADS["prefill_chunk_llama3_8b_32k"], torch.device("cuda", 0)
+    QL = 2048
+    cfg, cache, lengths, comp = bench.build_workload(w, w["rank"], device, decode_variant=variant)
+    T, Hq, Hkv = lengths[0], w["n_q_heads"], w["n_kv_heads"]
+    G = Hq // Hkv
+    g = torch.Generator(device="cpu").manual_seed(bench.SEED + 77)
+    q = torch.randn((1, QL, Hq, 128), generator=g).to(torch.bfloat16).to(device)
+    out32 = torch.empty(q.shape, dtype=torch.float32, device=device)
+    out = torch.empty_like(q)
+    cache.decode_attention_multi(0, [0], QL, q, out, out32)
+    again = torch.empty_like(out32)
+    cache.decode_attention_multi(0, [0], QL, q, None, again)
+    torch.cuda.synchronize()
+    assert torch.equal(again, out32) and not out32.isnan().any()
+    scale = 1.0 / np.sqrt(cfg.head_dim)
+    positions = [0, 1, 31, 32, 63, 64, 65, 127, 128, 1000, 1023, 1024, 1999, 2046, 2047]
+    worst = 0.0
+    for head in (0, 5):
+        K_all, V_all, _ = stored_kv(cache, 0, 0, head)
+        for j in positions:
+            vis = T - (QL - 1 - j)
+            for gq in range(G):
+                h = head * G + gq
+                ref = oatt.attention_plain(f64(q[0, j, h]), K_all[:vis], V_all[:vis], scale)
+                e = rel_err(f64(out32[0, j, h]), ref)
+                assert e <= 4e-3, (variant, head, j, gq, e)
+                assert rel_err(f64(out[0, j, h]), ref) <= ATT_TOL
+                worst = max(worst, e)
+    record("prefill_chunk_llama3_8b_32k", decode_variant=variant, kernel_gate_worst=worst, rows_checked=2 * len(positions) * G)
+    if variant == 0:
+        _PREFILL_OUT["tcgen05"] = out32.cpu()
+    elif "tcgen05" in _PREFILL_OUT:
+        a, b = _PREFILL_OUT.pop("tcgen05").double().numpy(), out32.cpu().double().numpy()
+        # every row of the launch: the two kernels differ by summation order and by where p and w are rounded
+        err = np.abs(a - b).max(axis=-1) / np.abs(b).max(axis=-1)
+        assert err.max() <= 8e-3, err.max()          # both are within 4e-3 of the same reference
+        print("tcgen05 vs mma.sync over %d rows: worst %.2e, mean %.2e" % (err.size, err.max(), err.mean()))
+        record("prefill_chunk_llama3_8b_32k", tcgen05_vs_mma_sync_worst_row=float(err.max()), rows=int(err.size))
+    _finish(cache)
+
+
+_PREFILL_OUT = {}
+
+
 @pytest.mark.parametrize("rank", [8, 16, 24, 32])
 def test_ragged_serving_batch_rank_sweep(rank):
     """Ragged serving batch: 64 requests, lengths log-uniform in [2048, 65536], 2% outlier key tokens (x10)."""
