@@ -45,7 +45,7 @@ constexpr uint32_t kColQt = 0, kColS = 32, kColW = 96, kColO = 128, kTmemCols = 
 __host__ __device__ inline int umma_part_rows(const Geometry &g) { return g.rank_tiles <= 2 ? 16 : 32; }
 constexpr int kUStagePad = 1024;
 __host__ __device__ inline int umma_stage_bytes(const Geometry &g) {
-    const int factor = 3 * 128 * (g.rank_k + g.rank_v), dense = 4 * umma_part_rows(g) * 128;
+    const int factor = 3 * 128 * (((g.rank_k + 7) & ~7) + ((g.rank_v + 7) & ~7)), dense = 4 * umma_part_rows(g) * 128;
     return ((factor > dense ? factor : dense) + 1023) & ~1023;
 }
 // stages: the units u, u + 1 and u + 2 are in use at any time; the rest is the copies' lead
@@ -179,18 +179,21 @@ struct RowSoftmax {
 };
 constexpr float kFrameLag = 8.f;
 
-// Byte offsets of a unit's parts inside its stage.  A factor unit fills the stage without gaps,
+// Byte offsets of a unit's parts inside its stage.  A factor unit is
 //     [A_k^T: r_k rows][K side: 2 panels of r_k rows][A_v^T: r_v rows][V side: 2 panels of r_v rows]    (128-byte rows)
-// so a product that reads a rank padded to 16 or 32 rows runs into the next part: real data, multiplied by exact
-// zeros (or producing columns that are replaced by exact zeros).  A dense unit is [K side: 2 x RB rows][V side: 2 x RB rows].
+// with every part rounded up to a multiple of 8 rows, so a product that reads a rank padded to 16 or 32 rows reads
+// rows no copy of this unit wrote (what an earlier unit left there, or the zeros of the start) and runs into the
+// next part: finite data either way, multiplied by exact zeros (or producing columns that are replaced by exact
+// zeros).  A dense unit is [K side: 2 x RB rows][V side: 2 x RB rows].
 struct StageLayout {
     int ak, k, k_panel, av, v, v_panel;         // factor units
     int dk, dv, d_panel;                        // dense units
 };
 __host__ __device__ inline StageLayout umma_layout(const Geometry &g) {
     StageLayout L;
-    L.ak = 0; L.k = g.rank_k * 128; L.k_panel = g.rank_k * 128;
-    L.av = 3 * g.rank_k * 128; L.v = L.av + g.rank_v * 128; L.v_panel = g.rank_v * 128;
+    const int rk = (g.rank_k + 7) & ~7, rv = (g.rank_v + 7) & ~7;        // parts start on 1024-byte boundaries
+    L.ak = 0; L.k = rk * 128; L.k_panel = rk * 128;
+    L.av = 3 * rk * 128; L.v = L.av + rv * 128; L.v_panel = rv * 128;
     L.d_panel = umma_part_rows(g) * 128; L.dk = 0; L.dv = 2 * L.d_panel;
     return L;
 }
@@ -600,9 +603,9 @@ size_t umma_smem_bytes(const Geometry &g) {
 }  // namespace
 
 bool row_block_umma_supported(const Geometry &g) {
-    // A^T rows of 128 bytes (P = 64); every part of a blob on a 256-byte row of the pool, every part of a stage on a
-    // 1024-byte boundary (the swizzle pattern repeats every 8 rows): ranks that are multiples of 8
-    return g.page == 64 && g.factor_bits == 16 && g.global_rank == 0 && g.rank_k % 8 == 0 && g.rank_v % 8 == 0 &&
+    // A^T rows of 128 bytes (P = 64); every part of a blob on a 256-byte row of the pool (the tiled copies address
+    // the pools in such rows): even ranks
+    return g.page == 64 && g.factor_bits == 16 && g.global_rank == 0 && g.rank_k % 2 == 0 && g.rank_v % 2 == 0 &&
            g.rank_v <= g.rank_k && g.rank_tiles >= 1 && g.rank_tiles <= 4 && g.bk_off % 256 == 0 && g.bv_off % 256 == 0 &&
            g.blob_bytes % 256 == 0 && umma_smem_bytes(g) <= (size_t)kSmemBudget / 2;
 }

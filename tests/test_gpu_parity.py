@@ -502,6 +502,8 @@ def test_many_tiny_segments_per_cta(rank, n_ctas):
     (64, 32, 32, 1, 70, 16),      # row-block kernel, one query head per KV head, full-width ranks
     (64, 24, 24, 8, 16, 16),      # row-block kernel, 128 rows, two tokens per 16-row tile
     (32, 8, 8, 4, 40, 16),        # row-block kernel, one rank tile, queries spanning two pages
+    (64, 16, 14, 4, 70, 16),      # tcgen05 row-block kernel, even ranks that are not multiples of 8 (parts of a stage padded)
+    (64, 8, 8, 8, 40, 16),        # tcgen05 row-block kernel, one rank tile (rank padded to 16 in the products), 320 rows
 ])
 def test_multi_query_attention(P, rk, rv, G, q_len, bits):
     """Several new positions per sequence in one call (causal among themselves): every query row against the
@@ -661,7 +663,8 @@ def test_sequence_sharded_attention_states(bits):
     print("sharded states bits=%d: merged kernel gate max %.2e, log-sum-exp max abs %.2e" % (bits, worst, worst_lse))
 
 
-@pytest.mark.parametrize("P,rk,rv,G,q_len", [(64, 24, 24, 4, 128), (32, 16, 14, 8, 33), (16, 16, 16, 2, 48), (64, 8, 5, 4, 17)])
+@pytest.mark.parametrize("P,rk,rv,G,q_len", [(64, 24, 24, 4, 128), (32, 16, 14, 8, 33), (16, 16, 16, 2, 48), (64, 8, 5, 4, 17),
+                                             (64, 16, 14, 4, 70), (64, 30, 26, 2, 96)])
 def test_row_block_kernel_agrees_with_the_column_kernel(P, rk, rv, G, q_len):
     """pkv_decode_attention_multi picks its kernel by shape; decode_variant = 2 pins the decode (column) kernel.  The
     two must agree to fp32-accumulation accuracy on the same cache contents (same compression kernel, same factors),
