@@ -268,12 +268,14 @@ def test_config_validation():
                         (dict(rank=65), pkv.PKV_ERR_INVALID_ARG), (dict(rank=33), pkv.PKV_ERR_UNSUPPORTED),
                         (dict(head_dim=64, page_size=64), pkv.PKV_ERR_UNSUPPORTED), (dict(page_size=48, sink_tokens=48, recent_tokens=48), pkv.PKV_ERR_UNSUPPORTED),
                         (dict(page_size=16, rank=17, sink_tokens=16, recent_tokens=16), pkv.PKV_ERR_INVALID_ARG),
-                        (dict(n_q_heads=16), pkv.PKV_ERR_UNSUPPORTED), (dict(rank=16, rank_v=8), pkv.PKV_ERR_UNSUPPORTED)]:
+                        (dict(n_q_heads=16), pkv.PKV_ERR_UNSUPPORTED), (dict(rank=16, rank_v=8), pkv.PKV_ERR_UNSUPPORTED),
+                        (dict(decode_variant=4), pkv.PKV_ERR_INVALID_ARG), (dict(decode_variant=-1), pkv.PKV_ERR_INVALID_ARG)]:
         with pytest.raises(pkv.PkvError) as e:
             pkv.pkv_query_sizes(pkv.make_config(**{**ok, **bad}))
         assert e.value.status == status, bad
     for good in (dict(rank=12), dict(rank=16, rank_v=14, page_size=32, sink_tokens=32, recent_tokens=32),
-                 dict(rank=9, page_size=16, sink_tokens=16, recent_tokens=16), dict(rank=27)):
+                 dict(rank=9, page_size=16, sink_tokens=16, recent_tokens=16), dict(rank=27), dict(decode_variant=2),
+                 dict(decode_variant=3)):
         pkv.pkv_query_sizes(pkv.make_config(**{**ok, **good}))
     with pytest.raises(pkv.PkvError):
         pkv.Cache(pkv.make_config(**ok), dry_run=True, dense_slot_order=[0, 0, 1, 2])   # not a permutation
