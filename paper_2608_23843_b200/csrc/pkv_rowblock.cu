@@ -18,14 +18,14 @@
 // Warps 0-3: the 128 query rows.  Warp 4, one lane: copies into the ring.  Warp 5, one lane: issues every
 // tcgen05.mma.  The four products of a factor page depend on one another through the row threads; the schedule
 // keeps the row threads waiting for as few of them as it can.  Per unit u the rows hand over three times (an
-// mbarrier of 128 arrivals each) and the issuer answers with tcgen05.commit on four mbarriers:
-//     rows: wait S(u); softmax -> p(u)                      hand-over A -> issuer: G3(u) | Gb(u); commit "G3"
+// mbarrier of 128 arrivals each) and the issuer answers with tcgen05.commit on three mbarriers:
+//     rows: wait "S"; softmax of s(u) -> p(u)               hand-over A -> issuer: G3(u) | Gb(u); commit "G3"
 //     rows: wait "Q"; q~(u+1) to two bf16 terms             hand-over B -> issuer: G2(u+1) | Ga(u+1); commit "S"
-//     rows: wait "G3"; w(u) to bf16                         hand-over C -> issuer: G4(u); commit "O"; G1(u+2); commit "Q"
-// so the conversion of q~(u+1) runs while G3(u) does, s(u+1) is being computed while w(u) is converted, and the rows
-// never wait for G4 or G1 unless o has to be rescaled (they meet commit "O" later in the unit, when it has long
-// arrived).  Two CTAs per SM overlap one another's remaining waits.  Every wait is bounded; tensor memory is
-// released on every path out.
+//     rows: wait "G3"; w(u) to bf16                         hand-over C -> issuer: G4(u); G1(u+2); commit "Q"
+// so the conversion of q~(u+1) runs while G3(u) does, s(u+1) is being computed while w(u) is converted, and G4 and
+// G1 are off the rows' path: their commit is met one hand-over later, when it has long arrived (earlier only if o
+// has to be rescaled).  Two CTAs per SM overlap one another's remaining waits.  Every wait is bounded; tensor
+// memory is released on every path out.
 #include "pkv_device.cuh"
 
 namespace pkv {
@@ -198,14 +198,36 @@ __host__ __device__ inline StageLayout umma_layout(const Geometry &g) {
     return L;
 }
 
+// RP fp32 values x (a row of q~ or w) times `scale`, as bf16 pairs; columns from `rank` on become exact zeros.  The
+// first KNOWN columns are known to lie below the rank (no test), the rest are tested against it.
+template <int RP, int KNOWN>
+__device__ __forceinline__ void scale_pack(const uint32_t *x, uint32_t *pk, float scale, int rank) {
+#pragma unroll
+    for (int k = 0; k < RP / 2; ++k) {
+        const bool in0 = 2 * k < KNOWN && 2 * k < rank, in1 = 2 * k + 1 < KNOWN && 2 * k + 1 < rank;
+        pk[k] = pack_bf16(in0 ? __uint_as_float(x[2 * k]) * scale : 0.f, in1 ? __uint_as_float(x[2 * k + 1]) * scale : 0.f);
+    }
+}
+// The same with the rounding error of each pair as a second bf16 term (hi + lo carries about 16 bits).
+template <int RP, int KNOWN>
+__device__ __forceinline__ void split_terms(const uint32_t *x, uint32_t *hi, uint32_t *lo, float scale, int rank) {
+#pragma unroll
+    for (int k = 0; k < RP / 2; ++k) {
+        const bool in0 = 2 * k < KNOWN && 2 * k < rank, in1 = 2 * k + 1 < KNOWN && 2 * k + 1 < rank;
+        const float x0 = in0 ? __uint_as_float(x[2 * k]) * scale : 0.f, x1 = in1 ? __uint_as_float(x[2 * k + 1]) * scale : 0.f;
+        hi[k] = pack_bf16(x0, x1);
+        lo[k] = pack_bf16(x0 - bf16lo_f(hi[k]), x1 - bf16hi_f(hi[k]));
+    }
+}
+
 // Online softmax of one row over N scores held in sv (already scaled and masked): updates (m, l), brings o to a
 // frame it may stay in (see RowSoftmax) - which, when some row of the warp needs it, means waiting (once per unit:
 // o_seen) for the product of the unit before that adds to o and rescaling o in tensor memory - and writes p as bf16
 // pairs over the first N / 2 columns the scores were read from.  o_valid: some product has already written o.
 // False if the wait ran out.
 template <int N, bool kDense>
-__device__ __forceinline__ bool softmax_row(float *sv, RowSoftmax &st, bool o_valid, uint32_t t_s, uint32_t t_o, uint32_t bar_O,
-                                            uint32_t &ph_O, bool &o_seen, volatile int *abort_flag, long long limit) {
+__device__ __forceinline__ bool softmax_row(float *sv, RowSoftmax &st, bool o_valid, uint32_t t_s, uint32_t t_o, uint32_t bar_Q,
+                                            uint32_t &ph_Q, bool &o_seen, volatile int *abort_flag, long long limit) {
     float mx4[4] = {sv[0], sv[1], sv[2], sv[3]};           // four chains: a thread has no other work to hide latencies with
 #pragma unroll
     for (int i = 4; i < N; ++i) mx4[i & 3] = fmaxf(mx4[i & 3], sv[i]);
@@ -215,8 +237,8 @@ __device__ __forceinline__ bool softmax_row(float *sv, RowSoftmax &st, bool o_va
         st.m_ref = st.m;
     } else if (__any_sync(0xffffffffu, kDense ? st.m != st.m_ref : st.m - st.m_ref > kFrameLag)) {
         if (!o_seen) {
-            if (!wait_warp(bar_O, ph_O, abort_flag, limit)) return false;
-            ph_O ^= 1;
+            if (!wait_warp(bar_Q, ph_Q, abort_flag, limit)) return false;
+            ph_Q ^= 1;
             o_seen = true;
             tc_fence_after();
         }
@@ -266,18 +288,18 @@ __global__ void __launch_bounds__(kUThreads, 2) block_umma_kernel(const __grid_c
     // (one more KiB behind the last stage: a padded product of the last stage's last part reads it)
     unsigned long long *full_bar = reinterpret_cast<unsigned long long *>(stages + (size_t)S * ustage + kUStagePad);
     unsigned long long *empty_bar = full_bar + S;
-    unsigned long long *bars = empty_bar + S;          // rows -> issuer: A, B, C; issuer -> rows: G3, S, O, Q; drain
+    unsigned long long *bars = empty_bar + S;          // rows -> issuer: A, B, C; issuer -> rows: G3, S, Q; drain
     StageDesc *descs = reinterpret_cast<StageDesc *>(bars + 8);
     volatile int *abort_flag = reinterpret_cast<volatile int *>(descs + S);
     uint32_t *tmem_slot = reinterpret_cast<uint32_t *>(const_cast<int *>(abort_flag) + 1);
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
     const uint32_t bar_A = smem_u32(bars + 0), bar_B = smem_u32(bars + 1), bar_C = smem_u32(bars + 2);
-    const uint32_t bar_G3 = smem_u32(bars + 3), bar_S = smem_u32(bars + 4), bar_O = smem_u32(bars + 5), bar_Q = smem_u32(bars + 6);
-    const uint32_t bar_drain = smem_u32(bars + 7);
+    const uint32_t bar_G3 = smem_u32(bars + 3), bar_S = smem_u32(bars + 4), bar_Q = smem_u32(bars + 5);
+    const uint32_t bar_drain = smem_u32(bars + 6);
     if (tid == 0) {
         for (int s = 0; s < S; ++s) { mbar_init(smem_u32(full_bar + s), 1); mbar_init(smem_u32(empty_bar + s), 1); }
         mbar_init(bar_A, kURows); mbar_init(bar_B, kURows); mbar_init(bar_C, kURows);
-        mbar_init(bar_G3, 1); mbar_init(bar_S, 1); mbar_init(bar_O, 1); mbar_init(bar_Q, 1); mbar_init(bar_drain, 1);
+        mbar_init(bar_G3, 1); mbar_init(bar_S, 1); mbar_init(bar_Q, 1); mbar_init(bar_drain, 1);
         *abort_flag = 0;
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     }
@@ -442,7 +464,6 @@ __global__ void __launch_bounds__(kUThreads, 2) block_umma_kernel(const __grid_c
                     pv(t_w, stage_of(u) + L.v, L.v_panel);
                     umma_commit(smem_u32(empty_bar + u % S));          // a factor unit's stage is free after G4
                 }
-                umma_commit(bar_O);
                 if (u + 2 < n_units) {
                     k2 = unit_kind(u + 2, ok);
                     if (!ok) break;
@@ -474,9 +495,10 @@ __global__ void __launch_bounds__(kUThreads, 2) block_umma_kernel(const __grid_c
         const uint32_t t_lane = tm + ((uint32_t)(warp * 32) << 16);
         const uint32_t t_qt = t_lane + kColQt, t_s = t_lane + kColS, t_w = t_lane + kColW, t_o = t_lane + kColO;
         RowSoftmax st{kNegInf, 0.f, kNegInf};
-        uint32_t ph_G3 = 0, ph_S = 0, ph_O = 0, ph_Q = 0;
+        uint32_t ph_G3 = 0, ph_S = 0, ph_Q = 0;
         bool ok = true;
         const float scale = geo.scale_log2e;
+        const bool full_tiles = geo.rank_k == 8 * NT && geo.rank_v == 8 * NT;     // then the rank bounds below are compile-time
         StageDesc cur{kKindDense, 0, 0, 0}, nxt{kKindDense, 0, 0, 0};
 #define PKV_ROWS_WAIT(bar, ph) { if (!wait_warp(bar, ph, abort_flag, limit)) { ok = false; break; } ph ^= 1; tc_fence_after(); }
 #define PKV_ROWS_ARRIVE(bar) { tc_fence_before(); mbar_arrive(bar); }
@@ -489,22 +511,20 @@ __global__ void __launch_bounds__(kUThreads, 2) block_umma_kernel(const __grid_c
                 if (cur.kind == kKindFactor) {
                     float sv[P];
                     tmem_ld<P>(t_s, reinterpret_cast<uint32_t *>(sv));
-                    fine = softmax_row<P, false>(sv, st, u > 0, t_s, t_o, bar_O, ph_O, o_seen, abort_flag, limit);
+                    fine = softmax_row<P, false>(sv, st, u > 0, t_s, t_o, bar_Q, ph_Q, o_seen, abort_flag, limit);
                 } else {
                     float sv[kDB];
                     tmem_ld<kDB>(t_s, reinterpret_cast<uint32_t *>(sv));
                     const int lim = cur.rows - max(0, hid - cur.after);
 #pragma unroll
                     for (int i = 0; i < kDB; ++i) sv[i] = i < lim ? sv[i] * scale : kMasked;
-                    fine = softmax_row<kDB, true>(sv, st, u > 0, t_s, t_o, bar_O, ph_O, o_seen, abort_flag, limit);
+                    fine = softmax_row<kDB, true>(sv, st, u > 0, t_s, t_o, bar_Q, ph_Q, o_seen, abort_flag, limit);
                 }
                 if (!fine) { ok = false; break; }
                 PKV_ROWS_ARRIVE(bar_A)
             }
-            if (u >= -1) {
-                if (!o_seen) PKV_ROWS_WAIT(bar_O, ph_O)          // (one wait per commit keeps the phases in step)
-                PKV_ROWS_WAIT(bar_Q, ph_Q)                       // G1(u+1) has written q~
-            }
+            if (u >= -1 && !o_seen) PKV_ROWS_WAIT(bar_Q, ph_Q)   // G4(u-1) has added to o, G1(u+1) has written q~
+
             if (u >= -1 && u + 1 < n_units) {
                 // ---- the next unit's descriptor; q~(u+1) as two bf16 terms -> hand-over B ----
                 const int s = (u + 1) % S;
@@ -514,13 +534,8 @@ __global__ void __launch_bounds__(kUThreads, 2) block_umma_kernel(const __grid_c
                 if (nxt.kind == kKindFactor) {      // columns past the rank are exact zeros
                     uint32_t rq[RP], hi[RP / 2], lo[RP / 2];
                     tmem_ld<RP>(t_qt, rq);
-#pragma unroll
-                    for (int k = 0; k < RP / 2; ++k) {
-                        const float x0 = 2 * k < geo.rank_k ? __uint_as_float(rq[2 * k]) * scale : 0.f;
-                        const float x1 = 2 * k + 1 < geo.rank_k ? __uint_as_float(rq[2 * k + 1]) * scale : 0.f;
-                        hi[k] = pack_bf16(x0, x1);
-                        lo[k] = pack_bf16(x0 - bf16lo_f(hi[k]), x1 - bf16hi_f(hi[k]));
-                    }
+                    if (full_tiles) split_terms<RP, 8 * NT>(rq, hi, lo, scale, 8 * NT);
+                    else split_terms<RP, RP>(rq, hi, lo, scale, geo.rank_k);
                     tmem_st<RP / 2>(t_qt, hi);
                     tmem_st<RP / 2>(t_qt + RP / 2, lo);
                     tmem_st_wait();
@@ -543,9 +558,8 @@ __global__ void __launch_bounds__(kUThreads, 2) block_umma_kernel(const __grid_c
                     uint32_t rw[RP], pk[RP / 2];
                     tmem_ld<RP>(t_w, rw);
                     const float c = exp2_fast(st.m - st.m_ref);
-#pragma unroll
-                    for (int k = 0; k < RP / 2; ++k)
-                        pk[k] = pack_bf16(2 * k < geo.rank_v ? __uint_as_float(rw[2 * k]) * c : 0.f, 2 * k + 1 < geo.rank_v ? __uint_as_float(rw[2 * k + 1]) * c : 0.f);
+                    if (full_tiles) scale_pack<RP, 8 * NT>(rw, pk, c, 8 * NT);
+                    else scale_pack<RP, RP>(rw, pk, c, geo.rank_v);
                     tmem_st<RP / 2>(t_w, pk);
                     tmem_st_wait();
                 }
@@ -554,7 +568,7 @@ __global__ void __launch_bounds__(kUThreads, 2) block_umma_kernel(const __grid_c
             cur = nxt;
         }
         if (ok) {                                                       // the last G4 | Gb
-            ok = wait_warp(bar_O, ph_O, abort_flag, limit);
+            ok = wait_warp(bar_Q, ph_Q, abort_flag, limit);
             tc_fence_after();
         }
 #undef PKV_ROWS_WAIT
