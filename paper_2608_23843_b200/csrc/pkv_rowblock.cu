@@ -61,6 +61,16 @@ __device__ __forceinline__ uint64_t umma_desc(uint32_t saddr, uint32_t lbo, uint
     return (uint64_t)((saddr >> 4) & 0x3FFF) | (uint64_t)((lbo >> 4) & 0x3FFF) << 16 | (uint64_t)((sbo >> 4) & 0x3FFF) << 32 |
            (uint64_t)1 << 46 | (uint64_t)layout << 61;
 }
+// The same descriptor `bytes` further on (a multiple of 16; the start-address field, in 16-byte units, is the lowest
+// field and the sum stays inside the 256 KB the field covers): one 32-bit add on the low word.
+__device__ __forceinline__ uint64_t umma_desc_step(uint64_t desc, uint32_t bytes) {
+    uint32_t lo, hi;
+    asm("mov.b64 {%0, %1}, %2;" : "=r"(lo), "=r"(hi) : "l"(desc));
+    lo += bytes >> 4;
+    uint64_t d;
+    asm("mov.b64 %0, {%1, %2};" : "=l"(d) : "r"(lo), "r"(hi));
+    return d;
+}
 // Instruction descriptor: bf16 x bf16 -> fp32, M x N, B operand K-major (0) or MN-major (1); A always K-major.
 __host__ __device__ constexpr uint32_t umma_idesc(int M, int N, int b_mn_major) {
     return (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)b_mn_major << 16) | ((uint32_t)(N >> 3) << 17) | ((uint32_t)(M >> 4) << 24);
@@ -394,6 +404,7 @@ __global__ void __launch_bounds__(kUThreads, 2) block_umma_kernel(const __grid_c
         // ------------------------------ products (one lane) ------------------------------
         if (elect_one()) {
             const uint32_t sq_a = smem_u32(sq);
+            const uint64_t dq0 = umma_desc(sq_a, 16, 1024, 2), dq1 = umma_desc(sq_a + kURows * 128, 16, 1024, 2);       // Q, channels 0-63 / 64-127
             const uint32_t t_qt = tm + kColQt, t_s = tm + kColS, t_w = tm + kColW, t_o = tm + kColO;
             uint32_t ph_A = 0, ph_B = 0, ph_C = 0;
             bool ok = true, o_valid = false;
@@ -401,16 +412,17 @@ __global__ void __launch_bounds__(kUThreads, 2) block_umma_kernel(const __grid_c
             // [128 x RP] = Q . (K side)^T: 8 steps of 16 channels; both operands K-major, 128-byte swizzle
             auto qk = [&](uint32_t t_dst, uint32_t kside, int panel) {
                 const uint32_t idesc = umma_idesc(128, RP, 0);
+                const uint64_t db0 = umma_desc(kside, 16, 1024, 2), db1 = umma_desc(kside + panel, 16, 1024, 2);
 #pragma unroll
                 for (int ks = 0; ks < 8; ++ks)
-                    umma_ss(t_dst, umma_desc(sq_a + (ks >> 2) * (kURows * 128) + (ks & 3) * 32, 16, 1024, 2),
-                            umma_desc(kside + (ks >> 2) * panel + (ks & 3) * 32, 16, 1024, 2), idesc, ks > 0);
+                    umma_ss(t_dst, umma_desc_step(ks < 4 ? dq0 : dq1, (ks & 3) * 32), umma_desc_step(ks < 4 ? db0 : db1, (ks & 3) * 32), idesc, ks > 0);
             };
             // o [128 x d] (+)= (rows of RP bf16 at t_src) . (V side): MN-major, two panels of 64 channels
             auto pv = [&](uint32_t t_src, uint32_t vside, int panel) {
+                const uint64_t dv = umma_desc(vside, panel, 1024, 2);
 #pragma unroll
                 for (int ks = 0; ks < RP / 16; ++ks)
-                    umma_ts(t_o, t_src + ks * 8, umma_desc(vside + ks * 2048, panel, 1024, 2), umma_idesc(128, 128, 1), o_valid || ks > 0);
+                    umma_ts(t_o, t_src + ks * 8, umma_desc_step(dv, ks * 2048), umma_idesc(128, 128, 1), o_valid || ks > 0);
                 o_valid = true;
             };
             // kind of a unit as the products see it: units without tokens run as dense units with every score masked
@@ -429,9 +441,10 @@ __global__ void __launch_bounds__(kUThreads, 2) block_umma_kernel(const __grid_c
                     tc_fence_after();
                     const uint32_t sb = stage_of(u);
                     if (k0 == kKindFactor) {
+                        const uint64_t da = umma_desc(sb + L.av, 16, 1024, 2);
 #pragma unroll
                         for (int ks = 0; ks < P / 16; ++ks)      // w = p . A_v, A_v^T in place (K-major)
-                            umma_ts(t_w, t_s + ks * 8, umma_desc(sb + L.av + ks * 32, 16, 1024, 2), umma_idesc(128, RP, 0), ks > 0);
+                            umma_ts(t_w, t_s + ks * 8, umma_desc_step(da, ks * 32), umma_idesc(128, RP, 0), ks > 0);
                     } else {
                         pv(t_s, sb + L.dv, L.d_panel);
                         umma_commit(smem_u32(empty_bar + u % S));      // a dense unit's stage is free after Gb
@@ -445,11 +458,12 @@ __global__ void __launch_bounds__(kUThreads, 2) block_umma_kernel(const __grid_c
                     tc_fence_after();
                     const uint32_t sb = stage_of(u + 1);
                     if (k1 == kKindFactor) {
+                        const uint64_t dak = umma_desc(sb + L.ak, 16, 1024, 2);
 #pragma unroll
                         for (int t = 0; t < 2; ++t)              // s = (q~_hi + q~_lo) . A_k^T, A_k^T in place (MN-major)
 #pragma unroll
                             for (int ks = 0; ks < RP / 16; ++ks)
-                                umma_ts(t_s, t_qt + t * (RP / 2) + ks * 8, umma_desc(sb + L.ak + ks * 2048, 16, 1024, 2),
+                                umma_ts(t_s, t_qt + t * (RP / 2) + ks * 8, umma_desc_step(dak, ks * 2048),
                                         umma_idesc(128, P, 1), (t | ks) > 0);
                     } else {
                         qk(t_s, sb + L.dk, L.d_panel);
