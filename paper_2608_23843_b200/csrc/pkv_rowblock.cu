@@ -348,9 +348,10 @@ __global__ void __launch_bounds__(kUThreads, 2) block_umma_kernel(const __grid_c
             const int *pt = a.page_table + ((long long)e.seq * geo.n_layers + a.layer) * geo.max_pages;
             bool ok = true;
             int u = 0;
-            for (; u < n_units; ++u) {
-                const int s = u % S;
-                if (u >= S && !wait_lane(smem_u32(empty_bar + s), ((u / S) - 1) & 1, abort_flag, limit)) { ok = false; break; }
+            // (stage and use count of a unit are counted along: S is not known at compile time and a division per
+            // unit is a hundred clocks of a single thread)
+            for (int s = 0, round = 0; u < n_units; ++u, s = s + 1 == S ? 0 : s + 1, round += s == 0) {
+                if (u >= S && !wait_lane(smem_u32(empty_bar + s), (round - 1) & 1, abort_flag, limit)) { ok = false; break; }
                 int page, blk, kind;
                 unit_to_page(geo, hu, u, page, blk, kind);
                 const int slot = pt[page];
@@ -408,7 +409,9 @@ __global__ void __launch_bounds__(kUThreads, 2) block_umma_kernel(const __grid_c
             const uint32_t t_qt = tm + kColQt, t_s = tm + kColS, t_w = tm + kColW, t_o = tm + kColO;
             uint32_t ph_A = 0, ph_B = 0, ph_C = 0;
             bool ok = true, o_valid = false;
-            auto stage_of = [&](int u) { return smem_u32(stages + (size_t)(u % S) * ustage); };
+            const uint32_t stages_a = smem_u32(stages);
+            int s0 = 0, s1 = 0, s2 = 0, round2 = 0;          // stages of the units u, u + 1, u + 2; times the stage of u + 2 has been used before
+            auto stage_at = [&](int s) { return stages_a + (uint32_t)(s * ustage); };
             // [128 x RP] = Q . (K side)^T: 8 steps of 16 channels; both operands K-major, 128-byte swizzle
             auto qk = [&](uint32_t t_dst, uint32_t kside, int panel) {
                 const uint32_t idesc = umma_idesc(128, RP, 0);
@@ -426,9 +429,8 @@ __global__ void __launch_bounds__(kUThreads, 2) block_umma_kernel(const __grid_c
                 o_valid = true;
             };
             // kind of a unit as the products see it: units without tokens run as dense units with every score masked
-            auto unit_kind = [&](int u, bool &good) -> int {
-                const int s = u % S;
-                if (!wait_lane(smem_u32(full_bar + s), (u / S) & 1, abort_flag, limit)) { good = false; return kKindDense; }
+            auto unit_kind = [&](int s, int round, bool &good) -> int {
+                if (!wait_lane(smem_u32(full_bar + s), round & 1, abort_flag, limit)) { good = false; return kKindDense; }
                 const StageDesc d = descs[s];
                 return d.kind == kKindFactor && d.rows > 0 ? kKindFactor : kKindDense;
             };
@@ -439,7 +441,7 @@ __global__ void __launch_bounds__(kUThreads, 2) block_umma_kernel(const __grid_c
                     if (!wait_lane(bar_A, ph_A, abort_flag, limit)) { ok = false; break; }
                     ph_A ^= 1;
                     tc_fence_after();
-                    const uint32_t sb = stage_of(u);
+                    const uint32_t sb = stage_at(s0);
                     if (k0 == kKindFactor) {
                         const uint64_t da = umma_desc(sb + L.av, 16, 1024, 2);
 #pragma unroll
@@ -447,7 +449,7 @@ __global__ void __launch_bounds__(kUThreads, 2) block_umma_kernel(const __grid_c
                             umma_ts(t_w, t_s + ks * 8, umma_desc_step(da, ks * 32), umma_idesc(128, RP, 0), ks > 0);
                     } else {
                         pv(t_s, sb + L.dv, L.d_panel);
-                        umma_commit(smem_u32(empty_bar + u % S));      // a dense unit's stage is free after Gb
+                        umma_commit(smem_u32(empty_bar + s0));         // a dense unit's stage is free after Gb
                     }
                     umma_commit(bar_G3);
                 }
@@ -456,7 +458,7 @@ __global__ void __launch_bounds__(kUThreads, 2) block_umma_kernel(const __grid_c
                     if (!wait_lane(bar_B, ph_B, abort_flag, limit)) { ok = false; break; }
                     ph_B ^= 1;
                     tc_fence_after();
-                    const uint32_t sb = stage_of(u + 1);
+                    const uint32_t sb = stage_at(s1);
                     if (k1 == kKindFactor) {
                         const uint64_t dak = umma_desc(sb + L.ak, 16, 1024, 2);
 #pragma unroll
@@ -475,16 +477,18 @@ __global__ void __launch_bounds__(kUThreads, 2) block_umma_kernel(const __grid_c
                 ph_C ^= 1;
                 tc_fence_after();
                 if (u >= 0 && k0 == kKindFactor) {
-                    pv(t_w, stage_of(u) + L.v, L.v_panel);
-                    umma_commit(smem_u32(empty_bar + u % S));          // a factor unit's stage is free after G4
+                    pv(t_w, stage_at(s0) + L.v, L.v_panel);
+                    umma_commit(smem_u32(empty_bar + s0));             // a factor unit's stage is free after G4
                 }
                 if (u + 2 < n_units) {
-                    k2 = unit_kind(u + 2, ok);
+                    k2 = unit_kind(s2, round2, ok);
                     if (!ok) break;
-                    if (k2 == kKindFactor) qk(t_qt, stage_of(u + 2) + L.k, L.k_panel);
+                    if (k2 == kKindFactor) qk(t_qt, stage_at(s2) + L.k, L.k_panel);
                 }
                 umma_commit(bar_Q);
                 k0 = k1; k1 = k2;
+                s0 = s1; s1 = s2;
+                if (++s2 == S) { s2 = 0; ++round2; }
             }
             if (!ok && !*abort_flag) { *abort_flag = 1; atomicAdd(a.status, 1); }
             // nothing of this CTA's may still be running on the tensor cores when tensor memory is given back
@@ -514,6 +518,7 @@ __global__ void __launch_bounds__(kUThreads, 2) block_umma_kernel(const __grid_c
         const float scale = geo.scale_log2e;
         const bool full_tiles = geo.rank_k == 8 * NT && geo.rank_v == 8 * NT;     // then the rank bounds below are compile-time
         StageDesc cur{kKindDense, 0, 0, 0}, nxt{kKindDense, 0, 0, 0};
+        int s_nxt = 0, round_nxt = 0;          // stage of the unit u + 1 and the times it has been used before
 #define PKV_ROWS_WAIT(bar, ph) { if (!wait_warp(bar, ph, abort_flag, limit)) { ok = false; break; } ph ^= 1; tc_fence_after(); }
 #define PKV_ROWS_ARRIVE(bar) { tc_fence_before(); mbar_arrive(bar); }
         for (int u = -2; u < n_units; ++u) {
@@ -541,8 +546,9 @@ __global__ void __launch_bounds__(kUThreads, 2) block_umma_kernel(const __grid_c
 
             if (u >= -1 && u + 1 < n_units) {
                 // ---- the next unit's descriptor; q~(u+1) as two bf16 terms -> hand-over B ----
-                const int s = (u + 1) % S;
-                if (!wait_warp(smem_u32(full_bar + s), ((u + 1) / S) & 1, abort_flag, limit)) { ok = false; break; }
+                const int s = s_nxt;
+                if (!wait_warp(smem_u32(full_bar + s), round_nxt & 1, abort_flag, limit)) { ok = false; break; }
+                if (++s_nxt == S) { s_nxt = 0; ++round_nxt; }
                 nxt = descs[s];
                 if (nxt.rows <= 0 || nxt.kind != kKindFactor) { nxt.kind = kKindDense; nxt.rows = max(0, min(nxt.rows, kDB)); }
                 if (nxt.kind == kKindFactor) {      // columns past the rank are exact zeros
