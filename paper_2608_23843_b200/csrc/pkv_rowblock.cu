@@ -208,12 +208,49 @@ __host__ __device__ inline StageLayout umma_layout(const Geometry &g) {
     return L;
 }
 
+// Two fp32 values in one 64-bit register, and the sm_100 instructions that work on both halves at once: the row
+// threads' arithmetic is issue-bound (two row warps per scheduler), so halving the instruction count of the
+// subtractions, sums and scalings shows.  Likewise the three-input maximum.
+__device__ __forceinline__ uint64_t f2_pack(float lo, float hi) {
+    uint64_t v;
+    asm("mov.b64 %0, {%1, %2};" : "=l"(v) : "f"(lo), "f"(hi));
+    return v;
+}
+__device__ __forceinline__ void f2_unpack(uint64_t v, float &lo, float &hi) { asm("mov.b64 {%0, %1}, %2;" : "=f"(lo), "=f"(hi) : "l"(v)); }
+__device__ __forceinline__ uint64_t f2_add(uint64_t a, uint64_t b) {
+    uint64_t d;
+    asm("add.rn.f32x2 %0, %1, %2;" : "=l"(d) : "l"(a), "l"(b));
+    return d;
+}
+__device__ __forceinline__ uint64_t f2_sub(uint64_t a, uint64_t b) {
+    uint64_t d;
+    asm("sub.rn.f32x2 %0, %1, %2;" : "=l"(d) : "l"(a), "l"(b));
+    return d;
+}
+__device__ __forceinline__ uint64_t f2_mul(uint64_t a, uint64_t b) {
+    uint64_t d;
+    asm("mul.rn.f32x2 %0, %1, %2;" : "=l"(d) : "l"(a), "l"(b));
+    return d;
+}
+__device__ __forceinline__ float max3(float a, float b, float c) {
+    float d;
+    asm("max.f32 %0, %1, %2, %3;" : "=f"(d) : "f"(a), "f"(b), "f"(c));
+    return d;
+}
+
 // RP fp32 values x (a row of q~ or w) times `scale`, as bf16 pairs; columns from `rank` on become exact zeros.  The
 // first KNOWN columns are known to lie below the rank (no test), the rest are tested against it.
 template <int RP, int KNOWN>
 __device__ __forceinline__ void scale_pack(const uint32_t *x, uint32_t *pk, float scale, int rank) {
 #pragma unroll
+    const uint64_t sc2 = f2_pack(scale, scale);
     for (int k = 0; k < RP / 2; ++k) {
+        if (KNOWN < RP && 2 * k + 1 < KNOWN) {            // the ranks fill their tiles: this pair lies below the rank
+            float y0, y1;
+            f2_unpack(f2_mul(f2_pack(__uint_as_float(x[2 * k]), __uint_as_float(x[2 * k + 1])), sc2), y0, y1);
+            pk[k] = pack_bf16(y0, y1);
+            continue;
+        }
         const bool in0 = 2 * k < KNOWN && 2 * k < rank, in1 = 2 * k + 1 < KNOWN && 2 * k + 1 < rank;
         pk[k] = pack_bf16(in0 ? __uint_as_float(x[2 * k]) * scale : 0.f, in1 ? __uint_as_float(x[2 * k + 1]) * scale : 0.f);
     }
@@ -222,7 +259,17 @@ __device__ __forceinline__ void scale_pack(const uint32_t *x, uint32_t *pk, floa
 template <int RP, int KNOWN>
 __device__ __forceinline__ void split_terms(const uint32_t *x, uint32_t *hi, uint32_t *lo, float scale, int rank) {
 #pragma unroll
+    const uint64_t sc2 = f2_pack(scale, scale);
     for (int k = 0; k < RP / 2; ++k) {
+        if (KNOWN < RP && 2 * k + 1 < KNOWN) {            // the ranks fill their tiles: this pair lies below the rank
+            const uint64_t y = f2_mul(f2_pack(__uint_as_float(x[2 * k]), __uint_as_float(x[2 * k + 1])), sc2);
+            float y0, y1, e0, e1;
+            f2_unpack(y, y0, y1);
+            hi[k] = pack_bf16(y0, y1);
+            f2_unpack(f2_sub(y, f2_pack(bf16lo_f(hi[k]), bf16hi_f(hi[k]))), e0, e1);
+            lo[k] = pack_bf16(e0, e1);
+            continue;
+        }
         const bool in0 = 2 * k < KNOWN && 2 * k < rank, in1 = 2 * k + 1 < KNOWN && 2 * k + 1 < rank;
         const float x0 = in0 ? __uint_as_float(x[2 * k]) * scale : 0.f, x1 = in1 ? __uint_as_float(x[2 * k + 1]) * scale : 0.f;
         hi[k] = pack_bf16(x0, x1);
@@ -240,8 +287,12 @@ __device__ __forceinline__ bool softmax_row(float *sv, RowSoftmax &st, bool o_va
                                             uint32_t &ph_Q, bool &o_seen, volatile int *abort_flag, long long limit) {
     float mx4[4] = {sv[0], sv[1], sv[2], sv[3]};           // four chains: a thread has no other work to hide latencies with
 #pragma unroll
-    for (int i = 4; i < N; ++i) mx4[i & 3] = fmaxf(mx4[i & 3], sv[i]);
-    const float mx = fmaxf(fmaxf(mx4[0], mx4[1]), fmaxf(mx4[2], mx4[3]));
+    for (int i = 4; i + 8 <= N; i += 8)
+#pragma unroll
+        for (int c = 0; c < 4; ++c) mx4[c] = max3(mx4[c], sv[i + c], sv[i + 4 + c]);
+#pragma unroll
+    for (int i = 4 + ((N - 4) / 8) * 8; i < N; ++i) mx4[i & 3] = fmaxf(mx4[i & 3], sv[i]);
+    const float mx = fmaxf(max3(mx4[0], mx4[1], mx4[2]), mx4[3]);
     if (mx > st.m) { st.l *= exp2_fast(st.m - mx); st.m = mx; }
     if (!o_valid) {
         st.m_ref = st.m;
@@ -264,18 +315,22 @@ __device__ __forceinline__ bool softmax_row(float *sv, RowSoftmax &st, bool o_va
             tmem_st32(t_o + 32 * c, r);
         }
     }
-    float sum4[4] = {0.f, 0.f, 0.f, 0.f};
-    const float m = st.m;
+    uint64_t sum2[4] = {0ull, 0ull, 0ull, 0ull};         // (0.f, 0.f) each
+    const uint64_t m2 = f2_pack(st.m, st.m);
     uint32_t pk[N / 2];
 #pragma unroll
     for (int e = 0; e < N / 2; ++e) {
-        const float p0 = exp2_fast(sv[2 * e] - m), p1 = exp2_fast(sv[2 * e + 1] - m);
-        sum4[e & 3] += p0 + p1;
+        float d0, d1;
+        f2_unpack(f2_sub(f2_pack(sv[2 * e], sv[2 * e + 1]), m2), d0, d1);
+        const float p0 = exp2_fast(d0), p1 = exp2_fast(d1);
+        sum2[e & 3] = f2_add(sum2[e & 3], f2_pack(p0, p1));
         pk[e] = pack_bf16(p0, p1);
     }
     tmem_st<N / 2>(t_s, pk);
     tmem_st_wait();
-    st.l += (sum4[0] + sum4[1]) + (sum4[2] + sum4[3]);
+    float s0, s1;
+    f2_unpack(f2_add(f2_add(sum2[0], sum2[1]), f2_add(sum2[2], sum2[3])), s0, s1);
+    st.l += s0 + s1;
     return true;
 }
 
