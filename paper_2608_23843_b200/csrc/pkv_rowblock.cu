@@ -239,13 +239,14 @@ __device__ __forceinline__ float max3(float a, float b, float c) {
 }
 
 // RP fp32 values x (a row of q~ or w) times `scale`, as bf16 pairs; columns from `rank` on become exact zeros.  The
-// first KNOWN columns are known to lie below the rank (no test), the rest are tested against it.
-template <int RP, int KNOWN>
+// kExact: the rank is KNOWN, a compile-time value (the ranks fill their tiles); otherwise KNOWN = RP and every column is
+// tested against `rank`.
+template <int RP, int KNOWN, bool kExact>
 __device__ __forceinline__ void scale_pack(const uint32_t *x, uint32_t *pk, float scale, int rank) {
 #pragma unroll
     const uint64_t sc2 = f2_pack(scale, scale);
     for (int k = 0; k < RP / 2; ++k) {
-        if (KNOWN < RP && 2 * k + 1 < KNOWN) {            // the ranks fill their tiles: this pair lies below the rank
+        if (kExact && 2 * k + 1 < KNOWN) {                // this pair lies below the rank
             float y0, y1;
             f2_unpack(f2_mul(f2_pack(__uint_as_float(x[2 * k]), __uint_as_float(x[2 * k + 1])), sc2), y0, y1);
             pk[k] = pack_bf16(y0, y1);
@@ -256,12 +257,12 @@ __device__ __forceinline__ void scale_pack(const uint32_t *x, uint32_t *pk, floa
     }
 }
 // The same with the rounding error of each pair as a second bf16 term (hi + lo carries about 16 bits).
-template <int RP, int KNOWN>
+template <int RP, int KNOWN, bool kExact>
 __device__ __forceinline__ void split_terms(const uint32_t *x, uint32_t *hi, uint32_t *lo, float scale, int rank) {
 #pragma unroll
     const uint64_t sc2 = f2_pack(scale, scale);
     for (int k = 0; k < RP / 2; ++k) {
-        if (KNOWN < RP && 2 * k + 1 < KNOWN) {            // the ranks fill their tiles: this pair lies below the rank
+        if (kExact && 2 * k + 1 < KNOWN) {                // this pair lies below the rank
             const uint64_t y = f2_mul(f2_pack(__uint_as_float(x[2 * k]), __uint_as_float(x[2 * k + 1])), sc2);
             float y0, y1, e0, e1;
             f2_unpack(y, y0, y1);
@@ -609,8 +610,8 @@ __global__ void __launch_bounds__(kUThreads, 2) block_umma_kernel(const __grid_c
                 if (nxt.kind == kKindFactor) {      // columns past the rank are exact zeros
                     uint32_t rq[RP], hi[RP / 2], lo[RP / 2];
                     tmem_ld<RP>(t_qt, rq);
-                    if (full_tiles) split_terms<RP, 8 * NT>(rq, hi, lo, scale, 8 * NT);
-                    else split_terms<RP, RP>(rq, hi, lo, scale, geo.rank_k);
+                    if (full_tiles) split_terms<RP, 8 * NT, true>(rq, hi, lo, scale, 8 * NT);
+                    else split_terms<RP, RP, false>(rq, hi, lo, scale, geo.rank_k);
                     tmem_st<RP / 2>(t_qt, hi);
                     tmem_st<RP / 2>(t_qt + RP / 2, lo);
                     tmem_st_wait();
@@ -633,8 +634,8 @@ __global__ void __launch_bounds__(kUThreads, 2) block_umma_kernel(const __grid_c
                     uint32_t rw[RP], pk[RP / 2];
                     tmem_ld<RP>(t_w, rw);
                     const float c = exp2_fast(st.m - st.m_ref);
-                    if (full_tiles) scale_pack<RP, 8 * NT>(rw, pk, c, 8 * NT);
-                    else scale_pack<RP, RP>(rw, pk, c, geo.rank_v);
+                    if (full_tiles) scale_pack<RP, 8 * NT, true>(rw, pk, c, 8 * NT);
+                    else scale_pack<RP, RP, false>(rw, pk, c, geo.rank_v);
                     tmem_st<RP / 2>(t_w, pk);
                     tmem_st_wait();
                 }
