@@ -798,7 +798,7 @@ def main():
                                            "block_tc_kernel<P=%d, rank tiles=%%d> (mma.sync, 64 query rows per CTA)" % P_) % ((rank + 7) // 8),
                                 "achieved": tach, "peak": tpeak, "unit": "TFLOP/s", "frac": tach / tpeak,
                                 "peak_source": tsrc + ("; the products are small (N = 32 to 128 per instruction, four dependent products per "
-                                                       "page through the row threads): ncu shows the tensor pipe about 25 % busy" if umma else
+                                                       "page through the row threads): ncu shows the tensor pipe about 30 % busy" if umma else
                                                        "; ncu showed the mma.sync pipe 50 % busy at this rate"),
                                 "traffic": None, "launch_us": launch_ms * 1e3, "algorithmic_flops_per_launch": flops}
         if not args.no_cpu_baseline and world == 1 and QL == 1 and not args.global_rank:
