@@ -1585,9 +1585,9 @@ __global__ void __launch_bounds__(kBlockThreads, 2) block_tc_kernel(const __grid
         const int *pt = a.page_table + ((long long)e.seq * geo.n_layers + a.layer) * geo.max_pages;
         bool ok = true;
         int u = 0;
-        for (; u < n_units && ok; ++u) {
-            const int s = u % S;
-            if (u >= S && !mbar_wait(smem_u32(empty_bar + s), ((u / S) - 1) & 1)) { ok = false; break; }
+        // (stage and use count of a unit are counted along: the number of stages is not known at compile time)
+        for (int s = 0, round = 0; u < n_units && ok; ++u, s = s + 1 == S ? 0 : s + 1, round += s == 0) {
+            if (u >= S && !mbar_wait(smem_u32(empty_bar + s), (round - 1) & 1)) { ok = false; break; }
             int page, blk, kind;
             unit_to_page(geo, hu, u, page, blk, kind);
             const int slot = pt[page];
@@ -1657,11 +1657,10 @@ __global__ void __launch_bounds__(kBlockThreads, 2) block_tc_kernel(const __grid
     st.m[0] = st.m[1] = kNegInf;
     st.l[0] = st.l[1] = 0.f;
     bool ok = true;
-    for (int u = 0; u < n_units; ++u) {
-        const int s = u % S;
+    for (int u = 0, s = 0, round = 0; u < n_units; ++u, s = s + 1 == S ? 0 : s + 1, round += s == 0) {
         // The only way out is this warp's own wait running out: if the producer gave up, every warp ends up at the
         // same unarmed unit, so no warp is left alone at the block barrier below.
-        if (!mbar_wait(smem_u32(full_bar + s), (u / S) & 1)) {
+        if (!mbar_wait(smem_u32(full_bar + s), round & 1)) {
             ok = false;
             if (lane == 0) { *abort_flag = 1; atomicAdd(a.status, 1); }
             break;
