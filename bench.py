@@ -48,6 +48,9 @@ WORKLOADS = {
     # dense window of that size) are the queries.  Use with --q-len 2048 (pkv_decode_attention_multi).
     "prefill_chunk_llama3_8b_32k": dict(n_layers=2, layers_per_step=1, n_kv_heads=8, n_q_heads=32, batch=1, T=32768,
                                         rank=24, sink=64, recent=2048, ragged=False, outliers=0.0),
+    # The same with the paper's default page shape (Section 4.1: P = 32, ranks (16, 14)) on the Qwen3-8B layer shape.
+    "prefill_chunk_qwen3_8b_16k_p32": dict(n_layers=2, layers_per_step=1, n_kv_heads=8, n_q_heads=32, batch=1, T=16384,
+                                           rank=16, rank_v=14, page=32, sink=32, recent=2048, ragged=False, outliers=0.0),
     # tiny single decode step (L2-resident; latency only)
     "tiny": dict(n_layers=1, n_kv_heads=1, n_q_heads=4, batch=1, T=1024, rank=16, sink=64, recent=128,
                  ragged=False, outliers=0.0),
@@ -790,11 +793,11 @@ def main():
                 flops += QL * Hq * (nf_ * 2 * (128 * rank + rank * P_ + P_ * rv_ + rv_ * 128) + dense_tok * 4 * 128)
             tpeak, tsrc = _tensor_peak()
             tach = flops / (launch_ms * 1e-3) / 1e12
-            # the library's own rule (row_block_umma_supported): tcgen05 kernel for P = 64, bf16 factors, even ranks;
+            # the library's own rule (row_block_umma_supported): tcgen05 kernel for P = 64 or 32, bf16 factors, even ranks;
             # the mma.sync kernel otherwise or when decode_variant 3 pins it
-            umma = args.decode_variant == 0 and P_ == 64 and rank % 2 == 0 and rv_ % 2 == 0 and rv_ <= rank
+            umma = args.decode_variant == 0 and P_ in (32, 64) and rank % 2 == 0 and rv_ % 2 == 0 and rv_ <= rank
             line["roofline"] = {"bound": "tensor",
-                                "kernel": ("block_umma_kernel<rank tiles=%d> (tcgen05, 128 query rows per CTA)" if umma else
+                                "kernel": (("block_umma_kernel<P=%d, rank tiles=%%d> (tcgen05, 128 query rows per CTA)" % P_) if umma else
                                            "block_tc_kernel<P=%d, rank tiles=%%d> (mma.sync, 64 query rows per CTA)" % P_) % ((rank + 7) // 8),
                                 "achieved": tach, "peak": tpeak, "unit": "TFLOP/s", "frac": tach / tpeak,
                                 "peak_source": tsrc + ("; the products are small (N = 32 to 128 per instruction, four dependent products per "

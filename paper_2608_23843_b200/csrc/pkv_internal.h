@@ -142,12 +142,12 @@ cudaError_t launch_compress(const Geometry &geo, const unsigned char *dense_pool
                             const int2 *worklist, int n_entries, int *status, cudaStream_t st);
 cudaError_t launch_decode(const DecodeArgs &a, int n_segs, cudaStream_t st);
 constexpr int kRowBlock = 64;          // query rows (token x query head) per CTA of the mma.sync row-block kernel
-// tcgen05 row-block kernel (pkv_rowblock.cu): 128 query rows per CTA; P = 64, bf16 page-wise factors, rank_k a multiple of 8
+// tcgen05 row-block kernel (pkv_rowblock.cu): 128 query rows per CTA; P = 64 or 32, bf16 page-wise factors, even ranks
 bool row_block_umma_supported(const Geometry &geo);
 cudaError_t row_block_umma_setup();
 // TMA descriptors of the pools for that kernel (B factors; dense K / V); valid = 0 where the shape is not covered or
 // the driver offers no encoder, and the mma.sync kernel is used instead
-struct RowBlockMaps { CUtensorMap bk, bv, dense; int valid; };
+struct RowBlockMaps { CUtensorMap bk, bv, bk_half, bv_half, dense; int valid; };   // *_half: origin 128 bytes into the pool
 void row_block_make_maps(const Geometry &geo, const void *factor_pool, const void *dense_pool, RowBlockMaps *maps);
 cudaError_t launch_decode_blocks_umma(const DecodeArgs &a, int n_seqs, const RowBlockMaps &maps, cudaStream_t st);
 cudaError_t launch_decode_blocks(const DecodeArgs &a, int n_seqs, const RowBlockMaps &maps, cudaStream_t st);

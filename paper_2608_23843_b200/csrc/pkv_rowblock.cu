@@ -44,8 +44,12 @@ constexpr uint32_t kColQt = 0, kColS = 32, kColW = 96, kColO = 128, kTmemCols = 
 // Rows of a dense block, and what a rank is padded to in the products (16 or 32):
 __host__ __device__ inline int umma_part_rows(const Geometry &g) { return g.rank_tiles <= 2 ? 16 : 32; }
 constexpr int kUStagePad = 1024;
+// bytes of an A^T part of a stage: rows of 2 P bytes, the rank rounded up to 8 rows, the part to 1024 bytes (the parts
+// behind it hold 128-byte-swizzled panels, whose pattern repeats every 1024 bytes)
+__host__ __device__ inline int umma_a_bytes(const Geometry &g, int rank) { return ((((rank + 7) & ~7) * 2 * g.page) + 1023) & ~1023; }
 __host__ __device__ inline int umma_stage_bytes(const Geometry &g) {
-    const int factor = 3 * 128 * (((g.rank_k + 7) & ~7) + ((g.rank_v + 7) & ~7)), dense = 4 * umma_part_rows(g) * 128;
+    const int factor = umma_a_bytes(g, g.rank_k) + umma_a_bytes(g, g.rank_v) + 2 * 128 * (((g.rank_k + 7) & ~7) + ((g.rank_v + 7) & ~7));
+    const int dense = 4 * umma_part_rows(g) * 128;
     return ((factor > dense ? factor : dense) + 1023) & ~1023;
 }
 // stages: the units u, u + 1 and u + 2 are in use at any time; the rest is the copies' lead
@@ -190,7 +194,7 @@ struct RowSoftmax {
 constexpr float kFrameLag = 8.f;
 
 // Byte offsets of a unit's parts inside its stage.  A factor unit is
-//     [A_k^T: r_k rows][K side: 2 panels of r_k rows][A_v^T: r_v rows][V side: 2 panels of r_v rows]    (128-byte rows)
+//     [A_k^T: r_k rows of 2 P bytes][K side: 2 panels of r_k rows][A_v^T: r_v rows][V side: 2 panels of r_v rows]    (panels: 128-byte rows)
 // with every part rounded up to a multiple of 8 rows, so a product that reads a rank padded to 16 or 32 rows reads
 // rows no copy of this unit wrote (what an earlier unit left there, or the zeros of the start) and runs into the
 // next part: finite data either way, multiplied by exact zeros (or producing columns that are replaced by exact
@@ -202,8 +206,8 @@ struct StageLayout {
 __host__ __device__ inline StageLayout umma_layout(const Geometry &g) {
     StageLayout L;
     const int rk = (g.rank_k + 7) & ~7, rv = (g.rank_v + 7) & ~7;        // parts start on 1024-byte boundaries
-    L.ak = 0; L.k = rk * 128; L.k_panel = rk * 128;
-    L.av = 3 * rk * 128; L.v = L.av + rv * 128; L.v_panel = rv * 128;
+    L.ak = 0; L.k = umma_a_bytes(g, g.rank_k); L.k_panel = rk * 128;
+    L.av = L.k + 2 * rk * 128; L.v = L.av + umma_a_bytes(g, g.rank_v); L.v_panel = rv * 128;
     L.d_panel = umma_part_rows(g) * 128; L.dk = 0; L.dv = 2 * L.d_panel;
     return L;
 }
@@ -335,12 +339,13 @@ __device__ __forceinline__ bool softmax_row(float *sv, RowSoftmax &st, bool o_va
     return true;
 }
 
-template <int NT>
+template <int P, int NT>
 __global__ void __launch_bounds__(kUThreads, 2) block_umma_kernel(const __grid_constant__ DecodeArgs a,
-                                                                  const __grid_constant__ CUtensorMap map_bk,
-                                                                  const __grid_constant__ CUtensorMap map_bv,
-                                                                  const __grid_constant__ CUtensorMap map_dense) {
-    constexpr int P = 64, RP = NT <= 2 ? 16 : 32, kDB = kDenseBlock<P, NT, 0>;
+                                                                  const __grid_constant__ RowBlockMaps maps) {
+    constexpr int RP = NT <= 2 ? 16 : 32, kDB = kDenseBlock<P, NT, 0>;
+    // A^T rows are 2 P bytes: the 128-byte swizzle for P = 64, the 64-byte one (8 rows = 512 bytes) for P = 32 - in both
+    // cases the XOR the pages are stored with
+    constexpr uint32_t kASwizzle = P == 64 ? 2 : 4, kAGroup = 8 * 2 * P;
     static_assert(kDB == RP, "dense blocks and padded ranks have the same number of rows");
     const Geometry &geo = a.geo;
     const StageLayout L = umma_layout(geo);
@@ -429,23 +434,27 @@ __global__ void __launch_bounds__(kUThreads, 2) block_umma_kernel(const __grid_c
                 if (kind == kKindFactor) {
                     const long long off = (long long)slot * geo.factor_slot_bytes + (long long)head * geo.blob_bytes;
                     const unsigned char *src = a.factor_pool + off;
-                    const int yk = (int)((off + geo.bk_off) >> 8), yv = (int)((off + geo.bv_off) >> 8);     // pool rows of 256 bytes
+                    // B_k, B_v as rows of the pool seen in 256-byte rows; a part that starts half a row in (the ranks
+                    // of P = 32 pages allow it) goes through the map whose origin is 128 bytes further on
+                    const long long ok_ = off + geo.bk_off, ov_ = off + geo.bv_off;
+                    const CUtensorMap *mk = (ok_ & 128) ? &maps.bk_half : &maps.bk, *mv = (ov_ & 128) ? &maps.bv_half : &maps.bv;
+                    const int yk = (int)(ok_ >> 8), yv = (int)(ov_ >> 8);
                     mbar_arrive_expect_tx(bar, geo.blob_bytes);
-                    bulk_g2s_keep(dst + L.ak, src + geo.ak_off, geo.rank_k * 128, bar);
-                    bulk_g2s_keep(dst + L.av, src + geo.av_off, geo.rank_v * 128, bar);
-                    tma_box(dst + L.k, &map_bk, 0, yk, bar);
-                    tma_box(dst + L.k + L.k_panel, &map_bk, 64, yk, bar);
-                    tma_box(dst + L.v, &map_bv, 0, yv, bar);
-                    tma_box(dst + L.v + L.v_panel, &map_bv, 64, yv, bar);
+                    bulk_g2s_keep(dst + L.ak, src + geo.ak_off, geo.rank_k * 2 * P, bar);
+                    bulk_g2s_keep(dst + L.av, src + geo.av_off, geo.rank_v * 2 * P, bar);
+                    tma_box(dst + L.k, mk, 0, yk, bar);
+                    tma_box(dst + L.k + L.k_panel, mk, 64, yk, bar);
+                    tma_box(dst + L.v, mv, 0, yv, bar);
+                    tma_box(dst + L.v + L.v_panel, mv, 64, yv, bar);
                 } else if (rows > 0) {
                     // whole blocks: rows past the sequence's end hold whatever the pool holds; the scores there are
                     // masked and the row threads clear those rows
                     const int y = (int)(((long long)slot * geo.dense_slot_bytes + (long long)head * geo.dense_head_bytes) >> 8) + blk * kDB;
                     mbar_arrive_expect_tx(bar, 4 * L.d_panel);
-                    tma_box(dst + L.dk, &map_dense, 0, y, bar);
-                    tma_box(dst + L.dk + L.d_panel, &map_dense, 64, y, bar);
-                    tma_box(dst + L.dv, &map_dense, 0, y + P, bar);
-                    tma_box(dst + L.dv + L.d_panel, &map_dense, 64, y + P, bar);
+                    tma_box(dst + L.dk, &maps.dense, 0, y, bar);
+                    tma_box(dst + L.dk + L.d_panel, &maps.dense, 64, y, bar);
+                    tma_box(dst + L.dv, &maps.dense, 0, y + P, bar);
+                    tma_box(dst + L.dv + L.d_panel, &maps.dense, 64, y + P, bar);
                 } else {
                     mbar_arrive(bar);
                 }
@@ -499,7 +508,7 @@ __global__ void __launch_bounds__(kUThreads, 2) block_umma_kernel(const __grid_c
                     tc_fence_after();
                     const uint32_t sb = stage_at(s0);
                     if (k0 == kKindFactor) {
-                        const uint64_t da = umma_desc(sb + L.av, 16, 1024, 2);
+                        const uint64_t da = umma_desc(sb + L.av, 16, kAGroup, kASwizzle);
 #pragma unroll
                         for (int ks = 0; ks < P / 16; ++ks)      // w = p . A_v, A_v^T in place (K-major)
                             umma_ts(t_w, t_s + ks * 8, umma_desc_step(da, ks * 32), umma_idesc(128, RP, 0), ks > 0);
@@ -516,12 +525,12 @@ __global__ void __launch_bounds__(kUThreads, 2) block_umma_kernel(const __grid_c
                     tc_fence_after();
                     const uint32_t sb = stage_at(s1);
                     if (k1 == kKindFactor) {
-                        const uint64_t dak = umma_desc(sb + L.ak, 16, 1024, 2);
+                        const uint64_t dak = umma_desc(sb + L.ak, 16, kAGroup, kASwizzle);
 #pragma unroll
                         for (int t = 0; t < 2; ++t)              // s = (q~_hi + q~_lo) . A_k^T, A_k^T in place (MN-major)
 #pragma unroll
                             for (int ks = 0; ks < RP / 16; ++ks)
-                                umma_ts(t_s, t_qt + t * (RP / 2) + ks * 8, umma_desc_step(dak, ks * 2048),
+                                umma_ts(t_s, t_qt + t * (RP / 2) + ks * 8, umma_desc_step(dak, ks * 2 * kAGroup),
                                         umma_idesc(128, P, 1), (t | ks) > 0);
                     } else {
                         qk(t_s, sb + L.dk, L.d_panel);
@@ -693,23 +702,28 @@ size_t umma_smem_bytes(const Geometry &g) {
 }  // namespace
 
 bool row_block_umma_supported(const Geometry &g) {
-    // A^T rows of 128 bytes (P = 64); every part of a blob on a 256-byte row of the pool (the tiled copies address
-    // the pools in such rows): even ranks
-    return g.page == 64 && g.factor_bits == 16 && g.global_rank == 0 && g.rank_k % 2 == 0 && g.rank_v % 2 == 0 &&
-           g.rank_v <= g.rank_k && g.rank_tiles >= 1 && g.rank_tiles <= 4 && g.bk_off % 256 == 0 && g.bv_off % 256 == 0 &&
-           g.blob_bytes % 256 == 0 && umma_smem_bytes(g) <= (size_t)kSmemBudget / 2;
+    // A^T rows of 128 or 64 bytes (P = 64, 32: the swizzles the tensor cores know for such rows); every part of a blob
+    // on a 128-byte boundary of the pool (the tiled copies address the pools in 256-byte rows, from either of two
+    // origins 128 bytes apart): even ranks
+    return (g.page == 64 || g.page == 32) && g.factor_bits == 16 && g.global_rank == 0 && g.rank_k % 2 == 0 && g.rank_v % 2 == 0 &&
+           g.rank_v <= g.rank_k && g.rank_tiles >= 1 && g.rank_tiles <= 4 && g.bk_off % 128 == 0 && g.bv_off % 128 == 0 &&
+           g.blob_bytes % 128 == 0 && g.factor_slot_bytes % 128 == 0 && umma_smem_bytes(g) <= (size_t)kSmemBudget / 2;
 }
+
+#define PKV_FOR_EACH_UMMA_SHAPE(X) X(64, 1) X(64, 2) X(64, 3) X(64, 4) X(32, 1) X(32, 2) X(32, 3) X(32, 4)
 
 cudaError_t row_block_umma_setup() {
     cudaError_t e;
-    if ((e = cudaFuncSetAttribute(block_umma_kernel<1>, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBudget / 2)) != cudaSuccess) return e;
-    if ((e = cudaFuncSetAttribute(block_umma_kernel<2>, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBudget / 2)) != cudaSuccess) return e;
-    if ((e = cudaFuncSetAttribute(block_umma_kernel<3>, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBudget / 2)) != cudaSuccess) return e;
-    return cudaFuncSetAttribute(block_umma_kernel<4>, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBudget / 2);
+#define PKV_UMMA_SETUP(P, NT) \
+    if ((e = cudaFuncSetAttribute(block_umma_kernel<P, NT>, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBudget / 2)) != cudaSuccess) return e;
+    PKV_FOR_EACH_UMMA_SHAPE(PKV_UMMA_SETUP)
+#undef PKV_UMMA_SETUP
+    return cudaSuccess;
 }
 
-// Tensor maps of the two pools seen as matrices of 256-byte rows (128 bf16), box = 64 channels x `rows`.  The
-// encoder is a driver entry point; it is looked up at run time so that the library does not link against the driver.
+// Tensor maps of the two pools seen as matrices of 256-byte rows (128 bf16), box = 64 channels x `rows`; for the factor
+// pool a second pair whose origin lies 128 bytes further on (see the copy lane).  The encoder is a driver entry
+// point; it is looked up at run time so that the library does not link against the driver.
 void row_block_make_maps(const Geometry &g, const void *factor_pool, const void *dense_pool, RowBlockMaps *maps) {
     typedef CUresult (*EncodeTiled)(CUtensorMap *, CUtensorMapDataType, cuuint32_t, void *, const cuuint64_t *, const cuuint64_t *,
                                     const cuuint32_t *, const cuuint32_t *, CUtensorMapInterleave, CUtensorMapSwizzle,
@@ -737,10 +751,16 @@ void row_block_make_maps(const Geometry &g, const void *factor_pool, const void 
     if (!make(&maps->dense, dense_pool, (long long)g.n_dense_slots * g.dense_slot_bytes, rb)) return;
     if (factor_pool && g.n_factor_slots > 0) {
         const long long bytes = (long long)g.n_factor_slots * g.factor_slot_bytes;
+        const unsigned char *half = static_cast<const unsigned char *>(factor_pool) + 128;
         if (!make(&maps->bk, factor_pool, bytes, g.rank_k) || !make(&maps->bv, factor_pool, bytes, g.rank_v)) return;
+        if (bytes >= 512) {
+            if (!make(&maps->bk_half, half, bytes - 128, g.rank_k) || !make(&maps->bv_half, half, bytes - 128, g.rank_v)) return;
+        } else {
+            maps->bk_half = maps->bk;
+            maps->bv_half = maps->bv;
+        }
     } else {
-        maps->bk = maps->dense;          // no factor pages: never used
-        maps->bv = maps->dense;
+        maps->bk = maps->bv = maps->bk_half = maps->bv_half = maps->dense;          // no factor pages: never used
     }
     maps->valid = 1;
 }
@@ -751,13 +771,12 @@ cudaError_t launch_decode_blocks_umma(const DecodeArgs &a, int n_seqs, const Row
     const long long n_ctas = (long long)n_seqs * a.geo.n_kv_heads * n_blk;
     if (!maps.valid || !row_block_umma_supported(a.geo) || n_ctas <= 0 || n_ctas > 0x7fffffffLL) return cudaErrorInvalidValue;
     const size_t smem = umma_smem_bytes(a.geo);
-    switch (a.geo.rank_tiles) {
-        case 1: block_umma_kernel<1><<<(unsigned)n_ctas, kUThreads, smem, st>>>(a, maps.bk, maps.bv, maps.dense); break;
-        case 2: block_umma_kernel<2><<<(unsigned)n_ctas, kUThreads, smem, st>>>(a, maps.bk, maps.bv, maps.dense); break;
-        case 3: block_umma_kernel<3><<<(unsigned)n_ctas, kUThreads, smem, st>>>(a, maps.bk, maps.bv, maps.dense); break;
-        default: block_umma_kernel<4><<<(unsigned)n_ctas, kUThreads, smem, st>>>(a, maps.bk, maps.bv, maps.dense); break;
-    }
-    return cudaGetLastError();
+    cudaError_t e = cudaErrorInvalidValue;
+#define PKV_UMMA_LAUNCH(P, NT) \
+    if (a.geo.page == P && a.geo.rank_tiles == NT) { block_umma_kernel<P, NT><<<(unsigned)n_ctas, kUThreads, smem, st>>>(a, maps); e = cudaGetLastError(); }
+    PKV_FOR_EACH_UMMA_SHAPE(PKV_UMMA_LAUNCH)
+#undef PKV_UMMA_LAUNCH
+    return e;
 }
 
 }  // namespace pkv

@@ -231,15 +231,17 @@ def test_paper_default_shape_qwen3_8b_16k():
 
 
 @pytest.mark.parametrize("variant", [0, 3])
-def test_prefill_chunk_2048_positions_against_32k(variant):
-    """The bench's prefill-chunk launch (`--workload prefill_chunk_llama3_8b_32k --q-len 2048`): one sequence of
-    32768 tokens whose last 2048 positions are the queries, 8192 query rows per KV head, served by the row-block
-    kernels (variant 0: tcgen05, 512 CTAs of 128 rows; 3: mma.sync, 1024 CTAs of 64 rows).  Sampled query rows -
+@pytest.mark.parametrize("workload", ["prefill_chunk_llama3_8b_32k", "prefill_chunk_qwen3_8b_16k_p32"])
+def test_prefill_chunk_2048_positions_against_a_long_context(workload, variant):
+    """The bench's prefill-chunk launches (`--workload prefill_chunk_llama3_8b_32k --q-len 2048`, and the same on the
+    paper's default page shape, P = 32 with ranks (16, 14)): one sequence whose last 2048 positions are the queries,
+    8192 query rows per KV head, served by the row-block kernels (variant 0: tcgen05, 512 CTAs of 128 rows; 3:
+    mma.sync, 1024 CTAs of 64 rows).  Sampled query rows -
     the first and last positions of the chunk, positions on either side of page and block boundaries, a row from every
     128-row block parity - against plain attention over the pages exactly as the GPU stores them (kernel gate; the
     causal limit is part of what is checked), the two kernels against one another on every row, and a rerun bit for
     bit."""
-    w, device = bench.WORKLOADS["prefill_chunk_llama3_8b_32k"], torch.device("cuda", 0)
+    w, device = bench.WORKLOADS[workload], torch.device("cuda", 0)
     QL = 2048
     cfg, cache, lengths, comp = bench.build_workload(w, w["rank"], device, decode_variant=variant)
     T, Hq, Hkv = lengths[0], w["n_q_heads"], w["n_kv_heads"]
@@ -267,16 +269,16 @@ def test_prefill_chunk_2048_positions_against_32k(variant):
                 assert e <= 4e-3, (variant, head, j, gq, e)
                 assert rel_err(f64(out[0, j, h]), ref) <= ATT_TOL
                 worst = max(worst, e)
-    record("prefill_chunk_llama3_8b_32k", decode_variant=variant, kernel_gate_worst=worst, rows_checked=2 * len(positions) * G)
+    record(workload, decode_variant=variant, kernel_gate_worst=worst, rows_checked=2 * len(positions) * G)
     if variant == 0:
-        _PREFILL_OUT["tcgen05"] = out32.cpu()
-    elif "tcgen05" in _PREFILL_OUT:
-        a, b = _PREFILL_OUT.pop("tcgen05").double().numpy(), out32.cpu().double().numpy()
+        _PREFILL_OUT[workload] = out32.cpu()
+    elif workload in _PREFILL_OUT:
+        a, b = _PREFILL_OUT.pop(workload).double().numpy(), out32.cpu().double().numpy()
         # every row of the launch: the two kernels differ by summation order and by where p and w are rounded
         err = np.abs(a - b).max(axis=-1) / np.abs(b).max(axis=-1)
         assert err.max() <= 8e-3, err.max()          # both are within 4e-3 of the same reference
         print("tcgen05 vs mma.sync over %d rows: worst %.2e, mean %.2e" % (err.size, err.max(), err.mean()))
-        record("prefill_chunk_llama3_8b_32k", tcgen05_vs_mma_sync_worst_row=float(err.max()), rows=int(err.size))
+        record(workload, tcgen05_vs_mma_sync_worst_row=float(err.max()), rows=int(err.size))
     _finish(cache)
 
 
