@@ -793,9 +793,9 @@ def main():
                 flops += QL * Hq * (nf_ * 2 * (128 * rank + rank * P_ + P_ * rv_ + rv_ * 128) + dense_tok * 4 * 128)
             tpeak, tsrc = _tensor_peak()
             tach = flops / (launch_ms * 1e-3) / 1e12
-            # the library's own rule (row_block_umma_supported): tcgen05 kernel for P = 64 or 32, bf16 factors, even ranks;
-            # the mma.sync kernel otherwise or when decode_variant 3 pins it
-            umma = args.decode_variant == 0 and P_ in (32, 64) and rank % 2 == 0 and rv_ % 2 == 0 and rv_ <= rank
+            # the library's own rule (row_block_umma_supported): tcgen05 kernel for bf16 factors whose matrices start on
+            # 128-byte boundaries of the pool; the mma.sync kernel otherwise or when decode_variant 3 pins it
+            umma = args.decode_variant == 0 and rv_ <= rank and all(x % 128 == 0 for x in (2 * P_ * rank, 2 * P_ * rv_, 256 * rank, 256 * rv_))
             line["roofline"] = {"bound": "tensor",
                                 "kernel": (("block_umma_kernel<P=%d, rank tiles=%%d> (tcgen05, 128 query rows per CTA)" % P_) if umma else
                                            "block_tc_kernel<P=%d, rank tiles=%%d> (mma.sync, 64 query rows per CTA)" % P_) % ((rank + 7) // 8),

@@ -304,9 +304,10 @@ pkv_status pkv_decode_attention(pkv_cache *c, int32_t layer, int32_t n_seqs, con
  * which reads the sequence's pages once for its block, the query rows being the row operand of every product of
  * Eq. 4 - runs when q_len * (H_q / H_kv) >= 64, the factors are bf16, and the call makes at least 128 blocks of 64
  * rows (enough to fill the GPU) or would exceed the limit above, which does not apply to this kernel.  For
- * page_size 64 or 32 and even ranks it is the tcgen05 kernel (128 rows per CTA, accumulators and
- * row operands in tensor memory, pages brought in by TMA in the layout the tensor cores read); for other shapes,
- * or with decode_variant 3, the mma.sync kernel (64 rows per CTA).  Otherwise the decode kernel runs
+ * page_size 64 (any rank), 32 (even ranks) and 16 (ranks that are multiples of 4) it is the tcgen05 kernel (128
+ * rows per CTA, accumulators and row operands in tensor memory, pages brought in by TMA in the layout the tensor
+ * cores read); for the other ranks, or with decode_variant 3, the mma.sync kernel (64 rows per CTA).  Otherwise
+ * the decode kernel runs
  * with its CTAs in groups of b = ceil(q_len / max(1, 8 / (H_q / H_kv))): the CTAs of a group walk the same pages at
  * the same time, one block of 8 / (H_q / H_kv) query tokens each, so HBM delivers a page once and L2 delivers it b
  * times (q_len = 2 at H_q / H_kv = 8 costs 1.3 single-query launches, q_len = 2 at H_q / H_kv = 4 costs one).

@@ -142,7 +142,8 @@ cudaError_t launch_compress(const Geometry &geo, const unsigned char *dense_pool
                             const int2 *worklist, int n_entries, int *status, cudaStream_t st);
 cudaError_t launch_decode(const DecodeArgs &a, int n_segs, cudaStream_t st);
 constexpr int kRowBlock = 64;          // query rows (token x query head) per CTA of the mma.sync row-block kernel
-// tcgen05 row-block kernel (pkv_rowblock.cu): 128 query rows per CTA; P = 64 or 32, bf16 page-wise factors, even ranks
+// tcgen05 row-block kernel (pkv_rowblock.cu): 128 query rows per CTA; bf16 page-wise factors whose matrices start on
+// 128-byte boundaries of the pool (every rank for P = 64, even ranks for P = 32, multiples of 4 for P = 16)
 bool row_block_umma_supported(const Geometry &geo);
 cudaError_t row_block_umma_setup();
 // TMA descriptors of the pools for that kernel (B factors; dense K / V); valid = 0 where the shape is not covered or

@@ -343,9 +343,9 @@ template <int P, int NT>
 __global__ void __launch_bounds__(kUThreads, 2) block_umma_kernel(const __grid_constant__ DecodeArgs a,
                                                                   const __grid_constant__ RowBlockMaps maps) {
     constexpr int RP = NT <= 2 ? 16 : 32, kDB = kDenseBlock<P, NT, 0>;
-    // A^T rows are 2 P bytes: the 128-byte swizzle for P = 64, the 64-byte one (8 rows = 512 bytes) for P = 32 - in both
-    // cases the XOR the pages are stored with
-    constexpr uint32_t kASwizzle = P == 64 ? 2 : 4, kAGroup = 8 * 2 * P;
+    // A^T rows are 2 P bytes: the 128-byte swizzle for P = 64, the 64-byte one (8 rows = 512 bytes) for P = 32, the
+    // 32-byte one for P = 16 - each time the XOR the pages are stored with
+    constexpr uint32_t kASwizzle = P == 64 ? 2 : (P == 32 ? 4 : 6), kAGroup = 8 * 2 * P;
     static_assert(kDB == RP, "dense blocks and padded ranks have the same number of rows");
     const Geometry &geo = a.geo;
     const StageLayout L = umma_layout(geo);
@@ -702,15 +702,15 @@ size_t umma_smem_bytes(const Geometry &g) {
 }  // namespace
 
 bool row_block_umma_supported(const Geometry &g) {
-    // A^T rows of 128 or 64 bytes (P = 64, 32: the swizzles the tensor cores know for such rows); every part of a blob
+    // A^T rows of 128, 64 or 32 bytes (P = 64, 32, 16: the swizzles the tensor cores know for such rows); every part of a blob
     // on a 128-byte boundary of the pool (the tiled copies address the pools in 256-byte rows, from either of two
-    // origins 128 bytes apart): even ranks
-    return (g.page == 64 || g.page == 32) && g.factor_bits == 16 && g.global_rank == 0 && g.rank_k % 2 == 0 && g.rank_v % 2 == 0 &&
+    // origins 128 bytes apart): every rank for P = 64, even ranks for P = 32, multiples of 4 for P = 16
+    return (g.page == 64 || g.page == 32 || g.page == 16) && g.factor_bits == 16 && g.global_rank == 0 &&
            g.rank_v <= g.rank_k && g.rank_tiles >= 1 && g.rank_tiles <= 4 && g.bk_off % 128 == 0 && g.bv_off % 128 == 0 &&
            g.blob_bytes % 128 == 0 && g.factor_slot_bytes % 128 == 0 && umma_smem_bytes(g) <= (size_t)kSmemBudget / 2;
 }
 
-#define PKV_FOR_EACH_UMMA_SHAPE(X) X(64, 1) X(64, 2) X(64, 3) X(64, 4) X(32, 1) X(32, 2) X(32, 3) X(32, 4)
+#define PKV_FOR_EACH_UMMA_SHAPE(X) X(64, 1) X(64, 2) X(64, 3) X(64, 4) X(32, 1) X(32, 2) X(32, 3) X(32, 4) X(16, 1) X(16, 2)
 
 cudaError_t row_block_umma_setup() {
     cudaError_t e;
