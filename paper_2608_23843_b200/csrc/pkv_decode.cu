@@ -773,9 +773,8 @@ __device__ __forceinline__ long long q_row(const DecodeArgs &a, int seg, int n) 
 
 // Loads the lane's share of the segment's queries.  Returns, packed in 16-bit halves, how many of the sequence's
 // newest positions the lane's columns 2t and 2t+1 must not see (q_len - 1 - the column's query token).
-__device__ __forceinline__ int load_q(const DecodeArgs &a, int seg, uint32_t (&qf)[8][2], int lane) {
+__device__ __forceinline__ int load_q(const DecodeArgs &a, int seg, uint32_t (&qf)[8][2], int lane, long long row) {
     const int t = lane & 3;
-    const long long row = q_row(a, seg, lane >> 2);
     if (row >= 0) {
         const uint32_t *q = reinterpret_cast<const uint32_t *>(reinterpret_cast<const __nv_bfloat16 *>(a.q) + row * kHeadDim);
 #pragma unroll
@@ -788,6 +787,9 @@ __device__ __forceinline__ int load_q(const DecodeArgs &a, int seg, uint32_t (&q
     const int G = a.geo.group, j0 = ((seg / a.geo.n_kv_heads) % a.q_nblk) * a.q_tpt;
     const int b0 = max(0, a.q_len - 1 - j0 - (2 * t) / G), b1 = max(0, a.q_len - 1 - j0 - (2 * t + 1) / G);
     return b0 | (b1 << 16);
+}
+__device__ __forceinline__ int load_q(const DecodeArgs &a, int seg, uint32_t (&qf)[8][2], int lane) {
+    return load_q(a, seg, qf, lane, q_row(a, seg, lane >> 2));
 }
 
 // Writes the final result of one (entry, KV head) for query column hq, dims d4..d4+3.
@@ -1192,6 +1194,9 @@ __global__ void __launch_bounds__(kDecodeThreads, 2) decode_tc_kernel(const __gr
             asm volatile("prefetch.global.L2 [%0];" ::"l"(a.tickets + rg.seg_first + rg.n_local_segs - 1));
         }
         auto seg_info = [&](int sg) { return sg == 0 ? ps_first : (sg == rg.n_local_segs - 1 ? ps_last : PlanSeg{(int)(blockIdx.x / a.q_group), 1}); };
+        // (where this lane's queries of the first segment lie is worked out before the wait: several divisions by
+        // run-time values, which a stand-alone launch would otherwise pay between its release and its first load)
+        const long long first_q_row = warp < W ? q_row(a, query_seg(a, rg.seg_first), lane >> 2) : -1;
         if (!a.overlap) asm volatile("griddepcontrol.wait;" ::: "memory");
         if (trace && tid == 0) trace[8] = clock64();
         if (warp >= W) {
@@ -1201,7 +1206,7 @@ __global__ void __launch_bounds__(kDecodeThreads, 2) decode_tc_kernel(const __gr
         }
         uint32_t qf[8][2];
         int cur_seg = 0;
-        int hidden = load_q(a, query_seg(a, rg.seg_first), qf, lane);
+        int hidden = load_q(a, query_seg(a, rg.seg_first), qf, lane, first_q_row);
         // Global SVD form: this warp's rank-space sum, and where it keeps q~ (its own part of the combine area, which it
         // overwrites with its state only at a flush, when q~ of that segment is no longer needed)
         float wacc[kGlobal ? NT : 1][2];
