@@ -765,6 +765,9 @@ __device__ __forceinline__ float *partial_slot(const DecodeArgs &a, int cta_rang
 // block; with one query per sequence (q_len = 1) that is query head n.  Row of q / out it maps to, or -1.
 // (`seg` here is a query_seg() index.)
 __device__ __forceinline__ long long q_row(const DecodeArgs &a, int seg, int n) {
+    // one query per sequence: seg = entry * H + head and H_q = H * G, so the row is seg * G + n - no division (this
+    // sits between a stand-alone launch's release and its first load, and on the merging CTA's way out)
+    if (a.q_len == 1) return n < a.geo.group ? (long long)seg * a.geo.group + n : -1;
     const int H = a.geo.n_kv_heads, G = a.geo.group;
     const int entry = seg / H, head = seg % H, jl = n / G, j = (entry % a.q_nblk) * a.q_tpt + jl;
     if (jl >= a.q_tpt || j >= a.q_len) return -1;
@@ -924,11 +927,12 @@ __device__ __forceinline__ void flush_segment(const DecodeArgs &a, float *comb, 
             mine[kMaxGroup * kHeadDim + kMaxGroup + 2 * t + 1] = l1;
         }
     }
+    // (where the state goes is worked out while the other warps arrive: divisions by run-time values)
+    const int qseg = query_seg(a, seg);
+    float *part = partial_slot(a, blockIdx.x / a.q_group, seg);
     PKV_CONSUMER_BARRIER();
     // overlap mode 1: partial states, tickets and `out` may still be in use by the preceding launch
     if (a.overlap == 1) asm volatile("griddepcontrol.wait;" ::: "memory");
-    const int qseg = query_seg(a, seg);
-    float *part = partial_slot(a, blockIdx.x / a.q_group, seg);
     for (int item = ctid; item < kItems; item += kThreads) {
         const int hq = item >> 5, d4 = (item & 31) * 4;
         float M = kNegInf;
