@@ -478,12 +478,15 @@ __global__ void __launch_bounds__(kUThreads, 2) block_umma_kernel(const __grid_c
             int s0 = 0, s1 = 0, s2 = 0, round2 = 0;          // stages of the units u, u + 1, u + 2; times the stage of u + 2 has been used before
             auto stage_at = [&](int s) { return stages_a + (uint32_t)(s * ustage); };
             // [128 x RP] = Q . (K side)^T: 8 steps of 16 channels; both operands K-major, 128-byte swizzle
-            auto qk = [&](uint32_t t_dst, uint32_t kside, int panel) {
+            // (steps ks0 .. ks1 - 1: the eight steps of G1 are issued in two halves, so that they stand in the way of the
+            // other CTA's products for half as long at a time)
+            auto qk = [&](uint32_t t_dst, uint32_t kside, int panel, int ks0 = 0, int ks1 = 8) {
                 const uint32_t idesc = umma_idesc(128, RP, 0);
                 const uint64_t db0 = umma_desc(kside, 16, 1024, 2), db1 = umma_desc(kside + panel, 16, 1024, 2);
 #pragma unroll
                 for (int ks = 0; ks < 8; ++ks)
-                    umma_ss(t_dst, umma_desc_step(ks < 4 ? dq0 : dq1, (ks & 3) * 32), umma_desc_step(ks < 4 ? db0 : db1, (ks & 3) * 32), idesc, ks > 0);
+                    if (ks >= ks0 && ks < ks1)
+                        umma_ss(t_dst, umma_desc_step(ks < 4 ? dq0 : dq1, (ks & 3) * 32), umma_desc_step(ks < 4 ? db0 : db1, (ks & 3) * 32), idesc, ks > 0);
             };
             // o [128 x d] (+)= (rows of RP bf16 at t_src) . (V side): MN-major, two panels of 64 channels
             auto pv = [&](uint32_t t_src, uint32_t vside, int panel) {
@@ -536,6 +539,12 @@ __global__ void __launch_bounds__(kUThreads, 2) block_umma_kernel(const __grid_c
                         qk(t_s, sb + L.dk, L.d_panel);
                     }
                     umma_commit(bar_S);
+                    // behind it, off the rows' path: the first half of G1(u+2), over the q~ columns G2(u+1) has just read
+                    if (u + 2 < n_units) {
+                        k2 = unit_kind(s2, round2, ok);
+                        if (!ok) break;
+                        if (k2 == kKindFactor) qk(t_qt, stage_at(s2) + L.k, L.k_panel, 0, 4);
+                    }
                 }
                 // hand-over C: w(u) is in tensor memory -> G4(u); then, off the rows' path, G1(u+2)
                 if (!wait_lane(bar_C, ph_C, abort_flag, limit)) { ok = false; break; }
@@ -546,9 +555,12 @@ __global__ void __launch_bounds__(kUThreads, 2) block_umma_kernel(const __grid_c
                     umma_commit(smem_u32(empty_bar + s0));             // a factor unit's stage is free after G4
                 }
                 if (u + 2 < n_units) {
-                    k2 = unit_kind(s2, round2, ok);
-                    if (!ok) break;
-                    if (k2 == kKindFactor) qk(t_qt, stage_at(s2) + L.k, L.k_panel);
+                    if (u < -1) {                                  // (before the first unit there is no hand-over B)
+                        k2 = unit_kind(s2, round2, ok);
+                        if (!ok) break;
+                        if (k2 == kKindFactor) qk(t_qt, stage_at(s2) + L.k, L.k_panel, 0, 4);
+                    }
+                    if (k2 == kKindFactor) qk(t_qt, stage_at(s2) + L.k, L.k_panel, 4, 8);       // the second half of G1(u+2)
                 }
                 umma_commit(bar_Q);
                 k0 = k1; k1 = k2;
