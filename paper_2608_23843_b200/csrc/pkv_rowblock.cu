@@ -361,7 +361,8 @@ __global__ void __launch_bounds__(kUThreads, 2) block_umma_kernel(const __grid_c
     unsigned long long *empty_bar = full_bar + S;
     unsigned long long *bars = empty_bar + S;          // rows -> issuer: A, B, C; issuer -> rows: G3, S, Q; drain
     StageDesc *descs = reinterpret_cast<StageDesc *>(bars + 8);
-    volatile int *abort_flag = reinterpret_cast<volatile int *>(descs + S);
+    StageDesc *info = descs + S;                       // [2]: the descriptor of a unit as the issuing lane read it, for the row threads
+    volatile int *abort_flag = reinterpret_cast<volatile int *>(info + 2);
     uint32_t *tmem_slot = reinterpret_cast<uint32_t *>(const_cast<int *>(abort_flag) + 1);
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
     const uint32_t bar_A = smem_u32(bars + 0), bar_B = smem_u32(bars + 1), bar_C = smem_u32(bars + 2);
@@ -497,9 +498,13 @@ __global__ void __launch_bounds__(kUThreads, 2) block_umma_kernel(const __grid_c
                 o_valid = true;
             };
             // kind of a unit as the products see it: units without tokens run as dense units with every score masked
-            auto unit_kind = [&](int s, int round, bool &good) -> int {
+            // (the descriptor is passed on to the row threads, who meet it behind the next commit "Q": they need not wait
+            // for the copies themselves)
+            auto unit_kind = [&](int s, int round, bool &good, int unit) -> int {
                 if (!wait_lane(smem_u32(full_bar + s), round & 1, abort_flag, limit)) { good = false; return kKindDense; }
                 const StageDesc d = descs[s];
+                info[unit & 1] = d;
+                __threadfence_block();
                 return d.kind == kKindFactor && d.rows > 0 ? kKindFactor : kKindDense;
             };
             int k0 = kKindDense, k1 = kKindDense, k2 = kKindDense;       // kinds of the units u, u + 1, u + 2
@@ -541,7 +546,7 @@ __global__ void __launch_bounds__(kUThreads, 2) block_umma_kernel(const __grid_c
                     umma_commit(bar_S);
                     // behind it, off the rows' path: the first half of G1(u+2), over the q~ columns G2(u+1) has just read
                     if (u + 2 < n_units) {
-                        k2 = unit_kind(s2, round2, ok);
+                        k2 = unit_kind(s2, round2, ok, u + 2);
                         if (!ok) break;
                         if (k2 == kKindFactor) qk(t_qt, stage_at(s2) + L.k, L.k_panel, 0, 4);
                     }
@@ -556,7 +561,7 @@ __global__ void __launch_bounds__(kUThreads, 2) block_umma_kernel(const __grid_c
                 }
                 if (u + 2 < n_units) {
                     if (u < -1) {                                  // (before the first unit there is no hand-over B)
-                        k2 = unit_kind(s2, round2, ok);
+                        k2 = unit_kind(s2, round2, ok, u + 2);
                         if (!ok) break;
                         if (k2 == kKindFactor) qk(t_qt, stage_at(s2) + L.k, L.k_panel, 0, 4);
                     }
@@ -623,10 +628,9 @@ __global__ void __launch_bounds__(kUThreads, 2) block_umma_kernel(const __grid_c
 
             if (u >= -1 && u + 1 < n_units) {
                 // ---- the next unit's descriptor; q~(u+1) as two bf16 terms -> hand-over B ----
-                const int s = s_nxt;
-                if (!wait_warp(smem_u32(full_bar + s), round_nxt & 1, abort_flag, limit)) { ok = false; break; }
+                const int s = s_nxt, round = round_nxt;
                 if (++s_nxt == S) { s_nxt = 0; ++round_nxt; }
-                nxt = descs[s];
+                nxt = info[(u + 1) & 1];                        // written by the issuing lane ahead of the commit just met
                 if (nxt.rows <= 0 || nxt.kind != kKindFactor) { nxt.kind = kKindDense; nxt.rows = max(0, min(nxt.rows, kDB)); }
                 if (nxt.kind == kKindFactor) {      // columns past the rank are exact zeros
                     uint32_t rq[RP], hi[RP / 2], lo[RP / 2];
@@ -638,7 +642,9 @@ __global__ void __launch_bounds__(kUThreads, 2) block_umma_kernel(const __grid_c
                     tmem_st_wait();
                 } else if (nxt.rows < kDB) {
                     // rows past the sequence's end hold whatever the pool held: p is 0 there, but the rows must be
-                    // finite (V), also for a padded product of the stage before this one (K)
+                    // finite (V), also for a padded product of the stage before this one (K).  (The copies have
+                    // landed: the issuing lane has seen them; the wait costs nothing and orders these stores behind them.)
+                    if (!wait_warp(smem_u32(full_bar + s), round & 1, abort_flag, limit)) { ok = false; break; }
                     unsigned char *st_base = stages + (size_t)s * ustage;
                     for (int i = tid; i < (kDB - nxt.rows) * 32; i += kURows) {
                         const int side = i & 1, panel = (i >> 1) & 1, chunk = (i >> 2) & 7, r = nxt.rows + (i >> 5);
@@ -708,7 +714,7 @@ __global__ void __launch_bounds__(kUThreads, 2) block_umma_kernel(const __grid_c
 
 size_t umma_smem_bytes(const Geometry &g) {
     const int S = umma_stages(g);
-    return (size_t)kUQBytes + (size_t)S * umma_stage_bytes(g) + kUStagePad + (2 * S + 8) * 8 + S * sizeof(StageDesc) + 64;
+    return (size_t)kUQBytes + (size_t)S * umma_stage_bytes(g) + kUStagePad + (2 * S + 8) * 8 + (S + 2) * sizeof(StageDesc) + 64;
 }
 
 }  // namespace
