@@ -351,7 +351,10 @@ __global__ void __launch_bounds__(kUThreads, 2) block_umma_kernel(const __grid_c
     const StageLayout L = umma_layout(geo);
     const int S = umma_stages(geo), ustage = umma_stage_bytes(geo), H = geo.n_kv_heads, G = geo.group;
     const int n_rows = a.q_len * G, n_blk = (n_rows + kURows - 1) / kURows;
-    const int rb = blockIdx.x % n_blk, head = (blockIdx.x / n_blk) % H, entry = blockIdx.x / (n_blk * H);
+    // (the later a block's rows, the more of the sequence they see: the longest blocks of every head are started first,
+    // so that what is left for the last wave of CTAs is the short ones)
+    const int n_he = (int)gridDim.x / n_blk;              // (entry, head) pairs
+    const int rb = n_blk - 1 - (int)blockIdx.x / n_he, head = ((int)blockIdx.x % n_he) % H, entry = ((int)blockIdx.x % n_he) / H;
     const PlanHeader hdr = *reinterpret_cast<const PlanHeader *>(a.plan);
     if (entry >= hdr.n_seqs) return;
     extern __shared__ __align__(1024) unsigned char smem[];
