@@ -1547,7 +1547,10 @@ __global__ void __launch_bounds__(kBlockThreads, 2) block_tc_kernel(const __grid
     const Geometry &geo = a.geo;
     const int S = block_stages(geo), H = geo.n_kv_heads, G = geo.group;
     const int n_rows = a.q_len * G, n_blk = (n_rows + kBlockRows - 1) / kBlockRows;
-    const int rb = blockIdx.x % n_blk, head = (blockIdx.x / n_blk) % H, entry = blockIdx.x / (n_blk * H);
+    // (the later a block's rows, the more of the sequence they see: the longest blocks of every head are started first,
+    // so that what is left for the last wave of CTAs is the short ones)
+    const int n_he = (int)gridDim.x / n_blk;              // (entry, head) pairs
+    const int rb = n_blk - 1 - (int)blockIdx.x / n_he, head = ((int)blockIdx.x % n_he) % H, entry = ((int)blockIdx.x % n_he) / H;
     const PlanHeader hdr = *reinterpret_cast<const PlanHeader *>(a.plan);
     if (entry >= hdr.n_seqs) return;
     extern __shared__ __align__(1024) unsigned char smem[];
