@@ -11,21 +11,24 @@
 // One thread owns one query row (= one lane of tensor memory): it reads its row of q~, s, w back from tensor memory,
 // does the scaling, the two-term bf16 split, the masking and the online softmax alone (no shuffles), and writes the
 // row of the next product's A operand over the columns it has just read (tcgen05.mma takes A from tensor memory).
-// A^T factors are used where the bulk copy put them: the storage swizzle of a 128-byte A^T row is the tensor core's
-// 128-byte swizzle (A_k^T as an MN-major B operand, A_v^T as a K-major one).  Rows of 256 bytes (B factors, dense
-// K / V) arrive as two panels of 128-byte rows (tiled TMA copies, 64 channels each), which is the same swizzle again.
+// A^T factors are used where the bulk copy put them: the storage swizzle of an A^T row of 128, 64 or 32 bytes (P =
+// 64, 32, 16) is the tensor core's swizzle for rows of that length (A_k^T as an MN-major B operand, A_v^T as a K-major
+// one).  Rows of 256 bytes (B factors, dense K / V) arrive as two panels of 128-byte rows (tiled TMA copies, 64
+// channels each), which is the 128-byte swizzle again.
 //
 // Warps 0-3: the 128 query rows.  Warp 4, one lane: copies into the ring.  Warp 5, one lane: issues every
 // tcgen05.mma.  The four products of a factor page depend on one another through the row threads; the schedule
 // keeps the row threads waiting for as few of them as it can.  Per unit u the rows hand over three times (an
 // mbarrier of 128 arrivals each) and the issuer answers with tcgen05.commit on three mbarriers:
 //     rows: wait "S"; softmax of s(u) -> p(u)               hand-over A -> issuer: G3(u) | Gb(u); commit "G3"
-//     rows: wait "Q"; q~(u+1) to two bf16 terms             hand-over B -> issuer: G2(u+1) | Ga(u+1); commit "S"
-//     rows: wait "G3"; w(u) to bf16                         hand-over C -> issuer: G4(u); G1(u+2); commit "Q"
+//     rows: wait "Q"; q~(u+1) to two bf16 terms             hand-over B -> issuer: G2(u+1) | Ga(u+1); commit "S";
+//                                                                          first half of G1(u+2)
+//     rows: wait "G3"; w(u) to bf16                         hand-over C -> issuer: G4(u); second half of G1(u+2); commit "Q"
 // so the conversion of q~(u+1) runs while G3(u) does, s(u+1) is being computed while w(u) is converted, and G4 and
 // G1 are off the rows' path: their commit is met one hand-over later, when it has long arrived (earlier only if o
-// has to be rescaled).  Two CTAs per SM overlap one another's remaining waits.  Every wait is bounded; tensor
-// memory is released on every path out.
+// has to be rescaled).  The issuing lane also waits for each unit's copies and passes the unit's descriptor on to
+// the row threads ahead of commit "Q".  Two CTAs per SM overlap one another's remaining waits; the blocks of a
+// launch are taken longest first.  Every wait is bounded; tensor memory is released on every path out.
 #include "pkv_device.cuh"
 
 namespace pkv {
