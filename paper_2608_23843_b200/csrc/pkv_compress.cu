@@ -12,6 +12,16 @@ namespace pkv {
 
 namespace {
 
+// Two fp32 values in one 64-bit register and the sm_100 instructions that multiply-add both halves at once.  Each half
+// is an ordinary round-to-nearest FMA, so a sum written with them has the bits of the scalar version; what changes is
+// the number of instructions (the dense 4 x 4 updates below are bound by instruction issue).
+struct F2 { unsigned long long v; };
+__device__ __forceinline__ F2 f2(float lo, float hi) { F2 r; asm("mov.b64 %0, {%1, %2};" : "=l"(r.v) : "f"(lo), "f"(hi)); return r; }
+__device__ __forceinline__ void f2_get(F2 a, float &lo, float &hi) { asm("mov.b64 {%0, %1}, %2;" : "=f"(lo), "=f"(hi) : "l"(a.v)); }
+__device__ __forceinline__ F2 f2_mul(F2 a, F2 b) { F2 r; asm("mul.rn.f32x2 %0, %1, %2;" : "=l"(r.v) : "l"(a.v), "l"(b.v)); return r; }
+__device__ __forceinline__ F2 f2_fma(F2 a, F2 b, F2 c) { F2 r; asm("fma.rn.f32x2 %0, %1, %2, %3;" : "=l"(r.v) : "l"(a.v), "l"(b.v), "l"(c.v)); return r; }
+
+
 constexpr int kXs = kHeadDim + 2;         // padded row stride of X (bf16): 65 words, odd
 
 // Rotation pairs of every round of the pair ordering (P = 16), written once per device by the host.  A pair is
@@ -355,30 +365,35 @@ compress_kernel(Geometry geo, const unsigned char *dense_pool, unsigned char *fa
 #pragma unroll
                         for (int i = 0; i < 4; ++i) { ma[i] = (ma4 >> (8 * i)) & 0xff; mb[i] = (mb4 >> (8 * i)) & 0xff; }
                         const float4 *Ma = S.M + Qd::mslot(h, ia, 0), *Mb = S.M + Qd::mslot(h, ib, 0);    // rows 0..3 of the quad
-                        float T[4][4];
+                        // (two values per instruction; per value the operations and their order are those of the scalar form)
+                        F2 Tlo[4], Thi[4];                             // (T[0][j], T[1][j]) and (T[2][j], T[3][j])
 #pragma unroll
-                        for (int i = 0; i < 4; ++i)
-#pragma unroll
-                            for (int j = 0; j < 4; ++j) T[i][j] = 0.f;
+                        for (int j = 0; j < 4; ++j) Tlo[j] = Thi[j] = f2(0.f, 0.f);
 #pragma unroll
                         for (int k = 0; k < 4; ++k) {                  // T = M_a^T X
                             const float4 mk = Ma[k];
+                            const F2 mlo = f2(mk.x, mk.y), mhi = f2(mk.z, mk.w);
                             const float *row = S.G + ma[k] * kGs;
 #pragma unroll
                             for (int j = 0; j < 4; ++j) {
                                 const float x = row[mb[j]];
-                                T[0][j] = fmaf(mk.x, x, T[0][j]); T[1][j] = fmaf(mk.y, x, T[1][j]);
-                                T[2][j] = fmaf(mk.z, x, T[2][j]); T[3][j] = fmaf(mk.w, x, T[3][j]);
+                                const F2 xx = f2(x, x);
+                                Tlo[j] = f2_fma(mlo, xx, Tlo[j]);
+                                Thi[j] = f2_fma(mhi, xx, Thi[j]);
                             }
                         }
+                        float T[4][4];
+#pragma unroll
+                        for (int j = 0; j < 4; ++j) { f2_get(Tlo[j], T[0][j], T[1][j]); f2_get(Thi[j], T[2][j], T[3][j]); }
                         const float4 b0 = Mb[0], b1 = Mb[1], b2 = Mb[2], b3 = Mb[3];
+                        const F2 b0a = f2(b0.x, b0.y), b0b = f2(b0.z, b0.w), b1a = f2(b1.x, b1.y), b1b = f2(b1.z, b1.w);
+                        const F2 b2a = f2(b2.x, b2.y), b2b = f2(b2.z, b2.w), b3a = f2(b3.x, b3.y), b3b = f2(b3.z, b3.w);
 #pragma unroll
                         for (int i = 0; i < 4; ++i) {                  // Y = T M_b, row i
                             float y[4];
-                            y[0] = fmaf(T[i][3], b3.x, fmaf(T[i][2], b2.x, fmaf(T[i][1], b1.x, T[i][0] * b0.x)));
-                            y[1] = fmaf(T[i][3], b3.y, fmaf(T[i][2], b2.y, fmaf(T[i][1], b1.y, T[i][0] * b0.y)));
-                            y[2] = fmaf(T[i][3], b3.z, fmaf(T[i][2], b2.z, fmaf(T[i][1], b1.z, T[i][0] * b0.z)));
-                            y[3] = fmaf(T[i][3], b3.w, fmaf(T[i][2], b2.w, fmaf(T[i][1], b1.w, T[i][0] * b0.w)));
+                            const F2 t0 = f2(T[i][0], T[i][0]), t1 = f2(T[i][1], T[i][1]), t2 = f2(T[i][2], T[i][2]), t3 = f2(T[i][3], T[i][3]);
+                            f2_get(f2_fma(t3, b3a, f2_fma(t2, b2a, f2_fma(t1, b1a, f2_mul(t0, b0a)))), y[0], y[1]);
+                            f2_get(f2_fma(t3, b3b, f2_fma(t2, b2b, f2_fma(t1, b1b, f2_mul(t0, b0b)))), y[2], y[3]);
 #pragma unroll
                             for (int j = 0; j < 4; ++j) {
                                 S.G[ma[i] * kGs + mb[j]] = y[j];
@@ -395,11 +410,15 @@ compress_kernel(Geometry geo, const unsigned char *dense_pool, unsigned char *fa
                         const float4 x0 = *r0, x1 = *r1, x2 = *r2, x3 = *r3;
                         const float4 *Mk = S.M + Qd::mslot(0, k, 0);
                         const float4 c0 = Mk[0], c1 = Mk[1], c2 = Mk[2], c3 = Mk[3];
-#define PKV_MIX(comp) make_float4(fmaf(c3.comp, x3.x, fmaf(c2.comp, x2.x, fmaf(c1.comp, x1.x, c0.comp * x0.x))), \
-                                  fmaf(c3.comp, x3.y, fmaf(c2.comp, x2.y, fmaf(c1.comp, x1.y, c0.comp * x0.y))), \
-                                  fmaf(c3.comp, x3.z, fmaf(c2.comp, x2.z, fmaf(c1.comp, x1.z, c0.comp * x0.z))), \
-                                  fmaf(c3.comp, x3.w, fmaf(c2.comp, x2.w, fmaf(c1.comp, x1.w, c0.comp * x0.w))))
-                        *r0 = PKV_MIX(x); *r1 = PKV_MIX(y); *r2 = PKV_MIX(z); *r3 = PKV_MIX(w);   // row i' = sum_k M[k][i] row k
+                        // row i' = sum_k M[k][i] row k, two channels per instruction (same order of operations per channel)
+                        const F2 x0a = f2(x0.x, x0.y), x0b = f2(x0.z, x0.w), x1a = f2(x1.x, x1.y), x1b = f2(x1.z, x1.w);
+                        const F2 x2a = f2(x2.x, x2.y), x2b = f2(x2.z, x2.w), x3a = f2(x3.x, x3.y), x3b = f2(x3.z, x3.w);
+#define PKV_MIX(dst, comp) { const F2 k0 = f2(c0.comp, c0.comp), k1 = f2(c1.comp, c1.comp), k2 = f2(c2.comp, c2.comp), k3 = f2(c3.comp, c3.comp); \
+                             float4 o; \
+                             f2_get(f2_fma(k3, x3a, f2_fma(k2, x2a, f2_fma(k1, x1a, f2_mul(k0, x0a)))), o.x, o.y); \
+                             f2_get(f2_fma(k3, x3b, f2_fma(k2, x2b, f2_fma(k1, x1b, f2_mul(k0, x0b)))), o.z, o.w); \
+                             *dst = o; }
+                        PKV_MIX(r0, x) PKV_MIX(r1, y) PKV_MIX(r2, z) PKV_MIX(r3, w)
 #undef PKV_MIX
                     }
                 }
