@@ -250,8 +250,8 @@ __device__ __forceinline__ float max3(float a, float b, float c) {
 // tested against `rank`.
 template <int RP, int KNOWN, bool kExact>
 __device__ __forceinline__ void scale_pack(const uint32_t *x, uint32_t *pk, float scale, int rank) {
-#pragma unroll
     const uint64_t sc2 = f2_pack(scale, scale);
+#pragma unroll
     for (int k = 0; k < RP / 2; ++k) {
         if (kExact && 2 * k + 1 < KNOWN) {                // this pair lies below the rank
             float y0, y1;
@@ -266,8 +266,8 @@ __device__ __forceinline__ void scale_pack(const uint32_t *x, uint32_t *pk, floa
 // The same with the rounding error of each pair as a second bf16 term (hi + lo carries about 16 bits).
 template <int RP, int KNOWN, bool kExact>
 __device__ __forceinline__ void split_terms(const uint32_t *x, uint32_t *hi, uint32_t *lo, float scale, int rank) {
-#pragma unroll
     const uint64_t sc2 = f2_pack(scale, scale);
+#pragma unroll
     for (int k = 0; k < RP / 2; ++k) {
         if (kExact && 2 * k + 1 < KNOWN) {                // this pair lies below the rank
             const uint64_t y = f2_mul(f2_pack(__uint_as_float(x[2 * k]), __uint_as_float(x[2 * k + 1])), sc2);
