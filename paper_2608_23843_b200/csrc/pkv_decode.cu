@@ -764,10 +764,13 @@ __device__ __forceinline__ float *partial_slot(const DecodeArgs &a, int cta_rang
 // Query column n of a segment's score tile = query head n % G of the (n / G)-th query token of the plan entry's
 // block; with one query per sequence (q_len = 1) that is query head n.  Row of q / out it maps to, or -1.
 // (`seg` here is a query_seg() index.)
+template <bool kFast = true>
 __device__ __forceinline__ long long q_row(const DecodeArgs &a, int seg, int n) {
     // one query per sequence: seg = entry * H + head and H_q = H * G, so the row is seg * G + n - no division (this
-    // sits between a stand-alone launch's release and its first load, and on the merging CTA's way out)
-    if (a.q_len == 1) return n < a.geo.group ? (long long)seg * a.geo.group + n : -1;
+    // sits between a stand-alone launch's release and its first load, and on the merging CTA's way out).  kFast = false
+    // leaves the shortcut out: the Global SVD form of the decode kernel has no register to spare for a second copy of
+    // the code behind it (its inner loop spills more with it).
+    if (kFast && a.q_len == 1) return n < a.geo.group ? (long long)seg * a.geo.group + n : -1;
     const int H = a.geo.n_kv_heads, G = a.geo.group;
     const int entry = seg / H, head = seg % H, jl = n / G, j = (entry % a.q_nblk) * a.q_tpt + jl;
     if (jl >= a.q_tpt || j >= a.q_len) return -1;
@@ -791,16 +794,18 @@ __device__ __forceinline__ int load_q(const DecodeArgs &a, int seg, uint32_t (&q
     const int b0 = max(0, a.q_len - 1 - j0 - (2 * t) / G), b1 = max(0, a.q_len - 1 - j0 - (2 * t + 1) / G);
     return b0 | (b1 << 16);
 }
+template <bool kFast = true>
 __device__ __forceinline__ int load_q(const DecodeArgs &a, int seg, uint32_t (&qf)[8][2], int lane) {
-    return load_q(a, seg, qf, lane, q_row(a, seg, lane >> 2));
+    return load_q(a, seg, qf, lane, q_row<kFast>(a, seg, lane >> 2));
 }
 
 // Writes the final result of one (entry, KV head) for query column hq, dims d4..d4+3.
 // With a.state set the call returns the softmax state instead (Eq. 5's inputs, for a merge across caches that
 // hold different token ranges of the sequence): row = o[0..d) unnormalised, then m (the running maximum of the
 // scaled scores in base-2 units, i.e. of s * softmax_scale * log2 e), then l.
+template <bool kFast = true>
 __device__ __forceinline__ void store_out(const DecodeArgs &a, int seg, int hq, int d4, float4 acc, float M, float L) {
-    const long long row = q_row(a, seg, hq);
+    const long long row = q_row<kFast>(a, seg, hq);
     if (row < 0) return;
     if (a.state) {
         float *st = a.state + row * (kHeadDim + 2);
@@ -834,7 +839,7 @@ __device__ __forceinline__ void fold_state(float4 &tot, float &Mr, float &Lr, co
 // Eq. 5 across CTAs: partial states summed in CTA order with a running maximum (one pass).
 // A thread owns E items (query head, four dims): ctid, ctid + kThreads, ...; kBatch parts' loads are in flight at a
 // time, because with dozens of parts it is the latency of these loads that the rest of the GPU waits for.
-template <int E, int kBatch>
+template <int E, int kBatch, bool kFast = true>
 __device__ __forceinline__ void merge_parts(const DecodeArgs &a, const float *first, int np, int seg, int ctid,
                                             float *dst) {
     const long long stride = (long long)a.q_group * kPartialFloats;     // between the states of consecutive ranges
@@ -881,7 +886,7 @@ __device__ __forceinline__ void merge_parts(const DecodeArgs &a, const float *fi
             *reinterpret_cast<float4 *>(dst + hq[e] * kHeadDim + d4) = tot[e];
             if (d4 == 0) { dst[kMaxGroup * kHeadDim + hq[e]] = Mr[e]; dst[kMaxGroup * kHeadDim + kMaxGroup + hq[e]] = Lr[e]; }
         } else {
-            store_out(a, seg, hq[e], d4, tot[e], Mr[e], Lr[e]);
+            store_out<kFast>(a, seg, hq[e], d4, tot[e], Mr[e], Lr[e]);
         }
     }
 }
@@ -899,6 +904,7 @@ __device__ __forceinline__ int draw_ticket(int *counter) {
 // lies wholly in this CTA the result is final; otherwise the CTA writes one partial state, takes a
 // ticket, and the CTA that draws the last ticket of the segment applies Eq. 5 across CTAs.  Partials
 // are always summed in CTA order, so the result does not depend on which CTA arrives last.
+template <bool kFast = true>
 __device__ __forceinline__ void flush_segment(const DecodeArgs &a, float *comb, volatile int *last_flag, WarpState &st,
                                               int seg, const PlanSeg ps, int warp, int lane, int ctid, int n_active,
                                               long long *trace) {
@@ -947,7 +953,7 @@ __device__ __forceinline__ void flush_segment(const DecodeArgs &a, float *comb, 
             L += f * cw[kMaxGroup * kHeadDim + kMaxGroup + hq];
         }
         if (ps.n_parts <= 1) {
-            if (hq < a.q_cols) store_out(a, qseg, hq, d4, acc, M, L);
+            if (hq < a.q_cols) store_out<kFast>(a, qseg, hq, d4, acc, M, L);
         } else {
             *reinterpret_cast<float4 *>(part + hq * kHeadDim + d4) = acc;
             if ((item & 31) == 0) {
@@ -980,8 +986,8 @@ __device__ __forceinline__ void flush_segment(const DecodeArgs &a, float *comb, 
             if (mine) {
                 float *dst = a.gpartials + (long long)(gslot0 + g) * kPartialFloats;
                 const float *gfirst = first + (long long)g * kMergeFan * kPartialFloats;
-                if (a.q_cols * 32 <= kThreads) merge_parts<1, 16>(a, gfirst, gsize, qseg, ctid, dst);
-                else merge_parts<2, 8>(a, gfirst, gsize, qseg, ctid, dst);
+                if (a.q_cols * 32 <= kThreads) merge_parts<1, 16, kFast>(a, gfirst, gsize, qseg, ctid, dst);
+                else merge_parts<2, 8, kFast>(a, gfirst, gsize, qseg, ctid, dst);
                 if (ctid == 0) a.gtickets[gslot0 + g] = 0;     // ready for the next launch
                 first = a.gpartials + (long long)gslot0 * kPartialFloats;
                 np = (ps.n_parts + kMergeFan - 1) / kMergeFan;
@@ -993,8 +999,8 @@ __device__ __forceinline__ void flush_segment(const DecodeArgs &a, float *comb, 
             PKV_CONSUMER_BARRIER();
             if (trace && ctid == 0) trace[10] = clock64();
             if (*last_flag) {
-                if (a.q_cols * 32 <= kThreads) merge_parts<1, 16>(a, first, np, qseg, ctid, nullptr);
-                else merge_parts<2, 8>(a, first, np, qseg, ctid, nullptr);
+                if (a.q_cols * 32 <= kThreads) merge_parts<1, 16, kFast>(a, first, np, qseg, ctid, nullptr);
+                else merge_parts<2, 8, kFast>(a, first, np, qseg, ctid, nullptr);
                 if (ctid == 0) a.tickets[qseg] = 0;         // ready for the next launch
                 if (trace && ctid == 0) trace[13] = clock64();
             }
@@ -1200,12 +1206,12 @@ __global__ void __launch_bounds__(kDecodeThreads, 2) decode_tc_kernel(const __gr
         auto seg_info = [&](int sg) { return sg == 0 ? ps_first : (sg == rg.n_local_segs - 1 ? ps_last : PlanSeg{(int)(blockIdx.x / a.q_group), 1}); };
         // (where this lane's queries of the first segment lie is worked out before the wait: several divisions by
         // run-time values, which a stand-alone launch would otherwise pay between its release and its first load)
-        const long long first_q_row = warp < W ? q_row(a, query_seg(a, rg.seg_first), lane >> 2) : -1;
+        const long long first_q_row = warp < W ? q_row<!kGlobal>(a, query_seg(a, rg.seg_first), lane >> 2) : -1;
         if (!a.overlap) asm volatile("griddepcontrol.wait;" ::: "memory");
         if (trace && tid == 0) trace[8] = clock64();
         if (warp >= W) {
             for (int sg = 0; sg < rg.n_local_segs; ++sg)
-                flush_segment(a, comb, last_flag, st, rg.seg_first + sg, seg_info(sg), warp, lane, tid, W, nullptr);
+                flush_segment<!kGlobal>(a, comb, last_flag, st, rg.seg_first + sg, seg_info(sg), warp, lane, tid, W, nullptr);
             return;
         }
         uint32_t qf[8][2];
@@ -1231,9 +1237,9 @@ __global__ void __launch_bounds__(kDecodeThreads, 2) decode_tc_kernel(const __gr
             if (cur_seg < dsc.seg) {
                 // the old segment's queries are no longer needed: fetch the new ones now, so that their latency
                 // hides behind the flush
-                if (dsc.seg < rg.n_local_segs) hidden = load_q(a, query_seg(a, rg.seg_first + dsc.seg), qf, lane);
+                if (dsc.seg < rg.n_local_segs) hidden = load_q<!kGlobal>(a, query_seg(a, rg.seg_first + dsc.seg), qf, lane);
                 while (cur_seg < dsc.seg) {
-                    flush_segment(a, comb, last_flag, st, rg.seg_first + cur_seg, seg_info(cur_seg), warp, lane, tid, W, trace);
+                    flush_segment<!kGlobal>(a, comb, last_flag, st, rg.seg_first + cur_seg, seg_info(cur_seg), warp, lane, tid, W, trace);
                     ++cur_seg;
                     reset_state(st);
                 }
