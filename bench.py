@@ -780,11 +780,16 @@ def main():
                                   "gpu_launches": lps * args.steps}
         P_, Gq = w.get("page", 64), Hq // w["n_kv_heads"]
         rows = QL * Gq
-        if QL > 1 and args.decode_variant in (0, 3) and args.factor_bits != 4 and rows >= 64 and w["batch"] * w["n_kv_heads"] * -(-rows // 64) >= 128:
+        rv_ = w.get("rank_v", rank)
+        # the library's own rule (row_block_umma_supported): tcgen05 kernel for bf16 factors whose matrices start on
+        # 128-byte boundaries of the pool; the mma.sync kernel otherwise or when decode_variant 3 pins it
+        umma = args.decode_variant == 0 and rv_ <= rank and all(x % 128 == 0 for x in (2 * P_ * rank, 2 * P_ * rv_, 256 * rank, 256 * rv_))
+        # (and its rule for the route: row blocks from 64 query rows per KV head on; the mma.sync kernel only if they fill the GPU)
+        if QL > 1 and args.decode_variant in (0, 3) and args.factor_bits != 4 and rows >= 64 and (
+                umma or w["batch"] * w["n_kv_heads"] * -(-rows // 64) >= 128):
             # Served by the row-block kernel, whose bound is the tensor pipe, not HBM: algorithmic FLOPs per launch =
             # query rows x (factor pages x 2 (d r_k + r_k P + P r_v + r_v d) + dense tokens x 4 d); the causal
             # triangle among the new positions is counted in full.
-            rv_ = w.get("rank_v", rank)
             flops = 0
             for T_ in lengths:
                 n_pages_ = -(-T_ // P_)
@@ -793,9 +798,6 @@ def main():
                 flops += QL * Hq * (nf_ * 2 * (128 * rank + rank * P_ + P_ * rv_ + rv_ * 128) + dense_tok * 4 * 128)
             tpeak, tsrc = _tensor_peak()
             tach = flops / (launch_ms * 1e-3) / 1e12
-            # the library's own rule (row_block_umma_supported): tcgen05 kernel for bf16 factors whose matrices start on
-            # 128-byte boundaries of the pool; the mma.sync kernel otherwise or when decode_variant 3 pins it
-            umma = args.decode_variant == 0 and rv_ <= rank and all(x % 128 == 0 for x in (2 * P_ * rank, 2 * P_ * rv_, 256 * rank, 256 * rv_))
             line["roofline"] = {"bound": "tensor",
                                 "kernel": (("block_umma_kernel<P=%d, rank tiles=%%d> (tcgen05, 128 query rows per CTA)" % P_) if umma else
                                            "block_tc_kernel<P=%d, rank tiles=%%d> (mma.sync, 64 query rows per CTA)" % P_) % ((rank + 7) // 8),

@@ -80,6 +80,7 @@ struct pkv_cache {
     MetaLayout ml;
     WorkspaceLayout wl;
     bool dry = false;
+    int n_sms = 148;                   // of the device the cache was created on
     bool trace = false;                // PKV_DECODE_TRACE=1: CTAs write time stamps into the workspace
     unsigned char *dense_pool = nullptr, *factor_pool = nullptr, *meta = nullptr, *workspace = nullptr;
     RowBlockMaps row_maps = {};        // TMA descriptors of the pools (tcgen05 row-block kernel)
@@ -271,6 +272,8 @@ void derive(const pkv_config &cfg, int n_ctas, Geometry &g, MetaLayout &ml, Work
     wl.tickets = w;  w += wl.tickets_stride * wl.n_sets;
     wl.gram = w;     w = align_up(w + (cfg.global_rank > 0 ? 4LL * cfg.n_kv_heads * 2 * d * d : 0), 256);
     wl.trace = w;    w = align_up(w + 8LL * kTraceSlots * n_ctas, 256);
+    wl.rb_partials = w;
+    w = align_up(w + (row_block_umma_supported(g) ? 4LL * kRbSplitItems * 128 * kRbStateFloats : 0), 256);
     wl.total = w;
 }
 
@@ -397,6 +400,8 @@ int block_slots_per_seq(const Geometry &g, int q_len) { return passes_per_seq(g,
 bool uses_row_blocks(const pkv_cache *c, int q_len, int n_seqs) {
     const long long rows = (long long)q_len * c->geo.group;
     if (q_len <= 1 || (c->cfg.decode_variant != 0 && c->cfg.decode_variant != 3) || c->geo.factor_bits == 4 || rows < kRowBlock) return false;
+    // (the tcgen05 kernel splits long sequences over several CTAs when the row blocks alone would not fill the GPU)
+    if (c->row_maps.valid && c->cfg.decode_variant == 0) return true;
     const long long n_ctas = (long long)n_seqs * c->geo.n_kv_heads * ((rows + kRowBlock - 1) / kRowBlock);
     return n_ctas >= 128 || (long long)n_seqs * block_slots_per_seq(c->geo, q_len) > c->cfg.max_seqs;
 }
@@ -550,7 +555,8 @@ pkv_status pkv_init_cache(const pkv_config *cfg, void *dense_pool, void *factor_
     { const char *t = getenv("PKV_TEST_DROP_UNIT"); if (t && t[0]) c->drop_unit = atoi(t); }
     // default grid: one CTA per SM when consecutive launches overlap (two launches share each SM),
     // otherwise two CTAs per SM
-    int n_ctas = cfg->n_ctas > 0 ? cfg->n_ctas : default_ctas(dry) * (cfg->decode_overlap ? 1 : 2);
+    c->n_sms = default_ctas(dry);
+    int n_ctas = cfg->n_ctas > 0 ? cfg->n_ctas : c->n_sms * (cfg->decode_overlap ? 1 : 2);
     if (cfg->n_ctas == 0 && n_ctas > 512) n_ctas = 512;      // pkv_query_sizes() sized the buffers for <= 512
     derive(*cfg, n_ctas, c->geo, c->ml, c->wl);
     {
@@ -1064,6 +1070,19 @@ static pkv_status decode_impl(pkv_cache *c, int32_t layer, int32_t n_seqs, const
         a.layer = layer;
         a.variant = c->cfg.decode_variant == 3 ? 3 : 0; a.overlap = 0; a.plain_launch = 1; a.trace = nullptr;
         c->cache_written = false;
+        // tcgen05 kernel: with fewer row blocks than half the CTAs the GPU holds, each block's sequence is cut into
+        // ranges of at least kRbMinPages pages, one CTA each
+        a.rb_splits = 1;
+        a.rb_partials = (float *)(c->workspace + c->wl.rb_partials);
+        if (a.variant == 0 && c->row_maps.valid) {
+            const long long n_blocks = (long long)n_seqs * c->geo.n_kv_heads * (((long long)q_len * c->geo.group + 127) / 128);
+            int longest = 0;
+            for (int i = 0; i < n_seqs; ++i) longest = std::max(longest, c->at(seq_ids[i], layer).n_tokens);
+            const long long by_fill = std::min<long long>(2LL * c->n_sms, kRbSplitItems) / n_blocks;
+            const long long by_length = (longest + c->cfg.page_size - 1) / c->cfg.page_size / kRbMinPages;
+            const long long ns = std::min<long long>(kRbMaxSplits, std::min(by_fill, by_length));
+            if (ns >= 2) a.rb_splits = (int)ns;
+        }
         PKV_CUDA(c, launch_decode_blocks(a, n_seqs, c->row_maps, st));
         return PKV_OK;
     }

@@ -93,6 +93,7 @@ struct WorkspaceLayout {
     long long tickets;                 // int [n_sets][n_seg_tickets + n_group]: per segment, then per group
     long long gram;                    // Global SVD form: float [H_kv][2][d][d], the region Gram matrices of one (sequence, layer)
     long long trace;                   // long long [n_ctas][kTraceSlots]
+    long long rb_partials;             // float [kRbSplitItems][128][kRbStateFloats]: states of row blocks split by token range (0 bytes if the tcgen05 kernel does not cover the shape)
     long long total;
 };
 
@@ -130,6 +131,10 @@ struct DecodeArgs {
     long long wait_clocks;             // limit of every in-kernel wait of the decode kernel (SM clocks)
     int drop_unit;                     // -1; test hook: CTA 0's producer never arms this unit (a wait must run out)
     long long *trace;                  // NULL, or [n_ctas][kTraceSlots] time stamps written by each CTA (debugging)
+    // tcgen05 row-block kernel: CTAs per row block (each with its own range of the sequence; 1 = no split) and where
+    // their states go
+    int rb_splits;
+    float *rb_partials;
 };
 
 // Launchers (defined in the .cu files); all return the launch error.
@@ -141,6 +146,9 @@ cudaError_t launch_append(const Geometry &geo, unsigned char *dense_pool, const 
 cudaError_t launch_compress(const Geometry &geo, const unsigned char *dense_pool, unsigned char *factor_pool,
                             const int2 *worklist, int n_entries, int *status, cudaStream_t st);
 cudaError_t launch_decode(const DecodeArgs &a, int n_segs, cudaStream_t st);
+// Row blocks split by token range: a state is d channels of o, then m and l, padded to 16-byte rows; at most
+// kRbSplitItems CTAs per launch when split, at most kRbMaxSplits per row block, at least kRbMinPages pages per range.
+constexpr int kRbStateFloats = kHeadDim + 4, kRbSplitItems = 512, kRbMaxSplits = 16, kRbMinPages = 8;
 constexpr int kRowBlock = 64;          // query rows (token x query head) per CTA of the mma.sync row-block kernel
 // tcgen05 row-block kernel (pkv_rowblock.cu): 128 query rows per CTA; bf16 page-wise factors whose matrices start on
 // 128-byte boundaries of the pool (every rank for P = 64, even ranks for P = 32, multiples of 4 for P = 16)

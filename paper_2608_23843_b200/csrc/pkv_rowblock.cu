@@ -356,8 +356,11 @@ __global__ void __launch_bounds__(kUThreads, 2) block_umma_kernel(const __grid_c
     const int n_rows = a.q_len * G, n_blk = (n_rows + kURows - 1) / kURows;
     // (the later a block's rows, the more of the sequence they see: the longest blocks of every head are started first,
     // so that what is left for the last wave of CTAs is the short ones)
-    const int n_he = (int)gridDim.x / n_blk;              // (entry, head) pairs
-    const int rb = n_blk - 1 - (int)blockIdx.x / n_he, head = ((int)blockIdx.x % n_he) % H, entry = ((int)blockIdx.x % n_he) / H;
+    // With a.rb_splits = ns > 1 (few row blocks, long sequences) ns consecutive CTAs share a row block, each with its own
+    // range of the block's units; they leave softmax states which rowblock_merge_kernel combines (Eq. 5).
+    const int ns = a.rb_splits, blk_id = (int)blockIdx.x / ns, split = (int)blockIdx.x - blk_id * ns;
+    const int n_he = (int)gridDim.x / ns / n_blk;         // (entry, head) pairs
+    const int rb = n_blk - 1 - blk_id / n_he, head = (blk_id % n_he) % H, entry = (blk_id % n_he) / H;
     const PlanHeader hdr = *reinterpret_cast<const PlanHeader *>(a.plan);
     if (entry >= hdr.n_seqs) return;
     extern __shared__ __align__(1024) unsigned char smem[];
@@ -408,6 +411,11 @@ __global__ void __launch_bounds__(kUThreads, 2) block_umma_kernel(const __grid_c
         else need = hu.d0 + hu.nf + (page - hu.fe) * geo.blocks_per_page + blk + 1;
         n_units = max(1, min(need, hu.units));
     }
+    int u_base = 0;                                       // first unit of this CTA's range
+    if (ns > 1) {
+        u_base = (int)((long long)n_units * split / ns);
+        n_units = (int)((long long)n_units * (split + 1) / ns) - u_base;          // may be 0: a state without weight
+    }
     const long long limit = a.wait_clocks;
 
     if (warp == 4) {
@@ -421,7 +429,7 @@ __global__ void __launch_bounds__(kUThreads, 2) block_umma_kernel(const __grid_c
             for (int s = 0, round = 0; u < n_units; ++u, s = s + 1 == S ? 0 : s + 1, round += s == 0) {
                 if (u >= S && !wait_lane(smem_u32(empty_bar + s), (round - 1) & 1, abort_flag, limit)) { ok = false; break; }
                 int page, blk, kind;
-                unit_to_page(geo, hu, u, page, blk, kind);
+                unit_to_page(geo, hu, u_base + u, page, blk, kind);
                 const int slot = pt[page];
                 int rows = 0, after = 0;
                 const bool bad = slot < 0 || slot >= (kind == kKindFactor ? geo.n_factor_slots : geo.n_dense_slots);
@@ -683,7 +691,25 @@ __global__ void __launch_bounds__(kUThreads, 2) block_umma_kernel(const __grid_c
 #undef PKV_ROWS_WAIT
 #undef PKV_ROWS_ARRIVE
         if (!ok && lane == 0 && !*abort_flag) { *abort_flag = 1; atomicAdd(a.status, 1); }
-        if (ok) {
+        if (ok && ns > 1) {
+            // this range's state: o in the frame of its own maximum m, then m and l (rows of kRbStateFloats floats)
+            const float f = st.l > 0.f ? exp2_fast(st.m_ref - st.m) : 0.f;
+            float *dst = a.rb_partials + ((size_t)blockIdx.x * kURows + tid) * kRbStateFloats;
+#pragma unroll 1
+            for (int c = 0; c < 4; ++c) {
+                uint32_t r[32];
+                if (n_units > 0) {                                      // (without units o was never written)
+                    tmem_ld32(t_o + 32 * c, r);
+                    tmem_ld_wait();
+                }
+#pragma unroll
+                for (int i = 0; i < 32; ++i) r[i] = n_units > 0 ? __float_as_uint(__uint_as_float(r[i]) * f) : 0u;
+#pragma unroll
+                for (int k = 0; k < 8; ++k)
+                    *reinterpret_cast<uint4 *>(dst + 32 * c + 4 * k) = make_uint4(r[4 * k], r[4 * k + 1], r[4 * k + 2], r[4 * k + 3]);
+            }
+            *reinterpret_cast<float2 *>(dst + kHeadDim) = make_float2(st.m, st.l);
+        } else if (ok) {
             const float inv = st.l > 0.f ? exp2_fast(st.m_ref - st.m) / st.l : 0.f;          // o is in the frame of m_ref
             __nv_bfloat16 *out = reinterpret_cast<__nv_bfloat16 *>(a.out);
 #pragma unroll 1
@@ -716,6 +742,43 @@ __global__ void __launch_bounds__(kUThreads, 2) block_umma_kernel(const __grid_c
     tc_fence_before();
     __syncthreads();
     if (warp == 0) asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tm), "r"(kTmemCols) : "memory");
+}
+
+// Eq. 5 over the ns ranges of a row block: one warp per query row, a lane per four channels; the ranges are taken in
+// token order, so the result does not depend on which CTA finished first.
+__global__ void __launch_bounds__(256) rowblock_merge_kernel(const __grid_constant__ DecodeArgs a) {
+    const Geometry &geo = a.geo;
+    const int ns = a.rb_splits, H = geo.n_kv_heads, G = geo.group;
+    const int n_rows = a.q_len * G, n_blk = (n_rows + kURows - 1) / kURows;
+    const int blk_id = (int)blockIdx.x / (kURows / 8), r = ((int)blockIdx.x % (kURows / 8)) * 8 + ((int)threadIdx.x >> 5);
+    const int n_he = (int)gridDim.x / (kURows / 8) / n_blk;
+    const int rb = n_blk - 1 - blk_id / n_he, head = (blk_id % n_he) % H, entry = (blk_id % n_he) / H;
+    const int row = rb * kURows + r, lane = threadIdx.x & 31;
+    if (row >= n_rows) return;
+    const long long qrow = ((long long)entry * a.q_len + row / G) * geo.n_q_heads + head * G + row % G;
+    const float *src = a.rb_partials + ((size_t)blk_id * ns * kURows + r) * kRbStateFloats;
+    const size_t stride = (size_t)kURows * kRbStateFloats;
+    float M = kNegInf;
+    for (int k = 0; k < ns; ++k) {
+        const float2 ml = *reinterpret_cast<const float2 *>(src + k * stride + kHeadDim);
+        if (ml.y > 0.f) M = fmaxf(M, ml.x);
+    }
+    float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
+    float L = 0.f;
+    for (int k = 0; k < ns; ++k) {
+        const float2 ml = *reinterpret_cast<const float2 *>(src + k * stride + kHeadDim);
+        if (!(ml.y > 0.f)) continue;
+        const float w = exp2f(ml.x - M);
+        const float4 o = *reinterpret_cast<const float4 *>(src + k * stride + 4 * lane);
+        acc.x += w * o.x; acc.y += w * o.y; acc.z += w * o.z; acc.w += w * o.w;
+        L += w * ml.y;
+    }
+    const float inv = L > 0.f ? 1.f / L : 0.f;
+    acc.x *= inv; acc.y *= inv; acc.z *= inv; acc.w *= inv;
+    if (a.out)
+        *reinterpret_cast<uint2 *>(reinterpret_cast<__nv_bfloat16 *>(a.out) + qrow * kHeadDim + 4 * lane) =
+            make_uint2(pack_bf16(acc.x, acc.y), pack_bf16(acc.z, acc.w));
+    if (a.out_f32) *reinterpret_cast<float4 *>(a.out_f32 + qrow * kHeadDim + 4 * lane) = acc;
 }
 
 size_t umma_smem_bytes(const Geometry &g) {
@@ -789,17 +852,24 @@ void row_block_make_maps(const Geometry &g, const void *factor_pool, const void 
     maps->valid = 1;
 }
 
-// One CTA per (sequence, KV head, block of 128 query rows).
+// One CTA per (sequence, KV head, block of 128 query rows), or a.rb_splits CTAs with a range of the sequence each and
+// a second launch that merges their states.
 cudaError_t launch_decode_blocks_umma(const DecodeArgs &a, int n_seqs, const RowBlockMaps &maps, cudaStream_t st) {
     const int n_blk = (a.q_len * a.geo.group + kURows - 1) / kURows;
-    const long long n_ctas = (long long)n_seqs * a.geo.n_kv_heads * n_blk;
-    if (!maps.valid || !row_block_umma_supported(a.geo) || n_ctas <= 0 || n_ctas > 0x7fffffffLL) return cudaErrorInvalidValue;
+    const long long n_blocks = (long long)n_seqs * a.geo.n_kv_heads * n_blk, n_ctas = n_blocks * a.rb_splits;
+    if (!maps.valid || !row_block_umma_supported(a.geo) || n_blocks <= 0 || n_ctas > 0x7fffffffLL || a.rb_splits < 1 ||
+        (a.rb_splits > 1 && (!a.rb_partials || n_ctas > kRbSplitItems)))
+        return cudaErrorInvalidValue;
     const size_t smem = umma_smem_bytes(a.geo);
     cudaError_t e = cudaErrorInvalidValue;
 #define PKV_UMMA_LAUNCH(P, NT) \
     if (a.geo.page == P && a.geo.rank_tiles == NT) { block_umma_kernel<P, NT><<<(unsigned)n_ctas, kUThreads, smem, st>>>(a, maps); e = cudaGetLastError(); }
     PKV_FOR_EACH_UMMA_SHAPE(PKV_UMMA_LAUNCH)
 #undef PKV_UMMA_LAUNCH
+    if (e == cudaSuccess && a.rb_splits > 1) {
+        rowblock_merge_kernel<<<(unsigned)(n_blocks * (kURows / 8)), 256, 0, st>>>(a);
+        e = cudaGetLastError();
+    }
     return e;
 }
 

@@ -668,9 +668,22 @@ def test_sequence_sharded_attention_states(bits):
 def test_row_block_kernel_agrees_with_the_column_kernel(P, rk, rv, G, q_len):
     """pkv_decode_attention_multi picks its kernel by shape; decode_variant = 2 pins the decode (column) kernel.  The
     two must agree to fp32-accumulation accuracy on the same cache contents (same compression kernel, same factors),
-    including sequences whose new positions start a page, end mid-block, or make up the whole sequence."""
+    including sequences whose new positions start a page, end mid-block, or make up the whole sequence.  (The longest
+    sequence has 31 pages: the tcgen05 kernel cuts every row block's sequence into three ranges, and the shortest
+    sequences leave some of those ranges empty.)"""
+    _row_block_against_column(P, rk, rv, G, q_len, [30 * P + 3, q_len, 5 * P, 12 * P + P // 2, q_len + 1], 40)
+
+
+@pytest.mark.parametrize("P,rk,rv,G,q_len", [(16, 16, 12, 4, 40), (64, 24, 24, 8, 16), (32, 16, 14, 4, 37)])
+def test_row_blocks_split_by_token_range(P, rk, rv, G, q_len):
+    """Few row blocks and long sequences: the tcgen05 kernel gives each row block 11 to 16 CTAs with a range of the
+    sequence each and merges their softmax states (Eq. 5) in a second launch.  Same agreement as above with the
+    column kernel and the unsplit mma.sync kernel; one sequence is so short that most of its ranges are empty."""
+    _row_block_against_column(P, rk, rv, G, q_len, [131 * P + 5, q_len + 2, 90 * P + P // 2], 140)
+
+
+def _row_block_against_column(P, rk, rv, G, q_len, lengths, max_pages):
     H = 2
-    lengths = [30 * P + 3, q_len, 5 * P, 12 * P + P // 2, q_len + 1]
     W = -(-q_len // P) * P
     outs = []
     for variant in (0, 2, 3):              # 0: row-block kernel the library picks (tcgen05 where the shape allows); 3: the mma.sync one
@@ -678,7 +691,8 @@ def test_row_block_kernel_agrees_with_the_column_kernel(P, rk, rv, G, q_len):
         # variant 0 with too few plan entries for the column kernel: the row-block kernel runs whatever the batch size
         cfg = pkv.make_config(n_layers=1, n_kv_heads=H, n_q_heads=H * G, rank=rk, rank_v=rv, page_size=P, sink_tokens=P,
                               recent_tokens=W, max_seqs=len(lengths) * (-(-q_len // tpt) if variant == 2 else 1),
-                              max_pages_per_seq=40, n_dense_slots=200, n_factor_slots=160, decode_variant=variant)
+                              max_pages_per_seq=max_pages, n_dense_slots=200, n_factor_slots=max(160, 2 * max_pages),
+                              decode_variant=variant)
         cache = pkv.Cache(cfg, "cuda")
         for s, T in enumerate(lengths):
             k, v = gen_kv(8, 0, s, T, cfg, outlier_prob=0.01)
@@ -689,9 +703,10 @@ def test_row_block_kernel_agrees_with_the_column_kernel(P, rk, rv, G, q_len):
         g = torch.Generator().manual_seed(5)
         q = torch.randn((len(lengths), q_len, H * G, 128), generator=g).to(torch.bfloat16).cuda()
         out32 = torch.empty(q.shape, dtype=torch.float32, device="cuda")
-        out = cache.decode_attention_multi(0, [4, 2, 0, 1, 3], q_len, q, None, out32)
+        order = [4, 2, 0, 1, 3][-len(lengths):] if len(lengths) == 5 else list(range(len(lengths)))[::-1]
+        out = cache.decode_attention_multi(0, order, q_len, q, None, out32)
         again = torch.empty_like(out32)
-        cache.decode_attention_multi(0, [4, 2, 0, 1, 3], q_len, q, None, again)
+        cache.decode_attention_multi(0, order, q_len, q, None, again)
         torch.cuda.synchronize()
         st = cache.stats()
         assert st["device_timeouts"] == 0 and st["bad_slot_indices"] == 0 and not out32.isnan().any()
