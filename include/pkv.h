@@ -300,13 +300,15 @@ pkv_status pkv_decode_attention(pkv_cache *c, int32_t layer, int32_t n_seqs, con
  * checked per call); n_seqs * b <= max_seqs with b = ceil(q_len / max(1, 8 / (H_q / H_kv))) blocks of query tokens
  * per sequence, b rounded up to a multiple of the grid size if it exceeds it (split-K partial states and tickets
  * are kept per sequence and block).
- * Two kinds of kernel serve this call.  A row-block kernel - one CTA per (sequence, KV head, block of query rows),
- * which reads the sequence's pages once for its block, the query rows being the row operand of every product of
- * Eq. 4 - runs when q_len * (H_q / H_kv) >= 64, the factors are bf16, and the call makes at least 128 blocks of 64
- * rows (enough to fill the GPU) or would exceed the limit above, which does not apply to this kernel.  For
- * page_size 64 (any rank), 32 (even ranks) and 16 (ranks that are multiples of 4) it is the tcgen05 kernel (128
- * rows per CTA, accumulators and row operands in tensor memory, pages brought in by TMA in the layout the tensor
- * cores read); for the other ranks, or with decode_variant 3, the mma.sync kernel (64 rows per CTA).  Otherwise
+ * Two kinds of kernel serve this call.  A row-block kernel - CTAs per (sequence, KV head, block of query rows),
+ * which read the sequence's pages once for the block, the query rows being the row operand of every product of
+ * Eq. 4 - runs when q_len * (H_q / H_kv) >= 64 and the factors are bf16.  For page_size 64 (any rank), 32 (even
+ * ranks) and 16 (ranks that are multiples of 4) it is the tcgen05 kernel (128 rows per CTA, accumulators and row
+ * operands in tensor memory, pages brought in by TMA in the layout the tensor cores read); where the blocks alone
+ * would not fill the GPU it cuts each block's sequence into up to 16 token ranges, one CTA each, and a second
+ * launch merges their softmax states by Eq. 5 in token order.  For the other ranks, or with decode_variant 3, it
+ * is the mma.sync kernel (64 rows per CTA, never split), and then only if the call makes at least 128 blocks
+ * (enough to fill the GPU) or would exceed the limit above, which does not apply to row blocks.  Otherwise
  * the decode kernel runs
  * with its CTAs in groups of b = ceil(q_len / max(1, 8 / (H_q / H_kv))): the CTAs of a group walk the same pages at
  * the same time, one block of 8 / (H_q / H_kv) query tokens each, so HBM delivers a page once and L2 delivers it b
