@@ -285,6 +285,46 @@ def test_prefill_chunk_2048_positions_against_a_long_context(workload, variant):
 _PREFILL_OUT = {}
 
 
+@pytest.mark.parametrize("q_len", [16, 64])
+def test_a_few_dozen_new_positions_per_sequence_at_full_size(q_len):
+    """The bench's `--workload llama3_8b_32k_b8 --q-len 16 / 64` launches: 8 sequences of 32K, 64 / 128 row blocks of 128
+    rows (half filled at q_len 16), which the tcgen05 kernel cuts into 4 / 2 token ranges of 128 / 256 units each and
+    merges by Eq. 5.  Sampled rows of every sequence against plain attention over the pages as the GPU stores them
+    (kernel gate), and a rerun bit for bit."""
+    w, device = bench.WORKLOADS["llama3_8b_32k_b8"], torch.device("cuda", 0)
+    cfg, cache, lengths, comp = bench.build_workload(w, w["rank"], device)
+    B, Hq, Hkv = w["batch"], w["n_q_heads"], w["n_kv_heads"]
+    G = Hq // Hkv
+    ids = list(range(B))
+    g = torch.Generator(device="cpu").manual_seed(bench.SEED + 78)
+    q = torch.randn((B, q_len, Hq, 128), generator=g).to(torch.bfloat16).to(device)
+    out32 = torch.empty(q.shape, dtype=torch.float32, device=device)
+    out = torch.empty_like(q)
+    cache.decode_attention_multi(0, ids, q_len, q, out, out32)
+    again = torch.empty_like(out32)
+    cache.decode_attention_multi(0, ids, q_len, q, None, again)
+    torch.cuda.synchronize()
+    st = cache.stats()
+    assert st["device_timeouts"] == 0 and st["bad_slot_indices"] == 0
+    assert torch.equal(again, out32) and not out32.isnan().any()
+    scale = 1.0 / np.sqrt(cfg.head_dim)
+    worst = 0.0
+    for i in ids:
+        head = (3 * i + 1) % Hkv
+        K_all, V_all, _ = stored_kv(cache, i, 0, head)
+        for j in sorted({0, 1, q_len // 2, q_len - 1}):
+            vis = lengths[i] - (q_len - 1 - j)
+            for gq in range(G):
+                h = head * G + gq
+                ref = oatt.attention_plain(f64(q[i, j, h]), K_all[:vis], V_all[:vis], scale)
+                e = rel_err(f64(out32[i, j, h]), ref)
+                assert e <= 4e-3, (i, head, j, gq, e)
+                assert rel_err(f64(out[i, j, h]), ref) <= ATT_TOL
+                worst = max(worst, e)
+    record("llama3_8b_32k_b8", q_len=q_len, kernel_gate_worst=worst, rows_checked=B * 4 * G)
+    _finish(cache)
+
+
 @pytest.mark.parametrize("rank", [8, 16, 24, 32])
 def test_ragged_serving_batch_rank_sweep(rank):
     """Ragged serving batch: 64 requests, lengths log-uniform in [2048, 65536], 2% outlier key tokens (x10)."""
