@@ -148,7 +148,7 @@ cudaError_t launch_compress(const Geometry &geo, const unsigned char *dense_pool
 cudaError_t launch_decode(const DecodeArgs &a, int n_segs, cudaStream_t st);
 // Row blocks split by token range: a state is d channels of o, then m and l, padded to 16-byte rows; at most
 // kRbSplitItems CTAs per launch when split, at most kRbMaxSplits per row block, at least kRbMinPages pages per range.
-constexpr int kRbStateFloats = kHeadDim + 4, kRbSplitItems = 512, kRbMaxSplits = 16, kRbMinPages = 8;
+constexpr int kRbStateFloats = kHeadDim + 4, kRbSplitItems = 512, kRbMaxSplits = 32, kRbMinPages = 8;
 constexpr int kRowBlock = 64;          // query rows (token x query head) per CTA of the mma.sync row-block kernel
 // tcgen05 row-block kernel (pkv_rowblock.cu): 128 query rows per CTA; bf16 page-wise factors whose matrices start on
 // 128-byte boundaries of the pool (every rank for P = 64, even ranks for P = 32, multiples of 4 for P = 16)

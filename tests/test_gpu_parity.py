@@ -676,7 +676,7 @@ def test_row_block_kernel_agrees_with_the_column_kernel(P, rk, rv, G, q_len):
 
 @pytest.mark.parametrize("P,rk,rv,G,q_len", [(16, 16, 12, 4, 40), (64, 24, 24, 8, 16), (32, 16, 14, 4, 37)])
 def test_row_blocks_split_by_token_range(P, rk, rv, G, q_len):
-    """Few row blocks and long sequences: the tcgen05 kernel gives each row block 11 to 16 CTAs with a range of the
+    """Few row blocks and long sequences: the tcgen05 kernel gives each row block 16 CTAs with a range of the
     sequence each and merges their softmax states (Eq. 5) in a second launch.  Same agreement as above with the
     column kernel and the unsplit mma.sync kernel; one sequence is so short that most of its ranges are empty."""
     _row_block_against_column(P, rk, rv, G, q_len, [131 * P + 5, q_len + 2, 90 * P + P // 2], 140)
