@@ -806,6 +806,14 @@ def main():
                                                        "page through the row threads): ncu shows the tensor pipe about 30 % busy" if umma else
                                                        "; ncu showed the mma.sync pipe 50 % busy at this rate"),
                                 "traffic": None, "launch_us": launch_ms * 1e3, "algorithmic_flops_per_launch": flops}
+            if umma:
+                # the library's rule for cutting row blocks into token ranges (a second, merging launch follows then)
+                n_blocks = w["batch"] * w["n_kv_heads"] * -(-rows // 128)
+                sms = torch.cuda.get_device_properties(device).multi_processor_count
+                ns = min(32, min(2 * sms, 512) // n_blocks, -(-max(lengths) // P_) // 8)
+                line["roofline"]["token_ranges_per_row_block"] = ns if ns >= 2 else 1
+                if ns >= 2:
+                    line["gpu_launches"] *= 2
         if not args.no_cpu_baseline and world == 1 and QL == 1 and not args.global_rank:
             o = oracle_sample(w, rank, 3, args.factor_bits)
             line["cpu_baseline"] = {"value": o["decode_s"] * 1e6 * o["slices_per_step"], "unit": "us",
