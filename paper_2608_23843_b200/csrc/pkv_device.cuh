@@ -30,11 +30,15 @@ __device__ __forceinline__ HeadUnits head_units(const Geometry &g, const PlanEnt
 }
 
 // unit index within an (entry, head) run -> logical page, block inside the page, kind
+// (bpp: blocks a dense page is cut into)
+__device__ __forceinline__ void unit_to_page(int bpp, const HeadUnits &h, int u, int &page, int &blk, int &kind) {
+    if (u < h.d0) { page = u / bpp; blk = u % bpp; kind = kKindDense; }
+    else if (u < h.d0 + h.nf) { page = h.fb + (u - h.d0); blk = 0; kind = kKindFactor; }
+    else { int v = u - h.d0 - h.nf; page = h.fe + v / bpp; blk = v % bpp; kind = kKindDense; }
+}
 __device__ __forceinline__ void unit_to_page(const Geometry &g, const HeadUnits &h, int u, int &page, int &blk,
                                              int &kind) {
-    if (u < h.d0) { page = u / g.blocks_per_page; blk = u % g.blocks_per_page; kind = kKindDense; }
-    else if (u < h.d0 + h.nf) { page = h.fb + (u - h.d0); blk = 0; kind = kKindFactor; }
-    else { int v = u - h.d0 - h.nf; page = h.fe + v / g.blocks_per_page; blk = v % g.blocks_per_page; kind = kKindDense; }
+    unit_to_page(g.blocks_per_page, h, u, page, blk, kind);
 }
 
 __device__ __forceinline__ uint32_t smem_u32(const void *p) { return (uint32_t)__cvta_generic_to_shared(p); }

@@ -44,20 +44,27 @@ constexpr uint32_t kColQt = 0, kColS = 32, kColW = 96, kColO = 128, kTmemCols = 
 // a block of dense K, V side = B_v or a block of dense V; a side is two panels of 64 channels, written by tiled TMA
 // copies (box = 64 channels x rows) straight from the pools' 256-byte rows: 16-byte chunk c of row j is stored at
 // chunk c ^ (j & 7), so each half of a row is a 128-byte row in the tensor core's 128-byte swizzle.
-// Rows of a dense block, and what a rank is padded to in the products (16 or 32):
-__host__ __device__ inline int umma_part_rows(const Geometry &g) { return g.rank_tiles <= 2 ? 16 : 32; }
-constexpr int kUStagePad = 1024;
+// Pages of 32 tokens with ranks up to 16 are taken two to a unit (64 tokens, like a page of 64): page j's B rows start
+// at row 16 j of panels of 32 rows, so that q~ and w of the pair are one row of 32 columns and the products with the
+// B factors are the same instructions as for a rank of 32; the products with the A factors are issued per page.
+__host__ __device__ inline bool umma_pair(const Geometry &g) { return g.page == 32 && g.rank_tiles <= 2; }
+// Rows of a dense block (a whole page of 32 tokens in the pair form), and what a rank - or a pair's two ranks - is padded to in the products:
+__host__ __device__ inline int umma_part_rows(const Geometry &g) { return g.rank_tiles <= 2 && !umma_pair(g) ? 16 : 32; }
+// Bytes kept free behind the last stage: a product that reads a rank padded to 16 or 32 rows may run past the last
+// part of a stage (a pair's panels hold exactly the rows its products read).
+__host__ __device__ inline int umma_stage_pad(const Geometry &g) { return umma_pair(g) ? 0 : 1024; }
 // bytes of an A^T part of a stage: rows of 2 P bytes, the rank rounded up to 8 rows, the part to 1024 bytes (the parts
 // behind it hold 128-byte-swizzled panels, whose pattern repeats every 1024 bytes)
 __host__ __device__ inline int umma_a_bytes(const Geometry &g, int rank) { return ((((rank + 7) & ~7) * 2 * g.page) + 1023) & ~1023; }
 __host__ __device__ inline int umma_stage_bytes(const Geometry &g) {
-    const int factor = umma_a_bytes(g, g.rank_k) + umma_a_bytes(g, g.rank_v) + 2 * 128 * (((g.rank_k + 7) & ~7) + ((g.rank_v + 7) & ~7));
+    const int factor = umma_pair(g) ? 2 * (umma_a_bytes(g, g.rank_k) + umma_a_bytes(g, g.rank_v)) + 4 * 32 * 128
+                                    : umma_a_bytes(g, g.rank_k) + umma_a_bytes(g, g.rank_v) + 2 * 128 * (((g.rank_k + 7) & ~7) + ((g.rank_v + 7) & ~7));
     const int dense = 4 * umma_part_rows(g) * 128;
     return ((factor > dense ? factor : dense) + 1023) & ~1023;
 }
 // stages: the units u, u + 1 and u + 2 are in use at any time; the rest is the copies' lead
 __host__ __device__ inline int umma_stages(const Geometry &g) {
-    const int room = 113 * 1024 - kUQBytes - kUStagePad - 512;
+    const int room = 113 * 1024 - kUQBytes - umma_stage_pad(g) - 512;
     return max(3, min(6, room / umma_stage_bytes(g)));
 }
 
@@ -211,6 +218,10 @@ __host__ __device__ inline StageLayout umma_layout(const Geometry &g) {
     const int rk = (g.rank_k + 7) & ~7, rv = (g.rank_v + 7) & ~7;        // parts start on 1024-byte boundaries
     L.ak = 0; L.k = umma_a_bytes(g, g.rank_k); L.k_panel = rk * 128;
     L.av = L.k + 2 * rk * 128; L.v = L.av + umma_a_bytes(g, g.rank_v); L.v_panel = rv * 128;
+    if (umma_pair(g)) {          // [A_k^T x 2][K side: 2 panels of 32 rows][A_v^T x 2][V side: 2 panels of 32 rows]
+        L.k = 2 * umma_a_bytes(g, g.rank_k); L.k_panel = 32 * 128;
+        L.av = L.k + 2 * L.k_panel; L.v = L.av + 2 * umma_a_bytes(g, g.rank_v); L.v_panel = 32 * 128;
+    }
     L.d_panel = umma_part_rows(g) * 128; L.dk = 0; L.dv = 2 * L.d_panel;
     return L;
 }
@@ -248,28 +259,31 @@ __device__ __forceinline__ float max3(float a, float b, float c) {
 // RP fp32 values x (a row of q~ or w) times `scale`, as bf16 pairs; columns from `rank` on become exact zeros.  The
 // kExact: the rank is KNOWN, a compile-time value (the ranks fill their tiles); otherwise KNOWN = RP and every column is
 // tested against `rank`.
-template <int RP, int KNOWN, bool kExact>
+// (kHalves: the row is two ranks of 16 columns side by side - a pair of pages -, each with its own pad columns)
+template <int RP, int KNOWN, bool kExact, bool kHalves = false>
 __device__ __forceinline__ void scale_pack(const uint32_t *x, uint32_t *pk, float scale, int rank) {
     const uint64_t sc2 = f2_pack(scale, scale);
+    constexpr int kMask = kHalves ? 15 : ~0;
 #pragma unroll
     for (int k = 0; k < RP / 2; ++k) {
-        if (kExact && 2 * k + 1 < KNOWN) {                // this pair lies below the rank
+        if (kExact && ((2 * k + 1) & kMask) < KNOWN) {    // this pair lies below the rank
             float y0, y1;
             f2_unpack(f2_mul(f2_pack(__uint_as_float(x[2 * k]), __uint_as_float(x[2 * k + 1])), sc2), y0, y1);
             pk[k] = pack_bf16(y0, y1);
             continue;
         }
-        const bool in0 = 2 * k < KNOWN && 2 * k < rank, in1 = 2 * k + 1 < KNOWN && 2 * k + 1 < rank;
+        const bool in0 = ((2 * k) & kMask) < KNOWN && ((2 * k) & kMask) < rank, in1 = ((2 * k + 1) & kMask) < KNOWN && ((2 * k + 1) & kMask) < rank;
         pk[k] = pack_bf16(in0 ? __uint_as_float(x[2 * k]) * scale : 0.f, in1 ? __uint_as_float(x[2 * k + 1]) * scale : 0.f);
     }
 }
 // The same with the rounding error of each pair as a second bf16 term (hi + lo carries about 16 bits).
-template <int RP, int KNOWN, bool kExact>
+template <int RP, int KNOWN, bool kExact, bool kHalves = false>
 __device__ __forceinline__ void split_terms(const uint32_t *x, uint32_t *hi, uint32_t *lo, float scale, int rank) {
     const uint64_t sc2 = f2_pack(scale, scale);
+    constexpr int kMask = kHalves ? 15 : ~0;
 #pragma unroll
     for (int k = 0; k < RP / 2; ++k) {
-        if (kExact && 2 * k + 1 < KNOWN) {                // this pair lies below the rank
+        if (kExact && ((2 * k + 1) & kMask) < KNOWN) {    // this pair lies below the rank
             const uint64_t y = f2_mul(f2_pack(__uint_as_float(x[2 * k]), __uint_as_float(x[2 * k + 1])), sc2);
             float y0, y1, e0, e1;
             f2_unpack(y, y0, y1);
@@ -278,7 +292,7 @@ __device__ __forceinline__ void split_terms(const uint32_t *x, uint32_t *hi, uin
             lo[k] = pack_bf16(e0, e1);
             continue;
         }
-        const bool in0 = 2 * k < KNOWN && 2 * k < rank, in1 = 2 * k + 1 < KNOWN && 2 * k + 1 < rank;
+        const bool in0 = ((2 * k) & kMask) < KNOWN && ((2 * k) & kMask) < rank, in1 = ((2 * k + 1) & kMask) < KNOWN && ((2 * k + 1) & kMask) < rank;
         const float x0 = in0 ? __uint_as_float(x[2 * k]) * scale : 0.f, x1 = in1 ? __uint_as_float(x[2 * k + 1]) * scale : 0.f;
         hi[k] = pack_bf16(x0, x1);
         lo[k] = pack_bf16(x0 - bf16lo_f(hi[k]), x1 - bf16hi_f(hi[k]));
@@ -345,7 +359,11 @@ __device__ __forceinline__ bool softmax_row(float *sv, RowSoftmax &st, bool o_va
 template <int P, int NT>
 __global__ void __launch_bounds__(kUThreads, 2) block_umma_kernel(const __grid_constant__ DecodeArgs a,
                                                                   const __grid_constant__ RowBlockMaps maps) {
-    constexpr int RP = NT <= 2 ? 16 : 32, kDB = kDenseBlock<P, NT, 0>;
+    // RP1: what a page's rank is padded to; RP: columns of q~ and w of a factor unit, and the rows of a dense block;
+    // PU: tokens of a factor unit (kPair: two pages of 32 tokens, see umma_pair()); bpp: blocks of a dense page
+    constexpr bool kPair = P == 32 && NT <= 2;
+    constexpr int RP1 = NT <= 2 ? 16 : 32, RP = kPair ? 32 : RP1, PU = kPair ? 2 * P : P;
+    constexpr int kDB = kPair ? 32 : kDenseBlock<P, NT, 0>, bpp = P / kDB;
     // A^T rows are 2 P bytes: the 128-byte swizzle for P = 64, the 64-byte one (8 rows = 512 bytes) for P = 32, the
     // 32-byte one for P = 16 - each time the XOR the pages are stored with
     constexpr uint32_t kASwizzle = P == 64 ? 2 : (P == 32 ? 4 : 6), kAGroup = 8 * 2 * P;
@@ -366,7 +384,8 @@ __global__ void __launch_bounds__(kUThreads, 2) block_umma_kernel(const __grid_c
     extern __shared__ __align__(1024) unsigned char smem[];
     unsigned char *sq = smem, *stages = smem + kUQBytes;
     // (one more KiB behind the last stage: a padded product of the last stage's last part reads it)
-    unsigned long long *full_bar = reinterpret_cast<unsigned long long *>(stages + (size_t)S * ustage + kUStagePad);
+    const int stage_pad = umma_stage_pad(geo);
+    unsigned long long *full_bar = reinterpret_cast<unsigned long long *>(stages + (size_t)S * ustage + stage_pad);
     unsigned long long *empty_bar = full_bar + S;
     unsigned long long *bars = empty_bar + S;          // rows -> issuer: A, B, C; issuer -> rows: G3, S, Q; drain
     StageDesc *descs = reinterpret_cast<StageDesc *>(bars + 8);
@@ -385,7 +404,7 @@ __global__ void __launch_bounds__(kUThreads, 2) block_umma_kernel(const __grid_c
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     }
     // What a padded product reads past a unit's own rows must be finite from the start.
-    for (int i = tid; i < (S * ustage + kUStagePad) / 16; i += kUThreads) reinterpret_cast<uint4 *>(stages)[i] = make_uint4(0u, 0u, 0u, 0u);
+    for (int i = tid; i < (S * ustage + stage_pad) / 16; i += kUThreads) reinterpret_cast<uint4 *>(stages)[i] = make_uint4(0u, 0u, 0u, 0u);
     fence_async_smem();
     if (warp == 0) {
         asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(tmem_slot)), "r"(kTmemCols) : "memory");
@@ -396,7 +415,12 @@ __global__ void __launch_bounds__(kUThreads, 2) block_umma_kernel(const __grid_c
     tc_fence_after();
     const uint32_t tm = *tmem_slot;
     const PlanEntry e = reinterpret_cast<const PlanEntry *>(a.plan + a.plan_entry)[entry];
-    const HeadUnits hu = head_units(geo, e);
+    HeadUnits hu = head_units(geo, e);
+    if (kPair) {          // factor pages two to a unit (the last unit of an odd number holds one), dense pages whole
+        hu.d0 = hu.fb * bpp;
+        hu.nf = (hu.nf + 1) >> 1;
+        hu.units = hu.d0 + hu.nf + (e.n_pages - hu.fe) * bpp;
+    }
     const int T = a.n_tokens[(long long)e.seq * geo.n_layers + a.layer];
     // Units are in token order and the block's last row sees the most: units that start after what it sees are
     // hidden from every row of the block and are left out (all roles agree on the count).
@@ -406,9 +430,9 @@ __global__ void __launch_bounds__(kUThreads, 2) block_umma_kernel(const __grid_c
         const int vis = T - (a.q_len - 1 - last_row / G);                 // tokens the last row sees (>= 1)
         const int page = (vis - 1) / P, blk = ((vis - 1) % P) / kDB;
         int need;
-        if (page < hu.fb) need = page * geo.blocks_per_page + blk + 1;
+        if (page < hu.fb) need = page * bpp + blk + 1;
         else if (page < hu.fe) need = hu.d0 + hu.nf;
-        else need = hu.d0 + hu.nf + (page - hu.fe) * geo.blocks_per_page + blk + 1;
+        else need = hu.d0 + hu.nf + (page - hu.fe) * bpp + blk + 1;
         n_units = max(1, min(need, hu.units));
     }
     int u_base = 0;                                       // first unit of this CTA's range
@@ -429,15 +453,19 @@ __global__ void __launch_bounds__(kUThreads, 2) block_umma_kernel(const __grid_c
             for (int s = 0, round = 0; u < n_units; ++u, s = s + 1 == S ? 0 : s + 1, round += s == 0) {
                 if (u >= S && !wait_lane(smem_u32(empty_bar + s), (round - 1) & 1, abort_flag, limit)) { ok = false; break; }
                 int page, blk, kind;
-                unit_to_page(geo, hu, u_base + u, page, blk, kind);
+                unit_to_page(bpp, hu, u_base + u, page, blk, kind);
+                if (kPair && kind == kKindFactor) page = hu.fb + 2 * (page - hu.fb);
                 const int slot = pt[page];
+                const int n_pg = kPair && kind == kKindFactor && page + 1 < hu.fe ? 2 : 1;          // pages of this unit
+                const int slot2 = n_pg == 2 ? pt[page + 1] : 0;
                 int rows = 0, after = 0;
-                const bool bad = slot < 0 || slot >= (kind == kKindFactor ? geo.n_factor_slots : geo.n_dense_slots);
+                const bool bad = slot < 0 || slot >= (kind == kKindFactor ? geo.n_factor_slots : geo.n_dense_slots) ||
+                                 slot2 < 0 || slot2 >= geo.n_factor_slots;
                 if (bad) {
                     atomicAdd(a.status + 2, 1);                  // corrupt page table: an empty unit, and a mark
                     kind = kKindDense;
                 } else if (kind == kKindFactor) {
-                    rows = P;
+                    rows = P * n_pg;
                 } else {
                     rows = max(0, min(kDB, T - page * P - blk * kDB));
                     after = max(0, T - page * P - blk * kDB - rows);
@@ -447,20 +475,24 @@ __global__ void __launch_bounds__(kUThreads, 2) block_umma_kernel(const __grid_c
                 const uint32_t bar = smem_u32(full_bar + s);
                 const uint32_t dst = smem_u32(stages + (size_t)s * ustage);
                 if (kind == kKindFactor) {
-                    const long long off = (long long)slot * geo.factor_slot_bytes + (long long)head * geo.blob_bytes;
-                    const unsigned char *src = a.factor_pool + off;
-                    // B_k, B_v as rows of the pool seen in 256-byte rows; a part that starts half a row in (the ranks
-                    // of P = 32 pages allow it) goes through the map whose origin is 128 bytes further on
-                    const long long ok_ = off + geo.bk_off, ov_ = off + geo.bv_off;
-                    const CUtensorMap *mk = (ok_ & 128) ? &maps.bk_half : &maps.bk, *mv = (ov_ & 128) ? &maps.bv_half : &maps.bv;
-                    const int yk = (int)(ok_ >> 8), yv = (int)(ov_ >> 8);
-                    mbar_arrive_expect_tx(bar, geo.blob_bytes);
-                    bulk_g2s_keep(dst + L.ak, src + geo.ak_off, geo.rank_k * 2 * P, bar);
-                    bulk_g2s_keep(dst + L.av, src + geo.av_off, geo.rank_v * 2 * P, bar);
-                    tma_box(dst + L.k, mk, 0, yk, bar);
-                    tma_box(dst + L.k + L.k_panel, mk, 64, yk, bar);
-                    tma_box(dst + L.v, mv, 0, yv, bar);
-                    tma_box(dst + L.v + L.v_panel, mv, 64, yv, bar);
+                    mbar_arrive_expect_tx(bar, geo.blob_bytes * n_pg);
+                    for (int j = 0; j < n_pg; ++j) {
+                        const long long off = (long long)(j ? slot2 : slot) * geo.factor_slot_bytes + (long long)head * geo.blob_bytes;
+                        const unsigned char *src = a.factor_pool + off;
+                        // B_k, B_v as rows of the pool seen in 256-byte rows; a part that starts half a row in (the ranks
+                        // of P = 32 pages allow it) goes through the map whose origin is 128 bytes further on
+                        const long long ok_ = off + geo.bk_off, ov_ = off + geo.bv_off;
+                        const CUtensorMap *mk = (ok_ & 128) ? &maps.bk_half : &maps.bk, *mv = (ov_ & 128) ? &maps.bv_half : &maps.bv;
+                        const int yk = (int)(ok_ >> 8), yv = (int)(ov_ >> 8);
+                        // (a pair: the second page's A^T parts follow the first's, its B rows start at row 16 of the panels)
+                        const uint32_t dk = dst + L.k + j * (16 * 128), dv = dst + L.v + j * (16 * 128);
+                        bulk_g2s_keep(dst + L.ak + j * umma_a_bytes(geo, geo.rank_k), src + geo.ak_off, geo.rank_k * 2 * P, bar);
+                        bulk_g2s_keep(dst + L.av + j * umma_a_bytes(geo, geo.rank_v), src + geo.av_off, geo.rank_v * 2 * P, bar);
+                        tma_box(dk, mk, 0, yk, bar);
+                        tma_box(dk + L.k_panel, mk, 64, yk, bar);
+                        tma_box(dv, mv, 0, yv, bar);
+                        tma_box(dv + L.v_panel, mv, 64, yv, bar);
+                    }
                 } else if (rows > 0) {
                     // whole blocks: rows past the sequence's end hold whatever the pool holds; the scores there are
                     // masked and the row threads clear those rows
@@ -530,10 +562,13 @@ __global__ void __launch_bounds__(kUThreads, 2) block_umma_kernel(const __grid_c
                     tc_fence_after();
                     const uint32_t sb = stage_at(s0);
                     if (k0 == kKindFactor) {
-                        const uint64_t da = umma_desc(sb + L.av, 16, kAGroup, kASwizzle);
 #pragma unroll
-                        for (int ks = 0; ks < P / 16; ++ks)      // w = p . A_v, A_v^T in place (K-major)
-                            umma_ts(t_w, t_s + ks * 8, umma_desc_step(da, ks * 32), umma_idesc(128, RP, 0), ks > 0);
+                        for (int j = 0; j < (kPair ? 2 : 1); ++j) {        // (a pair: page j's tokens are columns 32 j .. of p, its ranks columns 16 j .. of w)
+                            const uint64_t da = umma_desc(sb + L.av + j * umma_a_bytes(geo, geo.rank_v), 16, kAGroup, kASwizzle);
+#pragma unroll
+                            for (int ks = 0; ks < P / 16; ++ks)      // w = p . A_v, A_v^T in place (K-major)
+                                umma_ts(t_w + j * RP1, t_s + (j * (P / 16) + ks) * 8, umma_desc_step(da, ks * 32), umma_idesc(128, RP1, 0), ks > 0);
+                        }
                     } else {
                         pv(t_s, sb + L.dv, L.d_panel);
                         umma_commit(smem_u32(empty_bar + s0));         // a dense unit's stage is free after Gb
@@ -547,13 +582,23 @@ __global__ void __launch_bounds__(kUThreads, 2) block_umma_kernel(const __grid_c
                     tc_fence_after();
                     const uint32_t sb = stage_at(s1);
                     if (k1 == kKindFactor) {
-                        const uint64_t dak = umma_desc(sb + L.ak, 16, kAGroup, kASwizzle);
+                        if (kPair) {
 #pragma unroll
-                        for (int t = 0; t < 2; ++t)              // s = (q~_hi + q~_lo) . A_k^T, A_k^T in place (MN-major)
+                            for (int j = 0; j < 2; ++j) {        // page j: its 16 columns of either term of q~ -> columns 32 j .. of s
+                                const uint64_t dak = umma_desc(sb + L.ak + j * umma_a_bytes(geo, geo.rank_k), 16, kAGroup, kASwizzle);
 #pragma unroll
-                            for (int ks = 0; ks < RP / 16; ++ks)
-                                umma_ts(t_s, t_qt + t * (RP / 2) + ks * 8, umma_desc_step(dak, ks * 2 * kAGroup),
-                                        umma_idesc(128, P, 1), (t | ks) > 0);
+                                for (int t = 0; t < 2; ++t)
+                                    umma_ts(t_s + j * P, t_qt + t * (RP / 2) + j * 8, dak, umma_idesc(128, P, 1), t > 0);
+                            }
+                        } else {
+                            const uint64_t dak = umma_desc(sb + L.ak, 16, kAGroup, kASwizzle);
+#pragma unroll
+                            for (int t = 0; t < 2; ++t)              // s = (q~_hi + q~_lo) . A_k^T, A_k^T in place (MN-major)
+#pragma unroll
+                                for (int ks = 0; ks < RP / 16; ++ks)
+                                    umma_ts(t_s, t_qt + t * (RP / 2) + ks * 8, umma_desc_step(dak, ks * 2 * kAGroup),
+                                            umma_idesc(128, P, 1), (t | ks) > 0);
+                        }
                     } else {
                         qk(t_s, sb + L.dk, L.d_panel);
                     }
@@ -624,9 +669,13 @@ __global__ void __launch_bounds__(kUThreads, 2) block_umma_kernel(const __grid_c
                 PKV_ROWS_WAIT(bar_S, ph_S)
                 bool fine;
                 if (cur.kind == kKindFactor) {
-                    float sv[P];
-                    tmem_ld<P>(t_s, reinterpret_cast<uint32_t *>(sv));
-                    fine = softmax_row<P, false>(sv, st, u > 0, t_s, t_o, bar_Q, ph_Q, o_seen, abort_flag, limit);
+                    float sv[PU];
+                    tmem_ld<PU>(t_s, reinterpret_cast<uint32_t *>(sv));
+                    if (kPair && cur.rows < PU) {                 // the last page of an odd number: no second page
+#pragma unroll
+                        for (int i = P; i < PU; ++i) sv[i] = kMasked;
+                    }
+                    fine = softmax_row<PU, false>(sv, st, u > 0, t_s, t_o, bar_Q, ph_Q, o_seen, abort_flag, limit);
                 } else {
                     float sv[kDB];
                     tmem_ld<kDB>(t_s, reinterpret_cast<uint32_t *>(sv));
@@ -649,8 +698,8 @@ __global__ void __launch_bounds__(kUThreads, 2) block_umma_kernel(const __grid_c
                 if (nxt.kind == kKindFactor) {      // columns past the rank are exact zeros
                     uint32_t rq[RP], hi[RP / 2], lo[RP / 2];
                     tmem_ld<RP>(t_qt, rq);
-                    if (full_tiles) split_terms<RP, 8 * NT, true>(rq, hi, lo, scale, 8 * NT);
-                    else split_terms<RP, RP, false>(rq, hi, lo, scale, geo.rank_k);
+                    if (full_tiles) split_terms<RP, 8 * NT, true, kPair>(rq, hi, lo, scale, 8 * NT);
+                    else split_terms<RP, RP, false, kPair>(rq, hi, lo, scale, geo.rank_k);
                     tmem_st<RP / 2>(t_qt, hi);
                     tmem_st<RP / 2>(t_qt + RP / 2, lo);
                     tmem_st_wait();
@@ -675,8 +724,8 @@ __global__ void __launch_bounds__(kUThreads, 2) block_umma_kernel(const __grid_c
                     uint32_t rw[RP], pk[RP / 2];
                     tmem_ld<RP>(t_w, rw);
                     const float c = exp2_fast(st.m - st.m_ref);
-                    if (full_tiles) scale_pack<RP, 8 * NT, true>(rw, pk, c, 8 * NT);
-                    else scale_pack<RP, RP, false>(rw, pk, c, geo.rank_v);
+                    if (full_tiles) scale_pack<RP, 8 * NT, true, kPair>(rw, pk, c, 8 * NT);
+                    else scale_pack<RP, RP, false, kPair>(rw, pk, c, geo.rank_v);
                     tmem_st<RP / 2>(t_w, pk);
                     tmem_st_wait();
                 }
@@ -783,7 +832,7 @@ __global__ void __launch_bounds__(256) rowblock_merge_kernel(const __grid_consta
 
 size_t umma_smem_bytes(const Geometry &g) {
     const int S = umma_stages(g);
-    return (size_t)kUQBytes + (size_t)S * umma_stage_bytes(g) + kUStagePad + (2 * S + 8) * 8 + (S + 2) * sizeof(StageDesc) + 64;
+    return (size_t)kUQBytes + (size_t)S * umma_stage_bytes(g) + umma_stage_pad(g) + (2 * S + 8) * 8 + (S + 2) * sizeof(StageDesc) + 64;
 }
 
 }  // namespace
