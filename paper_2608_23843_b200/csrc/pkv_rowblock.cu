@@ -1,10 +1,11 @@
 // Row-block attention on the fifth-generation tensor cores (tcgen05.mma, accumulators and row operands in tensor
 // memory).
 //
-// Same job as the mma.sync row-block kernel of pkv_decode.cu — many queries per sequence (a chunk of a prefill), one
+// Same job as the mma.sync row-block kernel of pkv_decode.cu — many queries per sequence (a chunk of a prefill), a
 // CTA per (sequence, KV head, block of query rows), Eq. 4 for factor pages and plain attention for dense ones, the
-// pages in token order so that no split-K state is left to merge — but with 128 query rows per CTA as the M
-// dimension of every product:
+// pages in token order — but with 128 query rows per CTA as the M dimension of every product (and, where the row
+// blocks alone would not fill the GPU, several CTAs per block with a range of the sequence each, whose softmax
+// states rowblock_merge_kernel combines; pages of 32 tokens with ranks up to 16 are taken two to a unit):
 //     G1: q~ [128 x r] = Q [128 x d] . B_k^T        G2: s [128 x P] = (q~_hi + q~_lo) . A_k^T
 //     G3: w  [128 x r] = p [128 x P] . A_v          G4: o [128 x d] += w . B_v
 //     dense pages:  Ga: s = Q . K^T                 Gb: o += p . V
