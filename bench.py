@@ -51,6 +51,9 @@ WORKLOADS = {
     # The same with the paper's default page shape (Section 4.1: P = 32, ranks (16, 14)) on the Qwen3-8B layer shape.
     "prefill_chunk_qwen3_8b_16k_p32": dict(n_layers=2, layers_per_step=1, n_kv_heads=8, n_q_heads=32, batch=1, T=16384,
                                            rank=16, rank_v=14, page=32, sink=32, recent=2048, ragged=False, outliers=0.0),
+    # ... and with the smallest page of the paper's page-size ablation (P = 16) at the same rank per token (8, 8)
+    "prefill_chunk_qwen3_8b_16k_p16": dict(n_layers=2, layers_per_step=1, n_kv_heads=8, n_q_heads=32, batch=1, T=16384,
+                                           rank=8, rank_v=8, page=16, sink=16, recent=2048, ragged=False, outliers=0.0),
     # tiny single decode step (L2-resident; latency only)
     "tiny": dict(n_layers=1, n_kv_heads=1, n_q_heads=4, batch=1, T=1024, rank=16, sink=64, recent=128,
                  ragged=False, outliers=0.0),

@@ -45,12 +45,12 @@ constexpr uint32_t kColQt = 0, kColS = 32, kColW = 96, kColO = 128, kTmemCols = 
 // a block of dense K, V side = B_v or a block of dense V; a side is two panels of 64 channels, written by tiled TMA
 // copies (box = 64 channels x rows) straight from the pools' 256-byte rows: 16-byte chunk c of row j is stored at
 // chunk c ^ (j & 7), so each half of a row is a 128-byte row in the tensor core's 128-byte swizzle.
-// Pages of 32 tokens with ranks up to 16 are taken two to a unit (64 tokens, like a page of 64): page j's B rows start
+// Pages of 32 or 16 tokens with ranks up to 16 are taken two to a unit: page j's B rows start
 // at row 16 j of panels of 32 rows, so that q~ and w of the pair are one row of 32 columns and the products with the
 // B factors are the same instructions as for a rank of 32; the products with the A factors are issued per page.
-__host__ __device__ inline bool umma_pair(const Geometry &g) { return g.page == 32 && g.rank_tiles <= 2; }
-// Rows of a dense block (a whole page of 32 tokens in the pair form), and what a rank - or a pair's two ranks - is padded to in the products:
-__host__ __device__ inline int umma_part_rows(const Geometry &g) { return g.rank_tiles <= 2 && !umma_pair(g) ? 16 : 32; }
+__host__ __device__ inline bool umma_pair(const Geometry &g) { return g.page <= 32 && g.rank_tiles <= 2; }
+// Rows of a dense block (a whole page in the pair form; otherwise what a rank is padded to in the products):
+__host__ __device__ inline int umma_part_rows(const Geometry &g) { return umma_pair(g) ? g.page : (g.rank_tiles <= 2 ? 16 : 32); }
 // Bytes kept free behind the last stage: a product that reads a rank padded to 16 or 32 rows may run past the last
 // part of a stage (a pair's panels hold exactly the rows its products read).
 __host__ __device__ inline int umma_stage_pad(const Geometry &g) { return umma_pair(g) ? 0 : 1024; }
@@ -362,13 +362,13 @@ __global__ void __launch_bounds__(kUThreads, 2) block_umma_kernel(const __grid_c
                                                                   const __grid_constant__ RowBlockMaps maps) {
     // RP1: what a page's rank is padded to; RP: columns of q~ and w of a factor unit, and the rows of a dense block;
     // PU: tokens of a factor unit (kPair: two pages of 32 tokens, see umma_pair()); bpp: blocks of a dense page
-    constexpr bool kPair = P == 32 && NT <= 2;
+    constexpr bool kPair = P <= 32 && NT <= 2;
     constexpr int RP1 = NT <= 2 ? 16 : 32, RP = kPair ? 32 : RP1, PU = kPair ? 2 * P : P;
-    constexpr int kDB = kPair ? 32 : kDenseBlock<P, NT, 0>, bpp = P / kDB;
+    constexpr int kDB = kPair ? P : kDenseBlock<P, NT, 0>, bpp = P / kDB;
     // A^T rows are 2 P bytes: the 128-byte swizzle for P = 64, the 64-byte one (8 rows = 512 bytes) for P = 32, the
     // 32-byte one for P = 16 - each time the XOR the pages are stored with
     constexpr uint32_t kASwizzle = P == 64 ? 2 : (P == 32 ? 4 : 6), kAGroup = 8 * 2 * P;
-    static_assert(kDB == RP, "dense blocks and padded ranks have the same number of rows");
+    static_assert(kDB == RP || kPair, "dense blocks and padded ranks have the same number of rows unless pages come in pairs");
     const Geometry &geo = a.geo;
     const StageLayout L = umma_layout(geo);
     const int S = umma_stages(geo), ustage = umma_stage_bytes(geo), H = geo.n_kv_heads, G = geo.group;
@@ -528,8 +528,9 @@ __global__ void __launch_bounds__(kUThreads, 2) block_umma_kernel(const __grid_c
             // [128 x RP] = Q . (K side)^T: 8 steps of 16 channels; both operands K-major, 128-byte swizzle
             // (steps ks0 .. ks1 - 1: the eight steps of G1 are issued in two halves, so that they stand in the way of the
             // other CTA's products for half as long at a time)
-            auto qk = [&](uint32_t t_dst, uint32_t kside, int panel, int ks0 = 0, int ks1 = 8) {
-                const uint32_t idesc = umma_idesc(128, RP, 0);
+            // (n: rows of the K side - RP for G1, the rows of a block for a dense unit)
+            auto qk = [&](uint32_t t_dst, uint32_t kside, int panel, int ks0, int ks1, int n) {
+                const uint32_t idesc = umma_idesc(128, n, 0);
                 const uint64_t db0 = umma_desc(kside, 16, 1024, 2), db1 = umma_desc(kside + panel, 16, 1024, 2);
 #pragma unroll
                 for (int ks = 0; ks < 8; ++ks)
@@ -537,11 +538,12 @@ __global__ void __launch_bounds__(kUThreads, 2) block_umma_kernel(const __grid_c
                         umma_ss(t_dst, umma_desc_step(ks < 4 ? dq0 : dq1, (ks & 3) * 32), umma_desc_step(ks < 4 ? db0 : db1, (ks & 3) * 32), idesc, ks > 0);
             };
             // o [128 x d] (+)= (rows of RP bf16 at t_src) . (V side): MN-major, two panels of 64 channels
-            auto pv = [&](uint32_t t_src, uint32_t vside, int panel) {
+            // (k: rows of the V side - RP for G4, the rows of a block for a dense unit)
+            auto pv = [&](uint32_t t_src, uint32_t vside, int panel, int k) {
                 const uint64_t dv = umma_desc(vside, panel, 1024, 2);
 #pragma unroll
                 for (int ks = 0; ks < RP / 16; ++ks)
-                    umma_ts(t_o, t_src + ks * 8, umma_desc_step(dv, ks * 2048), umma_idesc(128, 128, 1), o_valid || ks > 0);
+                    if (ks * 16 < k) umma_ts(t_o, t_src + ks * 8, umma_desc_step(dv, ks * 2048), umma_idesc(128, 128, 1), o_valid || ks > 0);
                 o_valid = true;
             };
             // kind of a unit as the products see it: units without tokens run as dense units with every score masked
@@ -571,7 +573,7 @@ __global__ void __launch_bounds__(kUThreads, 2) block_umma_kernel(const __grid_c
                                 umma_ts(t_w + j * RP1, t_s + (j * (P / 16) + ks) * 8, umma_desc_step(da, ks * 32), umma_idesc(128, RP1, 0), ks > 0);
                         }
                     } else {
-                        pv(t_s, sb + L.dv, L.d_panel);
+                        pv(t_s, sb + L.dv, L.d_panel, kDB);
                         umma_commit(smem_u32(empty_bar + s0));         // a dense unit's stage is free after Gb
                     }
                     umma_commit(bar_G3);
@@ -601,14 +603,14 @@ __global__ void __launch_bounds__(kUThreads, 2) block_umma_kernel(const __grid_c
                                             umma_idesc(128, P, 1), (t | ks) > 0);
                         }
                     } else {
-                        qk(t_s, sb + L.dk, L.d_panel);
+                        qk(t_s, sb + L.dk, L.d_panel, 0, 8, kDB);
                     }
                     umma_commit(bar_S);
                     // behind it, off the rows' path: the first half of G1(u+2), over the q~ columns G2(u+1) has just read
                     if (u + 2 < n_units) {
                         k2 = unit_kind(s2, round2, ok, u + 2);
                         if (!ok) break;
-                        if (k2 == kKindFactor) qk(t_qt, stage_at(s2) + L.k, L.k_panel, 0, 4);
+                        if (k2 == kKindFactor) qk(t_qt, stage_at(s2) + L.k, L.k_panel, 0, 4, RP);
                     }
                 }
                 // hand-over C: w(u) is in tensor memory -> G4(u); then, off the rows' path, G1(u+2)
@@ -616,16 +618,16 @@ __global__ void __launch_bounds__(kUThreads, 2) block_umma_kernel(const __grid_c
                 ph_C ^= 1;
                 tc_fence_after();
                 if (u >= 0 && k0 == kKindFactor) {
-                    pv(t_w, stage_at(s0) + L.v, L.v_panel);
+                    pv(t_w, stage_at(s0) + L.v, L.v_panel, RP);
                     umma_commit(smem_u32(empty_bar + s0));             // a factor unit's stage is free after G4
                 }
                 if (u + 2 < n_units) {
                     if (u < -1) {                                  // (before the first unit there is no hand-over B)
                         k2 = unit_kind(s2, round2, ok, u + 2);
                         if (!ok) break;
-                        if (k2 == kKindFactor) qk(t_qt, stage_at(s2) + L.k, L.k_panel, 0, 4);
+                        if (k2 == kKindFactor) qk(t_qt, stage_at(s2) + L.k, L.k_panel, 0, 4, RP);
                     }
-                    if (k2 == kKindFactor) qk(t_qt, stage_at(s2) + L.k, L.k_panel, 4, 8);       // the second half of G1(u+2)
+                    if (k2 == kKindFactor) qk(t_qt, stage_at(s2) + L.k, L.k_panel, 4, 8, RP);       // the second half of G1(u+2)
                 }
                 umma_commit(bar_Q);
                 k0 = k1; k1 = k2;
