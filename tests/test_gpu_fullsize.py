@@ -26,7 +26,7 @@ import pytest
 import torch
 
 import bench
-from gpu_helpers import E2E_FLOOR_CAP, E2E_FLOOR_FACTOR, f64, rel_err
+from gpu_helpers import E2E_FLOOR_CAP, E2E_FLOOR_FACTOR, f64, kernel_tolerances, rel_err
 from oracle import attention as oatt
 from oracle import svd as osvd
 from oracle.cache import FACTOR, OracleCache, OracleConfig
@@ -231,7 +231,7 @@ def test_paper_default_shape_qwen3_8b_16k():
 
 
 @pytest.mark.parametrize("variant", [0, 3])
-@pytest.mark.parametrize("workload", ["prefill_chunk_llama3_8b_32k", "prefill_chunk_qwen3_8b_16k_p32"])
+@pytest.mark.parametrize("workload", ["prefill_chunk_llama3_8b_32k", "prefill_chunk_qwen3_8b_16k_p32", "prefill_chunk_qwen3_8b_16k_p16"])
 def test_prefill_chunk_2048_positions_against_a_long_context(workload, variant):
     """The bench's prefill-chunk launches (`--workload prefill_chunk_llama3_8b_32k --q-len 2048`, and the same on the
     paper's default page shape, P = 32 with ranks (16, 14)): one sequence whose last 2048 positions are the queries,
@@ -240,7 +240,9 @@ def test_prefill_chunk_2048_positions_against_a_long_context(workload, variant):
     the first and last positions of the chunk, positions on either side of page and block boundaries, a row from every
     128-row block parity - against plain attention over the pages exactly as the GPU stores them (kernel gate; the
     causal limit is part of what is checked), the two kernels against one another on every row, and a rerun bit for
-    bit."""
+    bit.  The third workload, pages of 16 tokens with ranks (8, 8), is judged by the rule for arbitrary shapes: with
+    1024 units per row both kernels sit at 4.0e-3 of ||out||_inf on one sampled row (the same row, to four digits:
+    the bf16 rounding of the softmax numerators, which they share)."""
     w, device = bench.WORKLOADS[workload], torch.device("cuda", 0)
     QL = 2048
     cfg, cache, lengths, comp = bench.build_workload(w, w["rank"], device, decode_variant=variant)
@@ -266,7 +268,13 @@ def test_prefill_chunk_2048_positions_against_a_long_context(workload, variant):
                 h = head * G + gq
                 ref = oatt.attention_plain(f64(q[0, j, h]), K_all[:vis], V_all[:vis], scale)
                 e = rel_err(f64(out32[0, j, h]), ref)
-                assert e <= 4e-3, (variant, head, j, gq, e)
+                if workload.endswith("_p16"):
+                    # not one of the benchmark configurations the stated 4e-3 was set for: the rule for arbitrary
+                    # shapes (4e-3 of ||out||_inf or one bf16 unit of the largest value read, whichever is larger)
+                    tol32, _ = kernel_tolerances(float(np.abs(ref).max()), float(np.abs(V_all[:vis]).max()))
+                    assert np.abs(f64(out32[0, j, h]) - ref).max() <= tol32, (variant, head, j, gq, e)
+                else:
+                    assert e <= 4e-3, (variant, head, j, gq, e)
                 assert rel_err(f64(out[0, j, h]), ref) <= ATT_TOL
                 worst = max(worst, e)
     record(workload, decode_variant=variant, kernel_gate_worst=worst, rows_checked=2 * len(positions) * G)
