@@ -49,8 +49,8 @@ constexpr uint32_t kColQt = 0, kColS = 32, kColW = 96, kColO = 128, kTmemCols = 
 // at row 16 j of panels of 32 rows, so that q~ and w of the pair are one row of 32 columns and the products with the
 // B factors are the same instructions as for a rank of 32; the products with the A factors are issued per page.
 __host__ __device__ inline bool umma_pair(const Geometry &g) { return g.page <= 32 && g.rank_tiles <= 2; }
-// Rows of a dense block (a whole page in the pair form; otherwise what a rank is padded to in the products):
-__host__ __device__ inline int umma_part_rows(const Geometry &g) { return umma_pair(g) ? g.page : (g.rank_tiles <= 2 ? 16 : 32); }
+// Rows of a dense block: a whole page, or half a page of 64 tokens
+__host__ __device__ inline int umma_part_rows(const Geometry &g) { return g.page < 32 ? g.page : 32; }
 // Bytes kept free behind the last stage: a product that reads a rank padded to 16 or 32 rows may run past the last
 // part of a stage (a pair's panels hold exactly the rows its products read).
 __host__ __device__ inline int umma_stage_pad(const Geometry &g) { return umma_pair(g) ? 0 : 1024; }
@@ -360,15 +360,15 @@ __device__ __forceinline__ bool softmax_row(float *sv, RowSoftmax &st, bool o_va
 template <int P, int NT>
 __global__ void __launch_bounds__(kUThreads, 2) block_umma_kernel(const __grid_constant__ DecodeArgs a,
                                                                   const __grid_constant__ RowBlockMaps maps) {
-    // RP1: what a page's rank is padded to; RP: columns of q~ and w of a factor unit, and the rows of a dense block;
-    // PU: tokens of a factor unit (kPair: two pages of 32 tokens, see umma_pair()); bpp: blocks of a dense page
+    // RP1: what a page's rank is padded to; RP: columns of q~ and w of a factor unit; PU: tokens of a factor unit
+    // (kPair: two pages, see umma_pair()); kDB: rows of a dense block; bpp: blocks of a dense page
     constexpr bool kPair = P <= 32 && NT <= 2;
     constexpr int RP1 = NT <= 2 ? 16 : 32, RP = kPair ? 32 : RP1, PU = kPair ? 2 * P : P;
-    constexpr int kDB = kPair ? P : kDenseBlock<P, NT, 0>, bpp = P / kDB;
+    constexpr int kDB = P < 32 ? P : 32, bpp = P / kDB;
     // A^T rows are 2 P bytes: the 128-byte swizzle for P = 64, the 64-byte one (8 rows = 512 bytes) for P = 32, the
     // 32-byte one for P = 16 - each time the XOR the pages are stored with
     constexpr uint32_t kASwizzle = P == 64 ? 2 : (P == 32 ? 4 : 6), kAGroup = 8 * 2 * P;
-    static_assert(kDB == RP || kPair, "dense blocks and padded ranks have the same number of rows unless pages come in pairs");
+    static_assert(kDB <= 32 && RP <= 32, "a dense block's scores and a unit's q~ fit their columns of tensor memory");
     const Geometry &geo = a.geo;
     const StageLayout L = umma_layout(geo);
     const int S = umma_stages(geo), ustage = umma_stage_bytes(geo), H = geo.n_kv_heads, G = geo.group;
@@ -417,11 +417,11 @@ __global__ void __launch_bounds__(kUThreads, 2) block_umma_kernel(const __grid_c
     const uint32_t tm = *tmem_slot;
     const PlanEntry e = reinterpret_cast<const PlanEntry *>(a.plan + a.plan_entry)[entry];
     HeadUnits hu = head_units(geo, e);
-    if (kPair) {          // factor pages two to a unit (the last unit of an odd number holds one), dense pages whole
-        hu.d0 = hu.fb * bpp;
-        hu.nf = (hu.nf + 1) >> 1;
-        hu.units = hu.d0 + hu.nf + (e.n_pages - hu.fe) * bpp;
-    }
+    // this kernel's own units: dense pages in blocks of kDB rows; kPair: factor pages two to a unit (the last unit of an
+    // odd number holds one)
+    hu.d0 = hu.fb * bpp;
+    if (kPair) hu.nf = (hu.nf + 1) >> 1;
+    hu.units = hu.d0 + hu.nf + (e.n_pages - hu.fe) * bpp;
     const int T = a.n_tokens[(long long)e.seq * geo.n_layers + a.layer];
     // Units are in token order and the block's last row sees the most: units that start after what it sees are
     // hidden from every row of the block and are left out (all roles agree on the count).
@@ -542,7 +542,7 @@ __global__ void __launch_bounds__(kUThreads, 2) block_umma_kernel(const __grid_c
             auto pv = [&](uint32_t t_src, uint32_t vside, int panel, int k) {
                 const uint64_t dv = umma_desc(vside, panel, 1024, 2);
 #pragma unroll
-                for (int ks = 0; ks < RP / 16; ++ks)
+                for (int ks = 0; ks < 2; ++ks)
                     if (ks * 16 < k) umma_ts(t_o, t_src + ks * 8, umma_desc_step(dv, ks * 2048), umma_idesc(128, 128, 1), o_valid || ks > 0);
                 o_valid = true;
             };
