@@ -810,11 +810,11 @@ def main():
                                                        "; ncu showed the mma.sync pipe 50 % busy at this rate"),
                                 "traffic": None, "launch_us": launch_ms * 1e3, "algorithmic_flops_per_launch": flops}
             if umma:
-                # the library's rule for cutting row blocks into token ranges (a second, merging launch follows then)
+                # (row blocks cut into token ranges: a second, merging launch follows)
                 n_blocks = w["batch"] * w["n_kv_heads"] * -(-rows // 128)
                 sms = torch.cuda.get_device_properties(device).multi_processor_count
-                ns = min(32, min(2 * sms, 512) // n_blocks, -(-max(lengths) // P_) // 8)
-                line["roofline"]["token_ranges_per_row_block"] = ns if ns >= 2 else 1
+                ns = pkv.pkv_get_row_block_ranges(n_blocks, max(lengths), P_, sms)
+                line["roofline"]["token_ranges_per_row_block"] = ns
                 if ns >= 2:
                     line["gpu_launches"] *= 2
         if not args.no_cpu_baseline and world == 1 and QL == 1 and not args.global_rank:

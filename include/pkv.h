@@ -473,6 +473,21 @@ pkv_status pkv_read_basis(pkv_cache *c, int32_t seq, int32_t layer, int32_t kv_h
 pkv_status pkv_get_rotation_schedule(int32_t page_size, uint8_t *members, int64_t capacity, int32_t *n_rounds,
                                      int32_t *groups_per_round, int32_t *group_size);
 
+/*
+ * How many token ranges pkv_decode_attention_multi() cuts each row block's sequence into when its tcgen05 row-block
+ * kernel serves a call (see there; Eq. 5 merges the ranges), for inspection and tests.  Host only: no cache, no GPU
+ * work.  (The paper fixes the merge rule, not how work is spread over a GPU; this describes this library's launch.)
+ *   n_row_blocks    blocks of 128 query rows in the call: n_seqs * H_kv * ceil(q_len * (H_q / H_kv) / 128)
+ *   longest_tokens  tokens of the longest listed sequence;  page_size as in the configuration
+ *   n_sms           multiprocessors of the GPU (two CTAs of the kernel fit one)
+ * *n_ranges = min(32, min(2 n_sms, 512) / n_row_blocks, ceil(longest_tokens / page_size) / 8) (integer divisions) if
+ * that is at least 2, else 1: ranges only when the row blocks alone leave half the GPU idle, at least eight pages
+ * per range, at most 512 states in the workspace.
+ * Returns PKV_ERR_INVALID_ARG for a NULL pointer or an argument below 1 (nothing written).
+ */
+pkv_status pkv_get_row_block_ranges(int64_t n_row_blocks, int32_t longest_tokens, int32_t page_size, int32_t n_sms,
+                                    int32_t *n_ranges);
+
 #ifdef __cplusplus
 }
 #endif

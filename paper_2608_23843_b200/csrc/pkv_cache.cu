@@ -397,6 +397,14 @@ int block_slots_per_seq(const Geometry &g, int q_len) { return passes_per_seq(g,
 // rows of a KV head, which walks the whole sequence alone) instead of the pipeline kernel (eight query columns per
 // pass over the pages, split over all CTAs).  The row-block kernel needs enough CTAs to fill the GPU; below that the
 // pipeline kernel is used if its plan entries fit.
+// Token ranges per row block of a tcgen05 row-block launch (documented with pkv_get_row_block_ranges()).
+int row_block_ranges(long long n_blocks, int longest_tokens, int page_size, int n_sms) {
+    const long long by_fill = std::min<long long>(2LL * n_sms, kRbSplitItems) / n_blocks;
+    const long long by_length = (longest_tokens + page_size - 1) / page_size / kRbMinPages;
+    const long long ns = std::min<long long>(kRbMaxSplits, std::min(by_fill, by_length));
+    return ns >= 2 ? (int)ns : 1;
+}
+
 bool uses_row_blocks(const pkv_cache *c, int q_len, int n_seqs) {
     const long long rows = (long long)q_len * c->geo.group;
     if (q_len <= 1 || (c->cfg.decode_variant != 0 && c->cfg.decode_variant != 3) || c->geo.factor_bits == 4 || rows < kRowBlock) return false;
@@ -1078,10 +1086,7 @@ static pkv_status decode_impl(pkv_cache *c, int32_t layer, int32_t n_seqs, const
             const long long n_blocks = (long long)n_seqs * c->geo.n_kv_heads * (((long long)q_len * c->geo.group + 127) / 128);
             int longest = 0;
             for (int i = 0; i < n_seqs; ++i) longest = std::max(longest, c->at(seq_ids[i], layer).n_tokens);
-            const long long by_fill = std::min<long long>(2LL * c->n_sms, kRbSplitItems) / n_blocks;
-            const long long by_length = (longest + c->cfg.page_size - 1) / c->cfg.page_size / kRbMinPages;
-            const long long ns = std::min<long long>(kRbMaxSplits, std::min(by_fill, by_length));
-            if (ns >= 2) a.rb_splits = (int)ns;
+            a.rb_splits = row_block_ranges(n_blocks, longest, c->cfg.page_size, c->n_sms);
         }
         PKV_CUDA(c, launch_decode_blocks(a, n_seqs, c->row_maps, st));
         return PKV_OK;
@@ -1269,6 +1274,13 @@ pkv_status pkv_write_factors(pkv_cache *c, int64_t slot, int32_t head, const voi
     unsigned char *blob = c->factor_pool + slot * c->geo.factor_slot_bytes + (int64_t)head * c->geo.blob_bytes;
     c->cache_written = true;                     // the next decode launch must not start ahead of this kernel
     PKV_CUDA(c, launch_write_factors(c->geo, blob, A_k, B_k, A_v, B_v, (cudaStream_t)stream));
+    return PKV_OK;
+}
+
+pkv_status pkv_get_row_block_ranges(int64_t n_row_blocks, int32_t longest_tokens, int32_t page_size, int32_t n_sms,
+                                    int32_t *n_ranges) {
+    if (!n_ranges || n_row_blocks < 1 || longest_tokens < 1 || page_size < 1 || n_sms < 1) return PKV_ERR_INVALID_ARG;
+    *n_ranges = row_block_ranges(n_row_blocks, longest_tokens, page_size, n_sms);
     return PKV_OK;
 }
 

@@ -31,7 +31,7 @@ EXPORTS = [
     "pkv_read_dense", "pkv_get_decode_plan", "pkv_decode_attention_static_scratch", "pkv_get_decode_trace",
     "pkv_decode_attention_multi", "pkv_compress_begin", "pkv_compress_commit",
     "pkv_decode_attention_partial", "pkv_merge_attention_states",
-    "pkv_get_rotation_schedule", "pkv_read_basis",
+    "pkv_get_rotation_schedule", "pkv_read_basis", "pkv_get_row_block_ranges",
 ]
 
 
@@ -104,6 +104,7 @@ def lib():
         L.pkv_get_decode_plan.argtypes = [vp, i32, ip, ip, ip, ip]
         L.pkv_get_decode_trace.argtypes = [vp, ctypes.POINTER(ctypes.c_int64), i32, vp]
         L.pkv_get_rotation_schedule.argtypes = [i32, ctypes.POINTER(ctypes.c_uint8), i64, ip, ip, ip]
+        L.pkv_get_row_block_ranges.argtypes = [i64, i32, i32, i32, ip]
         for name in EXPORTS:
             if name != "pkv_last_error":
                 getattr(L, name).restype = ctypes.c_int32
@@ -310,6 +311,15 @@ def pkv_get_rotation_schedule(page_size):
     flat = list(buf[:nr.value * ng.value * gs.value])
     it = iter(flat)
     return [[tuple(next(it) for _ in range(gs.value)) for _ in range(ng.value)] for _ in range(nr.value)]
+
+
+def pkv_get_row_block_ranges(n_row_blocks, longest_tokens, page_size, n_sms):
+    """-> token ranges per row block of a tcgen05 row-block launch (1 = the blocks are not cut)."""
+    n = ctypes.c_int32()
+    rc = lib().pkv_get_row_block_ranges(int(n_row_blocks), int(longest_tokens), int(page_size), int(n_sms), ctypes.byref(n))
+    if rc != PKV_OK:
+        raise PkvError(rc, "pkv_get_row_block_ranges(%r, %r, %r, %r)" % (n_row_blocks, longest_tokens, page_size, n_sms))
+    return n.value
 
 
 def pkv_read_dense(handle, slot, kv_head, K, V, stream=None):

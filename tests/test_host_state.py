@@ -456,3 +456,27 @@ def test_buffers_promised_by_query_sizes_always_suffice(overlap):
                     assert sz.workspace_bytes <= (192 << 20) + 64 * 4160 * (max(512, n_ctas) + max_seqs * H)
                 handle = pkv.pkv_init_cache(cfg, None, None, None, None, None, None)      # dry run: host logic only
                 pkv.pkv_destroy_cache(handle)
+
+
+def test_token_ranges_of_a_row_block_launch():
+    """pkv_get_row_block_ranges(): the rule by which the tcgen05 row-block kernel's launch cuts row blocks into token
+    ranges, pinned by hand-worked cases (148 SMs = 296 CTAs in flight; a range has at least eight pages; at most 32
+    ranges per block and 512 states per launch)."""
+    f = pkv.pkv_get_row_block_ranges
+    assert f(64, 32768, 64, 148) == 4            # 8 sequences x 8 KV heads, 32 queries of 4 heads each: 296 // 64
+    assert f(128, 32768, 64, 148) == 2           # 64 queries: two blocks per (sequence, head)
+    assert f(512, 32768, 64, 148) == 1           # a 2048-position chunk fills the GPU by itself
+    assert f(149, 32768, 64, 148) == 1           # more than half the CTAs in flight: no ranges
+    assert f(148, 32768, 64, 148) == 2
+    assert f(8, 32768, 64, 148) == 32            # one sequence: 296 // 8 = 37, capped at 32
+    assert f(8, 4096, 64, 148) == 8              # 64 pages: eight pages per range
+    assert f(8, 1000, 64, 148) == 2              # 16 pages
+    assert f(8, 1023, 64, 148) == 2
+    assert f(8, 960, 64, 148) == 1               # 15 pages: not two ranges of eight
+    assert f(8, 16384, 16, 148) == 32            # 1024 pages of 16 tokens
+    assert f(1, 1 << 20, 64, 1000) == 32         # a bigger GPU: 512 states bound the launch, 32 ranges the block
+    assert f(20, 1 << 20, 64, 1000) == 25        # 512 // 20
+    assert f(1, 64, 64, 1) == 1
+    for bad in [(0, 100, 64, 148), (1, 0, 64, 148), (1, 100, 0, 148), (1, 100, 64, 0)]:
+        with pytest.raises(pkv.PkvError):
+            f(*bad)
