@@ -164,7 +164,9 @@ typedef struct pkv_sizes {
     int64_t factor_pool_bytes;
     int64_t meta_bytes;         /* device page tables, token counts, decode plans, status words; with global_rank
                                    also the bases: max_seqs * n_layers * H_kv * 2 * global_rank * d * 2 bytes */
-    int64_t workspace_bytes;    /* split-K partial states, merge tickets, compression work list */
+    int64_t workspace_bytes;    /* split-K partial states, merge tickets, compression work list; where the tcgen05
+                                   row-block kernel applies (see pkv_decode_attention_multi), 34.6 MB for the states of
+                                   row blocks cut into token ranges */
 } pkv_sizes;
 
 typedef struct pkv_stats {
