@@ -537,6 +537,18 @@ def max_over_ranks(values, world, device="cpu"):
     return [float(x) for x in t.tolist()]
 
 
+def row_block_flops(w, rank, lengths, q_len):
+    """Algorithmic FLOPs of one pkv_decode_attention_multi launch served by a row-block kernel: query rows x (factor
+    pages x 2 (d r_k + r_k P + P r_v + r_v d) + dense tokens x 4 d); the causal triangle among the new positions is
+    counted in full."""
+    P_, rv_ = w.get("page", 64), w.get("rank_v", rank)
+    flops = 0
+    for T_ in lengths:
+        nf_ = max(0, T_ // P_ - w["recent"] // P_ - w["sink"] // P_)
+        flops += q_len * w["n_q_heads"] * (nf_ * 2 * (128 * rank + rank * P_ + P_ * rv_ + rv_ * 128) + (T_ - nf_ * P_) * 4 * 128)
+    return flops
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
@@ -726,6 +738,35 @@ def main():
     if st["device_timeouts"] or st["bad_slot_indices"] or (outs[0].float().isnan().any().item()):
         raise SystemExit("decode produced timeouts or NaNs: %r" % st)
 
+    # Several new positions per sequence on the same cache (pkv_decode_attention_multi, served by the tcgen05 row-block
+    # kernel): a sub-record of the default line, so that one run also carries the tensor-bound kernel's figure.
+    multi = None
+    MQ = 64
+    if (QL == 1 and not args.seq_sharded and not args.graph and not args.no_standalone and not args.global_rank
+            and args.factor_bits == 16 and args.decode_variant == 0 and not w["ragged"] and w["recent"] >= MQ
+            and MQ * (Hq // w["n_kv_heads"]) >= 64 and min(lengths) > w["recent"] + w["sink"]):
+        mq_q = [synth.make_q(SEED + 1, layer, 0, w["batch"] * MQ, Hq, 128, device).view(w["batch"], MQ, Hq, 128) for layer in range(min(L, 2))]
+        mq_out = torch.empty_like(mq_q[0])
+        mq_steps = max(2, min(args.steps, 5))
+
+        def mq_step():
+            for layer in range(lps):
+                cache.decode_attention_multi(layer % L, ids, MQ, mq_q[layer % len(mq_q)], mq_out)
+        for _ in range(3):
+            mq_step()
+        barrier()
+        m0, m1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        m0.record()
+        for _ in range(mq_steps):
+            mq_step()
+        m1.record()
+        barrier()
+        mq_ms = m0.elapsed_time(m1) / mq_steps
+        st = cache.stats()
+        if st["device_timeouts"] or st["bad_slot_indices"] or mq_out.float().isnan().any().item():
+            raise SystemExit("multi-query decode produced timeouts or NaNs: %r" % st)
+        multi = (mq_ms, mq_steps)
+
     # The same step with every launch standing alone (decode_overlap = 0: a launch starts computing only when the
     # kernel before it has finished, as in a decoder whose queries come from the layer before): a second cache of
     # the same workload, timed the same way in this run.
@@ -753,6 +794,8 @@ def main():
     ms, e2e_ms, launch_ms = max_over_ranks([ms, e2e_ms, launch_ms], world, device)
     if standalone_ms is not None:
         standalone_ms = max_over_ranks([standalone_ms], world, device)[0]
+    if multi is not None:
+        multi = (max_over_ranks([multi[0]], world, device)[0], multi[1])
 
     if rk == 0:
         bytes_per_launch = bytes_per_step / lps
@@ -781,6 +824,22 @@ def main():
                                   "hbm_gbs": bytes_per_step / (standalone_ms * 1e-3) / 1e9 * world,
                                   "frac_of_8tbs": r0["frac_of_8tbs"], "frac": r0["frac"], "launch_us": r0["launch_us"],
                                   "gpu_launches": lps * args.steps}
+        if multi is not None:
+            mq_ms = multi[0]
+            fl = row_block_flops(w, rank, lengths, MQ)
+            tpeak, tsrc = _tensor_peak()
+            n_blocks = w["batch"] * w["n_kv_heads"] * -(-(MQ * (Hq // w["n_kv_heads"])) // 128)
+            ns = pkv.pkv_get_row_block_ranges(n_blocks, max(lengths), w.get("page", 64),
+                                              torch.cuda.get_device_properties(device).multi_processor_count)
+            tach = fl * lps / (mq_ms * 1e-3) / 1e12
+            line["multi_query"] = {"queries_per_sequence": MQ, "value": mq_ms * 1e3, "unit": "us", "steps": multi[1],
+                                   "launch_us": mq_ms * 1e3 / lps, "bound": "tensor", "achieved": tach, "peak": tpeak,
+                                   "frac": tach / tpeak, "peak_source": tsrc, "kernel_unit": "TFLOP/s",
+                                   "kernel": "block_umma_kernel (tcgen05, 128 query rows per CTA) + rowblock_merge_kernel"
+                                             if ns >= 2 else "block_umma_kernel (tcgen05, 128 query rows per CTA)",
+                                   "row_blocks": n_blocks, "token_ranges_per_row_block": ns,
+                                   "algorithmic_flops_per_launch": fl,
+                                   "gpu_launches": lps * multi[1] * (2 if ns >= 2 else 1)}
         P_, Gq = w.get("page", 64), Hq // w["n_kv_heads"]
         rows = QL * Gq
         rv_ = w.get("rank_v", rank)
@@ -790,15 +849,8 @@ def main():
         # (and its rule for the route: row blocks from 64 query rows per KV head on; the mma.sync kernel only if they fill the GPU)
         if QL > 1 and args.decode_variant in (0, 3) and args.factor_bits != 4 and rows >= 64 and (
                 umma or w["batch"] * w["n_kv_heads"] * -(-rows // 64) >= 128):
-            # Served by the row-block kernel, whose bound is the tensor pipe, not HBM: algorithmic FLOPs per launch =
-            # query rows x (factor pages x 2 (d r_k + r_k P + P r_v + r_v d) + dense tokens x 4 d); the causal
-            # triangle among the new positions is counted in full.
-            flops = 0
-            for T_ in lengths:
-                n_pages_ = -(-T_ // P_)
-                nf_ = max(0, T_ // P_ - w["recent"] // P_ - w["sink"] // P_)
-                dense_tok = T_ - nf_ * P_
-                flops += QL * Hq * (nf_ * 2 * (128 * rank + rank * P_ + P_ * rv_ + rv_ * 128) + dense_tok * 4 * 128)
+            # Served by the row-block kernel, whose bound is the tensor pipe, not HBM.
+            flops = row_block_flops(w, rank, lengths, QL)
             tpeak, tsrc = _tensor_peak()
             tach = flops / (launch_ms * 1e-3) / 1e12
             line["roofline"] = {"bound": "tensor",
