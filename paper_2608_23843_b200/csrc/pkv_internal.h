@@ -150,13 +150,13 @@ cudaError_t launch_decode(const DecodeArgs &a, int n_segs, cudaStream_t st);
 // kRbSplitItems CTAs per launch when split, at most kRbMaxSplits per row block, at least kRbMinPages pages per range.
 constexpr int kRbStateFloats = kHeadDim + 4, kRbSplitItems = 512, kRbMaxSplits = 32, kRbMinPages = 8;
 constexpr int kRowBlock = 64;          // query rows (token x query head) per CTA of the mma.sync row-block kernel
-// tcgen05 row-block kernel (pkv_rowblock.cu): 128 query rows per CTA; bf16 page-wise factors whose matrices start on
-// 128-byte boundaries of the pool (every rank for P = 64, even ranks for P = 32, multiples of 4 for P = 16)
+// tcgen05 row-block kernel (pkv_rowblock.cu): 128 query rows per CTA; bf16 page-wise factors with rank_v <= rank_k
 bool row_block_umma_supported(const Geometry &geo);
 cudaError_t row_block_umma_setup();
 // TMA descriptors of the pools for that kernel (B factors; dense K / V); valid = 0 where the shape is not covered or
 // the driver offers no encoder, and the mma.sync kernel is used instead
-struct RowBlockMaps { CUtensorMap bk, bv, bk_half, bv_half, dense; int valid; };   // *_half: origin 128 bytes into the pool
+// (bk[i], bv[i]: the factor pool from an origin 32 i bytes in - a B matrix may start on any 32-byte boundary of a 256-byte row)
+struct RowBlockMaps { CUtensorMap bk[8], bv[8], dense; int valid; };
 void row_block_make_maps(const Geometry &geo, const void *factor_pool, const void *dense_pool, RowBlockMaps *maps);
 cudaError_t launch_decode_blocks_umma(const DecodeArgs &a, int n_seqs, const RowBlockMaps &maps, cudaStream_t st);
 cudaError_t launch_decode_blocks(const DecodeArgs &a, int n_seqs, const RowBlockMaps &maps, cudaStream_t st);

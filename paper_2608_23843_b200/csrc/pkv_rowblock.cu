@@ -480,10 +480,10 @@ __global__ void __launch_bounds__(kUThreads, 2) block_umma_kernel(const __grid_c
                     for (int j = 0; j < n_pg; ++j) {
                         const long long off = (long long)(j ? slot2 : slot) * geo.factor_slot_bytes + (long long)head * geo.blob_bytes;
                         const unsigned char *src = a.factor_pool + off;
-                        // B_k, B_v as rows of the pool seen in 256-byte rows; a part that starts half a row in (the ranks
-                        // of P = 32 pages allow it) goes through the map whose origin is 128 bytes further on
+                        // B_k, B_v as rows of the pool seen in 256-byte rows; a part that starts 32 i bytes into such a row
+                        // (A^T parts of 2 P r bytes come before it) goes through the map whose origin is that much further on
                         const long long ok_ = off + geo.bk_off, ov_ = off + geo.bv_off;
-                        const CUtensorMap *mk = (ok_ & 128) ? &maps.bk_half : &maps.bk, *mv = (ov_ & 128) ? &maps.bv_half : &maps.bv;
+                        const CUtensorMap *mk = &maps.bk[(ok_ >> 5) & 7], *mv = &maps.bv[(ov_ >> 5) & 7];
                         const int yk = (int)(ok_ >> 8), yv = (int)(ov_ >> 8);
                         // (a pair: the second page's A^T parts follow the first's, its B rows start at row 16 of the panels)
                         const uint32_t dk = dst + L.k + j * (16 * 128), dv = dst + L.v + j * (16 * 128);
@@ -842,11 +842,11 @@ size_t umma_smem_bytes(const Geometry &g) {
 
 bool row_block_umma_supported(const Geometry &g) {
     // A^T rows of 128, 64 or 32 bytes (P = 64, 32, 16: the swizzles the tensor cores know for such rows); every part of a blob
-    // on a 128-byte boundary of the pool (the tiled copies address the pools in 256-byte rows, from either of two
-    // origins 128 bytes apart): every rank for P = 64, even ranks for P = 32, multiples of 4 for P = 16
+    // on a 32-byte boundary of the pool (the tiled copies address the pools in 256-byte rows, from one of eight origins
+    // 32 bytes apart), which every rank gives
     return (g.page == 64 || g.page == 32 || g.page == 16) && g.factor_bits == 16 && g.global_rank == 0 &&
-           g.rank_v <= g.rank_k && g.rank_tiles >= 1 && g.rank_tiles <= 4 && g.bk_off % 128 == 0 && g.bv_off % 128 == 0 &&
-           g.blob_bytes % 128 == 0 && g.factor_slot_bytes % 128 == 0 && umma_smem_bytes(g) <= (size_t)kSmemBudget / 2;
+           g.rank_v <= g.rank_k && g.rank_tiles >= 1 && g.rank_tiles <= 4 && g.bk_off % 32 == 0 && g.bv_off % 32 == 0 &&
+           g.blob_bytes % 32 == 0 && g.factor_slot_bytes % 32 == 0 && umma_smem_bytes(g) <= (size_t)kSmemBudget / 2;
 }
 
 #define PKV_FOR_EACH_UMMA_SHAPE(X) X(64, 1) X(64, 2) X(64, 3) X(64, 4) X(32, 1) X(32, 2) X(32, 3) X(32, 4) X(16, 1) X(16, 2)
@@ -861,7 +861,7 @@ cudaError_t row_block_umma_setup() {
 }
 
 // Tensor maps of the two pools seen as matrices of 256-byte rows (128 bf16), box = 64 channels x `rows`; for the factor
-// pool a second pair whose origin lies 128 bytes further on (see the copy lane).  The encoder is a driver entry
+// pool eight pairs with origins 32 bytes apart (see the copy lane).  The encoder is a driver entry
 // point; it is looked up at run time so that the library does not link against the driver.
 void row_block_make_maps(const Geometry &g, const void *factor_pool, const void *dense_pool, RowBlockMaps *maps) {
     typedef CUresult (*EncodeTiled)(CUtensorMap *, CUtensorMapDataType, cuuint32_t, void *, const cuuint64_t *, const cuuint64_t *,
@@ -890,16 +890,17 @@ void row_block_make_maps(const Geometry &g, const void *factor_pool, const void 
     if (!make(&maps->dense, dense_pool, (long long)g.n_dense_slots * g.dense_slot_bytes, rb)) return;
     if (factor_pool && g.n_factor_slots > 0) {
         const long long bytes = (long long)g.n_factor_slots * g.factor_slot_bytes;
-        const unsigned char *half = static_cast<const unsigned char *>(factor_pool) + 128;
-        if (!make(&maps->bk, factor_pool, bytes, g.rank_k) || !make(&maps->bv, factor_pool, bytes, g.rank_v)) return;
-        if (bytes >= 512) {
-            if (!make(&maps->bk_half, half, bytes - 128, g.rank_k) || !make(&maps->bv_half, half, bytes - 128, g.rank_v)) return;
-        } else {
-            maps->bk_half = maps->bk;
-            maps->bv_half = maps->bv;
+        for (int i = 0; i < 8; ++i) {
+            const unsigned char *origin = static_cast<const unsigned char *>(factor_pool) + 32 * i;
+            if (i > 0 && bytes - 32 * i < 512) {          // (a pool of one or two rows: nothing can start there)
+                maps->bk[i] = maps->bk[0];
+                maps->bv[i] = maps->bv[0];
+            } else if (!make(&maps->bk[i], origin, bytes - 32 * i, g.rank_k) || !make(&maps->bv[i], origin, bytes - 32 * i, g.rank_v)) {
+                return;
+            }
         }
     } else {
-        maps->bk = maps->bv = maps->bk_half = maps->bv_half = maps->dense;          // no factor pages: never used
+        for (int i = 0; i < 8; ++i) maps->bk[i] = maps->bv[i] = maps->dense;          // no factor pages: never used
     }
     maps->valid = 1;
 }

@@ -502,7 +502,7 @@ def test_many_tiny_segments_per_cta(rank, n_ctas):
     (64, 32, 32, 1, 70, 16),      # row-block kernel, one query head per KV head, full-width ranks
     (64, 24, 24, 8, 16, 16),      # row-block kernel, 128 rows, two tokens per 16-row tile
     (32, 8, 8, 4, 40, 16),        # row-block kernel, one rank tile, queries spanning two pages
-    (64, 16, 14, 4, 70, 16),      # tcgen05 row-block kernel, even ranks that are not multiples of 8 (parts of a stage padded)
+    (64, 16, 14, 4, 70, 16),      # tcgen05 row-block kernel, ranks that are not multiples of 8 (parts of a stage padded)
     (64, 8, 8, 8, 40, 16),        # tcgen05 row-block kernel, one rank tile (rank padded to 16 in the products), 320 rows
 ])
 def test_multi_query_attention(P, rk, rv, G, q_len, bits):
