@@ -843,9 +843,9 @@ def main():
         P_, Gq = w.get("page", 64), Hq // w["n_kv_heads"]
         rows = QL * Gq
         rv_ = w.get("rank_v", rank)
-        # the library's own rule (row_block_umma_supported): tcgen05 kernel for bf16 factors with rank_v <= rank_k; the
-        # mma.sync kernel otherwise or when decode_variant 3 pins it
-        umma = args.decode_variant == 0 and rv_ <= rank
+        # the library's own rule (row_block_umma_supported): the tcgen05 kernel for bf16 factors unless decode_variant 3
+        # pins the mma.sync kernel
+        umma = args.decode_variant == 0
         # (and its rule for the route: row blocks from 64 query rows per KV head on; the mma.sync kernel only if they fill the GPU)
         if QL > 1 and args.decode_variant in (0, 3) and args.factor_bits != 4 and rows >= 64 and (
                 umma or w["batch"] * w["n_kv_heads"] * -(-rows // 64) >= 128):

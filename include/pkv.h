@@ -304,12 +304,12 @@ pkv_status pkv_decode_attention(pkv_cache *c, int32_t layer, int32_t n_seqs, con
  * are kept per sequence and block).
  * Two kinds of kernel serve this call.  A row-block kernel - CTAs per (sequence, KV head, block of query rows),
  * which read the sequence's pages once for the block, the query rows being the row operand of every product of
- * Eq. 4 - runs when q_len * (H_q / H_kv) >= 64 and the factors are bf16.  With rank_v <= rank_k (any page size
- * and rank) it is the tcgen05 kernel (128 rows per CTA, accumulators and row
+ * Eq. 4 - runs when q_len * (H_q / H_kv) >= 64 and the factors are bf16.  It is the tcgen05 kernel (any page
+ * size and ranks; 128 rows per CTA, accumulators and row
  * operands in tensor memory, pages brought in by TMA in the layout the tensor cores read); where the blocks alone
  * would not fill the GPU it cuts each block's sequence into up to 32 token ranges, one CTA each, and a second
- * launch merges their softmax states by Eq. 5 in token order.  With rank_v > rank_k, or with decode_variant 3, it
- * is the mma.sync kernel (64 rows per CTA, never split), and then only if the call makes at least 128 blocks
+ * launch merges their softmax states by Eq. 5 in token order.  With decode_variant 3 (or a driver without the
+ * tensor-map encoder) it is the mma.sync kernel (64 rows per CTA, never split), and then only if the call makes at least 128 blocks
  * (enough to fill the GPU) or would exceed the limit above, which does not apply to row blocks.  Otherwise
  * the decode kernel runs
  * with its CTAs in groups of b = ceil(q_len / max(1, 8 / (H_q / H_kv))): the CTAs of a group walk the same pages at

@@ -150,7 +150,7 @@ cudaError_t launch_decode(const DecodeArgs &a, int n_segs, cudaStream_t st);
 // kRbSplitItems CTAs per launch when split, at most kRbMaxSplits per row block, at least kRbMinPages pages per range.
 constexpr int kRbStateFloats = kHeadDim + 4, kRbSplitItems = 512, kRbMaxSplits = 32, kRbMinPages = 8;
 constexpr int kRowBlock = 64;          // query rows (token x query head) per CTA of the mma.sync row-block kernel
-// tcgen05 row-block kernel (pkv_rowblock.cu): 128 query rows per CTA; bf16 page-wise factors with rank_v <= rank_k
+// tcgen05 row-block kernel (pkv_rowblock.cu): 128 query rows per CTA; bf16 page-wise factors
 bool row_block_umma_supported(const Geometry &geo);
 cudaError_t row_block_umma_setup();
 // TMA descriptors of the pools for that kernel (B factors; dense K / V); valid = 0 where the shape is not covered or

@@ -845,7 +845,7 @@ bool row_block_umma_supported(const Geometry &g) {
     // on a 32-byte boundary of the pool (the tiled copies address the pools in 256-byte rows, from one of eight origins
     // 32 bytes apart), which every rank gives
     return (g.page == 64 || g.page == 32 || g.page == 16) && g.factor_bits == 16 && g.global_rank == 0 &&
-           g.rank_v <= g.rank_k && g.rank_tiles >= 1 && g.rank_tiles <= 4 && g.bk_off % 32 == 0 && g.bv_off % 32 == 0 &&
+           g.rank_tiles >= 1 && g.rank_tiles <= 4 && g.bk_off % 32 == 0 && g.bv_off % 32 == 0 &&
            g.blob_bytes % 32 == 0 && g.factor_slot_bytes % 32 == 0 && umma_smem_bytes(g) <= (size_t)kSmemBudget / 2;
 }
 

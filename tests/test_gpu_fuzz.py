@@ -227,9 +227,12 @@ def test_random_schedules_with_two_step_compression_multi_query_and_states(seed)
         pair.gpu.close()
 
 
+@pytest.mark.parametrize("variant", [0, 3])
 @pytest.mark.parametrize("seed", [1, 2])
-def test_random_configurations_row_block_kernel(seed):
-    """Random shapes for the row-block kernel of pkv_decode_attention_multi (queries as tensor-core rows): page
+def test_random_configurations_row_block_kernel(seed, variant):
+    """Random shapes for the row-block kernels of pkv_decode_attention_multi (queries as tensor-core rows; variant 0:
+    the tcgen05 kernel, which serves every shape, with its token ranges where the sequences are long enough; 3: the
+    mma.sync kernel): page
     sizes, ranks with ragged last tiles, group sizes, query counts that leave the last block or the last 16-row
     tile partly empty, new positions spanning pages and dense blocks, sequences that consist of nothing but the
     new positions.  max_seqs is kept too small for the column route, so the row-block kernel serves every call.
@@ -252,8 +255,9 @@ def test_random_configurations_row_block_kernel(seed):
         cfg = pkv.make_config(n_layers=1, n_kv_heads=H, n_q_heads=H * G, rank=rk, rank_v=rv, page_size=P,
                               sink_tokens=P * rng.choice([0, 1, 2]), recent_tokens=W, max_seqs=nseq,
                               max_pages_per_seq=max_pages, n_dense_slots=nseq * max_pages + 2,
-                              n_factor_slots=nseq * max_pages + 2, decode_overlap=rng.choice([0, 1, 2]))
-        what = (seed, case, P, rk, rv, H, G, q_len, lengths, W, cfg.sink_tokens)
+                              n_factor_slots=nseq * max_pages + 2, decode_overlap=rng.choice([0, 1, 2]),
+                              decode_variant=variant)
+        what = (seed, variant, case, P, rk, rv, H, G, q_len, lengths, W, cfg.sink_tokens)
         pair = Pair(cfg, seed=case)
         for s, T in enumerate(lengths):
             k, v = gen_kv(500 + case, 0, s, T, cfg)
