@@ -810,21 +810,26 @@ __global__ void __launch_bounds__(256) rowblock_merge_kernel(const __grid_consta
     const long long qrow = ((long long)entry * a.q_len + row / G) * geo.n_q_heads + head * G + row % G;
     const float *src = a.rb_partials + ((size_t)blk_id * ns * kURows + r) * kRbStateFloats;
     const size_t stride = (size_t)kURows * kRbStateFloats;
-    float M = kNegInf;
-    for (int k = 0; k < ns; ++k) {
-        const float2 ml = *reinterpret_cast<const float2 *>(src + k * stride + kHeadDim);
-        if (ml.y > 0.f) M = fmaxf(M, ml.x);
-    }
+    // lane k holds (m, l) of range k (at most 32 ranges) and works out the range's weight 2^(m_k - M); the sum over
+    // the ranges then takes each weight by a shuffle, so that the loads of the o rows do not wait for one another
+    static_assert(kRbMaxSplits <= 32, "one lane per range");
+    float2 ml = make_float2(kNegInf, 0.f);
+    if (lane < ns) ml = *reinterpret_cast<const float2 *>(src + lane * stride + kHeadDim);
+    float M = ml.y > 0.f ? ml.x : kNegInf;
+#pragma unroll
+    for (int d = 16; d > 0; d >>= 1) M = fmaxf(M, __shfl_xor_sync(0xffffffffu, M, d));
+    const float wk = ml.y > 0.f ? exp2f(ml.x - M) : 0.f;          // weight of range `lane`
+    float L = wk * ml.y;
     float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
-    float L = 0.f;
-    for (int k = 0; k < ns; ++k) {
-        const float2 ml = *reinterpret_cast<const float2 *>(src + k * stride + kHeadDim);
-        if (!(ml.y > 0.f)) continue;
-        const float w = exp2f(ml.x - M);
+#pragma unroll 4
+    for (int k = 0; k < ns; ++k) {                                  // token order: the sum is the same whoever ran first
+        const float w = __shfl_sync(0xffffffffu, wk, k);
         const float4 o = *reinterpret_cast<const float4 *>(src + k * stride + 4 * lane);
         acc.x += w * o.x; acc.y += w * o.y; acc.z += w * o.z; acc.w += w * o.w;
-        L += w * ml.y;
     }
+    // (l: summed in lane order by a fixed tree, the same for every launch)
+#pragma unroll
+    for (int d = 16; d > 0; d >>= 1) L += __shfl_xor_sync(0xffffffffu, L, d);
     const float inv = L > 0.f ? 1.f / L : 0.f;
     acc.x *= inv; acc.y *= inv; acc.z *= inv; acc.w *= inv;
     if (a.out)
